@@ -1,0 +1,445 @@
+/*
+ * CPU checker for outlier channel splitting (arXiv:1901.09504).  TEST INFRASTRUCTURE ONLY:
+ * plain scalar C, no blocking, no fusion; see ocs_oracle.h for the conventions.
+ * Build: gcc -O2 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC (OpenMP is used
+ * only on the outermost independent loop of the integer contractions).
+ */
+#include "ocs_oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------ Section 3.4: split count */
+int ocs_oracle_num_splits(int C, double ratio) {
+  if (C <= 0 || !(ratio > 0.0)) return 0;
+  return (int)ceil(ratio * (double)C - 1e-9);
+}
+
+/* ------------------------------------------------------------------ Section 3.3: one split */
+/* The two halves of one value.  d = 0 is the Net2WiderNet rule (w/2, w/2); d = half a grid
+ * step is the quantization-aware rule ((w - 0.5)/2, (w + 0.5)/2) written in weight units.
+ * Each operation rounds once to fp32. */
+static inline float split_keep(float w, float d) {
+  volatile float t = w - d;
+  return t * 0.5f;
+}
+static inline float split_new(float w, float d) {
+  volatile float t = w + d;
+  return t * 0.5f;
+}
+
+static float channel_maxabs(const float* Wc, int O, int Ctot, int R, int j) {
+  float m = 0.0f;
+  for (int o = 0; o < O; ++o)
+    for (int r = 0; r < R; ++r) {
+      float a = fabsf(Wc[((size_t)o * Ctot + j) * R + r]);
+      if (a > m) m = a;
+    }
+  return m;
+}
+
+static void split_channel(float* Wc, int O, int Ctot, int R, int j, int jnew, float d) {
+  for (int o = 0; o < O; ++o)
+    for (int r = 0; r < R; ++r) {
+      size_t src = ((size_t)o * Ctot + j) * R + r;
+      size_t dst = ((size_t)o * Ctot + jnew) * R + r;
+      float w = Wc[src];
+      Wc[src] = split_keep(w, d);
+      Wc[dst] = split_new(w, d);
+    }
+}
+
+static int split_common(const float* W, int O, int C, int R, int S, float qa_step, float* W_out,
+                        int32_t* idx_map, int32_t* split_order, float* max_abs, int cached) {
+  if (!W || !W_out || !idx_map || O <= 0 || C <= 0 || R <= 0 || S < 0 || !(qa_step >= 0.0f))
+    return 1;
+  const int Ctot = C + S;
+  const float d = qa_step * 0.5f;
+  /* current tensor: channels [0, C) hold W, [C, C+S) are not alive yet */
+  for (int o = 0; o < O; ++o)
+    for (int j = 0; j < Ctot; ++j)
+      for (int r = 0; r < R; ++r)
+        W_out[((size_t)o * Ctot + j) * R + r] =
+            (j < C) ? W[((size_t)o * C + j) * R + r] : 0.0f;
+  for (int j = 0; j < C; ++j) idx_map[j] = j;
+  if (max_abs) {
+    float m = 0.0f;
+    for (int j = 0; j < C; ++j) {
+      float c = channel_maxabs(W_out, O, Ctot, R, j);
+      if (c > m) m = c;
+    }
+    max_abs[0] = m;
+  }
+  float* cmax = NULL;
+  if (cached) {
+    cmax = (float*)malloc(sizeof(float) * (size_t)Ctot);
+    if (!cmax) return 2;
+    for (int j = 0; j < C; ++j) cmax[j] = channel_maxabs(W_out, O, Ctot, R, j);
+  }
+  for (int s = 0; s < S; ++s) {
+    const int alive = C + s;
+    int jbest = 0;
+    float best = -1.0f;
+    for (int j = 0; j < alive; ++j) { /* ascending j + strict '>' : ties go to the smallest index */
+      float c = cached ? cmax[j] : channel_maxabs(W_out, O, Ctot, R, j);
+      if (c > best) { best = c; jbest = j; }
+    }
+    split_channel(W_out, O, Ctot, R, jbest, alive, d);
+    idx_map[alive] = idx_map[jbest];
+    if (split_order) split_order[s] = jbest;
+    if (cached) {
+      cmax[jbest] = channel_maxabs(W_out, O, Ctot, R, jbest);
+      cmax[alive] = channel_maxabs(W_out, O, Ctot, R, alive);
+    }
+  }
+  if (max_abs) {
+    float m = 0.0f;
+    for (int j = 0; j < Ctot; ++j) {
+      float c = channel_maxabs(W_out, O, Ctot, R, j);
+      if (c > m) m = c;
+    }
+    max_abs[1] = m;
+  }
+  free(cmax);
+  return 0;
+}
+
+int ocs_oracle_split_literal(const float* W, int O, int C, int R, int S, float qa_step,
+                             float* W_out, int32_t* idx_map, int32_t* split_order,
+                             float* max_abs) {
+  return split_common(W, O, C, R, S, qa_step, W_out, idx_map, split_order, max_abs, 0);
+}
+int ocs_oracle_split_cached(const float* W, int O, int C, int R, int S, float qa_step,
+                            float* W_out, int32_t* idx_map, int32_t* split_order,
+                            float* max_abs) {
+  return split_common(W, O, C, R, S, qa_step, W_out, idx_map, split_order, max_abs, 1);
+}
+
+/* ------------------------------------------------------------------ Eq. 1: linear quantization */
+float ocs_oracle_maxabs(const float* T, int64_t n) {
+  float m = 0.0f;
+  for (int64_t i = 0; i < n; ++i) {
+    float a = fabsf(T[i]);
+    if (a > m) m = a;
+  }
+  return m;
+}
+
+static int code_limit(int bits, int is_signed) {
+  return is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
+}
+
+int ocs_oracle_quantize(const float* T, int64_t n, int bits, int is_signed, float alpha,
+                        int8_t* codes, float* scale) {
+  if (!T || !codes || n < 0 || bits < 2 || bits > 8 || !(alpha >= 0.0f)) return 1;
+  const int L = code_limit(bits, is_signed);
+  if (alpha == 0.0f) {
+    memset(codes, 0, (size_t)n);
+    if (scale) *scale = 0.0f;
+    return 0;
+  }
+  volatile float step = alpha / (float)L;
+  volatile float inv = (float)L / alpha;
+  const float lo = is_signed ? -(float)L : 0.0f, hi = (float)L;
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float t = T[i] * inv;
+    float q = nearbyintf(t); /* default rounding mode: half to even */
+    if (q < lo) q = lo;
+    if (q > hi) q = hi;
+    int c = (int)q;
+    if (is_signed) codes[i] = (int8_t)c;
+    else ((uint8_t*)codes)[i] = (uint8_t)c;
+  }
+  if (scale) *scale = step;
+  return 0;
+}
+
+/* ------------------------------------------------------------------ Section 4.1: MSE clip search */
+int ocs_oracle_clip_mse(const float* T, int64_t n, int bits, int is_signed, int n_bins,
+                        int n_candidates, float* alpha, float* max_abs, uint64_t* hist,
+                        double* scores) {
+  if (!T || !alpha || n < 0 || bits < 2 || bits > 8 || n_bins < 1 || n_candidates < 1) return 1;
+  const int L = code_limit(bits, is_signed);
+  const int B = n_bins;
+  const float m = ocs_oracle_maxabs(T, n);
+  if (max_abs) *max_abs = m;
+  uint64_t* h = (uint64_t*)calloc((size_t)B, sizeof(uint64_t));
+  if (!h) return 2;
+  if (m == 0.0f) {
+    *alpha = 0.0f;
+    if (hist) { memset(hist, 0, sizeof(uint64_t) * (size_t)B); hist[0] = (uint64_t)n; }
+    if (scores) for (int c = 0; c < n_candidates; ++c) scores[c] = 0.0;
+    free(h);
+    return 0;
+  }
+  /* histogram of |x|: B equal bins on [0, m] */
+  volatile float invw = (float)B / m;
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float t = fabsf(T[i]) * invw;
+    int b = (int)t; /* truncation */
+    if (b > B - 1) b = B - 1;
+    h[b] += 1;
+  }
+  if (hist) memcpy(hist, h, sizeof(uint64_t) * (size_t)B);
+  const double width = (double)m / (double)B;
+  const double lo = is_signed ? -(double)L : 0.0, hi = (double)L;
+  double best = 0.0;
+  int cbest = -1;
+  for (int c = 1; c <= n_candidates; ++c) {
+    const float alpha_c = (float)((double)m * (double)c / (double)n_candidates);
+    const double step = (double)alpha_c / (double)L;
+    double score = 0.0;
+    for (int b = 0; b < B; ++b) {
+      const double xb = ((double)b + 0.5) * width;
+      double q = nearbyint(xb / step);
+      if (q < lo) q = lo;
+      if (q > hi) q = hi;
+      const double e = xb - q * step;
+      score += (double)h[b] * e * e;
+    }
+    if (scores) scores[c - 1] = score;
+    if (cbest < 0 || score <= best) { best = score; cbest = c; } /* '<=' : ties to the largest alpha */
+  }
+  *alpha = (float)((double)m * (double)cbest / (double)n_candidates);
+  free(h);
+  return 0;
+}
+
+int ocs_oracle_clip_mse_exact(const float* T, int64_t n, int bits, int is_signed,
+                              int n_candidates, float* alpha, double* scores) {
+  if (!T || !alpha || n < 0 || bits < 2 || bits > 8 || n_candidates < 1) return 1;
+  const int L = code_limit(bits, is_signed);
+  const float m = ocs_oracle_maxabs(T, n);
+  if (m == 0.0f) {
+    *alpha = 0.0f;
+    if (scores) for (int c = 0; c < n_candidates; ++c) scores[c] = 0.0;
+    return 0;
+  }
+  const double lo = is_signed ? -(double)L : 0.0, hi = (double)L;
+  double best = 0.0;
+  int cbest = -1;
+  for (int c = 1; c <= n_candidates; ++c) {
+    const float alpha_c = (float)((double)m * (double)c / (double)n_candidates);
+    const double step = (double)alpha_c / (double)L;
+    double score = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+      const double x = (double)T[i];
+      double q = nearbyint(x / step);
+      if (q < lo) q = lo;
+      if (q > hi) q = hi;
+      const double e = x - q * step;
+      score += e * e;
+    }
+    if (scores) scores[c - 1] = score;
+    if (cbest < 0 || score <= best) { best = score; cbest = c; }
+  }
+  *alpha = (float)((double)m * (double)cbest / (double)n_candidates);
+  return 0;
+}
+
+/* ------------------------------------------------------------------ Eq. 2 / Eq. 3 on codes */
+static inline int32_t act_code(const void* A, int a_signed, size_t i) {
+  return a_signed ? (int32_t)((const int8_t*)A)[i] : (int32_t)((const uint8_t*)A)[i];
+}
+
+static inline float dequant(int32_t acc, float a_scale, float w_scale, float bias) {
+  volatile float s = a_scale * w_scale; /* one rounded multiply */
+  return fmaf((float)acc, s, bias);
+}
+
+static int qlinear_one(const void* A, int a_signed, int C, const int8_t* Wc, int S,
+                       const int32_t* idx_map, int m, int n, int32_t* out) {
+  const int K = C + S;
+  int64_t acc = 0;
+  for (int j = 0; j < K; ++j) {
+    const int src = idx_map[j];
+    if (src < 0 || src >= C) return 3;
+    acc += (int64_t)act_code(A, a_signed, (size_t)m * C + src) * (int64_t)Wc[(size_t)n * K + j];
+  }
+  if (acc > INT32_MAX || acc < INT32_MIN) return 4;
+  *out = (int32_t)acc;
+  return 0;
+}
+
+int ocs_oracle_qlinear(const void* A, int a_signed, float a_scale, int M, int C,
+                       const int8_t* Wc, float w_scale, int N, int S, const int32_t* idx_map,
+                       const float* bias, float* Y, int32_t* acc) {
+  if (!A || !Wc || !idx_map || M < 0 || C <= 0 || N < 0 || S < 0) return 1;
+  int err = 0;
+#pragma omp parallel for schedule(static)
+  for (int m = 0; m < M; ++m)
+    for (int n = 0; n < N; ++n) {
+      int32_t v = 0;
+      int e = qlinear_one(A, a_signed, C, Wc, S, idx_map, m, n, &v);
+      if (e) {
+#pragma omp atomic write
+        err = e;
+        continue;
+      }
+      if (acc) acc[(size_t)m * N + n] = v;
+      if (Y) Y[(size_t)m * N + n] = dequant(v, a_scale, w_scale, bias ? bias[n] : 0.0f);
+    }
+  return err;
+}
+
+int ocs_oracle_qlinear_samples(const void* A, int a_signed, float a_scale, int M, int C,
+                               const int8_t* Wc, float w_scale, int N, int S,
+                               const int32_t* idx_map, const float* bias, const int32_t* ms,
+                               const int32_t* ns, int count, float* Y, int32_t* acc) {
+  if (!A || !Wc || !idx_map || !ms || !ns || C <= 0 || S < 0 || count < 0) return 1;
+  for (int i = 0; i < count; ++i) {
+    if (ms[i] < 0 || ms[i] >= M || ns[i] < 0 || ns[i] >= N) return 1;
+    int32_t v = 0;
+    int e = qlinear_one(A, a_signed, C, Wc, S, idx_map, ms[i], ns[i], &v);
+    if (e) return e;
+    if (acc) acc[i] = v;
+    if (Y) Y[i] = dequant(v, a_scale, w_scale, bias ? bias[ns[i]] : 0.0f);
+  }
+  return 0;
+}
+
+int ocs_oracle_qconv(const void* X, int a_signed, float a_scale, int Nb, int H, int Wd, int C,
+                     const int8_t* Wc, float w_scale, int O, int S, int kh, int kw, int stride,
+                     int pad, const int32_t* idx_map, const float* bias, float* Y, int32_t* acc) {
+  if (!X || !Wc || !idx_map || Nb < 0 || H <= 0 || Wd <= 0 || C <= 0 || O <= 0 || S < 0 ||
+      kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
+    return 1;
+  const int K = C + S;
+  const int Ho = (H + 2 * pad - kh) / stride + 1;
+  const int Wo = (Wd + 2 * pad - kw) / stride + 1;
+  if (Ho <= 0 || Wo <= 0) return 1;
+  for (int j = 0; j < K; ++j)
+    if (idx_map[j] < 0 || idx_map[j] >= C) return 3;
+  int err = 0;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int n = 0; n < Nb; ++n)
+    for (int oh = 0; oh < Ho; ++oh)
+      for (int ow = 0; ow < Wo; ++ow)
+        for (int o = 0; o < O; ++o) {
+          int64_t a = 0;
+          for (int y = 0; y < kh; ++y)
+            for (int x = 0; x < kw; ++x) {
+              const int ih = oh * stride + y - pad, iw = ow * stride + x - pad;
+              if (ih < 0 || ih >= H || iw < 0 || iw >= Wd) continue; /* zero padding */
+              const size_t px = (((size_t)n * H + ih) * Wd + iw) * C;
+              for (int j = 0; j < K; ++j)
+                a += (int64_t)act_code(X, a_signed, px + idx_map[j]) *
+                     (int64_t)Wc[(((size_t)o * K + j) * kh + y) * kw + x];
+            }
+          if (a > INT32_MAX || a < INT32_MIN) {
+#pragma omp atomic write
+            err = 4;
+            continue;
+          }
+          const size_t oi = (((size_t)n * Ho + oh) * Wo + ow) * O + o;
+          if (acc) acc[oi] = (int32_t)a;
+          if (Y) Y[oi] = dequant((int32_t)a, a_scale, w_scale, bias ? bias[o] : 0.0f);
+        }
+  return err;
+}
+
+/* ------------------------------------------------------------------ glue */
+void ocs_oracle_relu(const float* x, int64_t n, float* y) {
+  for (int64_t i = 0; i < n; ++i) y[i] = x[i] > 0.0f ? x[i] : 0.0f;
+}
+
+void ocs_oracle_add_relu(const float* a, const float* b, int64_t n, int relu, float* y) {
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float s = a[i] + b[i];
+    y[i] = (relu && !(s > 0.0f)) ? 0.0f : s;
+  }
+}
+
+void ocs_oracle_maxpool3x3s2(const float* x, int Nb, int H, int Wd, int C, float* y) {
+  const int Ho = (H + 2 - 3) / 2 + 1, Wo = (Wd + 2 - 3) / 2 + 1;
+  for (int n = 0; n < Nb; ++n)
+    for (int oh = 0; oh < Ho; ++oh)
+      for (int ow = 0; ow < Wo; ++ow)
+        for (int c = 0; c < C; ++c) {
+          float m = -INFINITY;
+          for (int dy = 0; dy < 3; ++dy)
+            for (int dx = 0; dx < 3; ++dx) {
+              const int ih = oh * 2 + dy - 1, iw = ow * 2 + dx - 1;
+              if (ih < 0 || ih >= H || iw < 0 || iw >= Wd) continue; /* padding never wins */
+              const float v = x[(((size_t)n * H + ih) * Wd + iw) * C + c];
+              if (v > m) m = v;
+            }
+          y[(((size_t)n * Ho + oh) * Wo + ow) * C + c] = m;
+        }
+}
+
+void ocs_oracle_global_avgpool(const float* x, int Nb, int H, int Wd, int C, float* y) {
+  volatile float inv = 1.0f / (float)(H * Wd);
+  for (int n = 0; n < Nb; ++n)
+    for (int c = 0; c < C; ++c) {
+      volatile float s = 0.0f;
+      for (int h = 0; h < H; ++h)
+        for (int w = 0; w < Wd; ++w) s = s + x[(((size_t)n * H + h) * Wd + w) * C + c];
+      y[(size_t)n * C + c] = s * inv;
+    }
+}
+
+void ocs_oracle_nchw_to_nhwc(const float* x, int Nb, int C, int H, int Wd, float* y) {
+  for (int n = 0; n < Nb; ++n)
+    for (int c = 0; c < C; ++c)
+      for (int h = 0; h < H; ++h)
+        for (int w = 0; w < Wd; ++w)
+          y[(((size_t)n * H + h) * Wd + w) * C + c] = x[(((size_t)n * C + c) * H + h) * Wd + w];
+}
+
+/* exp(x) for x <= 0 clamped at -87: t = x*log2(e), n = rint(t), f = t - n in [-0.5, 0.5],
+ * 2^f by a degree-6 Taylor polynomial in f*ln2 evaluated with fmaf (Horner), scaled by 2^n. */
+static float exp_neg(float x) {
+  if (x < -87.0f) x = -87.0f;
+  volatile float t = x * 1.44269504088896341f;
+  const float n = nearbyintf(t);
+  volatile float f = t - n;
+  volatile float g = f * 0.693147180559945309f;
+  float p = 1.0f / 720.0f;
+  p = fmaf(p, g, 1.0f / 120.0f);
+  p = fmaf(p, g, 1.0f / 24.0f);
+  p = fmaf(p, g, 1.0f / 6.0f);
+  p = fmaf(p, g, 0.5f);
+  p = fmaf(p, g, 1.0f);
+  p = fmaf(p, g, 1.0f);
+  return ldexpf(p, (int)n);
+}
+
+float ocs_oracle_sigmoid(float x) {
+  /* 1/(1+e^-|x|) on the negative side, mirrored */
+  const float e = exp_neg(-fabsf(x));
+  volatile float den = 1.0f + e;
+  volatile float s = 1.0f / den;        /* sigmoid(|x|) */
+  if (x >= 0.0f) return s;
+  volatile float r = e / den;           /* sigmoid(-|x|) */
+  return r;
+}
+
+float ocs_oracle_tanh(float x) {
+  volatile float a = -2.0f * fabsf(x);
+  const float e = exp_neg(a);
+  volatile float num = 1.0f - e;
+  volatile float den = 1.0f + e;
+  volatile float r = num / den;
+  return x < 0.0f ? -r : r;
+}
+
+void ocs_oracle_lstm_cell(const float* g_ih, const float* g_hh, int batch, int hidden, float* c,
+                          float* h) {
+  for (int b = 0; b < batch; ++b)
+    for (int k = 0; k < hidden; ++k) {
+      const size_t base = (size_t)b * 4 * hidden;
+      volatile float zi = g_ih[base + k] + g_hh[base + k];
+      volatile float zf = g_ih[base + hidden + k] + g_hh[base + hidden + k];
+      volatile float zg = g_ih[base + 2 * hidden + k] + g_hh[base + 2 * hidden + k];
+      volatile float zo = g_ih[base + 3 * hidden + k] + g_hh[base + 3 * hidden + k];
+      const float i = ocs_oracle_sigmoid(zi), f = ocs_oracle_sigmoid(zf);
+      const float g = ocs_oracle_tanh(zg), o = ocs_oracle_sigmoid(zo);
+      volatile float ig = i * g;
+      const float cn = fmaf(f, c[(size_t)b * hidden + k], ig);
+      c[(size_t)b * hidden + k] = cn;
+      volatile float hn = o * ocs_oracle_tanh(cn);
+      h[(size_t)b * hidden + k] = hn;
+    }
+}

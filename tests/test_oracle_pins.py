@@ -1,0 +1,402 @@
+"""Pins for the CPU checker: every function is tied to something other than itself --
+values the paper prints, closed forms, invariants, library routines or brute force."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from ocs_inputs import configs, prng
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_golden(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                rows.append(line.split())
+    return rows
+
+
+# ----------------------------------------------------------------------------- Section 3.4
+def test_split_count_is_ceil_rC():
+    assert orc.num_splits(512, 0.05) == 26
+    assert orc.num_splits(256, 0.02) == 6
+    assert [orc.num_splits(25088, r) for r in (0, .01, .02, .05, .1)] == [0, 251, 502, 1255, 2509]
+    assert orc.num_splits(650, 0.02) == 13          # 0.02*650 is 13 in exact arithmetic
+    assert [orc.num_splits(c, .01) for c in (3, 64, 128, 256, 512, 1024, 2048)] == [1, 1, 2, 3, 6, 11, 21]
+    for c in range(1, 300):
+        for num in range(0, 40):
+            r = num / 100.0
+            assert orc.num_splits(c, r) == math.ceil(Fraction(num, 100) * c)
+
+
+def test_resnet50_size_overhead_matches_table5():
+    """Table 5: relative weight size of ResNet-50 at r = .01/.02/.05/.1 is 1.01/1.02/1.05/1.1;
+    Section 5.2: r = 0.01 is a single split in many layers."""
+    layers, fc = configs.resnet50_layers()
+    alls = layers + [fc]
+    base = sum(l.O * l.C * l.k * l.k for l in alls)
+    for ratio, printed in _read_golden("table5_resnet50_weight_overhead.txt"):
+        tot = sum(l.O * (l.C + orc.num_splits(l.C, float(ratio))) * l.k * l.k for l in alls)
+        skip = sum(l.O * (l.C + (0 if l.name == "conv1" else orc.num_splits(l.C, float(ratio)))) * l.k * l.k
+                   for l in alls)
+        assert tot / base >= 1 + float(ratio)           # Section 5.4: r is a lower bound
+        assert round(tot / base, len(printed.split(".")[1])) == float(printed)
+        assert round(skip / base, len(printed.split(".")[1])) == float(printed)
+    assert sum(1 for l in alls if orc.num_splits(l.C, 0.01) == 1) >= 4
+
+
+# ----------------------------------------------------------------------------- Section 3.3
+def _Q(x: Fraction) -> int:
+    return math.floor(x + Fraction(1, 2))
+
+
+def test_paper_worked_example_w3():
+    """Section 3.3: w = 3 splits into 1.5 and 1.5, both rounded the same way, so the naive
+    halves no longer sum to Q(w)."""
+    W = np.array([[3.0]], dtype=np.float32)
+    out, idx, order, _ = orc.split(W, 1, qa_step=0.0)
+    assert out.tolist() == [[1.5, 1.5]] and idx.tolist() == [0, 0] and order.tolist() == [0]
+    assert _Q(Fraction(1.5)) + _Q(Fraction(1.5)) == 4 != _Q(Fraction(3))
+    qa, _, _, _ = orc.split(W, 1, qa_step=1.0)
+    assert qa.tolist() == [[1.25, 1.75]]          # (w - .5)/2 stays in place, (w + .5)/2 is appended
+    assert _Q(Fraction(1.25)) + _Q(Fraction(1.75)) == 3
+
+
+def test_qa_identity_and_hermite_bruteforce():
+    """Q((w-.5)/2) + Q((w+.5)/2) = Q(w) for Q = floor(x + 1/2) on a fine grid, evaluated exactly on
+    what the checker's split produced; the naive rule fails somewhere; Hermite with n = 2."""
+    ws = np.arange(-40 * 64, 40 * 64 + 1, dtype=np.float64) / 64.0
+    # one column per value: a [1, n] matrix, one split each -> do them one at a time through
+    # the checker so that each value is the channel maximum
+    naive_fail = 0
+    for chunk in np.array_split(ws, 64):
+        for w in chunk[:: max(1, len(chunk) // 12)]:
+            W = np.array([[w]], dtype=np.float32)
+            qa, _, _, _ = orc.split(W, 1, qa_step=1.0)
+            a, b = Fraction(float(qa[0, 0])), Fraction(float(qa[0, 1]))
+            assert a == (Fraction(w) - Fraction(1, 2)) / 2 and b == (Fraction(w) + Fraction(1, 2)) / 2
+            assert _Q(a) + _Q(b) == _Q(Fraction(w))
+            nv, _, _, _ = orc.split(W, 1, qa_step=0.0)
+            naive_fail += (_Q(Fraction(float(nv[0, 0]))) + _Q(Fraction(float(nv[0, 1]))) != _Q(Fraction(w)))
+    assert naive_fail > 0
+    for k in range(-40 * 64, 40 * 64 + 1):
+        x = Fraction(k, 64)
+        assert math.floor(x) + math.floor(x + Fraction(1, 2)) == math.floor(2 * x)
+        assert _Q((x - Fraction(1, 2)) / 2) + _Q((x + Fraction(1, 2)) / 2) == _Q(x)
+
+
+def test_qa_split_whole_channel_in_grid_units():
+    """A whole channel moves together (Section 3.2) and every element gets the QA pair."""
+    rng = np.random.default_rng(5)
+    W = (rng.integers(-200, 200, size=(7, 5)) / 8.0).astype(np.float32)
+    W[3, 2] = 50.0
+    out, idx, order, mx = orc.split(W, 1, qa_step=1.0)
+    assert order.tolist() == [2] and idx.tolist() == [0, 1, 2, 3, 4, 2]
+    np.testing.assert_array_equal(out[:, [0, 1, 3, 4]], W[:, [0, 1, 3, 4]])
+    np.testing.assert_array_equal(out[:, 2], (W[:, 2] - 0.5) / 2)
+    np.testing.assert_array_equal(out[:, 5], (W[:, 2] + 0.5) / 2)
+    assert mx == (50.0, max(25.25, float(np.abs(out).max())))
+
+
+# ----------------------------------------------------------------------------- Eq. 3
+@pytest.mark.parametrize("shape,S", [((33, 20), 7), ((16, 12, 3, 3), 5), ((9, 1), 4), ((5, 6), 0), ((4, 3), 9)])
+def test_functional_identity_and_exact_halving(shape, S):
+    rng = np.random.default_rng(11)
+    W = rng.laplace(0, 0.02, size=shape).astype(np.float32)
+    W.reshape(-1)[rng.integers(0, W.size, 3)] *= 30
+    out, idx, order, mx = orc.split(W, S, qa_step=0.0, literal=True)
+    Cn = shape[1]
+    assert idx[:Cn].tolist() == list(range(Cn))
+    # every entry is the source value times an exact power of two, per-source sums are exact
+    src = W[:, idx]
+    ratio = np.where(src != 0, out / np.where(src == 0, 1, src), 1.0)
+    assert np.all(np.log2(ratio) == np.round(np.log2(ratio)))
+    summed = np.zeros(W.shape, dtype=np.float64)
+    np.add.at(summed, (slice(None), idx), out.astype(np.float64))   # exact: binary fractions of one value
+    np.testing.assert_array_equal(summed, W.astype(np.float64))
+    # layer output unchanged (Eq. 3 equals Eq. 2) for a random activation vector
+    x = rng.standard_normal(Cn)
+    W2 = W.reshape(shape[0], Cn, -1).astype(np.float64)
+    o2 = out.reshape(shape[0], Cn + S, -1).astype(np.float64)
+    y_ref = np.einsum("c,ocr->or", x, W2)
+    y_new = np.einsum("c,ocr->or", x[idx], o2)
+    np.testing.assert_allclose(y_new, y_ref, rtol=0, atol=1e-12 * np.abs(W2).sum())
+    assert mx[0] == np.abs(W).max() and mx[1] == np.abs(out).max()
+
+
+def test_greedy_is_monotone_and_targets_the_outlier():
+    """Section 3.4 / 5.2: each split halves the current maximum's channel; the maximum never
+    rises; with a unique largest outlier the first split strictly narrows the range."""
+    c1 = configs.config1()
+    W = c1["W"]
+    prev = np.abs(W).max()
+    j0 = int(np.unravel_index(np.abs(W).argmax(), W.shape)[1])
+    for S in range(1, 27):
+        out, idx, order, mx = orc.split(W, S)
+        cur = np.abs(out).max()
+        assert cur <= prev
+        prev = cur
+        if S == 1:
+            assert order[0] == j0 and cur < np.abs(W).max()
+            assert np.abs(out[:, j0]).max() == np.abs(W[:, j0]).max() / 2
+    # literal rescans and cached maxima agree, naive and QA
+    for qa in (0.0, float(np.abs(W).max()) / 127):
+        a = orc.split(W, 26, qa, literal=True)
+        b = orc.split(W, 26, qa, literal=False)
+        np.testing.assert_array_equal(a[0], b[0])
+        np.testing.assert_array_equal(a[1], b[1])
+        np.testing.assert_array_equal(a[2], b[2])
+    # config 1 re-splits at least one copy (an appended index appears in split_order)
+    assert (orc.split(W, 26)[2] >= 512).any()
+
+
+def test_greedy_bruteforce_python():
+    """Independent re-derivation of the greedy loop with python floats on a tiny tensor, ties
+    included (equal magnitudes: smallest current index first)."""
+    W = np.array([[4, -4, 1, 0.5], [1, 2, -4, 0.25]], dtype=np.float32)
+    S = 6
+    cols = [list(map(float, W[:, j])) for j in range(4)]
+    src = [0, 1, 2, 3]
+    order = []
+    for _ in range(S):
+        mags = [max(abs(v) for v in c) for c in cols]
+        j = max(range(len(cols)), key=lambda t: (mags[t], -t))
+        order.append(j)
+        half = [v / 2 for v in cols[j]]
+        cols[j] = half
+        cols.append(list(half))
+        src.append(src[j])
+    out, idx, so, _ = orc.split(W, S, literal=True)
+    assert so.tolist() == order and idx.tolist() == src
+    np.testing.assert_array_equal(out, np.array(cols, dtype=np.float32).T)
+
+
+def test_split_degenerate():
+    Z = np.zeros((3, 4), dtype=np.float32)
+    out, idx, order, mx = orc.split(Z, 5)
+    assert not out.any() and order.tolist() == [0] * 5 and idx.tolist() == [0, 1, 2, 3, 0, 0, 0, 0, 0]
+    W = np.array([[2.0], [-6.0]], dtype=np.float32)            # C = 1, S > C
+    out, idx, order, mx = orc.split(W, 3)
+    assert idx.tolist() == [0, 0, 0, 0] and order.tolist() == [0, 0, 1]
+    np.testing.assert_array_equal(out, np.array([[.5, .5, .5, .5], [-1.5, -1.5, -1.5, -1.5]], dtype=np.float32))
+    np.testing.assert_array_equal(out.sum(axis=1), W[:, 0])
+
+
+# ----------------------------------------------------------------------------- Eq. 1
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 8])
+def test_linear_quant_grid(bits):
+    """Eq. 1: 2^k - 1 grid points spanning [-max, max]; error at most half an increment."""
+    rng = np.random.default_rng(bits)
+    x = rng.uniform(-1, 1, 10000).astype(np.float32)
+    x = np.concatenate([x, -x])
+    alpha = orc.maxabs(x)
+    assert alpha == np.abs(x).max()
+    codes, scale = orc.quantize(x, bits, True, alpha)
+    L = 2 ** (bits - 1) - 1
+    assert codes.min() >= -L and codes.max() <= L
+    assert len(np.unique(codes)) <= 2 ** bits - 1
+    if bits <= 6:
+        assert len(np.unique(codes)) == 2 ** bits - 1
+    assert scale == np.float32(alpha) / np.float32(L)
+    err = np.abs(x.astype(np.float64) - codes.astype(np.float64) * scale)
+    assert err.max() <= 0.5 * scale * (1 + 1e-5)
+    # textbook form round(x L / max) * max / L, in double, away from rounding ties
+    t = x.astype(np.float64) * L / float(alpha)
+    safe = np.abs(t - np.floor(t) - 0.5) > 1e-4
+    assert np.array_equal(codes[safe], np.rint(t[safe]).astype(np.int8))
+    assert codes[np.abs(x).argmax()] in (-L, L)
+
+
+def test_quantize_clip_saturates_and_rne():
+    x = np.array([-3.0, -1.0, -0.5, 0.0, 0.5, 1.0, 1.5, 2.5, 3.0, 100.0], dtype=np.float32)
+    codes, scale = orc.quantize(x, 3, True, 3.0)               # L = 3, step 1
+    assert scale == 1.0
+    assert codes.tolist() == [-3, -1, 0, 0, 0, 1, 2, 2, 3, 3]     # halves to even, 100 saturates
+    ucodes, uscale = orc.quantize(x, 2, False, 3.0)            # L_u = 3
+    assert ucodes.dtype == np.uint8 and ucodes.tolist() == [0, 0, 0, 0, 0, 1, 2, 2, 3, 3]
+    z, s = orc.quantize(np.zeros(5, np.float32), 8, True, 0.0)
+    assert not z.any() and s == 0.0
+
+
+# ----------------------------------------------------------------------------- Section 4.1
+def _brute_clip(values, counts, m: Fraction, bits, n_cand, signed=True):
+    """Exact rational evaluation of the histogram MSE for every candidate."""
+    L = 2 ** (bits - 1) - 1 if signed else 2 ** bits - 1
+    best, cbest, scores = None, None, []
+    for c in range(1, n_cand + 1):
+        alpha = Fraction(float(np.float32(float(m * c / n_cand))))   # thresholds are fp32 values
+        assert abs(alpha - m * c / n_cand) <= m * Fraction(1, 2 ** 23)  # evenly spaced on (0, max]
+        step = alpha / L
+        sc = Fraction(0)
+        for xb, h in zip(values, counts):
+            t = xb / step
+            q = math.floor(t + Fraction(1, 2))
+            if t + Fraction(1, 2) == q and q % 2 == 1:   # exact tie: to even
+                q -= 1
+            q = max(-L if signed else 0, min(L, q))
+            sc += h * (xb - q * step) ** 2
+        scores.append(sc)
+        if best is None or sc <= best:
+            best, cbest = sc, c
+    return cbest, scores
+
+
+@pytest.mark.parametrize("bits,n_cand,seed", [(2, 8, 0), (3, 16, 1), (4, 16, 2), (3, 5, 3), (2, 16, 4)])
+def test_clip_mse_bruteforce(bits, n_cand, seed):
+    """Tiny tensors whose values sit on bin centres: the histogram is the data, so the search
+    must agree with an exact enumeration of every (threshold, grid point)."""
+    B = 64
+    rng = np.random.default_rng(seed)
+    m = 2.0                                         # power of two: bin edges exact in fp32
+    bins = np.unique(np.concatenate([rng.integers(0, 20, 40), rng.integers(0, B - 1, 6), [B - 1]]))
+    counts = rng.integers(1, 9, size=bins.size)
+    vals = []
+    for b, h in zip(bins, counts):
+        centre = (b + 0.5) * m / B
+        vals += [centre] * int(h)
+    vals = np.array(vals, dtype=np.float32)
+    vals[-1] = m                                    # the maximum itself falls in the last bin
+    vals *= rng.choice([-1.0, 1.0], size=vals.size).astype(np.float32)
+    res = orc.clip_mse(vals, bits, True, n_bins=B, n_candidates=n_cand)
+    hist = res["hist"]
+    assert hist.sum() == vals.size and res["max_abs"] == m
+    expect = np.zeros(B, dtype=np.uint64)
+    expect[bins] = counts.astype(np.uint64)
+    np.testing.assert_array_equal(hist, expect)
+    centres = [Fraction(int(b) * 2 + 1, 2) * Fraction(2, B) for b in range(B)]
+    cbest, scores = _brute_clip(centres, [int(h) for h in hist], Fraction(2), bits, n_cand)
+    np.testing.assert_allclose(res["scores"], [float(s) for s in scores], rtol=1e-12, atol=1e-15)
+    gaps = sorted(float(s) for s in scores)
+    if gaps[1] - gaps[0] > 1e-9:                    # unambiguous minimum
+        assert res["alpha"] == np.float32(2.0 * cbest / n_cand)
+
+
+def test_clip_mse_properties():
+    rng = np.random.default_rng(7)
+    x = rng.laplace(0, 0.01, 50000).astype(np.float32)
+    x[17] = 1.0                                     # one huge outlier, few bits -> must clip
+    r = orc.clip_mse(x, 3, True)
+    assert 0 < r["alpha"] < 1.0
+    assert r["hist"].sum() == x.size
+    # candidates are evenly spaced on (0, max]; the last one is "no clipping"
+    r8 = orc.clip_mse(x, 8, True, n_candidates=4)
+    assert r8["alpha"] in [np.float32(0.25 * k) for k in (1, 2, 3, 4)]
+    # the same search on the raw elements picks a nearby candidate
+    ex = orc.clip_mse_exact(x[:5000], 4, True, 64)
+    hs = orc.clip_mse(x[:5000], 4, True, 2048, 64)
+    assert abs(ex["alpha"] - hs["alpha"]) <= 2 * orc.maxabs(x[:5000]) / 64 + 1e-9
+    # scoring really is sum h * (x - Q(x))^2 at the bin centres: recompute with numpy
+    m, B, L = r["max_abs"], 2048, 3
+    centres = (np.arange(B) + 0.5) * (m / B)
+    for c in (1, 37, 128):
+        step = float(np.float32(m * c / 128)) / L
+        q = np.clip(np.rint(centres / step), -L, L)
+        np.testing.assert_allclose(r["scores"][c - 1], (r["hist"] * (centres - q * step) ** 2).sum(), rtol=1e-10)
+    assert orc.clip_mse(np.zeros(10, np.float32), 4)["alpha"] == 0.0
+
+
+def test_clip_none_is_last_candidate():
+    """With every value on the 8-bit grid of its own maximum, no clipping has zero error and
+    wins (ties go to the largest threshold)."""
+    x = (np.arange(-127, 128) / 127.0).astype(np.float32)
+    r = orc.clip_mse_exact(x, 8, True, 16)
+    assert r["alpha"] == 1.0
+
+
+# ----------------------------------------------------------------------------- Eq. 2 / 3 on codes
+def test_qlinear_matches_expanded_and_folded_matmul():
+    M, Cn, N, S = 9, 37, 13, 6
+    A = configs.random_codes(1, 0, (M, Cn), 0, 255, np.uint8)
+    Wc = configs.random_codes(1, 1, (N, Cn + S), -127, 127, np.int8)
+    idx = np.concatenate([np.arange(Cn), configs.random_codes(1, 2, (S,), 0, Cn - 1, np.int32)]).astype(np.int32)
+    bias = prng.normal(1, 9, (N,))
+    Y, acc = orc.qlinear(A, False, 0.013, Wc, 0.0007, idx, bias)
+    expanded = A.astype(np.int64)[:, idx] @ Wc.astype(np.int64).T
+    np.testing.assert_array_equal(acc, expanded)
+    folded = np.zeros((N, Cn), dtype=np.int64)
+    np.add.at(folded, (slice(None), idx), Wc.astype(np.int64))
+    np.testing.assert_array_equal(acc, A.astype(np.int64) @ folded.T)
+    s = np.float32(0.013) * np.float32(0.0007)
+    np.testing.assert_allclose(Y, acc.astype(np.float64) * float(s) + bias, rtol=2e-7, atol=1e-9)
+    # signed activations, identity map = plain integer matmul
+    As = configs.random_codes(2, 0, (M, Cn), -127, 127, np.int8)
+    _, acc0 = orc.qlinear(As, True, 1.0, Wc[:, :Cn].copy(), 1.0, np.arange(Cn, dtype=np.int32))
+    np.testing.assert_array_equal(acc0, As.astype(np.int64) @ Wc[:, :Cn].astype(np.int64).T)
+    ms, ns = np.array([0, 3, 8], np.int32), np.array([12, 0, 5], np.int32)
+    Ys, accs = orc.qlinear_samples(A, False, 0.013, Wc, 0.0007, idx, ms, ns, bias)
+    np.testing.assert_array_equal(accs, acc[ms, ns])
+    np.testing.assert_array_equal(Ys, Y[ms, ns])
+
+
+@pytest.mark.parametrize("k,stride,pad,H", [(3, 1, 1, 7), (3, 2, 1, 8), (1, 2, 0, 6), (7, 2, 3, 11), (1, 1, 0, 5)])
+def test_qconv_matches_library_conv(k, stride, pad, H):
+    torch = pytest.importorskip("torch")
+    Nb, Cn, O, S = 2, 5, 4, 3
+    X = configs.random_codes(3, 0, (Nb, H, H + 1, Cn), 0, 255, np.uint8)
+    Wc = configs.random_codes(3, 1, (O, Cn + S, k, k), -127, 127, np.int8)
+    idx = np.concatenate([np.arange(Cn), [4, 0, 4]]).astype(np.int32)
+    bias = prng.normal(3, 9, (O,))
+    Y, acc = orc.qconv(X, False, 0.5, Wc, 0.25, idx, stride, pad, bias)
+    xe = torch.from_numpy(X.astype(np.float64)[..., idx]).permute(0, 3, 1, 2)
+    ref = torch.nn.functional.conv2d(xe, torch.from_numpy(Wc.astype(np.float64)), stride=stride, padding=pad)
+    ref = ref.permute(0, 2, 3, 1).numpy()
+    np.testing.assert_array_equal(acc, ref.astype(np.int64))
+    np.testing.assert_allclose(Y, ref * 0.125 + bias, rtol=2e-7, atol=1e-9)
+
+
+# ----------------------------------------------------------------------------- glue
+def test_glue_against_library_routines():
+    torch = pytest.importorskip("torch")
+    x = prng.normal(5, 0, (2, 9, 11, 6))
+    np.testing.assert_array_equal(orc.relu(x), np.maximum(x, 0))
+    y = prng.normal(5, 1, (2, 9, 11, 6))
+    np.testing.assert_array_equal(orc.add_relu(x, y, True), np.maximum(x + y, 0))
+    np.testing.assert_array_equal(orc.add_relu(x, y, False), x + y)
+    t = torch.from_numpy(x).permute(0, 3, 1, 2)
+    mp = torch.nn.functional.max_pool2d(t, 3, 2, 1).permute(0, 2, 3, 1).numpy()
+    np.testing.assert_array_equal(orc.maxpool3x3s2(x), mp)
+    np.testing.assert_allclose(orc.global_avgpool(x), x.astype(np.float64).mean(axis=(1, 2)), rtol=1e-5, atol=1e-6)
+    nchw = prng.normal(5, 2, (2, 3, 4, 5))
+    np.testing.assert_array_equal(orc.nchw_to_nhwc(nchw), nchw.transpose(0, 2, 3, 1))
+
+
+def test_lstm_cell_against_libm():
+    xs = np.linspace(-30, 30, 2001)
+    sg = np.array([orc.sigmoid(float(v)) for v in xs])
+    th = np.array([orc.tanh(float(v)) for v in xs])
+    np.testing.assert_allclose(sg, 1 / (1 + np.exp(-xs)), rtol=0, atol=3e-7)
+    np.testing.assert_allclose(th, np.tanh(xs), rtol=0, atol=3e-7)
+    assert orc.sigmoid(0.0) == 0.5 and orc.tanh(0.0) == 0.0
+    b, hdim = 3, 5
+    gi, gh = prng.normal(6, 0, (b, 4 * hdim)), prng.normal(6, 1, (b, 4 * hdim))
+    c0 = prng.normal(6, 2, (b, hdim))
+    c1, h1 = orc.lstm_cell(gi, gh, c0)
+    z = (gi + gh).astype(np.float64)
+    i, f, g, o = (z[:, k * hdim:(k + 1) * hdim] for k in range(4))
+    sig = lambda v: 1 / (1 + np.exp(-v))
+    c_ref = sig(f) * c0 + sig(i) * np.tanh(g)
+    np.testing.assert_allclose(c1, c_ref, atol=2e-6)
+    np.testing.assert_allclose(h1, sig(o) * np.tanh(c_ref), atol=2e-6)
+
+
+# ----------------------------------------------------------------------------- inputs
+def test_input_streams_are_reproducible_and_shaped():
+    a, b = configs.config1(), configs.config1()
+    np.testing.assert_array_equal(a["W"], b["W"])
+    W = a["W"]
+    std = 0.02 * np.sqrt(2)
+    assert (np.abs(W) > 9.9 * std).sum() == 8 and np.abs(W).max() <= 20 * std * 1.0001
+    assert a["A"].min() >= 0
+    c3 = configs.config3(O=256, C=1568, M=8)
+    big = np.abs(c3["W"]) == np.float32(15 * 0.005 * np.sqrt(2))
+    assert big.sum() == round(1e-4 * 256 * 1568)
+    u = prng.Stream(9, 0).uniform(0, 100000)
+    assert abs(u.mean() - 0.5) < 5e-3 and 0 < u.min() and u.max() < 1
+    np.testing.assert_array_equal(prng.Stream(9, 0).bits(1000, 10), prng.Stream(9, 0).bits(0, 1010)[1000:])
