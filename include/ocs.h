@@ -1,0 +1,168 @@
+/*
+ * ocs.h -- C ABI of the B200 (sm_100a) library for outlier channel splitting (OCS)
+ * post-training quantization, after Zhao et al., "Improving Neural Network Quantization
+ * without Retraining using Outlier Channel Splitting", ICML 2019 (arXiv:1901.09504).
+ *
+ * Common rules for every call
+ *  - Every pointer is a DEVICE pointer owned by the caller unless it is marked "host".
+ *    The library allocates nothing; scratch memory comes in through (ws, ws_bytes), whose
+ *    minimum size the matching *_workspace_bytes() query returns (host call, no GPU work).
+ *    ws must be 256-byte aligned.  Inputs are never modified; outputs must not alias inputs.
+ *  - Every call only enqueues work on `stream` (a cudaStream_t passed as void*) and returns
+ *    without synchronising.  Scalar results (scales, thresholds, maxima) are written to
+ *    device memory.
+ *  - The return value reports what the host can see before launching (ocs_status).
+ *    Conditions only the device can see are OR-ed into the caller's device status word
+ *    `dev_status` (OCS_DEV_* bits; may be NULL to ignore); read it with ocs_poll_status().
+ *    A kernel that gives up on a bounded wait sets OCS_DEV_TIMEOUT and returns normally.
+ *  - There is no CPU fallback: on a machine without an sm_100 GPU the calls return
+ *    OCS_ERR_UNSUPPORTED or OCS_ERR_CUDA.
+ *
+ * Notation: W fp32 [O][C][R] (O outputs, C input channels, R = kh*kw filter taps, R = 1 for
+ * fully-connected and LSTM matrices); "channel" = input channel (Section 3.2).  S splits
+ * give C+S expanded channels.  L = 2^(k-1)-1 for signed k-bit codes (Eq. 1: 2^k-1 grid
+ * points), L_u = 2^k-1 for unsigned codes.
+ */
+#ifndef OCS_H
+#define OCS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  OCS_OK = 0,
+  OCS_ERR_INVALID_ARG = 1, /* null pointer, bits outside [2,8], negative ratio, n_candidates < 1 ... */
+  OCS_ERR_SHAPE = 2,       /* non-positive dims, leading dimension too small, misaligned pointer / ld */
+  OCS_ERR_WORKSPACE = 3,   /* ws NULL, misaligned or smaller than the query result */
+  OCS_ERR_UNSUPPORTED = 4, /* device is not sm_100, or a documented size limit is exceeded */
+  OCS_ERR_CUDA = 5         /* a CUDA runtime / driver call failed */
+} ocs_status;
+
+/* bits of the device status word */
+#define OCS_DEV_NONFINITE 1 /* an input held NaN or Inf; outputs unspecified */
+#define OCS_DEV_BAD_INDEX 2 /* an idx_map entry was outside [0, C); it was read as channel 0 */
+#define OCS_DEV_TIMEOUT 4   /* a bounded pipeline wait expired; outputs unspecified */
+#define OCS_DEV_DEPTH 8     /* a channel was re-split more than 63 times under the QA rule */
+
+typedef enum {
+  OCS_CLIP_NONE = 0, /* alpha = max|T| (Eq. 1) */
+  OCS_CLIP_MSE = 1   /* histogram MSE search (Section 4.1) */
+} ocs_clip_mode;
+
+/* Host helpers ------------------------------------------------------------------------- */
+
+/* Section 3.4: number of splits for a layer with C channels at expansion ratio r,
+ * ceil(r*C), evaluated in double as ceil(r*C - 1e-9) so that products that are integers in
+ * exact arithmetic do not round up; 0 for r <= 0.  Host only. */
+int ocs_num_splits(int C, double ratio);
+
+/* Copies the device status word to *host_out (host pointer) after synchronising `stream`.
+ * Returns OCS_ERR_CUDA if the copy fails. */
+ocs_status ocs_poll_status(const int* dev_status, void* stream, int* host_out);
+
+/* Version string of the build (host). */
+const char* ocs_version(void);
+
+/* ocs_split -------------------------------------------------------------------------------
+ * Weight OCS (Section 3.2 Eq. 3, Section 3.3, Section 3.4): S times, take the channel that
+ * holds the largest |w| of the CURRENT expanded tensor (ties: the smallest current channel
+ * index), duplicate it, and replace every value w of it by the pair
+ *      kept in place  : fl(fl(w - d) * 0.5)        appended at index C+s : fl(fl(w + d) * 0.5)
+ * with d = qa_step/2.  d = 0 is plain halving (Net2WiderNet); d = half a quantization step
+ * is the quantization-aware split ((w-0.5)/2, (w+0.5)/2) of Section 3.3 in weight units.
+ *   qa_bits = 0 : use the given qa_step (>= 0).
+ *   qa_bits in [2,8] : the step is chosen on the device: the greedy loop is first run with
+ *       d = 0 on the channel extrema, qa_step = (max|W'| predicted by that run) / L(qa_bits),
+ *       then the loop is run again with that step (qa_step argument ignored).
+ * Layouts: W [O][C][R] with row stride ld_in >= C*R floats; W_out [O][C+S][R] with row
+ * stride ld_out >= (C+S)*R floats (when both strides are multiples of 4 and both bases are
+ * 16-byte aligned the kernels use 128-bit accesses).  idx_map [C+S]: ORIGINAL source channel of
+ * each expanded channel (idx_map[j] = j for j < C).  split_order [S] (nullable): expanded
+ * index chosen at each step.  max_abs_out [3] (nullable): max|W|, max|W_out|, qa_step used.
+ * Limits: C*R and (C+S)*R below 2^31; S may exceed C.
+ * Errors: INVALID_ARG, SHAPE, WORKSPACE as above.  Device flags: NONFINITE, DEPTH. */
+size_t ocs_split_workspace_bytes(int O, int C, int R, int S);
+ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step,
+                     int qa_bits, float* W_out, int64_t ld_out, int32_t* idx_map,
+                     int32_t* split_order, float* max_abs_out, void* ws, size_t ws_bytes,
+                     int* dev_status, void* stream);
+
+/* ocs_quantize ----------------------------------------------------------------------------
+ * k-bit linear quantization (Eq. 1) with the clip threshold alpha in place of max|x|
+ * (Section 4): step = alpha/L, inv = L/alpha (fp32), code = clamp(rint(x*inv), -L, L) with
+ * round-half-to-even; unsigned (is_signed = 0): clamp to [0, L_u].  Codes live in 8-bit
+ * containers for every k (uint8 bit pattern when unsigned).
+ *   mode NONE: alpha = max|T|.   mode MSE (Section 4.1): histogram of |x| with n_bins equal
+ *   bins on [0, max|T|]; candidates alpha_c = max*c/n_candidates, c = 1..n_candidates;
+ *   score_c = sum_b h[b]*(x_b - Q_c(x_b))^2 at the bin centres x_b, in double; the smallest
+ *   score wins, ties go to the largest alpha.
+ * T [rows][cols] fp32 with row stride ld_in; codes [rows][cols] with row stride ld_codes bytes
+ * (bytes beyond cols in a row are left untouched).  max_abs_in (nullable): device scalar
+ * holding max|T| if the caller already has it (saves one pass over T).  *scale = step,
+ * *alpha = chosen threshold (device scalars; alpha nullable).  An all-zero tensor gives zero
+ * codes, scale 0, alpha 0.  n_bins <= 4096, n_candidates <= 1024 (ignored for mode NONE).
+ * Device flags: NONFINITE. */
+size_t ocs_quantize_workspace_bytes(int n_bins, int n_candidates);
+ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, int64_t ld_in, int bits,
+                        int is_signed, ocs_clip_mode mode, int n_candidates, int n_bins,
+                        const float* max_abs_in, int8_t* codes, int64_t ld_codes, float* scale,
+                        float* alpha, void* ws, size_t ws_bytes, int* dev_status, void* stream);
+
+/* Reads back the search's intermediate results after an MSE-mode ocs_quantize on the same
+ * workspace (for tests and reports): hist [n_bins] uint64 and scores [n_candidates] double,
+ * both device pointers into ws.  Host call, no GPU work. */
+void ocs_quantize_workspace_views(void* ws, int n_bins, int n_candidates, uint64_t** hist,
+                                  double** scores);
+
+/* ocs_qlinear -----------------------------------------------------------------------------
+ * The split layer of Eq. 3 evaluated on integer codes (Eq. 2 on low-precision MACs):
+ *     acc[m][n] = sum_{j < C+S} A[m][idx_map[j]] * Wc[n][j]          (int32, exact)
+ *     Y[m][n]   = fmaf((float)acc[m][n], a_scale * w_scale, bias[n])  (bias 0 if NULL)
+ * The duplicated activation channels (Section 3.5: "copies ... the appropriate channels")
+ * are gathered through idx_map while the operand tiles are staged; an expanded activation
+ * tensor is never written.  idx_map[j] must equal j for j < C (as ocs_split produces).
+ * A codes [M][C], row stride lda bytes, uint8 when a_signed = 0 else int8; Wc int8 [N][C+S],
+ * row stride ldw bytes, ldw a multiple of 16 and Wc 16-byte aligned; a_scale / w_scale
+ * device scalars; Y fp32 [M][N] row stride ldy floats; acc_out (nullable) int32 [M][N] with
+ * the same stride.  Limits: (C+S) * 255 * 127 must fit int32.
+ * Device flags: BAD_INDEX, TIMEOUT. */
+size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S);
+ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C,
+                       int64_t lda, const int8_t* W_codes, const float* w_scale, int N, int S,
+                       int64_t ldw, const int32_t* idx_map, const float* bias, float* Y,
+                       int64_t ldy, int32_t* acc_out, void* ws, size_t ws_bytes,
+                       int* dev_status, void* stream);
+
+/* ocs_pack_conv_weights -------------------------------------------------------------------
+ * Reorders quantized conv weights from the split's layout [O][C+S][kh*kw] (row stride
+ * ld_src bytes) into the contraction order ocs_qconv consumes: for each output o, first the
+ * C original channels of every tap, k = tap*C + c, then the S duplicated channels of every
+ * tap, k = kh*kw*C + tap*S + s; row stride ld_dst bytes (multiple of 16), bytes between the
+ * last k and ld_dst set to zero.  A pure permutation of Eq. 3's terms. */
+ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, int S, int kh, int kw,
+                                 int64_t ld_src, int8_t* packed, int64_t ld_dst, void* stream);
+
+/* ocs_qconv -------------------------------------------------------------------------------
+ * Convolution form of ocs_qlinear (Section 3.2: a split duplicates a whole 2-D activation
+ * channel and all filters connected to it):
+ *   acc[(n,oh,ow)][o] = sum_{kh,kw} sum_{j<C+S} X[n][oh*s+kh-p][ow*s+kw-p][idx_map[j]] * W'[o][j][kh][kw]
+ * with zeros outside the image, and the same fp32 epilogue.  X codes NHWC [Nb][H][Wd][C]
+ * (dense, 16-byte aligned when C is a multiple of 16); W_packed from ocs_pack_conv_weights with row
+ * stride ldw bytes; Y fp32 NHWC [Nb][Ho][Wo][O] dense; acc_out (nullable) int32, same shape.
+ * Device flags: BAD_INDEX, TIMEOUT. */
+size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O, int S, int kh, int kw,
+                                 int stride, int pad);
+ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H,
+                     int Wd, int C, const int8_t* W_packed, const float* w_scale, int O, int S,
+                     int kh, int kw, int stride, int pad, int64_t ldw, const int32_t* idx_map,
+                     const float* bias, float* Y, int32_t* acc_out, void* ws, size_t ws_bytes,
+                     int* dev_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OCS_H */

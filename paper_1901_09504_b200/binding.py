@@ -1,0 +1,202 @@
+"""Thin Python binding of the C ABI in include/ocs.h.
+
+Argument marshalling only: every function takes torch CUDA tensors (used purely as device
+buffers), allocates the outputs and the scratch workspace through torch, passes raw device
+pointers and the current CUDA stream to the library and returns the output tensors.  All
+arithmetic runs in the library's kernels.  There is no fallback: if the shared library is
+missing or the device is not sm_100 the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libocs_b200.so")
+
+OCS_OK = 0
+STATUS_NAMES = {0: "OCS_OK", 1: "OCS_ERR_INVALID_ARG", 2: "OCS_ERR_SHAPE", 3: "OCS_ERR_WORKSPACE",
+                4: "OCS_ERR_UNSUPPORTED", 5: "OCS_ERR_CUDA"}
+DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT, DEV_DEPTH = 1, 2, 4, 8
+CLIP_NONE, CLIP_MSE = 0, 1
+
+EXPORTS = [
+    "ocs_num_splits", "ocs_poll_status", "ocs_version",
+    "ocs_split_workspace_bytes", "ocs_split",
+    "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views",
+    "ocs_qlinear_workspace_bytes", "ocs_qlinear",
+    "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
+]
+
+_lib = None
+
+
+class OcsError(RuntimeError):
+    def __init__(self, what: str, status: int):
+        super().__init__(f"{what}: {STATUS_NAMES.get(status, status)}")
+        self.status = status
+
+
+def lib():
+    """Loads the in-tree shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise OcsError(f"{LIB_PATH} not built (run python -m paper_1901_09504_b200.build)", 5)
+        L = C.CDLL(LIB_PATH)
+        L.ocs_num_splits.argtypes = [C.c_int, C.c_double]
+        L.ocs_version.restype = C.c_char_p
+        for name in ("ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
+                     "ocs_qconv_workspace_bytes"):
+            getattr(L, name).restype = C.c_size_t
+        L.ocs_quantize_workspace_views.restype = None
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ws(nbytes: int, device):
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def _check(status: int, what: str):
+    if status != OCS_OK:
+        raise OcsError(what, status)
+
+
+def new_status(device="cuda"):
+    """A zeroed device status word."""
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def ocs_num_splits(channels: int, ratio: float) -> int:
+    return int(lib().ocs_num_splits(int(channels), float(ratio)))
+
+
+def ocs_poll_status(dev_status) -> int:
+    out = C.c_int(0)
+    _check(lib().ocs_poll_status(_ptr(dev_status), _stream(), C.byref(out)), "ocs_poll_status")
+    return int(out.value)
+
+
+def round_up(x: int, m: int) -> int:
+    return (x + m - 1) // m * m
+
+
+def ocs_split(W, S: int, qa_step: float = 0.0, qa_bits: int = 0, ld_out: int | None = None, dev_status=None,
+              want_order: bool = True):
+    """W fp32 [O, C] or [O, C, kh, kw] (contiguous).  Returns (W_out [O, ld_out] fp32 whose first
+    (C+S)*R columns are W', idx_map int32 [C+S], split_order int32 [S], max_abs fp32 [3])."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+    O, Cn = W.shape[0], W.shape[1]
+    R = 1
+    for d in W.shape[2:]:
+        R *= d
+    cols_out = (Cn + S) * R
+    if ld_out is None:
+        ld_out = round_up(cols_out, 4)
+    W_out = torch.empty((O, ld_out), dtype=torch.float32, device=W.device)
+    idx_map = torch.empty(Cn + S, dtype=torch.int32, device=W.device)
+    order = torch.empty(max(S, 1), dtype=torch.int32, device=W.device) if want_order else None
+    max_abs = torch.zeros(3, dtype=torch.float32, device=W.device)
+    nws = lib().ocs_split_workspace_bytes(O, Cn, R, int(S))
+    ws = _ws(nws, W.device)
+    st = lib().ocs_split(_ptr(W), O, Cn, R, C.c_int64(Cn * R), int(S), C.c_float(qa_step), int(qa_bits),
+                         _ptr(W_out), C.c_int64(ld_out), _ptr(idx_map), _ptr(order), _ptr(max_abs), _ptr(ws),
+                         C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
+    _check(st, "ocs_split")
+    return W_out, idx_map, (order[:S] if want_order else None), max_abs
+
+
+def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_candidates: int = 128,
+                 n_bins: int = 2048, cols: int | None = None, ld_codes: int | None = None, max_abs_in=None,
+                 dev_status=None, return_search: bool = False):
+    """T fp32 2-D [rows, ld_in] (row stride = T.stride(0)); `cols` valid columns per row (default all).
+    Returns (codes int8/uint8 [rows, ld_codes], scale fp32 [1], alpha fp32 [1]) and, with
+    return_search, also (hist uint64 [n_bins] as int64, scores float64 [n_candidates])."""
+    assert T.is_cuda and T.dtype == torch.float32 and T.dim() == 2 and T.stride(1) == 1
+    rows, ld_in = T.shape[0], T.stride(0)
+    if cols is None:
+        cols = T.shape[1]
+    if ld_codes is None:
+        ld_codes = round_up(cols, 16)
+    codes = torch.zeros((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=T.device)
+    scale = torch.zeros(1, dtype=torch.float32, device=T.device)
+    alpha = torch.zeros(1, dtype=torch.float32, device=T.device)
+    nws = lib().ocs_quantize_workspace_bytes(int(n_bins), int(n_candidates))
+    ws = _ws(nws, T.device)
+    st = lib().ocs_quantize(_ptr(T), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_in), int(bits),
+                            int(bool(is_signed)), int(mode), int(n_candidates), int(n_bins), _ptr(max_abs_in),
+                            _ptr(codes), C.c_int64(ld_codes), _ptr(scale), _ptr(alpha), _ptr(ws),
+                            C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
+    _check(st, "ocs_quantize")
+    if not return_search:
+        return codes, scale, alpha
+    hp, sp = C.c_void_p(0), C.c_void_p(0)
+    lib().ocs_quantize_workspace_views(_ptr(ws), int(n_bins), int(n_candidates), C.byref(hp), C.byref(sp))
+    base = ws.data_ptr()
+    hist = ws[hp.value - base: hp.value - base + 8 * n_bins].view(torch.int64).clone()
+    scores = ws[sp.value - base: sp.value - base + 8 * n_candidates].view(torch.float64).clone()
+    return codes, scale, alpha, hist, scores
+
+
+def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, bias=None, want_acc: bool = False,
+                dev_status=None):
+    """A_codes uint8/int8 [M, lda>=C]; W_codes int8 [N, ldw>=C+S].  Returns Y fp32 [M, N] (and acc int32)."""
+    assert A_codes.is_cuda and A_codes.dim() == 2 and A_codes.stride(1) == 1
+    assert W_codes.dtype == torch.int8 and W_codes.dim() == 2 and W_codes.stride(1) == 1
+    M, N = A_codes.shape[0], W_codes.shape[0]
+    a_signed = 1 if A_codes.dtype == torch.int8 else 0
+    Y = torch.empty((M, N), dtype=torch.float32, device=A_codes.device)
+    acc = torch.empty((M, N), dtype=torch.int32, device=A_codes.device) if want_acc else None
+    nws = lib().ocs_qlinear_workspace_bytes(M, N, int(C_in), int(S))
+    ws = _ws(nws, A_codes.device)
+    st = lib().ocs_qlinear(_ptr(A_codes), a_signed, _ptr(a_scale), M, int(C_in), C.c_int64(A_codes.stride(0)),
+                           _ptr(W_codes), _ptr(w_scale), N, int(S), C.c_int64(W_codes.stride(0)), _ptr(idx_map),
+                           _ptr(bias), _ptr(Y), C.c_int64(N), _ptr(acc), _ptr(ws), C.c_size_t(ws.numel()),
+                           _ptr(dev_status), _stream())
+    _check(st, "ocs_qlinear")
+    return (Y, acc) if want_acc else Y
+
+
+def ocs_pack_conv_weights(codes, O: int, C_in: int, S: int, kh: int, kw: int, ld_dst: int | None = None):
+    """codes int8 [O, ld_src] in [C+S][kh*kw] order per row -> packed int8 [O, ld_dst]."""
+    assert codes.is_cuda and codes.dtype == torch.int8 and codes.dim() == 2 and codes.stride(1) == 1
+    Kt = kh * kw * (C_in + S)
+    if ld_dst is None:
+        ld_dst = round_up(Kt, 16)
+    packed = torch.empty((O, ld_dst), dtype=torch.int8, device=codes.device)
+    st = lib().ocs_pack_conv_weights(_ptr(codes), O, int(C_in), int(S), int(kh), int(kw),
+                                     C.c_int64(codes.stride(0)), _ptr(packed), C.c_int64(ld_dst), _stream())
+    _check(st, "ocs_pack_conv_weights")
+    return packed
+
+
+def ocs_qconv(X_codes, a_scale, W_packed, w_scale, idx_map, S: int, kh: int, kw: int, stride: int, pad: int,
+              bias=None, want_acc: bool = False, dev_status=None):
+    """X_codes uint8/int8 NHWC [Nb, H, W, C] contiguous; W_packed from ocs_pack_conv_weights.
+    Returns Y fp32 NHWC [Nb, Ho, Wo, O] (and acc int32)."""
+    assert X_codes.is_cuda and X_codes.dim() == 4 and X_codes.is_contiguous()
+    Nb, H, Wd, Cn = X_codes.shape
+    O = W_packed.shape[0]
+    Ho = (H + 2 * pad - kh) // stride + 1
+    Wo = (Wd + 2 * pad - kw) // stride + 1
+    a_signed = 1 if X_codes.dtype == torch.int8 else 0
+    Y = torch.empty((Nb, Ho, Wo, O), dtype=torch.float32, device=X_codes.device)
+    acc = torch.empty((Nb, Ho, Wo, O), dtype=torch.int32, device=X_codes.device) if want_acc else None
+    nws = lib().ocs_qconv_workspace_bytes(Nb, H, Wd, Cn, O, int(S), kh, kw, stride, pad)
+    ws = _ws(nws, X_codes.device)
+    st = lib().ocs_qconv(_ptr(X_codes), a_signed, _ptr(a_scale), Nb, H, Wd, Cn, _ptr(W_packed), _ptr(w_scale), O,
+                         int(S), kh, kw, stride, pad, C.c_int64(W_packed.stride(0)), _ptr(idx_map), _ptr(bias),
+                         _ptr(Y), _ptr(acc), _ptr(ws), C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
+    _check(st, "ocs_qconv")
+    return (Y, acc) if want_acc else Y

@@ -1,0 +1,789 @@
+// ocs_qlinear / ocs_qconv: the split layer of Eq. 3 on integer codes, as one tcgen05 int8 GEMM /
+// implicit-GEMM convolution (Section 3.2, Section 3.5).
+//
+//   acc[m][n] = sum_k Aexp[m][k] * Wc[n][k]      int8/uint8 x int8 -> int32 in tensor memory
+//   Y[m][n]   = fmaf((float)acc, a_scale*w_scale, bias[n])
+//
+// The expanded activation operand Aexp (activations with the duplicated channels appended) is never
+// written to global memory: K-blocks that hold only original channels are fetched by TMA straight
+// from the unexpanded tensor, and K-blocks that hold duplicated channels (or that the TMA alignment
+// rules cannot serve) are assembled in shared memory by four producer warps that read the source
+// channels through idx_map and store them in the 128-byte-swizzled layout the tensor core reads.
+//
+// One CTA = one 128 x BN output tile (x one K slice when split-K is on).  Warp roles:
+//   warp 0      TMA producer (weights always, activations when the block is TMA-able)
+//   warp 1      allocates tensor memory, issues tcgen05.mma, commits to the stage barriers
+//   warps 2..5  gather producers during the main loop, then the epilogue (tcgen05.ld -> global)
+// Every mbarrier wait is bounded by a clock limit; on expiry the CTA sets OCS_DEV_TIMEOUT, lets its
+// outstanding copies land, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace ocs {
+namespace {
+
+constexpr int BM = 128;        // UMMA M
+constexpr int BK = 128;        // bytes (= int8 elements) per K-block: one 128-byte swizzle span
+constexpr int UMMA_K = 32;     // K of one tcgen05.mma.kind::i8
+constexpr int kGemmThreads = 192;
+constexpr int kGatherThreads = 128;
+constexpr long long kWaitCycles = 2000000000ll;  // about one second
+
+enum { MODE_LINEAR = 0, MODE_CONV = 1 };
+
+struct GemmParams {
+  int mode;
+  int M, N, Ktot;   // Ktot = number of valid contraction indices
+  int C, S, R;
+  const uint8_t* A;  // linear: [M][lda] ; conv: NHWC codes
+  long long lda;
+  int a_signed;
+  const int32_t* idx_map;
+  int a_vec16;       // 16-byte loads of A allowed (alignment)
+  // convolution geometry
+  int Nb, H, Wd, Ho, Wo, kh, kw, stride, pad;
+  int bw, bh, bn;               // output-pixel box of one M tile: bw*bh*bn <= 128
+  int tiles_w, tiles_h, tiles_n;
+  // k-blocks
+  int num_kb;
+  int kb_tma_a;      // K-blocks [0, kb_tma_a) get their A tile by TMA
+  int split_k;
+  // epilogue
+  const float* a_scale;
+  const float* w_scale;
+  const float* bias;
+  float* Y;
+  long long ldy;
+  int32_t* acc_out;
+  int32_t* acc_ws;              // [split_k][rows][N] partial sums when split_k > 1
+  long long out_rows;           // rows of Y
+  unsigned int* tile_counters;  // one per output tile when split_k > 1
+  int a_box_bytes;              // bytes one TMA load of A delivers
+  int* dev_status;
+};
+
+// ------------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the CTA is aborting (this wait or another one ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread t of the warp receives lane (base + t)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t v[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of
+// 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFFu);        // start address
+  d |= (uint64_t)1 << 16;                         // leading byte offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset: next 8-row group
+  d |= (uint64_t)1 << 46;                         // descriptor version
+  d |= (uint64_t)2 << 61;                         // SWIZZLE_128B
+  return d;
+}
+__host__ __device__ constexpr uint32_t instr_desc_i8(int n, int a_signed) {
+  return (2u << 4)                         // accumulator S32
+         | ((uint32_t)(a_signed ? 1 : 0) << 7)   // A: uint8 / int8
+         | (1u << 10)                      // B: int8
+         | ((uint32_t)(n >> 3) << 17)      // N
+         | ((uint32_t)(BM >> 4) << 24);    // M
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row r of M tile `mt` -> what it reads and where it writes.
+struct RowInfo {
+  long long out_row;   // linear: m ; conv: output pixel index (n*Ho+oh)*Wo+ow ; -1 = padding row
+  int n, ih0, iw0;     // conv: image and top-left input coordinate of the receptive field
+};
+
+__device__ __forceinline__ RowInfo row_info(const GemmParams& p, int mt, int r) {
+  RowInfo ri;
+  ri.n = 0; ri.ih0 = 0; ri.iw0 = 0;
+  if (p.mode == MODE_LINEAR) {
+    const long long m = (long long)mt * BM + r;
+    ri.out_row = m < p.M ? m : -1;
+    return ri;
+  }
+  const int tw = mt % p.tiles_w;
+  const int th = (mt / p.tiles_w) % p.tiles_h;
+  const int tn = mt / (p.tiles_w * p.tiles_h);
+  const int wl = r % p.bw;
+  const int hl = (r / p.bw) % p.bh;
+  const int nl = r / (p.bw * p.bh);
+  const int ow = tw * p.bw + wl, oh = th * p.bh + hl, n = tn * p.bn + nl;
+  if (nl >= p.bn || ow >= p.Wo || oh >= p.Ho || n >= p.Nb) { ri.out_row = -1; return ri; }
+  ri.out_row = ((long long)n * p.Ho + oh) * p.Wo + ow;
+  ri.n = n; ri.ih0 = oh * p.stride - p.pad; ri.iw0 = ow * p.stride - p.pad;
+  return ri;
+}
+
+__device__ __forceinline__ uint32_t checked_src(const GemmParams& p, int j, bool* bad) {
+  int c = __ldg(p.idx_map + j);
+  if ((unsigned)c >= (unsigned)p.C) { *bad = true; c = 0; }
+  return (uint32_t)c;
+}
+
+// The 16 operand bytes of row `ri` for contraction indices [k0, k0 + 16).
+__device__ __forceinline__ uint4 gather_chunk(const GemmParams& p, const RowInfo& ri, int k0, bool* bad) {
+  uint4 out = make_uint4(0u, 0u, 0u, 0u);
+  if (ri.out_row < 0 || k0 >= p.Ktot) return out;
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  if (p.mode == MODE_LINEAR) {
+    const uint8_t* row = p.A + ri.out_row * p.lda;
+    if (p.a_vec16 && k0 + 16 <= p.C) return __ldg(reinterpret_cast<const uint4*>(row + k0));
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int k = k0 + i;
+      if (k < p.Ktot) {
+        const uint32_t c = k < p.C ? (uint32_t)k : checked_src(p, k, bad);
+        w[i >> 2] |= (uint32_t)__ldg(row + c) << (8 * (i & 3));
+      }
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  // convolution: contraction order is [tap][c < C] then [tap][s < S]
+  const int KO = p.R * p.C;
+  const uint8_t* img = p.A + (long long)ri.n * p.H * p.Wd * p.C;
+  if (k0 + 16 <= KO && p.a_vec16) {  // C % 16 == 0: the chunk lies inside one tap
+    const int tap = k0 / p.C, c0 = k0 - tap * p.C;
+    const int ih = ri.ih0 + tap / p.kw, iw = ri.iw0 + tap % p.kw;
+    if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd)
+      return __ldg(reinterpret_cast<const uint4*>(img + ((long long)ih * p.Wd + iw) * p.C + c0));
+    return out;
+  }
+  int k = k0;
+  int tap, sub, width;  // position inside the current region: sub in [0, width)
+  if (k < KO) { tap = k / p.C; sub = k - tap * p.C; width = p.C; }
+  else { const int kd = k - KO; tap = kd / p.S; sub = kd - tap * p.S; width = p.S; }
+#pragma unroll
+  for (int i = 0; i < 16; ++i, ++k) {
+    if (k >= p.Ktot) break;
+    if (k == KO) { tap = 0; sub = 0; width = p.S; }
+    const int ih = ri.ih0 + tap / p.kw, iw = ri.iw0 + tap % p.kw;
+    if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd) {
+      const uint32_t c = k < KO ? (uint32_t)sub : checked_src(p, p.C + sub, bad);
+      w[i >> 2] |= (uint32_t)__ldg(img + ((long long)ih * p.Wd + iw) * p.C + c) << (8 * (i & 3));
+    }
+    if (++sub == width) { sub = 0; ++tap; }
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <int BN>
+struct SmemLayout {
+  static constexpr int kABytes = BM * BK;
+  static constexpr int kBBytes = BN * BK;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int kTileBytes = kStages * kStageBytes;
+  static constexpr int kCtrlBytes = 1024;               // barriers, tensor-memory slot, flags
+  static constexpr int kRowTableBytes = BM * 24;        // RowInfo per tile row
+  static constexpr int kDynBytes = kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmA, const GemmParams p) {
+  using L = SmemLayout<BN>;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t raw = smem_u32(smem_dyn);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* tiles = smem_dyn + (base - raw);
+  unsigned char* ctrl = tiles + L::kTileBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);           // full[kStages], empty[kStages], accum
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * L::kStages + 1));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * L::kStages + 1) + 8);
+  int* last_flag = const_cast<int*>(abort_flag) + 1;
+  RowInfo* rows = reinterpret_cast<RowInfo*>(ctrl + L::kCtrlBytes);
+  auto full_bar = [&](int s) { return smem_u32(bars + s); };
+  auto empty_bar = [&](int s) { return smem_u32(bars + L::kStages + s); };
+  const uint32_t accum_bar = smem_u32(bars + 2 * L::kStages);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int mt = blockIdx.x, nt = blockIdx.y, kz = blockIdx.z;
+  // this CTA's K-blocks: kz, kz + split_k, ...
+  const int my_kb = (p.num_kb - kz + p.split_k - 1) / p.split_k;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < L::kStages; ++s) {
+      mbar_init(full_bar(s), 1 + kGatherThreads / 32);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(accum_bar, 1);
+    *abort_flag = 0;
+    *last_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmB);
+    if (p.kb_tma_a > 0) prefetch_tmap(&tmA);
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), BN);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int issued = 0;
+      for (int i = 0; i < my_kb; ++i) {
+        const int kb = kz + i * p.split_k;
+        const int s = i % L::kStages;
+        const uint32_t par = ((i / L::kStages) & 1) ^ 1;
+        if (!mbar_wait(empty_bar(s), par, abort_flag)) break;
+        const uint32_t a_dst = base + s * L::kStageBytes;
+        const uint32_t b_dst = a_dst + L::kABytes;
+        const bool a_tma = kb < p.kb_tma_a;
+        mbar_arrive_expect_tx(full_bar(s), L::kBBytes + (a_tma ? p.a_box_bytes : 0));
+        tma_load_2d(b_dst, &tmB, full_bar(s), kb * BK, nt * BN);
+        if (a_tma) {
+          if (p.mode == MODE_LINEAR) {
+            tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, mt * BM);
+          } else {
+            const int k0 = kb * BK;
+            const int tap = k0 / p.C, c0 = k0 - tap * p.C;
+            const int tw = mt % p.tiles_w, th = (mt / p.tiles_w) % p.tiles_h, tn = mt / (p.tiles_w * p.tiles_h);
+            tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw + tap % p.kw - p.pad, th * p.bh + tap / p.kw - p.pad,
+                        tn * p.bn);
+          }
+        }
+        ++issued;
+      }
+      if (*abort_flag && issued > 0) {
+        // give copies that are still in flight time to land before the CTA's shared memory is released
+        for (int i = 0; i < 2000; ++i) __nanosleep(100);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_i8(BN, p.a_signed);
+      bool ok = true;
+      for (int i = 0; i < my_kb && ok; ++i) {
+        const int s = i % L::kStages;
+        const uint32_t par = (i / L::kStages) & 1;
+        if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t a_addr = base + s * L::kStageBytes;
+        const uint32_t b_addr = a_addr + L::kABytes;
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k) {
+          umma_i8(tmem_base, smem_desc_sw128(a_addr + k * UMMA_K), smem_desc_sw128(b_addr + k * UMMA_K), idesc,
+                  (i > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
+      }
+      if (ok) umma_commit(accum_bar);
+    }
+  } else {
+    // ---------------------------------------------------------------- gather producers, then epilogue
+    const int gt = threadIdx.x - 64;   // 0..127
+    rows[gt] = row_info(p, mt, gt);
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    const int chunk = gt & 7;          // 16-byte chunk of the 128-byte row
+    const int rbase = gt >> 3;         // rows rbase + 16*i
+    bool bad = false;
+    bool ok = true;
+    for (int i = 0; i < my_kb; ++i) {
+      const int kb = kz + i * p.split_k;
+      const int s = i % L::kStages;
+      const uint32_t par = ((i / L::kStages) & 1) ^ 1;
+      if (!mbar_wait(empty_bar(s), par, abort_flag)) { ok = false; break; }
+      if (kb >= p.kb_tma_a) {
+        unsigned char* a_tile = tiles + s * L::kStageBytes;
+        uint4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = gather_chunk(p, rows[rbase + 16 * j], kb * BK + chunk * 16, &bad);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int r = rbase + 16 * j;
+          *reinterpret_cast<uint4*>(a_tile + r * 128 + ((chunk ^ (r & 7)) << 4)) = v[j];
+        }
+        fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_bar(s));
+    }
+    if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
+
+    // epilogue: warp w may read tensor-memory lanes 32*(w%4) .. +31
+    if (ok) ok = mbar_wait(accum_bar, 0, abort_flag);
+    const int q = warp & 3;
+    const float sc = __fmul_rn(__ldg(p.a_scale), __ldg(p.w_scale));
+    const bool direct = p.split_k == 1;
+    if (ok) {
+      tc_fence_after();
+      const RowInfo ri = rows[q * 32 + lane];
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        const int n0 = nt * BN + c0;
+        if (n0 >= p.N) break;  // warp-uniform
+        uint32_t v[32];
+        __syncwarp();
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        if (ri.out_row >= 0) {
+          if (direct) {
+            float* y = p.Y + ri.out_row * p.ldy + n0;
+            int32_t* ao = p.acc_out ? p.acc_out + ri.out_row * p.ldy + n0 : nullptr;
+            const bool vec = (n0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(y) & 15) == 0);
+            if (vec) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                float4 o;
+                o.x = fmaf((float)(int)v[j + 0], sc, p.bias ? __ldg(p.bias + n0 + j + 0) : 0.0f);
+                o.y = fmaf((float)(int)v[j + 1], sc, p.bias ? __ldg(p.bias + n0 + j + 1) : 0.0f);
+                o.z = fmaf((float)(int)v[j + 2], sc, p.bias ? __ldg(p.bias + n0 + j + 2) : 0.0f);
+                o.w = fmaf((float)(int)v[j + 3], sc, p.bias ? __ldg(p.bias + n0 + j + 3) : 0.0f);
+                *reinterpret_cast<float4*>(y + j) = o;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (n0 + j < p.N) y[j] = fmaf((float)(int)v[j], sc, p.bias ? __ldg(p.bias + n0 + j) : 0.0f);
+            }
+            if (ao) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (n0 + j < p.N) ao[j] = (int)v[j];
+            }
+          } else {
+            // this slice's partial sums, [kz][row][n]
+            int32_t* part = p.acc_ws + ((long long)kz * p.out_rows + ri.out_row) * p.N + n0;
+            if ((n0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(part) & 15) == 0)) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                __stcg(reinterpret_cast<int4*>(part + j), make_int4((int)v[j], (int)v[j + 1], (int)v[j + 2], (int)v[j + 3]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (n0 + j < p.N) __stcg(part + j, (int)v[j]);
+            }
+          }
+        }
+      }
+    }
+    if (!direct) {
+      // the last K slice to finish a tile sums all slices' partials (integer sums: exact in any order)
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (gt == 0) {
+        int last = 0;
+        if (!*abort_flag) {
+          const unsigned int tile = blockIdx.y * gridDim.x + blockIdx.x;
+          last = (atomicAdd(p.tile_counters + tile, 1u) == (unsigned int)p.split_k - 1u) ? 1 : 0;
+        }
+        *last_flag = last;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (*last_flag) {
+        __threadfence();
+        const int ncols = min(BN, p.N - nt * BN);
+        for (int rr = 0; rr < 32; ++rr) {
+          const long long orow = rows[q * 32 + rr].out_row;
+          if (orow < 0) continue;  // warp-uniform
+          for (int c = lane; c < ncols; c += 32) {
+            const int n = nt * BN + c;
+            int a = 0;
+            for (int z = 0; z < p.split_k; ++z) a += __ldcg(p.acc_ws + ((long long)z * p.out_rows + orow) * p.N + n);
+            p.Y[orow * p.ldy + n] = fmaf((float)a, sc, p.bias ? __ldg(p.bias + n) : 0.0f);
+            if (p.acc_out) p.acc_out[orow * p.ldy + n] = a;
+          }
+        }
+      }
+    }
+    tc_fence_before();
+  }
+
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, BN);
+  }
+  if (threadIdx.x == 0 && *abort_flag) flag(p.dev_status, OCS_DEV_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+bool encode_u8(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+               const cuuint32_t* box) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct GemmPlan {
+  int BN;
+  int split_k;
+  int m_tiles, n_tiles;
+};
+
+GemmPlan choose_plan(int m_tiles, int N, int num_kb) {
+  GemmPlan best{64, 1, m_tiles, (N + 63) / 64};
+  double best_score = -1.0;
+  const int bns[3] = {256, 128, 64};
+  for (int bi = 0; bi < 3; ++bi) {
+    const int BN = bns[bi];
+    if (BN > 64 && N <= BN / 2) continue;  // tile mostly empty
+    const long long tiles = (long long)m_tiles * ((N + BN - 1) / BN);
+    int max_split = num_kb / 4;            // keep at least 4 K-blocks per slice
+    if (max_split < 1) max_split = 1;
+    if (max_split > 32) max_split = 32;
+    for (int sk = 1; sk <= max_split; ++sk) {
+      const long long ctas = tiles * sk;
+      const long long waves = (ctas + kNumSMs - 1) / kNumSMs;
+      const double eff = (double)ctas / (double)(waves * kNumSMs);
+      // prefer full waves, then wide tiles, then little splitting
+      const double score = eff + 0.02 * (2 - bi) - 0.004 * (sk - 1) - (sk > 1 && tiles >= kNumSMs ? 1.0 : 0.0);
+      if (score > best_score) {
+        best_score = score;
+        best = GemmPlan{BN, sk, m_tiles, (N + BN - 1) / BN};
+      }
+    }
+  }
+  return best;
+}
+
+template <int BN>
+ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const GemmParams& p, const GemmPlan& plan,
+                       cudaStream_t stream) {
+  using L = SmemLayout<BN>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(ocs_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynBytes) != cudaSuccess)
+      return OCS_ERR_CUDA;
+    attr_set = true;
+  }
+  dim3 grid(plan.m_tiles, plan.n_tiles, plan.split_k);
+  ocs_gemm_kernel<BN><<<grid, kGemmThreads, L::kDynBytes, stream>>>(tmB, tmA, p);
+  return launch_status();
+}
+
+struct GemmWs {
+  int32_t* acc_ws;
+  unsigned int* counters;
+  size_t total;
+};
+
+GemmWs carve_gemm_ws(void* ws, long long rows, int N, long long m_tiles, int split_k) {
+  GemmWs w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    unsigned char* q = ws ? reinterpret_cast<unsigned char*>(ws) + off : nullptr;
+    off += align_up(bytes, 256);
+    return q;
+  };
+  w.acc_ws = reinterpret_cast<int32_t*>(take(4 * (size_t)split_k * (size_t)rows * (size_t)N));
+  w.counters = reinterpret_cast<unsigned int*>(take(4 * (size_t)m_tiles * (size_t)((N + 63) / 64)));
+  w.total = off;
+  return w;
+}
+
+ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long long out_rows, int m_tiles, bool tma_a_ok,
+                    const CUtensorMap* tmA_in, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  p.num_kb = (p.Ktot + BK - 1) / BK;
+  const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb);
+  p.split_k = plan.split_k;
+  if (!tma_a_ok) p.kb_tma_a = 0;
+
+  CUtensorMap tmB;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)p.Ktot, (cuuint64_t)p.N};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldw};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)plan.BN};
+    if (!encode_u8(&tmB, W_codes, 2, dims, strides, box)) return OCS_ERR_CUDA;
+  }
+  CUtensorMap tmA = tmB;  // a valid map even when unused
+  if (p.kb_tma_a > 0) tmA = *tmA_in;
+
+  p.out_rows = out_rows;
+  if (plan.split_k > 1) {
+    const GemmWs w = carve_gemm_ws(ws, out_rows, p.N, m_tiles, plan.split_k);
+    if (!ws || !aligned(ws, 256) || ws_bytes < w.total) return OCS_ERR_WORKSPACE;
+    p.acc_ws = w.acc_ws;
+    p.tile_counters = w.counters;
+    if (cudaMemsetAsync(w.counters, 0, 4 * (size_t)m_tiles * (size_t)((p.N + 63) / 64), stream) != cudaSuccess)
+      return OCS_ERR_CUDA;
+  }
+  switch (plan.BN) {
+    case 256: return launch_gemm<256>(tmB, tmA, p, plan, stream);
+    case 128: return launch_gemm<128>(tmB, tmA, p, plan, stream);
+    default: return launch_gemm<64>(tmB, tmA, p, plan, stream);
+  }
+}
+
+// M-tile box for the convolution: the (bw, bh, bn) with bw*bh*bn <= 128 that needs the fewest tiles.
+void choose_conv_box(int Wo, int Ho, int Nb, int* bw_o, int* bh_o, int* bn_o) {
+  long long best_tiles = -1;
+  int bbw = 1, bbh = 1, bbn = 1;
+  for (int bw = 1; bw <= Wo && bw <= BM; ++bw) {
+    for (int bh = 1; bh <= Ho && bw * bh <= BM; ++bh) {
+      int bn = BM / (bw * bh);
+      if (bn > Nb) bn = Nb;
+      if (bn > 256) bn = 256;
+      const long long tiles = (long long)((Wo + bw - 1) / bw) * ((Ho + bh - 1) / bh) * ((Nb + bn - 1) / bn);
+      if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && bw > bbw)) {
+        best_tiles = tiles; bbw = bw; bbh = bh; bbn = bn;
+      }
+    }
+  }
+  *bw_o = bbw; *bh_o = bbh; *bn_o = bbn;
+}
+
+__global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, int S, int R, long long ld_src,
+                                 int8_t* __restrict__ dst, long long ld_dst) {
+  const long long total = (long long)O * ld_dst;
+  const int KO = R * C, Kt = R * (C + S);
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long o = i / ld_dst;
+    const int k = (int)(i - o * ld_dst);
+    int8_t v = 0;
+    if (k < Kt) {
+      int tap, j;
+      if (k < KO) { tap = k / C; j = k - tap * C; }
+      else { const int kd = k - KO; tap = kd / S; j = C + (kd - tap * S); }
+      v = src[o * ld_src + (long long)j * R + tap];
+    }
+    dst[i] = v;
+  }
+}
+
+}  // namespace
+}  // namespace ocs
+
+using namespace ocs;
+
+extern "C" size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S) {
+  if (M <= 0 || N <= 0 || C <= 0 || S < 0) return 256;
+  const int m_tiles = (M + BM - 1) / BM;
+  const GemmPlan plan = choose_plan(m_tiles, N, (int)(((long long)C + S + BK - 1) / BK));
+  if (plan.split_k == 1) return 256;
+  return carve_gemm_ws(nullptr, M, N, m_tiles, plan.split_k).total;
+}
+
+extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C, int64_t lda,
+                                  const int8_t* W_codes, const float* w_scale, int N, int S, int64_t ldw,
+                                  const int32_t* idx_map, const float* bias, float* Y, int64_t ldy, int32_t* acc_out,
+                                  void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!A_codes || !a_scale || !W_codes || !w_scale || !idx_map || !Y) return OCS_ERR_INVALID_ARG;
+  if (S < 0) return OCS_ERR_INVALID_ARG;
+  if (M <= 0 || C <= 0 || N <= 0) return OCS_ERR_SHAPE;
+  const long long Ktot = (long long)C + S;
+  if (lda < C || ldw < Ktot || ldy < N) return OCS_ERR_SHAPE;
+  if (ldw % 16 != 0 || !aligned(W_codes, 16) || !aligned(Y, 4)) return OCS_ERR_SHAPE;
+  if (Ktot * 255ll * 127ll > 2147483647ll) return OCS_ERR_UNSUPPORTED;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+
+  GemmParams p{};
+  p.mode = MODE_LINEAR;
+  p.M = M; p.N = N; p.Ktot = (int)Ktot; p.C = C; p.S = S; p.R = 1;
+  p.A = reinterpret_cast<const uint8_t*>(A_codes); p.lda = lda; p.a_signed = a_signed ? 1 : 0;
+  p.idx_map = idx_map;
+  p.a_vec16 = (lda % 16 == 0) && aligned(A_codes, 16);
+  p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = ldy; p.acc_out = acc_out;
+  p.dev_status = dev_status;
+  const int m_tiles = (M + BM - 1) / BM;
+  p.kb_tma_a = C / BK;  // K-blocks made of original channels only
+  p.a_box_bytes = BM * BK;
+  CUtensorMap tmA;
+  bool tma_ok = p.a_vec16 && p.kb_tma_a > 0;
+  if (tma_ok) {
+    const cuuint64_t dims[2] = {(cuuint64_t)C, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)lda};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    if (!encode_u8(&tmA, A_codes, 2, dims, strides, box)) return OCS_ERR_CUDA;
+  }
+  return run_gemm(p, W_codes, ldw, M, m_tiles, tma_ok, &tmA, ws, ws_bytes, stream);
+}
+
+extern "C" ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, int S, int kh, int kw, int64_t ld_src,
+                                            int8_t* packed, int64_t ld_dst, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!codes || !packed || S < 0) return OCS_ERR_INVALID_ARG;
+  if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0) return OCS_ERR_SHAPE;
+  const long long Kt = (long long)kh * kw * ((long long)C + S);
+  if (ld_src < Kt || ld_dst < Kt || ld_dst % 16 != 0 || Kt >= (1ll << 31)) return OCS_ERR_SHAPE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  const long long total = (long long)O * ld_dst;
+  const int grid = (int)((total + 255) / 256 < kNumSMs * 8 ? (total + 255) / 256 : kNumSMs * 8);
+  pack_conv_kernel<<<grid, 256, 0, stream>>>(codes, O, C, S, kh * kw, ld_src, packed, ld_dst);
+  return launch_status();
+}
+
+namespace {
+struct ConvGeom {
+  int Ho, Wo, bw, bh, bn, tiles_w, tiles_h, tiles_n;
+  long long m_tiles, out_rows;
+};
+bool conv_geom(int Nb, int H, int Wd, int kh, int kw, int stride, int pad, ConvGeom* g) {
+  g->Ho = (H + 2 * pad - kh) / stride + 1;
+  g->Wo = (Wd + 2 * pad - kw) / stride + 1;
+  if (g->Ho <= 0 || g->Wo <= 0) return false;
+  choose_conv_box(g->Wo, g->Ho, Nb, &g->bw, &g->bh, &g->bn);
+  g->tiles_w = (g->Wo + g->bw - 1) / g->bw;
+  g->tiles_h = (g->Ho + g->bh - 1) / g->bh;
+  g->tiles_n = (Nb + g->bn - 1) / g->bn;
+  g->m_tiles = (long long)g->tiles_w * g->tiles_h * g->tiles_n;
+  g->out_rows = (long long)Nb * g->Ho * g->Wo;
+  return true;
+}
+}  // namespace
+
+extern "C" size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O, int S, int kh, int kw, int stride,
+                                            int pad) {
+  ConvGeom g;
+  if (Nb <= 0 || H <= 0 || Wd <= 0 || C <= 0 || S < 0 || O <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0 ||
+      !conv_geom(Nb, H, Wd, kh, kw, stride, pad, &g))
+    return 256;
+  const long long Ktot = (long long)kh * kw * ((long long)C + S);
+  const GemmPlan plan = choose_plan((int)g.m_tiles, O, (int)((Ktot + BK - 1) / BK));
+  if (plan.split_k == 1) return 256;
+  return carve_gemm_ws(nullptr, g.out_rows, O, g.m_tiles, plan.split_k).total;
+}
+
+extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H, int Wd, int C,
+                                const int8_t* W_packed, const float* w_scale, int O, int S, int kh, int kw, int stride,
+                                int pad, int64_t ldw, const int32_t* idx_map, const float* bias, float* Y,
+                                int32_t* acc_out, void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!X_codes || !a_scale || !W_packed || !w_scale || !idx_map || !Y) return OCS_ERR_INVALID_ARG;
+  if (S < 0) return OCS_ERR_INVALID_ARG;
+  if (Nb <= 0 || H <= 0 || Wd <= 0 || C <= 0 || O <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
+    return OCS_ERR_SHAPE;
+  const long long Ktot = (long long)kh * kw * ((long long)C + S);
+  if (ldw < Ktot || ldw % 16 != 0 || !aligned(W_packed, 16) || !aligned(Y, 4)) return OCS_ERR_SHAPE;
+  if (Ktot * 255ll * 127ll > 2147483647ll) return OCS_ERR_UNSUPPORTED;
+  ConvGeom g;
+  if (!conv_geom(Nb, H, Wd, kh, kw, stride, pad, &g)) return OCS_ERR_SHAPE;
+  if (g.m_tiles >= (1ll << 31) || g.out_rows * (long long)O >= (1ll << 40)) return OCS_ERR_UNSUPPORTED;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+
+  GemmParams p{};
+  p.mode = MODE_CONV;
+  p.M = (int)(g.out_rows < (1ll << 31) ? g.out_rows : 0x7fffffff);
+  p.N = O; p.Ktot = (int)Ktot; p.C = C; p.S = S; p.R = kh * kw;
+  p.A = reinterpret_cast<const uint8_t*>(X_codes); p.lda = C; p.a_signed = a_signed ? 1 : 0;
+  p.idx_map = idx_map;
+  p.a_vec16 = (C % 16 == 0) && aligned(X_codes, 16);
+  p.Nb = Nb; p.H = H; p.Wd = Wd; p.Ho = g.Ho; p.Wo = g.Wo; p.kh = kh; p.kw = kw; p.stride = stride; p.pad = pad;
+  p.bw = g.bw; p.bh = g.bh; p.bn = g.bn; p.tiles_w = g.tiles_w; p.tiles_h = g.tiles_h; p.tiles_n = g.tiles_n;
+  p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = O; p.acc_out = acc_out;
+  p.dev_status = dev_status;
+
+  // TMA serves the K-blocks that lie inside one tap's original channels: stride 1 and C % 128 == 0
+  CUtensorMap tmA;
+  bool tma_ok = (stride == 1) && (C % BK == 0) && aligned(X_codes, 16);
+  p.kb_tma_a = tma_ok ? (kh * kw * C) / BK : 0;
+  p.a_box_bytes = g.bw * g.bh * g.bn * BK;
+  if (tma_ok) {
+    const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)Wd, (cuuint64_t)H, (cuuint64_t)Nb};
+    const cuuint64_t strides[3] = {(cuuint64_t)C, (cuuint64_t)C * Wd, (cuuint64_t)C * Wd * H};
+    const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)g.bw, (cuuint32_t)g.bh, (cuuint32_t)g.bn};
+    if (!encode_u8(&tmA, X_codes, 4, dims, strides, box)) return OCS_ERR_CUDA;
+  }
+  return run_gemm(p, W_packed, ldw, g.out_rows, (int)g.m_tiles, tma_ok, &tmA, ws, ws_bytes, stream);
+}

@@ -1,0 +1,311 @@
+// ocs_quantize: k-bit linear quantization (Eq. 1) with an optional MSE clip-threshold search
+// (Section 4.1).
+//
+// Kernels (each a streaming pass over T in tiles of one row segment of 4096 columns):
+//   maxabs_kernel     max|x|, combined with atomicMax on the bits of the non-negative value
+//   hist_kernel       histogram of |x| in privatised shared-memory counters, flushed with 64-bit atomics
+//   score_kernel      one CTA per candidate threshold: sum_b h[b]*(x_b - Q(x_b))^2 in double
+//   pick_kernel       smallest score, ties to the largest threshold
+//   quantize_kernel   code = clamp(rint(x * L/alpha)), round-half-to-even, saturating
+#include "common.cuh"
+
+namespace ocs {
+namespace {
+
+constexpr int kTileQuads = 4;                     // float4 per thread per tile
+constexpr int kTileCols = 256 * 4 * kTileQuads;   // 4096 columns per tile
+constexpr int kMaxBins = 4096;
+constexpr int kMaxCandidates = 1024;
+constexpr int kHistCopies = 2;
+
+struct View {
+  const float* T;
+  long long rows, cols, ld;
+  long long tiles_per_row, tiles;
+  bool vec;  // 128-bit loads allowed
+};
+
+View make_view(const float* T, int64_t rows, int64_t cols, int64_t ld) {
+  View v;
+  v.T = T;
+  if (ld == cols) {  // dense: one long row
+    v.rows = 1; v.cols = rows * cols; v.ld = rows * cols;
+    v.vec = aligned(T, 16);
+  } else {
+    v.rows = rows; v.cols = cols; v.ld = ld;
+    v.vec = aligned(T, 16) && (ld % 4 == 0);
+  }
+  v.tiles_per_row = (v.cols + kTileCols - 1) / kTileCols;
+  v.tiles = v.rows * v.tiles_per_row;
+  return v;
+}
+
+int grid_for(long long tiles) {
+  const long long cap = (long long)kNumSMs * 8;
+  return (int)(tiles < cap ? (tiles > 0 ? tiles : 1) : cap);
+}
+
+// Loads the thread's u-th quad of tile t; n = number of valid elements (0..4); col = first column.
+__device__ __forceinline__ int load_quad(const View& v, long long t, int u, float x[4], long long* row_out,
+                                         long long* col_out) {
+  const long long row = t / v.tiles_per_row;
+  const long long seg = t - row * v.tiles_per_row;
+  const long long col = seg * kTileCols + (long long)(u * 256 + threadIdx.x) * 4;
+  *row_out = row;
+  *col_out = col;
+  if (col >= v.cols) return 0;
+  const float* p = v.T + row * v.ld + col;
+  if (v.vec && col + 3 < v.cols) {
+    const float4 q = __ldcs(reinterpret_cast<const float4*>(p));
+    x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
+    return 4;
+  }
+  const int n = (int)min(4ll, v.cols - col);
+  for (int i = 0; i < 4; ++i) x[i] = i < n ? __ldcs(p + i) : 0.0f;
+  return n;
+}
+
+__global__ void __launch_bounds__(256) maxabs_kernel(View v, unsigned int* maxbits) {
+  float m = 0.0f;
+  for (long long t = blockIdx.x; t < v.tiles; t += gridDim.x) {
+#pragma unroll
+    for (int u = 0; u < kTileQuads; ++u) {
+      float x[4];
+      long long row, col;
+      const int n = load_quad(v, t, u, x, &row, &col);
+      if (n) m = fmaxf(m, fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3]))));
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  __shared__ float red[8];
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) m = fmaxf(m, red[w]);
+    atomicMax(maxbits, __float_as_uint(m));  // m >= 0: bit order is value order
+  }
+}
+
+__global__ void __launch_bounds__(256)
+hist_kernel(View v, const float* __restrict__ maxp, int n_bins, unsigned long long* __restrict__ hist) {
+  extern __shared__ unsigned int sh[];  // kHistCopies * n_bins
+  for (int i = threadIdx.x; i < kHistCopies * n_bins; i += 256) sh[i] = 0u;
+  __syncthreads();
+  const float m = *maxp;
+  if (m > 0.0f) {
+    const float invw = __fdiv_rn((float)n_bins, m);
+    unsigned int* mine = sh + ((threadIdx.x >> 5) % kHistCopies) * n_bins;
+    const int last = n_bins - 1;
+    for (long long t = blockIdx.x; t < v.tiles; t += gridDim.x) {
+      float x[kTileQuads][4];
+      int n[kTileQuads];
+#pragma unroll
+      for (int u = 0; u < kTileQuads; ++u) {
+        long long row, col;
+        n[u] = load_quad(v, t, u, x[u], &row, &col);
+      }
+#pragma unroll
+      for (int u = 0; u < kTileQuads; ++u) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (i < n[u]) {
+            const int b = min(last, (int)__fmul_rn(fabsf(x[u][i]), invw));  // truncation
+            atomicAdd(&mine[b], 1u);
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < n_bins; b += 256) {
+    unsigned int c = 0u;
+#pragma unroll
+    for (int k = 0; k < kHistCopies; ++k) c += sh[k * n_bins + b];
+    if (c) atomicAdd(&hist[b], (unsigned long long)c);
+  }
+}
+
+// grid = n_candidates, block = 256.  Fixed per-thread bin assignment and a fixed reduction tree:
+// the result does not depend on scheduling.
+__global__ void __launch_bounds__(256)
+score_kernel(const unsigned long long* __restrict__ hist, const float* __restrict__ maxp, int n_bins,
+             int n_candidates, int L, int is_signed, double* __restrict__ scores) {
+  __shared__ double red[256];
+  const int c = blockIdx.x + 1;
+  const float m = *maxp;
+  double acc = 0.0;
+  if (m > 0.0f) {
+    const float alpha_c = __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)c), (double)n_candidates));
+    const double step = __ddiv_rn((double)alpha_c, (double)L);
+    const double width = __ddiv_rn((double)m, (double)n_bins);
+    const double lo = is_signed ? -(double)L : 0.0, hi = (double)L;
+    for (int b = threadIdx.x; b < n_bins; b += 256) {
+      const double xb = __dmul_rn(__dadd_rn((double)b, 0.5), width);
+      double q = rint(__ddiv_rn(xb, step));
+      q = fmin(fmax(q, lo), hi);
+      const double e = __dsub_rn(xb, __dmul_rn(q, step));
+      acc = __dadd_rn(acc, __dmul_rn(__dmul_rn((double)hist[b], e), e));
+    }
+  }
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] = __dadd_rn(red[threadIdx.x], red[threadIdx.x + s]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) scores[blockIdx.x] = red[0];
+}
+
+__global__ void pick_kernel(const double* __restrict__ scores, const float* __restrict__ maxp, int n_candidates,
+                            float* __restrict__ alpha_sel) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const float m = *maxp;
+  if (!(m > 0.0f)) { *alpha_sel = 0.0f; return; }
+  int best = 1;
+  double bs = scores[0];
+  for (int c = 2; c <= n_candidates; ++c) {
+    const double s = scores[c - 1];
+    if (s <= bs) { bs = s; best = c; }  // ties to the largest threshold
+  }
+  *alpha_sel = __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)best), (double)n_candidates));
+}
+
+__global__ void __launch_bounds__(256)
+quantize_kernel(View v, const float* __restrict__ alpha_p, int L, int is_signed, int8_t* __restrict__ codes,
+                long long ld_codes, int packed_ok, float* __restrict__ scale_out, float* __restrict__ alpha_out,
+                int* dev_status) {
+  const float alpha = *alpha_p;
+  const bool zero = !(alpha > 0.0f);
+  const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)L);
+  const float inv = zero ? 0.0f : __fdiv_rn((float)L, alpha);
+  const float lo = is_signed ? -(float)L : 0.0f, hi = (float)L;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *scale_out = step;
+    if (alpha_out) *alpha_out = zero ? 0.0f : alpha;
+  }
+  bool bad = false;
+  for (long long t = blockIdx.x; t < v.tiles; t += gridDim.x) {
+    float x[kTileQuads][4];
+    int n[kTileQuads];
+    long long row[kTileQuads], col[kTileQuads];
+#pragma unroll
+    for (int u = 0; u < kTileQuads; ++u) n[u] = load_quad(v, t, u, x[u], &row[u], &col[u]);
+#pragma unroll
+    for (int u = 0; u < kTileQuads; ++u) {
+      if (!n[u]) continue;
+      unsigned int word = 0u;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        bad |= (i < n[u]) && !is_finite(x[u][i]);
+        float q = rintf(__fmul_rn(x[u][i], inv));  // round half to even
+        q = fminf(fmaxf(q, lo), hi);
+        word |= ((unsigned int)((int)q) & 0xFFu) << (8 * i);
+      }
+      // the dense view flattens rows, so its code offset is the flat index
+      int8_t* out = codes + row[u] * ld_codes + col[u];
+      if (packed_ok && n[u] == 4) {
+        *reinterpret_cast<unsigned int*>(out) = word;
+      } else {
+        for (int i = 0; i < n[u]; ++i) out[i] = (int8_t)((word >> (8 * i)) & 0xFFu);
+      }
+    }
+  }
+  if (bad) flag(dev_status, OCS_DEV_NONFINITE);
+}
+
+struct QuantWs {
+  unsigned int* maxbits;       // fp32 bits of max|T|
+  float* alpha_sel;
+  unsigned long long* hist;
+  double* scores;
+  size_t total;
+};
+
+QuantWs carve_quant_ws(void* ws, int n_bins, int n_candidates) {
+  QuantWs w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    unsigned char* p = ws ? reinterpret_cast<unsigned char*>(ws) + off : nullptr;
+    off += align_up(bytes, 256);
+    return p;
+  };
+  w.maxbits = reinterpret_cast<unsigned int*>(take(256));
+  w.alpha_sel = reinterpret_cast<float*>(take(256));
+  w.hist = reinterpret_cast<unsigned long long*>(take(8 * (size_t)(n_bins > 0 ? n_bins : 1)));
+  w.scores = reinterpret_cast<double*>(take(8 * (size_t)(n_candidates > 0 ? n_candidates : 1)));
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+}  // namespace ocs
+
+using namespace ocs;
+
+extern "C" size_t ocs_quantize_workspace_bytes(int n_bins, int n_candidates) {
+  return carve_quant_ws(nullptr, n_bins, n_candidates).total;
+}
+
+extern "C" void ocs_quantize_workspace_views(void* ws, int n_bins, int n_candidates, uint64_t** hist,
+                                             double** scores) {
+  const QuantWs w = carve_quant_ws(ws, n_bins, n_candidates);
+  if (hist) *hist = reinterpret_cast<uint64_t*>(w.hist);
+  if (scores) *scores = w.scores;
+}
+
+extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, int64_t ld_in, int bits, int is_signed,
+                                   ocs_clip_mode mode, int n_candidates, int n_bins, const float* max_abs_in,
+                                   int8_t* codes, int64_t ld_codes, float* scale, float* alpha, void* ws,
+                                   size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!T || !codes || !scale) return OCS_ERR_INVALID_ARG;
+  if (bits < 2 || bits > 8) return OCS_ERR_INVALID_ARG;
+  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE) return OCS_ERR_INVALID_ARG;
+  if (mode == OCS_CLIP_MSE && (n_candidates < 1 || n_candidates > kMaxCandidates || n_bins < 1 || n_bins > kMaxBins))
+    return OCS_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ld_in < cols || ld_codes < cols) return OCS_ERR_SHAPE;
+  if (!aligned(T, 4)) return OCS_ERR_SHAPE;
+  if (mode == OCS_CLIP_NONE) { n_bins = 1; n_candidates = 1; }
+  const QuantWs w = carve_quant_ws(ws, n_bins, n_candidates);
+  if (!ws || !aligned(ws, 256) || ws_bytes < w.total) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+
+  const View v = make_view(T, rows, cols, ld_in);
+  const int grid = grid_for(v.tiles);
+  const int L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
+
+  const float* maxp = max_abs_in;
+  if (!maxp) {
+    if (cudaMemsetAsync(w.maxbits, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
+    maxabs_kernel<<<grid, 256, 0, stream>>>(v, w.maxbits);
+    if ((st = launch_status()) != OCS_OK) return st;
+    maxp = reinterpret_cast<const float*>(w.maxbits);
+  }
+  const float* alpha_p = maxp;
+  if (mode == OCS_CLIP_MSE) {
+    if (cudaMemsetAsync(w.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
+    hist_kernel<<<grid, 256, sizeof(unsigned int) * kHistCopies * n_bins, stream>>>(v, maxp, n_bins, w.hist);
+    if ((st = launch_status()) != OCS_OK) return st;
+    score_kernel<<<n_candidates, 256, 0, stream>>>(w.hist, maxp, n_bins, n_candidates, L, is_signed, w.scores);
+    if ((st = launch_status()) != OCS_OK) return st;
+    pick_kernel<<<1, 32, 0, stream>>>(w.scores, maxp, n_candidates, w.alpha_sel);
+    if ((st = launch_status()) != OCS_OK) return st;
+    alpha_p = w.alpha_sel;
+  }
+  // the dense view addresses codes by flat index; that is only valid when the codes are dense too
+  View vq = v;
+  long long ldc = ld_codes;
+  if (ld_in == cols && ld_codes != cols) {  // dense input, padded output: keep the 2-D view
+    vq.rows = rows; vq.cols = cols; vq.ld = ld_in;
+    vq.vec = aligned(T, 16) && (ld_in % 4 == 0);
+    vq.tiles_per_row = (cols + kTileCols - 1) / kTileCols;
+    vq.tiles = rows * vq.tiles_per_row;
+  } else if (ld_in == cols) {
+    ldc = rows * cols;
+  }
+  const int packed_ok = aligned(codes, 4) && (ldc % 4 == 0);
+  quantize_kernel<<<grid_for(vq.tiles), 256, 0, stream>>>(vq, alpha_p, L, is_signed, codes, ldc, packed_ok, scale,
+                                                         alpha, dev_status);
+  return launch_status();
+}

@@ -1,0 +1,152 @@
+"""GPU parity: ocs_qlinear / ocs_qconv against the CPU checker, through the C ABI.
+Bars: int32 accumulators bit-exact; Y <= 1e-5 relative (it is one fmaf of exact inputs on both
+sides, so equality is asserted too)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_1901_09504_b200 as ocs
+from ocs_inputs import configs, prng
+from oracle import oracle as orc
+
+from gpu_util import dev, host
+
+pytestmark = pytest.mark.gpu
+
+
+def _rand_idx(seed, Cn, S):
+    return np.concatenate([np.arange(Cn), configs.random_codes(seed, 7, (S,), 0, Cn - 1, np.int32)]).astype(np.int32) \
+        if S else np.arange(Cn, dtype=np.int32)
+
+
+def _check_linear(seed, M, Cn, N, S, a_signed=False, lda=None, bias=True, a_scale=0.013, w_scale=0.0007):
+    A = configs.random_codes(seed, 0, (M, Cn), -127 if a_signed else 0, 127 if a_signed else 255,
+                             np.int8 if a_signed else np.uint8)
+    Wc = configs.random_codes(seed, 1, (N, Cn + S), -127, 127, np.int8)
+    idx = _rand_idx(seed, Cn, S)
+    b = prng.normal(seed, 9, (N,)) if bias else None
+    Yo, acco = orc.qlinear(A, a_signed, a_scale, Wc, w_scale, idx, b)
+    lda = lda or Cn
+    Ad = torch.zeros((M, lda), dtype=torch.int8 if a_signed else torch.uint8, device="cuda")
+    Ad[:, :Cn] = dev(A)
+    ldw = ocs.round_up(Cn + S, 16)
+    Wd = torch.zeros((N, ldw), dtype=torch.int8, device="cuda")
+    Wd[:, :Cn + S] = dev(Wc)
+    st = ocs.new_status()
+    Y, acc = ocs.ocs_qlinear(Ad, dev(np.array([a_scale], np.float32)), Wd, dev(np.array([w_scale], np.float32)),
+                             dev(idx), Cn, S, bias=None if b is None else dev(b), want_acc=True, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    np.testing.assert_array_equal(host(acc), acco)
+    np.testing.assert_allclose(host(Y), Yo, rtol=1e-5, atol=0)
+    np.testing.assert_array_equal(host(Y), Yo)
+
+
+@pytest.mark.parametrize("M,Cn,N,S", [(64, 512, 256, 26), (128, 256, 128, 0), (1, 16, 8, 0), (5, 130, 70, 3),
+                                      (200, 384, 300, 140), (20, 650, 2600, 13), (128, 1000, 64, 17)])
+def test_qlinear_tma_path(M, Cn, N, S):
+    _check_linear(M + Cn, M, Cn, N, S, lda=ocs.round_up(Cn, 16))
+
+
+@pytest.mark.parametrize("M,Cn,N,S", [(64, 515, 256, 26), (3, 7, 5, 2), (130, 129, 33, 1)])
+def test_qlinear_gather_path(M, Cn, N, S):
+    _check_linear(M + Cn + 1, M, Cn, N, S, lda=Cn + 1)       # unaligned rows: every block is assembled by threads
+
+
+def test_qlinear_signed_nobias_and_splitk():
+    _check_linear(11, 20, 650, 2600, 13, a_signed=True, lda=656)
+    _check_linear(12, 128, 6272, 512, 314, bias=False, lda=6272)    # few tiles, long K: split-K
+    _check_linear(13, 100, 4099, 200, 77, lda=4112)
+
+
+def test_qlinear_config1_end_to_end():
+    """split -> quantize -> activation quantize -> qlinear, every stage compared."""
+    c = configs.config1()
+    W, A = c["W"], c["A"]
+    S = 26
+    Wp, idx, _, _ = orc.split(W, S)
+    wc, ws_ = orc.quantize(Wp, 8, True, orc.maxabs(Wp))
+    ac, as_ = orc.quantize(A, 8, False, orc.maxabs(A))
+    Yo, acco = orc.qlinear(ac, False, as_, wc, ws_, idx)
+    Wout, idx_d, _, mx = ocs.ocs_split(dev(W), S)
+    codes, scale, _ = ocs.ocs_quantize(Wout, 8, True, ocs.CLIP_NONE, cols=512 + S, max_abs_in=mx[1:2])
+    acodes, ascale, _ = ocs.ocs_quantize(dev(A), 8, False, ocs.CLIP_NONE)
+    Y, acc = ocs.ocs_qlinear(acodes, ascale, codes, scale, idx_d, 512, S, want_acc=True)
+    np.testing.assert_array_equal(host(codes)[:, :512 + S], wc)
+    np.testing.assert_array_equal(host(acc), acco)
+    np.testing.assert_array_equal(host(Y), Yo)
+    # the quantized split layer tracks the float layer (Eq. 3 = Eq. 2 up to quantization error)
+    ref = A.astype(np.float64) @ W.astype(np.float64).T
+    assert np.abs(host(Y) - ref).max() < 0.02 * np.abs(ref).max()
+
+
+def test_qlinear_bad_index_flag_and_args():
+    A = torch.zeros((8, 32), dtype=torch.uint8, device="cuda")
+    Wd = torch.zeros((8, 48), dtype=torch.int8, device="cuda")
+    idx = np.arange(34, dtype=np.int32)
+    idx[33] = 99
+    one = dev(np.ones(1, np.float32))
+    st = ocs.new_status()
+    ocs.ocs_qlinear(A, one, Wd, one, dev(idx), 32, 2, dev_status=st)
+    assert ocs.ocs_poll_status(st) & ocs.DEV_BAD_INDEX
+    with pytest.raises(ocs.OcsError):
+        ocs.ocs_qlinear(A, one, Wd[:, :40], one, dev(idx), 32, 20)       # ldw too small
+
+
+def _check_conv(seed, Nb, H, Wd_, Cn, O, S, k, stride, pad, a_signed=False):
+    X = configs.random_codes(seed, 0, (Nb, H, Wd_, Cn), -127 if a_signed else 0, 127 if a_signed else 255,
+                             np.int8 if a_signed else np.uint8)
+    Wc = configs.random_codes(seed, 1, (O, Cn + S, k, k), -127, 127, np.int8)
+    idx = _rand_idx(seed, Cn, S)
+    b = prng.normal(seed, 9, (O,))
+    Yo, acco = orc.qconv(X, a_signed, 0.02, Wc, 0.003, idx, stride, pad, b)
+    packed = ocs.ocs_pack_conv_weights(dev(Wc.reshape(O, -1)), O, Cn, S, k, k)
+    # the packing is a pure permutation: check it against numpy
+    ref_pack = np.concatenate([Wc[:, :Cn].transpose(0, 2, 3, 1).reshape(O, -1),
+                               Wc[:, Cn:].transpose(0, 2, 3, 1).reshape(O, -1)], axis=1)
+    np.testing.assert_array_equal(host(packed)[:, :ref_pack.shape[1]], ref_pack)
+    assert not host(packed)[:, ref_pack.shape[1]:].any()
+    st = ocs.new_status()
+    Y, acc = ocs.ocs_qconv(dev(X), dev(np.array([0.02], np.float32)), packed, dev(np.array([0.003], np.float32)),
+                           dev(idx), S, k, k, stride, pad, bias=dev(b), want_acc=True, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    np.testing.assert_array_equal(host(acc), acco)
+    np.testing.assert_array_equal(host(Y), Yo)
+
+
+@pytest.mark.parametrize("Nb,H,W,Cn,O,S,k,stride,pad", [
+    (2, 7, 8, 5, 4, 3, 3, 1, 1),        # tiny, odd channels
+    (2, 11, 11, 3, 16, 1, 7, 2, 3),     # first-layer shape: 3 channels, 7x7 stride 2
+    (3, 14, 14, 128, 64, 2, 3, 1, 1),   # C = 128: original channels by TMA, duplicates by threads
+    (2, 9, 9, 256, 40, 3, 1, 1, 0),     # 1x1
+    (2, 14, 14, 64, 32, 1, 3, 1, 1),    # C = 64: blocks straddle taps
+    (2, 16, 16, 128, 24, 2, 3, 2, 1),   # stride 2
+    (2, 8, 8, 256, 24, 3, 1, 2, 0),     # 1x1 stride 2 (downsample)
+    (1, 5, 6, 32, 8, 0, 3, 1, 1),       # no splits
+])
+def test_qconv_shapes(Nb, H, W, Cn, O, S, k, stride, pad):
+    _check_conv(Nb * 100 + Cn, Nb, H, W, Cn, O, S, k, stride, pad)
+
+
+def test_qconv_signed_input():
+    _check_conv(5, 2, 9, 9, 3, 8, 1, 7, 2, 3, a_signed=True)
+
+
+def test_qconv_config2_reduced_batch():
+    """Config 2's layer (256 -> 256, 3x3, 14x14, r = 0.02, 6-bit MSE-clipped weights) on 4 images."""
+    c = configs.config2(batch=4)
+    W, X = c["W"], c["X"]
+    S = 6
+    Wp, idx, _, _ = orc.split(W, S)
+    alpha = orc.clip_mse(Wp, 6, True, 2048, 128)["alpha"]
+    wc, wscale = orc.quantize(Wp, 6, True, alpha)
+    Xh = orc.nchw_to_nhwc(X)
+    xc, xscale = orc.quantize(Xh, 8, False, orc.maxabs(Xh))
+    Yo, acco = orc.qconv(xc, False, xscale, wc, wscale, idx, 1, 1)
+    Wout, idx_d, _, mx = ocs.ocs_split(dev(W), S)
+    codes, scale, al = ocs.ocs_quantize(Wout, 6, True, ocs.CLIP_MSE, cols=(256 + S) * 9, max_abs_in=mx[1:2])
+    assert np.float32(host(al)[0]) == np.float32(alpha)
+    packed = ocs.ocs_pack_conv_weights(codes, 256, 256, S, 3, 3)
+    xcodes, xs, _ = ocs.ocs_quantize(dev(Xh).reshape(-1, 256), 8, False, ocs.CLIP_NONE)
+    Y, acc = ocs.ocs_qconv(xcodes.reshape(4, 14, 14, 256), xs, packed, scale, idx_d, S, 3, 3, 1, 1, want_acc=True)
+    np.testing.assert_array_equal(host(acc), acco)
+    np.testing.assert_array_equal(host(Y), Yo)
