@@ -67,6 +67,24 @@ ocs_status ocs_poll_status(const int* dev_status, void* stream, int* host_out);
 /* Version string of the build (host). */
 const char* ocs_version(void);
 
+/* Launch accounting and tracing (host; no counterpart in the paper, used by reports) ------
+ * ocs_kernel_launches(): number of kernels this process has launched through the library.
+ * ocs_trace_start(max_records): from now on every kernel launch of the library is bracketed
+ * by a pair of CUDA events on its stream (at most max_records launches are recorded; the
+ * events are created on first use and reused).  ocs_trace_stop(rows, capacity): ends the
+ * trace, waits for the recorded launches and writes one row per kernel name (launch count,
+ * summed device time in ms) into rows[0..capacity); returns the number of rows written, or
+ * -1 if an event could not be read.  Tracing is process-wide and meant for one stream at a
+ * time; it is off by default and costs nothing then. */
+typedef struct {
+  char name[48];
+  long long launches;
+  double total_ms;
+} ocs_trace_row;
+long long ocs_kernel_launches(void);
+ocs_status ocs_trace_start(int max_records);
+int ocs_trace_stop(ocs_trace_row* rows, int capacity);
+
 /* ocs_split -------------------------------------------------------------------------------
  * Weight OCS (Section 3.2 Eq. 3, Section 3.3, Section 3.4): S times, take the channel that
  * holds the largest |w| of the CURRENT expanded tensor (ties: the smallest current channel

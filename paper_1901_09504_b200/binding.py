@@ -24,6 +24,7 @@ CLIP_NONE, CLIP_MSE = 0, 1
 
 EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
+    "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
     "ocs_split_workspace_bytes", "ocs_split",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
@@ -52,6 +53,7 @@ def lib():
                      "ocs_qconv_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.ocs_quantize_workspace_views.restype = None
+        L.ocs_kernel_launches.restype = C.c_longlong
         _lib = L
     return _lib
 
@@ -88,14 +90,36 @@ def ocs_poll_status(dev_status) -> int:
     return int(out.value)
 
 
+class _TraceRow(C.Structure):
+    _fields_ = [("name", C.c_char * 48), ("launches", C.c_longlong), ("total_ms", C.c_double)]
+
+
+def ocs_kernel_launches() -> int:
+    return int(lib().ocs_kernel_launches())
+
+
+def ocs_trace_start(max_records: int = 65536) -> None:
+    _check(lib().ocs_trace_start(int(max_records)), "ocs_trace_start")
+
+
+def ocs_trace_stop(capacity: int = 64) -> dict:
+    """-> {kernel name: (launches, total device ms)} of the launches since ocs_trace_start."""
+    rows = (_TraceRow * capacity)()
+    n = lib().ocs_trace_stop(rows, capacity)
+    if n < 0:
+        raise OcsError("ocs_trace_stop", 5)
+    return {rows[i].name.decode(): (int(rows[i].launches), float(rows[i].total_ms)) for i in range(n)}
+
+
 def round_up(x: int, m: int) -> int:
     return (x + m - 1) // m * m
 
 
 def ocs_split(W, S: int, qa_step: float = 0.0, qa_bits: int = 0, ld_out: int | None = None, dev_status=None,
-              want_order: bool = True):
+              want_order: bool = True, out=None, ws=None):
     """W fp32 [O, C] or [O, C, kh, kw] (contiguous).  Returns (W_out [O, ld_out] fp32 whose first
-    (C+S)*R columns are W', idx_map int32 [C+S], split_order int32 [S], max_abs fp32 [3])."""
+    (C+S)*R columns are W', idx_map int32 [C+S], split_order int32 [S], max_abs fp32 [3]).
+    `out` = (W_out, idx_map, order, max_abs) and `ws` reuse caller-held buffers instead of allocating."""
     assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
     O, Cn = W.shape[0], W.shape[1]
     R = 1
@@ -104,12 +128,19 @@ def ocs_split(W, S: int, qa_step: float = 0.0, qa_bits: int = 0, ld_out: int | N
     cols_out = (Cn + S) * R
     if ld_out is None:
         ld_out = round_up(cols_out, 4)
-    W_out = torch.empty((O, ld_out), dtype=torch.float32, device=W.device)
-    idx_map = torch.empty(Cn + S, dtype=torch.int32, device=W.device)
-    order = torch.empty(max(S, 1), dtype=torch.int32, device=W.device) if want_order else None
-    max_abs = torch.zeros(3, dtype=torch.float32, device=W.device)
+    if out is not None:
+        W_out, idx_map, order, max_abs = out
+        ld_out = W_out.stride(0)
+        assert W_out.shape[0] == O and ld_out >= cols_out and idx_map.numel() >= Cn + S and max_abs.numel() >= 3
+        want_order = order is not None
+    else:
+        W_out = torch.empty((O, ld_out), dtype=torch.float32, device=W.device)
+        idx_map = torch.empty(Cn + S, dtype=torch.int32, device=W.device)
+        order = torch.empty(max(S, 1), dtype=torch.int32, device=W.device) if want_order else None
+        max_abs = torch.zeros(3, dtype=torch.float32, device=W.device)
     nws = lib().ocs_split_workspace_bytes(O, Cn, R, int(S))
-    ws = _ws(nws, W.device)
+    if ws is None:
+        ws = _ws(nws, W.device)
     st = lib().ocs_split(_ptr(W), O, Cn, R, C.c_int64(Cn * R), int(S), C.c_float(qa_step), int(qa_bits),
                          _ptr(W_out), C.c_int64(ld_out), _ptr(idx_map), _ptr(order), _ptr(max_abs), _ptr(ws),
                          C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
@@ -119,7 +150,7 @@ def ocs_split(W, S: int, qa_step: float = 0.0, qa_bits: int = 0, ld_out: int | N
 
 def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_candidates: int = 128,
                  n_bins: int = 2048, cols: int | None = None, ld_codes: int | None = None, max_abs_in=None,
-                 dev_status=None, return_search: bool = False):
+                 dev_status=None, return_search: bool = False, out=None, ws=None):
     """T fp32 2-D [rows, ld_in] (row stride = T.stride(0)); `cols` valid columns per row (default all).
     Returns (codes int8/uint8 [rows, ld_codes], scale fp32 [1], alpha fp32 [1]) and, with
     return_search, also (hist uint64 [n_bins] as int64, scores float64 [n_candidates])."""
@@ -129,11 +160,17 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
         cols = T.shape[1]
     if ld_codes is None:
         ld_codes = round_up(cols, 16)
-    codes = torch.zeros((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=T.device)
-    scale = torch.zeros(1, dtype=torch.float32, device=T.device)
-    alpha = torch.zeros(1, dtype=torch.float32, device=T.device)
+    if out is not None:
+        codes, scale, alpha = out
+        ld_codes = codes.stride(0)
+        assert codes.shape[0] == rows and ld_codes >= cols
+    else:
+        codes = torch.empty((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=T.device)
+        scale = torch.zeros(1, dtype=torch.float32, device=T.device)
+        alpha = torch.zeros(1, dtype=torch.float32, device=T.device)
     nws = lib().ocs_quantize_workspace_bytes(int(n_bins), int(n_candidates))
-    ws = _ws(nws, T.device)
+    if ws is None:
+        ws = _ws(nws, T.device)
     st = lib().ocs_quantize(_ptr(T), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_in), int(bits),
                             int(bool(is_signed)), int(mode), int(n_candidates), int(n_bins), _ptr(max_abs_in),
                             _ptr(codes), C.c_int64(ld_codes), _ptr(scale), _ptr(alpha), _ptr(ws),
@@ -150,16 +187,18 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
 
 
 def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, bias=None, want_acc: bool = False,
-                dev_status=None):
+                dev_status=None, out=None, ws=None):
     """A_codes uint8/int8 [M, lda>=C]; W_codes int8 [N, ldw>=C+S].  Returns Y fp32 [M, N] (and acc int32)."""
     assert A_codes.is_cuda and A_codes.dim() == 2 and A_codes.stride(1) == 1
     assert W_codes.dtype == torch.int8 and W_codes.dim() == 2 and W_codes.stride(1) == 1
     M, N = A_codes.shape[0], W_codes.shape[0]
     a_signed = 1 if A_codes.dtype == torch.int8 else 0
-    Y = torch.empty((M, N), dtype=torch.float32, device=A_codes.device)
+    Y = out if out is not None else torch.empty((M, N), dtype=torch.float32, device=A_codes.device)
+    assert Y.stride(0) == N and Y.stride(1) == 1
     acc = torch.empty((M, N), dtype=torch.int32, device=A_codes.device) if want_acc else None
     nws = lib().ocs_qlinear_workspace_bytes(M, N, int(C_in), int(S))
-    ws = _ws(nws, A_codes.device)
+    if ws is None:
+        ws = _ws(nws, A_codes.device)
     st = lib().ocs_qlinear(_ptr(A_codes), a_signed, _ptr(a_scale), M, int(C_in), C.c_int64(A_codes.stride(0)),
                            _ptr(W_codes), _ptr(w_scale), N, int(S), C.c_int64(W_codes.stride(0)), _ptr(idx_map),
                            _ptr(bias), _ptr(Y), C.c_int64(N), _ptr(acc), _ptr(ws), C.c_size_t(ws.numel()),
@@ -168,13 +207,15 @@ def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, 
     return (Y, acc) if want_acc else Y
 
 
-def ocs_pack_conv_weights(codes, O: int, C_in: int, S: int, kh: int, kw: int, ld_dst: int | None = None):
+def ocs_pack_conv_weights(codes, O: int, C_in: int, S: int, kh: int, kw: int, ld_dst: int | None = None, out=None):
     """codes int8 [O, ld_src] in [C+S][kh*kw] order per row -> packed int8 [O, ld_dst]."""
     assert codes.is_cuda and codes.dtype == torch.int8 and codes.dim() == 2 and codes.stride(1) == 1
     Kt = kh * kw * (C_in + S)
     if ld_dst is None:
         ld_dst = round_up(Kt, 16)
-    packed = torch.empty((O, ld_dst), dtype=torch.int8, device=codes.device)
+    if out is not None:
+        ld_dst = out.stride(0)
+    packed = out if out is not None else torch.empty((O, ld_dst), dtype=torch.int8, device=codes.device)
     st = lib().ocs_pack_conv_weights(_ptr(codes), O, int(C_in), int(S), int(kh), int(kw),
                                      C.c_int64(codes.stride(0)), _ptr(packed), C.c_int64(ld_dst), _stream())
     _check(st, "ocs_pack_conv_weights")
@@ -182,7 +223,7 @@ def ocs_pack_conv_weights(codes, O: int, C_in: int, S: int, kh: int, kw: int, ld
 
 
 def ocs_qconv(X_codes, a_scale, W_packed, w_scale, idx_map, S: int, kh: int, kw: int, stride: int, pad: int,
-              bias=None, want_acc: bool = False, dev_status=None):
+              bias=None, want_acc: bool = False, dev_status=None, out=None, ws=None):
     """X_codes uint8/int8 NHWC [Nb, H, W, C] contiguous; W_packed from ocs_pack_conv_weights.
     Returns Y fp32 NHWC [Nb, Ho, Wo, O] (and acc int32)."""
     assert X_codes.is_cuda and X_codes.dim() == 4 and X_codes.is_contiguous()
@@ -191,10 +232,11 @@ def ocs_qconv(X_codes, a_scale, W_packed, w_scale, idx_map, S: int, kh: int, kw:
     Ho = (H + 2 * pad - kh) // stride + 1
     Wo = (Wd + 2 * pad - kw) // stride + 1
     a_signed = 1 if X_codes.dtype == torch.int8 else 0
-    Y = torch.empty((Nb, Ho, Wo, O), dtype=torch.float32, device=X_codes.device)
+    Y = out if out is not None else torch.empty((Nb, Ho, Wo, O), dtype=torch.float32, device=X_codes.device)
     acc = torch.empty((Nb, Ho, Wo, O), dtype=torch.int32, device=X_codes.device) if want_acc else None
     nws = lib().ocs_qconv_workspace_bytes(Nb, H, Wd, Cn, O, int(S), kh, kw, stride, pad)
-    ws = _ws(nws, X_codes.device)
+    if ws is None:
+        ws = _ws(nws, X_codes.device)
     st = lib().ocs_qconv(_ptr(X_codes), a_signed, _ptr(a_scale), Nb, H, Wd, Cn, _ptr(W_packed), _ptr(w_scale), O,
                          int(S), kh, kw, stride, pad, C.c_int64(W_packed.stride(0)), _ptr(idx_map), _ptr(bias),
                          _ptr(Y), _ptr(acc), _ptr(ws), C.c_size_t(ws.numel()), _ptr(dev_status), _stream())

@@ -54,4 +54,15 @@ inline ocs_status launch_status() {
   return cudaGetLastError() == cudaSuccess ? OCS_OK : OCS_ERR_CUDA;
 }
 
+// Launch accounting (defined in api.cu).  Every kernel launch of the library sits inside one
+// LaunchScope: it bumps the process-wide launch counter and, while a trace is active, brackets
+// the launch with a pair of CUDA events on the launch stream.
+void trace_begin(const char* name, cudaStream_t stream);
+void trace_end(cudaStream_t stream);
+struct LaunchScope {
+  cudaStream_t stream;
+  LaunchScope(const char* name, cudaStream_t s) : stream(s) { trace_begin(name, s); }
+  ~LaunchScope() { trace_end(stream); }
+};
+
 }  // namespace ocs

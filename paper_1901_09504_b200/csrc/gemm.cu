@@ -556,6 +556,7 @@ ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const Gem
     attr_set = true;
   }
   dim3 grid(plan.m_tiles, plan.n_tiles, plan.split_k);
+  LaunchScope ls(p.mode == MODE_CONV ? "ocs_gemm_kernel(conv)" : "ocs_gemm_kernel(linear)", stream);
   ocs_gemm_kernel<BN><<<grid, kGemmThreads, L::kDynBytes, stream>>>(tmB, tmA, p);
   return launch_status();
 }
@@ -710,6 +711,7 @@ extern "C" ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, i
   if (st != OCS_OK) return st;
   const long long total = (long long)O * ld_dst;
   const int grid = (int)((total + 255) / 256 < kNumSMs * 8 ? (total + 255) / 256 : kNumSMs * 8);
+  LaunchScope ls("pack_conv_kernel", stream);
   pack_conv_kernel<<<grid, 256, 0, stream>>>(codes, O, C, S, kh * kw, ld_src, packed, ld_dst);
   return launch_status();
 }

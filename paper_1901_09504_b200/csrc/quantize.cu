@@ -278,6 +278,7 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   const float* maxp = max_abs_in;
   if (!maxp) {
     if (cudaMemsetAsync(w.maxbits, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
+    LaunchScope ls("maxabs_kernel", stream);
     maxabs_kernel<<<grid, 256, 0, stream>>>(v, w.maxbits);
     if ((st = launch_status()) != OCS_OK) return st;
     maxp = reinterpret_cast<const float*>(w.maxbits);
@@ -285,11 +286,20 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   const float* alpha_p = maxp;
   if (mode == OCS_CLIP_MSE) {
     if (cudaMemsetAsync(w.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
-    hist_kernel<<<grid, 256, sizeof(unsigned int) * kHistCopies * n_bins, stream>>>(v, maxp, n_bins, w.hist);
+    {
+      LaunchScope ls("hist_kernel", stream);
+      hist_kernel<<<grid, 256, sizeof(unsigned int) * kHistCopies * n_bins, stream>>>(v, maxp, n_bins, w.hist);
+    }
     if ((st = launch_status()) != OCS_OK) return st;
-    score_kernel<<<n_candidates, 256, 0, stream>>>(w.hist, maxp, n_bins, n_candidates, L, is_signed, w.scores);
+    {
+      LaunchScope ls("score_kernel", stream);
+      score_kernel<<<n_candidates, 256, 0, stream>>>(w.hist, maxp, n_bins, n_candidates, L, is_signed, w.scores);
+    }
     if ((st = launch_status()) != OCS_OK) return st;
-    pick_kernel<<<1, 32, 0, stream>>>(w.scores, maxp, n_candidates, w.alpha_sel);
+    {
+      LaunchScope ls("pick_kernel", stream);
+      pick_kernel<<<1, 32, 0, stream>>>(w.scores, maxp, n_candidates, w.alpha_sel);
+    }
     if ((st = launch_status()) != OCS_OK) return st;
     alpha_p = w.alpha_sel;
   }
@@ -305,6 +315,7 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
     ldc = rows * cols;
   }
   const int packed_ok = aligned(codes, 4) && (ldc % 4 == 0);
+  LaunchScope ls("quantize_kernel", stream);
   quantize_kernel<<<grid_for(vq.tiles), 256, 0, stream>>>(vq, alpha_p, L, is_signed, codes, ldc, packed_ok, scale,
                                                          alpha, dev_status);
   return launch_status();

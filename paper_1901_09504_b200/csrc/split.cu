@@ -509,6 +509,7 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     const int rows = rows_per_cta_for(O, col_blocks);
     dim3 grid(col_blocks, (O + rows - 1) / rows);
     const bool vec = (ld_in % 4 == 0) && aligned(W, 16);
+    LaunchScope ls("col_minmax_kernel", stream);
     if (vec)
       col_minmax_kernel<true><<<grid, 256, 0, stream>>>(W, O, ncols, ld_in, rows, w.colmin, w.colmax, dev_status);
     else
@@ -538,6 +539,7 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
         return OCS_ERR_CUDA;
       attr_set = true;
     }
+    LaunchScope ls("split_plan_kernel", stream);
     split_plan_kernel<<<1, kPlanThreads, smem, stream>>>(a);
     if ((st = launch_status()) != OCS_OK) return st;
   }
@@ -547,6 +549,7 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     const int rows = rows_per_cta_for(O, col_blocks);
     dim3 grid(col_blocks, (O + rows - 1) / rows);
     const bool vec = (ld_in % 4 == 0) && (ld_out % 4 == 0) && aligned(W, 16) && aligned(W_out, 16);
+    LaunchScope ls("split_scatter_kernel", stream);
     if (vec)
       split_scatter_kernel<true><<<grid, 256, 0, stream>>>(W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth,
                                                            w.bits, w.qa_step_dev, rows);
