@@ -58,7 +58,6 @@ struct GemmParams {
   int32_t* acc_out;
   int32_t* acc_ws;              // [split_k][rows][N] partial sums when split_k > 1
   long long out_rows;           // rows of Y
-  unsigned int* tile_counters;  // one per output tile when split_k > 1
   int a_box_bytes;              // bytes one TMA load of A delivers
   int* dev_status;
 };
@@ -201,56 +200,72 @@ __device__ __forceinline__ RowInfo row_info(const GemmParams& p, int mt, int r) 
   return ri;
 }
 
-__device__ __forceinline__ uint32_t checked_src(const GemmParams& p, int j, bool* bad) {
+// Where contraction index k of a K-block reads from, relative to the row's base address (linear:
+// the row of A; convolution: the top-left pixel of the output pixel's receptive field).
+struct KSrc {
+  int off;   // byte offset from the row base; negative: this k contributes zero
+  int dydx;  // convolution: dy | dx << 8 of the filter tap (for the image-border test)
+};
+
+__device__ __forceinline__ int checked_src(const GemmParams& p, int j, bool* bad) {
   int c = __ldg(p.idx_map + j);
   if ((unsigned)c >= (unsigned)p.C) { *bad = true; c = 0; }
-  return (uint32_t)c;
+  return c;
 }
 
-// The 16 operand bytes of row `ri` for contraction indices [k0, k0 + 16).
-__device__ __forceinline__ uint4 gather_chunk(const GemmParams& p, const RowInfo& ri, int k0, bool* bad) {
-  uint4 out = make_uint4(0u, 0u, 0u, 0u);
-  if (ri.out_row < 0 || k0 >= p.Ktot) return out;
-  uint32_t w[4] = {0u, 0u, 0u, 0u};
+__device__ __forceinline__ KSrc k_source(const GemmParams& p, int k, bool* bad) {
+  KSrc e;
+  e.off = -1; e.dydx = 0;
+  if (k >= p.Ktot) return e;
   if (p.mode == MODE_LINEAR) {
-    const uint8_t* row = p.A + ri.out_row * p.lda;
-    if (p.a_vec16 && k0 + 16 <= p.C) return __ldg(reinterpret_cast<const uint4*>(row + k0));
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int k = k0 + i;
-      if (k < p.Ktot) {
-        const uint32_t c = k < p.C ? (uint32_t)k : checked_src(p, k, bad);
-        w[i >> 2] |= (uint32_t)__ldg(row + c) << (8 * (i & 3));
-      }
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
+    e.off = k < p.C ? k : checked_src(p, k, bad);
+    return e;
   }
   // convolution: contraction order is [tap][c < C] then [tap][s < S]
   const int KO = p.R * p.C;
-  const uint8_t* img = p.A + (long long)ri.n * p.H * p.Wd * p.C;
-  if (k0 + 16 <= KO && p.a_vec16) {  // C % 16 == 0: the chunk lies inside one tap
-    const int tap = k0 / p.C, c0 = k0 - tap * p.C;
-    const int ih = ri.ih0 + tap / p.kw, iw = ri.iw0 + tap % p.kw;
-    if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd)
-      return __ldg(reinterpret_cast<const uint4*>(img + ((long long)ih * p.Wd + iw) * p.C + c0));
-    return out;
-  }
-  int k = k0;
-  int tap, sub, width;  // position inside the current region: sub in [0, width)
-  if (k < KO) { tap = k / p.C; sub = k - tap * p.C; width = p.C; }
-  else { const int kd = k - KO; tap = kd / p.S; sub = kd - tap * p.S; width = p.S; }
+  int tap, c;
+  if (k < KO) { tap = k / p.C; c = k - tap * p.C; }
+  else { const int kd = k - KO; tap = kd / p.S; c = checked_src(p, p.C + (kd - tap * p.S), bad); }
+  const int dy = tap / p.kw, dx = tap - dy * p.kw;
+  e.off = (dy * p.Wd + dx) * p.C + c;
+  e.dydx = dy | (dx << 8);
+  return e;
+}
+
+// The operand bytes of one tile row for the 16 contraction indices whose sources are tab[0..16).
+// Every load is unconditional (a source that contributes zero reads the tensor's first byte and is
+// masked afterwards), so the 16 loads are independent and in flight together.
+__device__ __forceinline__ uint4 gather_chunk(const GemmParams& p, const RowInfo& ri, const uint8_t* base,
+                                              const KSrc* __restrict__ tab) {
+  uint32_t b[16];
 #pragma unroll
-  for (int i = 0; i < 16; ++i, ++k) {
-    if (k >= p.Ktot) break;
-    if (k == KO) { tap = 0; sub = 0; width = p.S; }
-    const int ih = ri.ih0 + tap / p.kw, iw = ri.iw0 + tap % p.kw;
-    if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd) {
-      const uint32_t c = k < KO ? (uint32_t)sub : checked_src(p, p.C + sub, bad);
-      w[i >> 2] |= (uint32_t)__ldg(img + ((long long)ih * p.Wd + iw) * p.C + c) << (8 * (i & 3));
+  for (int i = 0; i < 16; ++i) {
+    const KSrc e = tab[i];
+    bool ok = ri.out_row >= 0 && e.off >= 0;
+    if (p.mode == MODE_CONV) {
+      const int ih = ri.ih0 + (e.dydx & 255), iw = ri.iw0 + (e.dydx >> 8);
+      ok = ok && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd;
     }
-    if (++sub == width) { sub = 0; ++tap; }
+    const uint8_t* addr = ok ? base + e.off : p.A;
+    const uint32_t v = (uint32_t)__ldg(addr);
+    b[i] = ok ? v : 0u;
   }
+  uint32_t w[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) w[q] = b[4 * q] | (b[4 * q + 1] << 8) | (b[4 * q + 2] << 16) | (b[4 * q + 3] << 24);
   return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// A 16-byte chunk that is one aligned run of original channels (no duplicate, one filter tap).
+__device__ __forceinline__ uint4 direct_chunk(const GemmParams& p, const RowInfo& ri, int k0) {
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  if (ri.out_row < 0) return zero;
+  if (p.mode == MODE_LINEAR) return __ldg(reinterpret_cast<const uint4*>(p.A + ri.out_row * p.lda + k0));
+  const int tap = k0 / p.C, c0 = k0 - tap * p.C;
+  const int ih = ri.ih0 + tap / p.kw, iw = ri.iw0 + tap % p.kw;
+  if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd)
+    return __ldg(reinterpret_cast<const uint4*>(p.A + (((long long)ri.n * p.H + ih) * p.Wd + iw) * p.C + c0));
+  return zero;
 }
 
 template <int BN>
@@ -262,7 +277,9 @@ struct SmemLayout {
   static constexpr int kTileBytes = kStages * kStageBytes;
   static constexpr int kCtrlBytes = 1024;               // barriers, tensor-memory slot, flags
   static constexpr int kRowTableBytes = BM * 24;        // RowInfo per tile row
-  static constexpr int kDynBytes = kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes;
+  static constexpr int kSrcTableBytes = BK * 8;         // KSrc per contraction index of a gathered K-block
+  static constexpr int kDynBytes =
+      kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes + kSrcTableBytes;
 };
 
 template <int BN>
@@ -277,8 +294,8 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);           // full[kStages], empty[kStages], accum
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * L::kStages + 1));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * L::kStages + 1) + 8);
-  int* last_flag = const_cast<int*>(abort_flag) + 1;
   RowInfo* rows = reinterpret_cast<RowInfo*>(ctrl + L::kCtrlBytes);
+  KSrc* ksrc = reinterpret_cast<KSrc*>(ctrl + L::kCtrlBytes + L::kRowTableBytes);
   auto full_bar = [&](int s) { return smem_u32(bars + s); };
   auto empty_bar = [&](int s) { return smem_u32(bars + L::kStages + s); };
   const uint32_t accum_bar = smem_u32(bars + 2 * L::kStages);
@@ -295,7 +312,6 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     }
     mbar_init(accum_bar, 1);
     *abort_flag = 0;
-    *last_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmB);
     if (p.kb_tma_a > 0) prefetch_tmap(&tmA);
@@ -364,8 +380,12 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     const int gt = threadIdx.x - 64;   // 0..127
     rows[gt] = row_info(p, mt, gt);
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    const int chunk = gt & 7;          // 16-byte chunk of the 128-byte row
-    const int rbase = gt >> 3;         // rows rbase + 16*i
+    // gather thread gt builds tile row gt: consecutive contraction indices of one row are close in
+    // memory (one pixel's channels), so its loads share cache lines
+    const RowInfo my_row = rows[gt];
+    const uint8_t* my_base;
+    if (p.mode == MODE_LINEAR) my_base = p.A + (my_row.out_row >= 0 ? my_row.out_row : 0) * p.lda;
+    else my_base = p.A + (((long long)my_row.n * p.H + my_row.ih0) * p.Wd + my_row.iw0) * p.C;
     bool bad = false;
     bool ok = true;
     for (int i = 0; i < my_kb; ++i) {
@@ -374,14 +394,20 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       const uint32_t par = ((i / L::kStages) & 1) ^ 1;
       if (!mbar_wait(empty_bar(s), par, abort_flag)) { ok = false; break; }
       if (kb >= p.kb_tma_a) {
-        unsigned char* a_tile = tiles + s * L::kStageBytes;
-        uint4 v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = gather_chunk(p, rows[rbase + 16 * j], kb * BK + chunk * 16, &bad);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int r = rbase + 16 * j;
-          *reinterpret_cast<uint4*>(a_tile + r * 128 + ((chunk ^ (r & 7)) << 4)) = v[j];
+        unsigned char* a_row = tiles + s * L::kStageBytes + gt * 128;
+        // chunks of 16 original channels inside one tap move as one 16-byte load; the rest goes
+        // through the block's source table
+        const int direct_chunks = p.a_vec16 ? min(8, max(0, (p.R * p.C - kb * BK) >> 4)) : 0;
+        if (direct_chunks < 8) {  // uniform over the gather threads
+          asm volatile("bar.sync 1, 128;" ::: "memory");  // the previous block's table is no longer read
+          ksrc[gt] = k_source(p, kb * BK + gt, &bad);
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+#pragma unroll 2
+        for (int c = 0; c < 8; ++c) {
+          const uint4 v = c < direct_chunks ? direct_chunk(p, my_row, kb * BK + c * 16)
+                                            : gather_chunk(p, my_row, my_base, ksrc + c * 16);
+          *reinterpret_cast<uint4*>(a_row + ((c ^ (gt & 7)) << 4)) = v;
         }
         fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
       }
@@ -445,35 +471,6 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         }
       }
     }
-    if (!direct) {
-      // the last K slice to finish a tile sums all slices' partials (integer sums: exact in any order)
-      __threadfence();
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (gt == 0) {
-        int last = 0;
-        if (!*abort_flag) {
-          const unsigned int tile = blockIdx.y * gridDim.x + blockIdx.x;
-          last = (atomicAdd(p.tile_counters + tile, 1u) == (unsigned int)p.split_k - 1u) ? 1 : 0;
-        }
-        *last_flag = last;
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (*last_flag) {
-        __threadfence();
-        const int ncols = min(BN, p.N - nt * BN);
-        for (int rr = 0; rr < 32; ++rr) {
-          const long long orow = rows[q * 32 + rr].out_row;
-          if (orow < 0) continue;  // warp-uniform
-          for (int c = lane; c < ncols; c += 32) {
-            const int n = nt * BN + c;
-            int a = 0;
-            for (int z = 0; z < p.split_k; ++z) a += __ldcg(p.acc_ws + ((long long)z * p.out_rows + orow) * p.N + n);
-            p.Y[orow * p.ldy + n] = fmaf((float)a, sc, p.bias ? __ldg(p.bias + n) : 0.0f);
-            if (p.acc_out) p.acc_out[orow * p.ldy + n] = a;
-          }
-        }
-      }
-    }
     tc_fence_before();
   }
 
@@ -484,6 +481,46 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     tmem_dealloc(tmem_base, BN);
   }
   if (threadIdx.x == 0 && *abort_flag) flag(p.dev_status, OCS_DEV_TIMEOUT);
+}
+
+// Sums the K slices' partial accumulators (integer sums: exact in any order) and applies the epilogue.
+// Thread = 4 consecutive columns of one output row when N % 4 == 0, else one element.
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long rows, int N,
+                     const float* __restrict__ a_scale, const float* __restrict__ w_scale,
+                     const float* __restrict__ bias, float* __restrict__ Y, long long ldy, int32_t* __restrict__ acc_out) {
+  const float sc = __fmul_rn(__ldg(a_scale), __ldg(w_scale));
+  const long long slice = rows * (long long)N;
+  const int per_row = VEC ? (N >> 2) : N;
+  const long long total = rows * per_row;
+  for (long long t = blockIdx.x * 256ll + threadIdx.x; t < total; t += (long long)gridDim.x * 256) {
+    const long long row = t / per_row;
+    const int n = (int)(t - row * per_row) * (VEC ? 4 : 1);
+    const int32_t* p = part + row * N + n;
+    if (VEC) {
+      int4 a = __ldcg(reinterpret_cast<const int4*>(p));
+#pragma unroll 4
+      for (int z = 1; z < split_k; ++z) {
+        const int4 b = __ldcg(reinterpret_cast<const int4*>(p + z * slice));
+        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+      }
+      float* y = Y + row * ldy + n;
+      y[0] = fmaf((float)a.x, sc, bias ? __ldg(bias + n + 0) : 0.0f);
+      y[1] = fmaf((float)a.y, sc, bias ? __ldg(bias + n + 1) : 0.0f);
+      y[2] = fmaf((float)a.z, sc, bias ? __ldg(bias + n + 2) : 0.0f);
+      y[3] = fmaf((float)a.w, sc, bias ? __ldg(bias + n + 3) : 0.0f);
+      if (acc_out) {
+        int32_t* ao = acc_out + row * ldy + n;
+        ao[0] = a.x; ao[1] = a.y; ao[2] = a.z; ao[3] = a.w;
+      }
+    } else {
+      int a = __ldcg(p);
+      for (int z = 1; z < split_k; ++z) a += __ldcg(p + z * slice);
+      Y[row * ldy + n] = fmaf((float)a, sc, bias ? __ldg(bias + n) : 0.0f);
+      if (acc_out) acc_out[row * ldy + n] = a;
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------------ host
@@ -563,11 +600,10 @@ ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const Gem
 
 struct GemmWs {
   int32_t* acc_ws;
-  unsigned int* counters;
   size_t total;
 };
 
-GemmWs carve_gemm_ws(void* ws, long long rows, int N, long long m_tiles, int split_k) {
+GemmWs carve_gemm_ws(void* ws, long long rows, int N, int split_k) {
   GemmWs w{};
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -576,7 +612,6 @@ GemmWs carve_gemm_ws(void* ws, long long rows, int N, long long m_tiles, int spl
     return q;
   };
   w.acc_ws = reinterpret_cast<int32_t*>(take(4 * (size_t)split_k * (size_t)rows * (size_t)N));
-  w.counters = reinterpret_cast<unsigned int*>(take(4 * (size_t)m_tiles * (size_t)((N + 63) / 64)));
   w.total = off;
   return w;
 }
@@ -600,18 +635,28 @@ ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long lo
 
   p.out_rows = out_rows;
   if (plan.split_k > 1) {
-    const GemmWs w = carve_gemm_ws(ws, out_rows, p.N, m_tiles, plan.split_k);
+    const GemmWs w = carve_gemm_ws(ws, out_rows, p.N, plan.split_k);
     if (!ws || !aligned(ws, 256) || ws_bytes < w.total) return OCS_ERR_WORKSPACE;
     p.acc_ws = w.acc_ws;
-    p.tile_counters = w.counters;
-    if (cudaMemsetAsync(w.counters, 0, 4 * (size_t)m_tiles * (size_t)((p.N + 63) / 64), stream) != cudaSuccess)
-      return OCS_ERR_CUDA;
   }
+  ocs_status st;
   switch (plan.BN) {
-    case 256: return launch_gemm<256>(tmB, tmA, p, plan, stream);
-    case 128: return launch_gemm<128>(tmB, tmA, p, plan, stream);
-    default: return launch_gemm<64>(tmB, tmA, p, plan, stream);
+    case 256: st = launch_gemm<256>(tmB, tmA, p, plan, stream); break;
+    case 128: st = launch_gemm<128>(tmB, tmA, p, plan, stream); break;
+    default: st = launch_gemm<64>(tmB, tmA, p, plan, stream); break;
   }
+  if (st != OCS_OK || plan.split_k == 1) return st;
+  const bool vec = (p.N % 4 == 0);
+  const long long work = out_rows * (long long)(vec ? p.N / 4 : p.N);
+  const int grid = (int)min((work + 255) / 256, (long long)kNumSMs * 8);
+  LaunchScope ls("splitk_reduce_kernel", stream);
+  if (vec)
+    splitk_reduce_kernel<true><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
+                                                         p.bias, p.Y, p.ldy, p.acc_out);
+  else
+    splitk_reduce_kernel<false><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
+                                                          p.bias, p.Y, p.ldy, p.acc_out);
+  return launch_status();
 }
 
 // M-tile box for the convolution: the (bw, bh, bn) with bw*bh*bn <= 128 that needs the fewest tiles.
@@ -660,7 +705,7 @@ extern "C" size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S) {
   const int m_tiles = (M + BM - 1) / BM;
   const GemmPlan plan = choose_plan(m_tiles, N, (int)(((long long)C + S + BK - 1) / BK));
   if (plan.split_k == 1) return 256;
-  return carve_gemm_ws(nullptr, M, N, m_tiles, plan.split_k).total;
+  return carve_gemm_ws(nullptr, M, N, plan.split_k).total;
 }
 
 extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C, int64_t lda,
@@ -744,7 +789,7 @@ extern "C" size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O,
   const long long Ktot = (long long)kh * kw * ((long long)C + S);
   const GemmPlan plan = choose_plan((int)g.m_tiles, O, (int)((Ktot + BK - 1) / BK));
   if (plan.split_k == 1) return 256;
-  return carve_gemm_ws(nullptr, g.out_rows, O, g.m_tiles, plan.split_k).total;
+  return carve_gemm_ws(nullptr, g.out_rows, O, plan.split_k).total;
 }
 
 extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H, int Wd, int C,

@@ -5,8 +5,8 @@
 //   maxabs_kernel     max|x|, combined with atomicMax on the bits of the non-negative value
 //   hist_kernel       histogram of |x| in privatised shared-memory counters, flushed with 64-bit atomics
 //   score_kernel      one CTA per candidate threshold: sum_b h[b]*(x_b - Q(x_b))^2 in double
-//   pick_kernel       smallest score, ties to the largest threshold
-//   quantize_kernel   code = clamp(rint(x * L/alpha)), round-half-to-even, saturating
+//   quantize_kernel   picks the winning threshold (smallest score, ties to the largest threshold), then
+//                     code = clamp(rint(x * L/alpha)), round-half-to-even, saturating
 #include "common.cuh"
 
 namespace ocs {
@@ -40,8 +40,13 @@ View make_view(const float* T, int64_t rows, int64_t cols, int64_t ld) {
   return v;
 }
 
-int grid_for(long long tiles) {
-  const long long cap = (long long)kNumSMs * 8;
+// Grid of a tile-strided kernel: one resident wave at most.
+template <typename K>
+int grid_for(K kernel, long long tiles, size_t dyn_smem = 0) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, dyn_smem) != cudaSuccess || per_sm < 1)
+    per_sm = 4;
+  const long long cap = (long long)kNumSMs * per_sm;
   return (int)(tiles < cap ? (tiles > 0 ? tiles : 1) : cap);
 }
 
@@ -156,25 +161,40 @@ score_kernel(const unsigned long long* __restrict__ hist, const float* __restric
   if (threadIdx.x == 0) scores[blockIdx.x] = red[0];
 }
 
-__global__ void pick_kernel(const double* __restrict__ scores, const float* __restrict__ maxp, int n_candidates,
-                            float* __restrict__ alpha_sel) {
-  if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  const float m = *maxp;
-  if (!(m > 0.0f)) { *alpha_sel = 0.0f; return; }
-  int best = 1;
-  double bs = scores[0];
-  for (int c = 2; c <= n_candidates; ++c) {
-    const double s = scores[c - 1];
-    if (s <= bs) { bs = s; best = c; }  // ties to the largest threshold
+// The search's winner: smallest score, ties to the largest threshold.  Every CTA of the quantize
+// kernel evaluates it (n_candidates doubles) instead of a separate single-thread launch.
+__device__ float pick_alpha(const double* __restrict__ scores, float m, int n_candidates) {
+  __shared__ double s_best[8];
+  __shared__ int c_best[8];
+  double bs = INFINITY;
+  int bc = 0;
+  for (int c = threadIdx.x + 1; c <= n_candidates; c += 256) {
+    const double v = scores[c - 1];
+    if (v < bs || (v == bs && c > bc)) { bs = v; bc = c; }
   }
-  *alpha_sel = __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)best), (double)n_candidates));
+  for (int o = 16; o > 0; o >>= 1) {
+    const double v = __shfl_xor_sync(0xffffffffu, bs, o);
+    const int c = __shfl_xor_sync(0xffffffffu, bc, o);
+    if (c != 0 && (bc == 0 || v < bs || (v == bs && c > bc))) { bs = v; bc = c; }
+  }
+  if ((threadIdx.x & 31) == 0) { s_best[threadIdx.x >> 5] = bs; c_best[threadIdx.x >> 5] = bc; }
+  __syncthreads();
+  bs = s_best[0]; bc = c_best[0];
+  for (int w = 1; w < 8; ++w) {
+    const double v = s_best[w];
+    const int c = c_best[w];
+    if (c != 0 && (bc == 0 || v < bs || (v == bs && c > bc))) { bs = v; bc = c; }
+  }
+  return __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)bc), (double)n_candidates));
 }
 
 __global__ void __launch_bounds__(256)
-quantize_kernel(View v, const float* __restrict__ alpha_p, int L, int is_signed, int8_t* __restrict__ codes,
-                long long ld_codes, int packed_ok, float* __restrict__ scale_out, float* __restrict__ alpha_out,
-                int* dev_status) {
-  const float alpha = *alpha_p;
+quantize_kernel(View v, const float* __restrict__ alpha_p, const double* __restrict__ scores, int n_candidates, int L,
+                int is_signed, int8_t* __restrict__ codes, long long ld_codes, int packed_ok,
+                float* __restrict__ scale_out, float* __restrict__ alpha_out, int* dev_status) {
+  // alpha_p holds max|T|; with scores given the threshold is the search's winner
+  float alpha = *alpha_p;
+  if (scores && alpha > 0.0f) alpha = pick_alpha(scores, alpha, n_candidates);
   const bool zero = !(alpha > 0.0f);
   const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)L);
   const float inv = zero ? 0.0f : __fdiv_rn((float)L, alpha);
@@ -215,7 +235,6 @@ quantize_kernel(View v, const float* __restrict__ alpha_p, int L, int is_signed,
 
 struct QuantWs {
   unsigned int* maxbits;       // fp32 bits of max|T|
-  float* alpha_sel;
   unsigned long long* hist;
   double* scores;
   size_t total;
@@ -230,7 +249,6 @@ QuantWs carve_quant_ws(void* ws, int n_bins, int n_candidates) {
     return p;
   };
   w.maxbits = reinterpret_cast<unsigned int*>(take(256));
-  w.alpha_sel = reinterpret_cast<float*>(take(256));
   w.hist = reinterpret_cast<unsigned long long*>(take(8 * (size_t)(n_bins > 0 ? n_bins : 1)));
   w.scores = reinterpret_cast<double*>(take(8 * (size_t)(n_candidates > 0 ? n_candidates : 1)));
   w.total = off;
@@ -272,23 +290,23 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   if (st != OCS_OK) return st;
 
   const View v = make_view(T, rows, cols, ld_in);
-  const int grid = grid_for(v.tiles);
   const int L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
 
   const float* maxp = max_abs_in;
   if (!maxp) {
     if (cudaMemsetAsync(w.maxbits, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
     LaunchScope ls("maxabs_kernel", stream);
-    maxabs_kernel<<<grid, 256, 0, stream>>>(v, w.maxbits);
+    maxabs_kernel<<<grid_for(maxabs_kernel, v.tiles), 256, 0, stream>>>(v, w.maxbits);
     if ((st = launch_status()) != OCS_OK) return st;
     maxp = reinterpret_cast<const float*>(w.maxbits);
   }
-  const float* alpha_p = maxp;
+  const double* scores = nullptr;
   if (mode == OCS_CLIP_MSE) {
     if (cudaMemsetAsync(w.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
     {
+      const size_t smem = sizeof(unsigned int) * kHistCopies * n_bins;
       LaunchScope ls("hist_kernel", stream);
-      hist_kernel<<<grid, 256, sizeof(unsigned int) * kHistCopies * n_bins, stream>>>(v, maxp, n_bins, w.hist);
+      hist_kernel<<<grid_for(hist_kernel, v.tiles, smem), 256, smem, stream>>>(v, maxp, n_bins, w.hist);
     }
     if ((st = launch_status()) != OCS_OK) return st;
     {
@@ -296,12 +314,7 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
       score_kernel<<<n_candidates, 256, 0, stream>>>(w.hist, maxp, n_bins, n_candidates, L, is_signed, w.scores);
     }
     if ((st = launch_status()) != OCS_OK) return st;
-    {
-      LaunchScope ls("pick_kernel", stream);
-      pick_kernel<<<1, 32, 0, stream>>>(w.scores, maxp, n_candidates, w.alpha_sel);
-    }
-    if ((st = launch_status()) != OCS_OK) return st;
-    alpha_p = w.alpha_sel;
+    scores = w.scores;
   }
   // the dense view addresses codes by flat index; that is only valid when the codes are dense too
   View vq = v;
@@ -316,7 +329,8 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   }
   const int packed_ok = aligned(codes, 4) && (ldc % 4 == 0);
   LaunchScope ls("quantize_kernel", stream);
-  quantize_kernel<<<grid_for(vq.tiles), 256, 0, stream>>>(vq, alpha_p, L, is_signed, codes, ldc, packed_ok, scale,
-                                                         alpha, dev_status);
+  quantize_kernel<<<grid_for(quantize_kernel, vq.tiles), 256, 0, stream>>>(vq, maxp, scores, n_candidates, L, is_signed,
+                                                                          codes, ldc, packed_ok, scale, alpha,
+                                                                          dev_status);
   return launch_status();
 }

@@ -6,61 +6,86 @@
 //                        combined across CTAs with integer atomics on order-preserving bits.
 //   split_plan_kernel    the greedy loop of Section 3.4 run on channel extrema only.  Both halves
 //                        of a split are monotone in w, so a copy's extrema are the images of its
-//                        parent's extrema and the whole loop needs no further pass over W.
-//   split_scatter_kernel one streaming pass that writes W' = path(W[:, idx_map[j], :]).
+//                        parent's extrema and the whole loop needs no further pass over W.  The
+//                        dependent steps are grouped into rounds whose members are independent.
+//   split_rows_kernel    one streaming pass that writes W' = path(W[:, idx_map[j], :]): whole rows staged
+//                        in shared memory by bulk copies, duplicated channels gathered there
+//   split_scatter_kernel the same pass with plain loads and stores, for shapes the bulk copies
+//                        cannot serve (rows longer than the buffers, unaligned rows)
 #include "common.cuh"
 
 namespace ocs {
 namespace {
 
 constexpr int kPlanThreads = 1024;
-constexpr int kPlanSmemSplits = 4096;  // up to this many splits the plan's queues live in shared memory
+constexpr int kPlanSmemSplits = 3072;  // up to this many splits the plan's live set lives in shared memory
+constexpr int kPlanSmemBytes = 220 * 1024;  // dynamic shared memory the plan kernel may use
+constexpr size_t kRowSmemBytes = 226 * 1024;       // shared memory the bulk-copy scatter may use (two row-group buffers)
 constexpr int kMaxHalvings = 320;      // 2^-320 * any finite fp32 is zero: deeper plain halvings change nothing
 
 __device__ __forceinline__ float split_keep(float w, float d) { return __fmul_rn(__fsub_rn(w, d), 0.5f); }
 __device__ __forceinline__ float split_new(float w, float d) { return __fmul_rn(__fadd_rn(w, d), 0.5f); }
 
 // ------------------------------------------------------------------------------------------------
+// Work partition of the two streaming kernels: the matrix is cut into column blocks of 1024
+// columns (a thread owns 4 consecutive columns); the (column block, row) pairs are numbered
+// column-block-major and every CTA of a grid sized to one resident wave takes one contiguous
+// range of them, so all CTAs stream the same number of rows (to within one).
+__device__ __forceinline__ void cta_range(long long total, long long* u0, long long* u1) {
+  *u0 = total * (long long)blockIdx.x / (long long)gridDim.x;
+  *u1 = total * ((long long)blockIdx.x + 1) / (long long)gridDim.x;
+}
+
 // K1: per-column signed extrema of a row-major [O][ncols] fp32 matrix.
 template <bool VEC>
 __global__ void __launch_bounds__(256)
-col_minmax_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, int rows_per_cta,
-                  uint32_t* __restrict__ colmin, uint32_t* __restrict__ colmax, int* dev_status) {
-  const int col0 = (blockIdx.x * 256 + threadIdx.x) * 4;
-  if (col0 >= ncols) return;
-  const int r0 = blockIdx.y * rows_per_cta;
-  const int r1 = min(O, r0 + rows_per_cta);
-  float mn[4], mx[4];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) { mn[c] = INFINITY; mx[c] = -INFINITY; }
+col_minmax_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
+                  uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map, int32_t* __restrict__ depth,
+                  unsigned long long* __restrict__ bits, int* dev_status) {
+  // identity part of the plan's outputs: original channel c maps to itself and has no split yet
+  for (int c = blockIdx.x * 256 + threadIdx.x; c < C; c += gridDim.x * 256) {
+    idx_map[c] = c; depth[c] = 0; bits[c] = 0ull;
+  }
+  const int col_blocks = (ncols + 1023) / 1024;
+  long long u, u1;
+  cta_range((long long)col_blocks * O, &u, &u1);
   bool bad = false;
-  if (VEC && col0 + 3 < ncols) {
-    const float4* p = reinterpret_cast<const float4*>(W + (int64_t)r0 * ld + col0);
-    const int64_t stride = ld >> 2;
-#pragma unroll 8
-    for (int r = r0; r < r1; ++r) {
-      const float4 v = __ldcs(p);
-      p += stride;
-      mn[0] = fminf(mn[0], v.x); mx[0] = fmaxf(mx[0], v.x);
-      mn[1] = fminf(mn[1], v.y); mx[1] = fmaxf(mx[1], v.y);
-      mn[2] = fminf(mn[2], v.z); mx[2] = fmaxf(mx[2], v.z);
-      mn[3] = fminf(mn[3], v.w); mx[3] = fmaxf(mx[3], v.w);
-      bad |= !(is_finite(v.x) && is_finite(v.y) && is_finite(v.z) && is_finite(v.w));
-    }
-  } else {
-    for (int r = r0; r < r1; ++r) {
+  while (u < u1) {
+    const int cb = (int)(u / O);
+    const int r0 = (int)(u - (long long)cb * O);
+    const int r1 = (int)min((long long)O, r0 + (u1 - u));
+    u += r1 - r0;
+    const int col0 = (cb * 256 + threadIdx.x) * 4;
+    if (col0 >= ncols) continue;
+    float mn[4], mx[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        if (col0 + c < ncols) {
-          const float v = __ldcs(W + (int64_t)r * ld + col0 + c);
-          mn[c] = fminf(mn[c], v);
-          mx[c] = fmaxf(mx[c], v);
-          bad |= !is_finite(v);
+    for (int c = 0; c < 4; ++c) { mn[c] = INFINITY; mx[c] = -INFINITY; }
+    if (VEC && col0 + 3 < ncols) {
+      const float4* p = reinterpret_cast<const float4*>(W + (int64_t)r0 * ld + col0);
+      const int64_t stride = ld >> 2;
+#pragma unroll 8
+      for (int r = r0; r < r1; ++r) {
+        const float4 v = __ldcs(p);
+        p += stride;
+        mn[0] = fminf(mn[0], v.x); mx[0] = fmaxf(mx[0], v.x);
+        mn[1] = fminf(mn[1], v.y); mx[1] = fmaxf(mx[1], v.y);
+        mn[2] = fminf(mn[2], v.z); mx[2] = fmaxf(mx[2], v.z);
+        mn[3] = fminf(mn[3], v.w); mx[3] = fmaxf(mx[3], v.w);
+        bad |= !(is_finite(v.x) && is_finite(v.y) && is_finite(v.z) && is_finite(v.w));
+      }
+    } else {
+      for (int r = r0; r < r1; ++r) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (col0 + c < ncols) {
+            const float v = __ldcs(W + (int64_t)r * ld + col0 + c);
+            mn[c] = fminf(mn[c], v);
+            mx[c] = fmaxf(mx[c], v);
+            bad |= !is_finite(v);
+          }
         }
       }
     }
-  }
-  if (r1 > r0) {
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       if (col0 + c < ncols) {
@@ -73,13 +98,23 @@ col_minmax_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, int
 }
 
 // ------------------------------------------------------------------------------------------------
-// K2: the greedy loop on channel extrema.
+// K2: the greedy loop of Section 3.4 on channel extrema, in rounds.
 //
 // A live channel is (expanded index j, min, max).  Its priority is the 64-bit word
-// (bits(max(|min|,|max|)) << 32) | (0xFFFFFFFF - j): larger word = larger |w|, ties broken toward the
-// smallest current index.  Only the S largest original channels can ever be chosen (before every
-// step at least one of them is still untouched and it outranks every other original), so they
-// are selected and sorted once; copies created by splits go to a binary heap.
+// (bits(max(|min|,|max|)) << 32) | (0xFFFFFFFF - j): a larger word is a larger |w|, ties broken
+// toward the smallest current index -- the order in which the one-at-a-time loop picks channels.
+// Only the min(S, C) highest-priority original channels can ever be picked (before every step at
+// least one of them is untouched and outranks every other original), so they are selected once
+// (radix select) and form the initial live set.
+//
+// One round: let kmax be the largest live key and B = fl(fl(kmax + d) * 0.5), an upper bound on
+// the key of any child of any live channel.  Every live channel whose key is strictly above B is
+// picked before any child created from now on, and before every live channel at or below B; so
+// the next steps of the one-at-a-time loop are exactly those channels in priority order.  The
+// round sorts them (bitonic, shared memory), assigns step numbers base + rank, and performs all
+// their splits in parallel.  The top channel itself always joins the batch, so a round makes at
+// least one step even when d >= kmax or all keys are zero.  Typical tensors need a handful of
+// rounds (each halves the largest key), instead of S dependent steps.
 
 struct PlanArgs {
   const uint32_t* colmin;  // [C*R] order-preserving bits
@@ -87,24 +122,26 @@ struct PlanArgs {
   int C, R, S;
   float qa_step;
   int qa_bits;
-  float* chmin;  // [C]
-  float* chmax;  // [C]
-  float* chkey;  // [C]
-  int32_t* idx_map;       // [C+S]
+  float* chmin;  // [C+S] current extrema of the selected originals and of every channel a split creates
+  float* chmax;
+  float* chkey;  // [C] keys, used when they do not fit in shared memory
+  int32_t* idx_map;       // [C+S]  (entries below C are written by the extrema kernel)
   int32_t* split_order;   // [S] or null
   int32_t* depth;         // [C+S]
   unsigned long long* bits;  // [C+S]
   float* max_abs_out;     // [3] or null
   float* qa_step_dev;     // [1] step actually used (read by the scatter kernel)
-  // queues for S > kPlanSmemSplits
-  unsigned long long* g_sorted;
-  float* g_omin;
-  float* g_omax;
-  unsigned long long* g_hcomp;
-  float* g_hmin;
-  float* g_hmax;
+  int32_t* touched;       // [min(S, C)] original channels that were split at least once
+  int* n_touched;         // [1]
+  unsigned long long* g_buf;  // sel | live0 | live1 | batch in global memory, used when S > kPlanSmemSplits
+  int cap, npad, Sp;      // live capacity Sp + S, sort capacity (power of two >= cap), min(S, C)
+  int hist_off, keys_off; // byte offsets in dynamic shared memory: selection histograms; keys (-1: chkey)
   int* dev_status;
 };
+
+constexpr int kSelBins = 2048;    // bins of one selection level
+constexpr int kSelCopies = 8;     // private histogram copies (one per four warps)
+constexpr int kSelHistBytes = kSelBins * kSelCopies * 4;
 
 __device__ __forceinline__ unsigned long long make_prio(float key, int j) {
   return ((unsigned long long)__float_as_uint(key) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)j);
@@ -112,247 +149,363 @@ __device__ __forceinline__ unsigned long long make_prio(float key, int j) {
 __device__ __forceinline__ float prio_key(unsigned long long p) { return __uint_as_float((uint32_t)(p >> 32)); }
 __device__ __forceinline__ int prio_index(unsigned long long p) { return (int)(0xFFFFFFFFu - (uint32_t)p); }
 
-struct Heap {
-  unsigned long long* comp;
-  float* mn;
-  float* mx;
-  int n;
-  __device__ void sift_up(int i, unsigned long long c, float a, float b) {
-    while (i > 0) {
-      const int parent = (i - 1) >> 1;
-      const unsigned long long pc = comp[parent];
-      if (pc >= c) break;
-      comp[i] = pc; mn[i] = mn[parent]; mx[i] = mx[parent];
-      i = parent;
-    }
-    comp[i] = c; mn[i] = a; mx[i] = b;
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o);
+    v = t > v ? t : v;
   }
-  __device__ void push(unsigned long long c, float a, float b) { sift_up(n++, c, a, b); }
-  __device__ void replace_top(unsigned long long c, float a, float b) {
-    int i = 0;
-    for (;;) {
-      int l = 2 * i + 1;
-      if (l >= n) break;
-      unsigned long long lc = comp[l];
-      if (l + 1 < n) {
-        const unsigned long long rc = comp[l + 1];
-        if (rc > lc) { lc = rc; ++l; }
-      }
-      if (lc <= c) break;
-      comp[i] = lc; mn[i] = mn[l]; mx[i] = mx[l];
-      i = l;
-    }
-    comp[i] = c; mn[i] = a; mx[i] = b;
-  }
+  return v;
+}
+
+struct PlanShared {
+  unsigned long long red[32];
+  unsigned long long scan[32];
+  unsigned int digit, count;
+  int n_batch, n_next;
+  int n_touched;
+  int bad;
 };
 
-// One run of the S greedy steps by a single thread.  Returns max|W'| after the last step.
-__device__ float greedy_run(const PlanArgs& a, const unsigned long long* sorted, const float* omin,
-                            const float* omax, int Sp, Heap heap, float d, float rest_max, bool write) {
-  int p = 0;
-  heap.n = 0;
-  for (int s = 0; s < a.S; ++s) {
-    const unsigned long long co = p < Sp ? sorted[p] : 0ull;
-    const unsigned long long ch = heap.n > 0 ? heap.comp[0] : 0ull;
-    const bool from_heap = !(p < Sp && co >= ch);
-    int j, src, dep;
-    unsigned long long bt;
-    float mn, mx;
-    if (!from_heap) {
-      j = prio_index(co); src = j; dep = 0; bt = 0ull;
-      mn = omin[p]; mx = omax[p];
-      ++p;
-    } else {
-      j = prio_index(ch);
-      mn = heap.mn[0]; mx = heap.mx[0];
-      if (write) { src = a.idx_map[j]; dep = a.depth[j]; bt = a.bits[j]; } else { src = 0; dep = 0; bt = 0ull; }
-    }
-    const int jn = a.C + s;
-    const float amn = split_keep(mn, d), amx = split_keep(mx, d);
-    const float bmn = split_new(mn, d), bmx = split_new(mx, d);
-    if (write) {
-      if (dep >= 63 && d != 0.0f) flag(a.dev_status, OCS_DEV_DEPTH);
-      const unsigned long long nb = dep < 64 ? (bt | (1ull << dep)) : bt;
-      a.idx_map[jn] = src;
-      if (a.split_order) a.split_order[s] = j;
-      a.depth[j] = dep + 1;   // bits[j] unchanged: the kept copy's new step is a 0 bit
-      a.depth[jn] = dep + 1;
-      a.bits[jn] = nb;
-      if (!from_heap) a.bits[j] = 0ull;
-    }
-    const unsigned long long ca = make_prio(fmaxf(fabsf(amn), fabsf(amx)), j);
-    const unsigned long long cb = make_prio(fmaxf(fabsf(bmn), fabsf(bmx)), jn);
-    if (from_heap) heap.replace_top(ca, amn, amx); else heap.push(ca, amn, amx);
-    heap.push(cb, bmn, bmx);
+// Largest of the threads' words over the whole CTA, returned to every thread.
+__device__ unsigned long long block_max_u64(unsigned long long m, unsigned long long* red) {
+  m = warp_max_u64(m);
+  __syncthreads();  // red may still be read by the previous call
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  return warp_max_u64(red[threadIdx.x & 31]);
+}
+
+// Exclusive prefix sum of v over the CTA in thread order (both 32-bit halves of v are summed
+// independently as long as neither overflows); *total receives the sum over all threads.
+__device__ unsigned long long block_excl_scan(unsigned long long v, unsigned long long* scan,
+                                              unsigned long long* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned long long incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
   }
-  float m = rest_max;
-  if (p < Sp) m = fmaxf(m, prio_key(sorted[p]));
-  // the heap's top has the largest key among the copies
-  if (heap.n > 0) m = fmaxf(m, prio_key(heap.comp[0]));
-  return m;
+  __syncthreads();  // scan may still be read by the previous call
+  if (lane == 31) scan[warp] = incl;
+  __syncthreads();
+  unsigned long long w = scan[lane];
+  unsigned long long wincl = w;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long t = __shfl_up_sync(0xffffffffu, wincl, o);
+    if (lane >= o) wincl += t;
+  }
+  *total = __shfl_sync(0xffffffffu, wincl, 31);
+  const unsigned long long warp_base = __shfl_sync(0xffffffffu, wincl - w, warp);
+  return warp_base + incl - v;
+}
+
+// One compare-exchange of a descending bitonic network on a[0..): pair number t of stage (k, jj).
+__device__ __forceinline__ void bitonic_pair(unsigned long long* a, int t, int k, int jj) {
+  const int i = ((t & ~(jj - 1)) << 1) | (t & (jj - 1));
+  const int ixj = i | jj;
+  const unsigned long long x = a[i], y = a[ixj];
+  const bool desc = (i & k) == 0;
+  if (desc ? (x < y) : (x > y)) { a[i] = y; a[ixj] = x; }
+}
+
+// Sorts a[0..npad) descending; npad a power of two >= 2.  Every warp owns a contiguous chunk:
+// stages whose partners lie inside one chunk need only a warp barrier.  Ends with a CTA barrier.
+__device__ void bitonic_sort_desc(unsigned long long* a, int npad) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int chunk = max(64, npad / (kPlanThreads / 32));   // elements per warp
+  const int warps_used = max(1, npad / chunk);
+  const int local_n = min(chunk, npad);
+  unsigned long long* mine = a + (size_t)warp * chunk;
+  for (int k = 2; k <= npad; k <<= 1) {
+    int jj = k >> 1;
+    for (; jj >= chunk; jj >>= 1) {                       // partners in different chunks
+      for (int t = threadIdx.x; t < (npad >> 1); t += kPlanThreads) bitonic_pair(a, t, k, jj);
+      __syncthreads();
+    }
+    if (warp < warps_used) {
+      for (; jj > 0; jj >>= 1) {                          // partners inside this warp's chunk
+        for (int t = lane; t < (local_n >> 1); t += 32) {
+          const int i = ((t & ~(jj - 1)) << 1) | (t & (jj - 1));
+          const int gi = warp * chunk + i;                // the direction depends on the global index
+          const unsigned long long x = mine[i], y = mine[i | jj];
+          const bool desc = (gi & k) == 0;
+          if (desc ? (x < y) : (x > y)) { mine[i] = y; mine[i | jj] = x; }
+        }
+        __syncwarp();
+      }
+    }
+    if (k >= chunk) __syncthreads();                      // the next cross-chunk stage reads other chunks
+  }
+  __syncthreads();
+}
+
+// Runs the S greedy steps in rounds on the live set `live` (n_live entries).  With write = false
+// (plain halving, d = 0) only keys are tracked: both children of key k have key fl(k * 0.5).
+// Returns the largest key among the live channels after the last step.
+__device__ float greedy_rounds(const PlanArgs& a, PlanShared& sh, unsigned long long* live, unsigned long long* next,
+                               unsigned long long* batch, int n_live, float d, bool write) {
+  const int tid = threadIdx.x, lane = threadIdx.x & 31;
+  const unsigned int lt = (1u << lane) - 1u;
+  int base = 0;
+  while (base < a.S) {
+    unsigned long long m = 0ull;
+    for (int i = tid; i < n_live; i += kPlanThreads) m = live[i] > m ? live[i] : m;
+    const unsigned long long pmax = block_max_u64(m, sh.red);
+    const float bound = __fmul_rn(__fadd_rn(prio_key(pmax), d), 0.5f);
+    if (tid == 0) { sh.n_batch = 0; sh.n_next = 0; }
+    __syncthreads();
+    for (int i0 = 0; i0 < n_live; i0 += kPlanThreads) {   // whole warps iterate together
+      const int i = i0 + tid;
+      const unsigned long long p = i < n_live ? live[i] : 0ull;
+      const bool in_batch = i < n_live && (prio_key(p) > bound || p == pmax);
+      const bool in_next = i < n_live && !in_batch;
+      const unsigned int mb = __ballot_sync(0xffffffffu, in_batch), mn = __ballot_sync(0xffffffffu, in_next);
+      int bb = 0, nn = 0;
+      if (lane == 0) {
+        if (mb) bb = atomicAdd(&sh.n_batch, __popc(mb));
+        if (mn) nn = atomicAdd(&sh.n_next, __popc(mn));
+      }
+      bb = __shfl_sync(0xffffffffu, bb, 0);
+      nn = __shfl_sync(0xffffffffu, nn, 0);
+      if (in_batch) batch[bb + __popc(mb & lt)] = p;
+      if (in_next) next[nn + __popc(mn & lt)] = p;
+    }
+    __syncthreads();
+    const int nb = sh.n_batch, n_keep = sh.n_next;
+    int npad = 1;
+    while (npad < nb) npad <<= 1;
+    for (int i = nb + tid; i < npad; i += kPlanThreads) batch[i] = 0ull;  // below every real priority word
+    __syncthreads();
+    if (npad > 1) bitonic_sort_desc(batch, npad);
+    const int take = min(nb, a.S - base);
+    // rank i < take performs step base + i; its children go to next[n_keep + 2i, +1]; channels
+    // beyond `take` (the last round only) stay live unchanged
+    for (int i0 = 0; i0 < nb; i0 += kPlanThreads) {
+      const int i = i0 + tid;
+      const bool act = i < nb;
+      const unsigned long long p = act ? batch[i] : 0ull;
+      bool first = false;
+      int j = 0;
+      if (act && i >= take) next[n_keep + 2 * take + (i - take)] = p;
+      if (act && i < take) {
+        j = prio_index(p);
+        const int s = base + i;
+        const int jn = a.C + s;
+        unsigned long long ca, cb;
+        if (write) {
+          const float mn = a.chmin[j], mx = a.chmax[j];
+          const float amn = split_keep(mn, d), amx = split_keep(mx, d);
+          const float bmn = split_new(mn, d), bmx = split_new(mx, d);
+          const int dep = a.depth[j];
+          const unsigned long long bt = a.bits[j];
+          if (dep >= 63 && d != 0.0f) flag(a.dev_status, OCS_DEV_DEPTH);
+          first = dep == 0;   // an original channel's first split
+          a.chmin[j] = amn; a.chmax[j] = amx;
+          a.chmin[jn] = bmn; a.chmax[jn] = bmx;
+          a.idx_map[jn] = a.idx_map[j];
+          if (a.split_order) a.split_order[s] = j;
+          a.depth[j] = dep + 1;   // bits[j] unchanged: the kept copy's new step is a 0 bit
+          a.depth[jn] = dep + 1;
+          a.bits[jn] = dep < 64 ? (bt | (1ull << dep)) : bt;
+          ca = make_prio(fmaxf(fabsf(amn), fabsf(amx)), j);
+          cb = make_prio(fmaxf(fabsf(bmn), fabsf(bmx)), jn);
+        } else {
+          const float half = __fmul_rn(prio_key(p), 0.5f);
+          ca = make_prio(half, j);
+          cb = make_prio(half, jn);
+        }
+        next[n_keep + 2 * i] = ca;
+        next[n_keep + 2 * i + 1] = cb;
+      }
+      const unsigned int mf = __ballot_sync(0xffffffffu, first);
+      if (mf) {
+        int tb = 0;
+        if (lane == 0) tb = atomicAdd(&sh.n_touched, __popc(mf));
+        tb = __shfl_sync(0xffffffffu, tb, 0);
+        if (first) a.touched[tb + __popc(mf & lt)] = j;
+      }
+    }
+    __syncthreads();
+    n_live = n_keep + nb + take;
+    base += take;
+    unsigned long long* t = live; live = next; next = t;
+  }
+  unsigned long long m = 0ull;
+  for (int i = tid; i < n_live; i += kPlanThreads) m = live[i] > m ? live[i] : m;
+  return prio_key(block_max_u64(m, sh.red));
 }
 
 __global__ void __launch_bounds__(kPlanThreads, 1) split_plan_kernel(PlanArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ unsigned int hist[256];
-  __shared__ float red[kPlanThreads / 32];
-  __shared__ unsigned long long sh_thresh;
-  __shared__ unsigned int sh_count;
-  __shared__ float sh_maxw, sh_rest;
-  __shared__ int sh_bad;
+  __shared__ PlanShared sh;
 
   const int tid = threadIdx.x;
-  const int C = a.C, R = a.R, S = a.S;
-  const int Sp = min(S, C);
-  int npad = 1;
-  while (npad < Sp) npad <<= 1;
+  const int C = a.C, R = a.R, S = a.S, Sp = a.Sp;
+  unsigned long long* buf = (S <= kPlanSmemSplits) ? reinterpret_cast<unsigned long long*>(smem_raw) : a.g_buf;
+  unsigned long long* sel = buf;                 // [Sp]   the selected originals
+  unsigned long long* live0 = sel + Sp;          // [cap]
+  unsigned long long* live1 = live0 + a.cap;     // [cap]
+  unsigned long long* batch = live1 + a.cap;     // [npad]
+  // during the selection the space behind sel holds the histograms and (when they fit) the keys
+  unsigned int* hist = reinterpret_cast<unsigned int*>(smem_raw + a.hist_off);
+  float* keys = a.keys_off >= 0 ? reinterpret_cast<float*>(smem_raw + a.keys_off) : a.chkey;
+  const uint32_t* __restrict__ colmin = a.colmin;
+  const uint32_t* __restrict__ colmax = a.colmax;
 
-  unsigned long long* sorted;
-  float *omin, *omax;
-  Heap heap;
-  if (S <= kPlanSmemSplits) {
-    unsigned char* q = smem_raw;
-    sorted = reinterpret_cast<unsigned long long*>(q); q += sizeof(unsigned long long) * npad;
-    heap.comp = reinterpret_cast<unsigned long long*>(q); q += sizeof(unsigned long long) * 2 * (size_t)S;
-    omin = reinterpret_cast<float*>(q); q += sizeof(float) * Sp;
-    omax = reinterpret_cast<float*>(q); q += sizeof(float) * Sp;
-    heap.mn = reinterpret_cast<float*>(q); q += sizeof(float) * 2 * (size_t)S;
-    heap.mx = reinterpret_cast<float*>(q);
-  } else {
-    sorted = a.g_sorted; omin = a.g_omin; omax = a.g_omax;
-    heap.comp = a.g_hcomp; heap.mn = a.g_hmin; heap.mx = a.g_hmax;
-  }
-  heap.n = 0;
-
-  // ---- phase A: fold the R taps of each channel, priorities, identity part of the outputs
-  if (tid == 0) sh_bad = 0;
-  float lmax = 0.0f;
+  // ---- phase A: fold the R taps of each channel into its key max(|min|, |max|)
+  if (tid == 0) { sh.bad = 0; sh.n_touched = 0; }
+  __syncthreads();
+  unsigned long long lmax = 0ull;
   bool bad = false;
-  for (int c = tid; c < C; c += kPlanThreads) {
-    uint32_t umin = 0xFFFFFFFFu, umax = 0u;
-    for (int r = 0; r < R; ++r) {
-      umin = min(umin, a.colmin[(size_t)c * R + r]);
-      umax = max(umax, a.colmax[(size_t)c * R + r]);
+  for (int c0 = 0; c0 < C; c0 += 8 * kPlanThreads) {
+    uint32_t umin[8], umax[8];
+    if (R == 1) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {   // sixteen independent loads in flight
+        const int c = c0 + u * kPlanThreads + tid;
+        umin[u] = c < C ? __ldg(colmin + c) : 0xFFFFFFFFu;
+        umax[u] = c < C ? __ldg(colmax + c) : 0u;
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = c0 + u * kPlanThreads + tid;
+        umin[u] = 0xFFFFFFFFu; umax[u] = 0u;
+        if (c < C) {
+          for (int r = 0; r < R; ++r) {
+            umin[u] = min(umin[u], __ldg(colmin + (size_t)c * R + r));
+            umax[u] = max(umax[u], __ldg(colmax + (size_t)c * R + r));
+          }
+        }
+      }
     }
-    const float mn = ord_decode(umin), mx = ord_decode(umax);
-    const float key = fmaxf(fabsf(mn), fabsf(mx));
-    bad |= !is_finite(key);
-    a.chmin[c] = mn; a.chmax[c] = mx; a.chkey[c] = key;
-    a.idx_map[c] = c; a.depth[c] = 0; a.bits[c] = 0ull;
-    lmax = fmaxf(lmax, key);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int c = c0 + u * kPlanThreads + tid;
+      if (c >= C) continue;
+      const float key = fmaxf(fabsf(ord_decode(umin[u])), fabsf(ord_decode(umax[u])));
+      bad |= !is_finite(key);
+      keys[c] = key;
+      const unsigned long long kb = (unsigned long long)__float_as_uint(key);
+      lmax = kb > lmax ? kb : lmax;
+    }
   }
-  for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));
-  if ((tid & 31) == 0) red[tid >> 5] = lmax;
-  __syncthreads();
-  if (tid < 32) {
-    float v = red[tid];
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    if (tid == 0) sh_maxw = v;
-  }
-  if (bad) sh_bad = 1;
-  __syncthreads();
-  const float maxw = sh_maxw;
+  if (bad) sh.bad = 1;
+  const float maxw = __uint_as_float((uint32_t)block_max_u64(lmax, sh.red));
 
   if (S == 0) {
     if (tid == 0) {
       const float step = a.qa_bits >= 2 ? __fdiv_rn(maxw, (float)((1 << (a.qa_bits - 1)) - 1)) : a.qa_step;
       if (a.max_abs_out) { a.max_abs_out[0] = maxw; a.max_abs_out[1] = maxw; a.max_abs_out[2] = step; }
       *a.qa_step_dev = step;
-      if (sh_bad) flag(a.dev_status, OCS_DEV_NONFINITE);
+      *a.n_touched = 0;
+      if (sh.bad) flag(a.dev_status, OCS_DEV_NONFINITE);
     }
     return;
   }
 
-  // ---- phase B: radix select of the Sp-th largest priority word (8 digits of 8 bits, high first)
-  unsigned long long prefix = 0ull, mask = 0ull;
+  // ---- phase B: the Sp-th largest key, by a three-level histogram select on the key bits
+  // (keys are non-negative floats: their bit patterns order like their values)
+  uint32_t prefix = 0u, pmask = 0u;
   unsigned int remaining = (unsigned int)Sp;
-  for (int pass = 7; pass >= 0; --pass) {
-    const int shift = pass * 8;
-    if (tid < 256) hist[tid] = 0u;
+  for (int lvl = 0; lvl < 3; ++lvl) {
+    const int shift = lvl == 0 ? 21 : (lvl == 1 ? 10 : 0);
+    const int nbins = lvl == 2 ? 1024 : 2048;
+    for (int i = tid; i < kSelBins * kSelCopies; i += kPlanThreads) hist[i] = 0u;
     __syncthreads();
+    unsigned int* copy = hist + ((tid >> 5) & (kSelCopies - 1)) * kSelBins;
     for (int c = tid; c < C; c += kPlanThreads) {
-      const unsigned long long w = make_prio(a.chkey[c], c);
-      if ((w & mask) == prefix) atomicAdd(&hist[(unsigned int)(w >> shift) & 255u], 1u);
+      const uint32_t kb = __float_as_uint(keys[c]);
+      if ((kb & pmask) == prefix) atomicAdd(&copy[(kb >> shift) & (uint32_t)(nbins - 1)], 1u);
     }
     __syncthreads();
-    if (tid == 0) {
-      unsigned int cum = 0u;
-      int dsel = 0;
-      for (int dgt = 255; dgt >= 0; --dgt) {
-        if (cum + hist[dgt] >= remaining) { dsel = dgt; break; }
-        cum += hist[dgt];
+    // thread t owns bins nbins-1-2t and nbins-2-2t (descending), summed over the copies
+    unsigned int hi = 0u, lo = 0u;
+    if (2 * tid < nbins) {
+      for (int k = 0; k < kSelCopies; ++k) {
+        hi += hist[k * kSelBins + nbins - 1 - 2 * tid];
+        lo += hist[k * kSelBins + nbins - 2 - 2 * tid];
       }
-      sh_thresh = prefix | ((unsigned long long)dsel << shift);
-      sh_count = remaining - cum;
+    }
+    unsigned long long total;
+    const unsigned int above = (unsigned int)block_excl_scan((unsigned long long)(hi + lo), sh.scan, &total);
+    if (above < remaining && remaining <= above + hi + lo) {   // exactly one thread
+      if (above + hi >= remaining) { sh.digit = (unsigned int)(nbins - 1 - 2 * tid); sh.count = remaining - above; }
+      else { sh.digit = (unsigned int)(nbins - 2 - 2 * tid); sh.count = remaining - above - hi; }
     }
     __syncthreads();
-    prefix = sh_thresh;
-    remaining = sh_count;
-    mask |= 255ull << shift;
+    prefix |= sh.digit << shift;
+    pmask |= (uint32_t)(nbins - 1) << shift;
+    remaining = sh.count;
     __syncthreads();
   }
-  const unsigned long long thresh = prefix;  // exactly Sp priority words are >= thresh
+  const uint32_t kthr = prefix;          // bit pattern of the Sp-th largest key
+  const unsigned int ties_taken = remaining;  // that many channels with exactly this key are selected ...
+  const unsigned int n_above = (unsigned int)Sp - ties_taken;   // ... after all channels with a larger key
 
-  // ---- selection + largest key left outside
-  if (tid == 0) sh_count = 0u;
-  for (int i = tid; i < npad; i += kPlanThreads) sorted[i] = 0ull;
-  __syncthreads();
-  float lrest = 0.0f;
-  for (int c = tid; c < C; c += kPlanThreads) {
-    const float key = a.chkey[c];
-    const unsigned long long w = make_prio(key, c);
-    if (w >= thresh) {
-      const unsigned int pos = atomicAdd(&sh_count, 1u);
-      if (pos < (unsigned int)npad) sorted[pos] = w;
+  // ---- selection: channels with a larger key, then the lowest-index channels with the threshold
+  // key.  Threads own contiguous index ranges, so tie ranks follow the channel index.
+  const int cpt = ((C + kPlanThreads - 1) / kPlanThreads) | 1;   // odd: conflict-free strided reads
+  const int c_begin = min(C, tid * cpt), c_end = min(C, c_begin + cpt);
+  unsigned int my_above = 0u, my_ties = 0u;
+  for (int c = c_begin; c < c_end; ++c) {
+    const uint32_t kb = __float_as_uint(keys[c]);
+    my_above += kb > kthr;
+    my_ties += kb == kthr;
+  }
+  unsigned long long total;
+  const unsigned long long pre = block_excl_scan(((unsigned long long)my_above << 32) | my_ties, sh.scan, &total);
+  unsigned int pos_above = (unsigned int)(pre >> 32), tie_rank = (unsigned int)pre;
+  unsigned long long lrest = 0ull;
+  for (int c = c_begin; c < c_end; ++c) {
+    const float key = keys[c];
+    const uint32_t kb = __float_as_uint(key);
+    int slot = -1;
+    if (kb > kthr) slot = (int)pos_above++;
+    else if (kb == kthr && tie_rank++ < ties_taken) slot = (int)(n_above + tie_rank - 1);
+    if (slot >= 0) {
+      sel[slot] = make_prio(key, c);
     } else {
-      lrest = fmaxf(lrest, key);
+      lrest = (unsigned long long)kb > lrest ? (unsigned long long)kb : lrest;
     }
   }
-  for (int o = 16; o > 0; o >>= 1) lrest = fmaxf(lrest, __shfl_xor_sync(0xffffffffu, lrest, o));
+  const float rest_max = __uint_as_float((uint32_t)block_max_u64(lrest, sh.red));
   __syncthreads();
-  if ((tid & 31) == 0) red[tid >> 5] = lrest;
-  __syncthreads();
-  if (tid < 32) {
-    float v = red[tid];
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    if (tid == 0) sh_rest = v;
-  }
-  __syncthreads();
-
-  // ---- phase C: bitonic sort, descending
-  for (int k = 2; k <= npad; k <<= 1) {
-    for (int jj = k >> 1; jj > 0; jj >>= 1) {
-      for (int i = tid; i < npad; i += kPlanThreads) {
-        const int ixj = i ^ jj;
-        if (ixj > i) {
-          const unsigned long long x = sorted[i], y = sorted[ixj];
-          const bool desc = (i & k) == 0;
-          if (desc ? (x < y) : (x > y)) { sorted[i] = y; sorted[ixj] = x; }
-        }
-      }
-      __syncthreads();
-    }
-  }
+  // signed extrema of the selected channels (the only originals the greedy steps can touch)
   for (int i = tid; i < Sp; i += kPlanThreads) {
-    const int c = prio_index(sorted[i]);
-    omin[i] = a.chmin[c];
-    omax[i] = a.chmax[c];
+    const int c = prio_index(sel[i]);
+    uint32_t umin = 0xFFFFFFFFu, umax = 0u;
+    for (int r = 0; r < R; ++r) {
+      umin = min(umin, __ldg(colmin + (size_t)c * R + r));
+      umax = max(umax, __ldg(colmax + (size_t)c * R + r));
+    }
+    a.chmin[c] = ord_decode(umin);
+    a.chmax[c] = ord_decode(umax);
   }
   __syncthreads();
 
-  // ---- phase D: the sequential greedy loop
+  // ---- phase C: the greedy steps
+  float step = a.qa_step;
+  if (a.qa_bits >= 2) {
+    // two-pass rule: the grid step is max|W'| of a plain-halving run divided by L
+    for (int i = tid; i < Sp; i += kPlanThreads) live0[i] = sel[i];
+    __syncthreads();
+    const float predicted = fmaxf(rest_max, greedy_rounds(a, sh, live0, live1, batch, Sp, 0.0f, false));
+    step = __fdiv_rn(predicted, (float)((1 << (a.qa_bits - 1)) - 1));
+    __syncthreads();
+  }
+  const float d = __fmul_rn(step, 0.5f);
+  for (int i = tid; i < Sp; i += kPlanThreads) live0[i] = sel[i];
+  __syncthreads();
+  const float maxwp = fmaxf(rest_max, greedy_rounds(a, sh, live0, live1, batch, Sp, d, true));
   if (tid == 0) {
-    float step = a.qa_step;
-    if (a.qa_bits >= 2) {
-      const float predicted = greedy_run(a, sorted, omin, omax, Sp, heap, 0.0f, sh_rest, false);
-      const int L = (1 << (a.qa_bits - 1)) - 1;
-      step = __fdiv_rn(predicted, (float)L);
-    }
-    const float d = __fmul_rn(step, 0.5f);
-    const float maxwp = greedy_run(a, sorted, omin, omax, Sp, heap, d, sh_rest, true);
     if (a.max_abs_out) { a.max_abs_out[0] = maxw; a.max_abs_out[1] = maxwp; a.max_abs_out[2] = step; }
     *a.qa_step_dev = step;
-    if (sh_bad) flag(a.dev_status, OCS_DEV_NONFINITE);
+    *a.n_touched = sh.n_touched;
+    if (sh.bad) flag(a.dev_status, OCS_DEV_NONFINITE);
   }
 }
 
@@ -363,42 +516,80 @@ __global__ void __launch_bounds__(256)
 split_scatter_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_in, int S,
                      float* __restrict__ Wout, int64_t ld_out, const int32_t* __restrict__ idx_map,
                      const int32_t* __restrict__ depth, const unsigned long long* __restrict__ bits,
-                     const float* __restrict__ qa_step_dev, int rows_per_cta) {
+                     const float* __restrict__ qa_step_dev) {
   const int ncols_out = (C + S) * R;
-  const int e0 = (blockIdx.x * 256 + threadIdx.x) * 4;
-  if (e0 >= ncols_out) return;
+  const int col_blocks = (ncols_out + 1023) / 1024;
+  long long u, u1;
+  cta_range((long long)col_blocks * O, &u, &u1);
   const float d = __fmul_rn(*qa_step_dev, 0.5f);
-  int src[4], dep[4];
-  unsigned long long bt[4];
-  int any = 0;
+  while (u < u1) {
+    const int cb = (int)(u / O);
+    const int r0 = (int)(u - (long long)cb * O);
+    const int r1 = (int)min((long long)O, r0 + (u1 - u));
+    u += r1 - r0;
+    const int e0 = (cb * 256 + threadIdx.x) * 4;
+    if (e0 >= ncols_out) continue;
+    const bool full = e0 + 3 < ncols_out;
+    if (VEC && full && e0 + 3 < C * R) {
+      // four original columns: they move as one 16-byte word; only split channels change value
+      int dep[4];
+      unsigned long long bt[4];
+      int any = 0;
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    const int e = e0 + c;
-    if (e < ncols_out) {
-      const int j = e / R, r = e - j * R;
-      src[c] = idx_map[j] * R + r;
-      dep[c] = min(depth[j], d == 0.0f ? kMaxHalvings : 64);
-      bt[c] = bits[j];
-    } else {
-      src[c] = 0; dep[c] = 0; bt[c] = 0ull;
+      for (int c = 0; c < 4; ++c) {
+        const int j = (e0 + c) / R;
+        dep[c] = min(depth[j], d == 0.0f ? kMaxHalvings : 64);
+        bt[c] = bits[j];
+        any |= dep[c];
+      }
+      const float4* src = reinterpret_cast<const float4*>(W + (int64_t)r0 * ld_in + e0);
+      float4* dst = reinterpret_cast<float4*>(Wout + (int64_t)r0 * ld_out + e0);
+      const int64_t sstride = ld_in >> 2, dstride = ld_out >> 2;
+      if (!any) {
+#pragma unroll 8
+        for (int row = r0; row < r1; ++row) {
+          __stcs(dst, __ldcs(src));
+          src += sstride;
+          dst += dstride;
+        }
+      } else {
+#pragma unroll 2
+        for (int row = r0; row < r1; ++row) {
+          const float4 t = __ldcs(src);
+          float v[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            float w = v[c];
+            for (int i = 0; i < dep[c]; ++i)
+              w = (i < 64 && ((bt[c] >> i) & 1ull)) ? split_new(w, d) : split_keep(w, d);
+            v[c] = w;
+          }
+          __stcs(dst, make_float4(v[0], v[1], v[2], v[3]));
+          src += sstride;
+          dst += dstride;
+        }
+      }
+      continue;
     }
-    any |= dep[c];
-  }
-  const bool full = e0 + 3 < ncols_out;
-  const bool identity = VEC && full && (e0 + 3 < C * R);
-  const int r0 = blockIdx.y * rows_per_cta;
-  const int r1 = min(O, r0 + rows_per_cta);
+    int src[4], dep[4];
+    unsigned long long bt[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int e = e0 + c;
+      if (e < ncols_out) {
+        const int j = e / R, r = e - j * R;
+        src[c] = idx_map[j] * R + r;
+        dep[c] = min(depth[j], d == 0.0f ? kMaxHalvings : 64);
+        bt[c] = bits[j];
+      } else {
+        src[c] = 0; dep[c] = 0; bt[c] = 0ull;
+      }
+    }
 #pragma unroll 4
-  for (int row = r0; row < r1; ++row) {
-    float v[4];
-    if (identity) {
-      const float4 t = __ldcs(reinterpret_cast<const float4*>(W + (int64_t)row * ld_in + e0));
-      v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-    } else {
+    for (int row = r0; row < r1; ++row) {
+      float v[4];
 #pragma unroll
       for (int c = 0; c < 4; ++c) v[c] = (e0 + c < ncols_out) ? __ldg(W + (int64_t)row * ld_in + src[c]) : 0.0f;
-    }
-    if (any) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         float w = v[c];
@@ -406,16 +597,204 @@ split_scatter_kernel(const float* __restrict__ W, int O, int C, int R, int64_t l
           w = (i < 64 && ((bt[c] >> i) & 1ull)) ? split_new(w, d) : split_keep(w, d);
         v[c] = w;
       }
-    }
-    float* out = Wout + (int64_t)row * ld_out + e0;
-    if (VEC && full) {
-      __stcs(reinterpret_cast<float4*>(out), make_float4(v[0], v[1], v[2], v[3]));
-    } else {
+      float* out = Wout + (int64_t)row * ld_out + e0;
+      if (VEC && full) {
+        __stcs(reinterpret_cast<float4*>(out), make_float4(v[0], v[1], v[2], v[3]));
+      } else {
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
-        if (e0 + c < ncols_out) out[c] = v[c];
+        for (int c = 0; c < 4; ++c)
+          if (e0 + c < ncols_out) out[c] = v[c];
+      }
     }
   }
+}
+
+// ------------------------------------------------------------------------------------------------
+// K3, bulk-copy form.  A group of whole rows is brought into shared memory by the copy engine
+// (cp.async.bulk, one copy per row, completion on an mbarrier), laid out with the output's row
+// length; threads only compute the 2S channels per row that change -- the S appended copies, read
+// from their source channels in shared memory, then the split originals in place -- and the
+// finished rows leave by bulk stores.  Every byte of W is read from DRAM once, every byte of W'
+// written once, and the duplicated channels are gathered from shared memory, not from global.
+// Two row-group buffers alternate: the load of group i+1 and the store of group i-1 overlap the
+// (small) compute of group i.  One CTA per SM; row groups are dealt round-robin.
+constexpr int kRowThreads = 512;
+constexpr long long kRowWaitCycles = 2000000000ll;  // about one second
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ float apply_path(float w, int dep, unsigned long long bt, float d) {
+  for (int i = 0; i < dep; ++i) w = (i < 64 && ((bt >> i) & 1ull)) ? split_new(w, d) : split_keep(w, d);
+  return w;
+}
+
+__device__ __forceinline__ bool row_bar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+
+__global__ void __launch_bounds__(kRowThreads, 1)
+split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_in, int S, float* __restrict__ Wout,
+                  int64_t ld_out, const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
+                  const unsigned long long* __restrict__ bits, const float* __restrict__ qa_step_dev,
+                  const int32_t* __restrict__ touched, const int* __restrict__ n_touched, int rows_per_group,
+                  int srow /*floats between rows in shared memory*/, int* dev_status) {
+  extern __shared__ __align__(128) unsigned char row_smem[];
+  __shared__ __align__(8) unsigned long long bars[2];
+  __shared__ int abort_flag;
+  float* buf[2] = {reinterpret_cast<float*>(row_smem),
+                   reinterpret_cast<float*>(row_smem) + (size_t)rows_per_group * srow};
+  const int tid = threadIdx.x;
+  const int in_cols = C * R;                 // a multiple of 4 (checked by the host)
+  const int out_cols = (C + S) * R;
+  const int out_bulk = out_cols & ~3;        // floats per row that leave by bulk store
+  const int n_groups = (O + rows_per_group - 1) / rows_per_group;
+  const int my_groups = blockIdx.x < n_groups ? (n_groups - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+  const float d = __fmul_rn(*qa_step_dev, 0.5f);
+  const int nt = *n_touched;
+  const int dep_cap = d == 0.0f ? kMaxHalvings : 64;
+
+  if (tid == 0) {
+    for (int b = 0; b < 2; ++b)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[b])) : "memory");
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  auto issue_load = [&](int i) {   // thread 0 only
+    const int g = blockIdx.x + i * gridDim.x;
+    const int r0 = g * rows_per_group;
+    const int gn = min(rows_per_group, O - r0);
+    const uint32_t bar = smem_addr(&bars[i & 1]);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)gn * in_cols * 4u)
+                 : "memory");
+    for (int rl = 0; rl < gn; ++rl) {
+      const float* src = W + (int64_t)(r0 + rl) * ld_in;
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+          ::"r"(smem_addr(buf[i & 1] + (size_t)rl * srow)), "l"(src), "r"((uint32_t)in_cols * 4u), "r"(bar)
+          : "memory");
+    }
+  };
+
+  // With one row per group every row needs the same (source, path) items: a thread keeps its
+  // share of them in registers instead of re-reading the plan's arrays for every row.
+  constexpr int kItems = 8;
+  const int tail_items = S * R;
+  const int orig_items = nt * R;
+  const bool cached = rows_per_group == 1 && tail_items <= kItems * kRowThreads && orig_items <= kItems * kRowThreads;
+  int t_src[kItems], t_dep[kItems], o_off[kItems], o_dep[kItems];
+  unsigned long long t_bits[kItems];
+  if (cached) {
+#pragma unroll
+    for (int k = 0; k < kItems; ++k) {
+      const int e = tid + k * kRowThreads;
+      t_src[k] = -1; t_dep[k] = 0; t_bits[k] = 0ull; o_off[k] = -1; o_dep[k] = 0;
+      if (e < tail_items) {
+        const int sidx = e / R, r = e - sidx * R;
+        const int j = C + sidx;
+        t_src[k] = __ldg(idx_map + j) * R + r;
+        t_dep[k] = min(__ldg(depth + j), dep_cap);
+        t_bits[k] = __ldg(bits + j);
+      }
+      if (e < orig_items) {
+        const int t = e / R, r = e - t * R;
+        const int j = __ldg(touched + t);
+        o_off[k] = j * R + r;
+        o_dep[k] = min(__ldg(depth + j), dep_cap);
+      }
+    }
+  }
+
+  if (tid == 0 && my_groups > 0) issue_load(0);
+  int issued = my_groups > 0 ? 1 : 0;
+  for (int i = 0; i < my_groups; ++i) {
+    const int b = i & 1;
+    if (tid == 0) {
+      // the stores issued from the other buffer have finished reading it
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      if (i + 1 < my_groups) { issue_load(i + 1); ++issued; }
+    }
+    {  // bounded wait for this group's rows
+      const uint32_t bar = smem_addr(&bars[b]);
+      const uint32_t parity = (uint32_t)(i >> 1) & 1u;
+      if (!row_bar_try(bar, parity)) {
+        const long long t0 = clock64();
+        for (uint32_t it = 1;; ++it) {
+          if (row_bar_try(bar, parity)) break;
+          if ((it & 63u) == 0u && (abort_flag || clock64() - t0 > kRowWaitCycles)) { abort_flag = 1; break; }
+        }
+      }
+    }
+    __syncthreads();
+    if (abort_flag) break;
+    const int g = blockIdx.x + i * gridDim.x;
+    const int r0 = g * rows_per_group;
+    const int gn = min(rows_per_group, O - r0);
+    float* rows = buf[b];
+    if (cached) {
+      // appended copies: channel C + s reads its source channel's original values
+#pragma unroll
+      for (int k = 0; k < kItems; ++k) {
+        if (t_src[k] >= 0) {
+          const float v = apply_path(rows[t_src[k]], t_dep[k], t_bits[k], d);
+          const int col = in_cols + tid + k * kRowThreads;
+          rows[col] = v;
+          if (col >= out_bulk) Wout[(int64_t)r0 * ld_out + col] = v;   // the last 1-3 floats of a row
+        }
+      }
+      __syncthreads();
+      // split originals, in place: the kept copy takes the (w - d)/2 branch at every level
+#pragma unroll
+      for (int k = 0; k < kItems; ++k)
+        if (o_off[k] >= 0) rows[o_off[k]] = apply_path(rows[o_off[k]], o_dep[k], 0ull, d);
+    } else {
+      for (int it = tid; it < gn * tail_items; it += kRowThreads) {
+        const int rl = it / tail_items, e = it - rl * tail_items;
+        const int sidx = e / R, r = e - sidx * R;
+        const int j = C + sidx;
+        const float v = apply_path(rows[(size_t)rl * srow + (size_t)__ldg(idx_map + j) * R + r],
+                                   min(__ldg(depth + j), dep_cap), __ldg(bits + j), d);
+        const int col = in_cols + e;
+        rows[(size_t)rl * srow + col] = v;
+        if (col >= out_bulk) Wout[(int64_t)(r0 + rl) * ld_out + col] = v;
+      }
+      __syncthreads();
+      for (int it = tid; it < gn * orig_items; it += kRowThreads) {
+        const int rl = it / orig_items, e = it - rl * orig_items;
+        const int t = e / R, r = e - t * R;
+        const int j = __ldg(touched + t);
+        float* q = rows + (size_t)rl * srow + (size_t)j * R + r;
+        *q = apply_path(*q, min(__ldg(depth + j), dep_cap), 0ull, d);
+      }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the bulk store
+    __syncthreads();
+    if (tid == 0 && out_bulk > 0) {
+      for (int rl = 0; rl < gn; ++rl) {
+        float* dst = Wout + (int64_t)(r0 + rl) * ld_out;
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                     ::"l"(dst), "r"(smem_addr(rows + (size_t)rl * srow)), "r"((uint32_t)out_bulk * 4u)
+                     : "memory");
+      }
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+  }
+  if (tid == 0) {
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (abort_flag) {
+      flag(dev_status, OCS_DEV_TIMEOUT);
+      if (issued > 0)
+        for (int k = 0; k < 2000; ++k) __nanosleep(100);   // let copies still in flight land
+    }
+  }
+  __syncthreads();
 }
 
 struct SplitWs {
@@ -423,8 +802,10 @@ struct SplitWs {
   float* chmin; float* chmax; float* chkey;
   int32_t* depth; unsigned long long* bits;
   float* qa_step_dev;
-  unsigned long long* g_sorted; float* g_omin; float* g_omax;
-  unsigned long long* g_hcomp; float* g_hmin; float* g_hmax;
+  int32_t* touched; int* n_touched;
+  unsigned long long* g_buf;
+  int cap, npad, Sp;
+  size_t plan_words;
   size_t total;
 };
 
@@ -439,32 +820,32 @@ SplitWs carve_split_ws(void* ws, int C, int R, int S) {
   const size_t ncols = (size_t)C * R;
   w.colmin = reinterpret_cast<uint32_t*>(take(4 * ncols));
   w.colmax = reinterpret_cast<uint32_t*>(take(4 * ncols));
-  w.chmin = reinterpret_cast<float*>(take(4 * (size_t)C));
-  w.chmax = reinterpret_cast<float*>(take(4 * (size_t)C));
+  w.chmin = reinterpret_cast<float*>(take(4 * ((size_t)C + S)));
+  w.chmax = reinterpret_cast<float*>(take(4 * ((size_t)C + S)));
   w.chkey = reinterpret_cast<float*>(take(4 * (size_t)C));
   w.depth = reinterpret_cast<int32_t*>(take(4 * ((size_t)C + S)));
   w.bits = reinterpret_cast<unsigned long long*>(take(8 * ((size_t)C + S)));
   w.qa_step_dev = reinterpret_cast<float*>(take(256));
-  if (S > kPlanSmemSplits) {
-    size_t npad = 1;
-    while (npad < (size_t)(S < C ? S : C)) npad <<= 1;
-    w.g_sorted = reinterpret_cast<unsigned long long*>(take(8 * npad));
-    w.g_omin = reinterpret_cast<float*>(take(4 * (size_t)S));
-    w.g_omax = reinterpret_cast<float*>(take(4 * (size_t)S));
-    w.g_hcomp = reinterpret_cast<unsigned long long*>(take(16 * (size_t)S));
-    w.g_hmin = reinterpret_cast<float*>(take(8 * (size_t)S));
-    w.g_hmax = reinterpret_cast<float*>(take(8 * (size_t)S));
-  }
+  w.n_touched = reinterpret_cast<int*>(take(256));
+  w.Sp = S < C ? S : C;
+  w.touched = reinterpret_cast<int32_t*>(take(4 * (size_t)(w.Sp > 0 ? w.Sp : 1)));
+  w.cap = w.Sp + S;
+  w.npad = 1;
+  while (w.npad < w.cap) w.npad <<= 1;
+  w.plan_words = (size_t)w.Sp + 2 * (size_t)w.cap + (size_t)w.npad;
+  if (S > kPlanSmemSplits) w.g_buf = reinterpret_cast<unsigned long long*>(take(8 * w.plan_words));
   w.total = off;
   return w;
 }
 
-int rows_per_cta_for(int O, int col_blocks) {
-  // aim at ~8 CTAs per SM in total, at least 16 rows per CTA so the atomics stay cheap
-  const int target_row_chunks = max(1, (kNumSMs * 8 + col_blocks - 1) / col_blocks);
-  int rows = (O + target_row_chunks - 1) / target_row_chunks;
-  rows = max(rows, 16);
-  return min(rows, max(O, 1));
+// Grid of a streaming kernel: one resident wave, but no more CTAs than there are 8-row slices.
+template <typename K>
+int wave_grid(K kernel, long long units) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 4;
+  const long long cap = (long long)kNumSMs * per_sm;
+  const long long want = (units + 7) / 8;
+  return (int)(want < cap ? (want > 0 ? want : 1) : cap);
 }
 
 }  // namespace
@@ -505,15 +886,15 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
   if (cudaMemsetAsync(w.colmax, 0x00, 4 * (size_t)ncols, stream) != cudaSuccess) return OCS_ERR_CUDA;
 
   {
-    const int col_blocks = (ncols + 1023) / 1024;
-    const int rows = rows_per_cta_for(O, col_blocks);
-    dim3 grid(col_blocks, (O + rows - 1) / rows);
+    const long long units = (long long)((ncols + 1023) / 1024) * O;
     const bool vec = (ld_in % 4 == 0) && aligned(W, 16);
     LaunchScope ls("col_minmax_kernel", stream);
     if (vec)
-      col_minmax_kernel<true><<<grid, 256, 0, stream>>>(W, O, ncols, ld_in, rows, w.colmin, w.colmax, dev_status);
+      col_minmax_kernel<true><<<wave_grid(col_minmax_kernel<true>, units), 256, 0, stream>>>(
+          W, O, ncols, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
     else
-      col_minmax_kernel<false><<<grid, 256, 0, stream>>>(W, O, ncols, ld_in, rows, w.colmin, w.colmax, dev_status);
+      col_minmax_kernel<false><<<wave_grid(col_minmax_kernel<false>, units), 256, 0, stream>>>(
+          W, O, ncols, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
     if ((st = launch_status()) != OCS_OK) return st;
   }
   {
@@ -523,19 +904,22 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     a.chmin = w.chmin; a.chmax = w.chmax; a.chkey = w.chkey;
     a.idx_map = idx_map; a.split_order = split_order; a.depth = w.depth; a.bits = w.bits;
     a.max_abs_out = max_abs_out; a.qa_step_dev = w.qa_step_dev;
-    a.g_sorted = w.g_sorted; a.g_omin = w.g_omin; a.g_omax = w.g_omax;
-    a.g_hcomp = w.g_hcomp; a.g_hmin = w.g_hmin; a.g_hmax = w.g_hmax;
+    a.touched = w.touched; a.n_touched = w.n_touched;
+    a.g_buf = w.g_buf; a.cap = w.cap; a.npad = w.npad; a.Sp = w.Sp;
     a.dev_status = dev_status;
-    size_t smem = 0;
-    if (S <= kPlanSmemSplits && S > 0) {
-      const int Sp = S < C ? S : C;
-      size_t npad = 1;
-      while (npad < (size_t)Sp) npad <<= 1;
-      smem = 8 * npad + 16 * (size_t)S + 8 * (size_t)Sp + 16 * (size_t)S;
-    }
+    // dynamic shared memory: the plan buffer (when S is small enough) and, overlapping the part of
+    // it that the live sets only use after the selection, the selection histograms and the keys
+    const size_t plan_bytes = (S <= kPlanSmemSplits) ? 8 * w.plan_words : 0;
+    const size_t hist_off = (S <= kPlanSmemSplits) ? align_up(8 * (size_t)w.Sp, 16) : 0;
+    const size_t keys_off = hist_off + kSelHistBytes;
+    const bool keys_fit = keys_off + 4 * (size_t)C <= (size_t)kPlanSmemBytes;
+    a.hist_off = (int)hist_off;
+    a.keys_off = keys_fit ? (int)keys_off : -1;
+    size_t smem = keys_fit ? keys_off + 4 * (size_t)C : keys_off;
+    if (plan_bytes > smem) smem = plan_bytes;
     static bool attr_set = false;
     if (!attr_set) {
-      if (cudaFuncSetAttribute(split_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+      if (cudaFuncSetAttribute(split_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPlanSmemBytes) != cudaSuccess)
         return OCS_ERR_CUDA;
       attr_set = true;
     }
@@ -545,17 +929,35 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
   }
   {
     const int ncols_out = (C + S) * R;
-    const int col_blocks = (ncols_out + 1023) / 1024;
-    const int rows = rows_per_cta_for(O, col_blocks);
-    dim3 grid(col_blocks, (O + rows - 1) / rows);
     const bool vec = (ld_in % 4 == 0) && (ld_out % 4 == 0) && aligned(W, 16) && aligned(W_out, 16);
+    const int srow = (ncols_out + 3) & ~3;
+    const size_t row_bytes = 4 * (size_t)srow;
     LaunchScope ls("split_scatter_kernel", stream);
-    if (vec)
-      split_scatter_kernel<true><<<grid, 256, 0, stream>>>(W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth,
-                                                           w.bits, w.qa_step_dev, rows);
-    else
-      split_scatter_kernel<false><<<grid, 256, 0, stream>>>(W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth,
-                                                            w.bits, w.qa_step_dev, rows);
+    if (vec && (C * R) % 4 == 0 && 2 * row_bytes <= kRowSmemBytes) {
+      // rows per group: as many as fit in half the buffer space, but keep at least one group per SM
+      long long g = (long long)(kRowSmemBytes / 2 / row_bytes);
+      g = min(g, (long long)max(1, O / kNumSMs));
+      g = min(g, 64ll);
+      const int n_groups = (int)((O + g - 1) / g);
+      static bool attr_set = false;
+      if (!attr_set) {
+        if (cudaFuncSetAttribute(split_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmemBytes) !=
+            cudaSuccess)
+          return OCS_ERR_CUDA;
+        attr_set = true;
+      }
+      split_rows_kernel<<<min(n_groups, kNumSMs), kRowThreads, 2 * (size_t)g * row_bytes, stream>>>(
+          W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g,
+          srow, dev_status);
+    } else {
+      const long long units = (long long)((ncols_out + 1023) / 1024) * O;
+      if (vec)
+        split_scatter_kernel<true><<<wave_grid(split_scatter_kernel<true>, units), 256, 0, stream>>>(
+            W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth, w.bits, w.qa_step_dev);
+      else
+        split_scatter_kernel<false><<<wave_grid(split_scatter_kernel<false>, units), 256, 0, stream>>>(
+            W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth, w.bits, w.qa_step_dev);
+    }
     if ((st = launch_status()) != OCS_OK) return st;
   }
   return OCS_OK;
