@@ -180,6 +180,37 @@ ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, in
                      const float* bias, float* Y, int32_t* acc_out, void* ws, size_t ws_bytes,
                      int* dev_status, void* stream);
 
+/* Steps between quantized layers ------------------------------------------------------------
+ * The paper runs whole networks through the split and quantized layers (Section 5: ImageNet
+ * CNNs; Section 6: a two-layer LSTM language model).  These calls are the float steps between
+ * the layers; each output element is produced by single IEEE-rounded fp32 operations in a
+ * fixed order, so a network's activations are reproducible bit for bit.  Tensors are dense;
+ * images are NHWC.  All pointers device, all calls asynchronous on `stream`.
+ *
+ * ocs_add_relu: y[i] = a[i] + b[i] (b NULL: y[i] = a[i]), then max(., 0) when relu != 0
+ *   (ReLU after a layer; the residual connection of a bottleneck block).  y may equal a.
+ * ocs_maxpool3x3s2: 3x3 window, stride 2, padding 1 (padding never wins);
+ *   y [Nb][(H-1)/2+1][(Wd-1)/2+1][C].
+ * ocs_global_avgpool: y[n][c] = (sum over (h, w), row-major, sequential) * (1 / (H*Wd)).
+ * ocs_nchw_to_nhwc: layout change of the network input.
+ * ocs_embedding: out[t][:] = table[ids[t]][:], table [V][E]; an id outside [0, V) reads row 0
+ *   and sets OCS_DEV_BAD_INDEX.
+ * ocs_lstm_cell (Section 6's LSTM): gates g_ih, g_hh [batch][4*hidden] in the order i, f, g, o,
+ *   each already holding its bias; z = g_ih + g_hh; c <- fmaf(sigmoid(z_f), c, sigmoid(z_i) *
+ *   tanh(z_g)); h <- sigmoid(z_o) * tanh(c); c [batch][hidden] updated in place, h written.
+ *   sigmoid and tanh are fixed routines: e = exp(-|x|) resp. exp(-2|x|) computed as 2^n * P(f ln 2)
+ *   with t = x * log2(e), n = rint(t), f = t - n, P the degree-6 Taylor polynomial of exp in
+ *   Horner form with fused multiply-adds (x clamped at -87); sigmoid = 1/(1+e) or e/(1+e),
+ *   tanh = (1-e)/(1+e) with the sign of x; divisions IEEE. */
+ocs_status ocs_add_relu(const float* a, const float* b, int64_t n, int relu, float* y, void* stream);
+ocs_status ocs_maxpool3x3s2(const float* x, int Nb, int H, int Wd, int C, float* y, void* stream);
+ocs_status ocs_global_avgpool(const float* x, int Nb, int H, int Wd, int C, float* y, void* stream);
+ocs_status ocs_nchw_to_nhwc(const float* x, int Nb, int C, int H, int Wd, float* y, void* stream);
+ocs_status ocs_embedding(const float* table, const int32_t* ids, int64_t n, int V, int E, float* out,
+                         int* dev_status, void* stream);
+ocs_status ocs_lstm_cell(const float* g_ih, const float* g_hh, int batch, int hidden, float* c, float* h,
+                         void* stream);
+
 #ifdef __cplusplus
 }
 #endif

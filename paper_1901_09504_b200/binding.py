@@ -29,6 +29,7 @@ EXPORTS = [
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
     "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
+    "ocs_add_relu", "ocs_maxpool3x3s2", "ocs_global_avgpool", "ocs_nchw_to_nhwc", "ocs_embedding", "ocs_lstm_cell",
 ]
 
 _lib = None
@@ -242,3 +243,60 @@ def ocs_qconv(X_codes, a_scale, W_packed, w_scale, idx_map, S: int, kh: int, kw:
                          _ptr(Y), _ptr(acc), _ptr(ws), C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
     _check(st, "ocs_qconv")
     return (Y, acc) if want_acc else Y
+
+
+def ocs_add_relu(a, b=None, relu: bool = True, out=None):
+    """y = a (+ b), then ReLU when relu; fp32 tensors of equal shape."""
+    assert a.is_cuda and a.dtype == torch.float32 and a.is_contiguous()
+    assert b is None or (b.shape == a.shape and b.dtype == torch.float32 and b.is_contiguous())
+    y = out if out is not None else torch.empty_like(a)
+    _check(lib().ocs_add_relu(_ptr(a), _ptr(b), C.c_int64(a.numel()), int(bool(relu)), _ptr(y), _stream()),
+           "ocs_add_relu")
+    return y
+
+
+def ocs_maxpool3x3s2(x):
+    """x fp32 NHWC -> 3x3 stride-2 pad-1 max pooling."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 4 and x.is_contiguous()
+    Nb, H, Wd, Cn = x.shape
+    y = torch.empty((Nb, (H - 1) // 2 + 1, (Wd - 1) // 2 + 1, Cn), dtype=torch.float32, device=x.device)
+    _check(lib().ocs_maxpool3x3s2(_ptr(x), Nb, H, Wd, Cn, _ptr(y), _stream()), "ocs_maxpool3x3s2")
+    return y
+
+
+def ocs_global_avgpool(x):
+    """x fp32 NHWC -> [Nb, C]."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 4 and x.is_contiguous()
+    Nb, H, Wd, Cn = x.shape
+    y = torch.empty((Nb, Cn), dtype=torch.float32, device=x.device)
+    _check(lib().ocs_global_avgpool(_ptr(x), Nb, H, Wd, Cn, _ptr(y), _stream()), "ocs_global_avgpool")
+    return y
+
+
+def ocs_nchw_to_nhwc(x):
+    assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 4 and x.is_contiguous()
+    Nb, Cn, H, Wd = x.shape
+    y = torch.empty((Nb, H, Wd, Cn), dtype=torch.float32, device=x.device)
+    _check(lib().ocs_nchw_to_nhwc(_ptr(x), Nb, Cn, H, Wd, _ptr(y), _stream()), "ocs_nchw_to_nhwc")
+    return y
+
+
+def ocs_embedding(table, ids, dev_status=None):
+    """table fp32 [V, E], ids int32 [...] -> fp32 [..., E]."""
+    assert table.is_cuda and table.dtype == torch.float32 and table.dim() == 2 and table.is_contiguous()
+    assert ids.is_cuda and ids.dtype == torch.int32 and ids.is_contiguous()
+    out = torch.empty(tuple(ids.shape) + (table.shape[1],), dtype=torch.float32, device=table.device)
+    _check(lib().ocs_embedding(_ptr(table), _ptr(ids), C.c_int64(ids.numel()), table.shape[0], table.shape[1],
+                               _ptr(out), _ptr(dev_status), _stream()), "ocs_embedding")
+    return out
+
+
+def ocs_lstm_cell(g_ih, g_hh, c, h=None):
+    """Gates fp32 [batch, 4*hidden] (i, f, g, o); c [batch, hidden] is updated IN PLACE; returns (c, h)."""
+    assert g_ih.is_cuda and g_ih.dtype == torch.float32 and g_ih.is_contiguous() and g_hh.is_contiguous()
+    batch, hidden = c.shape
+    assert g_ih.shape == (batch, 4 * hidden) and g_hh.shape == g_ih.shape and c.is_contiguous()
+    if h is None:
+        h = torch.empty_like(c)
+    _check(lib().ocs_lstm_cell(_ptr(g_ih), _ptr(g_hh), batch, hidden, _ptr(c), _ptr(h), _stream()), "ocs_lstm_cell")
+    return c, h

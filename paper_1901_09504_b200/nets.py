@@ -1,0 +1,150 @@
+"""Chains of C-ABI calls for whole networks: the ResNet-50 convolution stack (Section 5's CNN
+workloads) and the two-layer LSTM language model (Section 6).
+
+Only call sequencing lives here: which tensor feeds which layer.  Every arithmetic step -- split,
+clip search, quantization, the integer convolutions and GEMMs, ReLU, residual adds, pooling, the
+LSTM cell -- is one of the library's kernels, reached through the binding.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import torch
+
+from . import binding as B
+
+
+@dataclass
+class QLayer:
+    """One layer after the offline steps of Section 3.5: split, quantized and (for a convolution)
+    reordered weights, plus what the run-time layer needs to gather the duplicated channels."""
+    codes: torch.Tensor        # int8: conv [O, ld] packed for ocs_qconv; linear [O, ld]
+    w_scale: torch.Tensor      # fp32 [1]
+    idx_map: torch.Tensor      # int32 [C + S]
+    bias: torch.Tensor | None  # fp32 [O]
+    C: int
+    O: int
+    S: int
+    k: int = 1
+    stride: int = 1
+    pad: int = 0
+
+
+def prepare_layer(W, bias, ratio: float, bits: int, clip_mode: int = B.CLIP_NONE, qa_bits: int = 0, conv: bool = False,
+                  stride: int = 1, pad: int = 0, n_candidates: int = 128, n_bins: int = 2048, dev_status=None) -> QLayer:
+    """W fp32 [O, C] or [O, C, k, k] on the device -> QLayer (ocs_split, ocs_quantize, ocs_pack_conv_weights)."""
+    O, Cn = W.shape[0], W.shape[1]
+    k = W.shape[2] if W.dim() == 4 else 1
+    R = k * k
+    S = B.ocs_num_splits(Cn, ratio)
+    W_out, idx_map, _, mx = B.ocs_split(W.contiguous(), S, qa_bits=qa_bits, dev_status=dev_status, want_order=False)
+    codes, scale, _ = B.ocs_quantize(W_out, bits, True, clip_mode, n_candidates, n_bins, cols=(Cn + S) * R,
+                                     max_abs_in=mx[1:2], dev_status=dev_status)
+    if conv:
+        codes = B.ocs_pack_conv_weights(codes, O, Cn, S, k, k)
+    return QLayer(codes, scale, idx_map, bias, Cn, O, S, k, stride, pad)
+
+
+def quantize_activations(x, signed: bool, bits: int = 8, dev_status=None):
+    """Dynamic per-tensor grid (max |x| of the tensor handed to the layer): returns dense codes shaped
+    like x and the fp32 [1] scale."""
+    flat = x.reshape(1, -1)
+    codes, scale, _ = B.ocs_quantize(flat, bits, signed, B.CLIP_NONE, dev_status=dev_status)
+    return codes[0, :flat.shape[1]].view(x.shape), scale
+
+
+def conv_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None):
+    """x fp32 NHWC -> fp32 NHWC (activation quantization + ocs_qconv)."""
+    xc, xs = quantize_activations(x, a_signed, a_bits, dev_status)
+    return B.ocs_qconv(xc, xs, L.codes, L.w_scale, L.idx_map, L.S, L.k, L.k, L.stride, L.pad, bias=L.bias,
+                       dev_status=dev_status)
+
+
+def linear_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None):
+    """x fp32 [M, C] -> fp32 [M, O] (activation quantization + ocs_qlinear)."""
+    M, Cn = x.shape
+    ld = B.round_up(Cn, 16)
+    codes, scale, _ = B.ocs_quantize(x.contiguous(), a_bits, a_signed, B.CLIP_NONE, ld_codes=ld, dev_status=dev_status)
+    return B.ocs_qlinear(codes, scale, L.codes, L.w_scale, L.idx_map, Cn, L.S, bias=L.bias, dev_status=dev_status)
+
+
+# ------------------------------------------------------------------------------------------ ResNet-50
+def prepare_resnet50(cfg, device, dev_status=None):
+    """cfg from ocs_inputs.configs.config4 -> {layer name: QLayer}."""
+    mode = B.CLIP_MSE if cfg["clip"] == "mse" else B.CLIP_NONE
+    out = {}
+    for spec in cfg["layers"] + [cfg["fc"]]:
+        W, bias = cfg["params"][spec.name]
+        Wd = torch.from_numpy(W).to(device)
+        bd = torch.from_numpy(bias).to(device)
+        if spec.name == "fc":
+            out["fc"] = prepare_layer(Wd.reshape(spec.O, spec.C), bd, cfg["ratio"], cfg["w_bits"], mode,
+                                      dev_status=dev_status)
+        else:
+            out[spec.name] = prepare_layer(Wd, bd, cfg["ratio"], cfg["w_bits"], mode, conv=True, stride=spec.stride,
+                                           pad=spec.pad, dev_status=dev_status)
+    return out
+
+
+def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, dev_status=None):
+    """X fp32 NCHW on the device -> logits fp32 [Nb, 1000]; with keep, also every named tensor."""
+    t = {}
+    x = B.ocs_nchw_to_nhwc(X_nchw.contiguous())
+    first = True
+    for spec in cfg["layers"]:
+        src = t[spec.input_from] if spec.input_from else x
+        y = conv_forward(layers[spec.name], src, a_signed=first, a_bits=a_bits, dev_status=dev_status)
+        if spec.residual_from:
+            y = B.ocs_add_relu(y, t[spec.residual_from], relu=spec.relu, out=y)
+            t[spec.name.rsplit(".", 1)[0] + ".out"] = y
+        elif spec.relu:
+            y = B.ocs_add_relu(y, None, relu=True, out=y)
+        t[spec.name] = y
+        x = y
+        if first:
+            x = B.ocs_maxpool3x3s2(y)
+            t["pool"] = x
+            first = False
+    feat = B.ocs_global_avgpool(x)
+    t["avgpool"] = feat
+    logits = linear_forward(layers["fc"], feat, a_signed=False, a_bits=a_bits, dev_status=dev_status)
+    t["fc"] = logits
+    return (logits, t) if keep else logits
+
+
+# ------------------------------------------------------------------------------------------ LSTM
+def prepare_lstm(cfg, device, dev_status=None):
+    """cfg from ocs_inputs.configs.config5 -> dict of QLayers and the embedding table."""
+    p = cfg["params"]
+    mode = B.CLIP_MSE if cfg["clip"] == "mse" else B.CLIP_NONE
+    out = {"emb": torch.from_numpy(p["emb"]).to(device)}
+    for layer in range(2):
+        for nm, bn in (("W_ih", "b_ih"), ("W_hh", "b_hh")):
+            out[f"{nm}{layer}"] = prepare_layer(torch.from_numpy(p[f"{nm}{layer}"]).to(device),
+                                                torch.from_numpy(p[f"{bn}{layer}"]).to(device), cfg["ratio"],
+                                                cfg["w_bits"], mode, dev_status=dev_status)
+    out["W_dec"] = prepare_layer(torch.from_numpy(p["W_dec"]).to(device), torch.from_numpy(p["b_dec"]).to(device),
+                                 cfg["ratio"], cfg["w_bits"], mode, dev_status=dev_status)
+    return out
+
+
+def lstm_forward(cfg, layers, tokens, a_bits: int = 8, keep: bool = False, dev_status=None):
+    """tokens int32 [seq, batch] on the device -> logits fp32 [seq * batch, vocab] (h0 = c0 = 0)."""
+    seq, batch = tokens.shape
+    hidden = cfg["hidden"]
+    dev = tokens.device
+    emb = B.ocs_embedding(layers["emb"], tokens.contiguous(), dev_status=dev_status)
+    h = [torch.zeros((batch, hidden), dtype=torch.float32, device=dev) for _ in range(2)]
+    c = [torch.zeros((batch, hidden), dtype=torch.float32, device=dev) for _ in range(2)]
+    tops = torch.empty((seq, batch, hidden), dtype=torch.float32, device=dev)
+    for t in range(seq):
+        x = emb[t]
+        for l in range(2):
+            g_ih = linear_forward(layers[f"W_ih{l}"], x, True, a_bits, dev_status)
+            g_hh = linear_forward(layers[f"W_hh{l}"], h[l], True, a_bits, dev_status)
+            hn = tops[t] if l == 1 else torch.empty_like(h[l])
+            B.ocs_lstm_cell(g_ih, g_hh, c[l], hn)
+            h[l] = hn
+            x = hn
+    logits = linear_forward(layers["W_dec"], tops.view(seq * batch, hidden), True, a_bits, dev_status)
+    return (logits, dict(emb=emb, tops=tops, c=c)) if keep else logits
