@@ -71,6 +71,22 @@ class Ledger:
         return sum(self.bytes.values())
 
 
+def reduce_max(value: float, world: int, device) -> float:
+    """Max over ranks of a per-rank timing (the multi-GPU step time is the slowest rank's)."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank moves the same bytes per step (replicas, weak scaling)."""
+    return bytes_per_rank_step * world / (ms_per_step * 1e-3) / 1e9
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -375,10 +391,8 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item()) / steps, (ocs.ocs_kernel_launches() - n0) // steps
+        ms = reduce_max(e0.elapsed_time(e1), world, dev)
+        return ms / steps, (ocs.ocs_kernel_launches() - n0) // steps
 
     clk = sample_clocks_start() if rank == 0 else None
     ms_step, launches = timed(wl.step, args.steps, args.warmup)
@@ -431,7 +445,7 @@ def main():
                         avg_launch_ms=top_ms / top_cnt,
                         timed="second pass over the same steps with CUDA events around every kernel launch")
 
-    value = led.total * world / (ms_step * 1e-3) / 1e9
+    value = aggregate_gbs(led.total, world, ms_step)
     line = dict(
         metric=METRIC, value=value, unit="GB/s", n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None,
@@ -447,7 +461,7 @@ def main():
         roofline=roofline,
         kernels=kernels,
         cpu_baseline=cpu,
-        e2e=dict(value=led.total * world / (ms_e2e * 1e-3) / 1e9, unit="GB/s", ms_per_step=ms_e2e,
+        e2e=dict(value=aggregate_gbs(led.total, world, ms_e2e), unit="GB/s", ms_per_step=ms_e2e,
                  h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
         gpu_launches=int(launches) * args.steps,
         clocks=clocks,

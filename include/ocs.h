@@ -49,8 +49,9 @@ typedef enum {
 #define OCS_DEV_DEPTH 8     /* a channel was re-split more than 63 times under the QA rule */
 
 typedef enum {
-  OCS_CLIP_NONE = 0, /* alpha = max|T| (Eq. 1) */
-  OCS_CLIP_MSE = 1   /* histogram MSE search (Section 4.1) */
+  OCS_CLIP_NONE = 0,     /* alpha = max|T| (Eq. 1) */
+  OCS_CLIP_MSE = 1,      /* histogram MSE search (Section 4.1) */
+  OCS_CLIP_MSE_EXACT = 2 /* the same candidates scored on the elements themselves, no histogram */
 } ocs_clip_mode;
 
 /* Host helpers ------------------------------------------------------------------------- */
@@ -117,7 +118,10 @@ ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_in, int S, 
  *   mode NONE: alpha = max|T|.   mode MSE (Section 4.1): histogram of |x| with n_bins equal
  *   bins on [0, max|T|]; candidates alpha_c = max*c/n_candidates, c = 1..n_candidates;
  *   score_c = sum_b h[b]*(x_b - Q_c(x_b))^2 at the bin centres x_b, in double; the smallest
- *   score wins, ties go to the largest alpha.
+ *   score wins, ties go to the largest alpha.   mode MSE_EXACT: the same candidates with
+ *   score_c = sum_i (x_i - Q_c(x_i))^2 over the elements, in double (the MSE of Section 4.1
+ *   without the histogram approximation; bound by fp64 arithmetic, not by memory).  For this
+ *   mode n_bins is ignored and the workspace query is called with n_bins = 0.
  * T [rows][cols] fp32 with row stride ld_in; codes [rows][cols] with row stride ld_codes bytes
  * (bytes beyond cols in a row are left untouched).  max_abs_in (nullable): device scalar
  * holding max|T| if the caller already has it (saves one pass over T).  *scale = step,

@@ -20,7 +20,7 @@ OCS_OK = 0
 STATUS_NAMES = {0: "OCS_OK", 1: "OCS_ERR_INVALID_ARG", 2: "OCS_ERR_SHAPE", 3: "OCS_ERR_WORKSPACE",
                 4: "OCS_ERR_UNSUPPORTED", 5: "OCS_ERR_CUDA"}
 DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT, DEV_DEPTH = 1, 2, 4, 8
-CLIP_NONE, CLIP_MSE = 0, 1
+CLIP_NONE, CLIP_MSE, CLIP_MSE_EXACT = 0, 1, 2
 
 EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
@@ -169,6 +169,8 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
         codes = torch.empty((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=T.device)
         scale = torch.zeros(1, dtype=torch.float32, device=T.device)
         alpha = torch.zeros(1, dtype=torch.float32, device=T.device)
+    if mode == CLIP_MSE_EXACT:
+        n_bins = 0
     nws = lib().ocs_quantize_workspace_bytes(int(n_bins), int(n_candidates))
     if ws is None:
         ws = _ws(nws, T.device)
@@ -182,7 +184,7 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
     hp, sp = C.c_void_p(0), C.c_void_p(0)
     lib().ocs_quantize_workspace_views(_ptr(ws), int(n_bins), int(n_candidates), C.byref(hp), C.byref(sp))
     base = ws.data_ptr()
-    hist = ws[hp.value - base: hp.value - base + 8 * n_bins].view(torch.int64).clone()
+    hist = ws[hp.value - base: hp.value - base + 8 * max(n_bins, 1)].view(torch.int64).clone()
     scores = ws[sp.value - base: sp.value - base + 8 * n_candidates].view(torch.float64).clone()
     return codes, scale, alpha, hist, scores
 

@@ -161,6 +161,88 @@ score_kernel(const unsigned long long* __restrict__ hist, const float* __restric
   if (threadIdx.x == 0) scores[blockIdx.x] = red[0];
 }
 
+// The same candidates scored on the elements themselves (no histogram): score_c = sum_i (x_i - Q_c(x_i))^2
+// in double.  A CTA stages tiles of kExactTile elements in shared memory (as double); a thread owns up to
+// four candidates and one slice of the tile.  Per-CTA partial sums are combined in a fixed order by
+// exact_combine_kernel, so the scores do not depend on scheduling.  Bound by the fp64 pipe (one division
+// per element and candidate), not by HBM.
+constexpr int kExactTile = 2048;
+constexpr int kExactMaxGrid = 2 * kNumSMs;
+constexpr int kExactOwn = kMaxCandidates / 256;   // candidates per thread at most
+
+__global__ void __launch_bounds__(256)
+exact_score_kernel(View v, const float* __restrict__ maxp, int n_candidates, int L, int is_signed,
+                   double* __restrict__ partial) {
+  __shared__ double xs[kExactTile];
+  __shared__ double comb[256];
+  const float m = *maxp;
+  int slots = 1;                                   // candidate slots per pass: a power of two <= 256
+  while (slots < n_candidates && slots < 256) slots <<= 1;
+  const int slices = 256 / slots;
+  const int my_slot = threadIdx.x % slots, my_slice = threadIdx.x / slots;
+  double step[kExactOwn], acc[kExactOwn];
+#pragma unroll
+  for (int k = 0; k < kExactOwn; ++k) {
+    const int c = my_slot + k * slots + 1;
+    acc[k] = 0.0;
+    step[k] = 0.0;
+    if (c <= n_candidates && m > 0.0f) {
+      const float alpha_c = __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)c), (double)n_candidates));
+      step[k] = __ddiv_rn((double)alpha_c, (double)L);
+    }
+  }
+  const double lo = is_signed ? -(double)L : 0.0, hi = (double)L;
+  const long long total = v.rows * v.cols;
+  const long long n_tiles = (total + kExactTile - 1) / kExactTile;
+  for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    const long long e0 = t * kExactTile;
+    const int cnt = (int)min((long long)kExactTile, total - e0);
+    for (int i = threadIdx.x; i < cnt; i += 256) {
+      const long long e = e0 + i;
+      const long long row = e / v.cols;
+      xs[i] = (double)__ldcs(v.T + row * v.ld + (e - row * v.cols));
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kExactOwn; ++k) {
+      if (step[k] > 0.0) {
+        double a = acc[k];
+        for (int i = my_slice; i < cnt; i += slices) {   // ascending element order inside the slice
+          const double x = xs[i];
+          double q = rint(__ddiv_rn(x, step[k]));
+          q = fmin(fmax(q, lo), hi);
+          const double err = __dsub_rn(x, __dmul_rn(q, step[k]));
+          a = __dadd_rn(a, __dmul_rn(err, err));
+        }
+        acc[k] = a;
+      }
+    }
+    __syncthreads();
+  }
+  // slices of one candidate are added in slice order
+#pragma unroll
+  for (int k = 0; k < kExactOwn; ++k) {
+    comb[threadIdx.x] = acc[k];
+    __syncthreads();
+    const int c = my_slot + k * slots + 1;
+    if (my_slice == 0 && c <= n_candidates) {
+      double a = comb[my_slot];
+      for (int sl = 1; sl < slices; ++sl) a = __dadd_rn(a, comb[sl * slots + my_slot]);
+      partial[(size_t)blockIdx.x * n_candidates + (c - 1)] = a;
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(256)
+exact_combine_kernel(const double* __restrict__ partial, int n_parts, int n_candidates, double* __restrict__ scores) {
+  const int c = blockIdx.x * 256 + threadIdx.x;
+  if (c >= n_candidates) return;
+  double a = 0.0;
+  for (int b = 0; b < n_parts; ++b) a = __dadd_rn(a, partial[(size_t)b * n_candidates + c]);
+  scores[c] = a;
+}
+
 // The search's winner: smallest score, ties to the largest threshold.  Every CTA of the quantize
 // kernel evaluates it (n_candidates doubles) instead of a separate single-thread launch.
 __device__ float pick_alpha(const double* __restrict__ scores, float m, int n_candidates) {
@@ -237,6 +319,7 @@ struct QuantWs {
   unsigned int* maxbits;       // fp32 bits of max|T|
   unsigned long long* hist;
   double* scores;
+  double* partial;             // exact scorer only: [kExactMaxGrid][n_candidates]
   size_t total;
 };
 
@@ -251,6 +334,8 @@ QuantWs carve_quant_ws(void* ws, int n_bins, int n_candidates) {
   w.maxbits = reinterpret_cast<unsigned int*>(take(256));
   w.hist = reinterpret_cast<unsigned long long*>(take(8 * (size_t)(n_bins > 0 ? n_bins : 1)));
   w.scores = reinterpret_cast<double*>(take(8 * (size_t)(n_candidates > 0 ? n_candidates : 1)));
+  if (n_bins == 0)  // the exact scorer's layout
+    w.partial = reinterpret_cast<double*>(take(8 * (size_t)kExactMaxGrid * (size_t)(n_candidates > 0 ? n_candidates : 1)));
   w.total = off;
   return w;
 }
@@ -278,9 +363,11 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!T || !codes || !scale) return OCS_ERR_INVALID_ARG;
   if (bits < 2 || bits > 8) return OCS_ERR_INVALID_ARG;
-  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE) return OCS_ERR_INVALID_ARG;
+  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE && mode != OCS_CLIP_MSE_EXACT) return OCS_ERR_INVALID_ARG;
   if (mode == OCS_CLIP_MSE && (n_candidates < 1 || n_candidates > kMaxCandidates || n_bins < 1 || n_bins > kMaxBins))
     return OCS_ERR_INVALID_ARG;
+  if (mode == OCS_CLIP_MSE_EXACT && (n_candidates < 1 || n_candidates > kMaxCandidates)) return OCS_ERR_INVALID_ARG;
+  if (mode == OCS_CLIP_MSE_EXACT) n_bins = 0;
   if (rows <= 0 || cols <= 0 || ld_in < cols || ld_codes < cols) return OCS_ERR_SHAPE;
   if (!aligned(T, 4)) return OCS_ERR_SHAPE;
   if (mode == OCS_CLIP_NONE) { n_bins = 1; n_candidates = 1; }
@@ -312,6 +399,20 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
     {
       LaunchScope ls("score_kernel", stream);
       score_kernel<<<n_candidates, 256, 0, stream>>>(w.hist, maxp, n_bins, n_candidates, L, is_signed, w.scores);
+    }
+    if ((st = launch_status()) != OCS_OK) return st;
+    scores = w.scores;
+  } else if (mode == OCS_CLIP_MSE_EXACT) {
+    const long long n_tiles = (v.rows * v.cols + kExactTile - 1) / kExactTile;
+    const int grid = (int)(n_tiles < kExactMaxGrid ? n_tiles : kExactMaxGrid);
+    {
+      LaunchScope ls("exact_score_kernel", stream);
+      exact_score_kernel<<<grid, 256, 0, stream>>>(v, maxp, n_candidates, L, is_signed, w.partial);
+    }
+    if ((st = launch_status()) != OCS_OK) return st;
+    {
+      LaunchScope ls("exact_combine_kernel", stream);
+      exact_combine_kernel<<<(n_candidates + 255) / 256, 256, 0, stream>>>(w.partial, grid, n_candidates, w.scores);
     }
     if ((st = launch_status()) != OCS_OK) return st;
     scores = w.scores;

@@ -161,3 +161,41 @@ def test_quantize_config2_mse_and_config3_slice():
     Wp, _, _, _ = orc.split(c3["W"], orc.num_splits(6272, 0.05))
     for bits in (4, 5, 6, 8):
         _check_quant(Wp, bits, True, 1)
+
+
+def _check_quant_exact(T, bits, signed, n_cand=128, ld=None):
+    T = np.ascontiguousarray(T, dtype=np.float32)
+    rows, cols = T.shape
+    if ld is None:
+        Td = dev(T)
+    else:
+        Td = torch.full((rows, ld), -3.0e3, dtype=torch.float32, device="cuda")
+        Td[:, :cols] = dev(T)
+    st = ocs.new_status()
+    codes, scale, alpha, _, scores = ocs.ocs_quantize(Td, bits, signed, ocs.CLIP_MSE_EXACT, n_cand, cols=cols,
+                                                      dev_status=st, return_search=True)
+    assert ocs.ocs_poll_status(st) == 0
+    o = orc.clip_mse_exact(T, bits, signed, n_cand)
+    np.testing.assert_allclose(host(scores), o["scores"], rtol=1e-9, atol=1e-300)   # double sums, other order
+    assert np.float32(host(alpha)[0]) == np.float32(o["alpha"])
+    o_codes, o_scale = orc.quantize(T, bits, signed, o["alpha"])
+    assert float(host(scale)[0]) == np.float32(o_scale)
+    np.testing.assert_array_equal(host(codes)[:, :cols], o_codes)
+    return o["alpha"]
+
+
+def test_quantize_exact_mse_scorer():
+    """The element-wise scorer (no histogram) against the checker's, and next to the histogram search."""
+    c = configs.config1()
+    Wp, _, _, _ = orc.split(c["W"], 26)
+    for bits in (3, 4, 6, 8):
+        a_exact = _check_quant_exact(Wp, bits, True)
+        a_hist = orc.clip_mse(Wp, bits, True, 2048, 128)["alpha"]
+        assert abs(a_exact - a_hist) <= 1.5 * orc.maxabs(Wp) / 128          # within one candidate of each other
+    _check_quant_exact(c["A"], 8, False, n_cand=33)
+    _check_quant_exact(c["A"][:, :509], 5, False, n_cand=300, ld=512)
+    _check_quant_exact(prng.laplace(5, 0, (37, 4099), 0.01), 4, True, n_cand=1024, ld=4100)
+    _check_quant_exact(prng.laplace(5, 1, (1, 1), 1.0), 8, True, n_cand=1)
+    c2 = configs.config2(batch=1)
+    Wp2, _, _, _ = orc.split(c2["W"], 6)
+    _check_quant_exact(Wp2.reshape(256, -1), 6, True)
