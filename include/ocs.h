@@ -134,6 +134,30 @@ ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, int64_t ld_i
                         const float* max_abs_in, int8_t* codes, int64_t ld_codes, float* scale,
                         float* alpha, void* ws, size_t ws_bytes, int* dev_status, void* stream);
 
+/* ocs_quantize_noalloc ---------------------------------------------------------------------
+ * (No counterpart in the paper: a packaging variant of ocs_quantize.)
+ * Same operation, arguments and results as ocs_quantize, minus (ws, ws_bytes).  It is meant for
+ * callers that cannot obtain device memory where they need to quantize: code that runs inside
+ * another framework's execution callback where cudaMalloc is off limits because it stalls the
+ * whole device, a serving process that gave all device memory to its own planner at start-up,
+ * or a job so close to the memory limit that an allocation may fail.  Such callers still pass
+ * the input and output buffers; what they are spared is the scratch.
+ * The scratch (48 KB: running maximum, histogram, candidate scores) is a fixed array inside the
+ * library's device image, so every GPU that loads the library carries it until the process
+ * exits.  The call allocates nothing and frees nothing.
+ * Limits: modes OCS_CLIP_NONE and OCS_CLIP_MSE with n_bins <= 4096 and n_candidates <= 1024;
+ * anything larger, and OCS_CLIP_MSE_EXACT, returns OCS_ERR_UNSUPPORTED (use ocs_quantize).
+ * The first call on each device looks up the array's device address (with that device
+ * current) and remembers it; make that first call before starting any stream capture.
+ * All calls on a device share the one array, which keeps whatever the previous call left: each
+ * call re-clears the parts it needs to start from zero, but two calls whose kernels overlap on
+ * the GPU (different streams, no ordering between them) race on it -- order them, or use
+ * ocs_quantize with separate workspaces. */
+ocs_status ocs_quantize_noalloc(const float* T, int64_t rows, int64_t cols, int64_t ld_in, int bits,
+                                int is_signed, ocs_clip_mode mode, int n_candidates, int n_bins,
+                                const float* max_abs_in, int8_t* codes, int64_t ld_codes, float* scale,
+                                float* alpha, int* dev_status, void* stream);
+
 /* Reads back the search's intermediate results after an MSE-mode ocs_quantize on the same
  * workspace (for tests and reports): hist [n_bins] uint64 and scores [n_candidates] double,
  * both device pointers into ws.  Host call, no GPU work. */

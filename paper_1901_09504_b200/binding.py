@@ -26,7 +26,7 @@ EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
     "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
     "ocs_split_workspace_bytes", "ocs_split",
-    "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views",
+    "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
     "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
     "ocs_add_relu", "ocs_maxpool3x3s2", "ocs_global_avgpool", "ocs_nchw_to_nhwc", "ocs_embedding", "ocs_lstm_cell",
@@ -302,3 +302,32 @@ def ocs_lstm_cell(g_ih, g_hh, c, h=None):
         h = torch.empty_like(c)
     _check(lib().ocs_lstm_cell(_ptr(g_ih), _ptr(g_hh), batch, hidden, _ptr(c), _ptr(h), _stream()), "ocs_lstm_cell")
     return c, h
+
+
+def ocs_quantize_noalloc(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_candidates: int = 128,
+                         n_bins: int = 2048, cols: int | None = None, ld_codes: int | None = None, max_abs_in=None,
+                         dev_status=None, out=None):
+    """ocs_quantize without a workspace: for callers that must not allocate device memory where they
+    quantize (the library's built-in 48 KB scratch is used instead).  The outputs are still the
+    caller's: pass `out` = (codes, scale, alpha) to reuse buffers, otherwise this wrapper creates them
+    with torch for convenience -- the library call itself allocates nothing either way.
+    Returns (codes, scale, alpha)."""
+    assert T.is_cuda and T.dtype == torch.float32 and T.dim() == 2 and T.stride(1) == 1
+    rows, ld_in = T.shape[0], T.stride(0)
+    if cols is None:
+        cols = T.shape[1]
+    if out is not None:
+        codes, scale, alpha = out
+        ld_codes = codes.stride(0)
+    else:
+        if ld_codes is None:
+            ld_codes = round_up(cols, 16)
+        codes = torch.empty((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=T.device)
+        scale = torch.zeros(1, dtype=torch.float32, device=T.device)
+        alpha = torch.zeros(1, dtype=torch.float32, device=T.device)
+    st = lib().ocs_quantize_noalloc(_ptr(T), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_in), int(bits),
+                                    int(bool(is_signed)), int(mode), int(n_candidates), int(n_bins),
+                                    _ptr(max_abs_in), _ptr(codes), C.c_int64(ld_codes), _ptr(scale), _ptr(alpha),
+                                    _ptr(dev_status), _stream())
+    _check(st, "ocs_quantize_noalloc")
+    return codes, scale, alpha

@@ -435,3 +435,37 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
                                                                           dev_status);
   return launch_status();
 }
+
+// ------------------------------------------------------------------------------------------------
+// ocs_quantize_noalloc: ocs_quantize for callers that cannot hand over a workspace.  The scratch
+// (running maximum, histogram, candidate scores) lives in a fixed array that is part of the loaded
+// library image on every device; nothing is allocated, now or at load time beyond that image.
+namespace ocs {
+namespace {
+constexpr size_t kStaticScratchBytes = 48 * 1024;   // covers n_bins <= 4096 and n_candidates <= 1024
+static __device__ __align__(256) unsigned char g_quantize_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices] = {nullptr};       // device address of the array, per device
+}  // namespace
+}  // namespace ocs
+
+extern "C" ocs_status ocs_quantize_noalloc(const float* T, int64_t rows, int64_t cols, int64_t ld_in, int bits,
+                                           int is_signed, ocs_clip_mode mode, int n_candidates, int n_bins,
+                                           const float* max_abs_in, int8_t* codes, int64_t ld_codes, float* scale,
+                                           float* alpha, int* dev_status, void* stream) {
+  if (mode == OCS_CLIP_MSE_EXACT) return OCS_ERR_UNSUPPORTED;   // its partial sums need megabytes
+  if (mode == OCS_CLIP_MSE && (n_bins > kMaxBins || n_candidates > kMaxCandidates)) return OCS_ERR_UNSUPPORTED;
+  const int nb = mode == OCS_CLIP_MSE ? n_bins : 1, nc = mode == OCS_CLIP_MSE ? n_candidates : 1;
+  if (ocs_quantize_workspace_bytes(nb, nc) > kStaticScratchBytes) return OCS_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return OCS_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return OCS_ERR_UNSUPPORTED;
+  if (!g_scratch_addr[dev]) {
+    // in host code the array's name is only a handle: ask the runtime for its address on this device
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_quantize_scratch) != cudaSuccess || !p) return OCS_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  return ocs_quantize(T, rows, cols, ld_in, bits, is_signed, mode, n_candidates, n_bins, max_abs_in, codes, ld_codes,
+                      scale, alpha, g_scratch_addr[dev], kStaticScratchBytes, dev_status, stream);
+}
