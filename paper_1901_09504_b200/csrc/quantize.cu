@@ -50,36 +50,66 @@ int grid_for(K kernel, long long tiles, size_t dyn_smem = 0) {
   return (int)(tiles < cap ? (tiles > 0 ? tiles : 1) : cap);
 }
 
-// Loads the thread's u-th quad of tile t; n = number of valid elements (0..4); col = first column.
-__device__ __forceinline__ int load_quad(const View& v, long long t, int u, float x[4], long long* row_out,
-                                         long long* col_out) {
-  const long long row = t / v.tiles_per_row;
-  const long long seg = t - row * v.tiles_per_row;
-  const long long col = seg * kTileCols + (long long)(u * 256 + threadIdx.x) * 4;
-  *row_out = row;
-  *col_out = col;
-  if (col >= v.cols) return 0;
-  const float* p = v.T + row * v.ld + col;
-  if (v.vec && col + 3 < v.cols) {
-    const float4 q = __ldcs(reinterpret_cast<const float4*>(p));
-    x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
-    return 4;
+// A CTA's walk over its tiles (blockIdx.x, blockIdx.x + gridDim.x, ...) without per-tile divisions.
+struct TileWalk {
+  long long row, seg;     // current tile: row and tile index inside the row
+  long long drow, dseg;   // gridDim.x tiles further = drow rows and dseg tiles
+  long long left;         // tiles still to visit (including the current one)
+  __device__ TileWalk(const View& v) {
+    row = blockIdx.x / v.tiles_per_row;
+    seg = blockIdx.x - row * v.tiles_per_row;
+    drow = gridDim.x / v.tiles_per_row;
+    dseg = gridDim.x - drow * v.tiles_per_row;
+    left = (long long)blockIdx.x < v.tiles ? (v.tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
   }
-  const int n = (int)min(4ll, v.cols - col);
-  for (int i = 0; i < 4; ++i) x[i] = i < n ? __ldcs(p + i) : 0.0f;
-  return n;
+  __device__ void next(const View& v) {
+    row += drow;
+    seg += dseg;
+    if (seg >= v.tiles_per_row) { seg -= v.tiles_per_row; ++row; }
+    --left;
+  }
+};
+
+// The thread's kTileQuads quads of the current tile.  x[u] holds quad u, n[u] how many of its four
+// values exist (0..4); c[u] is the quad's first column inside the tile.
+__device__ __forceinline__ void load_tile(const View& v, const TileWalk& w, float4 x[kTileQuads], int n[kTileQuads]) {
+  const long long col0 = w.seg * kTileCols;
+  const float* base = v.T + w.row * v.ld + col0;
+  const long long rest = v.cols - col0;
+  if (v.vec && rest >= kTileCols) {          // a full tile: unconditional 128-bit loads
+#pragma unroll
+    for (int u = 0; u < kTileQuads; ++u) {
+      x[u] = __ldcs(reinterpret_cast<const float4*>(base) + u * 256 + threadIdx.x);
+      n[u] = 4;
+    }
+    return;
+  }
+  const int nt = (int)(rest < kTileCols ? rest : kTileCols);
+#pragma unroll
+  for (int u = 0; u < kTileQuads; ++u) {
+    const int c = (u * 256 + threadIdx.x) * 4;
+    n[u] = max(0, min(4, nt - c));
+    x[u] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    if (n[u] == 4 && v.vec) {
+      x[u] = __ldcs(reinterpret_cast<const float4*>(base + c));
+    } else if (n[u] > 0) {
+      x[u].x = __ldcs(base + c);
+      if (n[u] > 1) x[u].y = __ldcs(base + c + 1);
+      if (n[u] > 2) x[u].z = __ldcs(base + c + 2);
+      if (n[u] > 3) x[u].w = __ldcs(base + c + 3);
+    }
+  }
 }
 
 __global__ void __launch_bounds__(256) maxabs_kernel(View v, unsigned int* maxbits) {
   float m = 0.0f;
-  for (long long t = blockIdx.x; t < v.tiles; t += gridDim.x) {
+  for (TileWalk w(v); w.left > 0; w.next(v)) {
+    float4 x[kTileQuads];
+    int n[kTileQuads];
+    load_tile(v, w, x, n);
 #pragma unroll
-    for (int u = 0; u < kTileQuads; ++u) {
-      float x[4];
-      long long row, col;
-      const int n = load_quad(v, t, u, x, &row, &col);
-      if (n) m = fmaxf(m, fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3]))));
-    }
+    for (int u = 0; u < kTileQuads; ++u)   // missing values were loaded as 0: they cannot raise the maximum
+      m = fmaxf(m, fmaxf(fmaxf(fabsf(x[u].x), fabsf(x[u].y)), fmaxf(fabsf(x[u].z), fabsf(x[u].w))));
   }
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
   __shared__ float red[8];
@@ -101,22 +131,22 @@ hist_kernel(View v, const float* __restrict__ maxp, int n_bins, unsigned long lo
     const float invw = __fdiv_rn((float)n_bins, m);
     unsigned int* mine = sh + ((threadIdx.x >> 5) % kHistCopies) * n_bins;
     const int last = n_bins - 1;
-    for (long long t = blockIdx.x; t < v.tiles; t += gridDim.x) {
-      float x[kTileQuads][4];
+    auto count = [&](float xv) {
+      const int b = min(last, (int)__fmul_rn(fabsf(xv), invw));  // truncation
+      atomicAdd(&mine[b], 1u);
+    };
+    for (TileWalk w(v); w.left > 0; w.next(v)) {
+      float4 x[kTileQuads];
       int n[kTileQuads];
+      load_tile(v, w, x, n);
 #pragma unroll
       for (int u = 0; u < kTileQuads; ++u) {
-        long long row, col;
-        n[u] = load_quad(v, t, u, x[u], &row, &col);
-      }
-#pragma unroll
-      for (int u = 0; u < kTileQuads; ++u) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          if (i < n[u]) {
-            const int b = min(last, (int)__fmul_rn(fabsf(x[u][i]), invw));  // truncation
-            atomicAdd(&mine[b], 1u);
-          }
+        if (n[u] == 4) {
+          count(x[u].x); count(x[u].y); count(x[u].z); count(x[u].w);
+        } else {
+          if (n[u] > 0) count(x[u].x);
+          if (n[u] > 1) count(x[u].y);
+          if (n[u] > 2) count(x[u].z);
         }
       }
     }
@@ -270,6 +300,16 @@ __device__ float pick_alpha(const double* __restrict__ scores, float m, int n_ca
   return __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)bc), (double)n_candidates));
 }
 
+// code = clamp(rint(x * inv)): clamping first is the same thing (the bounds are integers) and leaves one
+// conversion with round-to-nearest-even
+__device__ __forceinline__ int quant_code(float x, float inv, float lo, float hi) {
+  return __float2int_rn(fminf(fmaxf(__fmul_rn(x, inv), lo), hi));
+}
+__device__ __forceinline__ unsigned int pack4(int c0, int c1, int c2, int c3) {
+  return __byte_perm(__byte_perm((unsigned)c0, (unsigned)c1, 0x0040), __byte_perm((unsigned)c2, (unsigned)c3, 0x0040),
+                     0x5410);
+}
+
 __global__ void __launch_bounds__(256)
 quantize_kernel(View v, const float* __restrict__ alpha_p, const double* __restrict__ scores, int n_candidates, int L,
                 int is_signed, int8_t* __restrict__ codes, long long ld_codes, int packed_ok,
@@ -286,25 +326,19 @@ quantize_kernel(View v, const float* __restrict__ alpha_p, const double* __restr
     if (alpha_out) *alpha_out = zero ? 0.0f : alpha;
   }
   bool bad = false;
-  for (long long t = blockIdx.x; t < v.tiles; t += gridDim.x) {
-    float x[kTileQuads][4];
+  for (TileWalk w(v); w.left > 0; w.next(v)) {
+    float4 x[kTileQuads];
     int n[kTileQuads];
-    long long row[kTileQuads], col[kTileQuads];
-#pragma unroll
-    for (int u = 0; u < kTileQuads; ++u) n[u] = load_quad(v, t, u, x[u], &row[u], &col[u]);
+    load_tile(v, w, x, n);
+    // the dense view flattens rows, so its code offset is the flat index
+    int8_t* out_tile = codes + w.row * ld_codes + w.seg * kTileCols;
 #pragma unroll
     for (int u = 0; u < kTileQuads; ++u) {
       if (!n[u]) continue;
-      unsigned int word = 0u;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        bad |= (i < n[u]) && !is_finite(x[u][i]);
-        float q = rintf(__fmul_rn(x[u][i], inv));  // round half to even
-        q = fminf(fmaxf(q, lo), hi);
-        word |= ((unsigned int)((int)q) & 0xFFu) << (8 * i);
-      }
-      // the dense view flattens rows, so its code offset is the flat index
-      int8_t* out = codes + row[u] * ld_codes + col[u];
+      bad |= !(is_finite(x[u].x) && is_finite(x[u].y) && is_finite(x[u].z) && is_finite(x[u].w));  // missing = 0
+      const unsigned int word = pack4(quant_code(x[u].x, inv, lo, hi), quant_code(x[u].y, inv, lo, hi),
+                                      quant_code(x[u].z, inv, lo, hi), quant_code(x[u].w, inv, lo, hi));
+      int8_t* out = out_tile + (u * 256 + threadIdx.x) * 4;
       if (packed_ok && n[u] == 4) {
         *reinterpret_cast<unsigned int*>(out) = word;
       } else {
