@@ -14,6 +14,11 @@
 //   warp 0      TMA producer (weights always, activations when the block is TMA-able)
 //   warp 1      allocates tensor memory, issues tcgen05.mma, commits to the stage barriers
 //   warps 2..5  gather producers during the main loop, then the epilogue (tcgen05.ld -> global)
+// The K-blocks whose A tile is assembled ("tail" blocks) come last in a CTA's K order and use two
+// dedicated A buffers, so the gather warps start at kernel begin and run ahead of the TMA-fed main
+// loop.  CTAs that share the M tile and the K slice (neighbouring N tiles) form a thread-block
+// cluster: each assembles 1/CL of a tail tile's rows and stores them into every peer's buffer
+// through distributed shared memory, so a tile is gathered once per cluster, not once per CTA.
 // Every mbarrier wait is bounded by a clock limit; on expiry the CTA sets OCS_DEV_TIMEOUT, lets its
 // outstanding copies land, frees its tensor memory and returns.
 #include <cuda.h>
@@ -97,8 +102,52 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// The same bounded wait for barriers that peer CTAs of the cluster arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((it & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) { *abort_flag = 1; return false; }
+    }
+  }
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Thread-block cluster: rank and size, a peer CTA's view of one of our shared-memory addresses,
+// stores and barrier arrivals into a peer's shared memory, cluster-wide barrier.
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_peer_v4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_peer(uint32_t addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
   asm volatile(
@@ -134,6 +183,11 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_
       "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+// Arrives on the barrier at the same shared-memory offset in every CTA of the mask.
+__device__ __forceinline__ void umma_commit_multicast(uint32_t bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(cta_mask) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -268,13 +322,20 @@ __device__ __forceinline__ uint4 direct_chunk(const GemmParams& p, const RowInfo
   return zero;
 }
 
+constexpr int kTailBufs = 2;   // A tiles assembled by the gather warps (shared across the cluster)
+
 template <int BN>
 struct SmemLayout {
   static constexpr int kABytes = BM * BK;
   static constexpr int kBBytes = BN * BK;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int kTileBytes = kStages * kStageBytes;
+  // ring depth: one stage fewer when the two tail buffers are needed
+  static constexpr int kStagesNoTail = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int kStagesTail = kStagesNoTail - 1;
+  static constexpr int kMaxStages = kStagesNoTail;
+  static constexpr int kTileBytes =
+      (kStagesNoTail * kStageBytes > kStagesTail * kStageBytes + kTailBufs * kABytes)
+          ? kStagesNoTail * kStageBytes : kStagesTail * kStageBytes + kTailBufs * kABytes;
   static constexpr int kCtrlBytes = 1024;               // barriers, tensor-memory slot, flags
   static constexpr int kRowTableBytes = BM * 24;        // RowInfo per tile row
   static constexpr int kSrcTableBytes = BK * 8;         // KSrc per contraction index of a gathered K-block
@@ -291,24 +352,39 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* tiles = smem_dyn + (base - raw);
   unsigned char* ctrl = tiles + L::kTileBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);           // full[kStages], empty[kStages], accum
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * (2 * L::kStages + 1));
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * (2 * L::kStages + 1) + 8);
+  // barriers: full[kMaxStages], empty[kMaxStages], gfull[kTailBufs], gempty[kTailBufs], accum
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);
+  constexpr int kNumBars = 2 * L::kMaxStages + 2 * kTailBufs + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * kNumBars + 8);
   RowInfo* rows = reinterpret_cast<RowInfo*>(ctrl + L::kCtrlBytes);
   KSrc* ksrc = reinterpret_cast<KSrc*>(ctrl + L::kCtrlBytes + L::kRowTableBytes);
   auto full_bar = [&](int s) { return smem_u32(bars + s); };
-  auto empty_bar = [&](int s) { return smem_u32(bars + L::kStages + s); };
-  const uint32_t accum_bar = smem_u32(bars + 2 * L::kStages);
+  auto empty_bar = [&](int s) { return smem_u32(bars + L::kMaxStages + s); };
+  auto gfull_bar = [&](int g) { return smem_u32(bars + 2 * L::kMaxStages + g); };
+  auto gempty_bar = [&](int g) { return smem_u32(bars + 2 * L::kMaxStages + kTailBufs + g); };
+  const uint32_t accum_bar = smem_u32(bars + 2 * L::kMaxStages + 2 * kTailBufs);
+  const int stages = p.num_kb > p.kb_tma_a ? L::kStagesTail : L::kStagesNoTail;
+  const uint32_t tail_base = base + stages * L::kStageBytes;   // kTailBufs A tiles (only with tail blocks)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int mt = blockIdx.x, nt = blockIdx.y, kz = blockIdx.z;
-  // this CTA's K-blocks: kz, kz + split_k, ...
+  // The CTAs of a cluster share the M tile and the K slice and differ in the N tile: they need the
+  // same assembled A tiles, so each assembles 1/CL of the rows and stores them into every peer.
+  const uint32_t crank = cluster_rank(), CL = cluster_size();
+  // this CTA's K-blocks kz, kz + split_k, ...: first those whose A tile comes by TMA, then the tail
   const int my_kb = (p.num_kb - kz + p.split_k - 1) / p.split_k;
+  const int n_tma = p.kb_tma_a > kz ? min(my_kb, (p.kb_tma_a - kz + p.split_k - 1) / p.split_k) : 0;
+  const int n_tail = my_kb - n_tma;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < L::kStages; ++s) {
-      mbar_init(full_bar(s), 1 + kGatherThreads / 32);
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
+    }
+    for (int g = 0; g < kTailBufs; ++g) {
+      mbar_init(gfull_bar(g), (kGatherThreads / 32) * CL);   // every gather warp of every CTA of the cluster
+      mbar_init(gempty_bar(g), CL);                          // every CTA's MMA issuer
     }
     mbar_init(accum_bar, 1);
     *abort_flag = 0;
@@ -319,6 +395,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), BN);
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();   // no peer touches our barriers or tiles before they are set up
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -328,12 +405,12 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       int issued = 0;
       for (int i = 0; i < my_kb; ++i) {
         const int kb = kz + i * p.split_k;
-        const int s = i % L::kStages;
-        const uint32_t par = ((i / L::kStages) & 1) ^ 1;
+        const int s = i % stages;
+        const uint32_t par = ((i / stages) & 1) ^ 1;
         if (!mbar_wait(empty_bar(s), par, abort_flag)) break;
         const uint32_t a_dst = base + s * L::kStageBytes;
         const uint32_t b_dst = a_dst + L::kABytes;
-        const bool a_tma = kb < p.kb_tma_a;
+        const bool a_tma = i < n_tma;
         mbar_arrive_expect_tx(full_bar(s), L::kBBytes + (a_tma ? p.a_box_bytes : 0));
         tma_load_2d(b_dst, &tmB, full_bar(s), kb * BK, nt * BN);
         if (a_tma) {
@@ -358,20 +435,28 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       const uint32_t idesc = instr_desc_i8(BN, p.a_signed);
+      const uint16_t all_ctas = (uint16_t)((1u << CL) - 1u);
       bool ok = true;
       for (int i = 0; i < my_kb && ok; ++i) {
-        const int s = i % L::kStages;
-        const uint32_t par = (i / L::kStages) & 1;
+        const int s = i % stages;
+        const uint32_t par = (i / stages) & 1;
         if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t a_addr = base + s * L::kStageBytes;
+        uint32_t a_addr = base + s * L::kStageBytes;
         const uint32_t b_addr = a_addr + L::kABytes;
+        const int t = i - n_tma;   // >= 0: the A tile is tail tile t, assembled by the cluster's gather warps
+        if (t >= 0) {
+          if (!mbar_wait_cluster(gfull_bar(t % kTailBufs), (uint32_t)(t / kTailBufs) & 1u, abort_flag)) { ok = false; break; }
+          a_addr = tail_base + (t % kTailBufs) * L::kABytes;
+        }
+        tc_fence_after();
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; ++k) {
           umma_i8(tmem_base, smem_desc_sw128(a_addr + k * UMMA_K), smem_desc_sw128(b_addr + k * UMMA_K), idesc,
                   (i > 0 || k > 0) ? 1u : 0u);
         }
         umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
+        // ... and tells every CTA of the cluster that this CTA is done with the tail buffer, if it is reused
+        if (t >= 0 && t + kTailBufs < n_tail) umma_commit_multicast(gempty_bar(t % kTailBufs), all_ctas);
       }
       if (ok) umma_commit(accum_bar);
     }
@@ -380,39 +465,49 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     const int gt = threadIdx.x - 64;   // 0..127
     rows[gt] = row_info(p, mt, gt);
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    // gather thread gt builds tile row gt: consecutive contraction indices of one row are close in
-    // memory (one pixel's channels), so its loads share cache lines
-    const RowInfo my_row = rows[gt];
-    const uint8_t* my_base;
-    if (p.mode == MODE_LINEAR) my_base = p.A + (my_row.out_row >= 0 ? my_row.out_row : 0) * p.lda;
-    else my_base = p.A + (((long long)my_row.n * p.H + my_row.ih0) * p.Wd + my_row.iw0) * p.C;
+    // This CTA assembles rows [crank * RP, (crank + 1) * RP) of every tail tile: RP * 8 chunks of 16
+    // bytes, dealt so that neighbouring threads work on the same rows (one pixel's channels share
+    // cache lines).  The tail buffers are separate from the TMA ring, so this starts at once and
+    // runs beside the TMA-fed main loop.
+    const int RP = BM / (int)CL;
+    const int items = RP * 8;
     bool bad = false;
     bool ok = true;
-    for (int i = 0; i < my_kb; ++i) {
-      const int kb = kz + i * p.split_k;
-      const int s = i % L::kStages;
-      const uint32_t par = ((i / L::kStages) & 1) ^ 1;
-      if (!mbar_wait(empty_bar(s), par, abort_flag)) { ok = false; break; }
-      if (kb >= p.kb_tma_a) {
-        unsigned char* a_row = tiles + s * L::kStageBytes + gt * 128;
-        // chunks of 16 original channels inside one tap move as one 16-byte load; the rest goes
-        // through the block's source table
-        const int direct_chunks = p.a_vec16 ? min(8, max(0, (p.R * p.C - kb * BK) >> 4)) : 0;
-        if (direct_chunks < 8) {  // uniform over the gather threads
-          asm volatile("bar.sync 1, 128;" ::: "memory");  // the previous block's table is no longer read
-          ksrc[gt] = k_source(p, kb * BK + gt, &bad);
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-        }
-#pragma unroll 2
-        for (int c = 0; c < 8; ++c) {
-          const uint4 v = c < direct_chunks ? direct_chunk(p, my_row, kb * BK + c * 16)
-                                            : gather_chunk(p, my_row, my_base, ksrc + c * 16);
-          *reinterpret_cast<uint4*>(a_row + ((c ^ (gt & 7)) << 4)) = v;
-        }
-        fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core
+    for (int t = 0; t < n_tail && ok; ++t) {
+      const int kb = kz + (n_tma + t) * p.split_k;
+      const int g = t % kTailBufs;
+      if (t >= kTailBufs && !mbar_wait_cluster(gempty_bar(g), (uint32_t)(t / kTailBufs - 1) & 1u, abort_flag)) {
+        ok = false;
+        break;
       }
+      // chunks of 16 original channels inside one tap move as one 16-byte load; the rest goes
+      // through the block's source table
+      const int direct_chunks = p.a_vec16 ? min(8, max(0, (p.R * p.C - kb * BK) >> 4)) : 0;
+      if (direct_chunks < 8) {  // uniform over the gather threads
+        asm volatile("bar.sync 1, 128;" ::: "memory");  // the previous block's table is no longer read
+        ksrc[gt] = k_source(p, kb * BK + gt, &bad);
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+      }
+      const uint32_t tile_local = tail_base + g * L::kABytes;
+      for (int it = gt; it < items; it += kGatherThreads) {
+        const int r = (int)crank * RP + (it >> 3), c = it & 7;
+        const RowInfo ri = rows[r];
+        uint4 v;
+        if (c < direct_chunks) {
+          v = direct_chunk(p, ri, kb * BK + c * 16);
+        } else {
+          const uint8_t* rbase;
+          if (p.mode == MODE_LINEAR) rbase = p.A + (ri.out_row >= 0 ? ri.out_row : 0) * p.lda;
+          else rbase = p.A + (((long long)ri.n * p.H + ri.ih0) * p.Wd + ri.iw0) * p.C;
+          v = gather_chunk(p, ri, rbase, ksrc + c * 16);
+        }
+        const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
+        for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), v);
+      }
+      fence_proxy_async_all();  // make the generic-proxy stores visible to the tensor cores that read them
       __syncwarp();
-      if (lane == 0) mbar_arrive(full_bar(s));
+      if (lane == 0)
+        for (uint32_t dst = 0; dst < CL; ++dst) mbar_arrive_peer(peer_addr(gfull_bar(g), dst));
     }
     if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
 
@@ -475,6 +570,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   }
 
   __syncthreads();
+  cluster_sync_all();   // no CTA leaves while a peer may still store into it or arrive on its barriers
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
@@ -553,33 +649,65 @@ bool encode_u8(CUtensorMap* map, const void* base, int rank, const cuuint64_t* d
 struct GemmPlan {
   int BN;
   int split_k;
+  int cluster;   // CTAs along N that share assembled A tiles
   int m_tiles, n_tiles;
 };
 
-GemmPlan choose_plan(int m_tiles, int N, int num_kb) {
-  GemmPlan best{64, 1, m_tiles, (N + 63) / 64};
-  double best_score = -1.0;
+// CTAs that can be resident at once for cluster sizes 1, 2, 4, 8 with one CTA per SM (B200: 148 SMs;
+// a cluster must fit inside one GPC, so larger clusters leave SMs unused).
+constexpr int kClusterSizes[4] = {1, 2, 4, 8};
+constexpr int kClusterCapacity[4] = {148, 148, 132, 120};
+constexpr int kMaxSplitCtas = 2 * kNumSMs;   // split-K never uses more than two waves of CTAs
+
+// Tile width, K split and cluster size by a small time model in units of one TMA-fed K-block of a
+// 128 x 256 tile: a wave costs max(main loop, gather beside it) plus a fixed prologue/epilogue; the
+// gather of one assembled K-block costs about `gather_cost` such units and is divided by the cluster
+// size; split-K adds the reduction pass.  n_tail = K-blocks whose A tile is assembled by threads.
+GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, bool conv) {
+  GemmPlan best{64, 1, 1, m_tiles, (N + 63) / 64};
+  double best_cost = 1e300;
   const int bns[3] = {256, 128, 64};
+  const double gather_cost = conv ? 16.0 : 40.0;
   for (int bi = 0; bi < 3; ++bi) {
     const int BN = bns[bi];
     if (BN > 64 && N <= BN / 2) continue;  // tile mostly empty
-    const long long tiles = (long long)m_tiles * ((N + BN - 1) / BN);
+    const int n_tiles = (N + BN - 1) / BN;
+    const long long tiles = (long long)m_tiles * n_tiles;
+    const double t_block = (128.0 + BN) / 384.0;
     int max_split = num_kb / 4;            // keep at least 4 K-blocks per slice
-    if (max_split < 1) max_split = 1;
+    if (max_split < 1 || tiles >= kNumSMs) max_split = 1;
     if (max_split > 32) max_split = 32;
     for (int sk = 1; sk <= max_split; ++sk) {
       const long long ctas = tiles * sk;
-      const long long waves = (ctas + kNumSMs - 1) / kNumSMs;
-      const double eff = (double)ctas / (double)(waves * kNumSMs);
-      // prefer full waves, then wide tiles, then little splitting
-      const double score = eff + 0.02 * (2 - bi) - 0.004 * (sk - 1) - (sk > 1 && tiles >= kNumSMs ? 1.0 : 0.0);
-      if (score > best_score) {
-        best_score = score;
-        best = GemmPlan{BN, sk, m_tiles, (N + BN - 1) / BN};
+      if (sk > 1 && ctas > kMaxSplitCtas) break;
+      const int main_blocks = (num_kb + sk - 1) / sk;
+      const int tail_blocks = (n_tail + sk - 1) / sk;
+      for (int ci = 0; ci < 4; ++ci) {
+        const int cl = kClusterSizes[ci];
+        if (cl > 1 && (n_tail == 0 || n_tiles % cl != 0)) continue;
+        const long long waves = (ctas + kClusterCapacity[ci] - 1) / kClusterCapacity[ci];
+        const double main_t = main_blocks * t_block;
+        const double gather_t = tail_blocks * gather_cost / cl;
+        double cost = (double)waves * ((main_t > gather_t ? main_t : gather_t) + 4.0 * t_block);
+        if (sk > 1) cost += 6.0;
+        cost *= 1.0 + 0.002 * ci + 0.001 * bi;   // ties: smaller cluster, wider tile
+        if (cost < best_cost) {
+          best_cost = cost;
+          best = GemmPlan{BN, sk, cl, m_tiles, n_tiles};
+        }
       }
     }
   }
   return best;
+}
+
+// Upper bound of the split-K scratch over every plan choose_plan can return for this output.
+size_t splitk_ws_bound(long long rows, int N, long long m_tiles) {
+  if (m_tiles * ((N + 255) / 256) >= kNumSMs) return 0;   // enough tiles: never split
+  long long ints = 32ll * rows * N;
+  const long long cap = (long long)kMaxSplitCtas * BM * 256;
+  if (ints > cap) ints = cap;
+  return 4 * (size_t)ints;
 }
 
 template <int BN>
@@ -592,9 +720,17 @@ ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const Gem
       return OCS_ERR_CUDA;
     attr_set = true;
   }
-  dim3 grid(plan.m_tiles, plan.n_tiles, plan.split_k);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(plan.m_tiles, plan.n_tiles, plan.split_k);
+  cfg.blockDim = dim3(kGemmThreads, 1, 1);
+  cfg.dynamicSmemBytes = L::kDynBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = plan.cluster; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
   LaunchScope ls(p.mode == MODE_CONV ? "ocs_gemm_kernel(conv)" : "ocs_gemm_kernel(linear)", stream);
-  ocs_gemm_kernel<BN><<<grid, kGemmThreads, L::kDynBytes, stream>>>(tmB, tmA, p);
+  if (cudaLaunchKernelEx(&cfg, ocs_gemm_kernel<BN>, tmB, tmA, p) != cudaSuccess) return OCS_ERR_CUDA;
   return launch_status();
 }
 
@@ -619,9 +755,9 @@ GemmWs carve_gemm_ws(void* ws, long long rows, int N, int split_k) {
 ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long long out_rows, int m_tiles, bool tma_a_ok,
                     const CUtensorMap* tmA_in, void* ws, size_t ws_bytes, cudaStream_t stream) {
   p.num_kb = (p.Ktot + BK - 1) / BK;
-  const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb);
-  p.split_k = plan.split_k;
   if (!tma_a_ok) p.kb_tma_a = 0;
+  const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb, p.num_kb - p.kb_tma_a, p.mode == MODE_CONV);
+  p.split_k = plan.split_k;
 
   CUtensorMap tmB;
   {
@@ -703,9 +839,7 @@ using namespace ocs;
 extern "C" size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S) {
   if (M <= 0 || N <= 0 || C <= 0 || S < 0) return 256;
   const int m_tiles = (M + BM - 1) / BM;
-  const GemmPlan plan = choose_plan(m_tiles, N, (int)(((long long)C + S + BK - 1) / BK));
-  if (plan.split_k == 1) return 256;
-  return carve_gemm_ws(nullptr, M, N, plan.split_k).total;
+  return 256 + align_up(splitk_ws_bound(M, N, m_tiles), 256);
 }
 
 extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C, int64_t lda,
@@ -787,9 +921,7 @@ extern "C" size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O,
       !conv_geom(Nb, H, Wd, kh, kw, stride, pad, &g))
     return 256;
   const long long Ktot = (long long)kh * kw * ((long long)C + S);
-  const GemmPlan plan = choose_plan((int)g.m_tiles, O, (int)((Ktot + BK - 1) / BK));
-  if (plan.split_k == 1) return 256;
-  return carve_gemm_ws(nullptr, g.out_rows, O, plan.split_k).total;
+  return 256 + align_up(splitk_ws_bound(g.out_rows, O, g.m_tiles), 256);
 }
 
 extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H, int Wd, int C,
