@@ -1,6 +1,6 @@
 """Benchmark of the OCS hot path on B200: split -> clip search -> quantize -> int8 GEMM/conv.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-small|fc] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-small|fc|conv|resnet50|lstm] [--impl reference]
 
 One step is one pass of the whole path over one batch of synthetic input:
   fc6   (default) the VGG-16-fc6-shaped sweep: W [4096, 25088], 5 expand ratios x 4 weight bit
@@ -8,6 +8,9 @@ One step is one pass of the whole path over one batch of synthetic input:
         the activation quantization and ocs_qlinear (nothing is cached between points).
   fc6-small  the same recipe on W [256, 6272] (quick checks).
   fc    the small fully-connected layer [256, 512], batch 64, r = 0.05, 8-bit, no clipping.
+  conv / resnet50 / lstm   the single 3x3 convolution, the ResNet-50 stack at batch 128 and the LSTM
+        language model: a step prepares every layer (split, quantize, pack) and runs the forward pass;
+        these report integer TOP/s of the quantized layers instead of bytes per second.
 The reported value is algorithmic bytes per second: the bytes the method must move (listed in
 `algorithmic_bytes` below) divided by the step time.  Rank 0 prints one JSON line.
 
@@ -165,18 +168,45 @@ class Fc6Sweep:
                             out=self.Y[i], ws=self.ws, dev_status=self.status)
 
     def e2e_buffers(self, host):
+        """End-to-end steps: every step's inputs travel from pinned host memory and its outputs travel
+        back.  The copy of step i+1's inputs runs on a second stream into a second pair of device
+        buffers while step i computes (one host-to-device copy of W and A per step)."""
         torch = self.torch
         self.hW = torch.from_numpy(host["W"]).pin_memory()
         self.hA = torch.from_numpy(host["A"]).pin_memory()
         self.hY = [torch.empty(y.shape, dtype=torch.float32).pin_memory() for y in self.Y]
+        self.copy_stream = torch.cuda.Stream()
+        self.Wd = [self.W, torch.empty_like(self.W)]
+        self.Ad = [self.A, torch.empty_like(self.A)]
+        self.ready = [torch.cuda.Event(), torch.cuda.Event()]
+        self.consumed = [torch.cuda.Event(), torch.cuda.Event()]
+        self.k = 0
+        torch.cuda.current_stream().synchronize()
+        for e in self.consumed:
+            e.record()
+        self._prefetch(0)
         return self.hW.numel() * 4 + self.hA.numel() * 4, sum(y.numel() * 4 for y in self.hY)
 
+    def _prefetch(self, slot):
+        torch = self.torch
+        with torch.cuda.stream(self.copy_stream):
+            self.copy_stream.wait_event(self.consumed[slot])      # the step that last read this slot is done
+            self.Wd[slot].copy_(self.hW, non_blocking=True)
+            self.Ad[slot].copy_(self.hA, non_blocking=True)
+            self.ready[slot].record(self.copy_stream)
+
     def step_e2e(self):
-        self.W.copy_(self.hW, non_blocking=True)
-        self.A.copy_(self.hA, non_blocking=True)
+        torch = self.torch
+        cur = self.k % 2
+        self._prefetch(1 - cur)                                   # next step's inputs, overlapping this step
+        main = torch.cuda.current_stream()
+        main.wait_event(self.ready[cur])
+        self.W, self.A = self.Wd[cur], self.Ad[cur]
         self.step()
+        self.consumed[cur].record(main)
         for h, y in zip(self.hY, self.Y):
             h.copy_(y, non_blocking=True)
+        self.k += 1
 
     # the CPU checker on a bounded sample of the same step
     oracle_sample_desc = "3 of the 20 sweep points on the full tensors: (r, bits) = (0.01, 4), (0.05, 6), (0.1, 8)"
@@ -261,6 +291,178 @@ class SmallFc(Fc6Sweep):
 
 
 # ----------------------------------------------------------------------------------------------
+# Whole-network workloads (configs[3], configs[4]) and the single convolution (configs[1]): reported
+# in integer TOP/s of the quantized layers, the unit of the GEMM/conv half of the metric.
+class NetWorkload:
+    kind = "net"
+    l2_note = "activations and weights of most layers fit in L2; nothing is flushed between steps"
+
+    def setup(self, ocs, torch, dev, host):
+        self.ocs, self.torch, self.dev = ocs, torch, dev
+        from paper_1901_09504_b200 import nets
+        self.nets = nets
+        self.status = ocs.new_status(dev)
+        self.dev_in = {k: torch.from_numpy(v).to(dev) for k, v in self.host_arrays().items()}
+
+    def e2e_buffers(self, host):
+        torch = self.torch
+        self.pinned = {k: torch.from_numpy(v).pin_memory() for k, v in self.host_arrays().items()}
+        out = self.step()
+        self.h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        return sum(v.numel() * v.element_size() for v in self.pinned.values()), out.numel() * out.element_size()
+
+    def step_e2e(self):
+        for k, v in self.pinned.items():
+            self.dev_in[k].copy_(v, non_blocking=True)
+        self.h_out.copy_(self.step(), non_blocking=True)
+
+
+class ResNet50(NetWorkload):
+    name = "resnet50"
+
+    def __init__(self, batch=128, image=224):
+        self.batch, self.image = batch, image
+        self.desc = (f"configs[3]: ResNet-50 conv/fc stack at random init (folded BN), batch {batch}, input "
+                     f"[{batch}, 3, {image}, {image}] fp32, OCS r = 0.01 on every layer, 8-bit weights and activations; "
+                     "a step splits, quantizes and packs all 54 layers, then runs the forward pass; seed 3")
+        self.oracle_sample_desc = "all 54 layers prepared + forward of 1 image at 64x64"
+
+    def host_inputs(self):
+        self.cfg = configs.config4(batch=self.batch, image=self.image)
+        return {}
+
+    def host_arrays(self):
+        return {"X": self.cfg["X"]}
+
+    def setup(self, ocs, torch, dev, host):
+        super().setup(ocs, torch, dev, host)
+        # the fp32 weights live on the device; preparing them (split, quantize, pack) is part of every step
+        self.Wd = {}
+        for spec in self.cfg["layers"] + [self.cfg["fc"]]:
+            W, b = self.cfg["params"][spec.name]
+            self.Wd[spec.name] = (torch.from_numpy(W).to(dev), torch.from_numpy(b).to(dev))
+        self.ops = 0
+        for spec in self.cfg["layers"]:
+            S = configs_num_splits(spec.C, self.cfg["ratio"])
+            self.ops += 2 * self.batch * spec.H_out ** 2 * spec.O * (spec.C + S) * spec.k ** 2
+        fc = self.cfg["fc"]
+        self.ops += 2 * self.batch * fc.O * (fc.C + configs_num_splits(fc.C, self.cfg["ratio"]))
+
+    def step(self):
+        nets, cfg = self.nets, self.cfg
+        layers = {}
+        for spec in cfg["layers"] + [cfg["fc"]]:
+            W, b = self.Wd[spec.name]
+            if spec.name == "fc":
+                layers["fc"] = nets.prepare_layer(W.reshape(spec.O, spec.C), b, cfg["ratio"], cfg["w_bits"],
+                                                  dev_status=self.status)
+            else:
+                layers[spec.name] = nets.prepare_layer(W, b, cfg["ratio"], cfg["w_bits"], conv=True, stride=spec.stride,
+                                                       pad=spec.pad, dev_status=self.status)
+        return nets.resnet50_forward(cfg, layers, self.dev_in["X"], dev_status=self.status)
+
+    def oracle_sample(self, orc, host):
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import net_oracle
+        small = configs.config4(batch=1, image=64)
+        t0 = time.perf_counter()
+        net_oracle.resnet50(small)
+        sec = time.perf_counter() - t0
+        ops = sum(2 * s.H_out ** 2 * s.O * (s.C + configs_num_splits(s.C, 0.01)) * s.k ** 2 for s in small["layers"])
+        return sec, ops
+
+
+class Lstm(NetWorkload):
+    name = "lstm"
+
+    def __init__(self):
+        self.desc = ("configs[4]: 2-layer LSTM language model, hidden 650, vocabulary 33278, batch 20, sequence 35, "
+                     "OCS r = 0.02 on W_ih, W_hh and the decoder, 6-bit weights, signed 8-bit activations, per-timestep "
+                     "quantized GEMMs; a step prepares the five weight matrices and runs the 35 time steps and the "
+                     "decoder; seed 4")
+        self.oracle_sample_desc = "the same model with vocabulary 3000, batch 4, 6 time steps"
+
+    def host_inputs(self):
+        self.cfg = configs.config5()
+        return {}
+
+    def host_arrays(self):
+        return {"tokens": self.cfg["tokens"]}
+
+    def setup(self, ocs, torch, dev, host):
+        super().setup(ocs, torch, dev, host)
+        self.Pd = {k: torch.from_numpy(v).to(dev) for k, v in self.cfg["params"].items()}
+        h, V = self.cfg["hidden"], self.cfg["vocab"]
+        seq, batch = self.cfg["tokens"].shape
+        S = configs_num_splits(h, self.cfg["ratio"])
+        self.ops = 2 * (h + S) * (seq * batch * 4 * h * 4 + seq * batch * V)
+
+    def step(self):
+        nets, cfg, P = self.nets, self.cfg, self.Pd
+        layers = {"emb": P["emb"]}
+        for l in range(2):
+            for nm, bn in (("W_ih", "b_ih"), ("W_hh", "b_hh")):
+                layers[f"{nm}{l}"] = nets.prepare_layer(P[f"{nm}{l}"], P[f"{bn}{l}"], cfg["ratio"], cfg["w_bits"],
+                                                        dev_status=self.status)
+        layers["W_dec"] = nets.prepare_layer(P["W_dec"], P["b_dec"], cfg["ratio"], cfg["w_bits"], dev_status=self.status)
+        return nets.lstm_forward(cfg, layers, self.dev_in["tokens"], dev_status=self.status)
+
+    def oracle_sample(self, orc, host):
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import net_oracle
+        small = configs.config5(vocab=3000, batch=4, seq=6)
+        t0 = time.perf_counter()
+        net_oracle.lstm(small)
+        sec = time.perf_counter() - t0
+        h = small["hidden"]
+        S = configs_num_splits(h, 0.02)
+        return sec, 2 * (h + S) * (6 * 4 * 4 * h * 4 + 6 * 4 * 3000)
+
+
+class Conv3x3(NetWorkload):
+    name = "conv"
+    l2_note = "everything fits in L2 (launch-bound); nothing is flushed between steps"
+
+    def __init__(self):
+        self.desc = ("configs[1]: conv 3x3 s1 p1, W [256, 256, 3, 3] fp32 (Student-t), input [32, 256, 14, 14], r = 0.02 "
+                     f"(6 splits), 6-bit weights with the MSE clip search ({N_CAND} candidates), 8-bit unsigned activations; "
+                     "a step splits, searches, quantizes, packs, converts the input layout and runs the convolution; seed 1")
+        self.oracle_sample_desc = "the same layer on 4 of the 32 images"
+
+    def host_inputs(self):
+        self.cfg = configs.config2()
+        return {}
+
+    def host_arrays(self):
+        return {"X": self.cfg["X"]}
+
+    def setup(self, ocs, torch, dev, host):
+        super().setup(ocs, torch, dev, host)
+        self.W = torch.from_numpy(self.cfg["W"]).to(dev)
+        self.ops = 2 * 32 * 14 * 14 * 256 * (256 + 6) * 9
+
+    def step(self):
+        nets, ocs = self.nets, self.ocs
+        L = nets.prepare_layer(self.W, None, 0.02, 6, ocs.CLIP_MSE, conv=True, stride=1, pad=1, dev_status=self.status)
+        x = ocs.ocs_nchw_to_nhwc(self.dev_in["X"])
+        return nets.conv_forward(L, x, a_signed=False, dev_status=self.status)
+
+    def oracle_sample(self, orc, host):
+        c = configs.config2(batch=4)
+        t0 = time.perf_counter()
+        Wp, idx, _, _ = orc.split(c["W"], 6)
+        alpha = orc.clip_mse(Wp, 6, True, N_BINS, N_CAND)["alpha"]
+        wc, ws = orc.quantize(Wp, 6, True, alpha)
+        xh = orc.nchw_to_nhwc(c["X"])
+        xc, xs = orc.quantize(xh, 8, False, orc.maxabs(xh))
+        orc.qconv(xc, False, xs, wc, ws, idx, 1, 1)
+        return time.perf_counter() - t0, 2 * 4 * 14 * 14 * 256 * (256 + 6) * 9
+
+
+NET_METRIC = "OCS quantized layers int8 TOP/s (whole step: split + quantize + pack of every layer, then the forward pass)"
+
+
+# ----------------------------------------------------------------------------------------------
 def sample_clocks_start():
     q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -311,14 +513,17 @@ def run_reference(args, wl):
         t, nbytes = wl.oracle_sample(orc, host)
         times.append(t)
     sec = sum(times) / len(times)
-    val = nbytes / sec / 1e9
-    line = dict(impl="reference", metric=METRIC, value=val, unit="GB/s", n_gpus=args.gpus, steps=args.steps,
+    net = getattr(wl, "kind", "") == "net"
+    val = nbytes / sec / (1e12 if net else 1e9)       # network workloads count integer ops, the others bytes
+    unit = "TOPS" if net else "GB/s"
+    line = dict(impl="reference", metric=NET_METRIC if net else METRIC, value=val, unit=unit, n_gpus=args.gpus,
+                steps=args.steps,
                 warmup=min(args.warmup, 1), ms_per_step=sec * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="int8 codes / int32 accumulate / fp32 scales", data="synthetic",
                 config=dict(workload=wl.desc, sample=wl.oracle_sample_desc),
-                cpu_baseline=dict(value=val, unit="GB/s", cores=orc.threads(), kind="oracle",
+                cpu_baseline=dict(value=val, unit=unit, cores=orc.threads(), kind="oracle",
                                   sample=wl.oracle_sample_desc),
-                e2e=dict(value=val, unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+                e2e=dict(value=val, unit=unit, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
 
 
@@ -330,7 +535,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-small", "fc"])
+    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-small", "fc", "conv", "resnet50", "lstm"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -339,7 +544,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    wl = {"fc6": Fc6Sweep, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc}[args.workload]()
+    wl = {"fc6": Fc6Sweep, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc, "conv": Conv3x3,
+          "resnet50": ResNet50, "lstm": Lstm}[args.workload]()
+    net = getattr(wl, "kind", "") == "net"
 
     if args.impl == "reference":
         if rank == 0:
@@ -354,8 +561,8 @@ def main():
         from oracle import oracle as orc
         orc.build()
         sec, nbytes = wl.oracle_sample(orc, host)
-        cpu = dict(value=nbytes / sec / 1e9, unit="GB/s", cores=orc.threads(), kind="oracle",
-                   sample=wl.oracle_sample_desc, seconds=sec)
+        cpu = dict(value=nbytes / sec / (1e12 if net else 1e9), unit="TOPS" if net else "GB/s", cores=orc.threads(),
+                   kind="oracle", sample=wl.oracle_sample_desc, seconds=sec)
 
     import torch
     import torch.distributed as dist
@@ -377,7 +584,9 @@ def main():
         torch.cuda.synchronize()
 
     wl.setup(ocs, torch, dev, {k: torch.from_numpy(v) for k, v in host.items()})
-    led = wl.ledger()
+    led = Ledger() if net else wl.ledger()
+    if net:
+        led.ops = wl.ops
     pk = peaks()
 
     def timed(fn, steps, warmup):
@@ -426,7 +635,8 @@ def main():
     top_cnt, top_ms = trace[top]
     int8_peak = pk["bf16_burst"] * INT8_OVER_BF16
     gemm_name = "ocs_gemm_kernel(linear)"
-    gemm_ms = trace.get(gemm_name, (0, 0.0))[1]
+    gemm_ms = sum(trace.get(k, (0, 0.0))[1] for k in ("ocs_gemm_kernel(linear)", "ocs_gemm_kernel(conv)",
+                                                     "splitk_reduce_kernel"))
     gemm_tops = (led.ops * args.steps / (gemm_ms * 1e-3) / 1e12) if gemm_ms > 0 else None
     sq_names = ("col_minmax_kernel", "split_scatter_kernel", "hist_kernel", "quantize_kernel", "maxabs_kernel")
     sq_ms = sum(trace[k][1] for k in sq_names if k in trace) + sum(
@@ -434,7 +644,16 @@ def main():
     sq_bytes = sum(led.bytes.get(k, 0) for k in sq_names) * args.steps
     sq_gbs = sq_bytes / (sq_ms * 1e-3) / 1e9 if sq_ms > 0 else None
     top_bytes = led.bytes.get(top, 0)
-    if top_bytes:
+    if net and top.startswith("ocs_gemm_kernel"):
+        # the contraction: integer ops of the step over the kernel's traced time, against the int8 peak
+        ach = led.ops * args.steps / (top_ms * 1e-3) / 1e12
+        roofline = dict(kernel=top, bound="tensor", achieved=ach, peak=int8_peak, unit="TOP/s", frac=ach / int8_peak,
+                        traffic=None, peak_source=f"{pk['source']} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16)",
+                        avg_launch_ms=top_ms / top_cnt, note="ops of every quantized layer of the step (linear and conv "
+                        "launches share one kernel); layers with few channels are bound by their output traffic, not by "
+                        "the tensor pipe",
+                        timed="second pass over the same steps with CUDA events around every kernel launch")
+    elif top_bytes:
         roof_achieved = top_bytes * args.steps / (top_ms * 1e-3) / 1e9
         roofline = dict(kernel=top, bound="hbm", achieved=roof_achieved, peak=pk["hbm"], unit="GB/s",
                         frac=roof_achieved / pk["hbm"], traffic=None, peak_source=f"of {pk['source']}",
@@ -445,14 +664,20 @@ def main():
                         avg_launch_ms=top_ms / top_cnt,
                         timed="second pass over the same steps with CUDA events around every kernel launch")
 
-    value = aggregate_gbs(led.total, world, ms_step)
+    if net:
+        scale = lambda ms: led.ops * world / (ms * 1e-3) / 1e12      # whole-job integer TOP/s
+        unit, metric = "TOPS", NET_METRIC
+    else:
+        scale = lambda ms: aggregate_gbs(led.total, world, ms)
+        unit, metric = "GB/s", METRIC
+    value = scale(ms_step)
     line = dict(
-        metric=METRIC, value=value, unit="GB/s", n_gpus=world, steps=args.steps, warmup=args.warmup,
+        metric=metric, value=value, unit=unit, n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype="int8 codes / int32 accumulate / fp32 scales", data="synthetic",
-        config=dict(workload=wl.desc, l2="inputs larger than L2 (no flush)" if wl.name == "fc6"
-                    else "inputs fit in L2; nothing is flushed between steps", bytes_per_step=led.total,
-                    int_ops_per_step=led.ops),
+        config=dict(workload=wl.desc, l2=getattr(wl, "l2_note", None) or (
+            "inputs larger than L2 (no flush)" if wl.name == "fc6" else "inputs fit in L2; nothing is flushed between steps"),
+                    bytes_per_step=led.total, int_ops_per_step=led.ops),
         parts=dict(split_quantize_gbs=sq_gbs, split_quantize_frac_of_hbm=(sq_gbs / pk["hbm"]) if sq_gbs else None,
                    gemm_tops=gemm_tops, gemm_frac_of_int8_peak=(gemm_tops / int8_peak) if gemm_tops else None,
                    int8_peak_tops=int8_peak,
@@ -461,7 +686,7 @@ def main():
         roofline=roofline,
         kernels=kernels,
         cpu_baseline=cpu,
-        e2e=dict(value=aggregate_gbs(led.total, world, ms_e2e), unit="GB/s", ms_per_step=ms_e2e,
+        e2e=dict(value=scale(ms_e2e), unit=unit, ms_per_step=ms_e2e,
                  h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h),
         gpu_launches=int(launches) * args.steps,
         clocks=clocks,
