@@ -10,10 +10,13 @@
 // rules cannot serve) are assembled in shared memory by four producer warps that read the source
 // channels through idx_map and store them in the 128-byte-swizzled layout the tensor core reads.
 //
-// One CTA = one 128 x BN output tile (x one K slice when split-K is on).  Warp roles:
-//   warp 0      TMA producer (weights always, activations when the block is TMA-able)
-//   warp 1      allocates tensor memory, issues tcgen05.mma, commits to the stage barriers
-//   warps 2..5  gather producers during the main loop, then the epilogue (tcgen05.ld -> global)
+// A work item = one 128 x BN output tile (x one K slice when split-K is on).  The grid is
+// persistent: one CTA per SM walks its share of the items.  Warp roles:
+//   warp 0      TMA producer (weights always, activations when the block is TMA-able); its ring of
+//               stages runs on across tiles
+//   warp 1      allocates tensor memory (two accumulators), issues tcgen05.mma, commits to barriers
+//   warps 2..5  gather producers: assemble the A tiles of the K-blocks that hold duplicated channels
+//   warps 6..9  epilogue (tcgen05.ld -> fmaf -> global) of tile i while the main loop of tile i+1 runs
 // The K-blocks whose A tile is assembled ("tail" blocks) come last in a CTA's K order and use two
 // dedicated A buffers, so the gather warps start at kernel begin and run ahead of the TMA-fed main
 // loop.  CTAs that share the M tile and the K slice (neighbouring N tiles) form a thread-block
@@ -31,7 +34,7 @@ namespace {
 constexpr int BM = 128;        // UMMA M
 constexpr int BK = 128;        // bytes (= int8 elements) per K-block: one 128-byte swizzle span
 constexpr int UMMA_K = 32;     // K of one tcgen05.mma.kind::i8
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 320;    // TMA warp, MMA warp, 4 gather warps, 4 epilogue warps
 constexpr int kGatherThreads = 128;
 constexpr long long kWaitCycles = 2000000000ll;  // about one second
 
@@ -54,6 +57,8 @@ struct GemmParams {
   int num_kb;
   int kb_tma_a;      // K-blocks [0, kb_tma_a) get their A tile by TMA
   int split_k;
+  // work items of the persistent grid: (K slice, M tile, group of CL neighbouring N tiles)
+  int m_tiles, n_groups, total_items;
   // epilogue
   const float* a_scale;
   const float* w_scale;
@@ -322,26 +327,48 @@ __device__ __forceinline__ uint4 direct_chunk(const GemmParams& p, const RowInfo
   return zero;
 }
 
-constexpr int kTailBufs = 2;   // A tiles assembled by the gather warps (shared across the cluster)
+constexpr int kTailBufs = 3;   // A tiles assembled by the gather warps (shared across the cluster)
 
 template <int BN>
 struct SmemLayout {
   static constexpr int kABytes = BM * BK;
   static constexpr int kBBytes = BN * BK;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  // ring depth: one stage fewer when the two tail buffers are needed
+  // ring depth: shallower when the tail buffers are needed
   static constexpr int kStagesNoTail = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int kStagesTail = kStagesNoTail - 1;
+  static constexpr int kStagesTail = (BN == 256) ? 3 : (BN == 128 ? 5 : 6);
   static constexpr int kMaxStages = kStagesNoTail;
   static constexpr int kTileBytes =
       (kStagesNoTail * kStageBytes > kStagesTail * kStageBytes + kTailBufs * kABytes)
           ? kStagesNoTail * kStageBytes : kStagesTail * kStageBytes + kTailBufs * kABytes;
   static constexpr int kCtrlBytes = 1024;               // barriers, tensor-memory slot, flags
-  static constexpr int kRowTableBytes = BM * 24;        // RowInfo per tile row
-  static constexpr int kSrcTableBytes = BK * 8;         // KSrc per contraction index of a gathered K-block
+  static constexpr int kRowTableBytes = 2 * BM * 24;    // RowInfo per tile row, two tiles
+  static constexpr int kSrcTableBytes = 2 * BK * 8;     // KSrc per contraction index, two gathered K-blocks
   static constexpr int kDynBytes =
       kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes + kSrcTableBytes;
 };
+
+// One work item of a CTA: an output tile and a K slice.
+struct WorkItem {
+  int mt, nt, kz;
+  int my_kb, n_tma, n_tail;   // K-blocks of the slice: first those with a TMA-fed A tile, then the tail
+};
+
+// Item j of this CTA's cluster (items are dealt round-robin to the clusters of the grid; the CTAs of
+// a cluster take neighbouring N tiles of the same M tile and K slice).
+__device__ __forceinline__ bool work_item(const GemmParams& p, int j, uint32_t crank, uint32_t CL, WorkItem* w) {
+  const long long idx = (long long)blockIdx.x + (long long)j * gridDim.x;
+  if (idx >= p.total_items) return false;
+  const int ntg = (int)(idx % p.n_groups);
+  const long long rest = idx / p.n_groups;
+  w->mt = (int)(rest % p.m_tiles);
+  w->kz = (int)(rest / p.m_tiles);
+  w->nt = ntg * (int)CL + (int)crank;
+  w->my_kb = (p.num_kb - w->kz + p.split_k - 1) / p.split_k;
+  w->n_tma = p.kb_tma_a > w->kz ? min(w->my_kb, (p.kb_tma_a - w->kz + p.split_k - 1) / p.split_k) : 0;
+  w->n_tail = w->my_kb - w->n_tma;
+  return true;
+}
 
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -352,9 +379,9 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* tiles = smem_dyn + (base - raw);
   unsigned char* ctrl = tiles + L::kTileBytes;
-  // barriers: full[kMaxStages], empty[kMaxStages], gfull[kTailBufs], gempty[kTailBufs], accum
+  // barriers: full[kMaxStages], empty[kMaxStages], gfull[kTailBufs], gempty[kTailBufs], acc_full[2], acc_empty[2]
   uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);
-  constexpr int kNumBars = 2 * L::kMaxStages + 2 * kTailBufs + 1;
+  constexpr int kNumBars = 2 * L::kMaxStages + 2 * kTailBufs + 4;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * kNumBars + 8);
   RowInfo* rows = reinterpret_cast<RowInfo*>(ctrl + L::kCtrlBytes);
@@ -363,19 +390,15 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   auto empty_bar = [&](int s) { return smem_u32(bars + L::kMaxStages + s); };
   auto gfull_bar = [&](int g) { return smem_u32(bars + 2 * L::kMaxStages + g); };
   auto gempty_bar = [&](int g) { return smem_u32(bars + 2 * L::kMaxStages + kTailBufs + g); };
-  const uint32_t accum_bar = smem_u32(bars + 2 * L::kMaxStages + 2 * kTailBufs);
+  auto accfull_bar = [&](int a) { return smem_u32(bars + 2 * L::kMaxStages + 2 * kTailBufs + a); };
+  auto accempty_bar = [&](int a) { return smem_u32(bars + 2 * L::kMaxStages + 2 * kTailBufs + 2 + a); };
   const int stages = p.num_kb > p.kb_tma_a ? L::kStagesTail : L::kStagesNoTail;
   const uint32_t tail_base = base + stages * L::kStageBytes;   // kTailBufs A tiles (only with tail blocks)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int mt = blockIdx.x, nt = blockIdx.y, kz = blockIdx.z;
   // The CTAs of a cluster share the M tile and the K slice and differ in the N tile: they need the
   // same assembled A tiles, so each assembles 1/CL of the rows and stores them into every peer.
   const uint32_t crank = cluster_rank(), CL = cluster_size();
-  // this CTA's K-blocks kz, kz + split_k, ...: first those whose A tile comes by TMA, then the tail
-  const int my_kb = (p.num_kb - kz + p.split_k - 1) / p.split_k;
-  const int n_tma = p.kb_tma_a > kz ? min(my_kb, (p.kb_tma_a - kz + p.split_k - 1) / p.split_k) : 0;
-  const int n_tail = my_kb - n_tma;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -386,14 +409,17 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       mbar_init(gfull_bar(g), (kGatherThreads / 32) * CL);   // every gather warp of every CTA of the cluster
       mbar_init(gempty_bar(g), CL);                          // every CTA's MMA issuer
     }
-    mbar_init(accum_bar, 1);
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accfull_bar(a), 1);    // the MMA issuer's commit
+      mbar_init(accempty_bar(a), 4);   // the four epilogue warps
+    }
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmB);
     if (p.kb_tma_a > 0) prefetch_tmap(&tmA);
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), BN);
-  tc_fence_before();
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 2 * BN);   // two accumulators: the epilogue of one tile
+  tc_fence_before();                                        // overlaps the main loop of the next
   __syncthreads();
   cluster_sync_all();   // no peer touches our barriers or tiles before they are set up
   tc_fence_after();
@@ -402,31 +428,34 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      int issued = 0;
-      for (int i = 0; i < my_kb; ++i) {
-        const int kb = kz + i * p.split_k;
-        const int s = i % stages;
-        const uint32_t par = ((i / stages) & 1) ^ 1;
-        if (!mbar_wait(empty_bar(s), par, abort_flag)) break;
-        const uint32_t a_dst = base + s * L::kStageBytes;
-        const uint32_t b_dst = a_dst + L::kABytes;
-        const bool a_tma = i < n_tma;
-        mbar_arrive_expect_tx(full_bar(s), L::kBBytes + (a_tma ? p.a_box_bytes : 0));
-        tma_load_2d(b_dst, &tmB, full_bar(s), kb * BK, nt * BN);
-        if (a_tma) {
-          if (p.mode == MODE_LINEAR) {
-            tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, mt * BM);
-          } else {
-            const int k0 = kb * BK;
-            const int tap = k0 / p.C, c0 = k0 - tap * p.C;
-            const int tw = mt % p.tiles_w, th = (mt / p.tiles_w) % p.tiles_h, tn = mt / (p.tiles_w * p.tiles_h);
-            tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw + tap % p.kw - p.pad, th * p.bh + tap / p.kw - p.pad,
-                        tn * p.bn);
+      int it = 0;   // K-blocks issued so far (the ring runs on across tiles)
+      WorkItem w;
+      bool ok = true;
+      for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
+        for (int i = 0; i < w.my_kb; ++i, ++it) {
+          const int kb = w.kz + i * p.split_k;
+          const int s = it % stages;
+          const uint32_t par = ((it / stages) & 1) ^ 1;
+          if (!mbar_wait(empty_bar(s), par, abort_flag)) { ok = false; break; }
+          const uint32_t a_dst = base + s * L::kStageBytes;
+          const uint32_t b_dst = a_dst + L::kABytes;
+          const bool a_tma = i < w.n_tma;
+          mbar_arrive_expect_tx(full_bar(s), L::kBBytes + (a_tma ? p.a_box_bytes : 0));
+          tma_load_2d(b_dst, &tmB, full_bar(s), kb * BK, w.nt * BN);
+          if (a_tma) {
+            if (p.mode == MODE_LINEAR) {
+              tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, w.mt * BM);
+            } else {
+              const int k0 = kb * BK;
+              const int tap = k0 / p.C, c0 = k0 - tap * p.C;
+              const int tw = w.mt % p.tiles_w, th = (w.mt / p.tiles_w) % p.tiles_h, tn = w.mt / (p.tiles_w * p.tiles_h);
+              tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw + tap % p.kw - p.pad, th * p.bh + tap / p.kw - p.pad,
+                          tn * p.bn);
+            }
           }
         }
-        ++issued;
       }
-      if (*abort_flag && issued > 0) {
+      if (*abort_flag && it > 0) {
         // give copies that are still in flight time to land before the CTA's shared memory is released
         for (int i = 0; i < 2000; ++i) __nanosleep(100);
       }
@@ -436,95 +465,141 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     if (lane == 0) {
       const uint32_t idesc = instr_desc_i8(BN, p.a_signed);
       const uint16_t all_ctas = (uint16_t)((1u << CL) - 1u);
+      WorkItem w;
+      int total_tail = 0;   // tail tiles this CTA consumes over all its items
+      for (int j = 0; work_item(p, j, crank, CL, &w); ++j) total_tail += w.n_tail;
+      int it = 0, tt = 0;
       bool ok = true;
-      for (int i = 0; i < my_kb && ok; ++i) {
-        const int s = i % stages;
-        const uint32_t par = (i / stages) & 1;
-        if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
-        uint32_t a_addr = base + s * L::kStageBytes;
-        const uint32_t b_addr = a_addr + L::kABytes;
-        const int t = i - n_tma;   // >= 0: the A tile is tail tile t, assembled by the cluster's gather warps
-        if (t >= 0) {
-          if (!mbar_wait_cluster(gfull_bar(t % kTailBufs), (uint32_t)(t / kTailBufs) & 1u, abort_flag)) { ok = false; break; }
-          a_addr = tail_base + (t % kTailBufs) * L::kABytes;
-        }
+      for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
+        const int acc = j & 1;
+        // the epilogue has drained this accumulator (two tiles ago)
+        if (!mbar_wait(accempty_bar(acc), (((uint32_t)j >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int i = 0; i < w.my_kb; ++i, ++it) {
+          const int s = it % stages;
+          const uint32_t par = (it / stages) & 1;
+          if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
+          uint32_t a_addr = base + s * L::kStageBytes;
+          const uint32_t b_addr = a_addr + L::kABytes;
+          const bool tail = i >= w.n_tma;   // the A tile is assembled by the cluster's gather warps
+          if (tail) {
+            if (!mbar_wait_cluster(gfull_bar(tt % kTailBufs), (uint32_t)(tt / kTailBufs) & 1u, abort_flag)) { ok = false; break; }
+            a_addr = tail_base + (tt % kTailBufs) * L::kABytes;
+          }
+          tc_fence_after();
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k) {
-          umma_i8(tmem_base, smem_desc_sw128(a_addr + k * UMMA_K), smem_desc_sw128(b_addr + k * UMMA_K), idesc,
-                  (i > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            umma_i8(d_tmem, smem_desc_sw128(a_addr + k * UMMA_K), smem_desc_sw128(b_addr + k * UMMA_K), idesc,
+                    (i > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
+          if (tail) {
+            // ... and tells every CTA of the cluster that this CTA is done with the tail buffer, if it is reused
+            if (tt + kTailBufs < total_tail) umma_commit_multicast(gempty_bar(tt % kTailBufs), all_ctas);
+            ++tt;
+          }
         }
-        umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
-        // ... and tells every CTA of the cluster that this CTA is done with the tail buffer, if it is reused
-        if (t >= 0 && t + kTailBufs < n_tail) umma_commit_multicast(gempty_bar(t % kTailBufs), all_ctas);
+        if (ok) umma_commit(accfull_bar(acc));
       }
-      if (ok) umma_commit(accum_bar);
     }
-  } else {
-    // ---------------------------------------------------------------- gather producers, then epilogue
-    const int gt = threadIdx.x - 64;   // 0..127
-    rows[gt] = row_info(p, mt, gt);
-    asm volatile("bar.sync 1, 128;" ::: "memory");
+  } else if (warp < 6) {
+    // ---------------------------------------------------------------- gather producers
     // This CTA assembles rows [crank * RP, (crank + 1) * RP) of every tail tile: RP * 8 chunks of 16
     // bytes, dealt so that neighbouring threads work on the same rows (one pixel's channels share
-    // cache lines).  The tail buffers are separate from the TMA ring, so this starts at once and
-    // runs beside the TMA-fed main loop.
+    // cache lines).  The tail buffers are separate from the TMA ring, so the gather runs ahead of
+    // the TMA-fed main loop (also across tiles).
+    const int gt = threadIdx.x - 64;   // 0..127
     const int RP = BM / (int)CL;
-    const int items = RP * 8;
     bool bad = false;
     bool ok = true;
-    for (int t = 0; t < n_tail && ok; ++t) {
-      const int kb = kz + (n_tma + t) * p.split_k;
-      const int g = t % kTailBufs;
-      if (t >= kTailBufs && !mbar_wait_cluster(gempty_bar(g), (uint32_t)(t / kTailBufs - 1) & 1u, abort_flag)) {
-        ok = false;
-        break;
-      }
-      // chunks of 16 original channels inside one tap move as one 16-byte load; the rest goes
-      // through the block's source table
-      const int direct_chunks = p.a_vec16 ? min(8, max(0, (p.R * p.C - kb * BK) >> 4)) : 0;
-      if (direct_chunks < 8) {  // uniform over the gather threads
-        asm volatile("bar.sync 1, 128;" ::: "memory");  // the previous block's table is no longer read
-        ksrc[gt] = k_source(p, kb * BK + gt, &bad);
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-      }
-      const uint32_t tile_local = tail_base + g * L::kABytes;
-      for (int it = gt; it < items; it += kGatherThreads) {
-        const int r = (int)crank * RP + (it >> 3), c = it & 7;
-        const RowInfo ri = rows[r];
-        uint4 v;
-        if (c < direct_chunks) {
-          v = direct_chunk(p, ri, kb * BK + c * 16);
-        } else {
-          const uint8_t* rbase;
-          if (p.mode == MODE_LINEAR) rbase = p.A + (ri.out_row >= 0 ? ri.out_row : 0) * p.lda;
-          else rbase = p.A + (((long long)ri.n * p.H + ri.ih0) * p.Wd + ri.iw0) * p.C;
-          v = gather_chunk(p, ri, rbase, ksrc + c * 16);
+    int tt = 0;          // tail tiles assembled so far
+    int n_tiles_done = 0;
+    int table_kb[2] = {-1, -1};   // which K-block each of the two source tables describes
+    WorkItem w;
+    for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
+      if (w.n_tail == 0) continue;
+      // row table of this tile (two tables alternate, so the previous tile's may still be in use)
+      RowInfo* trow = rows + (n_tiles_done & 1) * BM;
+      ++n_tiles_done;
+      trow[gt] = row_info(p, w.mt, gt);
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int t = 0; t < w.n_tail; ++t, ++tt) {
+        const int kb = w.kz + (w.n_tma + t) * p.split_k;
+        const int g = tt % kTailBufs;
+        if (tt >= kTailBufs && !mbar_wait_cluster(gempty_bar(g), (uint32_t)(tt / kTailBufs - 1) & 1u, abort_flag)) {
+          ok = false;
+          break;
         }
-        const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
-        for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), v);
+        // Chunks of 16 original channels inside one tap move as one 16-byte load; chunks past the
+        // last contraction index are zero; the rest goes through the block's source table, which
+        // is kept while the same K-block recurs (every tile of a layer has the same tail blocks).
+        const int direct_chunks = p.a_vec16 ? min(8, max(0, (p.R * p.C - kb * BK) >> 4)) : 0;
+        const int valid_chunks = min(8, (p.Ktot - kb * BK + 15) >> 4);
+        const KSrc* tab = ksrc + (t & 1) * BK;
+        if (direct_chunks < valid_chunks && table_kb[t & 1] != kb) {  // uniform over the gather threads
+          asm volatile("bar.sync 1, 128;" ::: "memory");  // nobody still reads the table being replaced
+          ksrc[(t & 1) * BK + gt] = k_source(p, kb * BK + gt, &bad);
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          table_kb[t & 1] = kb;
+        }
+        const uint32_t tile_local = tail_base + g * L::kABytes;
+        // (row, chunk) pairs with data, dealt evenly over the threads
+        const int n_valid = RP * valid_chunks;
+#pragma unroll 2
+        for (int it = gt; it < n_valid; it += kGatherThreads) {
+          const int rl = it / valid_chunks, c = it - rl * valid_chunks;
+          const int r = (int)crank * RP + rl;
+          const RowInfo ri = trow[r];
+          uint4 v;
+          if (ri.out_row < 0) {
+            v = make_uint4(0u, 0u, 0u, 0u);   // padding row
+          } else if (c < direct_chunks) {
+            v = direct_chunk(p, ri, kb * BK + c * 16);
+          } else {
+            const uint8_t* rbase;
+            if (p.mode == MODE_LINEAR) rbase = p.A + ri.out_row * p.lda;
+            else rbase = p.A + (((long long)ri.n * p.H + ri.ih0) * p.Wd + ri.iw0) * p.C;
+            v = gather_chunk(p, ri, rbase, tab + c * 16);
+          }
+          const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
+          for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), v);
+        }
+        // the K padding
+        const int zero_chunks = 8 - valid_chunks;
+        for (int it = gt; it < RP * zero_chunks; it += kGatherThreads) {
+          const int rl = it / zero_chunks, c = valid_chunks + (it - rl * zero_chunks);
+          const int r = (int)crank * RP + rl;
+          const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
+          for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), make_uint4(0u, 0u, 0u, 0u));
+        }
+        fence_proxy_async_all();  // make the generic-proxy stores visible to the tensor cores that read them
+        __syncwarp();
+        if (lane == 0)
+          for (uint32_t dst = 0; dst < CL; ++dst) mbar_arrive_peer(peer_addr(gfull_bar(g), dst));
       }
-      fence_proxy_async_all();  // make the generic-proxy stores visible to the tensor cores that read them
-      __syncwarp();
-      if (lane == 0)
-        for (uint32_t dst = 0; dst < CL; ++dst) mbar_arrive_peer(peer_addr(gfull_bar(g), dst));
     }
     if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
-
-    // epilogue: warp w may read tensor-memory lanes 32*(w%4) .. +31
-    if (ok) ok = mbar_wait(accum_bar, 0, abort_flag);
+  } else {
+    // ---------------------------------------------------------------- epilogue (tcgen05.ld -> global)
+    // warp w may read tensor-memory lanes 32*(w%4) .. +31
     const int q = warp & 3;
     const float sc = __fmul_rn(__ldg(p.a_scale), __ldg(p.w_scale));
     const bool direct = p.split_k == 1;
-    if (ok) {
+    WorkItem w;
+    bool ok = true;
+    for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
+      const int acc = j & 1;
+      if (!mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const RowInfo ri = rows[q * 32 + lane];
+      const RowInfo ri = row_info(p, w.mt, q * 32 + lane);
+      const int nt = w.nt, kz = w.kz;
       for (int c0 = 0; c0 < BN; c0 += 32) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
         uint32_t v[32];
         __syncwarp();
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
         if (ri.out_row >= 0) {
           if (direct) {
             float* y = p.Y + ri.out_row * p.ldy + n0;
@@ -532,39 +607,43 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             const bool vec = (n0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(y) & 15) == 0);
             if (vec) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 4) {
+              for (int jj = 0; jj < 32; jj += 4) {
                 float4 o;
-                o.x = fmaf((float)(int)v[j + 0], sc, p.bias ? __ldg(p.bias + n0 + j + 0) : 0.0f);
-                o.y = fmaf((float)(int)v[j + 1], sc, p.bias ? __ldg(p.bias + n0 + j + 1) : 0.0f);
-                o.z = fmaf((float)(int)v[j + 2], sc, p.bias ? __ldg(p.bias + n0 + j + 2) : 0.0f);
-                o.w = fmaf((float)(int)v[j + 3], sc, p.bias ? __ldg(p.bias + n0 + j + 3) : 0.0f);
-                *reinterpret_cast<float4*>(y + j) = o;
+                o.x = fmaf((float)(int)v[jj + 0], sc, p.bias ? __ldg(p.bias + n0 + jj + 0) : 0.0f);
+                o.y = fmaf((float)(int)v[jj + 1], sc, p.bias ? __ldg(p.bias + n0 + jj + 1) : 0.0f);
+                o.z = fmaf((float)(int)v[jj + 2], sc, p.bias ? __ldg(p.bias + n0 + jj + 2) : 0.0f);
+                o.w = fmaf((float)(int)v[jj + 3], sc, p.bias ? __ldg(p.bias + n0 + jj + 3) : 0.0f);
+                *reinterpret_cast<float4*>(y + jj) = o;
               }
             } else {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (n0 + j < p.N) y[j] = fmaf((float)(int)v[j], sc, p.bias ? __ldg(p.bias + n0 + j) : 0.0f);
+              for (int jj = 0; jj < 32; ++jj)
+                if (n0 + jj < p.N) y[jj] = fmaf((float)(int)v[jj], sc, p.bias ? __ldg(p.bias + n0 + jj) : 0.0f);
             }
             if (ao) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (n0 + j < p.N) ao[j] = (int)v[j];
+              for (int jj = 0; jj < 32; ++jj)
+                if (n0 + jj < p.N) ao[jj] = (int)v[jj];
             }
           } else {
             // this slice's partial sums, [kz][row][n]
             int32_t* part = p.acc_ws + ((long long)kz * p.out_rows + ri.out_row) * p.N + n0;
             if ((n0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(part) & 15) == 0)) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                __stcg(reinterpret_cast<int4*>(part + j), make_int4((int)v[j], (int)v[j + 1], (int)v[j + 2], (int)v[j + 3]));
+              for (int jj = 0; jj < 32; jj += 4)
+                __stcg(reinterpret_cast<int4*>(part + jj), make_int4((int)v[jj], (int)v[jj + 1], (int)v[jj + 2], (int)v[jj + 3]));
             } else {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (n0 + j < p.N) __stcg(part + j, (int)v[j]);
+              for (int jj = 0; jj < 32; ++jj)
+                if (n0 + jj < p.N) __stcg(part + jj, (int)v[jj]);
             }
           }
         }
       }
+      // the accumulator has been read out: hand it back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(accempty_bar(acc));
     }
     tc_fence_before();
   }
@@ -574,7 +653,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, BN);
+    tmem_dealloc(tmem_base, 2 * BN);
   }
   if (threadIdx.x == 0 && *abort_flag) flag(p.dev_status, OCS_DEV_TIMEOUT);
 }
@@ -720,8 +799,13 @@ ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const Gem
       return OCS_ERR_CUDA;
     attr_set = true;
   }
+  // persistent grid: as many clusters as fit on the device at once (or fewer, if there is less work)
+  int ci = 0;
+  while (ci < 3 && kClusterSizes[ci] != plan.cluster) ++ci;
+  const long long slots = kClusterCapacity[ci] / plan.cluster;
+  const long long n_clusters = p.total_items < slots ? p.total_items : slots;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(plan.m_tiles, plan.n_tiles, plan.split_k);
+  cfg.gridDim = dim3((unsigned)n_clusters, plan.cluster, 1);
   cfg.blockDim = dim3(kGemmThreads, 1, 1);
   cfg.dynamicSmemBytes = L::kDynBytes;
   cfg.stream = stream;
@@ -758,6 +842,9 @@ ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long lo
   if (!tma_a_ok) p.kb_tma_a = 0;
   const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb, p.num_kb - p.kb_tma_a, p.mode == MODE_CONV);
   p.split_k = plan.split_k;
+  p.m_tiles = plan.m_tiles;
+  p.n_groups = plan.n_tiles / plan.cluster;
+  p.total_items = (int)((long long)plan.m_tiles * p.n_groups * plan.split_k);
 
   CUtensorMap tmB;
   {
