@@ -449,8 +449,8 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
               const int k0 = kb * BK;
               const int tap = k0 / p.C, c0 = k0 - tap * p.C;
               const int tw = w.mt % p.tiles_w, th = (w.mt / p.tiles_w) % p.tiles_h, tn = w.mt / (p.tiles_w * p.tiles_h);
-              tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw + tap % p.kw - p.pad, th * p.bh + tap / p.kw - p.pad,
-                          tn * p.bn);
+              tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw * p.stride + tap % p.kw - p.pad,
+                          th * p.bh * p.stride + tap / p.kw - p.pad, tn * p.bn);
             }
           }
         }
@@ -715,11 +715,14 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// elem_strides (nullable): traversal stride per dimension; a box extent of N * stride then delivers N elements
 bool encode_u8(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-               const cuuint32_t* box) {
+               const cuuint32_t* box, const cuuint32_t* elem_strides = nullptr) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  if (elem_strides)
+    for (int i = 0; i < rank; ++i) estr[i] = elem_strides[i];
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box,
             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -1041,16 +1044,18 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = O; p.acc_out = acc_out;
   p.dev_status = dev_status;
 
-  // TMA serves the K-blocks that lie inside one tap's original channels: stride 1 and C % 128 == 0
+  // TMA serves the K-blocks that lie inside one tap's original channels (C % 128 == 0); a strided
+  // convolution walks the image with the tensor map's traversal stride
   CUtensorMap tmA;
-  bool tma_ok = (stride == 1) && (C % BK == 0) && aligned(X_codes, 16);
+  bool tma_ok = (C % BK == 0) && aligned(X_codes, 16) && stride <= 8 && g.bw * stride <= 256 && g.bh * stride <= 256;
   p.kb_tma_a = tma_ok ? (kh * kw * C) / BK : 0;
   p.a_box_bytes = g.bw * g.bh * g.bn * BK;
   if (tma_ok) {
     const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)Wd, (cuuint64_t)H, (cuuint64_t)Nb};
     const cuuint64_t strides[3] = {(cuuint64_t)C, (cuuint64_t)C * Wd, (cuuint64_t)C * Wd * H};
-    const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)g.bw, (cuuint32_t)g.bh, (cuuint32_t)g.bn};
-    if (!encode_u8(&tmA, X_codes, 4, dims, strides, box)) return OCS_ERR_CUDA;
+    const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)(g.bw * stride), (cuuint32_t)(g.bh * stride), (cuuint32_t)g.bn};
+    const cuuint32_t estr[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
+    if (!encode_u8(&tmA, X_codes, 4, dims, strides, box, estr)) return OCS_ERR_CUDA;
   }
   return run_gemm(p, W_packed, ldw, g.out_rows, (int)g.m_tiles, tma_ok, &tmA, ws, ws_bytes, stream);
 }
