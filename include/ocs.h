@@ -186,9 +186,14 @@ ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, 
 /* ocs_pack_conv_weights -------------------------------------------------------------------
  * Reorders quantized conv weights from the split's layout [O][C+S][kh*kw] (row stride
  * ld_src bytes) into the contraction order ocs_qconv consumes: for each output o, first the
- * C original channels of every tap, k = tap*C + c, then the S duplicated channels of every
- * tap, k = kh*kw*C + tap*S + s; row stride ld_dst bytes (multiple of 16), bytes between the
- * last k and ld_dst set to zero.  A pure permutation of Eq. 3's terms. */
+ * C original channels of every tap, k = tap*Cp + c, then the S duplicated channels of every
+ * tap, k = kh*kw*Cp + tap*S + s.  Cp is the per-tap stride: C, except that a C that is a
+ * multiple of 16 but not of 128 is padded up to the next multiple of 128 (zero weights), so
+ * that the activation tiles of such layers can be fetched as whole tiles.  Row stride ld_dst
+ * bytes (multiple of 16, at least ocs_conv_packed_k); bytes between the last k and ld_dst are
+ * set to zero.  A pure permutation (plus zero padding) of Eq. 3's terms.
+ * ocs_conv_packed_k (host): the packed contraction length kh*kw*(Cp + S). */
+int64_t ocs_conv_packed_k(int C, int S, int kh, int kw);
 ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, int S, int kh, int kw,
                                  int64_t ld_src, int8_t* packed, int64_t ld_dst, void* stream);
 

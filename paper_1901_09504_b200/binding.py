@@ -28,7 +28,7 @@ EXPORTS = [
     "ocs_split_workspace_bytes", "ocs_split",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
-    "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
+    "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
     "ocs_add_relu", "ocs_maxpool3x3s2", "ocs_global_avgpool", "ocs_nchw_to_nhwc", "ocs_embedding", "ocs_lstm_cell",
 ]
 
@@ -55,6 +55,7 @@ def lib():
             getattr(L, name).restype = C.c_size_t
         L.ocs_quantize_workspace_views.restype = None
         L.ocs_kernel_launches.restype = C.c_longlong
+        L.ocs_conv_packed_k.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -210,10 +211,15 @@ def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, 
     return (Y, acc) if want_acc else Y
 
 
+def ocs_conv_packed_k(C_in: int, S: int, kh: int, kw: int) -> int:
+    """Contraction length of the packed conv weights (taps may be padded to the K-block)."""
+    return int(lib().ocs_conv_packed_k(int(C_in), int(S), int(kh), int(kw)))
+
+
 def ocs_pack_conv_weights(codes, O: int, C_in: int, S: int, kh: int, kw: int, ld_dst: int | None = None, out=None):
     """codes int8 [O, ld_src] in [C+S][kh*kw] order per row -> packed int8 [O, ld_dst]."""
     assert codes.is_cuda and codes.dtype == torch.int8 and codes.dim() == 2 and codes.stride(1) == 1
-    Kt = kh * kw * (C_in + S)
+    Kt = ocs_conv_packed_k(C_in, S, kh, kw)
     if ld_dst is None:
         ld_dst = round_up(Kt, 16)
     if out is not None:

@@ -44,6 +44,7 @@ struct GemmParams {
   int mode;
   int M, N, Ktot;   // Ktot = number of valid contraction indices
   int C, S, R;
+  int Cp;            // contraction indices one filter tap occupies: C, or C padded to a K-block (see conv_tap_stride)
   const uint8_t* A;  // linear: [M][lda] ; conv: NHWC codes
   long long lda;
   int a_signed;
@@ -281,10 +282,14 @@ __device__ __forceinline__ KSrc k_source(const GemmParams& p, int k, bool* bad) 
     return e;
   }
   // convolution: contraction order is [tap][c < C] then [tap][s < S]
-  const int KO = p.R * p.C;
+  const int KO = p.R * p.Cp;
   int tap, c;
-  if (k < KO) { tap = k / p.C; c = k - tap * p.C; }
-  else { const int kd = k - KO; tap = kd / p.S; c = checked_src(p, p.C + (kd - tap * p.S), bad); }
+  if (k < KO) {
+    tap = k / p.Cp; c = k - tap * p.Cp;
+    if (c >= p.C) return e;   // padding between taps
+  } else {
+    const int kd = k - KO; tap = kd / p.S; c = checked_src(p, p.C + (kd - tap * p.S), bad);
+  }
   const int dy = tap / p.kw, dx = tap - dy * p.kw;
   e.off = (dy * p.Wd + dx) * p.C + c;
   e.dydx = dy | (dx << 8);
@@ -320,9 +325,9 @@ __device__ __forceinline__ uint4 direct_chunk(const GemmParams& p, const RowInfo
   const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
   if (ri.out_row < 0) return zero;
   if (p.mode == MODE_LINEAR) return __ldg(reinterpret_cast<const uint4*>(p.A + ri.out_row * p.lda + k0));
-  const int tap = k0 / p.C, c0 = k0 - tap * p.C;
+  const int tap = k0 / p.Cp, c0 = k0 - tap * p.Cp;
   const int ih = ri.ih0 + tap / p.kw, iw = ri.iw0 + tap % p.kw;
-  if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd)
+  if (c0 < p.C && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd)
     return __ldg(reinterpret_cast<const uint4*>(p.A + (((long long)ri.n * p.H + ih) * p.Wd + iw) * p.C + c0));
   return zero;
 }
@@ -447,7 +452,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
               tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, w.mt * BM);
             } else {
               const int k0 = kb * BK;
-              const int tap = k0 / p.C, c0 = k0 - tap * p.C;
+              const int tap = k0 / p.Cp, c0 = k0 - tap * p.Cp;
               const int tw = w.mt % p.tiles_w, th = (w.mt / p.tiles_w) % p.tiles_h, tn = w.mt / (p.tiles_w * p.tiles_h);
               tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw * p.stride + tap % p.kw - p.pad,
                           th * p.bh * p.stride + tap / p.kw - p.pad, tn * p.bn);
@@ -534,7 +539,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         // Chunks of 16 original channels inside one tap move as one 16-byte load; chunks past the
         // last contraction index are zero; the rest goes through the block's source table, which
         // is kept while the same K-block recurs (every tile of a layer has the same tail blocks).
-        const int direct_chunks = p.a_vec16 ? min(8, max(0, (p.R * p.C - kb * BK) >> 4)) : 0;
+        const int direct_chunks = p.a_vec16 ? min(8, max(0, (p.R * p.Cp - kb * BK) >> 4)) : 0;
         const int valid_chunks = min(8, (p.Ktot - kb * BK + 15) >> 4);
         const KSrc* tab = ksrc + (t & 1) * BK;
         if (direct_chunks < valid_chunks && table_kb[t & 1] != kb) {  // uniform over the gather threads
@@ -903,19 +908,25 @@ void choose_conv_box(int Wo, int Ho, int Nb, int* bw_o, int* bh_o, int* bn_o) {
   *bw_o = bbw; *bh_o = bbh; *bn_o = bbn;
 }
 
-__global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, int S, int R, long long ld_src,
+// Contraction indices one filter tap occupies in the packed weights: C, except that a channel count
+// that is a multiple of 16 but not of the K-block is padded up to the K-block, so that every K-block
+// lies inside one tap and its activation tile can come by TMA (the padding multiplies zero weights
+// with zero-filled out-of-range channels).
+int conv_tap_stride(int C) { return (C % 16 == 0 && C % BK != 0) ? (C + BK - 1) / BK * BK : C; }
+
+__global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, int Cp, int S, int R, long long ld_src,
                                  int8_t* __restrict__ dst, long long ld_dst) {
   const long long total = (long long)O * ld_dst;
-  const int KO = R * C, Kt = R * (C + S);
+  const int KO = R * Cp, Kt = KO + R * S;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
     const long long o = i / ld_dst;
     const int k = (int)(i - o * ld_dst);
     int8_t v = 0;
     if (k < Kt) {
       int tap, j;
-      if (k < KO) { tap = k / C; j = k - tap * C; }
+      if (k < KO) { tap = k / Cp; j = k - tap * Cp; }
       else { const int kd = k - KO; tap = kd / S; j = C + (kd - tap * S); }
-      v = src[o * ld_src + (long long)j * R + tap];
+      if (k >= KO || j < C) v = src[o * ld_src + (long long)j * R + tap];
     }
     dst[i] = v;
   }
@@ -949,7 +960,7 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
 
   GemmParams p{};
   p.mode = MODE_LINEAR;
-  p.M = M; p.N = N; p.Ktot = (int)Ktot; p.C = C; p.S = S; p.R = 1;
+  p.M = M; p.N = N; p.Ktot = (int)Ktot; p.C = C; p.Cp = C; p.S = S; p.R = 1;
   p.A = reinterpret_cast<const uint8_t*>(A_codes); p.lda = lda; p.a_signed = a_signed ? 1 : 0;
   p.idx_map = idx_map;
   p.a_vec16 = (lda % 16 == 0) && aligned(A_codes, 16);
@@ -969,19 +980,25 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
   return run_gemm(p, W_codes, ldw, M, m_tiles, tma_ok, &tmA, ws, ws_bytes, stream);
 }
 
+extern "C" int64_t ocs_conv_packed_k(int C, int S, int kh, int kw) {
+  if (C <= 0 || S < 0 || kh <= 0 || kw <= 0) return 0;
+  return (int64_t)kh * kw * ((int64_t)conv_tap_stride(C) + S);
+}
+
 extern "C" ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, int S, int kh, int kw, int64_t ld_src,
                                             int8_t* packed, int64_t ld_dst, void* stream_) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!codes || !packed || S < 0) return OCS_ERR_INVALID_ARG;
   if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0) return OCS_ERR_SHAPE;
-  const long long Kt = (long long)kh * kw * ((long long)C + S);
-  if (ld_src < Kt || ld_dst < Kt || ld_dst % 16 != 0 || Kt >= (1ll << 31)) return OCS_ERR_SHAPE;
+  const long long Ksrc = (long long)kh * kw * ((long long)C + S);
+  const long long Kt = (long long)kh * kw * ((long long)conv_tap_stride(C) + S);
+  if (ld_src < Ksrc || ld_dst < Kt || ld_dst % 16 != 0 || Kt >= (1ll << 31)) return OCS_ERR_SHAPE;
   ocs_status st = check_device();
   if (st != OCS_OK) return st;
   const long long total = (long long)O * ld_dst;
   const int grid = (int)((total + 255) / 256 < kNumSMs * 8 ? (total + 255) / 256 : kNumSMs * 8);
   LaunchScope ls("pack_conv_kernel", stream);
-  pack_conv_kernel<<<grid, 256, 0, stream>>>(codes, O, C, S, kh * kw, ld_src, packed, ld_dst);
+  pack_conv_kernel<<<grid, 256, 0, stream>>>(codes, O, C, conv_tap_stride(C), S, kh * kw, ld_src, packed, ld_dst);
   return launch_status();
 }
 
@@ -1023,7 +1040,8 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   if (S < 0) return OCS_ERR_INVALID_ARG;
   if (Nb <= 0 || H <= 0 || Wd <= 0 || C <= 0 || O <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
     return OCS_ERR_SHAPE;
-  const long long Ktot = (long long)kh * kw * ((long long)C + S);
+  const int Cp = conv_tap_stride(C);
+  const long long Ktot = (long long)kh * kw * ((long long)Cp + S);   // packed contraction length (ocs_conv_packed_k)
   if (ldw < Ktot || ldw % 16 != 0 || !aligned(W_packed, 16) || !aligned(Y, 4)) return OCS_ERR_SHAPE;
   if (Ktot * 255ll * 127ll > 2147483647ll) return OCS_ERR_UNSUPPORTED;
   ConvGeom g;
@@ -1035,7 +1053,7 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   GemmParams p{};
   p.mode = MODE_CONV;
   p.M = (int)(g.out_rows < (1ll << 31) ? g.out_rows : 0x7fffffff);
-  p.N = O; p.Ktot = (int)Ktot; p.C = C; p.S = S; p.R = kh * kw;
+  p.N = O; p.Ktot = (int)Ktot; p.C = C; p.Cp = Cp; p.S = S; p.R = kh * kw;
   p.A = reinterpret_cast<const uint8_t*>(X_codes); p.lda = C; p.a_signed = a_signed ? 1 : 0;
   p.idx_map = idx_map;
   p.a_vec16 = (C % 16 == 0) && aligned(X_codes, 16);
@@ -1044,11 +1062,12 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = O; p.acc_out = acc_out;
   p.dev_status = dev_status;
 
-  // TMA serves the K-blocks that lie inside one tap's original channels (C % 128 == 0); a strided
-  // convolution walks the image with the tensor map's traversal stride
+  // TMA serves the K-blocks of original channels: each lies inside one tap (the per-tap stride Cp is a
+  // multiple of the K-block; channels past C read as zero); a strided convolution walks the image
+  // with the tensor map's traversal stride
   CUtensorMap tmA;
-  bool tma_ok = (C % BK == 0) && aligned(X_codes, 16) && stride <= 8 && g.bw * stride <= 256 && g.bh * stride <= 256;
-  p.kb_tma_a = tma_ok ? (kh * kw * C) / BK : 0;
+  bool tma_ok = (Cp % BK == 0) && aligned(X_codes, 16) && stride <= 8 && g.bw * stride <= 256 && g.bh * stride <= 256;
+  p.kb_tma_a = tma_ok ? (kh * kw * Cp) / BK : 0;
   p.a_box_bytes = g.bw * g.bh * g.bn * BK;
   if (tma_ok) {
     const cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)Wd, (cuuint64_t)H, (cuuint64_t)Nb};

@@ -101,8 +101,11 @@ def _check_conv(seed, Nb, H, Wd_, Cn, O, S, k, stride, pad, a_signed=False):
     Yo, acco = orc.qconv(X, a_signed, 0.02, Wc, 0.003, idx, stride, pad, b)
     packed = ocs.ocs_pack_conv_weights(dev(Wc.reshape(O, -1)), O, Cn, S, k, k)
     # the packing is a pure permutation: check it against numpy
-    ref_pack = np.concatenate([Wc[:, :Cn].transpose(0, 2, 3, 1).reshape(O, -1),
-                               Wc[:, Cn:].transpose(0, 2, 3, 1).reshape(O, -1)], axis=1)
+    Cp = ocs.ocs_conv_packed_k(Cn, 0, 1, 1)          # per-tap stride: C, or C padded to the K-block
+    orig = np.zeros((O, k, k, Cp), np.int8)
+    orig[..., :Cn] = Wc[:, :Cn].transpose(0, 2, 3, 1)
+    ref_pack = np.concatenate([orig.reshape(O, -1), Wc[:, Cn:].transpose(0, 2, 3, 1).reshape(O, -1)], axis=1)
+    assert ref_pack.shape[1] == ocs.ocs_conv_packed_k(Cn, S, k, k)
     np.testing.assert_array_equal(host(packed)[:, :ref_pack.shape[1]], ref_pack)
     assert not host(packed)[:, ref_pack.shape[1]:].any()
     st = ocs.new_status()
