@@ -133,7 +133,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_cluster() { asm volatile("fence.proxy.async.shared::cluster;" ::: "memory"); }
 
 // Thread-block cluster: rank and size, a peer CTA's view of one of our shared-memory addresses,
 // stores and barrier arrivals into a peer's shared memory, cluster-wide barrier.
@@ -578,7 +578,8 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
           for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), make_uint4(0u, 0u, 0u, 0u));
         }
-        fence_proxy_async_all();  // make the generic-proxy stores visible to the tensor cores that read them
+        // make the generic-proxy stores visible to the tensor cores that read them
+        if (CL == 1) fence_proxy_async_smem(); else fence_proxy_async_cluster();
         __syncwarp();
         if (lane == 0)
           for (uint32_t dst = 0; dst < CL; ++dst) mbar_arrive_peer(peer_addr(gfull_bar(g), dst));
@@ -749,12 +750,13 @@ constexpr int kMaxSplitCtas = 2 * kNumSMs;   // split-K never uses more than two
 // Tile width, K split and cluster size by a small time model in units of one TMA-fed K-block of a
 // 128 x 256 tile: a wave costs max(main loop, gather beside it) plus a fixed prologue/epilogue; the
 // gather of one assembled K-block costs about `gather_cost` such units and is divided by the cluster
-// size; split-K adds the reduction pass.  n_tail = K-blocks whose A tile is assembled by threads.
-GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, bool conv) {
+// size; split-K adds the reduction pass.  n_tail = K-blocks whose A tile is assembled by threads,
+// tail_k = contraction indices in them (only 16-index chunks that hold data cost gather time).
+GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, bool conv) {
   GemmPlan best{64, 1, 1, m_tiles, (N + 63) / 64};
   double best_cost = 1e300;
   const int bns[3] = {256, 128, 64};
-  const double gather_cost = conv ? 16.0 : 40.0;
+  const double gather_cost = conv ? 16.0 : 60.0;
   for (int bi = 0; bi < 3; ++bi) {
     const int BN = bns[bi];
     if (BN > 64 && N <= BN / 2) continue;  // tile mostly empty
@@ -774,7 +776,9 @@ GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, bool conv) {
         if (cl > 1 && (n_tail == 0 || n_tiles % cl != 0)) continue;
         const long long waves = (ctas + kClusterCapacity[ci] - 1) / kClusterCapacity[ci];
         const double main_t = main_blocks * t_block;
-        const double gather_t = tail_blocks * gather_cost / cl;
+        // the most loaded CTA assembles tail_blocks K-blocks, of which at most tail_k indices hold data
+        const int cta_k = tail_k < tail_blocks * BK ? tail_k : tail_blocks * BK;
+        const double gather_t = (0.5 * tail_blocks + (cta_k / 128.0) * gather_cost) / cl;
         double cost = (double)waves * ((main_t > gather_t ? main_t : gather_t) + 4.0 * t_block);
         if (sk > 1) cost += 6.0;
         cost *= 1.0 + 0.002 * ci + 0.001 * bi;   // ties: smaller cluster, wider tile
@@ -848,7 +852,7 @@ ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long lo
                     const CUtensorMap* tmA_in, void* ws, size_t ws_bytes, cudaStream_t stream) {
   p.num_kb = (p.Ktot + BK - 1) / BK;
   if (!tma_a_ok) p.kb_tma_a = 0;
-  const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb, p.num_kb - p.kb_tma_a, p.mode == MODE_CONV);
+  const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb, p.num_kb - p.kb_tma_a, p.Ktot - p.kb_tma_a * BK, p.mode == MODE_CONV);
   p.split_k = plan.split_k;
   p.m_tiles = plan.m_tiles;
   p.n_groups = plan.n_tiles / plan.cluster;
