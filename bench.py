@@ -90,6 +90,33 @@ def aggregate_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float) -> f
     return bytes_per_rank_step * world / (ms_per_step * 1e-3) / 1e9
 
 
+# DRAM traffic of the dominant kernel from one ncu capture (profiles/split_rows_kernel_fc6.md): the launch
+# at r = 0.1 moved 811.6 MB for 863.2 MB of algorithmic bytes.  The figure is only reported while the
+# kernel's source text is the one that was profiled.
+NCU_TRAFFIC = {"split_scatter_kernel": dict(fingerprint="0865454ddbf393ff", dram_bytes=811.6e6, algorithmic_bytes=863.2e6)}
+
+
+def kernel_fingerprint(kernel: str):
+    if kernel != "split_scatter_kernel":
+        return None
+    import hashlib
+    try:
+        src = open(os.path.join(ROOT, "paper_1901_09504_b200", "csrc", "split.cu")).read()
+        a, b = src.index("// K3, bulk-copy form."), src.index("struct SplitWs {")
+    except (OSError, ValueError):
+        return None
+    return hashlib.sha256(src[a:b].encode()).hexdigest()[:16]
+
+
+def ncu_traffic(kernel: str, algorithmic_bytes_per_launch: float):
+    """Per-launch DRAM bytes, scaled from the captured launch by algorithmic bytes (traffic is
+    proportional to the rows moved); None when the kernel has changed since the capture."""
+    rec = NCU_TRAFFIC.get(kernel)
+    if not rec or kernel_fingerprint(kernel) != rec["fingerprint"]:
+        return None
+    return rec["dram_bytes"] / rec["algorithmic_bytes"] * algorithmic_bytes_per_launch
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -656,7 +683,9 @@ def main():
     elif top_bytes:
         roof_achieved = top_bytes * args.steps / (top_ms * 1e-3) / 1e9
         roofline = dict(kernel=top, bound="hbm", achieved=roof_achieved, peak=pk["hbm"], unit="GB/s",
-                        frac=roof_achieved / pk["hbm"], traffic=None, peak_source=f"of {pk['source']}",
+                        frac=roof_achieved / pk["hbm"], traffic=ncu_traffic(top, top_bytes * args.steps / top_cnt),
+                        traffic_unit="bytes per launch (ncu dram read + write, scaled from the r = 0.1 launch)",
+                        peak_source=f"of {pk['source']}",
                         avg_launch_ms=top_ms / top_cnt,
                         timed="second pass over the same steps with CUDA events around every kernel launch")
     else:   # a dependent-step kernel (greedy plan, scoring): no bytes to speak of

@@ -255,30 +255,33 @@ __device__ float greedy_rounds(const PlanArgs& a, PlanShared& sh, unsigned long 
     for (int i = tid; i < n_live; i += kPlanThreads) m = live[i] > m ? live[i] : m;
     const unsigned long long pmax = block_max_u64(m, sh.red);
     const float bound = __fmul_rn(__fadd_rn(prio_key(pmax), d), 0.5f);
-    if (tid == 0) { sh.n_batch = 0; sh.n_next = 0; }
-    __syncthreads();
+    // Stable partition (positions from prefix sums, not atomics): the selected originals arrive in
+    // index order, so a batch of equal keys -- the tie-break case -- comes out already in priority
+    // order and the sort below can be skipped.
+    int nb = 0, n_keep = 0;
     for (int i0 = 0; i0 < n_live; i0 += kPlanThreads) {   // whole warps iterate together
       const int i = i0 + tid;
       const unsigned long long p = i < n_live ? live[i] : 0ull;
       const bool in_batch = i < n_live && (prio_key(p) > bound || p == pmax);
       const bool in_next = i < n_live && !in_batch;
       const unsigned int mb = __ballot_sync(0xffffffffu, in_batch), mn = __ballot_sync(0xffffffffu, in_next);
-      int bb = 0, nn = 0;
-      if (lane == 0) {
-        if (mb) bb = atomicAdd(&sh.n_batch, __popc(mb));
-        if (mn) nn = atomicAdd(&sh.n_next, __popc(mn));
-      }
-      bb = __shfl_sync(0xffffffffu, bb, 0);
-      nn = __shfl_sync(0xffffffffu, nn, 0);
-      if (in_batch) batch[bb + __popc(mb & lt)] = p;
-      if (in_next) next[nn + __popc(mn & lt)] = p;
+      unsigned long long total;
+      const unsigned long long mine = lane == 0 ? (((unsigned long long)__popc(mb) << 32) | (unsigned long long)__popc(mn)) : 0ull;
+      unsigned long long pre = block_excl_scan(mine, sh.scan, &total);
+      pre = __shfl_sync(0xffffffffu, pre, 0);   // lane 0 holds the sum over the warps before this one
+      if (in_batch) batch[nb + (int)(pre >> 32) + __popc(mb & lt)] = p;
+      if (in_next) next[n_keep + (int)(unsigned int)pre + __popc(mn & lt)] = p;
+      nb += (int)(total >> 32);
+      n_keep += (int)(unsigned int)total;
     }
     __syncthreads();
-    const int nb = sh.n_batch, n_keep = sh.n_next;
     int npad = 1;
     while (npad < nb) npad <<= 1;
     for (int i = nb + tid; i < npad; i += kPlanThreads) batch[i] = 0ull;  // below every real priority word
     __syncthreads();
+    bool unsorted = false;
+    for (int i = tid + 1; i < nb; i += kPlanThreads) unsorted |= batch[i - 1] < batch[i];
+    if (!__syncthreads_or(unsorted)) npad = 1;   // already in descending priority order
     if (npad > 1) bitonic_sort_desc(batch, npad);
     const int take = min(nb, a.S - base);
     // rank i < take performs step base + i; its children go to next[n_keep + 2i, +1]; channels
