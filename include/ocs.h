@@ -134,6 +134,25 @@ ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, int64_t ld_i
                         const float* max_abs_in, int8_t* codes, int64_t ld_codes, float* scale,
                         float* alpha, void* ws, size_t ws_bytes, int* dev_status, void* stream);
 
+/* ocs_split_quantize -----------------------------------------------------------------------
+ * ocs_split followed by ocs_quantize on its result ("OCS followed by clipping", Section 5.2;
+ * Sections 3.2-3.4, Eq. 1, Section 4.1) in one call that never writes the fp32 W': the
+ * expanded rows exist only in shared memory, from where they are histogrammed (mode MSE) and
+ * quantized.  W is read three times (extrema, histogram, quantization) instead of W and W'
+ * being read and written five times.  Results are bit-identical to the two separate calls:
+ * codes int8 [O][(C+S)*R] in the split's layout with row stride ld_codes bytes, idx_map,
+ * split_order (nullable), max_abs_out [3] (nullable), *scale, *alpha (nullable).
+ * Arguments as in ocs_split and ocs_quantize (signed codes; modes NONE and MSE).
+ * Limits: W 16-byte aligned, ld_in and C*R multiples of 4, and two expanded rows (plus the
+ * histogram) must fit in shared memory ((C+S)*R up to about 27,000 floats); otherwise
+ * OCS_ERR_UNSUPPORTED -- use the two separate calls.  Device flags: NONFINITE, DEPTH, TIMEOUT. */
+size_t ocs_split_quantize_workspace_bytes(int O, int C, int R, int S, int n_bins, int n_candidates);
+ocs_status ocs_split_quantize(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step,
+                              int qa_bits, int bits, ocs_clip_mode mode, int n_candidates, int n_bins,
+                              int8_t* codes, int64_t ld_codes, int32_t* idx_map, int32_t* split_order,
+                              float* max_abs_out, float* scale, float* alpha, void* ws, size_t ws_bytes,
+                              int* dev_status, void* stream);
+
 /* ocs_quantize_noalloc ---------------------------------------------------------------------
  * (No counterpart in the paper: a packaging variant of ocs_quantize.)
  * Same operation, arguments and results as ocs_quantize, minus (ws, ws_bytes).  It is meant for

@@ -26,6 +26,7 @@ EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
     "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
     "ocs_split_workspace_bytes", "ocs_split",
+    "ocs_split_quantize_workspace_bytes", "ocs_split_quantize",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
     "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
@@ -50,7 +51,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.ocs_num_splits.argtypes = [C.c_int, C.c_double]
         L.ocs_version.restype = C.c_char_p
-        for name in ("ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
+        for name in ("ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
                      "ocs_qconv_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.ocs_quantize_workspace_views.restype = None
@@ -337,3 +338,38 @@ def ocs_quantize_noalloc(T, bits: int, is_signed: bool = True, mode: int = CLIP_
                                     _ptr(dev_status), _stream())
     _check(st, "ocs_quantize_noalloc")
     return codes, scale, alpha
+
+
+def ocs_split_quantize(W, S: int, bits: int, mode: int = CLIP_NONE, qa_step: float = 0.0, qa_bits: int = 0,
+                       n_candidates: int = 128, n_bins: int = 2048, ld_codes: int | None = None, dev_status=None,
+                       want_order: bool = True, out=None, ws=None):
+    """Split + clip search + quantization without the fp32 W'.  W fp32 [O, C] or [O, C, kh, kw].
+    Returns (codes int8 [O, ld_codes] in the split's layout, scale [1], alpha [1], idx_map int32 [C+S],
+    split_order int32 [S] or None, max_abs fp32 [3]).  `out` = (codes, scale, alpha, idx_map, order, max_abs)."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+    O, Cn = W.shape[0], W.shape[1]
+    R = 1
+    for d in W.shape[2:]:
+        R *= d
+    cols_out = (Cn + S) * R
+    if out is not None:
+        codes, scale, alpha, idx_map, order, max_abs = out
+        ld_codes = codes.stride(0)
+    else:
+        if ld_codes is None:
+            ld_codes = round_up(cols_out, 16)
+        codes = torch.empty((O, ld_codes), dtype=torch.int8, device=W.device)
+        scale = torch.zeros(1, dtype=torch.float32, device=W.device)
+        alpha = torch.zeros(1, dtype=torch.float32, device=W.device)
+        idx_map = torch.empty(Cn + S, dtype=torch.int32, device=W.device)
+        order = torch.empty(max(S, 1), dtype=torch.int32, device=W.device) if want_order else None
+        max_abs = torch.zeros(3, dtype=torch.float32, device=W.device)
+    nws = lib().ocs_split_quantize_workspace_bytes(O, Cn, R, int(S), int(n_bins), int(n_candidates))
+    if ws is None:
+        ws = _ws(nws, W.device)
+    st = lib().ocs_split_quantize(_ptr(W), O, Cn, R, C.c_int64(Cn * R), int(S), C.c_float(qa_step), int(qa_bits),
+                                  int(bits), int(mode), int(n_candidates), int(n_bins), _ptr(codes),
+                                  C.c_int64(ld_codes), _ptr(idx_map), _ptr(order), _ptr(max_abs), _ptr(scale),
+                                  _ptr(alpha), _ptr(ws), C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
+    _check(st, "ocs_split_quantize")
+    return codes, scale, alpha, idx_map, (order[:S] if order is not None else None), max_abs

@@ -273,43 +273,6 @@ exact_combine_kernel(const double* __restrict__ partial, int n_parts, int n_cand
   scores[c] = a;
 }
 
-// The search's winner: smallest score, ties to the largest threshold.  Every CTA of the quantize
-// kernel evaluates it (n_candidates doubles) instead of a separate single-thread launch.
-__device__ float pick_alpha(const double* __restrict__ scores, float m, int n_candidates) {
-  __shared__ double s_best[8];
-  __shared__ int c_best[8];
-  double bs = INFINITY;
-  int bc = 0;
-  for (int c = threadIdx.x + 1; c <= n_candidates; c += 256) {
-    const double v = scores[c - 1];
-    if (v < bs || (v == bs && c > bc)) { bs = v; bc = c; }
-  }
-  for (int o = 16; o > 0; o >>= 1) {
-    const double v = __shfl_xor_sync(0xffffffffu, bs, o);
-    const int c = __shfl_xor_sync(0xffffffffu, bc, o);
-    if (c != 0 && (bc == 0 || v < bs || (v == bs && c > bc))) { bs = v; bc = c; }
-  }
-  if ((threadIdx.x & 31) == 0) { s_best[threadIdx.x >> 5] = bs; c_best[threadIdx.x >> 5] = bc; }
-  __syncthreads();
-  bs = s_best[0]; bc = c_best[0];
-  for (int w = 1; w < 8; ++w) {
-    const double v = s_best[w];
-    const int c = c_best[w];
-    if (c != 0 && (bc == 0 || v < bs || (v == bs && c > bc))) { bs = v; bc = c; }
-  }
-  return __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)bc), (double)n_candidates));
-}
-
-// code = clamp(rint(x * inv)): clamping first is the same thing (the bounds are integers) and leaves one
-// conversion with round-to-nearest-even
-__device__ __forceinline__ int quant_code(float x, float inv, float lo, float hi) {
-  return __float2int_rn(fminf(fmaxf(__fmul_rn(x, inv), lo), hi));
-}
-__device__ __forceinline__ unsigned int pack4(int c0, int c1, int c2, int c3) {
-  return __byte_perm(__byte_perm((unsigned)c0, (unsigned)c1, 0x0040), __byte_perm((unsigned)c2, (unsigned)c3, 0x0040),
-                     0x5410);
-}
-
 __global__ void __launch_bounds__(256)
 quantize_kernel(View v, const float* __restrict__ alpha_p, const double* __restrict__ scores, int n_candidates, int L,
                 int is_signed, int8_t* __restrict__ codes, long long ld_codes, int packed_ok,
@@ -375,6 +338,14 @@ QuantWs carve_quant_ws(void* ws, int n_bins, int n_candidates) {
 }
 
 }  // namespace
+
+ocs_status launch_score_kernel(const unsigned long long* hist, const float* maxp, int n_bins, int n_candidates, int L,
+                               int is_signed, double* scores, cudaStream_t stream) {
+  LaunchScope ls("score_kernel", stream);
+  score_kernel<<<n_candidates, 256, 0, stream>>>(hist, maxp, n_bins, n_candidates, L, is_signed, scores);
+  return launch_status();
+}
+
 }  // namespace ocs
 
 using namespace ocs;

@@ -641,12 +641,35 @@ __device__ __forceinline__ bool row_bar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// What happens to a finished row of W' in shared memory:
+//   ROWS_STORE  it is written out as fp32 (ocs_split)
+//   ROWS_HIST   its |values| are added to the clip search's histogram, nothing is written
+//   ROWS_QUANT  it is quantized and only the codes are written
+// The last two serve ocs_split_quantize, which never materialises the fp32 W'.
+enum { ROWS_STORE = 0, ROWS_HIST = 1, ROWS_QUANT = 2 };
+
+struct RowsEpilogue {
+  const float* maxp;            // max|W'| (device scalar from the plan)
+  int n_bins;                   // HIST
+  unsigned long long* hist;     // HIST: global histogram [n_bins]
+  int hist_copies;              // HIST: private copies in shared memory behind the row buffers
+  const double* scores;         // QUANT: candidate scores (null: no clipping)
+  int n_candidates;
+  int L;                        // QUANT: code range [-L, L]
+  int8_t* codes;                // QUANT: [O][ld_codes]
+  long long ld_codes;
+  int packed_ok;                // QUANT: 32-bit stores of four codes allowed
+  float* scale_out;
+  float* alpha_out;
+};
+
+template <int MODE>
 __global__ void __launch_bounds__(kRowThreads, 1)
 split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_in, int S, float* __restrict__ Wout,
                   int64_t ld_out, const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
                   const unsigned long long* __restrict__ bits, const float* __restrict__ qa_step_dev,
                   const int32_t* __restrict__ touched, const int* __restrict__ n_touched, int rows_per_group,
-                  int srow /*floats between rows in shared memory*/, int* dev_status) {
+                  int srow /*floats between rows in shared memory*/, RowsEpilogue ep, int* dev_status) {
   extern __shared__ __align__(128) unsigned char row_smem[];
   __shared__ __align__(8) unsigned long long bars[2];
   __shared__ int abort_flag;
@@ -661,6 +684,27 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
   const float d = __fmul_rn(*qa_step_dev, 0.5f);
   const int nt = *n_touched;
   const int dep_cap = d == 0.0f ? kMaxHalvings : 64;
+
+  // epilogue state
+  unsigned int* hist_sh = reinterpret_cast<unsigned int*>(row_smem + 2 * (size_t)rows_per_group * srow * sizeof(float));
+  float invw = 0.0f, q_inv = 0.0f, q_lo = 0.0f, q_hi = 0.0f;
+  if (MODE == ROWS_HIST) {
+    for (int i = tid; i < ep.hist_copies * ep.n_bins; i += kRowThreads) hist_sh[i] = 0u;
+    const float m = *ep.maxp;
+    invw = m > 0.0f ? __fdiv_rn((float)ep.n_bins, m) : 0.0f;
+  }
+  if (MODE == ROWS_QUANT) {
+    float alpha = *ep.maxp;
+    if (ep.scores && alpha > 0.0f) alpha = pick_alpha(ep.scores, alpha, ep.n_candidates);
+    const bool zero = !(alpha > 0.0f);
+    const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)ep.L);
+    q_inv = zero ? 0.0f : __fdiv_rn((float)ep.L, alpha);
+    q_lo = -(float)ep.L; q_hi = (float)ep.L;
+    if (blockIdx.x == 0 && tid == 0) {
+      *ep.scale_out = step;
+      if (ep.alpha_out) *ep.alpha_out = zero ? 0.0f : alpha;
+    }
+  }
 
   if (tid == 0) {
     for (int b = 0; b < 2; ++b)
@@ -749,7 +793,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
           const float v = apply_path(rows[t_src[k]], t_dep[k], t_bits[k], d);
           const int col = in_cols + tid + k * kRowThreads;
           rows[col] = v;
-          if (col >= out_bulk) Wout[(int64_t)r0 * ld_out + col] = v;   // the last 1-3 floats of a row
+          if (MODE == ROWS_STORE && col >= out_bulk) Wout[(int64_t)r0 * ld_out + col] = v;   // the last 1-3 floats of a row
         }
       }
       __syncthreads();
@@ -766,7 +810,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
                                    min(__ldg(depth + j), dep_cap), __ldg(bits + j), d);
         const int col = in_cols + e;
         rows[(size_t)rl * srow + col] = v;
-        if (col >= out_bulk) Wout[(int64_t)(r0 + rl) * ld_out + col] = v;
+        if (MODE == ROWS_STORE && col >= out_bulk) Wout[(int64_t)(r0 + rl) * ld_out + col] = v;
       }
       __syncthreads();
       for (int it = tid; it < gn * orig_items; it += kRowThreads) {
@@ -777,16 +821,62 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
         *q = apply_path(*q, min(__ldg(depth + j), dep_cap), 0ull, d);
       }
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the bulk store
+    if (MODE == ROWS_STORE) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the bulk store
     __syncthreads();
-    if (tid == 0 && out_bulk > 0) {
-      for (int rl = 0; rl < gn; ++rl) {
-        float* dst = Wout + (int64_t)(r0 + rl) * ld_out;
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                     ::"l"(dst), "r"(smem_addr(rows + (size_t)rl * srow)), "r"((uint32_t)out_bulk * 4u)
-                     : "memory");
+    if (MODE == ROWS_STORE) {
+      if (tid == 0 && out_bulk > 0) {
+        for (int rl = 0; rl < gn; ++rl) {
+          float* dst = Wout + (int64_t)(r0 + rl) * ld_out;
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                       ::"l"(dst), "r"(smem_addr(rows + (size_t)rl * srow)), "r"((uint32_t)out_bulk * 4u)
+                       : "memory");
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
-      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    } else {
+      // the finished rows are consumed straight from shared memory
+      const int quads = out_cols >> 2;
+      for (int rl = 0; rl < gn; ++rl) {
+        const float* row = rows + (size_t)rl * srow;
+        if (MODE == ROWS_HIST) {
+          if (invw > 0.0f) {
+            unsigned int* mine = hist_sh + ((tid >> 5) % ep.hist_copies) * ep.n_bins;
+            const int last = ep.n_bins - 1;
+            auto count = [&](float xv) {
+              const int bin = min(last, (int)__fmul_rn(fabsf(xv), invw));  // truncation
+              atomicAdd(&mine[bin], 1u);
+            };
+            for (int q = tid; q < quads; q += kRowThreads) {
+              const float4 v = reinterpret_cast<const float4*>(row)[q];
+              count(v.x); count(v.y); count(v.z); count(v.w);
+            }
+            if (tid < (out_cols & 3)) count(row[(quads << 2) + tid]);
+          }
+        } else {
+          int8_t* out = ep.codes + (long long)(r0 + rl) * ep.ld_codes;
+          for (int q = tid; q < quads; q += kRowThreads) {
+            const float4 v = reinterpret_cast<const float4*>(row)[q];
+            const unsigned int word = pack4(quant_code(v.x, q_inv, q_lo, q_hi), quant_code(v.y, q_inv, q_lo, q_hi),
+                                            quant_code(v.z, q_inv, q_lo, q_hi), quant_code(v.w, q_inv, q_lo, q_hi));
+            if (ep.packed_ok) {
+              *reinterpret_cast<unsigned int*>(out + 4 * q) = word;
+            } else {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) out[4 * q + k] = (int8_t)((word >> (8 * k)) & 0xFFu);
+            }
+          }
+          if (tid < (out_cols & 3)) out[(quads << 2) + tid] = (int8_t)quant_code(row[(quads << 2) + tid], q_inv, q_lo, q_hi);
+        }
+      }
+      __syncthreads();   // the buffer may be refilled now
+    }
+  }
+  if (MODE == ROWS_HIST) {
+    __syncthreads();
+    for (int bin = tid; bin < ep.n_bins; bin += kRowThreads) {
+      unsigned int c = 0u;
+      for (int k = 0; k < ep.hist_copies; ++k) c += hist_sh[k * ep.n_bins + bin];
+      if (c) atomicAdd(&ep.hist[bin], (unsigned long long)c);
     }
   }
   if (tid == 0) {
@@ -867,23 +957,14 @@ extern "C" size_t ocs_split_workspace_bytes(int O, int C, int R, int S) {
   return carve_split_ws(nullptr, C, R, S).total;
 }
 
-extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step,
-                                int qa_bits, float* W_out, int64_t ld_out, int32_t* idx_map,
-                                int32_t* split_order, float* max_abs_out, void* ws, size_t ws_bytes,
-                                int* dev_status, void* stream_) {
-  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
-  if (!W || !W_out || !idx_map) return OCS_ERR_INVALID_ARG;
-  if (S < 0 || !(qa_step >= 0.0f) || !is_finite_host(qa_step)) return OCS_ERR_INVALID_ARG;
-  if (qa_bits != 0 && (qa_bits < 2 || qa_bits > 8)) return OCS_ERR_INVALID_ARG;
-  if (O <= 0 || C <= 0 || R <= 0) return OCS_ERR_SHAPE;
-  if ((int64_t)C * R >= (1ll << 31) || ((int64_t)C + S) * R >= (1ll << 31)) return OCS_ERR_SHAPE;
-  if (ld_in < (int64_t)C * R || ld_out < ((int64_t)C + S) * R) return OCS_ERR_SHAPE;
-  if (!aligned(W, 4) || !aligned(W_out, 4)) return OCS_ERR_SHAPE;
-  const SplitWs w = carve_split_ws(ws, C, R, S);
-  if (!ws || !aligned(ws, 256) || ws_bytes < w.total) return OCS_ERR_WORKSPACE;
-  ocs_status st = check_device();
-  if (st != OCS_OK) return st;
+namespace ocs {
+namespace {
 
+// The part ocs_split and ocs_split_quantize share: channel extrema and the greedy plan.
+ocs_status run_split_front(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step, int qa_bits,
+                           int32_t* idx_map, int32_t* split_order, float* max_abs_out, const SplitWs& w,
+                           int* dev_status, cudaStream_t stream) {
+  ocs_status st;
   const int ncols = C * R;
   if (cudaMemsetAsync(w.colmin, 0xFF, 4 * (size_t)ncols, stream) != cudaSuccess) return OCS_ERR_CUDA;
   if (cudaMemsetAsync(w.colmax, 0x00, 4 * (size_t)ncols, stream) != cudaSuccess) return OCS_ERR_CUDA;
@@ -930,6 +1011,32 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     split_plan_kernel<<<1, kPlanThreads, smem, stream>>>(a);
     if ((st = launch_status()) != OCS_OK) return st;
   }
+  return OCS_OK;
+}
+
+}  // namespace
+}  // namespace ocs
+
+extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step,
+                                int qa_bits, float* W_out, int64_t ld_out, int32_t* idx_map,
+                                int32_t* split_order, float* max_abs_out, void* ws, size_t ws_bytes,
+                                int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!W || !W_out || !idx_map) return OCS_ERR_INVALID_ARG;
+  if (S < 0 || !(qa_step >= 0.0f) || !is_finite_host(qa_step)) return OCS_ERR_INVALID_ARG;
+  if (qa_bits != 0 && (qa_bits < 2 || qa_bits > 8)) return OCS_ERR_INVALID_ARG;
+  if (O <= 0 || C <= 0 || R <= 0) return OCS_ERR_SHAPE;
+  if ((int64_t)C * R >= (1ll << 31) || ((int64_t)C + S) * R >= (1ll << 31)) return OCS_ERR_SHAPE;
+  if (ld_in < (int64_t)C * R || ld_out < ((int64_t)C + S) * R) return OCS_ERR_SHAPE;
+  if (!aligned(W, 4) || !aligned(W_out, 4)) return OCS_ERR_SHAPE;
+  const SplitWs w = carve_split_ws(ws, C, R, S);
+  if (!ws || !aligned(ws, 256) || ws_bytes < w.total) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+
+  if ((st = run_split_front(W, O, C, R, ld_in, S, qa_step, qa_bits, idx_map, split_order, max_abs_out, w, dev_status,
+                            stream)) != OCS_OK)
+    return st;
   {
     const int ncols_out = (C + S) * R;
     const bool vec = (ld_in % 4 == 0) && (ld_out % 4 == 0) && aligned(W, 16) && aligned(W_out, 16);
@@ -944,14 +1051,14 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
       const int n_groups = (int)((O + g - 1) / g);
       static bool attr_set = false;
       if (!attr_set) {
-        if (cudaFuncSetAttribute(split_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmemBytes) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(split_rows_kernel<ROWS_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kRowSmemBytes) != cudaSuccess)
           return OCS_ERR_CUDA;
         attr_set = true;
       }
-      split_rows_kernel<<<min(n_groups, kNumSMs), kRowThreads, 2 * (size_t)g * row_bytes, stream>>>(
+      split_rows_kernel<ROWS_STORE><<<min(n_groups, kNumSMs), kRowThreads, 2 * (size_t)g * row_bytes, stream>>>(
           W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g,
-          srow, dev_status);
+          srow, RowsEpilogue{}, dev_status);
     } else {
       const long long units = (long long)((ncols_out + 1023) / 1024) * O;
       if (vec)
@@ -964,4 +1071,125 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     if ((st = launch_status()) != OCS_OK) return st;
   }
   return OCS_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// ocs_split_quantize: split + clip search + quantization without the fp32 W'.
+namespace ocs {
+namespace {
+struct FusedWs {
+  SplitWs sp;
+  float* mx3;
+  unsigned long long* hist;
+  double* scores;
+  size_t total;
+};
+FusedWs carve_fused_ws(void* ws, int C, int R, int S, int n_bins, int n_candidates) {
+  FusedWs f{};
+  f.sp = carve_split_ws(ws, C, R, S);
+  size_t off = f.sp.total;
+  auto take = [&](size_t bytes) {
+    unsigned char* p = ws ? reinterpret_cast<unsigned char*>(ws) + off : nullptr;
+    off += align_up(bytes, 256);
+    return p;
+  };
+  f.mx3 = reinterpret_cast<float*>(take(256));
+  f.hist = reinterpret_cast<unsigned long long*>(take(8 * (size_t)(n_bins > 0 ? n_bins : 1)));
+  f.scores = reinterpret_cast<double*>(take(8 * (size_t)(n_candidates > 0 ? n_candidates : 1)));
+  f.total = off;
+  return f;
+}
+}  // namespace
+}  // namespace ocs
+
+extern "C" size_t ocs_split_quantize_workspace_bytes(int O, int C, int R, int S, int n_bins, int n_candidates) {
+  (void)O;
+  if (C <= 0 || R <= 0 || S < 0) return 0;
+  return carve_fused_ws(nullptr, C, R, S, n_bins, n_candidates).total;
+}
+
+extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step,
+                                         int qa_bits, int bits, ocs_clip_mode mode, int n_candidates, int n_bins,
+                                         int8_t* codes, int64_t ld_codes, int32_t* idx_map, int32_t* split_order,
+                                         float* max_abs_out, float* scale, float* alpha, void* ws, size_t ws_bytes,
+                                         int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!W || !codes || !idx_map || !scale) return OCS_ERR_INVALID_ARG;
+  if (S < 0 || !(qa_step >= 0.0f) || !is_finite_host(qa_step)) return OCS_ERR_INVALID_ARG;
+  if (qa_bits != 0 && (qa_bits < 2 || qa_bits > 8)) return OCS_ERR_INVALID_ARG;
+  if (bits < 2 || bits > 8) return OCS_ERR_INVALID_ARG;
+  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE) return OCS_ERR_INVALID_ARG;
+  if (mode == OCS_CLIP_MSE && (n_candidates < 1 || n_candidates > 1024 || n_bins < 1 || n_bins > 4096))
+    return OCS_ERR_INVALID_ARG;
+  if (O <= 0 || C <= 0 || R <= 0) return OCS_ERR_SHAPE;
+  if ((int64_t)C * R >= (1ll << 31) || ((int64_t)C + S) * R >= (1ll << 31)) return OCS_ERR_SHAPE;
+  const int ncols_out = (C + S) * R;
+  if (ld_in < (int64_t)C * R || ld_codes < ncols_out) return OCS_ERR_SHAPE;
+  if (mode == OCS_CLIP_NONE) { n_bins = 1; n_candidates = 1; }
+  // rows are staged whole in shared memory: they must be 16-byte addressable and fit twice
+  const int srow = (ncols_out + 3) & ~3;
+  const size_t row_bytes = 4 * (size_t)srow;
+  const size_t hist_bytes = mode == OCS_CLIP_MSE ? 4 * (size_t)n_bins : 0;
+  if (!(ld_in % 4 == 0 && aligned(W, 16) && (C * R) % 4 == 0 && 2 * row_bytes + hist_bytes <= kRowSmemBytes))
+    return OCS_ERR_UNSUPPORTED;
+  const FusedWs f = carve_fused_ws(ws, C, R, S, n_bins, n_candidates);
+  if (!ws || !aligned(ws, 256) || ws_bytes < f.total) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  const SplitWs& w = f.sp;
+  float* mx3 = max_abs_out ? max_abs_out : f.mx3;
+  if ((st = run_split_front(W, O, C, R, ld_in, S, qa_step, qa_bits, idx_map, split_order, mx3, w, dev_status, stream)) !=
+      OCS_OK)
+    return st;
+
+  long long g = (long long)((kRowSmemBytes - hist_bytes) / 2 / row_bytes);
+  g = min(g, (long long)max(1, O / kNumSMs));
+  g = min(g, 64ll);
+  const int n_groups = (int)((O + g - 1) / g);
+  const size_t rows_smem = 2 * (size_t)g * row_bytes;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(split_rows_kernel<ROWS_HIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kRowSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(split_rows_kernel<ROWS_QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kRowSmemBytes) != cudaSuccess)
+      return OCS_ERR_CUDA;
+    attr_set = true;
+  }
+  const int L = (1 << (bits - 1)) - 1;
+  RowsEpilogue ep{};
+  ep.maxp = mx3 + 1;   // max|W'| as the plan computed it
+  ep.L = L;
+  const double* scores = nullptr;
+  if (mode == OCS_CLIP_MSE) {
+    if (cudaMemsetAsync(f.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
+    ep.n_bins = n_bins;
+    ep.hist = f.hist;
+    int copies = (int)((kRowSmemBytes - rows_smem) / (4 * (size_t)n_bins));
+    ep.hist_copies = copies >= 4 ? 4 : (copies >= 2 ? 2 : 1);
+    {
+      LaunchScope ls("split_hist_kernel", stream);
+      split_rows_kernel<ROWS_HIST><<<min(n_groups, kNumSMs), kRowThreads,
+                                     rows_smem + 4 * (size_t)ep.hist_copies * n_bins, stream>>>(
+          W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g, srow,
+          ep, dev_status);
+    }
+    if ((st = launch_status()) != OCS_OK) return st;
+    if ((st = launch_score_kernel(f.hist, ep.maxp, n_bins, n_candidates, L, 1, f.scores, stream)) != OCS_OK) return st;
+    scores = f.scores;
+  }
+  ep.scores = scores;
+  ep.n_candidates = n_candidates;
+  ep.codes = codes;
+  ep.ld_codes = ld_codes;
+  ep.packed_ok = aligned(codes, 4) && (ld_codes % 4 == 0);
+  ep.scale_out = scale;
+  ep.alpha_out = alpha;
+  {
+    LaunchScope ls("split_quantize_kernel", stream);
+    split_rows_kernel<ROWS_QUANT><<<min(n_groups, kNumSMs), kRowThreads, rows_smem, stream>>>(
+        W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g, srow, ep,
+        dev_status);
+  }
+  return launch_status();
 }

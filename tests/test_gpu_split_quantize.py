@@ -199,3 +199,54 @@ def test_quantize_exact_mse_scorer():
     c2 = configs.config2(batch=1)
     Wp2, _, _, _ = orc.split(c2["W"], 6)
     _check_quant_exact(Wp2.reshape(256, -1), 6, True)
+
+
+# ------------------------------------------------------------------------------ fused split + quantize
+def _check_fused(W, S, bits, mode, qa_bits=0, n_cand=128, n_bins=2048):
+    """ocs_split_quantize against the checker's split -> search -> quantize, and against the two separate calls."""
+    o_out, o_idx, o_order, o_mx, step = oracle_split(W, S, qa_bits)
+    flat = o_out.reshape(o_out.shape[0], -1)
+    o_alpha = orc.clip_mse(flat, bits, True, n_bins, n_cand)["alpha"] if mode == ocs.CLIP_MSE else orc.maxabs(flat)
+    o_codes, o_scale = orc.quantize(flat, bits, True, o_alpha)
+    st = ocs.new_status()
+    codes, scale, alpha, idx, order, mx = ocs.ocs_split_quantize(dev(W), S, bits, mode, qa_bits=qa_bits,
+                                                                 n_candidates=n_cand, n_bins=n_bins, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    np.testing.assert_array_equal(host(idx), o_idx)
+    np.testing.assert_array_equal(host(order), o_order)
+    assert host(mx)[1] == np.float32(o_mx[1]) and host(mx)[2] == np.float32(step)
+    assert abs(float(host(alpha)[0]) - o_alpha) <= 1e-5 * abs(o_alpha)
+    assert np.float32(host(alpha)[0]) == np.float32(o_alpha)
+    assert float(host(scale)[0]) == np.float32(o_scale)
+    np.testing.assert_array_equal(host(codes)[:, :flat.shape[1]], o_codes)
+    # the separate calls give the same bytes
+    Wout, idx2, _, mx2 = ocs.ocs_split(dev(W), S, qa_bits=qa_bits)
+    codes2, scale2, alpha2 = ocs.ocs_quantize(Wout, bits, True, mode, n_cand, n_bins, cols=flat.shape[1],
+                                              max_abs_in=mx2[1:2])
+    np.testing.assert_array_equal(host(codes)[:, :flat.shape[1]], host(codes2)[:, :flat.shape[1]])
+    assert host(scale)[0] == host(scale2)[0] and host(alpha)[0] == host(alpha2)[0]
+
+
+def test_fused_split_quantize_matches_checker_and_separate_calls():
+    c1 = configs.config1()
+    for bits, mode in ((8, ocs.CLIP_NONE), (5, ocs.CLIP_MSE), (4, ocs.CLIP_MSE)):
+        _check_fused(c1["W"], 26, bits, mode)
+    _check_fused(c1["W"], 26, 6, ocs.CLIP_MSE, qa_bits=6)
+    c2 = configs.config2(batch=1)
+    _check_fused(c2["W"], 6, 6, ocs.CLIP_MSE)                                  # conv weights, R = 9
+    _check_fused(prng.laplace(17, 0, (33, 20), 0.02), 7, 5, ocs.CLIP_MSE, n_cand=33, n_bins=500)   # (C+S) odd: ragged rows
+    _check_fused(prng.laplace(17, 1, (5, 8), 0.02), 0, 8, ocs.CLIP_NONE)      # no splits
+    _check_fused(np.zeros((3, 4), np.float32), 5, 8, ocs.CLIP_MSE)            # all zero
+    c3 = configs.config3(O=256, C=25088, M=4)                                 # fc6-length rows: one row per buffer
+    _check_fused(c3["W"], ocs.ocs_num_splits(25088, 0.1), 4, ocs.CLIP_MSE)
+    _check_fused(c3["W"], ocs.ocs_num_splits(25088, 0.01), 8, ocs.CLIP_NONE)
+
+
+def test_fused_split_quantize_rejects_what_it_cannot_stage():
+    Wd = dev(prng.laplace(3, 0, (16, 30), 0.1))                                # C*R not a multiple of 4
+    with pytest.raises(ocs.OcsError) as e:
+        ocs.ocs_split_quantize(Wd, 2, 8)
+    assert e.value.status == 4
+    with pytest.raises(ocs.OcsError) as e:
+        ocs.ocs_split_quantize(dev(prng.laplace(3, 0, (16, 32), 0.1)), 2, 9)
+    assert e.value.status == 1
