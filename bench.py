@@ -1,11 +1,12 @@
 """Benchmark of the OCS hot path on B200: split -> clip search -> quantize -> int8 GEMM/conv.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-small|fc|conv|resnet50|lstm] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-fused|fc6-small|fc|conv|resnet50|lstm] [--impl reference]
 
 One step is one pass of the whole path over one batch of synthetic input:
   fc6   (default) the VGG-16-fc6-shaped sweep: W [4096, 25088], 5 expand ratios x 4 weight bit
         widths = 20 points; every point runs ocs_split, ocs_quantize with the MSE clip search,
         the activation quantization and ocs_qlinear (nothing is cached between points).
+  fc6-fused  the same sweep through ocs_split_quantize, which never writes the fp32 W'.
   fc6-small  the same recipe on W [256, 6272] (quick checks).
   fc    the small fully-connected layer [256, 512], batch 64, r = 0.05, 8-bit, no clipping.
   conv / resnet50 / lstm   the single 3x3 convolution, the ResNet-50 stack at batch 128 and the LSTM
@@ -50,6 +51,10 @@ def algorithmic_bytes(kernel: str, *, N=0, n=0, M=0, C=0, S=0, Nout=0, R=1, rows
         return 4 * N + 4 * n
     if kernel in ("hist_kernel", "maxabs_kernel"):
         return 4 * n
+    if kernel == "split_hist_kernel":          # fused path: W is read, the expanded rows live in shared memory
+        return 4 * N
+    if kernel == "split_quantize_kernel":
+        return 4 * N + n
     if kernel == "quantize_kernel":
         return 4 * n + n
     if kernel.startswith("ocs_gemm_kernel"):
@@ -262,6 +267,50 @@ class Fc6Sweep:
 def configs_num_splits(C, r):
     import math
     return 0 if r <= 0 else int(math.ceil(r * C - 1e-9))
+
+
+class Fc6Fused(Fc6Sweep):
+    """The same sweep through ocs_split_quantize (no fp32 W'): fewer bytes per point."""
+    name = "fc6-fused"
+
+    def __init__(self):
+        super().__init__()
+        self.desc = self.desc.replace("configs[2]:", "configs[2] through the fused ocs_split_quantize call:")
+
+    def setup(self, ocs, torch, dev, host):
+        super().setup(ocs, torch, dev, host)
+        nws = ocs.lib().ocs_split_quantize_workspace_bytes(self.O, self.C, 1, self.idx_map.numel() - self.C, N_BINS, N_CAND)
+        if nws + 256 > self.ws.numel():
+            self.ws = torch.empty(int(nws) + 256, dtype=torch.uint8, device=dev)
+        self.W_out = None      # never written
+
+    def ledger(self):
+        led = Ledger()
+        O, C, M = self.O, self.C, self.M
+        N = O * C
+        for r, _ in self.points:
+            S = configs_num_splits(C, r)
+            n = O * (C + S)
+            led.add("col_minmax_kernel", N=N)
+            led.add("split_hist_kernel", N=N)
+            led.add("split_quantize_kernel", N=N, n=n)
+            led.add("maxabs_kernel", n=M * C)
+            led.add("quantize_kernel", n=M * C)
+            led.add("ocs_gemm_kernel(linear)", rows=M, M=M, C=C, S=S, Nout=O)
+            led.ops += 2 * M * O * (C + S)
+        return led
+
+    def step(self):
+        ocs, C = self.ocs, self.C
+        for i, (r, bits) in enumerate(self.points):
+            S = ocs.ocs_num_splits(C, r)
+            ocs.ocs_split_quantize(self.W, S, bits, ocs.CLIP_MSE, n_candidates=N_CAND, n_bins=N_BINS,
+                                   out=(self.codes, self.scal[0:1], self.scal[1:2], self.idx_map, None, self.max_abs),
+                                   ws=self.ws, dev_status=self.status)
+            ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(self.a_codes, self.scal[2:3], self.scal[3:4]),
+                             ws=self.ws, dev_status=self.status)
+            ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S,
+                            out=self.Y[i], ws=self.ws, dev_status=self.status)
 
 
 class SmallFc(Fc6Sweep):
@@ -562,7 +611,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-small", "fc", "conv", "resnet50", "lstm"])
+    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -571,7 +620,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    wl = {"fc6": Fc6Sweep, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc, "conv": Conv3x3,
+    wl = {"fc6": Fc6Sweep, "fc6-fused": Fc6Fused, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc, "conv": Conv3x3,
           "resnet50": ResNet50, "lstm": Lstm}[args.workload]()
     net = getattr(wl, "kind", "") == "net"
 
@@ -665,7 +714,8 @@ def main():
     gemm_ms = sum(trace.get(k, (0, 0.0))[1] for k in ("ocs_gemm_kernel(linear)", "ocs_gemm_kernel(conv)",
                                                      "splitk_reduce_kernel"))
     gemm_tops = (led.ops * args.steps / (gemm_ms * 1e-3) / 1e12) if gemm_ms > 0 else None
-    sq_names = ("col_minmax_kernel", "split_scatter_kernel", "hist_kernel", "quantize_kernel", "maxabs_kernel")
+    sq_names = ("col_minmax_kernel", "split_scatter_kernel", "hist_kernel", "quantize_kernel", "maxabs_kernel",
+                "split_hist_kernel", "split_quantize_kernel")
     sq_ms = sum(trace[k][1] for k in sq_names if k in trace) + sum(
         trace[k][1] for k in ("split_plan_kernel", "score_kernel", "pick_kernel") if k in trace)
     sq_bytes = sum(led.bytes.get(k, 0) for k in sq_names) * args.steps
@@ -705,7 +755,7 @@ def main():
         ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype="int8 codes / int32 accumulate / fp32 scales", data="synthetic",
         config=dict(workload=wl.desc, l2=getattr(wl, "l2_note", None) or (
-            "inputs larger than L2 (no flush)" if wl.name == "fc6" else "inputs fit in L2; nothing is flushed between steps"),
+            "inputs larger than L2 (no flush)" if wl.name.startswith("fc6") else "inputs fit in L2; nothing is flushed between steps"),
                     bytes_per_step=led.total, int_ops_per_step=led.ops),
         parts=dict(split_quantize_gbs=sq_gbs, split_quantize_frac_of_hbm=(sq_gbs / pk["hbm"]) if sq_gbs else None,
                    gemm_tops=gemm_tops, gemm_frac_of_int8_peak=(gemm_tops / int8_peak) if gemm_tops else None,
