@@ -142,16 +142,32 @@ ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, int64_t ld_i
  * being read and written five times.  Results are bit-identical to the two separate calls:
  * codes int8 [O][(C+S)*R] in the split's layout with row stride ld_codes bytes, idx_map,
  * split_order (nullable), max_abs_out [3] (nullable), *scale, *alpha (nullable).
- * Arguments as in ocs_split and ocs_quantize (signed codes; modes NONE and MSE).
+ * Arguments as in ocs_split and ocs_quantize (modes NONE and MSE).
+ * Applied to an ACTIVATION matrix [rows][C] (R = 1, qa_bits = 0) this is the activation side
+ * of Eq. 4 with channels chosen on the batch at hand (the per-batch selection of Section 5.3):
+ * the chosen channels are duplicated and halved, and the codes come out already expanded,
+ * [rows][C+S]; ocs_dup_weight_columns provides the matching weight columns.
  * Limits: W 16-byte aligned, ld_in and C*R multiples of 4, and two expanded rows (plus the
  * histogram) must fit in shared memory ((C+S)*R up to about 27,000 floats); otherwise
  * OCS_ERR_UNSUPPORTED -- use the two separate calls.  Device flags: NONFINITE, DEPTH, TIMEOUT. */
 size_t ocs_split_quantize_workspace_bytes(int O, int C, int R, int S, int n_bins, int n_candidates);
 ocs_status ocs_split_quantize(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step,
-                              int qa_bits, int bits, ocs_clip_mode mode, int n_candidates, int n_bins,
+                              int qa_bits, int bits, int is_signed, ocs_clip_mode mode, int n_candidates, int n_bins,
                               int8_t* codes, int64_t ld_codes, int32_t* idx_map, int32_t* split_order,
                               float* max_abs_out, float* scale, float* alpha, void* ws, size_t ws_bytes,
                               int* dev_status, void* stream);
+
+/* ocs_dup_weight_columns ------------------------------------------------------------------
+ * Weight side of activation OCS (Eq. 4: the activation channel is halved in both copies, its
+ * weights are duplicated unchanged).  W_codes (device) int8 [N][ldw >= (C+S)*R] holds the layer's
+ * C weight channels, R taps each, in ocs_split's [channel][tap] order; channels C..C+S-1 are
+ * filled in place with W_codes[n][C+s][:] = W_codes[n][idx_map[C+s]][:].  With the expanded
+ * activation codes of ocs_split_quantize, ocs_qlinear (or, after ocs_pack_conv_weights,
+ * ocs_qconv) called with C+S plain channels and no gather evaluates the split layer.
+ * S = 0 is a no-op.  Device flag: BAD_INDEX (a source index outside [0, C); channel 0 is
+ * copied instead). */
+ocs_status ocs_dup_weight_columns(int8_t* W_codes, int N, int C, int R, int S, int64_t ldw, const int32_t* idx_map,
+                                  int* dev_status, void* stream);
 
 /* ocs_quantize_noalloc ---------------------------------------------------------------------
  * (No counterpart in the paper: a packaging variant of ocs_quantize.)

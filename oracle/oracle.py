@@ -128,6 +128,40 @@ def clip_mse_exact(T, bits: int, is_signed: bool = True, n_candidates: int = 128
     return dict(alpha=float(alpha.value), scores=scores)
 
 
+def act_ocs(A, S: int):
+    """Activation side of OCS (Eq. 4) with the channels chosen on the batch at hand (the
+    per-batch "Oracle OCS" of Section 5.3).  A [rows, C] holds one batch, one row per sample
+    (FC layer) or per pixel (conv layer, NHWC flattened): S times, the channel holding the largest
+    |a| of the batch is duplicated and BOTH copies are halved, which is the greedy rule of
+    Section 3.4 with the plain w/2 split.  -> (A' [rows, C+S], idx_map, split_order, (max|A|, max|A'|)).
+    A composition: the arithmetic is the checker's own split() on the matrix whose channel axis is
+    the activation's."""
+    A = _f32(A)
+    assert A.ndim == 2
+    return split(A, S, 0.0)
+
+
+def dup_weight_columns(Wc, idx_map):
+    """Weight side of Eq. 4: a duplicated activation channel meets an unchanged copy of its weights.
+    Wc [N, C] codes -> [N, C+S] with column j a copy of column idx_map[j]."""
+    Wc = np.asarray(Wc)
+    out = np.empty((Wc.shape[0], len(idx_map)), dtype=Wc.dtype)
+    for j, src in enumerate(idx_map):
+        out[:, j] = Wc[:, int(src)]
+    return out
+
+
+def act_ocs_linear(A, S: int, a_bits: int, a_signed: bool, Wc, w_scale, bias=None):
+    """One layer with per-batch activation OCS: split the batch (Eq. 4), quantize the expanded
+    activations on the grid of their own max |a'| (Section 3.1), duplicate the weight columns and
+    evaluate the integer layer.  -> (Y fp32 [rows, N], acc, A' codes, a_scale, idx_map)."""
+    Ap, idx, _, _ = act_ocs(A, S)
+    ac, a_scale = quantize(Ap, a_bits, a_signed, maxabs(Ap))
+    Wd = dup_weight_columns(Wc, idx)
+    Y, acc = qlinear(ac, a_signed, a_scale, Wd, w_scale, np.arange(len(idx), dtype=np.int32), bias)
+    return Y, acc, ac, a_scale, idx
+
+
 def _codes(a, signed):
     return np.ascontiguousarray(a, dtype=np.int8 if signed else np.uint8)
 

@@ -26,7 +26,7 @@ EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
     "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
     "ocs_split_workspace_bytes", "ocs_split",
-    "ocs_split_quantize_workspace_bytes", "ocs_split_quantize",
+    "ocs_split_quantize_workspace_bytes", "ocs_split_quantize", "ocs_dup_weight_columns",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
     "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
@@ -340,7 +340,8 @@ def ocs_quantize_noalloc(T, bits: int, is_signed: bool = True, mode: int = CLIP_
     return codes, scale, alpha
 
 
-def ocs_split_quantize(W, S: int, bits: int, mode: int = CLIP_NONE, qa_step: float = 0.0, qa_bits: int = 0,
+def ocs_split_quantize(W, S: int, bits: int, mode: int = CLIP_NONE, is_signed: bool = True, qa_step: float = 0.0,
+                       qa_bits: int = 0,
                        n_candidates: int = 128, n_bins: int = 2048, ld_codes: int | None = None, dev_status=None,
                        want_order: bool = True, out=None, ws=None):
     """Split + clip search + quantization without the fp32 W'.  W fp32 [O, C] or [O, C, kh, kw].
@@ -358,7 +359,7 @@ def ocs_split_quantize(W, S: int, bits: int, mode: int = CLIP_NONE, qa_step: flo
     else:
         if ld_codes is None:
             ld_codes = round_up(cols_out, 16)
-        codes = torch.empty((O, ld_codes), dtype=torch.int8, device=W.device)
+        codes = torch.empty((O, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=W.device)
         scale = torch.zeros(1, dtype=torch.float32, device=W.device)
         alpha = torch.zeros(1, dtype=torch.float32, device=W.device)
         idx_map = torch.empty(Cn + S, dtype=torch.int32, device=W.device)
@@ -368,8 +369,17 @@ def ocs_split_quantize(W, S: int, bits: int, mode: int = CLIP_NONE, qa_step: flo
     if ws is None:
         ws = _ws(nws, W.device)
     st = lib().ocs_split_quantize(_ptr(W), O, Cn, R, C.c_int64(Cn * R), int(S), C.c_float(qa_step), int(qa_bits),
-                                  int(bits), int(mode), int(n_candidates), int(n_bins), _ptr(codes),
+                                  int(bits), int(bool(is_signed)), int(mode), int(n_candidates), int(n_bins), _ptr(codes),
                                   C.c_int64(ld_codes), _ptr(idx_map), _ptr(order), _ptr(max_abs), _ptr(scale),
                                   _ptr(alpha), _ptr(ws), C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
     _check(st, "ocs_split_quantize")
     return codes, scale, alpha, idx_map, (order[:S] if order is not None else None), max_abs
+
+
+def ocs_dup_weight_columns(W_codes, C_in: int, S: int, idx_map, R: int = 1, dev_status=None):
+    """W_codes int8 [N, ldw >= (C+S)*R]: fills channels C..C+S-1 in place with copies of their sources."""
+    assert W_codes.is_cuda and W_codes.dtype == torch.int8 and W_codes.dim() == 2 and W_codes.stride(1) == 1
+    _check(lib().ocs_dup_weight_columns(_ptr(W_codes), W_codes.shape[0], int(C_in), int(R), int(S),
+                                        C.c_int64(W_codes.stride(0)), _ptr(idx_map), _ptr(dev_status), _stream()),
+           "ocs_dup_weight_columns")
+    return W_codes

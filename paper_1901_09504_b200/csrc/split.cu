@@ -655,7 +655,8 @@ struct RowsEpilogue {
   int hist_copies;              // HIST: private copies in shared memory behind the row buffers
   const double* scores;         // QUANT: candidate scores (null: no clipping)
   int n_candidates;
-  int L;                        // QUANT: code range [-L, L]
+  int L;                        // QUANT: code range [-L, L], or [0, L] for unsigned codes
+  int is_signed;
   int8_t* codes;                // QUANT: [O][ld_codes]
   long long ld_codes;
   int packed_ok;                // QUANT: 32-bit stores of four codes allowed
@@ -699,7 +700,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
     const bool zero = !(alpha > 0.0f);
     const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)ep.L);
     q_inv = zero ? 0.0f : __fdiv_rn((float)ep.L, alpha);
-    q_lo = -(float)ep.L; q_hi = (float)ep.L;
+    q_lo = ep.is_signed ? -(float)ep.L : 0.0f; q_hi = (float)ep.L;
     if (blockIdx.x == 0 && tid == 0) {
       *ep.scale_out = step;
       if (ep.alpha_out) *ep.alpha_out = zero ? 0.0f : alpha;
@@ -1109,7 +1110,8 @@ extern "C" size_t ocs_split_quantize_workspace_bytes(int O, int C, int R, int S,
 }
 
 extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step,
-                                         int qa_bits, int bits, ocs_clip_mode mode, int n_candidates, int n_bins,
+                                         int qa_bits, int bits, int is_signed, ocs_clip_mode mode, int n_candidates,
+                                         int n_bins,
                                          int8_t* codes, int64_t ld_codes, int32_t* idx_map, int32_t* split_order,
                                          float* max_abs_out, float* scale, float* alpha, void* ws, size_t ws_bytes,
                                          int* dev_status, void* stream_) {
@@ -1156,10 +1158,11 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
       return OCS_ERR_CUDA;
     attr_set = true;
   }
-  const int L = (1 << (bits - 1)) - 1;
+  const int L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
   RowsEpilogue ep{};
   ep.maxp = mx3 + 1;   // max|W'| as the plan computed it
   ep.L = L;
+  ep.is_signed = is_signed ? 1 : 0;
   const double* scores = nullptr;
   if (mode == OCS_CLIP_MSE) {
     if (cudaMemsetAsync(f.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
@@ -1175,7 +1178,7 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
           ep, dev_status);
     }
     if ((st = launch_status()) != OCS_OK) return st;
-    if ((st = launch_score_kernel(f.hist, ep.maxp, n_bins, n_candidates, L, 1, f.scores, stream)) != OCS_OK) return st;
+    if ((st = launch_score_kernel(f.hist, ep.maxp, n_bins, n_candidates, L, is_signed ? 1 : 0, f.scores, stream)) != OCS_OK) return st;
     scores = f.scores;
   }
   ep.scores = scores;
@@ -1191,5 +1194,45 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
         W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g, srow, ep,
         dev_status);
   }
+  return launch_status();
+}
+
+// ------------------------------------------------------------------------------------------------
+// ocs_dup_weight_columns: the weight side of activation OCS (Eq. 4): the duplicated channels'
+// weight columns are plain copies, Wc[n][C + s][:] = Wc[n][idx_map[C + s]][:] (R taps per channel).
+namespace ocs {
+namespace {
+__global__ void __launch_bounds__(256)
+dup_columns_kernel(int8_t* __restrict__ Wc, int N, int C, int R, int S, long long ldw,
+                   const int32_t* __restrict__ idx_map, int* dev_status) {
+  const long long per_row = (long long)S * R;
+  const long long total = (long long)N * per_row;
+  bool bad = false;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+    const long long n = i / per_row;
+    const int rem = (int)(i - n * per_row);
+    const int sidx = rem / R;
+    const int r = rem - sidx * R;
+    int src = __ldg(idx_map + C + sidx);
+    if ((unsigned)src >= (unsigned)C) { bad = true; src = 0; }
+    Wc[n * ldw + (long long)(C + sidx) * R + r] = Wc[n * ldw + (long long)src * R + r];
+  }
+  if (bad) flag(dev_status, OCS_DEV_BAD_INDEX);
+}
+}  // namespace
+}  // namespace ocs
+
+extern "C" ocs_status ocs_dup_weight_columns(int8_t* W_codes, int N, int C, int R, int S, int64_t ldw,
+                                             const int32_t* idx_map, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!W_codes || !idx_map || S < 0) return OCS_ERR_INVALID_ARG;
+  if (N <= 0 || C <= 0 || R <= 0 || ldw < ((int64_t)C + S) * R) return OCS_ERR_SHAPE;
+  if (S == 0) return OCS_OK;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  const long long total = (long long)N * S * R;
+  const int grid = (int)min((total + 255) / 256, (long long)kNumSMs * 8);
+  LaunchScope ls("dup_columns_kernel", stream);
+  dup_columns_kernel<<<grid, 256, 0, stream>>>(W_codes, N, C, R, S, ldw, idx_map, dev_status);
   return launch_status();
 }

@@ -148,3 +148,40 @@ def lstm_forward(cfg, layers, tokens, a_bits: int = 8, keep: bool = False, dev_s
             x = hn
     logits = linear_forward(layers["W_dec"], tops.view(seq * batch, hidden), True, a_bits, dev_status)
     return (logits, dict(emb=emb, tops=tops, c=c)) if keep else logits
+
+
+# ------------------------------------------------------------------------------ activation OCS
+def act_ocs_linear_forward(W_codes, w_scale, bias, x, S: int, a_bits: int, a_signed: bool, dev_status=None):
+    """Per-batch activation OCS (Eq. 4, Section 5.3) for a linear layer: x fp32 [M, C], W_codes int8
+    [N, ld >= C] unsplit weight codes.  The batch's S outlier channels are duplicated and halved while
+    being quantized (ocs_split_quantize on x), the weight columns are duplicated (ocs_dup_weight_columns)
+    and the integer layer runs on C+S plain channels.  -> (Y fp32 [M, N], idx_map)."""
+    M, Cn = x.shape
+    N = W_codes.shape[0]
+    ld = B.round_up(Cn + S, 16)
+    xc, xs, _, idx_map, _, _ = B.ocs_split_quantize(x.contiguous(), S, a_bits, B.CLIP_NONE, is_signed=a_signed,
+                                                    ld_codes=ld, dev_status=dev_status, want_order=False)
+    Wd = torch.zeros((N, ld), dtype=torch.int8, device=x.device)
+    Wd[:, :Cn] = W_codes[:, :Cn]
+    B.ocs_dup_weight_columns(Wd, Cn, S, idx_map, dev_status=dev_status)
+    ident = torch.arange(Cn + S, dtype=torch.int32, device=x.device)
+    return B.ocs_qlinear(xc, xs, Wd, w_scale, ident, Cn + S, 0, bias=bias, dev_status=dev_status), idx_map
+
+
+def act_ocs_conv_forward(W_codes, w_scale, bias, x, S: int, k: int, stride: int, pad: int, a_bits: int,
+                         a_signed: bool, dev_status=None):
+    """The same for a convolution: x fp32 NHWC, W_codes int8 [O, ld >= C*k*k] unsplit codes in
+    [channel][tap] order.  The batch's pixels are the rows of the activation matrix."""
+    Nb, H, Wd_, Cn = x.shape
+    O, R = W_codes.shape[0], k * k
+    xc, xs, _, idx_map, _, _ = B.ocs_split_quantize(x.reshape(Nb * H * Wd_, Cn), S, a_bits, B.CLIP_NONE,
+                                                    is_signed=a_signed, ld_codes=Cn + S, dev_status=dev_status,
+                                                    want_order=False)
+    Wdup = torch.zeros((O, B.round_up((Cn + S) * R, 16)), dtype=torch.int8, device=x.device)
+    Wdup[:, :Cn * R] = W_codes[:, :Cn * R]
+    B.ocs_dup_weight_columns(Wdup, Cn, S, idx_map, R=R, dev_status=dev_status)
+    packed = B.ocs_pack_conv_weights(Wdup, O, Cn + S, 0, k, k)
+    ident = torch.arange(Cn + S, dtype=torch.int32, device=x.device)
+    y = B.ocs_qconv(xc.view(Nb, H, Wd_, Cn + S), xs, packed, w_scale, ident, 0, k, k, stride, pad, bias=bias,
+                    dev_status=dev_status)
+    return y, idx_map

@@ -131,6 +131,53 @@ def test_functional_identity_and_exact_halving(shape, S):
     assert mx[0] == np.abs(W).max() and mx[1] == np.abs(out).max()
 
 
+# ----------------------------------------------------------------------------- Eq. 4
+def test_activation_ocs_keeps_the_layer_and_halves_the_outlier():
+    """Eq. 4: with the chosen activation channels duplicated and halved and their weight columns
+    duplicated unchanged, the layer output is the original one; on integer data every sum is exact."""
+    rng = np.random.default_rng(23)
+    M, Cn, N, S = 7, 12, 5, 6
+    A = (rng.integers(-8, 9, size=(M, Cn)) * 64).astype(np.float32)      # halvings stay integers
+    A[3, 4] = 64 * 40                                                      # the batch's outlier
+    W = rng.integers(-9, 10, size=(N, Cn)).astype(np.int8)
+    Ap, idx, order, mx = orc.act_ocs(A, S)
+    Wd = orc.dup_weight_columns(W, idx)
+    assert Wd.shape == (N, Cn + S) and np.array_equal(Wd[:, :Cn], W)
+    for s in range(S):
+        assert np.array_equal(Wd[:, Cn + s], W[:, idx[Cn + s]])
+    y_ref = A.astype(np.int64) @ W.astype(np.int64).T
+    y_new = Ap.astype(np.float64) @ Wd.astype(np.float64).T
+    np.testing.assert_array_equal(y_new, y_ref.astype(np.float64))
+    # both copies carry half of the value they were split from, the outlier's channel goes first
+    assert order[0] == 4 and idx[Cn] == 4
+    assert mx[0] == 64 * 40 and mx[1] < mx[0]
+    cols = np.zeros((M, Cn), dtype=np.float64)
+    np.add.at(cols, (slice(None), idx), Ap.astype(np.float64))
+    np.testing.assert_array_equal(cols, A.astype(np.float64))
+    # a channel split once: both copies are exactly a/2 (the plain split of Section 3.3)
+    A1, idx1, _, _ = orc.act_ocs(A, 1)
+    np.testing.assert_array_equal(A1[:, 4], A[:, 4] * 0.5)
+    np.testing.assert_array_equal(A1[:, Cn], A[:, 4] * 0.5)
+    others = [c for c in range(Cn) if c != 4]
+    np.testing.assert_array_equal(A1[:, others], A[:, others])
+
+
+def test_activation_ocs_layer_is_the_expanded_integer_layer():
+    """The composed layer against a plain integer matmul on its own outputs, and the grid refinement
+    the split buys: the expanded batch's max |a'| is what sets the scale."""
+    c1 = configs.config1()
+    A = c1["A"].copy()
+    A[2, 17] = 25.0
+    Wc, w_scale = orc.quantize(c1["W"], 8, True, orc.maxabs(c1["W"]))
+    S = 5
+    Y, acc, ac, a_scale, idx = orc.act_ocs_linear(A, S, 6, False, Wc, w_scale, None)
+    ref = ac.astype(np.int64) @ Wc[:, idx].astype(np.int64).T
+    np.testing.assert_array_equal(acc, ref)
+    _, a_scale0 = orc.quantize(A, 6, False, orc.maxabs(A))
+    assert a_scale < a_scale0 and idx[A.shape[1]] == 17
+    assert ac.max() == 63 and ac.min() >= 0
+
+
 def test_greedy_is_monotone_and_targets_the_outlier():
     """Section 3.4 / 5.2: each split halves the current maximum's channel; the maximum never
     rises; with a unique largest outlier the first split strictly narrows the range."""
