@@ -1,6 +1,6 @@
 """Benchmark of the OCS hot path on B200: split -> clip search -> quantize -> int8 GEMM/conv.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-fused|fc6-small|fc|conv|resnet50|lstm] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-fused|fc6-small|fc|conv|resnet50|lstm|act-ocs] [--impl reference]
 
 One step is one pass of the whole path over one batch of synthetic input:
   fc6   (default) the VGG-16-fc6-shaped sweep: W [4096, 25088], 5 expand ratios x 4 weight bit
@@ -12,6 +12,8 @@ One step is one pass of the whole path over one batch of synthetic input:
   conv / resnet50 / lstm   the single 3x3 convolution, the ResNet-50 stack at batch 128 and the LSTM
         language model: a step prepares every layer (split, quantize, pack) and runs the forward pass;
         these report integer TOP/s of the quantized layers instead of bytes per second.
+  act-ocs  per-batch activation OCS (Eq. 4) on a ResNet-50 stage-1 1x1 convolution at batch 128: channel
+        extrema, split plan, expanded 6-bit activation codes, duplicated weight columns, integer layer.
 The reported value is algorithmic bytes per second: the bytes the method must move (listed in
 `algorithmic_bytes` below) divided by the step time.  Rank 0 prints one JSON line.
 
@@ -34,7 +36,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from ocs_inputs import configs  # noqa: E402
+from ocs_inputs import configs, prng  # noqa: E402
 
 N_BINS, N_CAND = 2048, 128
 INT8_OVER_BF16 = 2.0          # nominal dense int8 rate / nominal dense bf16 rate of the part
@@ -311,6 +313,88 @@ class Fc6Fused(Fc6Sweep):
                              ws=self.ws, dev_status=self.status)
             ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S,
                             out=self.Y[i], ws=self.ws, dev_status=self.status)
+
+
+class ActOcs(Fc6Sweep):
+    """Per-batch activation OCS (Eq. 4, Section 5.3) on a ResNet-50 stage-1 1x1 convolution at batch 128."""
+    name = "act-ocs"
+    l2_note = "activations larger than L2 (no flush)"
+
+    def __init__(self):
+        self.Nb, self.H, self.C, self.O, self.S, self.bits = 128, 56, 256, 64, 6, 6
+        self.rows = self.Nb * self.H * self.H
+        self.desc = (f"per-batch activation OCS with Table 4's settings (r = 0.02 -> {self.S} splits, {self.bits} activation "
+                     f"bits, batch {self.Nb}) on a ResNet-50 stage-1 1x1 convolution: activations NHWC [{self.Nb}, {self.H}, "
+                     f"{self.H}, {self.C}] fp32 half-normal, weights [{self.O}, {self.C}] as 8-bit codes; a step = channel "
+                     "extrema + split plan + expanded unsigned codes (ocs_split_quantize), ocs_dup_weight_columns and the "
+                     "integer layer (ocs_qlinear over the pixels); seed 5")
+        self.oracle_sample_desc = "the same layer on 8 of the 128 images (its own batch: 25088 pixels)"
+
+    def host_inputs(self):
+        X = prng.normal(5, 0, (self.rows, self.C), 1.0, absolute=True)
+        W = prng.laplace(5, 1, (self.O, self.C), 0.02)
+        return dict(X=X, W=W)
+
+    def setup(self, ocs, torch, dev, host):
+        self.ocs, self.torch = ocs, torch
+        rows, C, O, S = self.rows, self.C, self.O, self.S
+        self.ld = ocs.round_up(C + S, 16)
+        self.X = host["X"].to(dev)
+        self.status = ocs.new_status(dev)
+        Wd = host["W"].to(dev)
+        self.w_codes, self.w_scale, _ = ocs.ocs_quantize(Wd, 8, True, ocs.CLIP_NONE, ld_codes=self.ld)
+        self.w_codes[:, C:] = 0
+        self.codes = torch.empty((rows, self.ld), dtype=torch.uint8, device=dev)
+        self.idx_map = torch.empty(C + S, dtype=torch.int32, device=dev)
+        self.ident = torch.arange(C + S, dtype=torch.int32, device=dev)
+        self.max_abs = torch.zeros(3, dtype=torch.float32, device=dev)
+        self.scal = torch.zeros(2, dtype=torch.float32, device=dev)
+        self.Y = torch.empty((rows, O), dtype=torch.float32, device=dev)
+        L = ocs.lib()
+        nws = max(L.ocs_split_quantize_workspace_bytes(rows, C, 1, S, N_BINS, N_CAND),
+                  L.ocs_qlinear_workspace_bytes(rows, O, C + S, 0))
+        self.ws = torch.empty(int(nws) + 256, dtype=torch.uint8, device=dev)
+
+    def ledger(self):
+        led = Ledger()
+        rows, C, O, S = self.rows, self.C, self.O, self.S
+        led.add("col_minmax_kernel", N=rows * C)
+        led.add("split_quantize_kernel", N=rows * C, n=rows * (C + S))
+        led.add("ocs_gemm_kernel(linear)", rows=rows, M=rows, C=C + S, S=0, Nout=O)
+        led.ops = 2 * rows * O * (C + S)
+        return led
+
+    def step(self):
+        ocs, C, S = self.ocs, self.C, self.S
+        ocs.ocs_split_quantize(self.X, S, self.bits, ocs.CLIP_NONE, is_signed=False,
+                               out=(self.codes, self.scal[0:1], self.scal[1:2], self.idx_map, None, self.max_abs),
+                               ws=self.ws, dev_status=self.status)
+        ocs.ocs_dup_weight_columns(self.w_codes, C, S, self.idx_map, dev_status=self.status)
+        ocs.ocs_qlinear(self.codes, self.scal[0:1], self.w_codes, self.w_scale, self.ident, C + S, 0, out=self.Y,
+                        ws=self.ws, dev_status=self.status)
+
+    def e2e_buffers(self, host):
+        self.hX = self.torch.from_numpy(host["X"]).pin_memory()
+        self.hY = self.torch.empty(self.Y.shape, dtype=self.torch.float32).pin_memory()
+        return self.hX.numel() * 4, self.hY.numel() * 4
+
+    def step_e2e(self):
+        self.X.copy_(self.hX, non_blocking=True)
+        self.step()
+        self.hY.copy_(self.Y, non_blocking=True)
+
+    def oracle_sample(self, orc, host):
+        rows = 8 * self.H * self.H
+        X, W = host["X"][:rows], host["W"]
+        t0 = time.perf_counter()
+        wc, ws = orc.quantize(W, 8, True, orc.maxabs(W))
+        orc.act_ocs_linear(X, self.S, self.bits, False, wc, ws, None)
+        sec = time.perf_counter() - t0
+        led = Ledger()
+        led.add("col_minmax_kernel", N=rows * self.C)
+        led.add("split_quantize_kernel", N=rows * self.C, n=rows * (self.C + self.S))
+        led.add("ocs_gemm_kernel(linear)", rows=rows, M=rows, C=self.C + self.S, S=0, Nout=self.O)
+        return sec, led.total
 
 
 class SmallFc(Fc6Sweep):
@@ -611,7 +695,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm"])
+    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm", "act-ocs"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -621,7 +705,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     wl = {"fc6": Fc6Sweep, "fc6-fused": Fc6Fused, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc, "conv": Conv3x3,
-          "resnet50": ResNet50, "lstm": Lstm}[args.workload]()
+          "resnet50": ResNet50, "lstm": Lstm, "act-ocs": ActOcs}[args.workload]()
     net = getattr(wl, "kind", "") == "net"
 
     if args.impl == "reference":
