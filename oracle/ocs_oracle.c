@@ -339,6 +339,64 @@ int ocs_oracle_qconv(const void* X, int a_signed, float a_scale, int Nb, int H, 
   return err;
 }
 
+/* ------------------------------------------------------------------ Section 5.3: static activation OCS */
+static int cmp_float_asc(const void* a, const void* b) {
+  const float x = *(const float*)a, y = *(const float*)b;
+  return (x > y) - (x < y);
+}
+
+int ocs_oracle_act_select(const float* P, int64_t rows, int C, int S, double quantile,
+                          int32_t* sel, int64_t* counts, float* thr) {
+  if (!P || !sel || rows <= 0 || C <= 0 || S < 0 || S > C) return 1;
+  if (!(quantile > 0.0) || !(quantile <= 1.0)) return 1;
+  const int64_t n = rows * (int64_t)C;
+  float* v = (float*)malloc(sizeof(float) * (size_t)n);
+  int64_t* cnt = (int64_t*)calloc((size_t)C, sizeof(int64_t));
+  char* taken = (char*)calloc((size_t)C, 1);
+  if (!v || !cnt || !taken) { free(v); free(cnt); free(taken); return 2; }
+  for (int64_t i = 0; i < n; ++i) v[i] = fabsf(P[i]);
+  qsort(v, (size_t)n, sizeof(float), cmp_float_asc);
+  int64_t k = (int64_t)ceil(quantile * (double)n - 1e-9);
+  if (k < 1) k = 1;
+  if (k > n) k = n;
+  const float t = v[k - 1];
+  for (int64_t m = 0; m < rows; ++m)
+    for (int c = 0; c < C; ++c)
+      if (fabsf(P[m * C + c]) > t) cnt[c] += 1;
+  for (int s = 0; s < S; ++s) {
+    int best = -1;
+    for (int c = 0; c < C; ++c)
+      if (!taken[c] && (best < 0 || cnt[c] > cnt[best])) best = c;
+    taken[best] = 1;
+    sel[s] = best;
+  }
+  if (counts) memcpy(counts, cnt, sizeof(int64_t) * (size_t)C);
+  if (thr) *thr = t;
+  free(v); free(cnt); free(taken);
+  return 0;
+}
+
+int ocs_oracle_act_split_static(const float* A, int64_t rows, int C, int S, const int32_t* sel,
+                                float* A_out, int32_t* idx_map) {
+  if (!A || !A_out || !idx_map || rows <= 0 || C <= 0 || S < 0 || S > C || (S > 0 && !sel)) return 1;
+  char* chosen = (char*)calloc((size_t)C, 1);
+  if (!chosen) return 2;
+  for (int s = 0; s < S; ++s) {
+    if (sel[s] < 0 || sel[s] >= C || chosen[sel[s]]) { free(chosen); return 1; }
+    chosen[sel[s]] = 1;
+  }
+  for (int c = 0; c < C; ++c) idx_map[c] = c;
+  for (int s = 0; s < S; ++s) idx_map[C + s] = sel[s];
+  for (int64_t m = 0; m < rows; ++m) {
+    const float* a = A + m * C;
+    float* o = A_out + m * (int64_t)(C + S);
+    for (int c = 0; c < C; ++c) o[c] = chosen[c] ? a[c] * 0.5f : a[c];
+    for (int s = 0; s < S; ++s) o[C + s] = a[sel[s]] * 0.5f;
+  }
+  free(chosen);
+  return 0;
+}
+
 /* ------------------------------------------------------------------ glue */
 void ocs_oracle_relu(const float* x, int64_t n, float* y) {
   for (int64_t i = 0; i < n; ++i) y[i] = x[i] > 0.0f ? x[i] : 0.0f;

@@ -13,9 +13,11 @@
  * unsigned codes.  All functions return 0 on success, non-zero on a bad argument.
  *
  * Pinned by tests (paper facts, closed forms, brute force): split, quantize, clip_mse,
- * qlinear, qconv, pools, relu/add.  Parity unpinned (conventions the paper does not fix,
+ * qlinear, qconv, pools, relu/add, act_select, act_split_static.  Parity unpinned (conventions the paper does not fix,
  * enforced only checker-vs-GPU): the QA grid-step policy, the unsigned activation grid,
- * the bin count and the tie rule of the clip search, the LSTM cell's sigmoid/tanh routines.
+ * the bin count and the tie rule of the clip search, the LSTM cell's sigmoid/tanh routines,
+ * the quantile convention of act_select (nearest rank on |a|; the paper says only "99th
+ * percentile").
  */
 #ifndef OCS_ORACLE_H
 #define OCS_ORACLE_H
@@ -90,6 +92,21 @@ int ocs_oracle_qlinear_samples(const void* A, int a_signed, float a_scale, int M
 int ocs_oracle_qconv(const void* X, int a_signed, float a_scale, int Nb, int H, int Wd, int C,
                      const int8_t* Wc, float w_scale, int O, int S, int kh, int kw, int stride,
                      int pad, const int32_t* idx_map, const float* bias, float* Y, int32_t* acc);
+
+/* Section 5.3, static activation OCS: which channels to split is decided once, on sampled
+ * activations P [rows][C].  t = the `quantile` (the paper uses 0.99) quantile of all |a| by
+ * nearest rank: the k-th smallest value, k = ceil(quantile * n - 1e-9) clamped to [1, n],
+ * n = rows * C.  counts[c] = number of samples of channel c with |a| > t.  sel[0..S) = the S
+ * channels with the highest counts (ties: smallest channel index), highest first.  S <= C.
+ * counts [C] and thr may be NULL. */
+int ocs_oracle_act_select(const float* P, int64_t rows, int C, int S, double quantile,
+                          int32_t* sel, int64_t* counts, float* thr);
+
+/* Eq. 4 for a fixed channel list: each channel in sel (distinct, in [0, C)) is duplicated and
+ * both copies become fl(a * 0.5); A_out [rows][C+S], the copy of sel[s] at index C + s;
+ * idx_map[C+S] as in the weight split. */
+int ocs_oracle_act_split_static(const float* A, int64_t rows, int C, int S, const int32_t* sel,
+                                float* A_out, int32_t* idx_map);
 
 /* Elementwise / pooling glue of the end-to-end networks, each a single rounded fp32 op per
  * output in a fixed order.  Tensors NHWC. */

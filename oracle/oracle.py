@@ -162,6 +162,36 @@ def act_ocs_linear(A, S: int, a_bits: int, a_signed: bool, Wc, w_scale, bias=Non
     return Y, acc, ac, a_scale, idx
 
 
+def act_select(P, S: int, quantile: float = 0.99):
+    """Static channel choice of Section 5.3 on sampled activations P [rows, C]
+    -> (sel int32 [S], counts int64 [C], threshold)."""
+    P = _f32(P)
+    assert P.ndim == 2
+    rows, Cn = P.shape
+    sel = np.empty(max(S, 1), dtype=np.int32)
+    counts = np.zeros(Cn, dtype=np.int64)
+    thr = C.c_float(0)
+    rc = lib().ocs_oracle_act_select(_p(P, _f32p), C.c_int64(rows), Cn, int(S), C.c_double(quantile),
+                                     _p(sel, _i32p), counts.ctypes.data_as(C.POINTER(C.c_int64)), C.byref(thr))
+    _check(rc, "act_select")
+    return sel[:S], counts, float(thr.value)
+
+
+def act_split_static(A, sel):
+    """Eq. 4 for a fixed channel list -> (A' [rows, C+S], idx_map)."""
+    A = _f32(A)
+    assert A.ndim == 2
+    rows, Cn = A.shape
+    sel = np.ascontiguousarray(sel, dtype=np.int32)
+    S = sel.size
+    out = np.empty((rows, Cn + S), dtype=np.float32)
+    idx = np.empty(Cn + S, dtype=np.int32)
+    rc = lib().ocs_oracle_act_split_static(_p(A, _f32p), C.c_int64(rows), Cn, S, _p(sel, _i32p), _p(out, _f32p),
+                                           _p(idx, _i32p))
+    _check(rc, "act_split_static")
+    return out, idx
+
+
 def _codes(a, signed):
     return np.ascontiguousarray(a, dtype=np.int8 if signed else np.uint8)
 

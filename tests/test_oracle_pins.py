@@ -178,6 +178,67 @@ def test_activation_ocs_layer_is_the_expanded_integer_layer():
     assert ac.max() == 63 and ac.min() >= 0
 
 
+# ----------------------------------------------------------------------------- Section 5.3
+@pytest.mark.parametrize("rows,Cn,S,q,seed", [(50, 16, 4, 0.99, 0), (7, 5, 5, 0.5, 1), (200, 33, 1, 0.9, 2),
+                                               (3, 4, 0, 0.99, 3), (64, 8, 3, 1.0, 4)])
+def test_static_channel_choice_against_library_routines(rows, Cn, S, q, seed):
+    """Threshold = numpy's nearest-rank quantile of |a|; counts and the top-S rule recomputed with
+    library routines (stable argsort on negated counts = highest count first, ties by index)."""
+    rng = np.random.default_rng(seed)
+    P = rng.standard_normal((rows, Cn)).astype(np.float32)
+    P[:, Cn // 2] *= 3.0                                  # one channel with heavier tails
+    P[rng.integers(0, rows, 5), rng.integers(0, Cn, 5)] = 0.0
+    sel, counts, thr = orc.act_select(P, S, q)
+    ref_thr = np.quantile(np.abs(P).ravel(), q, method="inverted_cdf")
+    assert np.float32(thr) == np.float32(ref_thr)
+    ref_counts = (np.abs(P) > ref_thr).sum(axis=0)
+    np.testing.assert_array_equal(counts, ref_counts)
+    assert counts.sum() == P.size - np.sum(np.abs(P).ravel() <= ref_thr)
+    np.testing.assert_array_equal(sel, np.argsort(-ref_counts, kind="stable")[:S])
+    if S and q < 1.0:
+        assert Cn // 2 in sel.tolist()
+
+
+def test_static_channel_choice_tiny_worked_case():
+    """Ten samples of three channels, by hand: 0.9-quantile of |a| is the 27th smallest of 30."""
+    P = np.zeros((10, 3), np.float32)
+    P[:, 0] = np.arange(1, 11)            # 1..10
+    P[:, 1] = -np.arange(11, 21)          # -11..-20: the largest magnitudes
+    P[:, 2] = np.arange(21, 31) * 0.01    # small
+    sel, counts, thr = orc.act_select(P, 2, 0.9)
+    assert thr == 17.0 and counts.tolist() == [0, 3, 0]
+    assert sel.tolist() == [1, 0]         # the tie between channels 0 and 2 goes to the smaller index
+
+
+def test_static_activation_split_is_eq4_with_a_fixed_list():
+    rng = np.random.default_rng(5)
+    M, Cn, N = 9, 10, 4
+    A = (rng.integers(-20, 21, size=(M, Cn)) * 2).astype(np.float32)
+    W = rng.integers(-9, 10, size=(N, Cn)).astype(np.int8)
+    sel = np.array([7, 2, 3], np.int32)
+    Ap, idx = orc.act_split_static(A, sel)
+    assert idx.tolist() == list(range(Cn)) + [7, 2, 3]
+    for s, c in enumerate(sel):
+        np.testing.assert_array_equal(Ap[:, c], A[:, c] / 2)
+        np.testing.assert_array_equal(Ap[:, Cn + s], A[:, c] / 2)
+    rest = [c for c in range(Cn) if c not in sel.tolist()]
+    np.testing.assert_array_equal(Ap[:, rest], A[:, rest])
+    Wd = orc.dup_weight_columns(W, idx)
+    np.testing.assert_array_equal(Ap.astype(np.float64) @ Wd.astype(np.float64).T,
+                                  (A.astype(np.int64) @ W.astype(np.int64).T).astype(np.float64))
+    # the same list applied through the greedy per-batch rule when that rule picks these channels once each
+    B = np.ones((2, 4), np.float32)
+    B[0, 3], B[1, 1] = 9.0, 8.0
+    Bp, bidx, order, _ = orc.act_ocs(B, 2)
+    Bs, sidx = orc.act_split_static(B, order)
+    np.testing.assert_array_equal(Bp, Bs)
+    np.testing.assert_array_equal(bidx, sidx)
+    with pytest.raises(RuntimeError):
+        orc.act_split_static(A, np.array([1, 1], np.int32))        # a channel listed twice
+    with pytest.raises(RuntimeError):
+        orc.act_split_static(A, np.array([Cn], np.int32))
+
+
 def test_greedy_is_monotone_and_targets_the_outlier():
     """Section 3.4 / 5.2: each split halves the current maximum's channel; the maximum never
     rises; with a unique largest outlier the first split strictly narrows the range."""
