@@ -169,6 +169,39 @@ ocs_status ocs_split_quantize(const float* W, int O, int C, int R, int64_t ld_in
 ocs_status ocs_dup_weight_columns(int8_t* W_codes, int N, int C, int R, int S, int64_t ldw, const int32_t* idx_map,
                                   int* dev_status, void* stream);
 
+/* ocs_act_select_channels --------------------------------------------------------------------
+ * Static channel choice for activation OCS (Section 5.3: count, per channel, the sampled values
+ * above the 99th percentile and split the channels with the highest counts).
+ * P (device) fp32 [rows][ldp >= C]: sampled activations, one row per sample or pixel.
+ * t = the `quantile` quantile (0 < quantile <= 1; the paper uses 0.99) of all |a| by nearest rank:
+ * the k-th smallest, k = ceil(quantile * rows * C - 1e-9) clamped to [1, rows * C] -- exact, found
+ * by a radix select over the bit patterns.  counts[c] = samples of channel c with |a| > t.
+ * sel (device, int32 [S], S <= C) = the S channels with the highest counts, highest first, ties to
+ * the smaller channel index.  counts (device, int64 [C]) and threshold (device, fp32 [1]) may be
+ * NULL.  Workspace (device, 256-byte aligned): ocs_act_select_workspace_bytes(C).  Four passes
+ * over P; asynchronous on `stream`.  Device flag: NONFINITE (such samples are left out). */
+size_t ocs_act_select_workspace_bytes(int C);
+ocs_status ocs_act_select_channels(const float* P, int64_t rows, int C, int64_t ldp, int S, double quantile,
+                                   int32_t* sel, int64_t* counts, float* threshold, void* ws, size_t ws_bytes,
+                                   int* dev_status, void* stream);
+
+/* ocs_act_split_quantize_static --------------------------------------------------------------
+ * Activation side of Eq. 4 for a channel list chosen ahead of time (Section 5.3's static variant;
+ * Section 3.5's "custom layer" that copies and scales the listed channels), fused with the
+ * quantization: A (device) fp32 [rows][ld_in >= C]; every channel in sel (device, int32 [S],
+ * distinct, in [0, C)) is duplicated and both copies carry a * 0.5; codes (device, int8 or the uint8
+ * bit pattern) [rows][ld_codes >= C+S], the copy of sel[s] at column C + s; idx_map (device,
+ * int32 [C+S]) as in ocs_split.  Grid: alpha_in (device, fp32 [1]) when given -- a threshold
+ * profiled ahead of time, values beyond it saturate -- else max |a'| of this batch (one extra pass
+ * over A).  *scale (device) = alpha / L.  Workspace: ocs_split_quantize_workspace_bytes(rows, C,
+ * 1, S, 1, 1).  Same staging limits as ocs_split_quantize (OCS_ERR_UNSUPPORTED otherwise).
+ * Device flags: BAD_INDEX (an entry of sel outside [0, C) or listed twice; outputs unspecified),
+ * NONFINITE (dynamic grid: non-finite input; static grid: alpha_in negative or non-finite). */
+ocs_status ocs_act_split_quantize_static(const float* A, int rows, int C, int64_t ld_in, int S, const int32_t* sel,
+                                         int bits, int is_signed, const float* alpha_in, int8_t* codes,
+                                         int64_t ld_codes, int32_t* idx_map, float* scale, void* ws, size_t ws_bytes,
+                                         int* dev_status, void* stream);
+
 /* ocs_quantize_noalloc ---------------------------------------------------------------------
  * (No counterpart in the paper: a packaging variant of ocs_quantize.)
  * Same operation, arguments and results as ocs_quantize, minus (ws, ws_bytes).  It is meant for

@@ -27,6 +27,7 @@ EXPORTS = [
     "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
     "ocs_split_workspace_bytes", "ocs_split",
     "ocs_split_quantize_workspace_bytes", "ocs_split_quantize", "ocs_dup_weight_columns",
+    "ocs_act_select_workspace_bytes", "ocs_act_select_channels", "ocs_act_split_quantize_static",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
     "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
@@ -51,7 +52,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.ocs_num_splits.argtypes = [C.c_int, C.c_double]
         L.ocs_version.restype = C.c_char_p
-        for name in ("ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
+        for name in ("ocs_act_select_workspace_bytes", "ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
                      "ocs_qconv_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.ocs_quantize_workspace_views.restype = None
@@ -383,3 +384,45 @@ def ocs_dup_weight_columns(W_codes, C_in: int, S: int, idx_map, R: int = 1, dev_
                                         C.c_int64(W_codes.stride(0)), _ptr(idx_map), _ptr(dev_status), _stream()),
            "ocs_dup_weight_columns")
     return W_codes
+
+
+def ocs_act_select_channels(P, S: int, quantile: float = 0.99, dev_status=None):
+    """P fp32 [rows, C] sampled activations -> (sel int32 [S], counts int64 [C], threshold fp32 [1])."""
+    assert P.is_cuda and P.dtype == torch.float32 and P.dim() == 2 and P.stride(1) == 1
+    rows, Cn = P.shape
+    sel = torch.empty(max(int(S), 1), dtype=torch.int32, device=P.device)
+    counts = torch.empty(Cn, dtype=torch.int64, device=P.device)
+    thr = torch.zeros(1, dtype=torch.float32, device=P.device)
+    ws = _ws(lib().ocs_act_select_workspace_bytes(Cn), P.device)
+    st = lib().ocs_act_select_channels(_ptr(P), C.c_int64(rows), Cn, C.c_int64(P.stride(0)), int(S), C.c_double(quantile),
+                                       _ptr(sel), _ptr(counts), _ptr(thr), _ptr(ws), C.c_size_t(ws.numel()),
+                                       _ptr(dev_status), _stream())
+    _check(st, "ocs_act_select_channels")
+    return sel[:int(S)], counts, thr
+
+
+def ocs_act_split_quantize_static(A, sel, bits: int, is_signed: bool, alpha_in=None, ld_codes: int | None = None,
+                                  dev_status=None, out=None, ws=None):
+    """A fp32 [rows, C], sel int32 [S] -> (expanded codes [rows, ld_codes], scale fp32 [1], idx_map int32 [C+S]).
+    `out` = (codes, scale, idx_map)."""
+    assert A.is_cuda and A.dtype == torch.float32 and A.dim() == 2 and A.stride(1) == 1
+    rows, Cn = A.shape
+    S = int(sel.numel())
+    if out is not None:
+        codes, scale, idx_map = out
+        ld_codes = codes.stride(0)
+    else:
+        if ld_codes is None:
+            ld_codes = round_up(Cn + S, 16)
+        codes = torch.empty((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=A.device)
+        scale = torch.zeros(1, dtype=torch.float32, device=A.device)
+        idx_map = torch.empty(Cn + S, dtype=torch.int32, device=A.device)
+    nws = lib().ocs_split_quantize_workspace_bytes(rows, Cn, 1, S, 1, 1)
+    if ws is None:
+        ws = _ws(nws, A.device)
+    st = lib().ocs_act_split_quantize_static(_ptr(A), rows, Cn, C.c_int64(A.stride(0)), S, _ptr(sel if S else None),
+                                             int(bits), int(bool(is_signed)), _ptr(alpha_in), _ptr(codes),
+                                             C.c_int64(ld_codes), _ptr(idx_map), _ptr(scale), _ptr(ws),
+                                             C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
+    _check(st, "ocs_act_split_quantize_static")
+    return codes, scale, idx_map

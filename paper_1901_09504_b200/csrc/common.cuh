@@ -71,13 +71,14 @@ ocs_status launch_score_kernel(const unsigned long long* hist, const float* maxp
 
 #ifdef __CUDACC__
 // The search's winner: smallest score, ties to the largest threshold.  Every CTA of the quantize
-// kernel evaluates it (n_candidates doubles) instead of a separate single-thread launch.
+// kernel evaluates it (n_candidates doubles) instead of a separate single-thread launch.  Works for
+// any one-dimensional block of up to 1024 threads; every thread of the block must call it.
 __device__ inline float pick_alpha(const double* __restrict__ scores, float m, int n_candidates) {
-  __shared__ double s_best[8];
-  __shared__ int c_best[8];
+  __shared__ double s_best[32];
+  __shared__ int c_best[32];
   double bs = INFINITY;
   int bc = 0;
-  for (int c = threadIdx.x + 1; c <= n_candidates; c += 256) {
+  for (int c = threadIdx.x + 1; c <= n_candidates; c += blockDim.x) {
     const double v = scores[c - 1];
     if (v < bs || (v == bs && c > bc)) { bs = v; bc = c; }
   }
@@ -88,8 +89,9 @@ __device__ inline float pick_alpha(const double* __restrict__ scores, float m, i
   }
   if ((threadIdx.x & 31) == 0) { s_best[threadIdx.x >> 5] = bs; c_best[threadIdx.x >> 5] = bc; }
   __syncthreads();
+  const int n_warps = (blockDim.x + 31) >> 5;
   bs = s_best[0]; bc = c_best[0];
-  for (int w = 1; w < 8; ++w) {
+  for (int w = 1; w < n_warps; ++w) {
     const double v = s_best[w];
     const int c = c_best[w];
     if (c != 0 && (bc == 0 || v < bs || (v == bs && c > bc))) { bs = v; bc = c; }

@@ -1103,6 +1103,56 @@ FusedWs carve_fused_ws(void* ws, int C, int R, int S, int n_bins, int n_candidat
 }  // namespace
 }  // namespace ocs
 
+namespace ocs {
+namespace {
+// Rows-per-buffer, row-group count and shared-memory bytes of the row-staged kernels.
+struct RowsGeometry {
+  long long g;
+  int n_groups;
+  size_t rows_smem;
+};
+RowsGeometry rows_geometry(int O, size_t row_bytes, size_t hist_bytes) {
+  RowsGeometry q{};
+  q.g = (long long)((kRowSmemBytes - hist_bytes) / 2 / row_bytes);
+  q.g = min(q.g, (long long)max(1, O / kNumSMs));
+  q.g = min(q.g, 64ll);
+  q.n_groups = (int)((O + q.g - 1) / q.g);
+  q.rows_smem = 2 * (size_t)q.g * row_bytes;
+  return q;
+}
+
+ocs_status rows_attr_once() {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(split_rows_kernel<ROWS_HIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kRowSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(split_rows_kernel<ROWS_QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kRowSmemBytes) != cudaSuccess)
+      return OCS_ERR_CUDA;
+    attr_set = true;
+  }
+  return OCS_OK;
+}
+
+// The code pass: rows staged in shared memory, split there, quantized and written as packed codes.
+ocs_status launch_rows_quant(const float* W, int O, int C, int R, int64_t ld_in, int S, const int32_t* idx_map,
+                             const SplitWs& w, RowsEpilogue ep, int8_t* codes, int64_t ld_codes, float* scale,
+                             float* alpha, int g, int srow, int n_groups, size_t rows_smem, int* dev_status,
+                             cudaStream_t stream) {
+  ep.codes = codes;
+  ep.ld_codes = ld_codes;
+  ep.packed_ok = aligned(codes, 4) && (ld_codes % 4 == 0);
+  ep.scale_out = scale;
+  ep.alpha_out = alpha;
+  LaunchScope ls("split_quantize_kernel", stream);
+  split_rows_kernel<ROWS_QUANT><<<min(n_groups, kNumSMs), kRowThreads, rows_smem, stream>>>(
+      W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, g, srow, ep,
+      dev_status);
+  return launch_status();
+}
+}  // namespace
+}  // namespace ocs
+
 extern "C" size_t ocs_split_quantize_workspace_bytes(int O, int C, int R, int S, int n_bins, int n_candidates) {
   (void)O;
   if (C <= 0 || R <= 0 || S < 0) return 0;
@@ -1144,20 +1194,11 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
       OCS_OK)
     return st;
 
-  long long g = (long long)((kRowSmemBytes - hist_bytes) / 2 / row_bytes);
-  g = min(g, (long long)max(1, O / kNumSMs));
-  g = min(g, 64ll);
-  const int n_groups = (int)((O + g - 1) / g);
-  const size_t rows_smem = 2 * (size_t)g * row_bytes;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(split_rows_kernel<ROWS_HIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kRowSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(split_rows_kernel<ROWS_QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kRowSmemBytes) != cudaSuccess)
-      return OCS_ERR_CUDA;
-    attr_set = true;
-  }
+  const RowsGeometry geo = rows_geometry(O, row_bytes, hist_bytes);
+  const long long g = geo.g;
+  const int n_groups = geo.n_groups;
+  const size_t rows_smem = geo.rows_smem;
+  if ((st = rows_attr_once()) != OCS_OK) return st;
   const int L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
   RowsEpilogue ep{};
   ep.maxp = mx3 + 1;   // max|W'| as the plan computed it
@@ -1183,18 +1224,118 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
   }
   ep.scores = scores;
   ep.n_candidates = n_candidates;
-  ep.codes = codes;
-  ep.ld_codes = ld_codes;
-  ep.packed_ok = aligned(codes, 4) && (ld_codes % 4 == 0);
-  ep.scale_out = scale;
-  ep.alpha_out = alpha;
-  {
-    LaunchScope ls("split_quantize_kernel", stream);
-    split_rows_kernel<ROWS_QUANT><<<min(n_groups, kNumSMs), kRowThreads, rows_smem, stream>>>(
-        W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g, srow, ep,
-        dev_status);
+  return launch_rows_quant(W, O, C, R, ld_in, S, idx_map, w, ep, codes, ld_codes, scale, alpha, (int)g, srow, n_groups,
+                           rows_smem, dev_status, stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// ocs_act_split_quantize_static: Eq. 4 for a channel list fixed ahead of time (Section 5.3).  The
+// list is turned into the plan arrays the row-staged kernel reads (every listed channel: one split,
+// both copies halved), then the code pass runs as in ocs_split_quantize.
+namespace ocs {
+namespace {
+constexpr int kStaticPlanThreads = 1024;
+
+__global__ void __launch_bounds__(kStaticPlanThreads)
+static_plan_kernel(const int32_t* __restrict__ sel, int C, int S, const uint32_t* __restrict__ colmin,
+                   const uint32_t* __restrict__ colmax, const float* __restrict__ alpha_in, int32_t* idx_map,
+                   int32_t* depth, unsigned long long* bits, float* qa_step_dev, int32_t* touched, int* n_touched,
+                   float* mx3, int* dev_status) {
+  __shared__ float s_m0[32], s_m1[32];
+  const int tid = threadIdx.x;
+  for (int j = tid; j < C + S; j += kStaticPlanThreads) {
+    idx_map[j] = j < C ? j : 0;
+    depth[j] = j < C ? 0 : 1;
+    bits[j] = 0ull;
   }
-  return launch_status();
+  __syncthreads();
+  bool bad = false;
+  for (int sidx = tid; sidx < S; sidx += kStaticPlanThreads) {
+    int c = sel[sidx];
+    if ((unsigned)c >= (unsigned)C) { bad = true; c = 0; }
+    if (atomicAdd(&depth[c], 1) != 0) bad = true;   // listed twice
+    touched[sidx] = c;
+    idx_map[C + sidx] = c;
+  }
+  if (bad) flag(dev_status, OCS_DEV_BAD_INDEX);
+  __syncthreads();
+  float m0 = 0.0f, m1 = 0.0f;
+  if (colmax) {
+    for (int c = tid; c < C; c += kStaticPlanThreads) {
+      const uint32_t lo = colmin[c], hi = colmax[c];
+      if (lo > hi) continue;                          // no finite sample seen in this column
+      const float m = fmaxf(fabsf(ord_decode(lo)), fabsf(ord_decode(hi)));
+      m0 = fmaxf(m0, m);
+      m1 = fmaxf(m1, depth[c] > 0 ? __fmul_rn(m, 0.5f) : m);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+      m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, o));
+    }
+    if ((tid & 31) == 0) { s_m0[tid >> 5] = m0; s_m1[tid >> 5] = m1; }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    if (colmax) {
+      for (int w = 1; w < kStaticPlanThreads / 32; ++w) { m0 = fmaxf(m0, s_m0[w]); m1 = fmaxf(m1, s_m1[w]); }
+    } else {
+      m1 = *alpha_in;
+      if (!(m1 >= 0.0f) || !is_finite(m1)) { flag(dev_status, OCS_DEV_NONFINITE); m1 = 0.0f; }
+    }
+    mx3[0] = m0; mx3[1] = m1; mx3[2] = 0.0f;
+    *qa_step_dev = 0.0f;
+    *n_touched = S;
+  }
+}
+}  // namespace
+}  // namespace ocs
+
+extern "C" ocs_status ocs_act_split_quantize_static(const float* A, int rows, int C, int64_t ld_in, int S,
+                                                    const int32_t* sel, int bits, int is_signed, const float* alpha_in,
+                                                    int8_t* codes, int64_t ld_codes, int32_t* idx_map, float* scale,
+                                                    void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!A || !codes || !idx_map || !scale || S < 0 || (S > 0 && !sel)) return OCS_ERR_INVALID_ARG;
+  if (bits < 2 || bits > 8) return OCS_ERR_INVALID_ARG;
+  if (rows <= 0 || C <= 0 || S > C) return OCS_ERR_SHAPE;
+  const int ncols_out = C + S;
+  if (ld_in < C || ld_codes < ncols_out) return OCS_ERR_SHAPE;
+  const int srow = (ncols_out + 3) & ~3;
+  const size_t row_bytes = 4 * (size_t)srow;
+  if (!(ld_in % 4 == 0 && aligned(A, 16) && C % 4 == 0 && 2 * row_bytes <= kRowSmemBytes)) return OCS_ERR_UNSUPPORTED;
+  const FusedWs f = carve_fused_ws(ws, C, 1, S, 1, 1);
+  if (!ws || !aligned(ws, 256) || ws_bytes < f.total) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  const SplitWs& w = f.sp;
+  if (!alpha_in) {
+    // dynamic grid: channel extrema of this batch (the kernel also flags non-finite input)
+    if (cudaMemsetAsync(w.colmin, 0xFF, 4 * (size_t)C, stream) != cudaSuccess) return OCS_ERR_CUDA;
+    if (cudaMemsetAsync(w.colmax, 0x00, 4 * (size_t)C, stream) != cudaSuccess) return OCS_ERR_CUDA;
+    const long long units = (long long)((C + 1023) / 1024) * rows;
+    LaunchScope ls("col_minmax_kernel", stream);
+    col_minmax_kernel<true><<<wave_grid(col_minmax_kernel<true>, units), 256, 0, stream>>>(
+        A, rows, C, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
+    if ((st = launch_status()) != OCS_OK) return st;
+  }
+  {
+    LaunchScope ls("static_plan_kernel", stream);
+    static_plan_kernel<<<1, kStaticPlanThreads, 0, stream>>>(sel, C, S, alpha_in ? nullptr : w.colmin,
+                                                             alpha_in ? nullptr : w.colmax, alpha_in, idx_map, w.depth,
+                                                             w.bits, w.qa_step_dev, w.touched, w.n_touched, f.mx3,
+                                                             dev_status);
+    if ((st = launch_status()) != OCS_OK) return st;
+  }
+  const RowsGeometry geo = rows_geometry(rows, row_bytes, 0);
+  if ((st = rows_attr_once()) != OCS_OK) return st;
+  RowsEpilogue ep{};
+  ep.maxp = f.mx3 + 1;
+  ep.L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
+  ep.is_signed = is_signed ? 1 : 0;
+  ep.scores = nullptr;
+  ep.n_candidates = 1;
+  return launch_rows_quant(A, rows, C, 1, ld_in, S, idx_map, w, ep, codes, ld_codes, scale, nullptr, (int)geo.g, srow,
+                           geo.n_groups, geo.rows_smem, dev_status, stream);
 }
 
 // ------------------------------------------------------------------------------------------------

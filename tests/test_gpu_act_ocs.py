@@ -122,3 +122,93 @@ def test_act_ocs_conv_layer(Nb, H, Cn, O, k, stride, pad, S):
     assert ocs.ocs_poll_status(st) == 0
     np.testing.assert_array_equal(host(idx), idx_o)
     np.testing.assert_allclose(host(Y), Y_o, rtol=1e-5, atol=1e-5 * np.abs(Y_o).max())
+
+
+# ------------------------------------------------------------------------------ static variant (Section 5.3)
+@pytest.mark.parametrize("rows,Cn,S,q,seed", [(64, 512, 11, 0.99, 0), (3000, 260, 6, 0.99, 1), (1, 8, 8, 0.5, 2),
+                                               (40000, 64, 2, 0.999, 3), (17, 1030, 0, 0.9, 4), (500, 96, 5, 1.0, 5)])
+def test_static_channel_choice_matches_checker(rows, Cn, S, q, seed):
+    P = prng.laplace(70 + seed, 0, (rows, Cn), 1.0)
+    P[:, Cn // 3] *= 2.5                                    # heavier tails in two channels
+    P[:, Cn - 1] *= 2.0
+    P[rows // 2, 0] = 0.0
+    P[0, Cn // 2] = -0.0
+    sel_o, counts_o, thr_o = orc.act_select(P, S, q)
+    st = ocs.new_status()
+    sel, counts, thr = ocs.ocs_act_select_channels(dev(P), S, q, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    assert host(thr)[0] == np.float32(thr_o)
+    np.testing.assert_array_equal(host(counts), counts_o)
+    np.testing.assert_array_equal(host(sel), sel_o)
+
+
+def test_static_channel_choice_with_padded_rows_and_ties():
+    base = np.zeros((32, 24), np.float32)                   # everything ties: the first S channels win
+    Pd = torch.full((32, 40), 7.0, dtype=torch.float32, device="cuda")
+    Pd[:, :24] = dev(base)
+    sel, counts, thr = ocs.ocs_act_select_channels(Pd[:, :24], 5, 0.99)
+    assert host(sel).tolist() == [0, 1, 2, 3, 4] and host(thr)[0] == 0.0 and not host(counts).any()
+    st = ocs.new_status()
+    bad = dev(np.array([[1.0, np.inf, 2.0, 3.0]], np.float32))
+    ocs.ocs_act_select_channels(bad, 1, 0.5, dev_status=st)
+    assert ocs.ocs_poll_status(st) & 1
+
+
+def _check_static_codes(A, sel, bits, signed, alpha=None):
+    Ap, idx_o = orc.act_split_static(A, sel)
+    a = float(np.float32(alpha)) if alpha is not None else orc.maxabs(Ap)
+    o_codes, o_scale = orc.quantize(Ap, bits, signed, a)
+    st = ocs.new_status()
+    alpha_d = None if alpha is None else dev(np.array([alpha], np.float32))
+    codes, scale, idx = ocs.ocs_act_split_quantize_static(dev(A), dev(np.asarray(sel, np.int32)), bits, signed,
+                                                          alpha_in=alpha_d, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    np.testing.assert_array_equal(host(idx), idx_o)
+    assert float(host(scale)[0]) == np.float32(o_scale)
+    np.testing.assert_array_equal(host(codes)[:, :Ap.shape[1]], o_codes)
+
+
+def test_static_activation_codes_match_checker():
+    A = np.abs(prng.laplace(81, 0, (300, 260), 1.0))
+    A[5, 100] = 33.0
+    _check_static_codes(A, [100, 7, 259, 0], 6, False)               # dynamic grid
+    _check_static_codes(A, [100, 7, 259, 0], 6, False, alpha=9.5)    # profiled threshold: the outlier's halves saturate
+    _check_static_codes(A, [], 8, False)
+    As = prng.laplace(82, 0, (70, 512), 1.0)
+    _check_static_codes(As, list(range(0, 512, 37)), 5, True)
+    _check_static_codes(As[:1], [3], 8, True, alpha=2.0)
+    _check_static_codes(np.zeros((8, 16), np.float32), [1, 2], 6, False)
+    _check_static_codes(As[:, :8], list(range(8)), 4, True)          # every channel split
+    # a channel listed twice or out of range is flagged
+    for bad in ([3, 3], [600]):
+        st = ocs.new_status()
+        ocs.ocs_act_split_quantize_static(dev(As), dev(np.array(bad, np.int32)), 6, True, dev_status=st)
+        assert ocs.ocs_poll_status(st) & 2
+    with pytest.raises(ocs.OcsError):
+        ocs.ocs_act_split_quantize_static(dev(As[:, :4]), dev(np.arange(5, dtype=np.int32) % 4), 6, True)   # S > C
+
+
+def test_static_act_ocs_layer_end_to_end():
+    """Profile on one batch, split another: selection -> expanded codes -> duplicated weights -> layer."""
+    Cn, N, S = 256, 96, 6
+    P = np.abs(prng.laplace(91, 0, (4096, Cn), 1.0))
+    P[:, 40] *= 3.0
+    A = np.abs(prng.laplace(92, 0, (128, Cn), 1.0))
+    A[:, 40] *= 3.0
+    Wc, ws = _weights(N, Cn, 1, 17)
+    sel_o, _, _ = orc.act_select(P, S, 0.99)
+    Ap, idx_o = orc.act_split_static(A, sel_o)
+    ac, a_scale = orc.quantize(Ap, 6, False, orc.maxabs(Ap))
+    Y_o, acc_o = orc.qlinear(ac, False, a_scale, orc.dup_weight_columns(Wc, idx_o), ws,
+                             np.arange(Cn + S, dtype=np.int32))
+    sel, _, _ = ocs.ocs_act_select_channels(dev(P), S, 0.99)
+    ld = ocs.round_up(Cn + S, 16)
+    codes, scale, idx = ocs.ocs_act_split_quantize_static(dev(A), sel, 6, False, ld_codes=ld)
+    Wd = torch.zeros((N, ld), dtype=torch.int8, device="cuda")
+    Wd[:, :Cn] = dev(Wc)
+    ocs.ocs_dup_weight_columns(Wd, Cn, S, idx)
+    ident = torch.arange(Cn + S, dtype=torch.int32, device="cuda")
+    Y, acc = ocs.ocs_qlinear(codes, scale, Wd, dev(np.array([ws], np.float32)), ident, Cn + S, 0, want_acc=True)
+    assert 40 in host(sel).tolist()
+    np.testing.assert_array_equal(host(acc), acc_o)
+    np.testing.assert_allclose(host(Y), Y_o, rtol=1e-5, atol=1e-5 * np.abs(Y_o).max())
