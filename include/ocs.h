@@ -47,6 +47,7 @@ typedef enum {
 #define OCS_DEV_BAD_INDEX 2 /* an idx_map entry was outside [0, C); it was read as channel 0 */
 #define OCS_DEV_TIMEOUT 4   /* a bounded pipeline wait expired; outputs unspecified */
 #define OCS_DEV_DEPTH 8     /* a channel was re-split more than 63 times under the QA rule */
+#define OCS_DEV_OVERFLOW 16 /* a folded sum of duplicated codes left int8; it was saturated */
 
 typedef enum {
   OCS_CLIP_NONE = 0,     /* alpha = max|T| (Eq. 1) */
@@ -168,6 +169,22 @@ ocs_status ocs_split_quantize(const float* W, int O, int C, int R, int64_t ld_in
  * copied instead). */
 ocs_status ocs_dup_weight_columns(int8_t* W_codes, int N, int C, int R, int S, int64_t ldw, const int32_t* idx_map,
                                   int* dev_status, void* stream);
+
+/* ocs_fold_duplicates ------------------------------------------------------------------------
+ * The copies of a split channel all multiply the same activation (Eq. 3), so their integer codes
+ * can be summed back into the source channel: W_folded[n][i][r] = sum over j with idx_map[j] = i
+ * of W_codes[n][j][r].  ocs_qlinear / ocs_qconv on W_folded with C plain channels (S = 0, no
+ * gather) give the same int32 accumulators as on W_codes with the index map -- while the codes
+ * still carry the finer grid the split bought.  W_codes (device) int8 [N][ldw >= (C+S)*R] in
+ * ocs_split's [channel][tap] order; W_folded (device) int8 [N][ld_out >= C*R], may not alias
+ * W_codes.  Two copies of k <= 7 bit codes always fit; a sum that leaves [-128, 127] (re-split
+ * channels, 8-bit codes) is saturated and sets OCS_DEV_OVERFLOW -- the caller then keeps the
+ * gathered form.  Workspace (device, 256-byte aligned): ocs_fold_workspace_bytes(C, S).
+ * The paper has no counterpart: it duplicates activation channels at run time (Section 3.5). */
+size_t ocs_fold_workspace_bytes(int C, int S);
+ocs_status ocs_fold_duplicates(const int8_t* W_codes, int N, int C, int R, int S, int64_t ldw, const int32_t* idx_map,
+                               int8_t* W_folded, int64_t ld_out, void* ws, size_t ws_bytes, int* dev_status,
+                               void* stream);
 
 /* ocs_act_select_channels --------------------------------------------------------------------
  * Static channel choice for activation OCS (Section 5.3: count, per channel, the sampled values

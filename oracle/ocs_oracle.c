@@ -339,6 +339,26 @@ int ocs_oracle_qconv(const void* X, int a_signed, float a_scale, int Nb, int H, 
   return err;
 }
 
+/* ------------------------------------------------------------------ folding duplicated codes */
+int64_t ocs_oracle_fold_duplicates(const int8_t* Wc, int N, int C, int R, int S,
+                                   const int32_t* idx_map, int8_t* Wf) {
+  if (!Wc || !Wf || !idx_map || N <= 0 || C <= 0 || R <= 0 || S < 0) return -1;
+  for (int j = 0; j < C + S; ++j)
+    if (idx_map[j] < 0 || idx_map[j] >= C) return -1;
+  int64_t overflow = 0;
+  for (int n = 0; n < N; ++n)
+    for (int i = 0; i < C; ++i)
+      for (int r = 0; r < R; ++r) {
+        int sum = 0;
+        for (int j = 0; j < C + S; ++j)
+          if (idx_map[j] == i) sum += Wc[((size_t)n * (C + S) + j) * R + r];
+        if (sum > 127) { sum = 127; ++overflow; }
+        if (sum < -128) { sum = -128; ++overflow; }
+        Wf[((size_t)n * C + i) * R + r] = (int8_t)sum;
+      }
+  return overflow;
+}
+
 /* ------------------------------------------------------------------ Section 5.3: static activation OCS */
 static int cmp_float_asc(const void* a, const void* b) {
   const float x = *(const float*)a, y = *(const float*)b;

@@ -13,7 +13,7 @@
  * unsigned codes.  All functions return 0 on success, non-zero on a bad argument.
  *
  * Pinned by tests (paper facts, closed forms, brute force): split, quantize, clip_mse,
- * qlinear, qconv, pools, relu/add, act_select, act_split_static.  Parity unpinned (conventions the paper does not fix,
+ * qlinear, qconv, fold_duplicates, pools, relu/add, act_select, act_split_static.  Parity unpinned (conventions the paper does not fix,
  * enforced only checker-vs-GPU): the QA grid-step policy, the unsigned activation grid,
  * the bin count and the tie rule of the clip search, the LSTM cell's sigmoid/tanh routines,
  * the quantile convention of act_select (nearest rank on |a|; the paper says only "99th
@@ -92,6 +92,14 @@ int ocs_oracle_qlinear_samples(const void* A, int a_signed, float a_scale, int M
 int ocs_oracle_qconv(const void* X, int a_signed, float a_scale, int Nb, int H, int Wd, int C,
                      const int8_t* Wc, float w_scale, int O, int S, int kh, int kw, int stride,
                      int pad, const int32_t* idx_map, const float* bias, float* Y, int32_t* acc);
+
+/* Folding the duplicates back (Eq. 3 read right to left on the integer codes): the copies of a
+ * split channel all multiply the same activation, so Wf[n][i][r] = sum over j with
+ * idx_map[j] = i of Wc[n][j][r] gives the same accumulators without any gather.
+ * Wc dense [N][C+S][R] int8 -> Wf dense [N][C][R] int8.  Returns the number of sums that left
+ * [-128, 127] (those entries are saturated), or -1 on a bad argument. */
+int64_t ocs_oracle_fold_duplicates(const int8_t* Wc, int N, int C, int R, int S,
+                                   const int32_t* idx_map, int8_t* Wf);
 
 /* Section 5.3, static activation OCS: which channels to split is decided once, on sampled
  * activations P [rows][C].  t = the `quantile` (the paper uses 0.99) quantile of all |a| by

@@ -162,6 +162,20 @@ def act_ocs_linear(A, S: int, a_bits: int, a_signed: bool, Wc, w_scale, bias=Non
     return Y, acc, ac, a_scale, idx
 
 
+def fold_duplicates(Wc, idx_map, Cn: int):
+    """Wc int8 [N, C+S] or [N, C+S, kh, kw] -> (Wf int8 [N, C, ...], number of saturated sums)."""
+    Wc = np.ascontiguousarray(Wc, dtype=np.int8)
+    idx_map = np.ascontiguousarray(idx_map, dtype=np.int32)
+    N, K = Wc.shape[0], Wc.shape[1]
+    R = int(np.prod(Wc.shape[2:])) if Wc.ndim > 2 else 1
+    out = np.empty((N, Cn) + tuple(Wc.shape[2:]), dtype=np.int8)
+    lib().ocs_oracle_fold_duplicates.restype = C.c_int64
+    rc = lib().ocs_oracle_fold_duplicates(_p(Wc, _i8p), N, int(Cn), R, K - int(Cn), _p(idx_map, _i32p), _p(out, _i8p))
+    if rc < 0:
+        raise RuntimeError("fold_duplicates: bad argument")
+    return out, int(rc)
+
+
 def act_select(P, S: int, quantile: float = 0.99):
     """Static channel choice of Section 5.3 on sampled activations P [rows, C]
     -> (sel int32 [S], counts int64 [C], threshold)."""

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libocs_b200.so")
 OCS_OK = 0
 STATUS_NAMES = {0: "OCS_OK", 1: "OCS_ERR_INVALID_ARG", 2: "OCS_ERR_SHAPE", 3: "OCS_ERR_WORKSPACE",
                 4: "OCS_ERR_UNSUPPORTED", 5: "OCS_ERR_CUDA"}
-DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT, DEV_DEPTH = 1, 2, 4, 8
+DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT, DEV_DEPTH, DEV_OVERFLOW = 1, 2, 4, 8, 16
 CLIP_NONE, CLIP_MSE, CLIP_MSE_EXACT = 0, 1, 2
 
 EXPORTS = [
@@ -27,6 +27,7 @@ EXPORTS = [
     "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
     "ocs_split_workspace_bytes", "ocs_split",
     "ocs_split_quantize_workspace_bytes", "ocs_split_quantize", "ocs_dup_weight_columns",
+    "ocs_fold_workspace_bytes", "ocs_fold_duplicates",
     "ocs_act_select_workspace_bytes", "ocs_act_select_channels", "ocs_act_split_quantize_static",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear",
@@ -52,7 +53,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.ocs_num_splits.argtypes = [C.c_int, C.c_double]
         L.ocs_version.restype = C.c_char_p
-        for name in ("ocs_act_select_workspace_bytes", "ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
+        for name in ("ocs_fold_workspace_bytes", "ocs_act_select_workspace_bytes", "ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
                      "ocs_qconv_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.ocs_quantize_workspace_views.restype = None
@@ -426,3 +427,18 @@ def ocs_act_split_quantize_static(A, sel, bits: int, is_signed: bool, alpha_in=N
                                              C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
     _check(st, "ocs_act_split_quantize_static")
     return codes, scale, idx_map
+
+
+def ocs_fold_duplicates(W_codes, C_in: int, S: int, idx_map, R: int = 1, ld_out: int | None = None, dev_status=None):
+    """W_codes int8 [N, ldw >= (C+S)*R] -> folded int8 [N, ld_out >= C*R] (copies summed into their sources)."""
+    assert W_codes.is_cuda and W_codes.dtype == torch.int8 and W_codes.dim() == 2 and W_codes.stride(1) == 1
+    N = W_codes.shape[0]
+    if ld_out is None:
+        ld_out = round_up(int(C_in) * int(R), 16)
+    out = torch.zeros((N, ld_out), dtype=torch.int8, device=W_codes.device)
+    ws = _ws(lib().ocs_fold_workspace_bytes(int(C_in), int(S)), W_codes.device)
+    st = lib().ocs_fold_duplicates(_ptr(W_codes), N, int(C_in), int(R), int(S), C.c_int64(W_codes.stride(0)), _ptr(idx_map),
+                                   _ptr(out), C.c_int64(ld_out), _ptr(ws), C.c_size_t(ws.numel()), _ptr(dev_status),
+                                   _stream())
+    _check(st, "ocs_fold_duplicates")
+    return out

@@ -37,6 +37,9 @@ constexpr int UMMA_K = 32;     // K of one tcgen05.mma.kind::i8
 constexpr int kGemmThreads = 320;    // TMA warp, MMA warp, 4 gather warps, 4 epilogue warps
 constexpr int kGatherThreads = 128;
 constexpr long long kWaitCycles = 2000000000ll;  // about one second
+// A waiting thread sleeps inside mbarrier.try_wait until the phase completes or about this many nanoseconds
+// pass, instead of spinning on the issue slots the epilogue warps of the same SM partition need.
+constexpr uint32_t kSuspendHintNs = 2000u;
 
 enum { MODE_LINEAR = 0, MODE_CONV = 1 };
 
@@ -89,10 +92,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }
@@ -112,10 +115,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
       : "memory");
   return ok != 0;
 }
@@ -211,6 +214,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t v[32]) {
       : "r"(taddr)
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// (float)acc with round-to-nearest-even, without the conversion unit (which is slow on this part and sits
+// on the epilogue's critical path): u = acc + 2^31 is split into two 16-bit halves, each placed by one byte
+// permute into the mantissa of 1.5 * 2^23, where it is exact; subtracting the offsets gives hi = floor(acc /
+// 65536) and lo exactly, and one fused multiply-add rounds the exact sum hi * 65536 + lo once -- the same
+// result as cvt.rn.f32.s32 for every int32.
+__device__ __forceinline__ float int_to_float_rn(int acc) {
+  const uint32_t u = (uint32_t)acc ^ 0x80000000u;
+  const float fh = __fsub_rn(__uint_as_float(__byte_perm(u, 0x4B400000u, 0x7632)), 12615680.0f);   // 1.5*2^23 + 2^15
+  const float fl = __fsub_rn(__uint_as_float(__byte_perm(u, 0x4B400000u, 0x7610)), 12582912.0f);
+  return fmaf(fh, 65536.0f, fl);
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of
@@ -341,7 +356,7 @@ struct SmemLayout {
   static constexpr int kStageBytes = kABytes + kBBytes;
   // ring depth: shallower when the tail buffers are needed
   static constexpr int kStagesNoTail = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int kStagesTail = (BN == 256) ? 3 : (BN == 128 ? 5 : 6);
+  static constexpr int kStagesTail = (BN == 256) ? 3 : (BN == 128 ? 4 : 6);
   static constexpr int kMaxStages = kStagesNoTail;
   static constexpr int kTileBytes =
       (kStagesNoTail * kStageBytes > kStagesTail * kStageBytes + kTailBufs * kABytes)
@@ -349,8 +364,14 @@ struct SmemLayout {
   static constexpr int kCtrlBytes = 1024;               // barriers, tensor-memory slot, flags
   static constexpr int kRowTableBytes = 2 * BM * 24;    // RowInfo per tile row, two tiles
   static constexpr int kSrcTableBytes = 2 * BK * 8;     // KSrc per contraction index, two gathered K-blocks
+  // epilogue staging: per epilogue warp a 32 x 32 tile of 32-bit words, rows padded to 36 words (16-byte
+  // aligned, conflict-free for 128-bit accesses by quarter warps), and the 32 output-row numbers
+  static constexpr int kEpiRowWords = 36;
+  static constexpr int kEpiWarpBytes = 32 * kEpiRowWords * 4 + 32 * 8;
+  static constexpr int kEpiBytes = 4 * kEpiWarpBytes;
   static constexpr int kDynBytes =
-      kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes + kSrcTableBytes;
+      kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes + kSrcTableBytes + kEpiBytes;
+  static_assert(kDynBytes <= 227 * 1024, "more dynamic shared memory than a CTA can have");
 };
 
 // One work item of a CTA: an output tile and a K slice.
@@ -391,6 +412,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * kNumBars + 8);
   RowInfo* rows = reinterpret_cast<RowInfo*>(ctrl + L::kCtrlBytes);
   KSrc* ksrc = reinterpret_cast<KSrc*>(ctrl + L::kCtrlBytes + L::kRowTableBytes);
+  unsigned char* epi_stage = ctrl + L::kCtrlBytes + L::kRowTableBytes + L::kSrcTableBytes;
   auto full_bar = [&](int s) { return smem_u32(bars + s); };
   auto empty_bar = [&](int s) { return smem_u32(bars + L::kMaxStages + s); };
   auto gfull_bar = [&](int g) { return smem_u32(bars + 2 * L::kMaxStages + g); };
@@ -600,48 +622,88 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       tc_fence_after();
       const RowInfo ri = row_info(p, w.mt, q * 32 + lane);
       const int nt = w.nt, kz = w.kz;
+      // Each lane holds one row of the 32 x 32 chunk; written out that way a store instruction would touch
+      // 32 rows with 16 bytes each.  The chunk goes through shared memory instead, so that every quarter
+      // warp writes one row's 128 contiguous bytes (lane -> row i*4 + lane/8, words (lane%8)*4 .. +3).
+      uint32_t* st_words = reinterpret_cast<uint32_t*>(epi_stage + (size_t)q * L::kEpiWarpBytes);
+      long long* st_rows = reinterpret_cast<long long*>(st_words + 32 * L::kEpiRowWords);
+      __syncwarp();
+      st_rows[lane] = ri.out_row;
+      __syncwarp();
+      const int sub = lane >> 3, cq = (lane & 7) * 4;
+      // destination of the chunk's words: Y (and acc_out), or this slice's partial sums [kz][row][n]
+      uint32_t* dst0 = direct ? reinterpret_cast<uint32_t*>(p.Y) : reinterpret_cast<uint32_t*>(p.acc_ws) + (long long)kz * p.out_rows * p.N;
+      const long long ldd = direct ? p.ldy : (long long)p.N;
+      const bool base_vec = ((reinterpret_cast<uintptr_t>(dst0) & 15) == 0) && (ldd % 4 == 0);
+      const bool acc_vec = p.acc_out && ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) && (p.ldy % 4 == 0);
       for (int c0 = 0; c0 < BN; c0 += 32) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
         uint32_t v[32];
         __syncwarp();
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
-        if (ri.out_row >= 0) {
-          if (direct) {
-            float* y = p.Y + ri.out_row * p.ldy + n0;
-            int32_t* ao = p.acc_out ? p.acc_out + ri.out_row * p.ldy + n0 : nullptr;
-            const bool vec = (n0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(y) & 15) == 0);
-            if (vec) {
+        const bool full = n0 + 32 <= p.N;   // warp-uniform
+        // raw accumulators -> shared memory, one row per lane
+        uint32_t* mine = st_words + lane * L::kEpiRowWords;
 #pragma unroll
-              for (int jj = 0; jj < 32; jj += 4) {
-                float4 o;
-                o.x = fmaf((float)(int)v[jj + 0], sc, p.bias ? __ldg(p.bias + n0 + jj + 0) : 0.0f);
-                o.y = fmaf((float)(int)v[jj + 1], sc, p.bias ? __ldg(p.bias + n0 + jj + 1) : 0.0f);
-                o.z = fmaf((float)(int)v[jj + 2], sc, p.bias ? __ldg(p.bias + n0 + jj + 2) : 0.0f);
-                o.w = fmaf((float)(int)v[jj + 3], sc, p.bias ? __ldg(p.bias + n0 + jj + 3) : 0.0f);
-                *reinterpret_cast<float4*>(y + jj) = o;
-              }
+        for (int jj = 0; jj < 32; jj += 4)
+          *reinterpret_cast<uint4*>(mine + jj) = make_uint4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
+        __syncwarp();
+        // this lane's four columns of every row it writes: their bias once per chunk
+        float b4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (direct && p.bias) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (n0 + cq + e < p.N) b4[e] = __ldg(p.bias + n0 + cq + e);
+        }
+        const bool vec0 = full && base_vec, vec1 = full && acc_vec;
+        long long orow[8];
+        uint4 a[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int r = i * 4 + sub;
+          orow[i] = st_rows[r];
+          a[i] = *reinterpret_cast<const uint4*>(st_words + r * L::kEpiRowWords + cq);
+        }
+        if (direct) {
+          uint4 o[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            o[i].x = __float_as_uint(fmaf(int_to_float_rn((int)a[i].x), sc, b4[0]));
+            o[i].y = __float_as_uint(fmaf(int_to_float_rn((int)a[i].y), sc, b4[1]));
+            o[i].z = __float_as_uint(fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]));
+            o[i].w = __float_as_uint(fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]));
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (orow[i] < 0) continue;
+            uint32_t* d = dst0 + orow[i] * ldd + n0 + cq;
+            if (vec0) {
+              *reinterpret_cast<uint4*>(d) = o[i];
             } else {
-#pragma unroll
-              for (int jj = 0; jj < 32; ++jj)
-                if (n0 + jj < p.N) y[jj] = fmaf((float)(int)v[jj], sc, p.bias ? __ldg(p.bias + n0 + jj) : 0.0f);
+              if (n0 + cq + 0 < p.N) d[0] = o[i].x;
+              if (n0 + cq + 1 < p.N) d[1] = o[i].y;
+              if (n0 + cq + 2 < p.N) d[2] = o[i].z;
+              if (n0 + cq + 3 < p.N) d[3] = o[i].w;
             }
-            if (ao) {
+          }
+        }
+        if (!direct || p.acc_out) {
+          // raw sums: this K slice's partials, or the caller's copy of the accumulators
+          uint32_t* rbase = direct ? reinterpret_cast<uint32_t*>(p.acc_out) : dst0;
+          const long long rld = direct ? p.ldy : ldd;
+          const bool rvec = direct ? vec1 : vec0;
 #pragma unroll
-              for (int jj = 0; jj < 32; ++jj)
-                if (n0 + jj < p.N) ao[jj] = (int)v[jj];
-            }
-          } else {
-            // this slice's partial sums, [kz][row][n]
-            int32_t* part = p.acc_ws + ((long long)kz * p.out_rows + ri.out_row) * p.N + n0;
-            if ((n0 + 32 <= p.N) && ((reinterpret_cast<uintptr_t>(part) & 15) == 0)) {
-#pragma unroll
-              for (int jj = 0; jj < 32; jj += 4)
-                __stcg(reinterpret_cast<int4*>(part + jj), make_int4((int)v[jj], (int)v[jj + 1], (int)v[jj + 2], (int)v[jj + 3]));
+          for (int i = 0; i < 8; ++i) {
+            if (orow[i] < 0) continue;
+            uint32_t* d = rbase + orow[i] * rld + n0 + cq;
+            if (rvec) {
+              __stcg(reinterpret_cast<uint4*>(d), a[i]);
             } else {
-#pragma unroll
-              for (int jj = 0; jj < 32; ++jj)
-                if (n0 + jj < p.N) __stcg(part + jj, (int)v[jj]);
+              if (n0 + cq + 0 < p.N) d[0] = a[i].x;
+              if (n0 + cq + 1 < p.N) d[1] = a[i].y;
+              if (n0 + cq + 2 < p.N) d[2] = a[i].z;
+              if (n0 + cq + 3 < p.N) d[3] = a[i].w;
             }
           }
         }

@@ -1377,3 +1377,73 @@ extern "C" ocs_status ocs_dup_weight_columns(int8_t* W_codes, int N, int C, int 
   dup_columns_kernel<<<grid, 256, 0, stream>>>(W_codes, N, C, R, S, ldw, idx_map, dev_status);
   return launch_status();
 }
+
+// ------------------------------------------------------------------------------------------------
+// ocs_fold_duplicates: the copies of a split channel all multiply the same activation, so their
+// integer codes can be summed back into the source channel (Eq. 3 read right to left):
+// Wf[n][i][r] = sum over j with idx_map[j] = i of Wc[n][j][r].  The layer on Wf needs no gather and
+// gives the same int32 accumulators.  Per-source lists of the appended copies are built with one
+// atomic exchange per copy; integer sums do not depend on the list order.
+namespace ocs {
+namespace {
+__global__ void __launch_bounds__(256)
+fold_lists_kernel(const int32_t* __restrict__ idx_map, int C, int S, int32_t* head, int32_t* next, int* dev_status) {
+  const int sidx = blockIdx.x * 256 + threadIdx.x;
+  if (sidx >= S) return;
+  int c = __ldg(idx_map + C + sidx);
+  if ((unsigned)c >= (unsigned)C) { flag(dev_status, OCS_DEV_BAD_INDEX); c = 0; }
+  next[sidx] = atomicExch(&head[c], sidx);
+}
+
+__global__ void __launch_bounds__(256)
+fold_kernel(const int8_t* __restrict__ Wc, int N, int C, int R, long long ldw, const int32_t* __restrict__ head,
+            const int32_t* __restrict__ next, int8_t* __restrict__ Wf, long long ld_out, int* dev_status) {
+  const int cols = C * R;
+  bool over = false;
+  for (int n = blockIdx.y; n < N; n += gridDim.y) {
+    const int8_t* src = Wc + (long long)n * ldw;
+    int8_t* dst = Wf + (long long)n * ld_out;
+    for (int e = blockIdx.x * 256 + threadIdx.x; e < cols; e += gridDim.x * 256) {
+      const int c = e / R, r = e - c * R;
+      int sum = src[e];
+      for (int sidx = __ldg(head + c); sidx >= 0; sidx = __ldg(next + sidx)) sum += src[(long long)(C + sidx) * R + r];
+      if (sum > 127) { sum = 127; over = true; }
+      if (sum < -128) { sum = -128; over = true; }
+      dst[e] = (int8_t)sum;
+    }
+  }
+  if (over) flag(dev_status, OCS_DEV_OVERFLOW);
+}
+}  // namespace
+}  // namespace ocs
+
+extern "C" size_t ocs_fold_workspace_bytes(int C, int S) {
+  if (C <= 0 || S < 0) return 0;
+  return align_up(4 * (size_t)C, 256) + align_up(4 * (size_t)(S > 0 ? S : 1), 256);
+}
+
+extern "C" ocs_status ocs_fold_duplicates(const int8_t* W_codes, int N, int C, int R, int S, int64_t ldw,
+                                          const int32_t* idx_map, int8_t* W_folded, int64_t ld_out, void* ws,
+                                          size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!W_codes || !W_folded || !idx_map || S < 0) return OCS_ERR_INVALID_ARG;
+  if (N <= 0 || C <= 0 || R <= 0) return OCS_ERR_SHAPE;
+  if ((int64_t)C * R >= (1ll << 31) || ldw < ((int64_t)C + S) * R || ld_out < (int64_t)C * R) return OCS_ERR_SHAPE;
+  if (!ws || !aligned(ws, 256) || ws_bytes < ocs_fold_workspace_bytes(C, S)) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  int32_t* head = reinterpret_cast<int32_t*>(ws);
+  int32_t* next = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(ws) + align_up(4 * (size_t)C, 256));
+  if (cudaMemsetAsync(head, 0xFF, 4 * (size_t)C, stream) != cudaSuccess) return OCS_ERR_CUDA;   // -1 = empty list
+  if (S > 0) {
+    LaunchScope ls("fold_lists_kernel", stream);
+    fold_lists_kernel<<<(S + 255) / 256, 256, 0, stream>>>(idx_map, C, S, head, next, dev_status);
+    if ((st = launch_status()) != OCS_OK) return st;
+  }
+  const int cols = C * R;
+  const int gx = min((cols + 255) / 256, 64);
+  const int gy = min(N, max(1, kNumSMs * 8 / gx));
+  LaunchScope ls("fold_kernel", stream);
+  fold_kernel<<<dim3(gx, gy), 256, 0, stream>>>(W_codes, N, C, R, ldw, head, next, W_folded, ld_out, dev_status);
+  return launch_status();
+}

@@ -443,6 +443,38 @@ def test_qlinear_matches_expanded_and_folded_matmul():
     np.testing.assert_array_equal(Ys, Y[ms, ns])
 
 
+def test_folded_codes_give_the_same_accumulators():
+    """Folding against numpy's add.at, and the folded layer against the gathered one (Eq. 3 both ways)."""
+    M, Cn, N, S = 9, 37, 13, 6
+    A = configs.random_codes(3, 0, (M, Cn), 0, 255, np.uint8)
+    Wc = configs.random_codes(3, 1, (N, Cn + S), -60, 60, np.int8)          # two or three copies still fit int8
+    idx = np.concatenate([np.arange(Cn), [5, 5, 0, 36, 17, 5]]).astype(np.int32)
+    Wc[:, [5, Cn, Cn + 1, Cn + 5]] //= 4                                      # channel 5 has four copies
+    Wf, over = orc.fold_duplicates(Wc, idx, Cn)
+    ref = np.zeros((N, Cn), dtype=np.int64)
+    np.add.at(ref, (slice(None), idx), Wc.astype(np.int64))
+    assert over == 0
+    np.testing.assert_array_equal(Wf, ref)
+    _, acc = orc.qlinear(A, False, 1.0, Wc, 1.0, idx)
+    _, acc_f = orc.qlinear(A, False, 1.0, Wf, 1.0, np.arange(Cn, dtype=np.int32))
+    np.testing.assert_array_equal(acc_f, acc)
+    # conv weights: taps fold independently
+    W4 = configs.random_codes(3, 2, (4, 6 + 2, 3, 3), -50, 50, np.int8)
+    idx4 = np.array([0, 1, 2, 3, 4, 5, 2, 4], np.int32)
+    W4f, over = orc.fold_duplicates(W4, idx4, 6)
+    ref4 = W4[:, :6].astype(np.int64).copy()
+    ref4[:, 2] += W4[:, 6]
+    ref4[:, 4] += W4[:, 7]
+    assert over == 0
+    np.testing.assert_array_equal(W4f, ref4)
+    # sums that leave int8 are counted and saturated
+    big = np.full((1, 3), 100, np.int8)
+    f, over = orc.fold_duplicates(big, np.array([0, 1, 0], np.int32), 2)
+    assert over == 1 and f.tolist() == [[127, 100]]
+    f, over = orc.fold_duplicates(-big, np.array([0, 1, 0], np.int32), 2)
+    assert over == 1 and f.tolist() == [[-128, -100]]
+
+
 @pytest.mark.parametrize("k,stride,pad,H", [(3, 1, 1, 7), (3, 2, 1, 8), (1, 2, 0, 6), (7, 2, 3, 11), (1, 1, 0, 5)])
 def test_qconv_matches_library_conv(k, stride, pad, H):
     torch = pytest.importorskip("torch")
