@@ -998,6 +998,48 @@ __global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, i
   }
 }
 
+
+// A convolution whose pixels TMA cannot address (a channel count that is not a multiple of 16 bytes, such
+// as a network's first layer) is run as a plain GEMM over its patch matrix: row m = output pixel
+// (n, oh, ow), column k = packed contraction index ([tap][c < C] then [tap][s < S], the order of the packed
+// weights), out-of-image taps zero.  Building it costs one pass of coalesced 32-bit stores; every byte of
+// the main loop then arrives by TMA instead of by byte gathers.  The duplicated channels are columns of
+// the matrix like any other, read through idx_map here.
+constexpr int kPatchMaxK = 4096;   // source table in shared memory: 8 bytes per contraction index
+
+__global__ void __launch_bounds__(256)
+conv_patches_kernel(GemmParams p, uint8_t* __restrict__ P, long long ldp, long long rows) {
+  extern __shared__ KSrc tab[];
+  bool bad = false;
+  for (int k = threadIdx.x; k < (int)ldp; k += 256) tab[k] = k_source(p, k, &bad);
+  if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
+  __syncthreads();
+  const int tpr = (int)(ldp >> 2);                 // threads per row: 4 contraction indices each
+  const int rows_par = 256 / tpr > 0 ? 256 / tpr : 1;
+  const int lane_row = threadIdx.x / tpr, q = threadIdx.x - lane_row * tpr;
+  if (tpr <= 256 && lane_row >= rows_par) return;
+  const long long HoWo = (long long)p.Ho * p.Wo;
+  for (long long m = (long long)blockIdx.x * rows_par + lane_row; m < rows; m += (long long)gridDim.x * rows_par) {
+    const int n = (int)(m / HoWo);
+    const int rem = (int)(m - (long long)n * HoWo);
+    const int oh = rem / p.Wo, ow = rem - oh * p.Wo;
+    const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
+    const uint8_t* base = p.A + (((long long)n * p.H + ih0) * p.Wd + iw0) * p.C;
+    for (int kq = q; kq < tpr; kq += 256) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const KSrc src = tab[kq * 4 + e];
+        const int ih = ih0 + (src.dydx & 255), iw = iw0 + (src.dydx >> 8);
+        const bool ok = src.off >= 0 && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd;
+        const uint32_t v = (uint32_t)__ldg(ok ? base + src.off : p.A);
+        word |= (ok ? v : 0u) << (8 * e);
+      }
+      *reinterpret_cast<uint32_t*>(P + m * ldp + kq * 4) = word;
+    }
+  }
+}
+
 }  // namespace
 }  // namespace ocs
 
@@ -1033,7 +1075,9 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
   p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = ldy; p.acc_out = acc_out;
   p.dev_status = dev_status;
   const int m_tiles = (M + BM - 1) / BM;
-  p.kb_tma_a = C / BK;  // K-blocks made of original channels only
+  // K-blocks made of original channels only; without duplicates the last, partial block is TMA-fed too (the
+  // tensor map zero-fills past C)
+  p.kb_tma_a = S == 0 ? (C + BK - 1) / BK : C / BK;
   p.a_box_bytes = BM * BK;
   CUtensorMap tmA;
   bool tma_ok = p.a_vec16 && p.kb_tma_a > 0;
@@ -1074,6 +1118,7 @@ struct ConvGeom {
   long long m_tiles, out_rows;
 };
 bool conv_geom(int Nb, int H, int Wd, int kh, int kw, int stride, int pad, ConvGeom* g) {
+
   g->Ho = (H + 2 * pad - kh) / stride + 1;
   g->Wo = (Wd + 2 * pad - kw) / stride + 1;
   if (g->Ho <= 0 || g->Wo <= 0) return false;
@@ -1085,6 +1130,18 @@ bool conv_geom(int Nb, int H, int Wd, int kh, int kw, int stride, int pad, ConvG
   g->out_rows = (long long)Nb * g->Ho * g->Wo;
   return true;
 }
+bool conv_tma_shape_ok(const ConvGeom& g, int C, int stride) {
+  return (conv_tap_stride(C) % BK == 0) && stride <= 8 && g.bw * stride <= 256 && g.bh * stride <= 256;
+}
+// Bytes of the patch matrix for layers TMA cannot address (0 when TMA can, or when the matrix would be
+// unreasonably wide or large: those layers keep the in-kernel gather).
+size_t patch_matrix_bytes(const ConvGeom& g, int C, int S, int kh, int kw, int stride) {
+  if (conv_tma_shape_ok(g, C, stride)) return 0;
+  const long long Kt = (long long)kh * kw * ((long long)C + S);
+  const long long ldp = (Kt + 15) / 16 * 16;
+  if (ldp > kPatchMaxK || g.out_rows * ldp > (8ll << 30)) return 0;
+  return align_up((size_t)(g.out_rows * ldp), 256);
+}
 }  // namespace
 
 extern "C" size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O, int S, int kh, int kw, int stride,
@@ -1093,8 +1150,10 @@ extern "C" size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O,
   if (Nb <= 0 || H <= 0 || Wd <= 0 || C <= 0 || S < 0 || O <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0 ||
       !conv_geom(Nb, H, Wd, kh, kw, stride, pad, &g))
     return 256;
-  const long long Ktot = (long long)kh * kw * ((long long)C + S);
-  return 256 + align_up(splitk_ws_bound(g.out_rows, O, g.m_tiles), 256);
+  size_t bytes = 256 + align_up(splitk_ws_bound(g.out_rows, O, (g.out_rows + BM - 1) / BM), 256) +
+                 align_up(splitk_ws_bound(g.out_rows, O, g.m_tiles), 256);
+  bytes += patch_matrix_bytes(g, C, S, kh, kw, stride);
+  return bytes;
 }
 
 extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H, int Wd, int C,
@@ -1132,7 +1191,37 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   // multiple of the K-block; channels past C read as zero); a strided convolution walks the image
   // with the tensor map's traversal stride
   CUtensorMap tmA;
-  bool tma_ok = (Cp % BK == 0) && aligned(X_codes, 16) && stride <= 8 && g.bw * stride <= 256 && g.bh * stride <= 256;
+  bool tma_ok = conv_tma_shape_ok(g, C, stride) && aligned(X_codes, 16);
+  // layers TMA cannot address: build the patch matrix (if the caller's workspace has room for it) and run
+  // the plain GEMM on it
+  const size_t patch_bytes = patch_matrix_bytes(g, C, S, kh, kw, stride);
+  if (patch_bytes > 0 && ws && aligned(ws, 256)) {
+    const size_t gemm_ws = 256 + align_up(splitk_ws_bound(g.out_rows, O, (g.out_rows + BM - 1) / BM), 256);
+    if (ws_bytes >= gemm_ws + patch_bytes) {
+      const long long ldp = (Ktot + 15) / 16 * 16;
+      uint8_t* P = reinterpret_cast<uint8_t*>(ws) + gemm_ws;
+      {
+        const int tpr = (int)(ldp / 4);
+        const int rows_par = 256 / tpr > 0 ? 256 / tpr : 1;
+        const long long blocks = (g.out_rows + rows_par - 1) / rows_par;
+        const int grid = (int)min(blocks, (long long)kNumSMs * 16);
+        LaunchScope ls("conv_patches_kernel", stream);
+        conv_patches_kernel<<<grid, 256, (size_t)ldp * sizeof(KSrc), stream>>>(p, P, ldp, g.out_rows);
+        if ((st = launch_status()) != OCS_OK) return st;
+      }
+      GemmParams q = p;
+      q.mode = MODE_LINEAR;
+      q.C = (int)Ktot; q.Cp = (int)Ktot; q.S = 0; q.R = 1;
+      q.A = P; q.lda = ldp; q.a_vec16 = 1;
+      q.kb_tma_a = (int)((Ktot + BK - 1) / BK);
+      q.a_box_bytes = BM * BK;
+      const cuuint64_t dims[2] = {(cuuint64_t)Ktot, (cuuint64_t)g.out_rows};
+      const cuuint64_t strides[1] = {(cuuint64_t)ldp};
+      const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+      if (!encode_u8(&tmA, P, 2, dims, strides, box)) return OCS_ERR_CUDA;
+      return run_gemm(q, W_packed, ldw, g.out_rows, (int)((g.out_rows + BM - 1) / BM), true, &tmA, ws, gemm_ws, stream);
+    }
+  }
   p.kb_tma_a = tma_ok ? (kh * kw * Cp) / BK : 0;
   p.a_box_bytes = g.bw * g.bh * g.bn * BK;
   if (tma_ok) {
