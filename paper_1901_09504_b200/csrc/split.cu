@@ -36,6 +36,79 @@ __device__ __forceinline__ void cta_range(long long total, long long* u0, long l
   *u1 = total * ((long long)blockIdx.x + 1) / (long long)gridDim.x;
 }
 
+// K1 for a narrow matrix (ncols <= 512): a row needs only ncols/4 threads, so the CTA walks 256 / (ncols/4)
+// rows side by side and combines them in shared memory before touching the global extrema.
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+col_minmax_narrow_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
+                         uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map,
+                         int32_t* __restrict__ depth, unsigned long long* __restrict__ bits, int* dev_status) {
+  for (int c = blockIdx.x * 256 + threadIdx.x; c < C; c += gridDim.x * 256) {
+    idx_map[c] = c; depth[c] = 0; bits[c] = 0ull;
+  }
+  bool bad = false;
+  {
+    // narrow matrix: a row needs only ncols/4 threads, so the CTA walks 256 / (ncols/4) rows side by side and
+    // combines them in shared memory before touching the global extrema
+    __shared__ uint32_t s_min[512], s_max[512];
+    for (int i = threadIdx.x; i < ncols; i += 256) { s_min[i] = 0xFFFFFFFFu; s_max[i] = 0u; }
+    __syncthreads();
+    const int tpr = (ncols + 3) >> 2;
+    const int side = 256 / tpr;
+    const int lr = threadIdx.x / tpr, col0 = (threadIdx.x - lr * tpr) * 4;
+    long long r0, r1;
+    cta_range((long long)O, &r0, &r1);
+    if (lr < side) {
+      float mn[4], mx[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) { mn[c] = INFINITY; mx[c] = -INFINITY; }
+      if (VEC && col0 + 3 < ncols) {
+        const float4* p = reinterpret_cast<const float4*>(W + (r0 + lr) * ld + col0);
+        const int64_t stride = (ld >> 2) * side;
+#pragma unroll 8
+        for (long long r = r0 + lr; r < r1; r += side) {
+          const float4 v = __ldcs(p);
+          p += stride;
+          mn[0] = fminf(mn[0], v.x); mx[0] = fmaxf(mx[0], v.x);
+          mn[1] = fminf(mn[1], v.y); mx[1] = fmaxf(mx[1], v.y);
+          mn[2] = fminf(mn[2], v.z); mx[2] = fmaxf(mx[2], v.z);
+          mn[3] = fminf(mn[3], v.w); mx[3] = fmaxf(mx[3], v.w);
+          bad |= !(is_finite(v.x) && is_finite(v.y) && is_finite(v.z) && is_finite(v.w));
+        }
+      } else {
+        for (long long r = r0 + lr; r < r1; r += side) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            if (col0 + c < ncols) {
+              const float v = __ldcs(W + r * ld + col0 + c);
+              mn[c] = fminf(mn[c], v);
+              mx[c] = fmaxf(mx[c], v);
+              bad |= !is_finite(v);
+            }
+          }
+        }
+      }
+      if (r0 + lr < r1) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (col0 + c < ncols) {
+            atomicMin(&s_min[col0 + c], ord_encode(mn[c]));
+            atomicMax(&s_max[col0 + c], ord_encode(mx[c]));
+          }
+        }
+      }
+    }
+    __syncthreads();
+    if (r0 < r1) {
+      for (int i = threadIdx.x; i < ncols; i += 256) {
+        atomicMin(&colmin[i], s_min[i]);
+        atomicMax(&colmax[i], s_max[i]);
+      }
+    }
+    if (bad) flag(dev_status, OCS_DEV_NONFINITE);
+  }
+}
+
 // K1: per-column signed extrema of a row-major [O][ncols] fp32 matrix.
 template <bool VEC>
 __global__ void __launch_bounds__(256)
@@ -46,10 +119,10 @@ col_minmax_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uin
   for (int c = blockIdx.x * 256 + threadIdx.x; c < C; c += gridDim.x * 256) {
     idx_map[c] = c; depth[c] = 0; bits[c] = 0ull;
   }
+  bool bad = false;
   const int col_blocks = (ncols + 1023) / 1024;
   long long u, u1;
   cta_range((long long)col_blocks * O, &u, &u1);
-  bool bad = false;
   while (u < u1) {
     const int cb = (int)(u / O);
     const int r0 = (int)(u - (long long)cb * O);
@@ -974,7 +1047,13 @@ ocs_status run_split_front(const float* W, int O, int C, int R, int64_t ld_in, i
     const long long units = (long long)((ncols + 1023) / 1024) * O;
     const bool vec = (ld_in % 4 == 0) && aligned(W, 16);
     LaunchScope ls("col_minmax_kernel", stream);
-    if (vec)
+    if (ncols <= 512 && vec)
+      col_minmax_narrow_kernel<true><<<wave_grid(col_minmax_narrow_kernel<true>, units), 256, 0, stream>>>(
+          W, O, ncols, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
+    else if (ncols <= 512)
+      col_minmax_narrow_kernel<false><<<wave_grid(col_minmax_narrow_kernel<false>, units), 256, 0, stream>>>(
+          W, O, ncols, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
+    else if (vec)
       col_minmax_kernel<true><<<wave_grid(col_minmax_kernel<true>, units), 256, 0, stream>>>(
           W, O, ncols, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
     else
@@ -1105,6 +1184,110 @@ FusedWs carve_fused_ws(void* ws, int C, int R, int S, int n_bins, int n_candidat
 
 namespace ocs {
 namespace {
+// Code pass for short rows under the plain w/2 split (the case of activation matrices: a row is one pixel's
+// or one sample's channels).  Staging whole rows in shared memory buys nothing when a row is a few hundred
+// bytes, so this form streams.  The warps of a CTA form two groups that walk the CTA's rows independently:
+// the main group converts the original columns (a thread owns one group of four columns for every row it
+// visits: one 128-bit load, halving counts in registers, one 32-bit store), the tail group the duplicated
+// channels (four loads of source columns whose lines the main group has just read).  Keeping the two kinds
+// of work in different warps keeps either from waiting on the other's divergent path.  Repeated halving
+// keeps the checker's rounding, subnormals included.
+__global__ void __launch_bounds__(256, 4)
+rows_quant_narrow_kernel(const float* __restrict__ W, int O, int C, int R, long long ld_in, int S,
+                         const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
+                         const float* __restrict__ maxp, const double* __restrict__ scores, int n_candidates, int L,
+                         int is_signed, int8_t* __restrict__ codes, long long ld_codes, int packed_ok, int vec_ok,
+                         int tail_warps, float* __restrict__ scale_out, float* __restrict__ alpha_out) {
+  float alpha = *maxp;
+  if (scores && alpha > 0.0f) alpha = pick_alpha(scores, alpha, n_candidates);
+  const bool zero = !(alpha > 0.0f);
+  const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)L);
+  const float inv = zero ? 0.0f : __fdiv_rn((float)L, alpha);
+  const float lo = is_signed ? -(float)L : 0.0f, hi = (float)L;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *scale_out = step;
+    if (alpha_out) *alpha_out = zero ? 0.0f : alpha;
+  }
+  const int in_cols = C * R, out_cols = (C + S) * R;
+  const int main_threads = 256 - 32 * tail_warps;
+  const bool is_tail = (int)threadIdx.x >= main_threads;
+  const int t = is_tail ? (int)threadIdx.x - main_threads : (int)threadIdx.x;
+  const int group = is_tail ? 32 * tail_warps : main_threads;
+  const int first_col = is_tail ? in_cols : 0;
+  const int n_quads = ((is_tail ? out_cols - in_cols : in_cols) + 3) >> 2;   // <= group (checked by the host)
+  const int side = group / n_quads;
+  const int lr = t / n_quads, col0 = first_col + (t - lr * n_quads) * 4;
+  if (lr >= side) return;
+  const int col_end = is_tail ? out_cols : in_cols;
+  int src[4], dep[4];
+  bool valid[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int col = col0 + e;
+    valid[e] = col < col_end;
+    src[e] = 0; dep[e] = 0;
+    if (valid[e]) {
+      const int ch = col / R, r = col - ch * R;
+      dep[e] = __ldg(depth + ch);
+      src[e] = (ch < C ? ch : __ldg(idx_map + ch)) * R + r;
+    }
+  }
+  const bool contiguous = !is_tail && vec_ok && valid[3];
+  const bool any_dep = (dep[0] | dep[1] | dep[2] | dep[3]) != 0;
+  long long r0, r1;
+  cta_range((long long)O, &r0, &r1);
+  auto emit = [&](long long r, float (&x)[4]) {
+    if (any_dep) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        for (int d = 0; d < dep[e]; ++d) x[e] = __fmul_rn(x[e], 0.5f);
+    }
+    const int c0 = quant_code(x[0], inv, lo, hi), c1 = quant_code(x[1], inv, lo, hi);
+    const int c2 = quant_code(x[2], inv, lo, hi), c3 = quant_code(x[3], inv, lo, hi);
+    int8_t* out = codes + r * ld_codes + col0;
+    if (packed_ok && valid[3]) {
+      *reinterpret_cast<unsigned int*>(out) = pack4(c0, c1, c2, c3);
+    } else {
+      if (valid[0]) out[0] = (int8_t)c0;
+      if (valid[1]) out[1] = (int8_t)c1;
+      if (valid[2]) out[2] = (int8_t)c2;
+      if (valid[3]) out[3] = (int8_t)c3;
+    }
+  };
+  if (contiguous) {
+    // eight rows' loads in flight per thread before the first is consumed
+    constexpr int kBatch = 8;
+    const long long stride = (long long)side * ld_in;
+    const float* p = W + (r0 + lr) * ld_in + col0;
+    for (long long r = r0 + lr; r < r1; r += (long long)kBatch * side, p += kBatch * stride) {
+      float4 v[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u)
+        v[u] = (r + (long long)u * side < r1) ? __ldcs(reinterpret_cast<const float4*>(p + u * stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        if (r + (long long)u * side < r1) {
+          float x[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+          emit(r + (long long)u * side, x);
+        }
+      }
+    }
+  } else {
+#pragma unroll 2
+    for (long long r = r0 + lr; r < r1; r += side) {
+      const float* row = W + r * ld_in;
+      float x[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) x[e] = valid[e] ? __ldg(row + src[e]) : 0.0f;
+      emit(r, x);
+    }
+  }
+}
+}  // namespace
+}  // namespace ocs
+
+namespace ocs {
+namespace {
 // Rows-per-buffer, row-group count and shared-memory bytes of the row-staged kernels.
 struct RowsGeometry {
   long long g;
@@ -1137,13 +1320,26 @@ ocs_status rows_attr_once() {
 // The code pass: rows staged in shared memory, split there, quantized and written as packed codes.
 ocs_status launch_rows_quant(const float* W, int O, int C, int R, int64_t ld_in, int S, const int32_t* idx_map,
                              const SplitWs& w, RowsEpilogue ep, int8_t* codes, int64_t ld_codes, float* scale,
-                             float* alpha, int g, int srow, int n_groups, size_t rows_smem, int* dev_status,
+                             float* alpha, int g, int srow, int n_groups, size_t rows_smem, bool naive, int* dev_status,
                              cudaStream_t stream) {
   ep.codes = codes;
   ep.ld_codes = ld_codes;
   ep.packed_ok = aligned(codes, 4) && (ld_codes % 4 == 0);
   ep.scale_out = scale;
   ep.alpha_out = alpha;
+  // short rows, plain halving: the streaming form (both column groups must fit their warps)
+  const int main_quads = (C * R + 3) / 4, tail_quads = (S * R + 3) / 4;
+  const int tail_warps = S == 0 ? 0 : (12 * tail_quads >= main_quads ? 2 : 1);
+  if (naive && (C * R) % 4 == 0 && main_quads <= 256 - 32 * tail_warps && tail_quads <= 32 * tail_warps) {
+    const int side = (256 - 32 * tail_warps) / main_quads;
+    const int grid = wave_grid(rows_quant_narrow_kernel, ((long long)O + side - 1) / side);   // one resident wave
+    const int vec_ok = (ld_in % 4 == 0) && aligned(W, 16);
+    LaunchScope ls("split_quantize_kernel", stream);
+    rows_quant_narrow_kernel<<<grid, 256, 0, stream>>>(W, O, C, R, ld_in, S, idx_map, w.depth, ep.maxp, ep.scores,
+                                                       ep.n_candidates, ep.L, ep.is_signed, codes, ld_codes, ep.packed_ok,
+                                                       vec_ok, tail_warps, scale, alpha);
+    return launch_status();
+  }
   LaunchScope ls("split_quantize_kernel", stream);
   split_rows_kernel<ROWS_QUANT><<<min(n_groups, kNumSMs), kRowThreads, rows_smem, stream>>>(
       W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, g, srow, ep,
@@ -1225,7 +1421,7 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
   ep.scores = scores;
   ep.n_candidates = n_candidates;
   return launch_rows_quant(W, O, C, R, ld_in, S, idx_map, w, ep, codes, ld_codes, scale, alpha, (int)g, srow, n_groups,
-                           rows_smem, dev_status, stream);
+                           rows_smem, qa_step == 0.0f && qa_bits == 0, dev_status, stream);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1314,8 +1510,12 @@ extern "C" ocs_status ocs_act_split_quantize_static(const float* A, int rows, in
     if (cudaMemsetAsync(w.colmax, 0x00, 4 * (size_t)C, stream) != cudaSuccess) return OCS_ERR_CUDA;
     const long long units = (long long)((C + 1023) / 1024) * rows;
     LaunchScope ls("col_minmax_kernel", stream);
-    col_minmax_kernel<true><<<wave_grid(col_minmax_kernel<true>, units), 256, 0, stream>>>(
-        A, rows, C, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
+    if (C <= 512)
+      col_minmax_narrow_kernel<true><<<wave_grid(col_minmax_narrow_kernel<true>, units), 256, 0, stream>>>(
+          A, rows, C, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
+    else
+      col_minmax_kernel<true><<<wave_grid(col_minmax_kernel<true>, units), 256, 0, stream>>>(
+          A, rows, C, ld_in, w.colmin, w.colmax, C, idx_map, w.depth, w.bits, dev_status);
     if ((st = launch_status()) != OCS_OK) return st;
   }
   {
@@ -1335,7 +1535,7 @@ extern "C" ocs_status ocs_act_split_quantize_static(const float* A, int rows, in
   ep.scores = nullptr;
   ep.n_candidates = 1;
   return launch_rows_quant(A, rows, C, 1, ld_in, S, idx_map, w, ep, codes, ld_codes, scale, nullptr, (int)geo.g, srow,
-                           geo.n_groups, geo.rows_smem, dev_status, stream);
+                           geo.n_groups, geo.rows_smem, true, dev_status, stream);
 }
 
 // ------------------------------------------------------------------------------------------------
