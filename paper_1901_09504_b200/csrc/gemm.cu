@@ -150,6 +150,9 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank) {
 __device__ __forceinline__ void st_peer_v4(uint32_t addr, uint4 v) {
   asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+__device__ __forceinline__ void st_local_v4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_peer(uint32_t addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
 }
@@ -543,6 +546,8 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     int tt = 0;          // tail tiles assembled so far
     int n_tiles_done = 0;
     int table_kb[2] = {-1, -1};   // which K-block each of the two source tables describes
+    int buf_kb[kTailBufs];        // which K-block each tail buffer held last (same for every CTA of the cluster)
+    for (int g = 0; g < kTailBufs; ++g) buf_kb[g] = -1;
     WorkItem w;
     for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
       if (w.n_tail == 0) continue;
@@ -590,15 +595,23 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             v = gather_chunk(p, ri, rbase, tab + c * 16);
           }
           const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
-          for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), v);
+          if (CL == 1) st_local_v4(off, v);   // a lone CTA: plain shared-memory stores
+          else
+            for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), v);
         }
-        // the K padding
+        // the K padding: zero, unless this buffer's last occupant was the same K-block (every tile of a layer
+        // has the same tail blocks, so the chunks that hold data are overwritten and the padding stays zero)
         const int zero_chunks = 8 - valid_chunks;
-        for (int it = gt; it < RP * zero_chunks; it += kGatherThreads) {
-          const int rl = it / zero_chunks, c = valid_chunks + (it - rl * zero_chunks);
-          const int r = (int)crank * RP + rl;
-          const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
-          for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), make_uint4(0u, 0u, 0u, 0u));
+        if (buf_kb[g] != kb) {
+          for (int it = gt; it < RP * zero_chunks; it += kGatherThreads) {
+            const int rl = it / zero_chunks, c = valid_chunks + (it - rl * zero_chunks);
+            const int r = (int)crank * RP + rl;
+            const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
+            if (CL == 1) st_local_v4(off, make_uint4(0u, 0u, 0u, 0u));
+            else
+              for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), make_uint4(0u, 0u, 0u, 0u));
+          }
+          buf_kb[g] = kb;
         }
         // make the generic-proxy stores visible to the tensor cores that read them
         if (CL == 1) fence_proxy_async_smem(); else fence_proxy_async_cluster();
