@@ -307,6 +307,9 @@ ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, in
  *
  * ocs_add_relu: y[i] = a[i] + b[i] (b NULL: y[i] = a[i]), then max(., 0) when relu != 0
  *   (ReLU after a layer; the residual connection of a bottleneck block).  y may equal a.
+ *   max_abs_out (device, fp32 [1], may be NULL) receives max |y| of the whole tensor: the next
+ *   layer's activation grid (pass it to ocs_quantize as max_abs_in), taken here to save a pass.
+ *   A NaN in y does not enter the maximum (ocs_quantize flags non-finite input itself).
  * ocs_maxpool3x3s2: 3x3 window, stride 2, padding 1 (padding never wins);
  *   y [Nb][(H-1)/2+1][(Wd-1)/2+1][C].
  * ocs_global_avgpool: y[n][c] = (sum over (h, w), row-major, sequential) * (1 / (H*Wd)).
@@ -320,7 +323,8 @@ ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, in
  *   with t = x * log2(e), n = rint(t), f = t - n, P the degree-6 Taylor polynomial of exp in
  *   Horner form with fused multiply-adds (x clamped at -87); sigmoid = 1/(1+e) or e/(1+e),
  *   tanh = (1-e)/(1+e) with the sign of x; divisions IEEE. */
-ocs_status ocs_add_relu(const float* a, const float* b, int64_t n, int relu, float* y, void* stream);
+ocs_status ocs_add_relu(const float* a, const float* b, int64_t n, int relu, float* y, float* max_abs_out,
+                        void* stream);
 ocs_status ocs_maxpool3x3s2(const float* x, int Nb, int H, int Wd, int C, float* y, void* stream);
 ocs_status ocs_global_avgpool(const float* x, int Nb, int H, int Wd, int C, float* y, void* stream);
 ocs_status ocs_nchw_to_nhwc(const float* x, int Nb, int C, int H, int Wd, float* y, void* stream);

@@ -256,13 +256,13 @@ def ocs_qconv(X_codes, a_scale, W_packed, w_scale, idx_map, S: int, kh: int, kw:
     return (Y, acc) if want_acc else Y
 
 
-def ocs_add_relu(a, b=None, relu: bool = True, out=None):
-    """y = a (+ b), then ReLU when relu; fp32 tensors of equal shape."""
+def ocs_add_relu(a, b=None, relu: bool = True, out=None, max_out=None):
+    """y = a (+ b), then ReLU when relu; fp32 tensors of equal shape.  max_out (fp32 [1]) receives max |y|."""
     assert a.is_cuda and a.dtype == torch.float32 and a.is_contiguous()
     assert b is None or (b.shape == a.shape and b.dtype == torch.float32 and b.is_contiguous())
     y = out if out is not None else torch.empty_like(a)
-    _check(lib().ocs_add_relu(_ptr(a), _ptr(b), C.c_int64(a.numel()), int(bool(relu)), _ptr(y), _stream()),
-           "ocs_add_relu")
+    _check(lib().ocs_add_relu(_ptr(a), _ptr(b), C.c_int64(a.numel()), int(bool(relu)), _ptr(y), _ptr(max_out),
+                              _stream()), "ocs_add_relu")
     return y
 
 

@@ -14,10 +14,15 @@ int ew_grid(long long n, int per_thread) {
 }
 
 // y = max(x, 0) (relu = 1) applied to a + b (b may be null: plain ReLU / copy)
+// max_bits (optional): fp32 bits of max|y| over the whole tensor, combined with atomicMax (the values are
+// non-negative, so their bit patterns order like the values); the next layer's activation grid needs it,
+// and taking it here saves that layer a pass over the tensor.
 template <bool VEC>
 __global__ void __launch_bounds__(256)
-add_relu_kernel(const float* __restrict__ a, const float* __restrict__ b, long long n, int relu, float* __restrict__ y) {
+add_relu_kernel(const float* __restrict__ a, const float* __restrict__ b, long long n, int relu, float* __restrict__ y,
+                unsigned int* __restrict__ max_bits) {
   const long long stride = (long long)gridDim.x * 256;
+  float m = 0.0f;
   if (VEC) {
     const long long n4 = n >> 2;
     for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n4; i += stride) {
@@ -30,19 +35,28 @@ add_relu_kernel(const float* __restrict__ a, const float* __restrict__ b, long l
         v.x = v.x > 0.0f ? v.x : 0.0f; v.y = v.y > 0.0f ? v.y : 0.0f;
         v.z = v.z > 0.0f ? v.z : 0.0f; v.w = v.w > 0.0f ? v.w : 0.0f;
       }
+      m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
       reinterpret_cast<float4*>(y)[i] = v;
     }
     for (long long i = (n4 << 2) + blockIdx.x * 256ll + threadIdx.x; i < n; i += stride) {
       float v = a[i];
       if (b) v = __fadd_rn(v, b[i]);
-      y[i] = (relu && !(v > 0.0f)) ? 0.0f : v;
+      v = (relu && !(v > 0.0f)) ? 0.0f : v;
+      m = fmaxf(m, fabsf(v));
+      y[i] = v;
     }
   } else {
     for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += stride) {
       float v = a[i];
       if (b) v = __fadd_rn(v, b[i]);
-      y[i] = (relu && !(v > 0.0f)) ? 0.0f : v;
+      v = (relu && !(v > 0.0f)) ? 0.0f : v;
+      m = fmaxf(m, fabsf(v));
+      y[i] = v;
     }
+  }
+  if (max_bits) {
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0 && m > 0.0f) atomicMax(max_bits, __float_as_uint(m));
   }
 }
 
@@ -175,16 +189,19 @@ lstm_cell_kernel(const float* __restrict__ g_ih, const float* __restrict__ g_hh,
 
 using namespace ocs;
 
-extern "C" ocs_status ocs_add_relu(const float* a, const float* b, int64_t n, int relu, float* y, void* stream_) {
+extern "C" ocs_status ocs_add_relu(const float* a, const float* b, int64_t n, int relu, float* y, float* max_abs_out,
+                                   void* stream_) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!a || !y) return OCS_ERR_INVALID_ARG;
   if (n <= 0) return OCS_ERR_SHAPE;
   ocs_status st = check_device();
   if (st != OCS_OK) return st;
+  if (max_abs_out && cudaMemsetAsync(max_abs_out, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
+  unsigned int* mb = reinterpret_cast<unsigned int*>(max_abs_out);
   const bool vec = aligned(a, 16) && aligned(y, 16) && (!b || aligned(b, 16));
   LaunchScope ls("add_relu_kernel", stream);
-  if (vec) add_relu_kernel<true><<<ew_grid(n, 8), 256, 0, stream>>>(a, b, n, relu, y);
-  else add_relu_kernel<false><<<ew_grid(n, 8), 256, 0, stream>>>(a, b, n, relu, y);
+  if (vec) add_relu_kernel<true><<<ew_grid(n, 8), 256, 0, stream>>>(a, b, n, relu, y, mb);
+  else add_relu_kernel<false><<<ew_grid(n, 8), 256, 0, stream>>>(a, b, n, relu, y, mb);
   return launch_status();
 }
 

@@ -312,6 +312,51 @@ quantize_kernel(View v, const float* __restrict__ alpha_p, const double* __restr
   if (bad) flag(dev_status, OCS_DEV_NONFINITE);
 }
 
+// Small tensors without a clip search (the per-step activations of a recurrent network, a classifier's
+// input): one CTA finds max|x| and writes the codes in the same launch -- the second read hits the cache,
+// and a launch of latency is saved where latency is all there is.
+constexpr long long kSmallQuantElems = 65536;
+
+__global__ void __launch_bounds__(1024)
+small_quantize_kernel(const float* __restrict__ T, int rows, int cols, long long ld_in, int L, int is_signed,
+                      int8_t* __restrict__ codes, long long ld_codes, float* __restrict__ scale_out,
+                      float* __restrict__ alpha_out, unsigned int* __restrict__ maxbits, int* dev_status) {
+  __shared__ float red[32];
+  __shared__ float s_alpha;
+  const int n = rows * cols;
+  float m = 0.0f;
+  bool bad = false;
+  for (int i = threadIdx.x; i < n; i += 1024) {
+    const int r = i / cols, c = i - r * cols;
+    const float x = T[r * ld_in + c];
+    bad |= !is_finite(x);
+    m = fmaxf(m, fabsf(x));
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 32; ++w) m = fmaxf(m, red[w]);
+    s_alpha = m;
+    *maxbits = __float_as_uint(m);
+  }
+  __syncthreads();
+  const float alpha = s_alpha;
+  const bool zero = !(alpha > 0.0f);
+  const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)L);
+  const float inv = zero ? 0.0f : __fdiv_rn((float)L, alpha);
+  const float lo = is_signed ? -(float)L : 0.0f, hi = (float)L;
+  if (threadIdx.x == 0) {
+    *scale_out = step;
+    if (alpha_out) *alpha_out = zero ? 0.0f : alpha;
+  }
+  for (int i = threadIdx.x; i < n; i += 1024) {
+    const int r = i / cols, c = i - r * cols;
+    codes[r * ld_codes + c] = (int8_t)quant_code(T[r * ld_in + c], inv, lo, hi);
+  }
+  if (bad) flag(dev_status, OCS_DEV_NONFINITE);
+}
+
 struct QuantWs {
   unsigned int* maxbits;       // fp32 bits of max|T|
   unsigned long long* hist;
@@ -384,6 +429,12 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   const View v = make_view(T, rows, cols, ld_in);
   const int L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
 
+  if (mode == OCS_CLIP_NONE && !max_abs_in && rows * cols <= kSmallQuantElems) {
+    LaunchScope ls("small_quantize_kernel", stream);
+    small_quantize_kernel<<<1, 1024, 0, stream>>>(T, (int)rows, (int)cols, ld_in, L, is_signed, codes, ld_codes, scale,
+                                                  alpha, w.maxbits, dev_status);
+    return launch_status();
+  }
   const float* maxp = max_abs_in;
   if (!maxp) {
     if (cudaMemsetAsync(w.maxbits, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;

@@ -45,17 +45,18 @@ def prepare_layer(W, bias, ratio: float, bits: int, clip_mode: int = B.CLIP_NONE
     return QLayer(codes, scale, idx_map, bias, Cn, O, S, k, stride, pad)
 
 
-def quantize_activations(x, signed: bool, bits: int = 8, dev_status=None):
+def quantize_activations(x, signed: bool, bits: int = 8, dev_status=None, max_abs=None):
     """Dynamic per-tensor grid (max |x| of the tensor handed to the layer): returns dense codes shaped
-    like x and the fp32 [1] scale."""
+    like x and the fp32 [1] scale.  max_abs (fp32 [1] on the device): max |x| when the producer of x
+    already took it."""
     flat = x.reshape(1, -1)
-    codes, scale, _ = B.ocs_quantize(flat, bits, signed, B.CLIP_NONE, dev_status=dev_status)
+    codes, scale, _ = B.ocs_quantize(flat, bits, signed, B.CLIP_NONE, max_abs_in=max_abs, dev_status=dev_status)
     return codes[0, :flat.shape[1]].view(x.shape), scale
 
 
-def conv_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None):
+def conv_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None, max_abs=None):
     """x fp32 NHWC -> fp32 NHWC (activation quantization + ocs_qconv)."""
-    xc, xs = quantize_activations(x, a_signed, a_bits, dev_status)
+    xc, xs = quantize_activations(x, a_signed, a_bits, dev_status, max_abs)
     return B.ocs_qconv(xc, xs, L.codes, L.w_scale, L.idx_map, L.S, L.k, L.k, L.stride, L.pad, bias=L.bias,
                        dev_status=dev_status)
 
@@ -89,16 +90,19 @@ def prepare_resnet50(cfg, device, dev_status=None):
 def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, dev_status=None):
     """X fp32 NCHW on the device -> logits fp32 [Nb, 1000]; with keep, also every named tensor."""
     t = {}
+    mx = {}     # max |tensor| of the tensors ocs_add_relu produced (it takes the maximum while it writes them)
     x = B.ocs_nchw_to_nhwc(X_nchw.contiguous())
     first = True
     for spec in cfg["layers"]:
         src = t[spec.input_from] if spec.input_from else x
-        y = conv_forward(layers[spec.name], src, a_signed=first, a_bits=a_bits, dev_status=dev_status)
-        if spec.residual_from:
-            y = B.ocs_add_relu(y, t[spec.residual_from], relu=spec.relu, out=y)
-            t[spec.name.rsplit(".", 1)[0] + ".out"] = y
-        elif spec.relu:
-            y = B.ocs_add_relu(y, None, relu=True, out=y)
+        y = conv_forward(layers[spec.name], src, a_signed=first, a_bits=a_bits, dev_status=dev_status,
+                         max_abs=mx.get(id(src)))
+        if spec.residual_from or spec.relu:
+            m = torch.zeros(1, dtype=torch.float32, device=y.device)
+            y = B.ocs_add_relu(y, t[spec.residual_from] if spec.residual_from else None, relu=spec.relu, out=y, max_out=m)
+            mx[id(y)] = m
+            if spec.residual_from:
+                t[spec.name.rsplit(".", 1)[0] + ".out"] = y
         t[spec.name] = y
         x = y
         if first:
