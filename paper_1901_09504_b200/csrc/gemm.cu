@@ -70,6 +70,8 @@ struct GemmParams {
   float* Y;
   long long ldy;
   int32_t* acc_out;
+  int relu;                     // max(., 0) applied to Y
+  unsigned int* max_bits;       // fp32 bits of max |Y| over the whole output (optional)
   int32_t* acc_ws;              // [split_k][rows][N] partial sums when split_k > 1
   long long out_rows;           // rows of Y
   int a_box_bytes;              // bytes one TMA load of A delivers
@@ -649,6 +651,8 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       const long long ldd = direct ? p.ldy : (long long)p.N;
       const bool base_vec = ((reinterpret_cast<uintptr_t>(dst0) & 15) == 0) && (ldd % 4 == 0);
       const bool acc_vec = p.acc_out && ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) && (p.ldy % 4 == 0);
+      float tile_max = 0.0f;
+      const bool want_max = direct && p.max_bits != nullptr;
       for (int c0 = 0; c0 < BN; c0 += 32) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
@@ -682,10 +686,25 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           uint4 o[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            o[i].x = __float_as_uint(fmaf(int_to_float_rn((int)a[i].x), sc, b4[0]));
-            o[i].y = __float_as_uint(fmaf(int_to_float_rn((int)a[i].y), sc, b4[1]));
-            o[i].z = __float_as_uint(fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]));
-            o[i].w = __float_as_uint(fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]));
+            float f0 = fmaf(int_to_float_rn((int)a[i].x), sc, b4[0]), f1 = fmaf(int_to_float_rn((int)a[i].y), sc, b4[1]);
+            float f2 = fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]), f3 = fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]);
+            if (p.relu) {
+              f0 = f0 > 0.0f ? f0 : 0.0f; f1 = f1 > 0.0f ? f1 : 0.0f;
+              f2 = f2 > 0.0f ? f2 : 0.0f; f3 = f3 > 0.0f ? f3 : 0.0f;
+            }
+            if (want_max) {   // padding rows and columns past N are not part of the output
+              float rm;
+              if (full) {
+                rm = fmaxf(fmaxf(fabsf(f0), fabsf(f1)), fmaxf(fabsf(f2), fabsf(f3)));
+              } else {
+                rm = n0 + cq + 0 < p.N ? fabsf(f0) : 0.0f;
+                if (n0 + cq + 1 < p.N) rm = fmaxf(rm, fabsf(f1));
+                if (n0 + cq + 2 < p.N) rm = fmaxf(rm, fabsf(f2));
+                if (n0 + cq + 3 < p.N) rm = fmaxf(rm, fabsf(f3));
+              }
+              tile_max = fmaxf(tile_max, orow[i] >= 0 ? rm : 0.0f);
+            }
+            o[i] = make_uint4(__float_as_uint(f0), __float_as_uint(f1), __float_as_uint(f2), __float_as_uint(f3));
           }
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
@@ -721,6 +740,10 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           }
         }
       }
+      if (want_max) {
+        for (int o = 16; o > 0; o >>= 1) tile_max = fmaxf(tile_max, __shfl_xor_sync(0xffffffffu, tile_max, o));
+        if (lane == 0 && tile_max > 0.0f) atomicMax(p.max_bits, __float_as_uint(tile_max));
+      }
       // the accumulator has been read out: hand it back to the MMA issuer
       tc_fence_before();
       __syncwarp();
@@ -745,7 +768,9 @@ template <bool VEC>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long rows, int N,
                      const float* __restrict__ a_scale, const float* __restrict__ w_scale,
-                     const float* __restrict__ bias, float* __restrict__ Y, long long ldy, int32_t* __restrict__ acc_out) {
+                     const float* __restrict__ bias, float* __restrict__ Y, long long ldy, int32_t* __restrict__ acc_out,
+                     int relu, unsigned int* __restrict__ max_bits) {
+  float m = 0.0f;
   const float sc = __fmul_rn(__ldg(a_scale), __ldg(w_scale));
   const long long slice = rows * (long long)N;
   const int per_row = VEC ? (N >> 2) : N;
@@ -762,10 +787,14 @@ splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long ro
         a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
       }
       float* y = Y + row * ldy + n;
-      y[0] = fmaf((float)a.x, sc, bias ? __ldg(bias + n + 0) : 0.0f);
-      y[1] = fmaf((float)a.y, sc, bias ? __ldg(bias + n + 1) : 0.0f);
-      y[2] = fmaf((float)a.z, sc, bias ? __ldg(bias + n + 2) : 0.0f);
-      y[3] = fmaf((float)a.w, sc, bias ? __ldg(bias + n + 3) : 0.0f);
+      float f[4] = {fmaf((float)a.x, sc, bias ? __ldg(bias + n + 0) : 0.0f), fmaf((float)a.y, sc, bias ? __ldg(bias + n + 1) : 0.0f),
+                    fmaf((float)a.z, sc, bias ? __ldg(bias + n + 2) : 0.0f), fmaf((float)a.w, sc, bias ? __ldg(bias + n + 3) : 0.0f)};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (relu) f[e] = f[e] > 0.0f ? f[e] : 0.0f;
+        m = fmaxf(m, fabsf(f[e]));
+        y[e] = f[e];
+      }
       if (acc_out) {
         int32_t* ao = acc_out + row * ldy + n;
         ao[0] = a.x; ao[1] = a.y; ao[2] = a.z; ao[3] = a.w;
@@ -773,9 +802,16 @@ splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long ro
     } else {
       int a = __ldcg(p);
       for (int z = 1; z < split_k; ++z) a += __ldcg(p + z * slice);
-      Y[row * ldy + n] = fmaf((float)a, sc, bias ? __ldg(bias + n) : 0.0f);
+      float f = fmaf((float)a, sc, bias ? __ldg(bias + n) : 0.0f);
+      if (relu) f = f > 0.0f ? f : 0.0f;
+      m = fmaxf(m, fabsf(f));
+      Y[row * ldy + n] = f;
       if (acc_out) acc_out[row * ldy + n] = a;
     }
+  }
+  if (max_bits) {
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0 && m > 0.0f) atomicMax(max_bits, __float_as_uint(m));
   }
 }
 
@@ -962,10 +998,10 @@ ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long lo
   LaunchScope ls("splitk_reduce_kernel", stream);
   if (vec)
     splitk_reduce_kernel<true><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
-                                                         p.bias, p.Y, p.ldy, p.acc_out);
+                                                         p.bias, p.Y, p.ldy, p.acc_out, p.relu, p.max_bits);
   else
     splitk_reduce_kernel<false><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
-                                                          p.bias, p.Y, p.ldy, p.acc_out);
+                                                          p.bias, p.Y, p.ldy, p.acc_out, p.relu, p.max_bits);
   return launch_status();
 }
 
@@ -1067,7 +1103,8 @@ extern "C" size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S) {
 extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C, int64_t lda,
                                   const int8_t* W_codes, const float* w_scale, int N, int S, int64_t ldw,
                                   const int32_t* idx_map, const float* bias, float* Y, int64_t ldy, int32_t* acc_out,
-                                  void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+                                  int relu, float* max_abs_out, void* ws, size_t ws_bytes, int* dev_status,
+                                  void* stream_) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!A_codes || !a_scale || !W_codes || !w_scale || !idx_map || !Y) return OCS_ERR_INVALID_ARG;
   if (S < 0) return OCS_ERR_INVALID_ARG;
@@ -1087,6 +1124,9 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
   p.a_vec16 = (lda % 16 == 0) && aligned(A_codes, 16);
   p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = ldy; p.acc_out = acc_out;
   p.dev_status = dev_status;
+  p.relu = relu ? 1 : 0;
+  p.max_bits = reinterpret_cast<unsigned int*>(max_abs_out);
+  if (max_abs_out && cudaMemsetAsync(max_abs_out, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
   const int m_tiles = (M + BM - 1) / BM;
   // K-blocks made of original channels only; without duplicates the last, partial block is TMA-fed too (the
   // tensor map zero-fills past C)
@@ -1172,7 +1212,8 @@ extern "C" size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O,
 extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H, int Wd, int C,
                                 const int8_t* W_packed, const float* w_scale, int O, int S, int kh, int kw, int stride,
                                 int pad, int64_t ldw, const int32_t* idx_map, const float* bias, float* Y,
-                                int32_t* acc_out, void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+                                int32_t* acc_out, int relu, float* max_abs_out, void* ws, size_t ws_bytes,
+                                int* dev_status, void* stream_) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!X_codes || !a_scale || !W_packed || !w_scale || !idx_map || !Y) return OCS_ERR_INVALID_ARG;
   if (S < 0) return OCS_ERR_INVALID_ARG;
@@ -1199,6 +1240,9 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   p.bw = g.bw; p.bh = g.bh; p.bn = g.bn; p.tiles_w = g.tiles_w; p.tiles_h = g.tiles_h; p.tiles_n = g.tiles_n;
   p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = O; p.acc_out = acc_out;
   p.dev_status = dev_status;
+  p.relu = relu ? 1 : 0;
+  p.max_bits = reinterpret_cast<unsigned int*>(max_abs_out);
+  if (max_abs_out && cudaMemsetAsync(max_abs_out, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
 
   // TMA serves the K-blocks of original channels: each lies inside one tap (the per-tap stride Cp is a
   // multiple of the K-block; channels past C read as zero); a strided convolution walks the image

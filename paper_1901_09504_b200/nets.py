@@ -54,11 +54,13 @@ def quantize_activations(x, signed: bool, bits: int = 8, dev_status=None, max_ab
     return codes[0, :flat.shape[1]].view(x.shape), scale
 
 
-def conv_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None, max_abs=None):
-    """x fp32 NHWC -> fp32 NHWC (activation quantization + ocs_qconv)."""
+def conv_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None, max_abs=None, relu: bool = False,
+                 max_out=None):
+    """x fp32 NHWC -> fp32 NHWC (activation quantization + ocs_qconv; ReLU and max |y| in the layer's epilogue
+    on request)."""
     xc, xs = quantize_activations(x, a_signed, a_bits, dev_status, max_abs)
     return B.ocs_qconv(xc, xs, L.codes, L.w_scale, L.idx_map, L.S, L.k, L.k, L.stride, L.pad, bias=L.bias,
-                       dev_status=dev_status)
+                       dev_status=dev_status, relu=relu, max_out=max_out)
 
 
 def linear_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None):
@@ -95,14 +97,15 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
     first = True
     for spec in cfg["layers"]:
         src = t[spec.input_from] if spec.input_from else x
+        m = torch.empty(1, dtype=torch.float32, device=x.device)
+        fused_relu = spec.relu and not spec.residual_from      # ReLU straight after the layer: in its epilogue
         y = conv_forward(layers[spec.name], src, a_signed=first, a_bits=a_bits, dev_status=dev_status,
-                         max_abs=mx.get(id(src)))
-        if spec.residual_from or spec.relu:
-            m = torch.zeros(1, dtype=torch.float32, device=y.device)
-            y = B.ocs_add_relu(y, t[spec.residual_from] if spec.residual_from else None, relu=spec.relu, out=y, max_out=m)
+                         max_abs=mx.get(id(src)), relu=fused_relu, max_out=m if fused_relu else None)
+        if spec.residual_from:
+            y = B.ocs_add_relu(y, t[spec.residual_from], relu=spec.relu, out=y, max_out=m)
+            t[spec.name.rsplit(".", 1)[0] + ".out"] = y
+        if fused_relu or spec.residual_from:
             mx[id(y)] = m
-            if spec.residual_from:
-                t[spec.name.rsplit(".", 1)[0] + ".out"] = y
         t[spec.name] = y
         x = y
         if first:

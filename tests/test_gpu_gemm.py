@@ -39,6 +39,15 @@ def _check_linear(seed, M, Cn, N, S, a_signed=False, lda=None, bias=True, a_scal
     np.testing.assert_array_equal(host(acc), acco)
     np.testing.assert_allclose(host(Y), Yo, rtol=1e-5, atol=0)
     np.testing.assert_array_equal(host(Y), Yo)
+    # ReLU and max |Y| taken in the layer's epilogue: the checker's relu and maxabs of its own output
+    m = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+    Yr = ocs.ocs_qlinear(Ad, dev(np.array([a_scale], np.float32)), Wd, dev(np.array([w_scale], np.float32)),
+                         dev(idx), Cn, S, bias=None if b is None else dev(b), relu=True, max_out=m, dev_status=st)
+    np.testing.assert_array_equal(host(Yr), orc.relu(Yo))
+    assert host(m)[0] == np.float32(orc.maxabs(orc.relu(Yo)))
+    ocs.ocs_qlinear(Ad, dev(np.array([a_scale], np.float32)), Wd, dev(np.array([w_scale], np.float32)),
+                    dev(idx), Cn, S, bias=None if b is None else dev(b), max_out=m, dev_status=st)
+    assert host(m)[0] == np.float32(orc.maxabs(Yo)) and ocs.ocs_poll_status(st) == 0
 
 
 @pytest.mark.parametrize("M,Cn,N,S", [(64, 512, 256, 26), (128, 256, 128, 0), (1, 16, 8, 0), (5, 130, 70, 3),
@@ -114,6 +123,11 @@ def _check_conv(seed, Nb, H, Wd_, Cn, O, S, k, stride, pad, a_signed=False):
     assert ocs.ocs_poll_status(st) == 0
     np.testing.assert_array_equal(host(acc), acco)
     np.testing.assert_array_equal(host(Y), Yo)
+    m = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
+    Yr = ocs.ocs_qconv(dev(X), dev(np.array([0.02], np.float32)), packed, dev(np.array([0.003], np.float32)),
+                       dev(idx), S, k, k, stride, pad, bias=dev(b), relu=True, max_out=m, dev_status=st)
+    np.testing.assert_array_equal(host(Yr), orc.relu(Yo))
+    assert host(m)[0] == np.float32(orc.maxabs(orc.relu(Yo))) and ocs.ocs_poll_status(st) == 0
 
 
 @pytest.mark.parametrize("Nb,H,W,Cn,O,S,k,stride,pad", [
