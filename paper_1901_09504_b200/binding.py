@@ -142,7 +142,7 @@ def ocs_split(W, S: int, qa_step: float = 0.0, qa_bits: int = 0, ld_out: int | N
         W_out = torch.empty((O, ld_out), dtype=torch.float32, device=W.device)
         idx_map = torch.empty(Cn + S, dtype=torch.int32, device=W.device)
         order = torch.empty(max(S, 1), dtype=torch.int32, device=W.device) if want_order else None
-        max_abs = torch.zeros(3, dtype=torch.float32, device=W.device)
+        max_abs = torch.empty(3, dtype=torch.float32, device=W.device)
     nws = lib().ocs_split_workspace_bytes(O, Cn, R, int(S))
     if ws is None:
         ws = _ws(nws, W.device)
@@ -171,8 +171,8 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
         assert codes.shape[0] == rows and ld_codes >= cols
     else:
         codes = torch.empty((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=T.device)
-        scale = torch.zeros(1, dtype=torch.float32, device=T.device)
-        alpha = torch.zeros(1, dtype=torch.float32, device=T.device)
+        scale = torch.empty(1, dtype=torch.float32, device=T.device)
+        alpha = torch.empty(1, dtype=torch.float32, device=T.device)
     if mode == CLIP_MSE_EXACT:
         n_bins = 0
     nws = lib().ocs_quantize_workspace_bytes(int(n_bins), int(n_candidates))
@@ -333,8 +333,8 @@ def ocs_quantize_noalloc(T, bits: int, is_signed: bool = True, mode: int = CLIP_
         if ld_codes is None:
             ld_codes = round_up(cols, 16)
         codes = torch.empty((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=T.device)
-        scale = torch.zeros(1, dtype=torch.float32, device=T.device)
-        alpha = torch.zeros(1, dtype=torch.float32, device=T.device)
+        scale = torch.empty(1, dtype=torch.float32, device=T.device)
+        alpha = torch.empty(1, dtype=torch.float32, device=T.device)
     st = lib().ocs_quantize_noalloc(_ptr(T), C.c_int64(rows), C.c_int64(cols), C.c_int64(ld_in), int(bits),
                                     int(bool(is_signed)), int(mode), int(n_candidates), int(n_bins),
                                     _ptr(max_abs_in), _ptr(codes), C.c_int64(ld_codes), _ptr(scale), _ptr(alpha),
@@ -363,11 +363,11 @@ def ocs_split_quantize(W, S: int, bits: int, mode: int = CLIP_NONE, is_signed: b
         if ld_codes is None:
             ld_codes = round_up(cols_out, 16)
         codes = torch.empty((O, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=W.device)
-        scale = torch.zeros(1, dtype=torch.float32, device=W.device)
-        alpha = torch.zeros(1, dtype=torch.float32, device=W.device)
+        scale = torch.empty(1, dtype=torch.float32, device=W.device)
+        alpha = torch.empty(1, dtype=torch.float32, device=W.device)
         idx_map = torch.empty(Cn + S, dtype=torch.int32, device=W.device)
         order = torch.empty(max(S, 1), dtype=torch.int32, device=W.device) if want_order else None
-        max_abs = torch.zeros(3, dtype=torch.float32, device=W.device)
+        max_abs = torch.empty(3, dtype=torch.float32, device=W.device)
     nws = lib().ocs_split_quantize_workspace_bytes(O, Cn, R, int(S), int(n_bins), int(n_candidates))
     if ws is None:
         ws = _ws(nws, W.device)
@@ -394,7 +394,7 @@ def ocs_act_select_channels(P, S: int, quantile: float = 0.99, dev_status=None):
     rows, Cn = P.shape
     sel = torch.empty(max(int(S), 1), dtype=torch.int32, device=P.device)
     counts = torch.empty(Cn, dtype=torch.int64, device=P.device)
-    thr = torch.zeros(1, dtype=torch.float32, device=P.device)
+    thr = torch.empty(1, dtype=torch.float32, device=P.device)
     ws = _ws(lib().ocs_act_select_workspace_bytes(Cn), P.device)
     st = lib().ocs_act_select_channels(_ptr(P), C.c_int64(rows), Cn, C.c_int64(P.stride(0)), int(S), C.c_double(quantile),
                                        _ptr(sel), _ptr(counts), _ptr(thr), _ptr(ws), C.c_size_t(ws.numel()),
@@ -417,7 +417,7 @@ def ocs_act_split_quantize_static(A, sel, bits: int, is_signed: bool, alpha_in=N
         if ld_codes is None:
             ld_codes = round_up(Cn + S, 16)
         codes = torch.empty((rows, ld_codes), dtype=torch.int8 if is_signed else torch.uint8, device=A.device)
-        scale = torch.zeros(1, dtype=torch.float32, device=A.device)
+        scale = torch.empty(1, dtype=torch.float32, device=A.device)
         idx_map = torch.empty(Cn + S, dtype=torch.int32, device=A.device)
     nws = lib().ocs_split_quantize_workspace_bytes(rows, Cn, 1, S, 1, 1)
     if ws is None:
