@@ -32,14 +32,25 @@ class QLayer:
 
 def prepare_layer(W, bias, ratio: float, bits: int, clip_mode: int = B.CLIP_NONE, qa_bits: int = 0, conv: bool = False,
                   stride: int = 1, pad: int = 0, n_candidates: int = 128, n_bins: int = 2048, dev_status=None) -> QLayer:
-    """W fp32 [O, C] or [O, C, k, k] on the device -> QLayer (ocs_split, ocs_quantize, ocs_pack_conv_weights)."""
+    """W fp32 [O, C] or [O, C, k, k] on the device -> QLayer (ocs_split_quantize, or ocs_split + ocs_quantize where
+    the fused call cannot stage the rows; ocs_pack_conv_weights)."""
     O, Cn = W.shape[0], W.shape[1]
     k = W.shape[2] if W.dim() == 4 else 1
     R = k * k
     S = B.ocs_num_splits(Cn, ratio)
-    W_out, idx_map, _, mx = B.ocs_split(W.contiguous(), S, qa_bits=qa_bits, dev_status=dev_status, want_order=False)
-    codes, scale, _ = B.ocs_quantize(W_out, bits, True, clip_mode, n_candidates, n_bins, cols=(Cn + S) * R,
-                                     max_abs_in=mx[1:2], dev_status=dev_status)
+    try:
+        # one call, no fp32 W' (rows that cannot be staged in shared memory are reported as unsupported)
+        if clip_mode not in (B.CLIP_NONE, B.CLIP_MSE):
+            raise B.OcsError("ocs_split_quantize", 4)
+        codes, scale, _, idx_map, _, _ = B.ocs_split_quantize(W.contiguous(), S, bits, clip_mode, qa_bits=qa_bits,
+                                                              n_candidates=n_candidates, n_bins=n_bins,
+                                                              dev_status=dev_status, want_order=False)
+    except B.OcsError as e:
+        if e.status != 4:
+            raise
+        W_out, idx_map, _, mx = B.ocs_split(W.contiguous(), S, qa_bits=qa_bits, dev_status=dev_status, want_order=False)
+        codes, scale, _ = B.ocs_quantize(W_out, bits, True, clip_mode, n_candidates, n_bins, cols=(Cn + S) * R,
+                                         max_abs_in=mx[1:2], dev_status=dev_status)
     if conv:
         codes = B.ocs_pack_conv_weights(codes, O, Cn, S, k, k)
     return QLayer(codes, scale, idx_map, bias, Cn, O, S, k, stride, pad)

@@ -167,3 +167,25 @@ def test_qconv_config2_reduced_batch():
     Y, acc = ocs.ocs_qconv(xcodes.reshape(4, 14, 14, 256), xs, packed, scale, idx_d, S, 3, 3, 1, 1, want_acc=True)
     np.testing.assert_array_equal(host(acc), acco)
     np.testing.assert_array_equal(host(Y), Yo)
+
+
+def test_qconv_first_layer_with_and_without_room_for_the_patch_matrix():
+    """A 3-channel 7x7 stride-2 layer runs over its patch matrix when the workspace has room for it and through
+    the in-kernel gather when it has not: the same accumulators either way."""
+    Nb, H, Cn, O, S, k, stride, pad = 3, 20, 3, 16, 1, 7, 2, 3
+    X = configs.random_codes(77, 0, (Nb, H, H, Cn), 0, 255, np.uint8)
+    Wc = configs.random_codes(77, 1, (O, Cn + S, k, k), -127, 127, np.int8)
+    idx = np.array([0, 1, 2, 1], np.int32)
+    Yo, acco = orc.qconv(X, False, 0.02, Wc, 0.003, idx, stride, pad, None)
+    packed = ocs.ocs_pack_conv_weights(dev(Wc.reshape(O, -1)), O, Cn, S, k, k)
+    full = ocs.lib().ocs_qconv_workspace_bytes(Nb, H, H, Cn, O, S, k, k, stride, pad)
+    Ho = (H + 2 * pad - k) // stride + 1
+    assert full >= Nb * Ho * Ho * 196                      # includes the patch matrix
+    for nbytes in (full, 1024):
+        ws = torch.empty(int(nbytes), dtype=torch.uint8, device="cuda")
+        st = ocs.new_status()
+        Y, acc = ocs.ocs_qconv(dev(X), dev(np.array([0.02], np.float32)), packed, dev(np.array([0.003], np.float32)),
+                               dev(idx), S, k, k, stride, pad, want_acc=True, dev_status=st, ws=ws)
+        assert ocs.ocs_poll_status(st) == 0
+        np.testing.assert_array_equal(host(acc), acco)
+        np.testing.assert_array_equal(host(Y), Yo)
