@@ -34,7 +34,9 @@ namespace {
 constexpr int BM = 128;        // UMMA M
 constexpr int BK = 128;        // bytes (= int8 elements) per K-block: one 128-byte swizzle span
 constexpr int UMMA_K = 32;     // K of one tcgen05.mma.kind::i8
-constexpr int kGemmThreads = 320;    // TMA warp, MMA warp, 4 gather warps, 4 epilogue warps
+constexpr int kGemmThreads = 448;    // TMA warp, MMA warp, 4 gather warps, 8 epilogue warps
+constexpr int kEpiWarps = 8;
+constexpr int kEpiCols = 16;         // accumulator columns an epilogue warp moves at a time
 constexpr int kGatherThreads = 128;
 constexpr long long kWaitCycles = 2000000000ll;  // about one second
 // A waiting thread sleeps inside mbarrier.try_wait until the phase completes or about this many nanoseconds
@@ -233,6 +235,18 @@ __device__ __forceinline__ float int_to_float_rn(int acc) {
   return fmaf(fh, 65536.0f, fl);
 }
 
+// 32 lanes x 16 consecutive 32-bit columns
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t v[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups of
 // 8 rows 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
@@ -371,9 +385,9 @@ struct SmemLayout {
   static constexpr int kSrcTableBytes = 2 * BK * 8;     // KSrc per contraction index, two gathered K-blocks
   // epilogue staging: per epilogue warp a 32 x 32 tile of 32-bit words, rows padded to 36 words (16-byte
   // aligned, conflict-free for 128-bit accesses by quarter warps), and the 32 output-row numbers
-  static constexpr int kEpiRowWords = 36;
+  static constexpr int kEpiRowWords = kEpiCols + 4;
   static constexpr int kEpiWarpBytes = 32 * kEpiRowWords * 4 + 32 * 8;
-  static constexpr int kEpiBytes = 4 * kEpiWarpBytes;
+  static constexpr int kEpiBytes = kEpiWarps * kEpiWarpBytes;
   static constexpr int kDynBytes =
       kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes + kSrcTableBytes + kEpiBytes;
   static_assert(kDynBytes <= 227 * 1024, "more dynamic shared memory than a CTA can have");
@@ -443,7 +457,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(accfull_bar(a), 1);    // the MMA issuer's commit
-      mbar_init(accempty_bar(a), 4);   // the four epilogue warps
+      mbar_init(accempty_bar(a), kEpiWarps);   // every epilogue warp
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -637,36 +651,39 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       tc_fence_after();
       const RowInfo ri = row_info(p, w.mt, q * 32 + lane);
       const int nt = w.nt, kz = w.kz;
-      // Each lane holds one row of the 32 x 32 chunk; written out that way a store instruction would touch
-      // 32 rows with 16 bytes each.  The chunk goes through shared memory instead, so that every quarter
-      // warp writes one row's 128 contiguous bytes (lane -> row i*4 + lane/8, words (lane%8)*4 .. +3).
-      uint32_t* st_words = reinterpret_cast<uint32_t*>(epi_stage + (size_t)q * L::kEpiWarpBytes);
+      // Each lane holds one row of a 32 x 16 piece of the accumulator; written out that way a store
+      // instruction would touch 32 rows with 16 bytes each.  The piece goes through shared memory instead, so
+      // that four neighbouring lanes write 64 contiguous bytes of one row (lane -> row i*8 + (qd&1)*4 + qd/2
+      // with qd = lane/4, words (lane%4)*4 .. +3; the row order keeps the shared-memory reads conflict-free).
+      // The two epilogue warps that share a tensor-memory lane quadrant take alternate pieces.
+      const int ew = warp - 6, half = ew >> 2;
+      uint32_t* st_words = reinterpret_cast<uint32_t*>(epi_stage + (size_t)ew * L::kEpiWarpBytes);
       long long* st_rows = reinterpret_cast<long long*>(st_words + 32 * L::kEpiRowWords);
       __syncwarp();
       st_rows[lane] = ri.out_row;
       __syncwarp();
-      const int sub = lane >> 3, cq = (lane & 7) * 4;
-      // destination of the chunk's words: Y (and acc_out), or this slice's partial sums [kz][row][n]
+      const int qd = lane >> 2, sub = (qd & 1) * 4 + (qd >> 1), cq = (lane & 3) * 4;
+      // destination of the words: Y (and acc_out), or this slice's partial sums [kz][row][n]
       uint32_t* dst0 = direct ? reinterpret_cast<uint32_t*>(p.Y) : reinterpret_cast<uint32_t*>(p.acc_ws) + (long long)kz * p.out_rows * p.N;
       const long long ldd = direct ? p.ldy : (long long)p.N;
       const bool base_vec = ((reinterpret_cast<uintptr_t>(dst0) & 15) == 0) && (ldd % 4 == 0);
       const bool acc_vec = p.acc_out && ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) && (p.ldy % 4 == 0);
       float tile_max = 0.0f;
       const bool want_max = direct && p.max_bits != nullptr;
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = half * kEpiCols; c0 < BN; c0 += 2 * kEpiCols) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
-        uint32_t v[32];
+        uint32_t v[kEpiCols];
         __syncwarp();
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
-        const bool full = n0 + 32 <= p.N;   // warp-uniform
+        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
+        const bool full = n0 + kEpiCols <= p.N;   // warp-uniform
         // raw accumulators -> shared memory, one row per lane
         uint32_t* mine = st_words + lane * L::kEpiRowWords;
 #pragma unroll
-        for (int jj = 0; jj < 32; jj += 4)
+        for (int jj = 0; jj < kEpiCols; jj += 4)
           *reinterpret_cast<uint4*>(mine + jj) = make_uint4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
         __syncwarp();
-        // this lane's four columns of every row it writes: their bias once per chunk
+        // this lane's four columns of every row it writes: their bias once per piece
         float b4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         if (direct && p.bias) {
 #pragma unroll
@@ -674,18 +691,18 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             if (n0 + cq + e < p.N) b4[e] = __ldg(p.bias + n0 + cq + e);
         }
         const bool vec0 = full && base_vec, vec1 = full && acc_vec;
-        long long orow[8];
-        uint4 a[8];
+        long long orow[4];
+        uint4 a[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int r = i * 4 + sub;
+        for (int i = 0; i < 4; ++i) {
+          const int r = i * 8 + sub;
           orow[i] = st_rows[r];
           a[i] = *reinterpret_cast<const uint4*>(st_words + r * L::kEpiRowWords + cq);
         }
         if (direct) {
-          uint4 o[8];
+          uint4 o[4];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
+          for (int i = 0; i < 4; ++i) {
             float f0 = fmaf(int_to_float_rn((int)a[i].x), sc, b4[0]), f1 = fmaf(int_to_float_rn((int)a[i].y), sc, b4[1]);
             float f2 = fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]), f3 = fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]);
             if (p.relu) {
@@ -707,7 +724,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             o[i] = make_uint4(__float_as_uint(f0), __float_as_uint(f1), __float_as_uint(f2), __float_as_uint(f3));
           }
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
+          for (int i = 0; i < 4; ++i) {
             if (orow[i] < 0) continue;
             uint32_t* d = dst0 + orow[i] * ldd + n0 + cq;
             if (vec0) {
@@ -726,7 +743,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           const long long rld = direct ? p.ldy : ldd;
           const bool rvec = direct ? vec1 : vec0;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
+          for (int i = 0; i < 4; ++i) {
             if (orow[i] < 0) continue;
             uint32_t* d = rbase + orow[i] * rld + n0 + cq;
             if (rvec) {
