@@ -3,6 +3,7 @@
 //
 //   acc[m][n] = sum_k Aexp[m][k] * Wc[n][k]      int8/uint8 x int8 -> int32 in tensor memory
 //   Y[m][n]   = fmaf((float)acc, a_scale*w_scale, bias[n])
+// A convolution whose pixels TMA cannot address runs as the same GEMM over a patch matrix built first.
 //
 // The expanded activation operand Aexp (activations with the duplicated channels appended) is never
 // written to global memory: K-blocks that hold only original channels are fetched by TMA straight
@@ -16,8 +17,10 @@
 //               stages runs on across tiles
 //   warp 1      allocates tensor memory (two accumulators), issues tcgen05.mma, commits to barriers
 //   warps 2..5  gather producers: assemble the A tiles of the K-blocks that hold duplicated channels
-//   warps 6..9  epilogue (tcgen05.ld -> fmaf -> global) of tile i while the main loop of tile i+1 runs
-// The K-blocks whose A tile is assembled ("tail" blocks) come last in a CTA's K order and use two
+//   warps 6..13 epilogue of tile i while the main loop of tile i+1 runs: tcgen05.ld, transposition through
+//               shared memory for full-sector stores, int32 -> fp32, fmaf (optionally ReLU and max |Y|);
+//               the two warps of a tensor-memory lane quadrant take alternate 16-column pieces
+// The K-blocks whose A tile is assembled ("tail" blocks) come last in a CTA's K order and use three
 // dedicated A buffers, so the gather warps start at kernel begin and run ahead of the TMA-fed main
 // loop.  CTAs that share the M tile and the K slice (neighbouring N tiles) form a thread-block
 // cluster: each assembles 1/CL of a tail tile's rows and stores them into every peer's buffer
