@@ -1076,35 +1076,76 @@ __global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, i
 // the matrix like any other, read through idx_map here.
 constexpr int kPatchMaxK = 4096;   // source table in shared memory: 8 bytes per contraction index
 
+// One CTA builds the patch rows of `tw` neighbouring output pixels of one output row: the kh input rows they
+// touch are staged in shared memory once (zero where the image ends), so every input byte is read from global
+// memory once per CTA instead of once per tap, and the gather runs on shared memory.
 __global__ void __launch_bounds__(256)
-conv_patches_kernel(GemmParams p, uint8_t* __restrict__ P, long long ldp, long long rows) {
-  extern __shared__ KSrc tab[];
+conv_patches_kernel(GemmParams p, uint8_t* __restrict__ P, long long ldp, int tw, int seg_per_row, long long n_units,
+                    int span_bytes) {
+  extern __shared__ unsigned char patch_smem[];
+  KSrc* tab = reinterpret_cast<KSrc*>(patch_smem);                  // [ldp]: off = dy * span + dx * C + c
+  uint8_t* img = patch_smem + (size_t)ldp * sizeof(KSrc);           // [kh][span_bytes]
   bool bad = false;
-  for (int k = threadIdx.x; k < (int)ldp; k += 256) tab[k] = k_source(p, k, &bad);
+  for (int k = threadIdx.x; k < (int)ldp; k += 256) {
+    KSrc e = k_source(p, k, &bad);
+    if (e.off >= 0) {
+      const int dy = e.dydx & 255, dx = e.dydx >> 8;
+      const int c = e.off - (dy * p.Wd + dx) * p.C;
+      e.off = dy * span_bytes + dx * p.C + c;
+    }
+    tab[k] = e;
+  }
   if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
-  __syncthreads();
-  const int tpr = (int)(ldp >> 2);                 // threads per row: 4 contraction indices each
-  const int rows_par = 256 / tpr > 0 ? 256 / tpr : 1;
-  const int lane_row = threadIdx.x / tpr, q = threadIdx.x - lane_row * tpr;
-  if (tpr <= 256 && lane_row >= rows_par) return;
-  const long long HoWo = (long long)p.Ho * p.Wo;
-  for (long long m = (long long)blockIdx.x * rows_par + lane_row; m < rows; m += (long long)gridDim.x * rows_par) {
-    const int n = (int)(m / HoWo);
-    const int rem = (int)(m - (long long)n * HoWo);
-    const int oh = rem / p.Wo, ow = rem - oh * p.Wo;
-    const int ih0 = oh * p.stride - p.pad, iw0 = ow * p.stride - p.pad;
-    const uint8_t* base = p.A + (((long long)n * p.H + ih0) * p.Wd + iw0) * p.C;
-    for (int kq = q; kq < tpr; kq += 256) {
-      uint32_t word = 0;
+  const int words_per_row = (int)(ldp >> 2);
+  for (long long u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int seg = (int)(u % seg_per_row);
+    const long long rest = u / seg_per_row;
+    const int oh = (int)(rest % p.Ho), n = (int)(rest / p.Ho);
+    const int ow0 = seg * tw, cnt = min(tw, p.Wo - ow0);
+    const int ih0 = oh * p.stride - p.pad, iw0 = ow0 * p.stride - p.pad;
+    __syncthreads();   // the previous unit's gather is done (and the table is complete)
+    // bytes [lo, hi) of a staged row lie inside the image
+    const int lo = max(0, -iw0) * p.C, hi = min(span_bytes, (p.Wd - iw0) * p.C);
+    for (int dy = 0; dy < p.kh; ++dy) {
+      const int ih = ih0 + dy;
+      const bool row_ok = (unsigned)ih < (unsigned)p.H;
+      const uint8_t* src = p.A + (((long long)n * p.H + ih) * p.Wd + iw0) * p.C;
+      uint8_t* dst = img + dy * span_bytes;
+      for (int bx = threadIdx.x; bx < span_bytes; bx += 256)
+        dst[bx] = (row_ok && bx >= lo && bx < hi) ? __ldg(src + bx) : (uint8_t)0;
+    }
+    __syncthreads();
+    const long long m0 = ((long long)n * p.Ho + oh) * p.Wo + ow0;
+    if (words_per_row <= 256) {
+      // a thread keeps one group of four contraction indices (their offsets in registers) and walks the pixels
+      const int side = 256 / words_per_row;
+      const int lp = threadIdx.x / words_per_row, kq = threadIdx.x - lp * words_per_row;
+      if (lp < side) {
+        int off[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const KSrc src = tab[kq * 4 + e];
-        const int ih = ih0 + (src.dydx & 255), iw = iw0 + (src.dydx >> 8);
-        const bool ok = src.off >= 0 && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd;
-        const uint32_t v = (uint32_t)__ldg(ok ? base + src.off : p.A);
-        word |= (ok ? v : 0u) << (8 * e);
+        for (int e = 0; e < 4; ++e) off[e] = tab[kq * 4 + e].off;
+        const int step = p.stride * p.C;
+        uint8_t* dst = P + (m0 + lp) * ldp + kq * 4;
+        const uint8_t* base = img + lp * step;
+        for (int px = lp; px < cnt; px += side, base += side * step, dst += side * ldp) {
+          uint32_t word = 0;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) word |= (off[e] >= 0 ? (uint32_t)base[off[e]] : 0u) << (8 * e);
+          *reinterpret_cast<uint32_t*>(dst) = word;
+        }
       }
-      *reinterpret_cast<uint32_t*>(P + m * ldp + kq * 4) = word;
+    } else {
+      for (int i = threadIdx.x; i < cnt * words_per_row; i += 256) {
+        const int px = i / words_per_row, kq = i - px * words_per_row;
+        const uint8_t* base = img + px * p.stride * p.C;
+        uint32_t word = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int off = tab[kq * 4 + e].off;
+          word |= (off >= 0 ? (uint32_t)base[off] : 0u) << (8 * e);
+        }
+        *reinterpret_cast<uint32_t*>(P + (m0 + px) * ldp + kq * 4) = word;
+      }
     }
   }
 }
@@ -1278,12 +1319,22 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
       const long long ldp = (Ktot + 15) / 16 * 16;
       uint8_t* P = reinterpret_cast<uint8_t*>(ws) + gemm_ws;
       {
-        const int tpr = (int)(ldp / 4);
-        const int rows_par = 256 / tpr > 0 ? 256 / tpr : 1;
-        const long long blocks = (g.out_rows + rows_par - 1) / rows_par;
-        const int grid = (int)min(blocks, (long long)kNumSMs * 16);
+        // output pixels per CTA: as many of one output row as keep the staged input rows within 40 KB
+        int tw = g.Wo;
+        auto span = [&](int t) { return ((t - 1) * stride + kw) * C; };
+        while (tw > 1 && (size_t)kh * span(tw) > 40 * 1024) tw = (tw + 1) / 2;
+        const int seg_per_row = (g.Wo + tw - 1) / tw;
+        const long long n_units = (long long)Nb * g.Ho * seg_per_row;
+        const size_t smem = (size_t)ldp * sizeof(KSrc) + (size_t)kh * span(tw);
+        static bool attr_set = false;
+        if (!attr_set) {
+          if (cudaFuncSetAttribute(conv_patches_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024) != cudaSuccess)
+            return OCS_ERR_CUDA;
+          attr_set = true;
+        }
+        const int grid = (int)min(n_units, (long long)kNumSMs * 8);
         LaunchScope ls("conv_patches_kernel", stream);
-        conv_patches_kernel<<<grid, 256, (size_t)ldp * sizeof(KSrc), stream>>>(p, P, ldp, g.out_rows);
+        conv_patches_kernel<<<grid, 256, smem, stream>>>(p, P, ldp, tw, seg_per_row, n_units, span(tw));
         if ((st = launch_status()) != OCS_OK) return st;
       }
       GemmParams q = p;
