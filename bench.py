@@ -201,6 +201,33 @@ class Fc6Sweep:
             ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S,
                             out=self.Y[i], ws=self.ws, dev_status=self.status)
 
+    # The step is a fixed chain of stream-ordered, allocation-free library calls on preallocated buffers: it is
+    # captured once in a CUDA graph (after an eager warm-up) and replayed, which removes the host work between
+    # the ~180 launches of a step.
+    graph = True
+    graph_obj = None
+
+    def _capture(self):
+        torch = self.torch
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.step()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        n0 = self.ocs.ocs_kernel_launches()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.step()
+        self.graph_launches = int(self.ocs.ocs_kernel_launches() - n0)
+        return g
+
+    def make_graph(self):
+        self.graph_obj = self._capture()
+
+    def step_graph(self):
+        self.graph_obj.replay()
+
     def e2e_buffers(self, host):
         """End-to-end steps: every step's inputs travel from pinned host memory and its outputs travel
         back.  The copy of step i+1's inputs runs on a second stream into a second pair of device
@@ -215,6 +242,7 @@ class Fc6Sweep:
         self.ready = [torch.cuda.Event(), torch.cuda.Event()]
         self.consumed = [torch.cuda.Event(), torch.cuda.Event()]
         self.k = 0
+        self.slot_graphs = {} if self.graph_obj is None else {0: self.graph_obj}
         torch.cuda.current_stream().synchronize()
         for e in self.consumed:
             e.record()
@@ -236,7 +264,12 @@ class Fc6Sweep:
         main = torch.cuda.current_stream()
         main.wait_event(self.ready[cur])
         self.W, self.A = self.Wd[cur], self.Ad[cur]
-        self.step()
+        if self.graph_obj is None:
+            self.step()
+        else:
+            if cur not in self.slot_graphs:      # one graph per input slot (the graph holds the buffers' addresses)
+                self.slot_graphs[cur] = self._capture()
+            self.slot_graphs[cur].replay()
         self.consumed[cur].record(main)
         for h, y in zip(self.hY, self.Y):
             h.copy_(y, non_blocking=True)
@@ -380,7 +413,10 @@ class ActOcs(Fc6Sweep):
 
     def step_e2e(self):
         self.X.copy_(self.hX, non_blocking=True)
-        self.step()
+        if self.graph_obj is None:
+            self.step()
+        else:
+            self.graph_obj.replay()
         self.hY.copy_(self.Y, non_blocking=True)
 
     def oracle_sample(self, orc, host):
@@ -504,6 +540,7 @@ class NetWorkload:
 
 class ResNet50(NetWorkload):
     name = "resnet50"
+    graph = True
 
     def __init__(self, batch=128, image=224):
         self.batch, self.image = batch, image
