@@ -217,7 +217,7 @@ class Fc6Sweep:
         torch.cuda.synchronize()
         n0 = self.ocs.ocs_kernel_launches()
         g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
+        with torch.cuda.graph(g, capture_error_mode="thread_local"):
             self.step()
         self.graph_launches = int(self.ocs.ocs_kernel_launches() - n0)
         return g
@@ -529,7 +529,7 @@ class NetWorkload:
         torch.cuda.synchronize()
         n0 = self.ocs.ocs_kernel_launches()
         self.graph_obj = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(self.graph_obj):
+        with torch.cuda.graph(self.graph_obj, capture_error_mode="thread_local"):
             self.graph_out = self.step()
         self.graph_launches = int(self.ocs.ocs_kernel_launches() - n0)
 
@@ -829,7 +829,13 @@ def main():
 
     use_graph = bool(getattr(wl, "graph", False))
     if use_graph:
-        wl.make_graph()
+        try:
+            wl.make_graph()
+        except RuntimeError as e:      # capture refused (another thread's CUDA call, an old driver): eager launches
+            print(f"bench: CUDA graph capture failed ({e}); timing eager launches", file=sys.stderr)
+            torch.cuda.synchronize()
+            wl.graph_obj = None
+            use_graph = False
     clk = sample_clocks_start() if rank == 0 else None
     ms_step, launches = timed(wl.step_graph if use_graph else wl.step, args.steps, args.warmup)
     if use_graph:
