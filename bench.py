@@ -203,7 +203,7 @@ class Fc6Sweep:
 
     # The step is a fixed chain of stream-ordered, allocation-free library calls on preallocated buffers: it is
     # captured once in a CUDA graph (after an eager warm-up) and replayed, which removes the host work between
-    # the ~180 launches of a step.
+    # the ~200 launches of a step.
     graph = True
     graph_obj = None
 

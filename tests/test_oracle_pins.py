@@ -239,6 +239,38 @@ def test_static_activation_split_is_eq4_with_a_fixed_list():
         orc.act_split_static(A, np.array([Cn], np.int32))
 
 
+def test_activation_ocs_lowers_the_layer_error_on_outlier_batches():
+    """Direction of Table 4 (6 activation bits, r = 0.02): on a batch with a few outlier channels the layer
+    output after per-batch activation OCS is closer to the float layer than without it, and a static choice
+    made on a profile batch with the same outlier channels does as well."""
+    rng = np.random.default_rng(29)
+    M, Cn, N = 64, 256, 32
+    A = np.abs(rng.standard_normal((M, Cn))).astype(np.float32)
+    hot = [17, 101, 200]
+    A[:, hot] *= 12.0
+    P = np.abs(rng.standard_normal((512, Cn))).astype(np.float32)
+    P[:, hot] *= 12.0
+    W = rng.laplace(0, 0.02, size=(N, Cn)).astype(np.float32)
+    Wc, ws = orc.quantize(W, 8, True, orc.maxabs(W))
+    y_ref = A.astype(np.float64) @ (Wc.astype(np.float64) * ws).T
+    S = orc.num_splits(Cn, 0.02)
+
+    def err(Y):
+        return float(np.mean((Y.astype(np.float64) - y_ref) ** 2))
+
+    ac0, as0 = orc.quantize(A, 6, False, orc.maxabs(A))
+    e_plain = err(orc.qlinear(ac0, False, as0, Wc, ws, np.arange(Cn, dtype=np.int32))[0])
+    e_batch = err(orc.act_ocs_linear(A, S, 6, False, Wc, ws)[0])
+    sel, counts, _ = orc.act_select(P, S, 0.99)
+    assert set(hot) <= set(sel.tolist())
+    Ap, idx = orc.act_split_static(A, sel)
+    acs, ass = orc.quantize(Ap, 6, False, orc.maxabs(Ap))
+    e_static = err(orc.qlinear(acs, False, ass, orc.dup_weight_columns(Wc, idx), ws,
+                               np.arange(Cn + S, dtype=np.int32))[0])
+    assert e_batch < 0.6 * e_plain
+    assert e_static < 0.6 * e_plain
+
+
 def test_greedy_is_monotone_and_targets_the_outlier():
     """Section 3.4 / 5.2: each split halves the current maximum's channel; the maximum never
     rises; with a unique largest outlier the first split strictly narrows the range."""
