@@ -1228,7 +1228,7 @@ rows_quant_narrow_kernel(const float* __restrict__ W, int O, int C, int R, long 
     src[e] = 0; dep[e] = 0;
     if (valid[e]) {
       const int ch = col / R, r = col - ch * R;
-      dep[e] = __ldg(depth + ch);
+      dep[e] = min(__ldg(depth + ch), kMaxHalvings);   // further halvings leave (signed) zero
       src[e] = (ch < C ? ch : __ldg(idx_map + ch)) * R + r;
     }
   }
