@@ -231,7 +231,8 @@ class Fc6Sweep:
     def e2e_buffers(self, host):
         """End-to-end steps: every step's inputs travel from pinned host memory and its outputs travel
         back.  The copy of step i+1's inputs runs on a second stream into a second pair of device
-        buffers while step i computes (one host-to-device copy of W and A per step)."""
+        buffers while step i computes (one host-to-device copy of W and A per step); step i's outputs travel
+        back on a third stream while step i+1 computes."""
         torch = self.torch
         self.hW = torch.from_numpy(host["W"]).pin_memory()
         self.hA = torch.from_numpy(host["A"]).pin_memory()
@@ -241,10 +242,16 @@ class Fc6Sweep:
         self.Ad = [self.A, torch.empty_like(self.A)]
         self.ready = [torch.cuda.Event(), torch.cuda.Event()]
         self.consumed = [torch.cuda.Event(), torch.cuda.Event()]
+        # the outputs are double-buffered too: step i's device-to-host copy runs on a third stream while step
+        # i+1 computes into the other set
+        self.out_stream = torch.cuda.Stream()
+        self.Yd = [self.Y, [torch.empty_like(y) for y in self.Y]]
+        self.done = [torch.cuda.Event(), torch.cuda.Event()]
+        self.copied = [torch.cuda.Event(), torch.cuda.Event()]
         self.k = 0
         self.slot_graphs = {} if self.graph_obj is None else {0: self.graph_obj}
         torch.cuda.current_stream().synchronize()
-        for e in self.consumed:
+        for e in self.consumed + self.copied:
             e.record()
         self._prefetch(0)
         return self.hW.numel() * 4 + self.hA.numel() * 4, sum(y.numel() * 4 for y in self.hY)
@@ -263,7 +270,8 @@ class Fc6Sweep:
         self._prefetch(1 - cur)                                   # next step's inputs, overlapping this step
         main = torch.cuda.current_stream()
         main.wait_event(self.ready[cur])
-        self.W, self.A = self.Wd[cur], self.Ad[cur]
+        main.wait_event(self.copied[cur])                          # this slot's outputs of two steps ago are home
+        self.W, self.A, self.Y = self.Wd[cur], self.Ad[cur], self.Yd[cur]
         if self.graph_obj is None:
             self.step()
         else:
@@ -271,8 +279,12 @@ class Fc6Sweep:
                 self.slot_graphs[cur] = self._capture()
             self.slot_graphs[cur].replay()
         self.consumed[cur].record(main)
-        for h, y in zip(self.hY, self.Y):
-            h.copy_(y, non_blocking=True)
+        self.done[cur].record(main)
+        with torch.cuda.stream(self.out_stream):
+            self.out_stream.wait_event(self.done[cur])
+            for h, y in zip(self.hY, self.Yd[cur]):
+                h.copy_(y, non_blocking=True)
+            self.copied[cur].record(self.out_stream)
         self.k += 1
 
     # the CPU checker on a bounded sample of the same step
