@@ -673,7 +673,9 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       const bool acc_vec = p.acc_out && ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) && (p.ldy % 4 == 0);
       float tile_max = 0.0f;
       const bool want_max = direct && p.max_bits != nullptr;
-      for (int c0 = half * kEpiCols; c0 < BN; c0 += 2 * kEpiCols) {
+      // a warp whose 32 rows are all padding (a short M tile) has nothing to write
+      const bool warp_has_rows = __any_sync(0xffffffffu, ri.out_row >= 0);
+      for (int c0 = half * kEpiCols; warp_has_rows && c0 < BN; c0 += 2 * kEpiCols) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
         uint32_t v[kEpiCols];

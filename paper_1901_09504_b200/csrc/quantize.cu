@@ -313,22 +313,33 @@ quantize_kernel(View v, const float* __restrict__ alpha_p, const double* __restr
 }
 
 // Small tensors without a clip search (the per-step activations of a recurrent network, a classifier's
-// input): one CTA finds max|x| and writes the codes in the same launch -- the second read hits the cache,
-// and a launch of latency is saved where latency is all there is.
+// input): one launch finds max|x| and writes the codes.  The launch is one thread-block cluster of eight CTAs:
+// each takes an eighth of the elements, the eight partial maxima are exchanged through distributed shared
+// memory (every CTA stores its maximum into every peer, then one cluster barrier), and each CTA quantizes
+// its own eighth -- the second read hits the cache, and a launch of latency is saved where latency is all
+// there is.
 constexpr long long kSmallQuantElems = 65536;
+constexpr int kSmallCluster = 8;
+constexpr int kSmallThreads = 512;
 
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(kSmallThreads)
 small_quantize_kernel(const float* __restrict__ T, int rows, int cols, long long ld_in, int L, int is_signed,
                       int8_t* __restrict__ codes, long long ld_codes, float* __restrict__ scale_out,
                       float* __restrict__ alpha_out, unsigned int* __restrict__ maxbits, int* dev_status) {
-  __shared__ float red[32];
-  __shared__ float s_alpha;
+  __shared__ float red[kSmallThreads / 32];
+  __shared__ float peer_max[kSmallCluster];
+  uint32_t crank, csize;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(csize));
   const int n = rows * cols;
+  const int per = (n + (int)csize - 1) / (int)csize;
+  const int i0 = (int)crank * per, i1 = min(n, i0 + per);
+  const bool dense = ld_in == cols;
   float m = 0.0f;
   bool bad = false;
-  for (int i = threadIdx.x; i < n; i += 1024) {
-    const int r = i / cols, c = i - r * cols;
-    const float x = T[r * ld_in + c];
+#pragma unroll 4
+  for (int i = i0 + threadIdx.x; i < i1; i += kSmallThreads) {
+    const float x = dense ? T[i] : T[(long long)(i / cols) * ld_in + (i % cols)];
     bad |= !is_finite(x);
     m = fmaxf(m, fabsf(x));
   }
@@ -336,23 +347,37 @@ small_quantize_kernel(const float* __restrict__ T, int rows, int cols, long long
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
   __syncthreads();
   if (threadIdx.x == 0) {
-    for (int w = 1; w < 32; ++w) m = fmaxf(m, red[w]);
-    s_alpha = m;
-    *maxbits = __float_as_uint(m);
+    for (int w = 1; w < kSmallThreads / 32; ++w) m = fmaxf(m, red[w]);
+    // this CTA's maximum into slot `crank` of every CTA of the cluster
+    const uint32_t local = (uint32_t)__cvta_generic_to_shared(&peer_max[crank]);
+    for (uint32_t dst = 0; dst < csize; ++dst) {
+      uint32_t remote;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(dst));
+      asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(m) : "memory");
+    }
   }
-  __syncthreads();
-  const float alpha = s_alpha;
+  // all stores of all CTAs are visible after the cluster barrier (release / acquire)
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+  float alpha = 0.0f;
+  for (uint32_t k = 0; k < csize; ++k) alpha = fmaxf(alpha, peer_max[k]);
   const bool zero = !(alpha > 0.0f);
   const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)L);
   const float inv = zero ? 0.0f : __fdiv_rn((float)L, alpha);
   const float lo = is_signed ? -(float)L : 0.0f, hi = (float)L;
-  if (threadIdx.x == 0) {
+  if (crank == 0 && threadIdx.x == 0) {
     *scale_out = step;
     if (alpha_out) *alpha_out = zero ? 0.0f : alpha;
+    *maxbits = __float_as_uint(alpha);
   }
-  for (int i = threadIdx.x; i < n; i += 1024) {
+  const bool dense_out = dense && ld_codes == cols;
+#pragma unroll 4
+  for (int i = i0 + threadIdx.x; i < i1; i += kSmallThreads) {
     const int r = i / cols, c = i - r * cols;
-    codes[r * ld_codes + c] = (int8_t)quant_code(T[r * ld_in + c], inv, lo, hi);
+    const float x = dense ? T[i] : T[(long long)r * ld_in + c];
+    const int8_t q = (int8_t)quant_code(x, inv, lo, hi);
+    if (dense_out) codes[i] = q;
+    else codes[(long long)r * ld_codes + c] = q;
   }
   if (bad) flag(dev_status, OCS_DEV_NONFINITE);
 }
@@ -430,9 +455,20 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   const int L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
 
   if (mode == OCS_CLIP_NONE && !max_abs_in && rows * cols <= kSmallQuantElems) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kSmallCluster, 1, 1);
+    cfg.blockDim = dim3(kSmallThreads, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kSmallCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
     LaunchScope ls("small_quantize_kernel", stream);
-    small_quantize_kernel<<<1, 1024, 0, stream>>>(T, (int)rows, (int)cols, ld_in, L, is_signed, codes, ld_codes, scale,
-                                                  alpha, w.maxbits, dev_status);
+    const int irows = (int)rows, icols = (int)cols;
+    const long long ldi = ld_in, ldc = ld_codes;
+    if (cudaLaunchKernelEx(&cfg, small_quantize_kernel, T, irows, icols, ldi, L, is_signed, codes, ldc, scale, alpha,
+                           w.maxbits, dev_status) != cudaSuccess)
+      return OCS_ERR_CUDA;
     return launch_status();
   }
   const float* maxp = max_abs_in;
