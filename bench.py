@@ -609,6 +609,7 @@ class ResNet50(NetWorkload):
 class Lstm(NetWorkload):
     name = "lstm"
     graph = True
+    fold = False
 
     def __init__(self):
         self.desc = ("configs[4]: 2-layer LSTM language model, hidden 650, vocabulary 33278, batch 20, sequence 35, "
@@ -638,8 +639,9 @@ class Lstm(NetWorkload):
         for l in range(2):
             for nm, bn in (("W_ih", "b_ih"), ("W_hh", "b_hh")):
                 layers[f"{nm}{l}"] = nets.prepare_layer(P[f"{nm}{l}"], P[f"{bn}{l}"], cfg["ratio"], cfg["w_bits"],
-                                                        dev_status=self.status)
-        layers["W_dec"] = nets.prepare_layer(P["W_dec"], P["b_dec"], cfg["ratio"], cfg["w_bits"], dev_status=self.status)
+                                                        dev_status=self.status, fold=self.fold)
+        layers["W_dec"] = nets.prepare_layer(P["W_dec"], P["b_dec"], cfg["ratio"], cfg["w_bits"], dev_status=self.status,
+                                             fold=self.fold)
         return nets.lstm_forward(cfg, layers, self.dev_in["tokens"], dev_status=self.status)
 
     def oracle_sample(self, orc, host):
@@ -652,6 +654,17 @@ class Lstm(NetWorkload):
         h = small["hidden"]
         S = configs_num_splits(h, 0.02)
         return sec, 2 * (h + S) * (6 * 4 * 4 * h * 4 + 6 * 4 * 3000)
+
+
+class LstmFolded(Lstm):
+    """The same model with the duplicated weight codes folded back into their source channels (6-bit codes:
+    the sums fit int8): no gather in any GEMM, identical outputs."""
+    name = "lstm-folded"
+    fold = True
+
+    def __init__(self):
+        super().__init__()
+        self.desc = self.desc.replace("configs[4]:", "configs[4] with ocs_fold_duplicates after the quantization:")
 
 
 class Conv3x3(NetWorkload):
@@ -771,7 +784,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm", "act-ocs"])
+    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm", "lstm-folded", "act-ocs"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -781,7 +794,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     wl = {"fc6": Fc6Sweep, "fc6-fused": Fc6Fused, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc, "conv": Conv3x3,
-          "resnet50": ResNet50, "lstm": Lstm, "act-ocs": ActOcs}[args.workload]()
+          "resnet50": ResNet50, "lstm": Lstm, "lstm-folded": LstmFolded, "act-ocs": ActOcs}[args.workload]()
     net = getattr(wl, "kind", "") == "net"
 
     if args.impl == "reference":

@@ -31,7 +31,8 @@ class QLayer:
 
 
 def prepare_layer(W, bias, ratio: float, bits: int, clip_mode: int = B.CLIP_NONE, qa_bits: int = 0, conv: bool = False,
-                  stride: int = 1, pad: int = 0, n_candidates: int = 128, n_bins: int = 2048, dev_status=None) -> QLayer:
+                  stride: int = 1, pad: int = 0, n_candidates: int = 128, n_bins: int = 2048, dev_status=None,
+                  fold: bool = False) -> QLayer:
     """W fp32 [O, C] or [O, C, k, k] on the device -> QLayer (ocs_split_quantize, or ocs_split + ocs_quantize where
     the fused call cannot stage the rows; ocs_pack_conv_weights)."""
     O, Cn = W.shape[0], W.shape[1]
@@ -51,6 +52,13 @@ def prepare_layer(W, bias, ratio: float, bits: int, clip_mode: int = B.CLIP_NONE
         W_out, idx_map, _, mx = B.ocs_split(W.contiguous(), S, qa_bits=qa_bits, dev_status=dev_status, want_order=False)
         codes, scale, _ = B.ocs_quantize(W_out, bits, True, clip_mode, n_candidates, n_bins, cols=(Cn + S) * R,
                                          max_abs_in=mx[1:2], dev_status=dev_status)
+    if fold and S > 0:
+        # k <= 7-bit codes: the copies are summed back into their source channel (ocs_fold_duplicates); the
+        # layer then runs on C plain channels with the same accumulators.  (A sum that leaves int8 sets
+        # OCS_DEV_OVERFLOW in dev_status.)
+        codes = B.ocs_fold_duplicates(codes, Cn, S, idx_map, R=R, dev_status=dev_status)
+        idx_map = idx_map[:Cn].contiguous()
+        S = 0
     if conv:
         codes = B.ocs_pack_conv_weights(codes, O, Cn, S, k, k)
     return QLayer(codes, scale, idx_map, bias, Cn, O, S, k, stride, pad)
@@ -131,7 +139,7 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
 
 
 # ------------------------------------------------------------------------------------------ LSTM
-def prepare_lstm(cfg, device, dev_status=None):
+def prepare_lstm(cfg, device, dev_status=None, fold: bool = False):
     """cfg from ocs_inputs.configs.config5 -> dict of QLayers and the embedding table."""
     p = cfg["params"]
     mode = B.CLIP_MSE if cfg["clip"] == "mse" else B.CLIP_NONE
@@ -140,9 +148,9 @@ def prepare_lstm(cfg, device, dev_status=None):
         for nm, bn in (("W_ih", "b_ih"), ("W_hh", "b_hh")):
             out[f"{nm}{layer}"] = prepare_layer(torch.from_numpy(p[f"{nm}{layer}"]).to(device),
                                                 torch.from_numpy(p[f"{bn}{layer}"]).to(device), cfg["ratio"],
-                                                cfg["w_bits"], mode, dev_status=dev_status)
+                                                cfg["w_bits"], mode, dev_status=dev_status, fold=fold)
     out["W_dec"] = prepare_layer(torch.from_numpy(p["W_dec"]).to(device), torch.from_numpy(p["b_dec"]).to(device),
-                                 cfg["ratio"], cfg["w_bits"], mode, dev_status=dev_status)
+                                 cfg["ratio"], cfg["w_bits"], mode, dev_status=dev_status, fold=fold)
     return out
 
 

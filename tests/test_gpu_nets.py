@@ -86,3 +86,16 @@ def test_lstm_language_model_reduced_end_to_end():
         np.testing.assert_array_equal(host(t["c"][l]), ref["c"][l])
     np.testing.assert_allclose(host(logits), ref_logits, rtol=1e-5, atol=0)
     np.testing.assert_array_equal(host(logits), ref_logits)
+
+
+def test_lstm_with_folded_duplicates_gives_the_same_logits():
+    """6-bit codes: the copies folded back into their source channels, no gather in any GEMM, same outputs."""
+    cfg = configs.config5(vocab=3000, batch=4, seq=6)
+    ref_logits, ref = net_oracle.lstm(cfg)
+    st = ocs.new_status()
+    layers = nets.prepare_lstm(cfg, torch.device("cuda"), dev_status=st, fold=True)
+    assert all(L.S == 0 for name, L in layers.items() if name != "emb")
+    logits, t = nets.lstm_forward(cfg, layers, dev(cfg["tokens"]), keep=True, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    np.testing.assert_array_equal(host(t["tops"]), ref["tops"])
+    np.testing.assert_array_equal(host(logits), ref_logits)
