@@ -581,18 +581,33 @@ class ResNet50(NetWorkload):
             self.ops += 2 * self.batch * spec.H_out ** 2 * spec.O * (spec.C + S) * spec.k ** 2
         fc = self.cfg["fc"]
         self.ops += 2 * self.batch * fc.O * (fc.C + configs_num_splits(fc.C, self.cfg["ratio"]))
+        self.prep_streams = [torch.cuda.Stream() for _ in range(8)]
+        self.ev_start = torch.cuda.Event()
+        self.ev_done = [torch.cuda.Event() for _ in self.prep_streams]
 
     def step(self):
-        nets, cfg = self.nets, self.cfg
+        """The 54 layers are prepared independently of one another: their small, latency-bound kernels (a single
+        CTA for the split plan) are spread over a few streams so that they run side by side; the forward pass
+        starts when all of them are done."""
+        nets, cfg, torch = self.nets, self.cfg, self.torch
+        main = torch.cuda.current_stream()
+        self.ev_start.record(main)
         layers = {}
-        for spec in cfg["layers"] + [cfg["fc"]]:
+        for i, spec in enumerate(cfg["layers"] + [cfg["fc"]]):
             W, b = self.Wd[spec.name]
-            if spec.name == "fc":
-                layers["fc"] = nets.prepare_layer(W.reshape(spec.O, spec.C), b, cfg["ratio"], cfg["w_bits"],
-                                                  dev_status=self.status)
-            else:
-                layers[spec.name] = nets.prepare_layer(W, b, cfg["ratio"], cfg["w_bits"], conv=True, stride=spec.stride,
-                                                       pad=spec.pad, dev_status=self.status)
+            side = self.prep_streams[i % len(self.prep_streams)]
+            with torch.cuda.stream(side):
+                if i < len(self.prep_streams):
+                    side.wait_event(self.ev_start)      # after everything the caller's stream has queued so far
+                if spec.name == "fc":
+                    layers["fc"] = nets.prepare_layer(W.reshape(spec.O, spec.C), b, cfg["ratio"], cfg["w_bits"],
+                                                      dev_status=self.status)
+                else:
+                    layers[spec.name] = nets.prepare_layer(W, b, cfg["ratio"], cfg["w_bits"], conv=True,
+                                                           stride=spec.stride, pad=spec.pad, dev_status=self.status)
+        for side, ev in zip(self.prep_streams, self.ev_done):
+            ev.record(side)
+            main.wait_event(ev)
         return nets.resnet50_forward(cfg, layers, self.dev_in["X"], dev_status=self.status)
 
     def oracle_sample(self, orc, host):
