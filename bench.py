@@ -647,17 +647,30 @@ class Lstm(NetWorkload):
         seq, batch = self.cfg["tokens"].shape
         S = configs_num_splits(h, self.cfg["ratio"])
         self.ops = 2 * (h + S) * (seq * batch * 4 * h * 4 + seq * batch * V)
+        self.prep_streams = [torch.cuda.Stream() for _ in range(5)]
+        self.ev_start = torch.cuda.Event()
+        self.ev_done = [torch.cuda.Event() for _ in self.prep_streams]
 
     def step(self):
-        nets, cfg, P = self.nets, self.cfg, self.Pd
+        """The five weight matrices are prepared side by side on their own streams; the decoder's (the largest)
+        keeps going beside the time steps and is waited for right before the decoder layer."""
+        nets, cfg, P, torch = self.nets, self.cfg, self.Pd, self.torch
+        main = torch.cuda.current_stream()
+        self.ev_start.record(main)
         layers = {"emb": P["emb"]}
-        for l in range(2):
-            for nm, bn in (("W_ih", "b_ih"), ("W_hh", "b_hh")):
-                layers[f"{nm}{l}"] = nets.prepare_layer(P[f"{nm}{l}"], P[f"{bn}{l}"], cfg["ratio"], cfg["w_bits"],
-                                                        dev_status=self.status, fold=self.fold)
-        layers["W_dec"] = nets.prepare_layer(P["W_dec"], P["b_dec"], cfg["ratio"], cfg["w_bits"], dev_status=self.status,
-                                             fold=self.fold)
-        return nets.lstm_forward(cfg, layers, self.dev_in["tokens"], dev_status=self.status)
+        names = [(f"{nm}{l}", f"{bn}{l}") for l in range(2) for nm, bn in (("W_ih", "b_ih"), ("W_hh", "b_hh"))]
+        names.append(("W_dec", "b_dec"))
+        for i, (wn, bname) in enumerate(names):
+            side = self.prep_streams[i]
+            with torch.cuda.stream(side):
+                side.wait_event(self.ev_start)
+                layers[wn] = nets.prepare_layer(P[wn], P[bname], cfg["ratio"], cfg["w_bits"], dev_status=self.status,
+                                                fold=self.fold)
+                self.ev_done[i].record(side)
+        for i in range(4):
+            main.wait_event(self.ev_done[i])
+        return nets.lstm_forward(cfg, layers, self.dev_in["tokens"], dev_status=self.status,
+                                 before_decoder=lambda: main.wait_event(self.ev_done[4]))
 
     def oracle_sample(self, orc, host):
         sys.path.insert(0, os.path.join(ROOT, "tests"))

@@ -154,8 +154,10 @@ def prepare_lstm(cfg, device, dev_status=None, fold: bool = False):
     return out
 
 
-def lstm_forward(cfg, layers, tokens, a_bits: int = 8, keep: bool = False, dev_status=None):
-    """tokens int32 [seq, batch] on the device -> logits fp32 [seq * batch, vocab] (h0 = c0 = 0)."""
+def lstm_forward(cfg, layers, tokens, a_bits: int = 8, keep: bool = False, dev_status=None, before_decoder=None):
+    """tokens int32 [seq, batch] on the device -> logits fp32 [seq * batch, vocab] (h0 = c0 = 0).
+    before_decoder: called right before the decoder layer (a caller that prepares the decoder's weights on
+    another stream while the time steps run makes its stream wait there)."""
     seq, batch = tokens.shape
     hidden = cfg["hidden"]
     dev = tokens.device
@@ -172,6 +174,8 @@ def lstm_forward(cfg, layers, tokens, a_bits: int = 8, keep: bool = False, dev_s
             B.ocs_lstm_cell(g_ih, g_hh, c[l], hn)
             h[l] = hn
             x = hn
+    if before_decoder is not None:
+        before_decoder()
     logits = linear_forward(layers["W_dec"], tops.view(seq * batch, hidden), True, a_bits, dev_status)
     return (logits, dict(emb=emb, tops=tops, c=c)) if keep else logits
 
