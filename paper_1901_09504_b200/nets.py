@@ -139,6 +139,17 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
 
 
 # ------------------------------------------------------------------------------------------ LSTM
+_SIDE_STREAMS = {}
+
+
+def _side_stream(device):
+    """One helper stream per device, created on first use."""
+    key = torch.device(device).index if torch.device(device).index is not None else torch.cuda.current_device()
+    if key not in _SIDE_STREAMS:
+        _SIDE_STREAMS[key] = torch.cuda.Stream(device=key)
+    return _SIDE_STREAMS[key]
+
+
 def prepare_lstm(cfg, device, dev_status=None, fold: bool = False):
     """cfg from ocs_inputs.configs.config5 -> dict of QLayers and the embedding table."""
     p = cfg["params"]
@@ -165,11 +176,21 @@ def lstm_forward(cfg, layers, tokens, a_bits: int = 8, keep: bool = False, dev_s
     h = [torch.zeros((batch, hidden), dtype=torch.float32, device=dev) for _ in range(2)]
     c = [torch.zeros((batch, hidden), dtype=torch.float32, device=dev) for _ in range(2)]
     tops = torch.empty((seq, batch, hidden), dtype=torch.float32, device=dev)
+    # The two gate GEMMs of a cell are independent: the hidden-to-hidden one runs on a second stream beside the
+    # input-to-hidden one (each a latency-bound chain of quantize + GEMM), and the cell waits for both.
+    main = torch.cuda.current_stream()
+    side = _side_stream(dev)
+    ev_in, ev_hh = torch.cuda.Event(), torch.cuda.Event()
     for t in range(seq):
         x = emb[t]
         for l in range(2):
+            ev_in.record(main)                       # x and h[l] are complete
+            with torch.cuda.stream(side):
+                side.wait_event(ev_in)
+                g_hh = linear_forward(layers[f"W_hh{l}"], h[l], True, a_bits, dev_status)
+                ev_hh.record(side)
             g_ih = linear_forward(layers[f"W_ih{l}"], x, True, a_bits, dev_status)
-            g_hh = linear_forward(layers[f"W_hh{l}"], h[l], True, a_bits, dev_status)
+            main.wait_event(ev_hh)
             hn = tops[t] if l == 1 else torch.empty_like(h[l])
             B.ocs_lstm_cell(g_ih, g_hh, c[l], hn)
             h[l] = hn
