@@ -142,11 +142,12 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
 _SIDE_STREAMS = {}
 
 
-def _side_stream(device):
-    """One helper stream per device, created on first use."""
-    key = torch.device(device).index if torch.device(device).index is not None else torch.cuda.current_device()
+def _side_stream(device, which: int = 0):
+    """Helper streams per device, created on first use."""
+    idx = torch.device(device).index if torch.device(device).index is not None else torch.cuda.current_device()
+    key = (idx, which)
     if key not in _SIDE_STREAMS:
-        _SIDE_STREAMS[key] = torch.cuda.Stream(device=key)
+        _SIDE_STREAMS[key] = torch.cuda.Stream(device=idx)
     return _SIDE_STREAMS[key]
 
 
@@ -173,28 +174,45 @@ def lstm_forward(cfg, layers, tokens, a_bits: int = 8, keep: bool = False, dev_s
     hidden = cfg["hidden"]
     dev = tokens.device
     emb = B.ocs_embedding(layers["emb"], tokens.contiguous(), dev_status=dev_status)
-    h = [torch.zeros((batch, hidden), dtype=torch.float32, device=dev) for _ in range(2)]
+    zero_h = torch.zeros((batch, hidden), dtype=torch.float32, device=dev)
     c = [torch.zeros((batch, hidden), dtype=torch.float32, device=dev) for _ in range(2)]
-    tops = torch.empty((seq, batch, hidden), dtype=torch.float32, device=dev)
-    # The two gate GEMMs of a cell are independent: the hidden-to-hidden one runs on a second stream beside the
-    # input-to-hidden one (each a latency-bound chain of quantize + GEMM), and the cell waits for both.
+    # hidden states of every step, preallocated (no buffer is recycled while another stream may still read it)
+    hs = [torch.empty((seq, batch, hidden), dtype=torch.float32, device=dev) for _ in range(2)]
+    tops = hs[1]
+    # Two kinds of concurrency, both plain stream forks and joins.  (1) The two gate GEMMs of a cell are
+    # independent: the hidden-to-hidden one runs on a helper stream beside the input-to-hidden one (each a
+    # latency-bound chain of quantize + GEMM), and the cell waits for both.  (2) Layer 1 of step t only needs
+    # layer 0's output of step t, so it runs on its own stream while layer 0 goes on with step t + 1.
     main = torch.cuda.current_stream()
-    side = _side_stream(dev)
-    ev_in, ev_hh = torch.cuda.Event(), torch.cuda.Event()
+    lay = [main, _side_stream(dev, 0)]
+    helper = [_side_stream(dev, 1), _side_stream(dev, 2)]
+    ev_start = torch.cuda.Event()
+    ev_start.record(main)
+    for st in (lay[1], helper[0], helper[1]):
+        st.wait_event(ev_start)                      # emb, the zero states and the layers' weights are complete
+    ev_in = [torch.cuda.Event(), torch.cuda.Event()]
+    ev_hh = [torch.cuda.Event(), torch.cuda.Event()]
+    ev_h0 = [torch.cuda.Event() for _ in range(seq)]
     for t in range(seq):
-        x = emb[t]
         for l in range(2):
-            ev_in.record(main)                       # x and h[l] are complete
-            with torch.cuda.stream(side):
-                side.wait_event(ev_in)
-                g_hh = linear_forward(layers[f"W_hh{l}"], h[l], True, a_bits, dev_status)
-                ev_hh.record(side)
-            g_ih = linear_forward(layers[f"W_ih{l}"], x, True, a_bits, dev_status)
-            main.wait_event(ev_hh)
-            hn = tops[t] if l == 1 else torch.empty_like(h[l])
-            B.ocs_lstm_cell(g_ih, g_hh, c[l], hn)
-            h[l] = hn
-            x = hn
+            with torch.cuda.stream(lay[l]):
+                if l == 1:
+                    lay[1].wait_event(ev_h0[t])      # layer 0's output of this step
+                x = emb[t] if l == 0 else hs[0][t]
+                h_prev = zero_h if t == 0 else hs[l][t - 1]
+                ev_in[l].record(lay[l])              # h_prev is complete on this layer's stream
+                with torch.cuda.stream(helper[l]):
+                    helper[l].wait_event(ev_in[l])
+                    g_hh = linear_forward(layers[f"W_hh{l}"], h_prev, True, a_bits, dev_status)
+                    ev_hh[l].record(helper[l])
+                g_ih = linear_forward(layers[f"W_ih{l}"], x, True, a_bits, dev_status)
+                lay[l].wait_event(ev_hh[l])
+                B.ocs_lstm_cell(g_ih, g_hh, c[l], hs[l][t])
+                if l == 0:
+                    ev_h0[t].record(lay[0])
+    ev_end = torch.cuda.Event()
+    ev_end.record(lay[1])
+    main.wait_event(ev_end)
     if before_decoder is not None:
         before_decoder()
     logits = linear_forward(layers["W_dec"], tops.view(seq * batch, hidden), True, a_bits, dev_status)
