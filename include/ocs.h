@@ -7,7 +7,8 @@
  *  - Every pointer is a DEVICE pointer owned by the caller unless it is marked "host".
  *    The library allocates nothing; scratch memory comes in through (ws, ws_bytes), whose
  *    minimum size the matching *_workspace_bytes() query returns (host call, no GPU work).
- *    ws must be 256-byte aligned.  Inputs are never modified; outputs must not alias inputs.
+ *    ws must be 256-byte aligned.  Inputs are never modified and outputs must not alias inputs,
+ *    unless an entry says otherwise (ocs_dup_weight_columns and ocs_add_relu work in place).
  *  - Every call only enqueues work on `stream` (a cudaStream_t passed as void*) and returns
  *    without synchronising.  Scalar results (scales, thresholds, maxima) are written to
  *    device memory.
