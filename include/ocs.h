@@ -261,16 +261,17 @@ void ocs_quantize_workspace_views(void* ws, int n_bins, int n_candidates, uint64
  * row stride ldw bytes, ldw a multiple of 16 and Wc 16-byte aligned; a_scale / w_scale
  * device scalars; Y fp32 [M][N] row stride ldy floats; acc_out (nullable) int32 [M][N] with
  * the same stride.  Limits: (C+S) * 255 * 127 must fit int32.
- * Two steps that usually follow a layer can be taken in its epilogue: relu != 0 stores
- * max(Y, 0) instead of Y, and max_abs_out (device, fp32 [1], may be NULL) receives max |Y| of
+ * Steps that usually follow a layer can be taken in its epilogue: residual (device, fp32, the
+ * shape and row stride of Y, may be NULL) is added to Y with one rounded addition (a block's
+ * shortcut connection; it may not alias Y), relu != 0 then stores max(., 0), and max_abs_out (device, fp32 [1], may be NULL) receives max |Y| of
  * the stored output -- the next layer's activation grid (ocs_quantize's max_abs_in).
  * Device flags: BAD_INDEX, TIMEOUT. */
 size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S);
 ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C,
                        int64_t lda, const int8_t* W_codes, const float* w_scale, int N, int S,
                        int64_t ldw, const int32_t* idx_map, const float* bias, float* Y,
-                       int64_t ldy, int32_t* acc_out, int relu, float* max_abs_out, void* ws,
-                       size_t ws_bytes, int* dev_status, void* stream);
+                       int64_t ldy, int32_t* acc_out, const float* residual, int relu,
+                       float* max_abs_out, void* ws, size_t ws_bytes, int* dev_status, void* stream);
 
 /* ocs_pack_conv_weights -------------------------------------------------------------------
  * Reorders quantized conv weights from the split's layout [O][C+S][kh*kw] (row stride
@@ -293,7 +294,7 @@ ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, int S, int k
  * with zeros outside the image, and the same fp32 epilogue.  X codes NHWC [Nb][H][Wd][C]
  * (dense, 16-byte aligned when C is a multiple of 16); W_packed from ocs_pack_conv_weights with row
  * stride ldw bytes; Y fp32 NHWC [Nb][Ho][Wo][O] dense; acc_out (nullable) int32, same shape.
- * relu and max_abs_out as in ocs_qlinear.  A layer whose pixels TMA cannot address (C not a
+ * residual, relu and max_abs_out as in ocs_qlinear.  A layer whose pixels TMA cannot address (C not a
  * multiple of 16 bytes) is run over its patch matrix, which is built in the workspace.
  * Device flags: BAD_INDEX, TIMEOUT. */
 size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O, int S, int kh, int kw,
@@ -301,8 +302,8 @@ size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O, int S, int
 ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H,
                      int Wd, int C, const int8_t* W_packed, const float* w_scale, int O, int S,
                      int kh, int kw, int stride, int pad, int64_t ldw, const int32_t* idx_map,
-                     const float* bias, float* Y, int32_t* acc_out, int relu, float* max_abs_out,
-                     void* ws, size_t ws_bytes, int* dev_status, void* stream);
+                     const float* bias, float* Y, int32_t* acc_out, const float* residual, int relu,
+                     float* max_abs_out, void* ws, size_t ws_bytes, int* dev_status, void* stream);
 
 /* Steps between quantized layers ------------------------------------------------------------
  * The paper runs whole networks through the split and quantized layers (Section 5: ImageNet

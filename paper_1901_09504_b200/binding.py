@@ -194,7 +194,7 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
 
 
 def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, bias=None, want_acc: bool = False,
-                dev_status=None, out=None, ws=None, relu: bool = False, max_out=None):
+                dev_status=None, out=None, ws=None, relu: bool = False, max_out=None, residual=None):
     """A_codes uint8/int8 [M, lda>=C]; W_codes int8 [N, ldw>=C+S].  Returns Y fp32 [M, N] (and acc int32)."""
     assert A_codes.is_cuda and A_codes.dim() == 2 and A_codes.stride(1) == 1
     assert W_codes.dtype == torch.int8 and W_codes.dim() == 2 and W_codes.stride(1) == 1
@@ -208,7 +208,7 @@ def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, 
         ws = _ws(nws, A_codes.device)
     st = lib().ocs_qlinear(_ptr(A_codes), a_signed, _ptr(a_scale), M, int(C_in), C.c_int64(A_codes.stride(0)),
                            _ptr(W_codes), _ptr(w_scale), N, int(S), C.c_int64(W_codes.stride(0)), _ptr(idx_map),
-                           _ptr(bias), _ptr(Y), C.c_int64(N), _ptr(acc), int(bool(relu)), _ptr(max_out), _ptr(ws),
+                           _ptr(bias), _ptr(Y), C.c_int64(N), _ptr(acc), _ptr(residual), int(bool(relu)), _ptr(max_out), _ptr(ws),
                            C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
     _check(st, "ocs_qlinear")
     return (Y, acc) if want_acc else Y
@@ -235,7 +235,8 @@ def ocs_pack_conv_weights(codes, O: int, C_in: int, S: int, kh: int, kw: int, ld
 
 
 def ocs_qconv(X_codes, a_scale, W_packed, w_scale, idx_map, S: int, kh: int, kw: int, stride: int, pad: int,
-              bias=None, want_acc: bool = False, dev_status=None, out=None, ws=None, relu: bool = False, max_out=None):
+              bias=None, want_acc: bool = False, dev_status=None, out=None, ws=None, relu: bool = False, max_out=None,
+              residual=None):
     """X_codes uint8/int8 NHWC [Nb, H, W, C] contiguous; W_packed from ocs_pack_conv_weights.
     Returns Y fp32 NHWC [Nb, Ho, Wo, O] (and acc int32)."""
     assert X_codes.is_cuda and X_codes.dim() == 4 and X_codes.is_contiguous()
@@ -251,7 +252,7 @@ def ocs_qconv(X_codes, a_scale, W_packed, w_scale, idx_map, S: int, kh: int, kw:
         ws = _ws(nws, X_codes.device)
     st = lib().ocs_qconv(_ptr(X_codes), a_signed, _ptr(a_scale), Nb, H, Wd, Cn, _ptr(W_packed), _ptr(w_scale), O,
                          int(S), kh, kw, stride, pad, C.c_int64(W_packed.stride(0)), _ptr(idx_map), _ptr(bias),
-                         _ptr(Y), _ptr(acc), int(bool(relu)), _ptr(max_out), _ptr(ws), C.c_size_t(ws.numel()),
+                         _ptr(Y), _ptr(acc), _ptr(residual), int(bool(relu)), _ptr(max_out), _ptr(ws), C.c_size_t(ws.numel()),
                          _ptr(dev_status), _stream())
     _check(st, "ocs_qconv")
     return (Y, acc) if want_acc else Y

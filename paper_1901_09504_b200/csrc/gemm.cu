@@ -75,6 +75,7 @@ struct GemmParams {
   float* Y;
   long long ldy;
   int32_t* acc_out;
+  const float* residual;        // optional fp32 tensor of Y's shape and stride, added before the ReLU
   int relu;                     // max(., 0) applied to Y
   unsigned int* max_bits;       // fp32 bits of max |Y| over the whole output (optional)
   int32_t* acc_ws;              // [split_k][rows][N] partial sums when split_k > 1
@@ -650,10 +651,17 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     bool ok = true;
     for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
       const int acc = j & 1;
-      if (!mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag)) { ok = false; break; }
-      tc_fence_after();
       const RowInfo ri = row_info(p, w.mt, q * 32 + lane);
       const int nt = w.nt, kz = w.kz;
+      if (p.residual && direct && ri.out_row >= 0) {
+        // the shortcut tensor's part of this tile is asked into L2 while the main loop still runs
+        const float* rrow = p.residual + ri.out_row * p.ldy + (long long)nt * BN;
+        const int n_left = p.N - nt * BN;
+        for (int c = (warp >= 10 ? 32 : 0); c < BN && c < n_left; c += 64)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(rrow + c));
+      }
+      if (!mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
       // Each lane holds one row of a 32 x 16 piece of the accumulator; written out that way a store
       // instruction would touch 32 rows with 16 bytes each.  The piece goes through shared memory instead, so
       // that four neighbouring lanes write 64 contiguous bytes of one row (lane -> row i*8 + (qd&1)*4 + qd/2
@@ -710,6 +718,18 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           for (int i = 0; i < 4; ++i) {
             float f0 = fmaf(int_to_float_rn((int)a[i].x), sc, b4[0]), f1 = fmaf(int_to_float_rn((int)a[i].y), sc, b4[1]);
             float f2 = fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]), f3 = fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]);
+            if (p.residual && orow[i] >= 0) {   // the block's shortcut: one more rounded addition per output
+              const float* rr = p.residual + orow[i] * p.ldy + n0 + cq;
+              if (vec0) {
+                const float4 r4 = __ldcs(reinterpret_cast<const float4*>(rr));
+                f0 = __fadd_rn(f0, r4.x); f1 = __fadd_rn(f1, r4.y); f2 = __fadd_rn(f2, r4.z); f3 = __fadd_rn(f3, r4.w);
+              } else {
+                if (n0 + cq + 0 < p.N) f0 = __fadd_rn(f0, rr[0]);
+                if (n0 + cq + 1 < p.N) f1 = __fadd_rn(f1, rr[1]);
+                if (n0 + cq + 2 < p.N) f2 = __fadd_rn(f2, rr[2]);
+                if (n0 + cq + 3 < p.N) f3 = __fadd_rn(f3, rr[3]);
+              }
+            }
             if (p.relu) {
               f0 = f0 > 0.0f ? f0 : 0.0f; f1 = f1 > 0.0f ? f1 : 0.0f;
               f2 = f2 > 0.0f ? f2 : 0.0f; f3 = f3 > 0.0f ? f3 : 0.0f;
@@ -791,7 +811,7 @@ __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long rows, int N,
                      const float* __restrict__ a_scale, const float* __restrict__ w_scale,
                      const float* __restrict__ bias, float* __restrict__ Y, long long ldy, int32_t* __restrict__ acc_out,
-                     int relu, unsigned int* __restrict__ max_bits) {
+                     const float* __restrict__ residual, int relu, unsigned int* __restrict__ max_bits) {
   float m = 0.0f;
   const float sc = __fmul_rn(__ldg(a_scale), __ldg(w_scale));
   const long long slice = rows * (long long)N;
@@ -813,6 +833,7 @@ splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long ro
                     fmaf((float)a.z, sc, bias ? __ldg(bias + n + 2) : 0.0f), fmaf((float)a.w, sc, bias ? __ldg(bias + n + 3) : 0.0f)};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
+        if (residual) f[e] = __fadd_rn(f[e], residual[row * ldy + n + e]);
         if (relu) f[e] = f[e] > 0.0f ? f[e] : 0.0f;
         m = fmaxf(m, fabsf(f[e]));
         y[e] = f[e];
@@ -825,6 +846,7 @@ splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long ro
       int a = __ldcg(p);
       for (int z = 1; z < split_k; ++z) a += __ldcg(p + z * slice);
       float f = fmaf((float)a, sc, bias ? __ldg(bias + n) : 0.0f);
+      if (residual) f = __fadd_rn(f, residual[row * ldy + n]);
       if (relu) f = f > 0.0f ? f : 0.0f;
       m = fmaxf(m, fabsf(f));
       Y[row * ldy + n] = f;
@@ -1020,10 +1042,10 @@ ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long lo
   LaunchScope ls("splitk_reduce_kernel", stream);
   if (vec)
     splitk_reduce_kernel<true><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
-                                                         p.bias, p.Y, p.ldy, p.acc_out, p.relu, p.max_bits);
+                                                         p.bias, p.Y, p.ldy, p.acc_out, p.residual, p.relu, p.max_bits);
   else
     splitk_reduce_kernel<false><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
-                                                          p.bias, p.Y, p.ldy, p.acc_out, p.relu, p.max_bits);
+                                                          p.bias, p.Y, p.ldy, p.acc_out, p.residual, p.relu, p.max_bits);
   return launch_status();
 }
 
@@ -1166,8 +1188,8 @@ extern "C" size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S) {
 extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C, int64_t lda,
                                   const int8_t* W_codes, const float* w_scale, int N, int S, int64_t ldw,
                                   const int32_t* idx_map, const float* bias, float* Y, int64_t ldy, int32_t* acc_out,
-                                  int relu, float* max_abs_out, void* ws, size_t ws_bytes, int* dev_status,
-                                  void* stream_) {
+                                  const float* residual, int relu, float* max_abs_out, void* ws, size_t ws_bytes,
+                                  int* dev_status, void* stream_) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!A_codes || !a_scale || !W_codes || !w_scale || !idx_map || !Y) return OCS_ERR_INVALID_ARG;
   if (S < 0) return OCS_ERR_INVALID_ARG;
@@ -1188,6 +1210,7 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
   p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = ldy; p.acc_out = acc_out;
   p.dev_status = dev_status;
   p.relu = relu ? 1 : 0;
+  p.residual = residual;
   p.max_bits = reinterpret_cast<unsigned int*>(max_abs_out);
   if (max_abs_out && cudaMemsetAsync(max_abs_out, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
   const int m_tiles = (M + BM - 1) / BM;
@@ -1275,8 +1298,8 @@ extern "C" size_t ocs_qconv_workspace_bytes(int Nb, int H, int Wd, int C, int O,
 extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* a_scale, int Nb, int H, int Wd, int C,
                                 const int8_t* W_packed, const float* w_scale, int O, int S, int kh, int kw, int stride,
                                 int pad, int64_t ldw, const int32_t* idx_map, const float* bias, float* Y,
-                                int32_t* acc_out, int relu, float* max_abs_out, void* ws, size_t ws_bytes,
-                                int* dev_status, void* stream_) {
+                                int32_t* acc_out, const float* residual, int relu, float* max_abs_out, void* ws,
+                                size_t ws_bytes, int* dev_status, void* stream_) {
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!X_codes || !a_scale || !W_packed || !w_scale || !idx_map || !Y) return OCS_ERR_INVALID_ARG;
   if (S < 0) return OCS_ERR_INVALID_ARG;
@@ -1304,6 +1327,7 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   p.a_scale = a_scale; p.w_scale = w_scale; p.bias = bias; p.Y = Y; p.ldy = O; p.acc_out = acc_out;
   p.dev_status = dev_status;
   p.relu = relu ? 1 : 0;
+  p.residual = residual;
   p.max_bits = reinterpret_cast<unsigned int*>(max_abs_out);
   if (max_abs_out && cudaMemsetAsync(max_abs_out, 0, 4, stream) != cudaSuccess) return OCS_ERR_CUDA;
 

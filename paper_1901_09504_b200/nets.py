@@ -74,12 +74,12 @@ def quantize_activations(x, signed: bool, bits: int = 8, dev_status=None, max_ab
 
 
 def conv_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None, max_abs=None, relu: bool = False,
-                 max_out=None):
-    """x fp32 NHWC -> fp32 NHWC (activation quantization + ocs_qconv; ReLU and max |y| in the layer's epilogue
-    on request)."""
+                 max_out=None, residual=None):
+    """x fp32 NHWC -> fp32 NHWC (activation quantization + ocs_qconv; the shortcut addition, ReLU and max |y|
+    in the layer's epilogue on request)."""
     xc, xs = quantize_activations(x, a_signed, a_bits, dev_status, max_abs)
     return B.ocs_qconv(xc, xs, L.codes, L.w_scale, L.idx_map, L.S, L.k, L.k, L.stride, L.pad, bias=L.bias,
-                       dev_status=dev_status, relu=relu, max_out=max_out)
+                       dev_status=dev_status, relu=relu, max_out=max_out, residual=residual)
 
 
 def linear_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None):
@@ -111,13 +111,16 @@ def prepare_resnet50(cfg, device, dev_status=None):
 def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, dev_status=None):
     """X fp32 NCHW on the device -> logits fp32 [Nb, 1000]; with keep, also every named tensor."""
     t = {}
-    mx = {}     # max |tensor| of the tensors ocs_add_relu produced (it takes the maximum while it writes them)
+    mx = {}     # max |tensor| of the tensors whose producing layer took it in its epilogue
     x = B.ocs_nchw_to_nhwc(X_nchw.contiguous())
     first = True
     for spec in cfg["layers"]:
         src = t[spec.input_from] if spec.input_from else x
         m = torch.empty(1, dtype=torch.float32, device=x.device)
-        fused_relu = spec.relu and not spec.residual_from      # ReLU straight after the layer: in its epilogue
+        # A ReLU straight after the layer is taken in its epilogue, with the maximum of the result.  The shortcut
+        # addition stays a separate streaming pass (ocs_add_relu, which also takes the maximum): in the epilogue
+        # it makes the output-bound layers wait for the shortcut tensor's loads and costs more than it saves.
+        fused_relu = spec.relu and not spec.residual_from
         y = conv_forward(layers[spec.name], src, a_signed=first, a_bits=a_bits, dev_status=dev_status,
                          max_abs=mx.get(id(src)), relu=fused_relu, max_out=m if fused_relu else None)
         if spec.residual_from:

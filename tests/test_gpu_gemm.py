@@ -48,6 +48,14 @@ def _check_linear(seed, M, Cn, N, S, a_signed=False, lda=None, bias=True, a_scal
     ocs.ocs_qlinear(Ad, dev(np.array([a_scale], np.float32)), Wd, dev(np.array([w_scale], np.float32)),
                     dev(idx), Cn, S, bias=None if b is None else dev(b), max_out=m, dev_status=st)
     assert host(m)[0] == np.float32(orc.maxabs(Yo)) and ocs.ocs_poll_status(st) == 0
+    # a shortcut tensor added in the epilogue: the checker's add_relu on its own output
+    res = prng.normal(seed, 11, (M, N))
+    Ys = ocs.ocs_qlinear(Ad, dev(np.array([a_scale], np.float32)), Wd, dev(np.array([w_scale], np.float32)),
+                         dev(idx), Cn, S, bias=None if b is None else dev(b), residual=dev(res), relu=True, max_out=m,
+                         dev_status=st)
+    ref = orc.add_relu(Yo, res, True)
+    np.testing.assert_array_equal(host(Ys), ref)
+    assert host(m)[0] == np.float32(orc.maxabs(ref)) and ocs.ocs_poll_status(st) == 0
 
 
 @pytest.mark.parametrize("M,Cn,N,S", [(64, 512, 256, 26), (128, 256, 128, 0), (1, 16, 8, 0), (5, 130, 70, 3),
@@ -128,6 +136,12 @@ def _check_conv(seed, Nb, H, Wd_, Cn, O, S, k, stride, pad, a_signed=False):
                        dev(idx), S, k, k, stride, pad, bias=dev(b), relu=True, max_out=m, dev_status=st)
     np.testing.assert_array_equal(host(Yr), orc.relu(Yo))
     assert host(m)[0] == np.float32(orc.maxabs(orc.relu(Yo))) and ocs.ocs_poll_status(st) == 0
+    res = prng.normal(seed, 11, Yo.shape)
+    Ys = ocs.ocs_qconv(dev(X), dev(np.array([0.02], np.float32)), packed, dev(np.array([0.003], np.float32)),
+                       dev(idx), S, k, k, stride, pad, bias=dev(b), residual=dev(res), relu=False, max_out=m, dev_status=st)
+    ref = orc.add_relu(Yo, res, False)
+    np.testing.assert_array_equal(host(Ys), ref)
+    assert host(m)[0] == np.float32(orc.maxabs(ref)) and ocs.ocs_poll_status(st) == 0
 
 
 @pytest.mark.parametrize("Nb,H,W,Cn,O,S,k,stride,pad", [
