@@ -49,7 +49,7 @@ def algorithmic_bytes(kernel: str, *, N=0, n=0, M=0, C=0, S=0, Nout=0, R=1, rows
     GEMM: M x Nout outputs over K' = (C+S)*R."""
     if kernel == "col_minmax_kernel":
         return 4 * N
-    if kernel == "split_scatter_kernel":
+    if kernel in ("split_rows_kernel", "split_scatter_kernel"):   # row-staged form / plain-load fallback
         return 4 * N + 4 * n
     if kernel in ("hist_kernel", "maxabs_kernel"):
         return 4 * n
@@ -100,11 +100,11 @@ def aggregate_gbs(bytes_per_rank_step: int, world: int, ms_per_step: float) -> f
 # DRAM traffic of the dominant kernel from one ncu capture (profiles/split_rows_kernel_fc6.md): the launch
 # at r = 0.1 moved 812.2 MB for 863.2 MB of algorithmic bytes.  The figure is only reported while the
 # kernel's source text is the one that was profiled.
-NCU_TRAFFIC = {"split_scatter_kernel": dict(fingerprint="01c86520fb09b5a5", dram_bytes=812.2e6, algorithmic_bytes=863.2e6)}
+NCU_TRAFFIC = {"split_rows_kernel": dict(fingerprint="01c86520fb09b5a5", dram_bytes=812.2e6, algorithmic_bytes=863.2e6)}
 
 
 def kernel_fingerprint(kernel: str):
-    if kernel != "split_scatter_kernel":
+    if kernel != "split_rows_kernel":
         return None
     import hashlib
     try:
@@ -178,7 +178,7 @@ class Fc6Sweep:
             S = configs_num_splits(C, r)
             n = O * (C + S)
             led.add("col_minmax_kernel", N=N)
-            led.add("split_scatter_kernel", N=N, n=n)
+            led.add("split_rows_kernel", N=N, n=n)
             led.add("hist_kernel", n=n)
             led.add("quantize_kernel", n=n)
             led.add("maxabs_kernel", n=M * C)
@@ -303,7 +303,7 @@ class Fc6Sweep:
             ac, asc = orc.quantize(A, 8, False, orc.maxabs(A))
             orc.qlinear(ac, False, asc, wc, wsc, idx)
             n = O * (C + S)
-            for k, kw in (("col_minmax_kernel", dict(N=O * C)), ("split_scatter_kernel", dict(N=O * C, n=n)),
+            for k, kw in (("col_minmax_kernel", dict(N=O * C)), ("split_rows_kernel", dict(N=O * C, n=n)),
                           ("hist_kernel", dict(n=n)), ("quantize_kernel", dict(n=n)), ("maxabs_kernel", dict(n=M * C)),
                           ("quantize_kernel", dict(n=M * C)),
                           ("ocs_gemm_kernel(linear)", dict(rows=M, M=M, C=C, S=S, Nout=O))):
@@ -476,7 +476,7 @@ class SmallFc(Fc6Sweep):
         S = configs_num_splits(C, 0.05)
         n = O * (C + S)
         led.add("col_minmax_kernel", N=O * C)
-        led.add("split_scatter_kernel", N=O * C, n=n)
+        led.add("split_rows_kernel", N=O * C, n=n)
         led.add("quantize_kernel", n=n)
         led.add("maxabs_kernel", n=M * C)
         led.add("quantize_kernel", n=M * C)
@@ -611,8 +611,7 @@ class ResNet50(NetWorkload):
         return nets.resnet50_forward(cfg, layers, self.dev_in["X"], dev_status=self.status)
 
     def oracle_sample(self, orc, host):
-        sys.path.insert(0, os.path.join(ROOT, "tests"))
-        import net_oracle
+        from oracle import net_oracle
         small = configs.config4(batch=1, image=64)
         t0 = time.perf_counter()
         net_oracle.resnet50(small)
@@ -673,8 +672,7 @@ class Lstm(NetWorkload):
                                  before_decoder=lambda: main.wait_event(self.ev_done[4]))
 
     def oracle_sample(self, orc, host):
-        sys.path.insert(0, os.path.join(ROOT, "tests"))
-        import net_oracle
+        from oracle import net_oracle
         small = configs.config5(vocab=3000, batch=4, seq=6)
         t0 = time.perf_counter()
         net_oracle.lstm(small)
@@ -926,7 +924,7 @@ def main():
     gemm_ms = sum(trace.get(k, (0, 0.0))[1] for k in ("ocs_gemm_kernel(linear)", "ocs_gemm_kernel(conv)",
                                                      "splitk_reduce_kernel"))
     gemm_tops = (led.ops * args.steps / (gemm_ms * 1e-3) / 1e12) if gemm_ms > 0 else None
-    sq_names = ("col_minmax_kernel", "split_scatter_kernel", "hist_kernel", "quantize_kernel", "maxabs_kernel",
+    sq_names = ("col_minmax_kernel", "split_rows_kernel", "split_scatter_kernel", "hist_kernel", "quantize_kernel", "maxabs_kernel",
                 "split_hist_kernel", "split_quantize_kernel")
     sq_ms = sum(trace[k][1] for k in sq_names if k in trace) + sum(
         trace[k][1] for k in ("split_plan_kernel", "score_kernel", "pick_kernel") if k in trace)

@@ -137,7 +137,7 @@ ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, int64_t ld_i
                         float* alpha, void* ws, size_t ws_bytes, int* dev_status, void* stream);
 
 /* ocs_split_quantize -----------------------------------------------------------------------
- * ocs_split followed by ocs_quantize on its result ("OCS followed by clipping", Section 5.2;
+ * ocs_split followed by ocs_quantize on its result (the split-then-clip order of Section 5.2;
  * Sections 3.2-3.4, Eq. 1, Section 4.1) in one call that never writes the fp32 W': the
  * expanded rows exist only in shared memory, from where they are histogrammed (mode MSE) and
  * quantized.  W is read three times (extrema, histogram, quantization) instead of W and W'
@@ -205,8 +205,8 @@ ocs_status ocs_act_select_channels(const float* P, int64_t rows, int C, int64_t 
 
 /* ocs_act_split_quantize_static --------------------------------------------------------------
  * Activation side of Eq. 4 for a channel list chosen ahead of time (Section 5.3's static variant;
- * Section 3.5's "custom layer" that copies and scales the listed channels), fused with the
- * quantization: A (device) fp32 [rows][ld_in >= C]; every channel in sel (device, int32 [S],
+ * the run-time duplication and scaling of the listed channels that Section 3.5 describes), fused with
+ * the quantization: A (device) fp32 [rows][ld_in >= C]; every channel in sel (device, int32 [S],
  * distinct, in [0, C)) is duplicated and both copies carry a * 0.5; codes (device, int8 or the uint8
  * bit pattern) [rows][ld_codes >= C+S], the copy of sel[s] at column C + s; idx_map (device,
  * int32 [C+S]) as in ocs_split.  Grid: alpha_in (device, fp32 [1]) when given -- a threshold
@@ -254,7 +254,7 @@ void ocs_quantize_workspace_views(void* ws, int n_bins, int n_candidates, uint64
  * The split layer of Eq. 3 evaluated on integer codes (Eq. 2 on low-precision MACs):
  *     acc[m][n] = sum_{j < C+S} A[m][idx_map[j]] * Wc[n][j]          (int32, exact)
  *     Y[m][n]   = fmaf((float)acc[m][n], a_scale * w_scale, bias[n])  (bias 0 if NULL)
- * The duplicated activation channels (Section 3.5: "copies ... the appropriate channels")
+ * The duplicated activation channels (the run-time channel duplication of Section 3.5)
  * are gathered through idx_map while the operand tiles are staged; an expanded activation
  * tensor is never written.  idx_map[j] must equal j for j < C (as ocs_split produces).
  * A codes [M][C], row stride lda bytes, uint8 when a_signed = 0 else int8; Wc int8 [N][C+S],

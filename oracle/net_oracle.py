@@ -1,5 +1,6 @@
-"""The end-to-end networks evaluated with the CPU checker only (test infrastructure): the same
-layer graphs as the CUDA drivers, written independently on top of oracle/oracle.py."""
+"""The end-to-end networks evaluated with the CPU checker only (TEST INFRASTRUCTURE: used by the
+tests and by the bench's CPU-baseline leg, never by the CUDA library): the same layer graphs as the
+CUDA drivers, written independently on top of oracle/oracle.py."""
 import numpy as np
 
 from oracle import oracle as orc

@@ -7,6 +7,12 @@
 #include "ocs_oracle.h"
 
 #include <math.h>
+#ifndef M_PI
+#define M_PI 3.14159265358979323846
+#endif
+#ifndef M_E
+#define M_E 2.71828182845904523536
+#endif
 #include <stdlib.h>
 #include <string.h>
 
@@ -235,6 +241,291 @@ int ocs_oracle_clip_mse_exact(const float* T, int64_t n, int bits, int is_signed
     if (cbest < 0 || score <= best) { best = score; cbest = c; }
   }
   *alpha = (float)((double)m * (double)cbest / (double)n_candidates);
+  return 0;
+}
+
+/* ------------------------------------------------------------------ Section 3.3: grid step of the QA split */
+/* The half step of the quantization-aware split is half a step of the grid the split tensor will
+ * be rounded on, and that grid depends on the split's outcome.  Reading taken ("two-pass rule"):
+ * run the greedy loop once with plain halving, take max|W'| of that run, qa_step = that / L
+ * (one fp32 division, L = 2^(bits-1) - 1), then run the loop again with d = qa_step / 2. */
+int ocs_oracle_split_qa(const float* W, int O, int C, int R, int S, int qa_bits, float* W_out,
+                        int32_t* idx_map, int32_t* split_order, float* max_abs3) {
+  if (qa_bits < 2 || qa_bits > 8) return 1;
+  float mx[2] = {0.0f, 0.0f};
+  int rc = split_common(W, O, C, R, S, 0.0f, W_out, idx_map, split_order, mx, 1);
+  if (rc) return rc;
+  volatile float step = mx[1] / (float)code_limit(qa_bits, 1);
+  rc = split_common(W, O, C, R, S, step, W_out, idx_map, split_order, mx, 1);
+  if (rc) return rc;
+  if (max_abs3) { max_abs3[0] = mx[0]; max_abs3[1] = mx[1]; max_abs3[2] = step; }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ Section 4.3: KL clip search */
+/* histogram of |x| exactly as in the MSE search */
+static uint64_t* abs_histogram(const float* T, int64_t n, int B, float m) {
+  uint64_t* h = (uint64_t*)calloc((size_t)B, sizeof(uint64_t));
+  if (!h) return NULL;
+  volatile float invw = (float)B / m;
+  for (int64_t i = 0; i < n; ++i) {
+    volatile float t = fabsf(T[i]) * invw;
+    int b = (int)t;
+    if (b > B - 1) b = B - 1;
+    h[b] += 1;
+  }
+  return h;
+}
+
+/* The paper describes the method only in general terms (histogram, candidate thresholds,
+ * divergence between the float and the quantized distribution, a little probability mass moved
+ * into empty bins so that the divergence is defined).  Reading taken, for candidate c of the
+ * same candidate list as the MSE search (alpha_c = max * c / n_candidates):
+ *   the first n_c = ceil(c * B / n_candidates) bins lie inside the threshold;
+ *   P: those bins' counts, with the count of everything beyond them added to the last one
+ *      (clipped values saturate), divided by the total count;
+ *   Q: the same bins WITHOUT the clipped mass, quantized and expanded again: bin i belongs to
+ *      level j(i) = clamp(rint(x_i / step_c)) (x_i the bin centre, step_c = alpha_c / L); a level's
+ *      count is spread evenly over its non-empty bins; divided by the kept count;
+ *   the only bin where P > 0 and Q = 0 can be the last one (empty itself, but holding clipped
+ *      mass): it then gets eps = 1e-4 and every other entry of Q is scaled by (1 - eps);
+ *   score_c = sum over bins with P > 0 of P * ln(P / Q), bins ascending, in double.
+ * Smallest score wins, ties to the largest threshold; a candidate that keeps no value at all
+ * scores +infinity. */
+int ocs_oracle_clip_kl(const float* T, int64_t n, int bits, int is_signed, int n_bins,
+                       int n_candidates, float* alpha, float* max_abs, uint64_t* hist,
+                       double* scores) {
+  if (!T || !alpha || n < 0 || bits < 2 || bits > 8 || n_bins < 1 || n_candidates < 1) return 1;
+  const int L = code_limit(bits, is_signed);
+  const int B = n_bins;
+  const float m = ocs_oracle_maxabs(T, n);
+  if (max_abs) *max_abs = m;
+  if (m == 0.0f) {
+    *alpha = 0.0f;
+    if (hist) { memset(hist, 0, sizeof(uint64_t) * (size_t)B); hist[0] = (uint64_t)n; }
+    if (scores) for (int c = 0; c < n_candidates; ++c) scores[c] = 0.0;
+    return 0;
+  }
+  uint64_t* h = abs_histogram(T, n, B, m);
+  uint64_t* level_count = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)(L + 1));
+  int* level_bins = (int*)malloc(sizeof(int) * (size_t)(L + 1));
+  int* level_of = (int*)malloc(sizeof(int) * (size_t)B);
+  if (!h || !level_count || !level_bins || !level_of) {
+    free(h); free(level_count); free(level_bins); free(level_of);
+    return 2;
+  }
+  if (hist) memcpy(hist, h, sizeof(uint64_t) * (size_t)B);
+  uint64_t total = 0;
+  for (int b = 0; b < B; ++b) total += h[b];
+  const double width = (double)m / (double)B;
+  const double eps = 1e-4;
+  double best = 0.0;
+  int cbest = -1;
+  for (int c = 1; c <= n_candidates; ++c) {
+    const float alpha_c = (float)((double)m * (double)c / (double)n_candidates);
+    const double step = (double)alpha_c / (double)L;
+    int nc = (int)(((int64_t)c * B + n_candidates - 1) / n_candidates);
+    if (nc < 1) nc = 1;
+    if (nc > B) nc = B;
+    uint64_t kept = 0;
+    for (int j = 0; j <= L; ++j) { level_count[j] = 0; level_bins[j] = 0; }
+    for (int b = 0; b < nc; ++b) {
+      const double xb = ((double)b + 0.5) * width;
+      double q = nearbyint(xb / step);
+      if (q < 0.0) q = 0.0;
+      if (q > (double)L) q = (double)L;
+      level_of[b] = (int)q;
+      kept += h[b];
+      level_count[(int)q] += h[b];
+      if (h[b] > 0) level_bins[(int)q] += 1;
+    }
+    double score;
+    if (kept == 0) {
+      score = INFINITY;
+    } else {
+      const uint64_t clipped = total - kept;
+      const int smooth = (h[nc - 1] == 0 && clipped > 0);
+      score = 0.0;
+      for (int b = 0; b < nc; ++b) {
+        const uint64_t pb = h[b] + (b == nc - 1 ? clipped : 0);
+        if (pb == 0) continue;
+        const double p = (double)pb / (double)total;
+        double q;
+        if (h[b] == 0) {
+          q = eps; /* the last bin: empty itself, but clipped values land on it */
+        } else {
+          const int j = level_of[b];
+          q = ((double)level_count[j] / (double)level_bins[j]) / (double)kept;
+          if (smooth) q = q * (1.0 - eps);
+        }
+        score += p * log(p / q);
+      }
+    }
+    if (scores) scores[c - 1] = score;
+    if (cbest < 0 || score <= best) { best = score; cbest = c; }
+  }
+  *alpha = (float)((double)m * (double)cbest / (double)n_candidates);
+  free(h); free(level_count); free(level_bins); free(level_of);
+  return 0;
+}
+
+/* ------------------------------------------------------------------ Section 4.2: ACIQ */
+/* The threshold, in units of the fitted scale, that minimises the model error
+ *     E(alpha) = (clipping noise of the fitted density beyond alpha) + step^2 / 12,
+ * step = 2 * alpha / n_intervals (a uniform grid of n_intervals steps across [-alpha, alpha]).
+ *   Laplace(0, b):  clipping noise 2 b^2 e^(-alpha/b);  dE/dalpha = 0  <=>  t e^t = 3 n_intervals^2,
+ *                   t = alpha / b  (a Lambert-W value), solved by Newton on t + ln t = ln(3 n^2).
+ *   Gauss(0, s):    clipping noise 2 [(s^2 + alpha^2) Qf(t) - alpha s phi(t)], t = alpha / s;
+ *                   dE/dalpha = 0  <=>  4 [phi(t) - t Qf(t)] = 2 t / (3 n_intervals^2), by bisection
+ *                   (the left side falls, the right side rises).
+ * With 2^M intervals this is the published analysis of the method; the paper's grid of 2^M - 1
+ * points has n_intervals = 2 L. */
+double ocs_oracle_aciq_multiplier(double n_intervals, int laplace) {
+  if (!(n_intervals > 0.0)) return 0.0;
+  const double z = 3.0 * n_intervals * n_intervals;
+  if (laplace) {
+    const double lz = log(z);
+    double t = lz > 1.0 ? lz : 1.0;
+    for (int it = 0; it < 100; ++it) {
+      const double g = t + log(t) - lz;
+      const double tn = t - g / (1.0 + 1.0 / t);
+      if (fabs(tn - t) <= 1e-16 * fabs(tn)) { t = tn; break; }
+      t = tn > 1e-300 ? tn : 1e-300;
+    }
+    return t;
+  }
+  double lo = 0.0, hi = 40.0;
+  for (int it = 0; it < 200; ++it) {
+    const double t = 0.5 * (lo + hi);
+    const double phi = exp(-0.5 * t * t) / sqrt(2.0 * M_PI);
+    const double tail = 0.5 * erfc(t / sqrt(2.0));
+    const double f = 4.0 * (phi - t * tail) - 2.0 * t / z;
+    if (f > 0.0) lo = t; else hi = t;
+  }
+  return 0.5 * (lo + hi);
+}
+
+/* Reading taken (the paper gives no formula): the two candidate densities are zero-location and
+ * are fitted to the histogram of |x| (same bins as the other searches, bin centres x_i):
+ * b = sum h x_i / n, s = sqrt(sum h x_i^2 / n), sums in double, bins ascending.  The density with
+ * the larger likelihood at its own fit is taken: Laplace iff b / s < sqrt(pi / (2 e)).
+ * alpha = multiplier(2 L) * (b or s), rounded to fp32, and never above max|x|.
+ * stats (nullable) = {b, s, 1 if Laplace else 0, multiplier}. */
+int ocs_oracle_clip_aciq(const float* T, int64_t n, int bits, int is_signed, int n_bins,
+                         float* alpha, float* max_abs, uint64_t* hist, double* stats) {
+  if (!T || !alpha || n < 0 || bits < 2 || bits > 8 || n_bins < 1) return 1;
+  const int L = code_limit(bits, is_signed);
+  const int B = n_bins;
+  const float m = ocs_oracle_maxabs(T, n);
+  if (max_abs) *max_abs = m;
+  if (m == 0.0f) {
+    *alpha = 0.0f;
+    if (hist) { memset(hist, 0, sizeof(uint64_t) * (size_t)B); hist[0] = (uint64_t)n; }
+    if (stats) { stats[0] = stats[1] = stats[2] = stats[3] = 0.0; }
+    return 0;
+  }
+  uint64_t* h = abs_histogram(T, n, B, m);
+  if (!h) return 2;
+  if (hist) memcpy(hist, h, sizeof(uint64_t) * (size_t)B);
+  const double width = (double)m / (double)B;
+  double cnt = 0.0, s1 = 0.0, s2 = 0.0;
+  for (int b = 0; b < B; ++b) {
+    const double xb = ((double)b + 0.5) * width;
+    const double hb = (double)h[b];
+    cnt += hb;
+    s1 += hb * xb;
+    s2 += hb * xb * xb;
+  }
+  free(h);
+  const double bb = s1 / cnt;
+  const double sd = sqrt(s2 / cnt);
+  const int laplace = bb / sd < sqrt(M_PI / (2.0 * M_E));
+  const double mult = ocs_oracle_aciq_multiplier(2.0 * (double)L, laplace);
+  float a = (float)(mult * (laplace ? bb : sd));
+  if (!(a < m)) a = m;
+  *alpha = a;
+  if (stats) { stats[0] = bb; stats[1] = sd; stats[2] = (double)laplace; stats[3] = mult; }
+  return 0;
+}
+
+/* ------------------------------------------------------------------ Section 3.4: knapsack allocation */
+/* curve[s] = max|W'| after s greedy plain-halving splits, s = 0..S_max: what the allocation's
+ * reward is made of.  The channel maxima are all the greedy loop sees under plain halving. */
+int ocs_oracle_range_curve(const float* W, int O, int C, int R, int S_max, float* curve) {
+  if (!W || !curve || O <= 0 || C <= 0 || R <= 0 || S_max < 0) return 1;
+  float* cmax = (float*)malloc(sizeof(float) * (size_t)(C + S_max));
+  if (!cmax) return 2;
+  for (int j = 0; j < C; ++j) cmax[j] = channel_maxabs(W, O, C, R, j);
+  for (int s = 0; s <= S_max; ++s) {
+    const int alive = C + s;
+    int jbest = 0;
+    float best = -1.0f;
+    for (int j = 0; j < alive; ++j)
+      if (cmax[j] > best) { best = cmax[j]; jbest = j; }
+    curve[s] = best;
+    if (s == S_max) break;
+    volatile float half = best * 0.5f;
+    cmax[jbest] = half;
+    cmax[alive] = half;
+  }
+  free(cmax);
+  return 0;
+}
+
+/* Section 3.4's alternative to ceil(r*C) per layer: choose the split counts of all layers at once.
+ * reward_l(s) = (curve_l[0] - curve_l[s]) / curve_l[0], the fraction by which s splits shrink the
+ * layer's dynamic range (0 for an all-zero layer); cost_l(s) = s * unit_cost[l] weight elements
+ * (unit_cost = O * R, one more input channel).  Maximise sum_l reward_l(s_l) subject to
+ * sum_l cost_l(s_l) <= budget, 0 <= s_l <= s_max[l]: a multiple-choice knapsack, solved exactly by
+ * dynamic programming over the budget in units of gcd(unit_cost): layers in order,
+ * best_l[b] = max over s (ascending; a later s must be strictly better) of
+ * best_{l-1}[b - s * cost] + reward_l(s), in double.  curves holds the layers' curves back to back
+ * (layer l at curve_off[l], s_max[l] + 1 entries).  S_out[l] = chosen count; *total_reward may be
+ * NULL.  The paper states the objective and the constraint, not the solver: parity unpinned beyond
+ * optimality. */
+static int64_t gcd64(int64_t a, int64_t b) { while (b) { int64_t t = a % b; a = b; b = t; } return a; }
+
+int ocs_oracle_knapsack(int n_layers, const float* curves, const int64_t* curve_off,
+                        const int32_t* s_max, const int64_t* unit_cost, int64_t budget,
+                        int32_t* S_out, double* total_reward) {
+  if (n_layers <= 0 || !curves || !curve_off || !s_max || !unit_cost || !S_out || budget < 0) return 1;
+  int64_t g = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    if (unit_cost[l] <= 0 || s_max[l] < 0) return 1;
+    g = gcd64(g, unit_cost[l]);
+  }
+  const int64_t Bu = budget / g; /* budget in units (a remainder cannot be spent) */
+  if (Bu > (int64_t)1 << 26) return 3;
+  double* prev = (double*)calloc((size_t)(Bu + 1), sizeof(double));
+  double* cur = (double*)malloc(sizeof(double) * (size_t)(Bu + 1));
+  int32_t* choice = (int32_t*)malloc(sizeof(int32_t) * (size_t)n_layers * (size_t)(Bu + 1));
+  if (!prev || !cur || !choice) { free(prev); free(cur); free(choice); return 2; }
+  for (int l = 0; l < n_layers; ++l) {
+    const float* cv = curves + curve_off[l];
+    const int64_t cu = unit_cost[l] / g;
+    const double c0 = (double)cv[0];
+    for (int64_t b = 0; b <= Bu; ++b) {
+      double best = prev[b]; /* s = 0: reward 0 */
+      int32_t sbest = 0;
+      for (int s = 1; s <= s_max[l]; ++s) {
+        if ((int64_t)s * cu > b) break;
+        const double reward = c0 > 0.0 ? (c0 - (double)cv[s]) / c0 : 0.0;
+        const double v = prev[b - (int64_t)s * cu] + reward;
+        if (v > best) { best = v; sbest = s; }
+      }
+      cur[b] = best;
+      choice[(size_t)l * (size_t)(Bu + 1) + (size_t)b] = sbest;
+    }
+    double* t = prev; prev = cur; cur = t;
+  }
+  if (total_reward) *total_reward = prev[Bu];
+  int64_t b = Bu;
+  for (int l = n_layers - 1; l >= 0; --l) {
+    const int32_t sc = choice[(size_t)l * (size_t)(Bu + 1) + (size_t)b];
+    S_out[l] = sc;
+    b -= (int64_t)sc * (unit_cost[l] / g);
+  }
+  free(prev); free(cur); free(choice);
   return 0;
 }
 

@@ -13,11 +13,14 @@
  * unsigned codes.  All functions return 0 on success, non-zero on a bad argument.
  *
  * Pinned by tests (paper facts, closed forms, brute force): split, quantize, clip_mse,
- * qlinear, qconv, fold_duplicates, pools, relu/add, act_select, act_split_static.  Parity unpinned (conventions the paper does not fix,
- * enforced only checker-vs-GPU): the QA grid-step policy, the unsigned activation grid,
- * the bin count and the tie rule of the clip search, the LSTM cell's sigmoid/tanh routines,
- * the quantile convention of act_select (nearest rank on |a|; the paper says only "99th
- * percentile").
+ * clip_mse_exact, clip_kl (as the function defined here), clip_aciq (the closed forms), qlinear,
+ * qconv, fold_duplicates, pools, relu/add, act_select, act_split_static, range_curve, knapsack
+ * (optimality).  Parity unpinned (conventions the paper does not fix, enforced only
+ * checker-vs-GPU): the QA grid-step policy (split_qa), the unsigned activation grid, the bin
+ * count and the tie rule of the clip searches, the construction of the two distributions of
+ * clip_kl and its smoothing constant, the density test and the histogram moments of clip_aciq,
+ * the reward sum and the tie rule of knapsack, the LSTM cell's sigmoid/tanh routines, the
+ * quantile convention of act_select (nearest rank on |a|; the paper says only which percentile).
  */
 #ifndef OCS_ORACLE_H
 #define OCS_ORACLE_H
@@ -72,6 +75,45 @@ int ocs_oracle_clip_mse(const float* T, int64_t n, int bits, int is_signed, int 
  * score_c = sum_i (x_i - Q_c(x_i))^2 in double, elements in storage order. */
 int ocs_oracle_clip_mse_exact(const float* T, int64_t n, int bits, int is_signed,
                               int n_candidates, float* alpha, double* scores);
+
+/* The split with the grid step of the quantization-aware rule chosen by the two-pass rule
+ * (Section 3.3 leaves open which grid the half step refers to): a plain-halving run of the
+ * greedy loop predicts max|W'|, qa_step = that / L(qa_bits) in fp32, and the loop is run again
+ * with that step.  max_abs3 (nullable) = max|W|, max|W'|, qa_step. */
+int ocs_oracle_split_qa(const float* W, int O, int C, int R, int S, int qa_bits, float* W_out,
+                        int32_t* idx_map, int32_t* split_order, float* max_abs3);
+
+/* Section 4.3: clip threshold by KL divergence, on the histogram and candidate list of the MSE
+ * search.  For candidate c the first n_c = ceil(c * n_bins / n_candidates) bins are inside the
+ * threshold; P = their counts with the clipped count added to the last of them; Q = their
+ * counts without it, grouped into the quantization levels of their bin centres and spread back
+ * evenly over each level's non-empty bins; both normalised; if the last bin is empty but takes
+ * clipped mass, Q gets 1e-4 there and is scaled by (1 - 1e-4) elsewhere; score_c = sum P ln(P/Q)
+ * in double, bins ascending.  Smallest score wins, ties to the largest threshold. */
+int ocs_oracle_clip_kl(const float* T, int64_t n, int bits, int is_signed, int n_bins,
+                       int n_candidates, float* alpha, float* max_abs, uint64_t* hist,
+                       double* scores);
+
+/* Section 4.2 (ACIQ): which of a zero-location Laplace or Gauss density fits the histogram of |x|
+ * better (likelihood at the fitted scale: Laplace iff b / s < sqrt(pi / (2e)), b = mean |x|,
+ * s = sqrt(mean x^2), both from the bin centres), then the threshold that minimises
+ * (clipping noise of that density) + step^2 / 12 in closed form: alpha = multiplier * scale,
+ * capped at max|x|.  stats (nullable) = {b, s, Laplace?, multiplier}.
+ * ocs_oracle_aciq_multiplier(n_intervals, laplace): the minimiser alpha / scale for a uniform grid
+ * of n_intervals steps across [-alpha, alpha] (the paper's 2^M - 1 grid points: n_intervals = 2L). */
+double ocs_oracle_aciq_multiplier(double n_intervals, int laplace);
+int ocs_oracle_clip_aciq(const float* T, int64_t n, int bits, int is_signed, int n_bins,
+                         float* alpha, float* max_abs, uint64_t* hist, double* stats);
+
+/* Section 3.4, knapsack allocation.  range_curve: curve[s] = max|W'| after s greedy plain-halving
+ * splits (s = 0..S_max).  knapsack: split counts for all layers at once, maximising the summed
+ * fractional reduction of each layer's dynamic range, (curve[0] - curve[s]) / curve[0], subject to
+ * sum_l S_out[l] * unit_cost[l] <= budget (weight elements; unit_cost = O * R) and
+ * S_out[l] <= s_max[l]; exact dynamic programme (ties: fewer splits in the later layer). */
+int ocs_oracle_range_curve(const float* W, int O, int C, int R, int S_max, float* curve);
+int ocs_oracle_knapsack(int n_layers, const float* curves, const int64_t* curve_off,
+                        const int32_t* s_max, const int64_t* unit_cost, int64_t budget,
+                        int32_t* S_out, double* total_reward);
 
 /* Eq. 2 / Eq. 3 on integer codes: acc[m][n] = sum_{j < C+S} A[m][idx_map[j]] * Wc[n][j]
  * (exact, checked to fit int32), Y = fmaf((float)acc, a_scale * w_scale, bias[n]).

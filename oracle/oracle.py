@@ -128,6 +128,81 @@ def clip_mse_exact(T, bits: int, is_signed: bool = True, n_candidates: int = 128
     return dict(alpha=float(alpha.value), scores=scores)
 
 
+def split_qa(W, S: int, qa_bits: int):
+    """Split with the two-pass grid-step rule -> (W', idx_map, split_order, (max|W|, max|W'|), qa_step)."""
+    W = _f32(W)
+    O, Cn = W.shape[0], W.shape[1]
+    R = int(np.prod(W.shape[2:])) if W.ndim > 2 else 1
+    out = np.empty((O, Cn + S) + tuple(W.shape[2:]), dtype=np.float32)
+    idx = np.empty(Cn + S, dtype=np.int32)
+    order = np.empty(max(S, 1), dtype=np.int32)
+    mx = np.zeros(3, dtype=np.float32)
+    rc = lib().ocs_oracle_split_qa(_p(W, _f32p), O, Cn, R, int(S), int(qa_bits), _p(out, _f32p), _p(idx, _i32p),
+                                   _p(order, _i32p), _p(mx, _f32p))
+    _check(rc, "split_qa")
+    return out, idx, order[:S], (float(mx[0]), float(mx[1])), float(mx[2])
+
+
+def clip_kl(T, bits: int, is_signed: bool = True, n_bins: int = 2048, n_candidates: int = 128):
+    """-> dict(alpha, max_abs, hist, scores) of the KL-divergence search (Section 4.3)."""
+    T = _f32(T)
+    hist = np.zeros(n_bins, dtype=np.uint64)
+    scores = np.zeros(n_candidates, dtype=np.float64)
+    alpha, mx = C.c_float(0), C.c_float(0)
+    rc = lib().ocs_oracle_clip_kl(_p(T, _f32p), C.c_int64(T.size), int(bits), int(bool(is_signed)), int(n_bins),
+                                  int(n_candidates), C.byref(alpha), C.byref(mx), _p(hist, _u64p), _p(scores, _f64p))
+    _check(rc, "clip_kl")
+    return dict(alpha=float(alpha.value), max_abs=float(mx.value), hist=hist, scores=scores)
+
+
+def aciq_multiplier(n_intervals: float, laplace: bool) -> float:
+    fn = lib().ocs_oracle_aciq_multiplier
+    fn.restype = C.c_double
+    fn.argtypes = [C.c_double, C.c_int]
+    return float(fn(float(n_intervals), int(bool(laplace))))
+
+
+def clip_aciq(T, bits: int, is_signed: bool = True, n_bins: int = 2048):
+    """-> dict(alpha, max_abs, hist, b, sigma, laplace, multiplier) of the ACIQ threshold (Section 4.2)."""
+    T = _f32(T)
+    hist = np.zeros(n_bins, dtype=np.uint64)
+    stats = np.zeros(4, dtype=np.float64)
+    alpha, mx = C.c_float(0), C.c_float(0)
+    rc = lib().ocs_oracle_clip_aciq(_p(T, _f32p), C.c_int64(T.size), int(bits), int(bool(is_signed)), int(n_bins),
+                                    C.byref(alpha), C.byref(mx), _p(hist, _u64p), _p(stats, _f64p))
+    _check(rc, "clip_aciq")
+    return dict(alpha=float(alpha.value), max_abs=float(mx.value), hist=hist, b=float(stats[0]), sigma=float(stats[1]),
+                laplace=bool(stats[2]), multiplier=float(stats[3]))
+
+
+def range_curve(W, S_max: int):
+    """max|W'| after s = 0..S_max greedy plain-halving splits -> float32 [S_max + 1]."""
+    W = _f32(W)
+    O, Cn = W.shape[0], W.shape[1]
+    R = int(np.prod(W.shape[2:])) if W.ndim > 2 else 1
+    curve = np.empty(S_max + 1, dtype=np.float32)
+    _check(lib().ocs_oracle_range_curve(_p(W, _f32p), O, Cn, R, int(S_max), _p(curve, _f32p)), "range_curve")
+    return curve
+
+
+def knapsack(curves, unit_cost, budget: int):
+    """curves: list of float32 arrays (one per layer, curve[s] for s = 0..s_max); unit_cost: elements one more
+    channel adds to each layer (O * R) -> (S per layer int32, total reward)."""
+    n = len(curves)
+    s_max = np.array([len(c) - 1 for c in curves], dtype=np.int32)
+    off = np.zeros(n, dtype=np.int64)
+    off[1:] = np.cumsum([len(c) for c in curves])[:-1]
+    flat = np.ascontiguousarray(np.concatenate([_f32(c) for c in curves]))
+    cost = np.ascontiguousarray(unit_cost, dtype=np.int64)
+    out = np.zeros(n, dtype=np.int32)
+    tot = C.c_double(0)
+    i64p = C.POINTER(C.c_int64)
+    rc = lib().ocs_oracle_knapsack(n, _p(flat, _f32p), off.ctypes.data_as(i64p), _p(s_max, _i32p),
+                                   cost.ctypes.data_as(i64p), C.c_int64(int(budget)), _p(out, _i32p), C.byref(tot))
+    _check(rc, "knapsack")
+    return out, float(tot.value)
+
+
 def act_ocs(A, S: int):
     """Activation side of OCS (Eq. 4) with the channels chosen on the batch at hand (the
     per-batch "Oracle OCS" of Section 5.3).  A [rows, C] holds one batch, one row per sample

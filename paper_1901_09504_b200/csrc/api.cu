@@ -11,6 +11,7 @@ namespace {
 struct TraceRecord {
   const char* name;
   cudaEvent_t start, stop;
+  bool closed = false;   // its stop event has been recorded
 };
 
 std::atomic<long long> g_launches{0};
@@ -33,22 +34,28 @@ cudaEvent_t take_event() {
 
 }  // namespace
 
-void trace_begin(const char* name, cudaStream_t stream) {
+int trace_begin(const char* name, cudaStream_t stream) {
   g_launches.fetch_add(1, std::memory_order_relaxed);
-  if (!g_trace_on) return;
+  if (!g_trace_on) return -1;
   std::lock_guard<std::mutex> lock(g_trace_mutex);
-  if (!g_trace_on || g_records.size() >= g_trace_cap) return;
+  if (!g_trace_on || g_records.size() >= g_trace_cap) return -1;
   TraceRecord r{name, take_event(), take_event()};
-  if (!r.start || !r.stop) return;
+  if (!r.start || !r.stop) {
+    if (r.start) g_event_pool.push_back(r.start);
+    if (r.stop) g_event_pool.push_back(r.stop);
+    return -1;
+  }
   cudaEventRecord(r.start, stream);
   g_records.push_back(r);
+  return (int)g_records.size() - 1;
 }
 
-void trace_end(cudaStream_t stream) {
-  if (!g_trace_on) return;
+void trace_end(int record, cudaStream_t stream) {
+  if (record < 0) return;
   std::lock_guard<std::mutex> lock(g_trace_mutex);
-  if (!g_trace_on || g_records.empty()) return;
-  cudaEventRecord(g_records.back().stop, stream);
+  if (!g_trace_on || (size_t)record >= g_records.size()) return;   // the trace ended, or a new one began, meanwhile
+  cudaEventRecord(g_records[record].stop, stream);
+  g_records[record].closed = true;
 }
 
 }  // namespace ocs
@@ -82,6 +89,7 @@ extern "C" int ocs_trace_stop(ocs_trace_row* rows, int capacity) {
   int n = 0;
   bool failed = false;
   for (const TraceRecord& r : g_records) {
+    if (!r.closed) continue;   // its launch had not returned when the trace ended
     float ms = 0.0f;
     if (cudaEventSynchronize(r.stop) != cudaSuccess || cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess)
       failed = true;

@@ -57,12 +57,15 @@ inline ocs_status launch_status() {
 // Launch accounting (defined in api.cu).  Every kernel launch of the library sits inside one
 // LaunchScope: it bumps the process-wide launch counter and, while a trace is active, brackets
 // the launch with a pair of CUDA events on the launch stream.
-void trace_begin(const char* name, cudaStream_t stream);
-void trace_end(cudaStream_t stream);
+// trace_begin returns the index of the record it opened, or -1 when nothing is recorded (tracing off, or the
+// trace is full); trace_end closes exactly that record.
+int trace_begin(const char* name, cudaStream_t stream);
+void trace_end(int record, cudaStream_t stream);
 struct LaunchScope {
   cudaStream_t stream;
-  LaunchScope(const char* name, cudaStream_t s) : stream(s) { trace_begin(name, s); }
-  ~LaunchScope() { trace_end(stream); }
+  int record;
+  LaunchScope(const char* name, cudaStream_t s) : stream(s), record(trace_begin(name, s)) {}
+  ~LaunchScope() { trace_end(record, stream); }
 };
 
 // One CTA per candidate threshold of the MSE clip search (defined in quantize.cu).

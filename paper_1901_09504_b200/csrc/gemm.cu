@@ -679,6 +679,9 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       const long long ldd = direct ? p.ldy : (long long)p.N;
       const bool base_vec = ((reinterpret_cast<uintptr_t>(dst0) & 15) == 0) && (ldd % 4 == 0);
       const bool acc_vec = p.acc_out && ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) && (p.ldy % 4 == 0);
+      // the shortcut tensor is read with 128-bit loads only when it is itself 16-byte aligned (a view that
+      // starts a few floats into a buffer takes the scalar loads)
+      const bool res_vec = p.residual && ((reinterpret_cast<uintptr_t>(p.residual) & 15) == 0) && (p.ldy % 4 == 0);
       float tile_max = 0.0f;
       const bool want_max = direct && p.max_bits != nullptr;
       // a warp whose 32 rows are all padding (a short M tile) has nothing to write
@@ -720,7 +723,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             float f2 = fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]), f3 = fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]);
             if (p.residual && orow[i] >= 0) {   // the block's shortcut: one more rounded addition per output
               const float* rr = p.residual + orow[i] * p.ldy + n0 + cq;
-              if (vec0) {
+              if (full && res_vec) {
                 const float4 r4 = __ldcs(reinterpret_cast<const float4*>(rr));
                 f0 = __fadd_rn(f0, r4.x); f1 = __fadd_rn(f1, r4.y); f2 = __fadd_rn(f2, r4.z); f3 = __fadd_rn(f3, r4.w);
               } else {
@@ -1197,6 +1200,8 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
   const long long Ktot = (long long)C + S;
   if (lda < C || ldw < Ktot || ldy < N) return OCS_ERR_SHAPE;
   if (ldw % 16 != 0 || !aligned(W_codes, 16) || !aligned(Y, 4)) return OCS_ERR_SHAPE;
+  if ((residual && !aligned(residual, 4)) || (acc_out && !aligned(acc_out, 4)) || (bias && !aligned(bias, 4)))
+    return OCS_ERR_SHAPE;
   if (Ktot * 255ll * 127ll > 2147483647ll) return OCS_ERR_UNSUPPORTED;
   ocs_status st = check_device();
   if (st != OCS_OK) return st;
@@ -1308,6 +1313,8 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   const int Cp = conv_tap_stride(C);
   const long long Ktot = (long long)kh * kw * ((long long)Cp + S);   // packed contraction length (ocs_conv_packed_k)
   if (ldw < Ktot || ldw % 16 != 0 || !aligned(W_packed, 16) || !aligned(Y, 4)) return OCS_ERR_SHAPE;
+  if ((residual && !aligned(residual, 4)) || (acc_out && !aligned(acc_out, 4)) || (bias && !aligned(bias, 4)))
+    return OCS_ERR_SHAPE;
   if (Ktot * 255ll * 127ll > 2147483647ll) return OCS_ERR_UNSUPPORTED;
   ConvGeom g;
   if (!conv_geom(Nb, H, Wd, kh, kw, stride, pad, &g)) return OCS_ERR_SHAPE;

@@ -895,7 +895,11 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
         *q = apply_path(*q, min(__ldg(depth + j), dep_cap), 0ull, d);
       }
     }
-    if (MODE == ROWS_STORE) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to the bulk store
+    // The threads' (generic-proxy) writes into the row buffer are ordered before what the copy engine (async
+    // proxy) does with the same bytes next: the bulk store that reads them (ROWS_STORE), and in every mode the
+    // bulk load that refills this buffer two groups later.  Each writing thread fences, then the CTA barrier
+    // orders the fences before thread 0's next copy.
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
     if (MODE == ROWS_STORE) {
       if (tid == 0 && out_bulk > 0) {
@@ -1122,8 +1126,9 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     const bool vec = (ld_in % 4 == 0) && (ld_out % 4 == 0) && aligned(W, 16) && aligned(W_out, 16);
     const int srow = (ncols_out + 3) & ~3;
     const size_t row_bytes = 4 * (size_t)srow;
-    LaunchScope ls("split_scatter_kernel", stream);
-    if (vec && (C * R) % 4 == 0 && 2 * row_bytes <= kRowSmemBytes) {
+    const bool staged = vec && (C * R) % 4 == 0 && 2 * row_bytes <= kRowSmemBytes;
+    LaunchScope ls(staged ? "split_rows_kernel" : "split_scatter_kernel", stream);
+    if (staged) {
       // rows per group: as many as fit in half the buffer space, but keep at least one group per SM
       long long g = (long long)(kRowSmemBytes / 2 / row_bytes);
       g = min(g, (long long)max(1, O / kNumSMs));

@@ -11,7 +11,7 @@ from ocs_inputs import configs
 from oracle import oracle as orc
 from paper_1901_09504_b200 import nets
 
-import net_oracle
+from oracle import net_oracle
 from gpu_util import dev, host
 
 pytestmark = pytest.mark.gpu

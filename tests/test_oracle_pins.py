@@ -572,3 +572,265 @@ def test_input_streams_are_reproducible_and_shaped():
     u = prng.Stream(9, 0).uniform(0, 100000)
     assert abs(u.mean() - 0.5) < 5e-3 and 0 < u.min() and u.max() < 1
     np.testing.assert_array_equal(prng.Stream(9, 0).bits(1000, 10), prng.Stream(9, 0).bits(0, 1010)[1000:])
+
+
+# ----------------------------------------------------------------------------- Section 4.1, element-wise scorer
+@pytest.mark.parametrize("bits,n_cand,seed", [(2, 8, 0), (3, 16, 1), (4, 16, 2), (3, 5, 3), (4, 7, 4)])
+def test_clip_mse_exact_bruteforce(bits, n_cand, seed):
+    """The element-wise scorer against an exact rational enumeration of every (threshold, element):
+    every element is its own 'bin' with count 1.  Values are small dyadic rationals, so the fp32
+    inputs are exact and only the candidates' fp32 rounding enters (reproduced by _brute_clip)."""
+    rng = np.random.default_rng(100 + seed)
+    vals = (rng.integers(-64, 65, size=40) / 32.0).astype(np.float32)
+    vals[7] = 2.0
+    vals[11] = -1.96875
+    m = Fraction(float(np.abs(vals).max()))
+    res = orc.clip_mse_exact(vals, bits, True, n_cand)
+    cbest, scores = _brute_clip([Fraction(float(v)) for v in vals], [1] * vals.size, m, bits, n_cand)
+    np.testing.assert_allclose(res["scores"], [float(s) for s in scores], rtol=1e-12, atol=1e-15)
+    gaps = sorted(float(s) for s in scores)
+    if gaps[1] - gaps[0] > 1e-9:
+        assert res["alpha"] == np.float32(float(m) * cbest / n_cand)
+    # unsigned codes: non-negative data, grid {0..2^k - 1}
+    uv = np.abs(vals)
+    resu = orc.clip_mse_exact(uv, bits, False, n_cand)
+    cb_u, sc_u = _brute_clip([Fraction(float(v)) for v in uv], [1] * uv.size, m, bits, n_cand, signed=False)
+    np.testing.assert_allclose(resu["scores"], [float(s) for s in sc_u], rtol=1e-12, atol=1e-15)
+
+
+# ----------------------------------------------------------------------------- Section 3.3, grid step of the QA split
+def test_split_qa_two_pass_rule_in_grid_units():
+    """Two-pass rule: the step is (max|W'| of a plain-halving run) / L.  The tensor is built so that this is
+    exactly 1.0 for 4-bit codes (L = 7); the QA pair of every split element must then satisfy the identity of
+    Section 3.3, Q((w - .5)/2) + Q((w + .5)/2) = Q(w) with Q = floor(x + 1/2), evaluated in exact rationals."""
+    rng = np.random.default_rng(31)
+    W = (rng.integers(-48, 49, size=(9, 12)) / 8.0).astype(np.float32)       # |w| <= 6
+    W[2, 3], W[5, 7], W[0, 10] = 13.5, -12.25, 9.75                          # three outlier channels
+    W[4, 1] = 7.0                                                            # the largest value left after 3 splits
+    S = 3
+    out, idx, order, mx, step = orc.split_qa(W, S, 4)
+    plain, _, order0, mx0 = orc.split(W, S, 0.0)
+    assert mx0[1] == 7.0 and step == 1.0                                     # predicted max / L
+    assert order.tolist() == order0.tolist() == [3, 7, 10]
+    ref, idx_r, order_r, mx_r = orc.split(W, S, 1.0)                          # same thing with the step given
+    np.testing.assert_array_equal(out, ref)
+    np.testing.assert_array_equal(idx, idx_r)
+    assert mx == mx_r
+    for s, ch in enumerate(order):
+        for o in range(W.shape[0]):
+            w, a, b = Fraction(float(W[o, ch])), Fraction(float(out[o, ch])), Fraction(float(out[o, 12 + s]))
+            assert a == (w - Fraction(1, 2)) / 2 and b == (w + Fraction(1, 2)) / 2
+            assert _Q(a) + _Q(b) == _Q(w)
+    # S = 0: the step is max|W| / L
+    _, _, _, mxz, stepz = orc.split_qa(W, 0, 4)
+    assert stepz == np.float32(13.5) / np.float32(7)
+
+
+# ----------------------------------------------------------------------------- Section 4.3 (KL)
+def _brute_kl(hist, m, L, n_cand, eps=1e-4):
+    """The divergence of every candidate, written out from the definition with exact integer level sums
+    (python ints / Fractions for the ratios, math.log on the final ratio)."""
+    B, n = len(hist), sum(hist)
+    scores = []
+    for c in range(1, n_cand + 1):
+        alpha = Fraction(float(np.float32(float(m) * c / n_cand)))
+        step = alpha / L
+        nc = -(-c * B // n_cand)
+        level = []
+        for i in range(nc):
+            t = Fraction(2 * i + 1, 2) * m / B / step
+            q = math.floor(t + Fraction(1, 2))
+            if t + Fraction(1, 2) == q and q % 2 == 1:
+                q -= 1
+            level.append(min(L, max(0, q)))
+        kept = sum(hist[:nc])
+        if kept == 0:
+            scores.append(math.inf)
+            continue
+        clipped = n - kept
+        P = [hist[i] + (clipped if i == nc - 1 else 0) for i in range(nc)]
+        mass, nnz = {}, {}
+        for i in range(nc):
+            mass[level[i]] = mass.get(level[i], 0) + hist[i]
+            nnz[level[i]] = nnz.get(level[i], 0) + (hist[i] > 0)
+        smooth = hist[nc - 1] == 0 and clipped > 0
+        kl = 0.0
+        for i in range(nc):
+            if P[i] == 0:
+                continue
+            p = Fraction(P[i], n)
+            if hist[i] == 0:
+                q = Fraction(eps)
+            else:
+                q = Fraction(mass[level[i]], nnz[level[i]] * kept)
+                if smooth:
+                    q = q * (1 - Fraction(eps))
+            kl += float(p) * math.log(p / q)
+        scores.append(kl)
+    return scores
+
+
+@pytest.mark.parametrize("bits,n_cand,B,seed", [(2, 8, 64, 0), (3, 16, 64, 1), (4, 16, 128, 2), (3, 5, 50, 3)])
+def test_clip_kl_bruteforce(bits, n_cand, B, seed):
+    rng = np.random.default_rng(200 + seed)
+    m = 2.0
+    counts = np.zeros(B, dtype=np.int64)
+    pick = np.unique(np.concatenate([rng.integers(0, B // 3, 30), rng.integers(0, B - 1, 8), [B - 1]]))
+    counts[pick] = rng.integers(1, 12, size=pick.size)
+    vals = []
+    for b in np.nonzero(counts)[0]:
+        vals += [(b + 0.5) * m / B] * int(counts[b])
+    vals = np.array(vals, dtype=np.float32)
+    vals[-1] = m
+    vals *= rng.choice([-1.0, 1.0], size=vals.size).astype(np.float32)
+    res = orc.clip_kl(vals, bits, True, n_bins=B, n_candidates=n_cand)
+    np.testing.assert_array_equal(res["hist"], counts.astype(np.uint64))
+    L = 2 ** (bits - 1) - 1
+    ref = _brute_kl([int(x) for x in counts], Fraction(2), L, n_cand)
+    np.testing.assert_allclose(res["scores"], ref, rtol=1e-11, atol=1e-14)
+    assert all(s >= -1e-15 for s in res["scores"])                       # a divergence
+    order = np.argsort(ref, kind="stable")
+    if ref[order[1]] - ref[order[0]] > 1e-9:
+        assert res["alpha"] == np.float32(2.0 * (order[0] + 1) / n_cand)
+    # the library's generic divergence routine on the same two distributions (one candidate, no empty last bin)
+    scipy_stats = pytest.importorskip("scipy.stats")
+    c = n_cand
+    P = counts.astype(np.float64)
+    lvl = np.clip(np.rint((np.arange(B) + 0.5) * (m / B) / (float(np.float32(m)) / L)), 0, L).astype(int)
+    mass = np.bincount(lvl, weights=P, minlength=L + 1)
+    nnz = np.bincount(lvl, weights=(P > 0).astype(float), minlength=L + 1)
+    Q = np.where(P > 0, mass[lvl] / np.maximum(nnz[lvl], 1), 0.0)
+    np.testing.assert_allclose(res["scores"][c - 1], scipy_stats.entropy(P, Q), rtol=1e-10, atol=1e-14)
+
+
+def test_clip_kl_properties():
+    # a tensor that already sits on the k-bit grid of its own maximum: quantizing it at the last candidate
+    # changes nothing, so the divergence there is exactly zero and the last candidate wins
+    for bits in (3, 4, 6):
+        L = 2 ** (bits - 1) - 1
+        rng = np.random.default_rng(bits)
+        codes = np.concatenate([rng.integers(-L, L + 1, 4000), [L, -L]])
+        x = (codes / L).astype(np.float32)
+        r = orc.clip_kl(x, bits, True, 2048, 128)
+        assert r["scores"][-1] == 0.0 and r["alpha"] == 1.0
+        assert (r["scores"][:-1] > 0).all()
+    # clipping is penalised through the mass that piles up in the last kept bin: with one far outlier
+    # and few bits the search clips, with many bits on clean data it does not clip much
+    rng = np.random.default_rng(9)
+    x = rng.laplace(0, 0.01, 60000).astype(np.float32)
+    x[5] = 1.0
+    r3 = orc.clip_kl(x, 3, True)
+    assert 0 < r3["alpha"] < 0.5
+    # scale covariance: powers of two change nothing but the scale
+    r3b = orc.clip_kl(x * np.float32(4.0), 3, True)
+    assert r3b["alpha"] == np.float32(4.0) * np.float32(r3["alpha"])
+    np.testing.assert_array_equal(r3b["scores"], r3["scores"])
+    assert orc.clip_kl(np.zeros(10, np.float32), 4)["alpha"] == 0.0
+
+
+# ----------------------------------------------------------------------------- Section 4.2 (ACIQ)
+def test_aciq_multipliers_closed_forms():
+    """The Laplace threshold is a Lambert-W value, the Gauss threshold the root of a monotone equation; both
+    minimise the model error (clipping noise + step^2/12).  With 2^M grid intervals they are the constants
+    the method's authors publish (Banner et al. 2018, the work Section 4.2 cites): 2.83 b, 3.89 b, 5.03 b and
+    1.71 s, 2.15 s, 2.56 s for M = 2, 3, 4."""
+    sp = pytest.importorskip("scipy.special")
+    so = pytest.importorskip("scipy.optimize")
+    ss = pytest.importorskip("scipy.stats")
+    for M, lap, gau in ((2, 2.83, 1.71), (3, 3.89, 2.15), (4, 5.03, 2.56)):
+        assert abs(orc.aciq_multiplier(2 ** M, True) - lap) < 0.01        # printed with two decimals
+        assert abs(orc.aciq_multiplier(2 ** M, False) - gau) < 0.01
+    for bits in range(2, 9):
+        for L in (2 ** (bits - 1) - 1, 2 ** bits - 1):
+            n_int = 2.0 * L
+            t = orc.aciq_multiplier(n_int, True)
+            assert abs(t - float(np.real(sp.lambertw(3 * n_int ** 2)))) < 1e-12 * t
+            lap_err = lambda a: 2 * math.exp(-a) + (2 * a / n_int) ** 2 / 12            # b = 1
+            opt = so.minimize_scalar(lap_err, bounds=(1e-3, 60), method="bounded", options=dict(xatol=1e-10))
+            assert abs(opt.x - t) < 1e-5 * t
+            g = orc.aciq_multiplier(n_int, False)
+            gau_err = lambda a: 2 * ((1 + a * a) * ss.norm.sf(a) - a * ss.norm.pdf(a)) + (2 * a / n_int) ** 2 / 12
+            optg = so.minimize_scalar(gau_err, bounds=(1e-3, 40), method="bounded", options=dict(xatol=1e-10))
+            assert abs(optg.x - g) < 1e-5 * g
+            # and the clipping-noise closed forms themselves, against numerical integration of (x - a)^2 f(x)
+            si = pytest.importorskip("scipy.integrate")
+            a = 1.7
+            num = 2 * si.quad(lambda x: (x - a) ** 2 * ss.norm.pdf(x), a, np.inf)[0]
+            assert abs(num - 2 * ((1 + a * a) * ss.norm.sf(a) - a * ss.norm.pdf(a))) < 1e-10
+            numl = 2 * si.quad(lambda x: (x - a) ** 2 * 0.5 * math.exp(-x), a, np.inf)[0]
+            assert abs(numl - 2 * math.exp(-a)) < 1e-10
+
+
+def test_clip_aciq_on_exact_laplace_and_gauss_samples():
+    """Deterministic quantile samples of the two densities: the fit recovers the scale, the likelihood test
+    picks the right density, alpha = multiplier * scale, and the measured quantization MSE of the sample at
+    that alpha is within a few percent of the best MSE over a fine sweep of thresholds."""
+    ss = pytest.importorskip("scipy.stats")
+    n = 200001
+    u = (np.arange(n) + 0.5) / n
+    for name, sample, scale_true in (("laplace", ss.laplace.ppf(u, scale=0.02), 0.02), ("gauss", ss.norm.ppf(u, scale=0.05), 0.05)):
+        x = sample.astype(np.float32)
+        for bits in (3, 4, 6):
+            L = 2 ** (bits - 1) - 1
+            r = orc.clip_aciq(x, bits, True, 2048)
+            assert r["laplace"] == (name == "laplace")
+            scale = r["b"] if name == "laplace" else r["sigma"]
+            assert abs(scale - scale_true) < 2e-3 * scale_true                   # histogram moments: bin-width error
+            assert r["multiplier"] == orc.aciq_multiplier(2 * L, name == "laplace")
+            expect = np.float32(r["multiplier"] * scale)
+            assert r["alpha"] == min(expect, np.float32(r["max_abs"]))
+
+            def mse(alpha):
+                codes, step = orc.quantize(x, bits, True, float(alpha))
+                return float(np.mean((x.astype(np.float64) - codes.astype(np.float64) * step) ** 2))
+            sweep = [mse(a) for a in np.linspace(0.3, 2.0, 35) * r["alpha"]]
+            assert mse(r["alpha"]) <= 1.10 * min(sweep)
+    # the threshold never exceeds the largest value; all-zero input
+    tiny = np.array([0.1, -0.1, 0.1, 0.1], np.float32)
+    assert orc.clip_aciq(tiny, 8, True)["alpha"] == np.float32(0.1)
+    assert orc.clip_aciq(np.zeros(8, np.float32), 4)["alpha"] == 0.0
+    # unsigned codes on non-negative data use L_u = 2^k - 1
+    xu = np.abs(ss.norm.ppf(u, scale=1.0)).astype(np.float32)
+    ru = orc.clip_aciq(xu, 4, False, 2048)
+    assert not ru["laplace"] and ru["multiplier"] == orc.aciq_multiplier(2 * 15, False)
+
+
+# ----------------------------------------------------------------------------- Section 3.4 (knapsack)
+def test_range_curve_follows_the_greedy_loop():
+    rng = np.random.default_rng(41)
+    for shape in ((8, 10), (6, 7, 3, 3)):
+        W = rng.laplace(0, 0.02, size=shape).astype(np.float32)
+        W.reshape(-1)[rng.integers(0, W.size, 4)] *= 25
+        curve = orc.range_curve(W, 9)
+        assert curve[0] == np.abs(W).max()
+        for s in range(10):
+            _, _, _, mx = orc.split(W, s, 0.0, literal=True)
+            assert curve[s] == np.float32(mx[1])
+        assert all(curve[s + 1] <= curve[s] for s in range(9))
+
+
+def test_knapsack_is_optimal_against_exhaustive_search():
+    import itertools
+    rng = np.random.default_rng(43)
+    for trial in range(6):
+        n_layers = int(rng.integers(3, 7))
+        curves, cost = [], []
+        for l in range(n_layers):
+            O, Cn, R = int(rng.integers(2, 6)) * 4, int(rng.integers(3, 7)), int(rng.choice([1, 9]))
+            W = rng.laplace(0, 0.02, size=(O, Cn * R)).astype(np.float32).reshape(O, Cn, R)
+            W.reshape(-1)[rng.integers(0, W.size, 2)] *= float(rng.uniform(3, 30))
+            curves.append(orc.range_curve(W, int(rng.integers(1, 4))))
+            cost.append(O * R)
+        budget = int(sum(c * (len(cv) - 1) for c, cv in zip(cost, curves)) * rng.uniform(0.2, 0.7))
+        S, total = orc.knapsack(curves, cost, budget)
+        assert sum(int(s) * c for s, c in zip(S, cost)) <= budget
+        assert all(0 <= s <= len(cv) - 1 for s, cv in zip(S, curves))
+        rew = lambda l, s: (Fraction(float(curves[l][0])) - Fraction(float(curves[l][s]))) / Fraction(float(curves[l][0]))
+        best = max(sum(rew(l, s) for l, s in enumerate(alloc))
+                   for alloc in itertools.product(*[range(len(cv)) for cv in curves])
+                   if sum(s * c for s, c in zip(alloc, cost)) <= budget)
+        got = sum(rew(l, int(s)) for l, s in enumerate(S))
+        assert abs(float(got - best)) < 1e-12 and abs(total - float(best)) < 1e-12
+    # zero budget: nothing is split; a budget that pays for everything: every layer takes what still helps
+    S0, t0 = orc.knapsack(curves, cost, 0)
+    assert not S0.any() and t0 == 0.0
