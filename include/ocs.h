@@ -53,7 +53,9 @@ typedef enum {
 typedef enum {
   OCS_CLIP_NONE = 0,     /* alpha = max|T| (Eq. 1) */
   OCS_CLIP_MSE = 1,      /* histogram MSE search (Section 4.1) */
-  OCS_CLIP_MSE_EXACT = 2 /* the same candidates scored on the elements themselves, no histogram */
+  OCS_CLIP_MSE_EXACT = 2,/* the same candidates scored on the elements themselves, no histogram */
+  OCS_CLIP_KL = 3,       /* KL-divergence search on the same histogram and candidates (Section 4.3) */
+  OCS_CLIP_ACIQ = 4      /* Laplace-or-Gauss fit and closed-form threshold (Section 4.2) */
 } ocs_clip_mode;
 
 /* Host helpers ------------------------------------------------------------------------- */
@@ -124,6 +126,24 @@ ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_in, int S, 
  *   score_c = sum_i (x_i - Q_c(x_i))^2 over the elements, in double (the MSE of Section 4.1
  *   without the histogram approximation; bound by fp64 arithmetic, not by memory).  For this
  *   mode n_bins is ignored and the workspace query is called with n_bins = 0.
+ *   mode KL (Section 4.3; the paper names the ingredients -- histogram, candidates, divergence
+ *   between the float and the quantized distribution, a little mass moved into empty bins --
+ *   the details here are this library's): same histogram and candidates as MSE.  Candidate c
+ *   keeps the first n_c = ceil(c*n_bins/n_candidates) bins.  P = their counts, with the count of
+ *   everything beyond added to the last one, over the total count.  Q = their counts alone,
+ *   grouped by the code of the bin centre (clamp(rint(x_b/step_c), 0, L)), each group's count
+ *   spread evenly over its non-empty bins, over the kept count; if the last kept bin is empty but
+ *   receives clipped mass, Q is 1e-4 there and scaled by (1 - 1e-4) elsewhere.  score_c =
+ *   sum over bins with P > 0 of P*ln(P/Q) in double; smallest wins, ties to the largest alpha;
+ *   a candidate that keeps no value scores +infinity.
+ *   mode ACIQ (Section 4.2: decide between a Gaussian and a Laplacian, then an approximate
+ *   closed form for the MSE-optimal threshold; the details are this library's): from the same
+ *   histogram, b = mean|x| and s = sqrt(mean x^2) at the bin centres (exact integer sums; up to
+ *   2^38 values); Laplace if b/s < sqrt(pi/2e) (the density with the larger likelihood at its own
+ *   fit), else Gauss; alpha = t*b resp. t*s, capped at max|T|, where t minimises
+ *   (clipping noise of the density) + step^2/12 for the grid of 2L intervals the codes span:
+ *   t*exp(t) = 12 L^2 for Laplace, 4*(phi(t) - t*Qf(t)) = t/(6 L^2) for Gauss.  n_candidates is
+ *   ignored (the workspace query takes 1).
  * T [rows][cols] fp32 with row stride ld_in; codes [rows][cols] with row stride ld_codes bytes
  * (bytes beyond cols in a row are left untouched).  max_abs_in (nullable): device scalar
  * holding max|T| if the caller already has it (saves one pass over T).  *scale = step,
@@ -144,7 +164,7 @@ ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, int64_t ld_i
  * being read and written five times.  Results are bit-identical to the two separate calls:
  * codes int8 [O][(C+S)*R] in the split's layout with row stride ld_codes bytes, idx_map,
  * split_order (nullable), max_abs_out [3] (nullable), *scale, *alpha (nullable).
- * Arguments as in ocs_split and ocs_quantize (modes NONE and MSE).
+ * Arguments as in ocs_split and ocs_quantize (modes NONE, MSE, KL and ACIQ).
  * Applied to an ACTIVATION matrix [rows][C] (R = 1, qa_bits = 0) this is the activation side
  * of Eq. 4 with channels chosen on the batch at hand (the per-batch selection of Section 5.3):
  * the chosen channels are duplicated and halved, and the codes come out already expanded,
@@ -231,8 +251,9 @@ ocs_status ocs_act_split_quantize_static(const float* A, int rows, int C, int64_
  * The scratch (48 KB: running maximum, histogram, candidate scores) is a fixed array inside the
  * library's device image, so every GPU that loads the library carries it until the process
  * exits.  The call allocates nothing and frees nothing.
- * Limits: modes OCS_CLIP_NONE and OCS_CLIP_MSE with n_bins <= 4096 and n_candidates <= 1024;
- * anything larger, and OCS_CLIP_MSE_EXACT, returns OCS_ERR_UNSUPPORTED (use ocs_quantize).
+ * Limits: modes OCS_CLIP_NONE, OCS_CLIP_MSE, OCS_CLIP_KL and OCS_CLIP_ACIQ with n_bins <= 4096
+ * and n_candidates <= 1024; anything larger, and OCS_CLIP_MSE_EXACT, returns
+ * OCS_ERR_UNSUPPORTED (use ocs_quantize).
  * The first call on each device looks up the array's device address (with that device
  * current) and remembers it; make that first call before starting any stream capture.
  * All calls on a device share the one array, which keeps whatever the previous call left: each

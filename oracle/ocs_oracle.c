@@ -407,7 +407,8 @@ double ocs_oracle_aciq_multiplier(double n_intervals, int laplace) {
 
 /* Reading taken (the paper gives no formula): the two candidate densities are zero-location and
  * are fitted to the histogram of |x| (same bins as the other searches, bin centres x_i):
- * b = sum h x_i / n, s = sqrt(sum h x_i^2 / n), sums in double, bins ascending.  The density with
+ * b = sum h x_i / n, s = sqrt(sum h x_i^2 / n), the sums taken exactly in integers (x_i is an odd
+ * multiple of half a bin width; n up to 2^38 values).  The density with
  * the larger likelihood at its own fit is taken: Laplace iff b / s < sqrt(pi / (2 e)).
  * alpha = multiplier(2 L) * (b or s), rounded to fp32, and never above max|x|.
  * stats (nullable) = {b, s, 1 if Laplace else 0, multiplier}. */
@@ -427,18 +428,19 @@ int ocs_oracle_clip_aciq(const float* T, int64_t n, int bits, int is_signed, int
   uint64_t* h = abs_histogram(T, n, B, m);
   if (!h) return 2;
   if (hist) memcpy(hist, h, sizeof(uint64_t) * (size_t)B);
+  /* moments of the bin centres x_i = (2i + 1) * width / 2 as exact integer sums (order-free):
+   * sum h x_i = I1 * width / 2, sum h x_i^2 = I2 * width^2 / 4 */
   const double width = (double)m / (double)B;
-  double cnt = 0.0, s1 = 0.0, s2 = 0.0;
+  uint64_t cnt = 0, I1 = 0, I2 = 0;
   for (int b = 0; b < B; ++b) {
-    const double xb = ((double)b + 0.5) * width;
-    const double hb = (double)h[b];
-    cnt += hb;
-    s1 += hb * xb;
-    s2 += hb * xb * xb;
+    const uint64_t odd = 2u * (uint64_t)b + 1u;
+    cnt += h[b];
+    I1 += h[b] * odd;
+    I2 += h[b] * odd * odd;
   }
   free(h);
-  const double bb = s1 / cnt;
-  const double sd = sqrt(s2 / cnt);
+  const double bb = ((double)I1 / (2.0 * (double)cnt)) * width;
+  const double sd = sqrt((double)I2 / (4.0 * (double)cnt)) * width;
   const int laplace = bb / sd < sqrt(M_PI / (2.0 * M_E));
   const double mult = ocs_oracle_aciq_multiplier(2.0 * (double)L, laplace);
   float a = (float)(mult * (laplace ? bb : sd));

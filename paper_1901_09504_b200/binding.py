@@ -20,7 +20,7 @@ OCS_OK = 0
 STATUS_NAMES = {0: "OCS_OK", 1: "OCS_ERR_INVALID_ARG", 2: "OCS_ERR_SHAPE", 3: "OCS_ERR_WORKSPACE",
                 4: "OCS_ERR_UNSUPPORTED", 5: "OCS_ERR_CUDA"}
 DEV_NONFINITE, DEV_BAD_INDEX, DEV_TIMEOUT, DEV_DEPTH, DEV_OVERFLOW = 1, 2, 4, 8, 16
-CLIP_NONE, CLIP_MSE, CLIP_MSE_EXACT = 0, 1, 2
+CLIP_NONE, CLIP_MSE, CLIP_MSE_EXACT, CLIP_KL, CLIP_ACIQ = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
@@ -175,6 +175,8 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
         alpha = torch.empty(1, dtype=torch.float32, device=T.device)
     if mode == CLIP_MSE_EXACT:
         n_bins = 0
+    if mode == CLIP_ACIQ:
+        n_candidates = 1
     nws = lib().ocs_quantize_workspace_bytes(int(n_bins), int(n_candidates))
     if ws is None:
         ws = _ws(nws, T.device)

@@ -68,9 +68,11 @@ struct LaunchScope {
   ~LaunchScope() { trace_end(record, stream); }
 };
 
-// One CTA per candidate threshold of the MSE clip search (defined in quantize.cu).
-ocs_status launch_score_kernel(const unsigned long long* hist, const float* maxp, int n_bins, int n_candidates, int L,
-                               int is_signed, double* scores, cudaStream_t stream);
+// The clip search that follows the histogram of |x| (defined in quantize.cu): candidate scores for the MSE and
+// KL searches, or the closed-form threshold of ACIQ written to *alpha_sel.
+ocs_status launch_clip_search(ocs_clip_mode mode, const unsigned long long* hist, const float* maxp, int n_bins,
+                              int n_candidates, int L, int is_signed, double* scores, float* alpha_sel,
+                              cudaStream_t stream);
 
 #ifdef __CUDACC__
 // The search's winner: smallest score, ties to the largest threshold.  Every CTA of the quantize

@@ -5,6 +5,9 @@
 //   maxabs_kernel     max|x|, combined with atomicMax on the bits of the non-negative value
 //   hist_kernel       histogram of |x| in privatised shared-memory counters, flushed with 64-bit atomics
 //   score_kernel      one CTA per candidate threshold: sum_b h[b]*(x_b - Q(x_b))^2 in double
+//   kl_score_kernel   one CTA per candidate threshold: KL divergence between the kept part of the histogram
+//                     (clipped mass added to its last bin) and its quantized-and-expanded form (Section 4.3)
+//   aciq_kernel       Laplace-or-Gauss fit to the histogram and the closed-form threshold (Section 4.2)
 //   quantize_kernel   picks the winning threshold (smallest score, ties to the largest threshold), then
 //                     code = clamp(rint(x * L/alpha)), round-half-to-even, saturating
 #include "common.cuh"
@@ -189,6 +192,124 @@ score_kernel(const unsigned long long* __restrict__ hist, const float* __restric
     __syncthreads();
   }
   if (threadIdx.x == 0) scores[blockIdx.x] = red[0];
+}
+
+// Section 4.3, KL divergence search on the histogram of |x| and the candidate list of the MSE search.
+// Candidate c keeps the first n_c = ceil(c * n_bins / n_candidates) bins.  P = their counts, the clipped count
+// added to the last one (clipped values saturate there), over the total; Q = their counts alone, grouped by the
+// quantization level of the bin centre (level = clamp(rint(x_b / step_c), 0, L)) and spread back evenly over each
+// level's non-empty bins, over the kept count.  Q can only be zero where P is not in the last kept bin (empty
+// itself but receiving clipped mass): that bin then gets kEps of Q's mass and the rest is scaled by 1 - kEps.
+// score_c = sum_{P > 0} P ln(P / Q).  Level sums are integers (exact, order-free); the terms are added in a fixed
+// per-thread order and a fixed tree.  A candidate that keeps nothing scores +infinity.
+constexpr int kMaxLevels = 256;
+constexpr double kKlEps = 1e-4;
+
+__global__ void __launch_bounds__(256)
+kl_score_kernel(const unsigned long long* __restrict__ hist, const float* __restrict__ maxp, int n_bins,
+                int n_candidates, int L, double* __restrict__ scores) {
+  __shared__ unsigned long long level_count[kMaxLevels];
+  __shared__ int level_bins[kMaxLevels];
+  __shared__ unsigned long long red_u[2][8];
+  __shared__ double red[256];
+  const int c = blockIdx.x + 1;
+  const float m = *maxp;
+  if (!(m > 0.0f)) {
+    if (threadIdx.x == 0) scores[blockIdx.x] = 0.0;
+    return;
+  }
+  const float alpha_c = __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)c), (double)n_candidates));
+  const double step = __ddiv_rn((double)alpha_c, (double)L);
+  const double width = __ddiv_rn((double)m, (double)n_bins);
+  int nc = (int)(((long long)c * n_bins + n_candidates - 1) / n_candidates);
+  nc = max(1, min(nc, n_bins));
+  for (int j = threadIdx.x; j <= L; j += 256) { level_count[j] = 0ull; level_bins[j] = 0; }
+  __syncthreads();
+  unsigned long long tot = 0ull, kept = 0ull;
+  for (int b = threadIdx.x; b < n_bins; b += 256) {
+    const unsigned long long h = hist[b];
+    tot += h;
+    if (b < nc) {
+      kept += h;
+      const double xb = __dmul_rn(__dadd_rn((double)b, 0.5), width);
+      const int lvl = (int)fmin(fmax(rint(__ddiv_rn(xb, step)), 0.0), (double)L);
+      if (h) { atomicAdd(&level_count[lvl], h); atomicAdd(&level_bins[lvl], 1); }
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    tot += __shfl_xor_sync(0xffffffffu, tot, o);
+    kept += __shfl_xor_sync(0xffffffffu, kept, o);
+  }
+  if ((threadIdx.x & 31) == 0) { red_u[0][threadIdx.x >> 5] = tot; red_u[1][threadIdx.x >> 5] = kept; }
+  __syncthreads();
+  tot = 0ull; kept = 0ull;
+  for (int w = 0; w < 8; ++w) { tot += red_u[0][w]; kept += red_u[1][w]; }
+  if (kept == 0ull) {
+    if (threadIdx.x == 0) scores[blockIdx.x] = INFINITY;
+    return;
+  }
+  const unsigned long long clipped = tot - kept;
+  const bool smooth = hist[nc - 1] == 0ull && clipped > 0ull;
+  double acc = 0.0;
+  for (int b = threadIdx.x; b < nc; b += 256) {
+    const unsigned long long h = hist[b];
+    const unsigned long long pb = h + (b == nc - 1 ? clipped : 0ull);
+    if (pb == 0ull) continue;
+    const double p = __ddiv_rn((double)pb, (double)tot);
+    double q;
+    if (h == 0ull) {
+      q = kKlEps;
+    } else {
+      const double xb = __dmul_rn(__dadd_rn((double)b, 0.5), width);
+      const int lvl = (int)fmin(fmax(rint(__ddiv_rn(xb, step)), 0.0), (double)L);
+      q = __ddiv_rn(__ddiv_rn((double)level_count[lvl], (double)level_bins[lvl]), (double)kept);
+      if (smooth) q = __dmul_rn(q, 1.0 - kKlEps);
+    }
+    acc = __dadd_rn(acc, __dmul_rn(p, log(__ddiv_rn(p, q))));
+  }
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  for (int sft = 128; sft > 0; sft >>= 1) {
+    if (threadIdx.x < sft) red[threadIdx.x] = __dadd_rn(red[threadIdx.x], red[threadIdx.x + sft]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) scores[blockIdx.x] = red[0];
+}
+
+// Section 4.2 (ACIQ).  Zero-location Laplace and Gauss densities are fitted to the histogram of |x| through the
+// bin centres x_b = (2b + 1) * width / 2: b_fit = mean |x|, s_fit = sqrt(mean x^2), with the sums taken exactly in
+// integers (I1 = sum h (2b+1), I2 = sum h (2b+1)^2: order-free).  The density with the larger likelihood at its own
+// fit wins (Laplace iff b_fit / s_fit < sqrt(pi / 2e)); alpha = multiplier * scale, capped at max|x|, where the
+// multiplier minimises clipping noise + step^2/12 for a grid of 2L intervals (solved on the host: it depends on
+// L only).  One CTA.
+__global__ void __launch_bounds__(256)
+aciq_kernel(const unsigned long long* __restrict__ hist, const float* __restrict__ maxp, int n_bins,
+            double mult_laplace, double mult_gauss, float* __restrict__ alpha_sel) {
+  __shared__ unsigned long long red_u[3][8];
+  const float m = *maxp;
+  unsigned long long cnt = 0ull, i1 = 0ull, i2 = 0ull;
+  for (int b = threadIdx.x; b < n_bins; b += 256) {
+    const unsigned long long h = hist[b], odd = 2ull * (unsigned long long)b + 1ull;
+    cnt += h; i1 += h * odd; i2 += h * odd * odd;
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    i1 += __shfl_xor_sync(0xffffffffu, i1, o);
+    i2 += __shfl_xor_sync(0xffffffffu, i2, o);
+  }
+  if ((threadIdx.x & 31) == 0) { red_u[0][threadIdx.x >> 5] = cnt; red_u[1][threadIdx.x >> 5] = i1; red_u[2][threadIdx.x >> 5] = i2; }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  cnt = 0ull; i1 = 0ull; i2 = 0ull;
+  for (int w = 0; w < 8; ++w) { cnt += red_u[0][w]; i1 += red_u[1][w]; i2 += red_u[2][w]; }
+  if (!(m > 0.0f) || cnt == 0ull) { *alpha_sel = m > 0.0f ? m : 0.0f; return; }
+  const double width = __ddiv_rn((double)m, (double)n_bins);
+  const double bfit = __dmul_rn(__ddiv_rn((double)i1, __dmul_rn(2.0, (double)cnt)), width);
+  const double sfit = __dmul_rn(sqrt(__ddiv_rn((double)i2, __dmul_rn(4.0, (double)cnt))), width);
+  const bool laplace = __ddiv_rn(bfit, sfit) < 0.7601734505331404;   // sqrt(pi / (2 e))
+  float a = __double2float_rn(laplace ? __dmul_rn(mult_laplace, bfit) : __dmul_rn(mult_gauss, sfit));
+  if (!(a < m)) a = m;
+  *alpha_sel = a;
 }
 
 // The same candidates scored on the elements themselves (no histogram): score_c = sum_i (x_i - Q_c(x_i))^2
@@ -384,6 +505,7 @@ small_quantize_kernel(const float* __restrict__ T, int rows, int cols, long long
 
 struct QuantWs {
   unsigned int* maxbits;       // fp32 bits of max|T|
+  float* alpha_sel;            // ACIQ: the chosen threshold (same 256-byte slot as maxbits)
   unsigned long long* hist;
   double* scores;
   double* partial;             // exact scorer only: [kExactMaxGrid][n_candidates]
@@ -399,6 +521,7 @@ QuantWs carve_quant_ws(void* ws, int n_bins, int n_candidates) {
     return p;
   };
   w.maxbits = reinterpret_cast<unsigned int*>(take(256));
+  w.alpha_sel = w.maxbits ? reinterpret_cast<float*>(w.maxbits) + 16 : nullptr;
   w.hist = reinterpret_cast<unsigned long long*>(take(8 * (size_t)(n_bins > 0 ? n_bins : 1)));
   w.scores = reinterpret_cast<double*>(take(8 * (size_t)(n_candidates > 0 ? n_candidates : 1)));
   if (n_bins == 0)  // the exact scorer's layout
@@ -409,11 +532,70 @@ QuantWs carve_quant_ws(void* ws, int n_bins, int n_candidates) {
 
 }  // namespace
 
-ocs_status launch_score_kernel(const unsigned long long* hist, const float* maxp, int n_bins, int n_candidates, int L,
-                               int is_signed, double* scores, cudaStream_t stream) {
-  LaunchScope ls("score_kernel", stream);
-  score_kernel<<<n_candidates, 256, 0, stream>>>(hist, maxp, n_bins, n_candidates, L, is_signed, scores);
-  return launch_status();
+namespace {
+// alpha / scale that minimises (clipping noise of the fitted density) + step^2 / 12 for a uniform grid of
+// n_int steps across [-alpha, alpha] (Section 4.2; step = 2 alpha / n_int, z = 3 n_int^2).
+//   Laplace(0, b): noise 2 b^2 exp(-t), t = alpha / b; stationary point t exp(t) = z, i.e. t = W(z): Halley's
+//                  iteration on w exp(w) - z.
+//   Gauss(0, s):   noise 2 [(1 + t^2) Qf(t) - t phi(t)] s^2; stationary point F(t) = 4 [phi(t) - t Qf(t)] - 2 t / z
+//                  = 0 with F' = -4 Qf(t) - 2 / z < 0: Newton steps kept inside a shrinking bracket.
+double aciq_multiplier_host(double n_int, bool laplace) {
+  const double z = 3.0 * n_int * n_int;
+  if (laplace) {
+    double w = log(z) - log(log(z) > 1.0 ? log(z) : 1.0);   // first terms of W's expansion for large z
+    if (!(w > 0.1)) w = 0.5;
+    for (int it = 0; it < 64; ++it) {
+      const double ew = exp(w), f = w * ew - z;
+      const double wn = w - f / (ew * (w + 1.0) - (w + 2.0) * f / (2.0 * w + 2.0));
+      if (fabs(wn - w) <= 4e-16 * fabs(wn)) { w = wn; break; }
+      w = wn;
+    }
+    return w;
+  }
+  double lo = 0.0, hi = 40.0, t = 2.0;
+  const double inv_sqrt_2pi = 0.3989422804014327, inv_sqrt2 = 0.7071067811865476;
+  for (int it = 0; it < 200; ++it) {
+    const double tail = 0.5 * erfc(t * inv_sqrt2);
+    const double f = 4.0 * (inv_sqrt_2pi * exp(-0.5 * t * t) - t * tail) - 2.0 * t / z;
+    if (f > 0.0) lo = t; else hi = t;
+    double tn = t - f / (-4.0 * tail - 2.0 / z);
+    if (!(tn > lo && tn < hi)) tn = 0.5 * (lo + hi);
+    if (fabs(tn - t) <= 4e-16 * fabs(tn)) { t = tn; break; }
+    t = tn;
+  }
+  return t;
+}
+}  // namespace
+
+// The clip search that follows the histogram: fills scores (MSE, KL) or *alpha_sel (ACIQ).
+ocs_status launch_clip_search(ocs_clip_mode mode, const unsigned long long* hist, const float* maxp, int n_bins,
+                              int n_candidates, int L, int is_signed, double* scores, float* alpha_sel,
+                              cudaStream_t stream) {
+  if (mode == OCS_CLIP_MSE) {
+    LaunchScope ls("score_kernel", stream);
+    score_kernel<<<n_candidates, 256, 0, stream>>>(hist, maxp, n_bins, n_candidates, L, is_signed, scores);
+    return launch_status();
+  }
+  if (mode == OCS_CLIP_KL) {
+    LaunchScope ls("kl_score_kernel", stream);
+    kl_score_kernel<<<n_candidates, 256, 0, stream>>>(hist, maxp, n_bins, n_candidates, L, scores);
+    return launch_status();
+  }
+  if (mode == OCS_CLIP_ACIQ) {
+    // the multipliers depend on the code range only: solved once per L on the host
+    static double cache[2][256];
+    static bool have[256] = {false};
+    if (L < 1 || L > 255) return OCS_ERR_INVALID_ARG;
+    if (!have[L]) {
+      cache[0][L] = aciq_multiplier_host(2.0 * L, true);
+      cache[1][L] = aciq_multiplier_host(2.0 * L, false);
+      have[L] = true;
+    }
+    LaunchScope ls("aciq_kernel", stream);
+    aciq_kernel<<<1, 256, 0, stream>>>(hist, maxp, n_bins, cache[0][L], cache[1][L], alpha_sel);
+    return launch_status();
+  }
+  return OCS_ERR_INVALID_ARG;
 }
 
 }  // namespace ocs
@@ -438,8 +620,12 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
   cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
   if (!T || !codes || !scale) return OCS_ERR_INVALID_ARG;
   if (bits < 2 || bits > 8) return OCS_ERR_INVALID_ARG;
-  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE && mode != OCS_CLIP_MSE_EXACT) return OCS_ERR_INVALID_ARG;
-  if (mode == OCS_CLIP_MSE && (n_candidates < 1 || n_candidates > kMaxCandidates || n_bins < 1 || n_bins > kMaxBins))
+  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE && mode != OCS_CLIP_MSE_EXACT && mode != OCS_CLIP_KL &&
+      mode != OCS_CLIP_ACIQ)
+    return OCS_ERR_INVALID_ARG;
+  const bool hist_mode = mode == OCS_CLIP_MSE || mode == OCS_CLIP_KL || mode == OCS_CLIP_ACIQ;
+  if (mode == OCS_CLIP_ACIQ) n_candidates = 1;   // no candidate list
+  if (hist_mode && (n_candidates < 1 || n_candidates > kMaxCandidates || n_bins < 1 || n_bins > kMaxBins))
     return OCS_ERR_INVALID_ARG;
   if (mode == OCS_CLIP_MSE_EXACT && (n_candidates < 1 || n_candidates > kMaxCandidates)) return OCS_ERR_INVALID_ARG;
   if (mode == OCS_CLIP_MSE_EXACT) n_bins = 0;
@@ -480,7 +666,7 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
     maxp = reinterpret_cast<const float*>(w.maxbits);
   }
   const double* scores = nullptr;
-  if (mode == OCS_CLIP_MSE) {
+  if (hist_mode) {
     if (cudaMemsetAsync(w.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
     {
       const size_t smem = sizeof(unsigned int) * kHistCopies * n_bins;
@@ -488,12 +674,11 @@ extern "C" ocs_status ocs_quantize(const float* T, int64_t rows, int64_t cols, i
       hist_kernel<<<grid_for(hist_kernel, v.tiles, smem), 256, smem, stream>>>(v, maxp, n_bins, w.hist);
     }
     if ((st = launch_status()) != OCS_OK) return st;
-    {
-      LaunchScope ls("score_kernel", stream);
-      score_kernel<<<n_candidates, 256, 0, stream>>>(w.hist, maxp, n_bins, n_candidates, L, is_signed, w.scores);
-    }
-    if ((st = launch_status()) != OCS_OK) return st;
-    scores = w.scores;
+    if ((st = launch_clip_search(mode, w.hist, maxp, n_bins, n_candidates, L, is_signed ? 1 : 0, w.scores, w.alpha_sel,
+                                 stream)) != OCS_OK)
+      return st;
+    if (mode == OCS_CLIP_ACIQ) maxp = w.alpha_sel;   // the threshold itself; nothing left to pick
+    else scores = w.scores;
   } else if (mode == OCS_CLIP_MSE_EXACT) {
     const long long n_tiles = (v.rows * v.cols + kExactTile - 1) / kExactTile;
     const int grid = (int)(n_tiles < kExactMaxGrid ? n_tiles : kExactMaxGrid);
@@ -546,8 +731,10 @@ extern "C" ocs_status ocs_quantize_noalloc(const float* T, int64_t rows, int64_t
                                            const float* max_abs_in, int8_t* codes, int64_t ld_codes, float* scale,
                                            float* alpha, int* dev_status, void* stream) {
   if (mode == OCS_CLIP_MSE_EXACT) return OCS_ERR_UNSUPPORTED;   // its partial sums need megabytes
-  if (mode == OCS_CLIP_MSE && (n_bins > kMaxBins || n_candidates > kMaxCandidates)) return OCS_ERR_UNSUPPORTED;
-  const int nb = mode == OCS_CLIP_MSE ? n_bins : 1, nc = mode == OCS_CLIP_MSE ? n_candidates : 1;
+  const bool searched = mode == OCS_CLIP_MSE || mode == OCS_CLIP_KL || mode == OCS_CLIP_ACIQ;
+  if (mode == OCS_CLIP_ACIQ) n_candidates = 1;
+  if (searched && (n_bins > kMaxBins || n_candidates > kMaxCandidates)) return OCS_ERR_UNSUPPORTED;
+  const int nb = searched ? n_bins : 1, nc = searched ? n_candidates : 1;
   if (ocs_quantize_workspace_bytes(nb, nc) > kStaticScratchBytes) return OCS_ERR_UNSUPPORTED;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return OCS_ERR_CUDA;

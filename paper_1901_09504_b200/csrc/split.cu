@@ -1371,8 +1371,11 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
   if (S < 0 || !(qa_step >= 0.0f) || !is_finite_host(qa_step)) return OCS_ERR_INVALID_ARG;
   if (qa_bits != 0 && (qa_bits < 2 || qa_bits > 8)) return OCS_ERR_INVALID_ARG;
   if (bits < 2 || bits > 8) return OCS_ERR_INVALID_ARG;
-  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE) return OCS_ERR_INVALID_ARG;
-  if (mode == OCS_CLIP_MSE && (n_candidates < 1 || n_candidates > 1024 || n_bins < 1 || n_bins > 4096))
+  if (mode != OCS_CLIP_NONE && mode != OCS_CLIP_MSE && mode != OCS_CLIP_KL && mode != OCS_CLIP_ACIQ)
+    return OCS_ERR_INVALID_ARG;
+  const bool hist_mode = mode != OCS_CLIP_NONE;
+  if (mode == OCS_CLIP_ACIQ) n_candidates = 1;
+  if (hist_mode && (n_candidates < 1 || n_candidates > 1024 || n_bins < 1 || n_bins > 4096))
     return OCS_ERR_INVALID_ARG;
   if (O <= 0 || C <= 0 || R <= 0) return OCS_ERR_SHAPE;
   if ((int64_t)C * R >= (1ll << 31) || ((int64_t)C + S) * R >= (1ll << 31)) return OCS_ERR_SHAPE;
@@ -1382,7 +1385,7 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
   // rows are staged whole in shared memory: they must be 16-byte addressable and fit twice
   const int srow = (ncols_out + 3) & ~3;
   const size_t row_bytes = 4 * (size_t)srow;
-  const size_t hist_bytes = mode == OCS_CLIP_MSE ? 4 * (size_t)n_bins : 0;
+  const size_t hist_bytes = hist_mode ? 4 * (size_t)n_bins : 0;
   if (!(ld_in % 4 == 0 && aligned(W, 16) && (C * R) % 4 == 0 && 2 * row_bytes + hist_bytes <= kRowSmemBytes))
     return OCS_ERR_UNSUPPORTED;
   const FusedWs f = carve_fused_ws(ws, C, R, S, n_bins, n_candidates);
@@ -1406,7 +1409,7 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
   ep.L = L;
   ep.is_signed = is_signed ? 1 : 0;
   const double* scores = nullptr;
-  if (mode == OCS_CLIP_MSE) {
+  if (hist_mode) {
     if (cudaMemsetAsync(f.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
     ep.n_bins = n_bins;
     ep.hist = f.hist;
@@ -1420,8 +1423,11 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
           ep, dev_status);
     }
     if ((st = launch_status()) != OCS_OK) return st;
-    if ((st = launch_score_kernel(f.hist, ep.maxp, n_bins, n_candidates, L, is_signed ? 1 : 0, f.scores, stream)) != OCS_OK) return st;
-    scores = f.scores;
+    if ((st = launch_clip_search(mode, f.hist, ep.maxp, n_bins, n_candidates, L, is_signed ? 1 : 0, f.scores,
+                                 f.mx3 + 8, stream)) != OCS_OK)
+      return st;
+    if (mode == OCS_CLIP_ACIQ) ep.maxp = f.mx3 + 8;   // the closed-form threshold replaces max|W'|
+    else scores = f.scores;
   }
   ep.scores = scores;
   ep.n_candidates = n_candidates;

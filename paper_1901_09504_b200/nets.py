@@ -41,7 +41,7 @@ def prepare_layer(W, bias, ratio: float, bits: int, clip_mode: int = B.CLIP_NONE
     S = B.ocs_num_splits(Cn, ratio)
     try:
         # one call, no fp32 W' (rows that cannot be staged in shared memory are reported as unsupported)
-        if clip_mode not in (B.CLIP_NONE, B.CLIP_MSE):
+        if clip_mode not in (B.CLIP_NONE, B.CLIP_MSE, B.CLIP_KL, B.CLIP_ACIQ):
             raise B.OcsError("ocs_split_quantize", 4)
         codes, scale, _, idx_map, _, _ = B.ocs_split_quantize(W.contiguous(), S, bits, clip_mode, qa_bits=qa_bits,
                                                               n_candidates=n_candidates, n_bins=n_bins,

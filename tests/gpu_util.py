@@ -20,10 +20,11 @@ def L_of(bits, signed=True):
 
 
 def oracle_split(W, S, qa_bits=0, qa_step=0.0, literal=False):
-    """The checker's split, with the two-pass grid-step rule when qa_bits is given."""
+    """The checker's split; with qa_bits the grid step comes from the checker's two-pass rule (split_qa)."""
     if qa_bits:
-        _, _, _, mx = orc.split(W, S, 0.0, literal=literal)
-        qa_step = float(np.float32(mx[1]) / np.float32(L_of(qa_bits)))
+        out, idx, order, mx, qa_step = orc.split_qa(W, S, qa_bits)
+        if not literal:
+            return out, idx, order, mx, qa_step
     out, idx, order, mx = orc.split(W, S, qa_step, literal=literal)
     return out, idx, order, mx, qa_step
 
@@ -49,3 +50,13 @@ def check_split(W, S, qa_bits=0, qa_step=0.0, ld_out=None, literal=False):
     assert g_mx[0] == np.float32(o_mx[0]) and g_mx[1] == np.float32(o_mx[1])
     assert g_mx[2] == np.float32(step)
     return o_out, o_idx, raw
+
+
+def clear_winner(scores, rel=1e-9):
+    """True when the smallest candidate score beats the runner-up by more than the rounding the two sides'
+    different summation orders can cause.  Only then is the chosen threshold a function of the scores that
+    both sides must agree on; a near-tie may legitimately flip and is compared through its scores alone."""
+    s = np.sort(np.asarray(scores, dtype=np.float64)[np.isfinite(scores)])
+    if s.size < 2:
+        return True
+    return (s[1] - s[0]) > rel * max(abs(s[1]), 1e-300)
