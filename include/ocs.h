@@ -114,6 +114,33 @@ ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_in, int S, 
                      int32_t* split_order, float* max_abs_out, void* ws, size_t ws_bytes,
                      int* dev_status, void* stream);
 
+/* ocs_range_curve / ocs_knapsack_allocate ---------------------------------------------------
+ * Section 3.4's second way of deciding how many channels each layer may add: instead of
+ * ceil(r*C) per layer, the counts of all layers are chosen together as a knapsack problem whose
+ * reward is the relative reduction of a layer's dynamic range and whose cost is the memory the
+ * extra channels take, under one overall memory constraint.
+ *   ocs_range_curve: curve (device, fp32 [S_max+1]), curve[s] = max|W'| after s steps of the
+ *   greedy loop with plain halving (curve[0] = max|W|).  W, O, C, R, ld_in as in ocs_split.  One
+ *   pass over W plus the split plan on channel maxima.  Device flag: NONFINITE.
+ *   ocs_knapsack_allocate: n_layers layers; curves (device) holds their curves back to back,
+ *   layer l at element curve_off[l] with s_max[l]+1 entries; unit_cost[l] = weight elements one
+ *   more input channel adds to layer l (O*R); curve_off, s_max, unit_cost are HOST arrays, read
+ *   before the call returns.  reward_l(s) = (curve_l[0] - curve_l[s]) / curve_l[0] (0 for an
+ *   all-zero layer), in double.  S_out (device, int32 [n_layers]) maximises sum_l reward_l(S_out[l])
+ *   subject to sum_l S_out[l]*unit_cost[l] <= budget (weight elements) and S_out[l] <= s_max[l]:
+ *   exact dynamic programme over the budget in units of gcd(unit_cost), layers in order, a larger
+ *   count taken only when strictly better.  total_reward (device, double [1], nullable) = the
+ *   optimum.  Limits: budget/gcd <= 2^22, n_layers <= 4096 (else OCS_ERR_UNSUPPORTED).
+ *   The paper states objective and constraint only (and reports no gain over the simple rule). */
+size_t ocs_range_curve_workspace_bytes(int C, int R, int S_max);
+ocs_status ocs_range_curve(const float* W, int O, int C, int R, int64_t ld_in, int S_max, float* curve,
+                           void* ws, size_t ws_bytes, int* dev_status, void* stream);
+size_t ocs_knapsack_workspace_bytes(int n_layers, const int64_t* unit_cost, int64_t budget);
+ocs_status ocs_knapsack_allocate(int n_layers, const float* curves, const int64_t* curve_off,
+                                 const int32_t* s_max, const int64_t* unit_cost, int64_t budget,
+                                 int32_t* S_out, double* total_reward, void* ws, size_t ws_bytes,
+                                 void* stream);
+
 /* ocs_quantize ----------------------------------------------------------------------------
  * k-bit linear quantization (Eq. 1) with the clip threshold alpha in place of max|x|
  * (Section 4): step = alpha/L, inv = L/alpha (fp32), code = clamp(rint(x*inv), -L, L) with

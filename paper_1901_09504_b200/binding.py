@@ -26,6 +26,7 @@ EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
     "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
     "ocs_split_workspace_bytes", "ocs_split",
+    "ocs_range_curve_workspace_bytes", "ocs_range_curve", "ocs_knapsack_workspace_bytes", "ocs_knapsack_allocate",
     "ocs_split_quantize_workspace_bytes", "ocs_split_quantize", "ocs_dup_weight_columns",
     "ocs_fold_workspace_bytes", "ocs_fold_duplicates",
     "ocs_act_select_workspace_bytes", "ocs_act_select_channels", "ocs_act_split_quantize_static",
@@ -53,7 +54,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.ocs_num_splits.argtypes = [C.c_int, C.c_double]
         L.ocs_version.restype = C.c_char_p
-        for name in ("ocs_fold_workspace_bytes", "ocs_act_select_workspace_bytes", "ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
+        for name in ("ocs_range_curve_workspace_bytes", "ocs_knapsack_workspace_bytes", "ocs_fold_workspace_bytes", "ocs_act_select_workspace_bytes", "ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
                      "ocs_qconv_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.ocs_quantize_workspace_views.restype = None
@@ -446,3 +447,39 @@ def ocs_fold_duplicates(W_codes, C_in: int, S: int, idx_map, R: int = 1, ld_out:
                                    _stream())
     _check(st, "ocs_fold_duplicates")
     return out
+
+
+def ocs_range_curve(W, S_max: int, out=None, dev_status=None):
+    """W fp32 [O, C] or [O, C, kh, kw] -> curve fp32 [S_max + 1]: max|W'| after s = 0..S_max greedy plain-halving splits."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+    O, Cn = W.shape[0], W.shape[1]
+    R = 1
+    for d in W.shape[2:]:
+        R *= d
+    curve = out if out is not None else torch.empty(int(S_max) + 1, dtype=torch.float32, device=W.device)
+    ws = _ws(lib().ocs_range_curve_workspace_bytes(Cn, R, int(S_max)), W.device)
+    st = lib().ocs_range_curve(_ptr(W), O, Cn, R, C.c_int64(Cn * R), int(S_max), _ptr(curve), _ptr(ws),
+                               C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
+    _check(st, "ocs_range_curve")
+    return curve
+
+
+def ocs_knapsack_allocate(curves, unit_cost, budget: int):
+    """curves: list of fp32 device tensors (one per layer, s_max + 1 entries each); unit_cost: list of ints (O * R per
+    layer); budget in weight elements -> (S int32 [n_layers] on the device, total reward float64 [1])."""
+    n = len(curves)
+    flat = torch.cat([c.reshape(-1) for c in curves]).contiguous()
+    sizes = [int(c.numel()) for c in curves]
+    off = (C.c_int64 * n)(*[sum(sizes[:i]) for i in range(n)])
+    smax = (C.c_int32 * n)(*[sz - 1 for sz in sizes])
+    cost = (C.c_int64 * n)(*[int(c) for c in unit_cost])
+    S = torch.empty(n, dtype=torch.int32, device=flat.device)
+    total = torch.empty(1, dtype=torch.float64, device=flat.device)
+    nws = lib().ocs_knapsack_workspace_bytes(n, cost, C.c_int64(int(budget)))
+    if nws == 0:
+        raise OcsError("ocs_knapsack_workspace_bytes", 4)
+    ws = _ws(nws, flat.device)
+    st = lib().ocs_knapsack_allocate(n, _ptr(flat), off, smax, cost, C.c_int64(int(budget)), _ptr(S), _ptr(total),
+                                     _ptr(ws), C.c_size_t(ws.numel()), _stream())
+    _check(st, "ocs_knapsack_allocate")
+    return S, total

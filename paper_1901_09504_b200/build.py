@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libocs_b200.so")
-SOURCES = ["split.cu", "actsel.cu", "quantize.cu", "gemm.cu", "glue.cu", "api.cu"]
+SOURCES = ["split.cu", "actsel.cu", "quantize.cu", "gemm.cu", "glue.cu", "knapsack.cu", "api.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -209,6 +209,8 @@ struct PlanArgs {
   unsigned long long* g_buf;  // sel | live0 | live1 | batch in global memory, used when S > kPlanSmemSplits
   int cap, npad, Sp;      // live capacity Sp + S, sort capacity (power of two >= cap), min(S, C)
   int hist_off, keys_off; // byte offsets in dynamic shared memory: selection histograms; keys (-1: chkey)
+  float* curve;           // [S + 1] or null: curve[s] = largest |w| after s plain-halving splits; when given, the
+                          // kernel only fills the curve (no index map, no extrema of the copies)
   int* dev_status;
 };
 
@@ -370,6 +372,7 @@ __device__ float greedy_rounds(const PlanArgs& a, PlanShared& sh, unsigned long 
         j = prio_index(p);
         const int s = base + i;
         const int jn = a.C + s;
+        if (!write && a.curve) a.curve[s] = prio_key(p);   // the value step s picks is the maximum before it
         unsigned long long ca, cb;
         if (write) {
           const float mn = a.chmin[j], mx = a.chmax[j];
@@ -472,6 +475,13 @@ __global__ void __launch_bounds__(kPlanThreads, 1) split_plan_kernel(PlanArgs a)
   if (bad) sh.bad = 1;
   const float maxw = __uint_as_float((uint32_t)block_max_u64(lmax, sh.red));
 
+  if (a.curve && S == 0) {
+    if (tid == 0) {
+      a.curve[0] = maxw;
+      if (sh.bad) flag(a.dev_status, OCS_DEV_NONFINITE);
+    }
+    return;
+  }
   if (S == 0) {
     if (tid == 0) {
       const float step = a.qa_bits >= 2 ? __fdiv_rn(maxw, (float)((1 << (a.qa_bits - 1)) - 1)) : a.qa_step;
@@ -550,6 +560,17 @@ __global__ void __launch_bounds__(kPlanThreads, 1) split_plan_kernel(PlanArgs a)
   }
   const float rest_max = __uint_as_float((uint32_t)block_max_u64(lrest, sh.red));
   __syncthreads();
+  if (a.curve) {
+    // range curve only: plain halving on the keys, every step's pick recorded
+    for (int i = tid; i < Sp; i += kPlanThreads) live0[i] = sel[i];
+    __syncthreads();
+    const float last = fmaxf(rest_max, greedy_rounds(a, sh, live0, live1, batch, Sp, 0.0f, false));
+    if (tid == 0) {
+      a.curve[S] = last;
+      if (sh.bad) flag(a.dev_status, OCS_DEV_NONFINITE);
+    }
+    return;
+  }
   // signed extrema of the selected channels (the only originals the greedy steps can touch)
   for (int i = tid; i < Sp; i += kPlanThreads) {
     const int c = prio_index(sel[i]);
@@ -1041,7 +1062,7 @@ namespace {
 // The part ocs_split and ocs_split_quantize share: channel extrema and the greedy plan.
 ocs_status run_split_front(const float* W, int O, int C, int R, int64_t ld_in, int S, float qa_step, int qa_bits,
                            int32_t* idx_map, int32_t* split_order, float* max_abs_out, const SplitWs& w,
-                           int* dev_status, cudaStream_t stream) {
+                           int* dev_status, cudaStream_t stream, float* curve = nullptr) {
   ocs_status st;
   const int ncols = C * R;
   if (cudaMemsetAsync(w.colmin, 0xFF, 4 * (size_t)ncols, stream) != cudaSuccess) return OCS_ERR_CUDA;
@@ -1074,6 +1095,7 @@ ocs_status run_split_front(const float* W, int O, int C, int R, int64_t ld_in, i
     a.max_abs_out = max_abs_out; a.qa_step_dev = w.qa_step_dev;
     a.touched = w.touched; a.n_touched = w.n_touched;
     a.g_buf = w.g_buf; a.cap = w.cap; a.npad = w.npad; a.Sp = w.Sp;
+    a.curve = curve;
     a.dev_status = dev_status;
     // dynamic shared memory: the plan buffer (when S is small enough) and, overlapping the part of
     // it that the live sets only use after the selection, the selection histograms and the keys
@@ -1156,6 +1178,32 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     if ((st = launch_status()) != OCS_OK) return st;
   }
   return OCS_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// ocs_range_curve: curve[s] = max|W'| after s greedy plain-halving splits (Section 3.4), s = 0..S_max: one pass
+// over W for the channel extrema, then the plan kernel's rounds on the keys alone.  This is what the knapsack
+// allocation's reward is made of.
+extern "C" size_t ocs_range_curve_workspace_bytes(int C, int R, int S_max) {
+  if (C <= 0 || R <= 0 || S_max < 0) return 0;
+  return carve_split_ws(nullptr, C, R, S_max).total + align_up(4 * ((size_t)C + S_max), 256);
+}
+
+extern "C" ocs_status ocs_range_curve(const float* W, int O, int C, int R, int64_t ld_in, int S_max, float* curve,
+                                      void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!W || !curve || S_max < 0) return OCS_ERR_INVALID_ARG;
+  if (O <= 0 || C <= 0 || R <= 0) return OCS_ERR_SHAPE;
+  if ((int64_t)C * R >= (1ll << 31) || ((int64_t)C + S_max) * R >= (1ll << 31) || ld_in < (int64_t)C * R) return OCS_ERR_SHAPE;
+  if (!aligned(W, 4)) return OCS_ERR_SHAPE;
+  const SplitWs w = carve_split_ws(ws, C, R, S_max);
+  const size_t total = w.total + align_up(4 * ((size_t)C + S_max), 256);
+  if (!ws || !aligned(ws, 256) || ws_bytes < total) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  // the extrema kernel also writes the identity part of an index map: it goes to scratch here
+  int32_t* idx_scratch = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(ws) + w.total);
+  return run_split_front(W, O, C, R, ld_in, S_max, 0.0f, 0, idx_scratch, nullptr, nullptr, w, dev_status, stream, curve);
 }
 
 // ------------------------------------------------------------------------------------------------
