@@ -39,7 +39,7 @@ if ROOT not in sys.path:
 from ocs_inputs import configs, prng  # noqa: E402
 
 N_BINS, N_CAND = 2048, 128
-INT8_OVER_BF16 = 2.0          # nominal dense int8 rate / nominal dense bf16 rate of the part
+INT8_OVER_BF16 = 2.0          # nominal dense int8 rate / nominal dense bf16 rate of the part (fallback only)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -134,11 +134,88 @@ def peaks():
 
 
 # ----------------------------------------------------------------------------------------------
+# The tensor half of the metric on shapes the tensor pipe bounds.  (1) The int8 peak of this GPU, measured in
+# the same run: the library int8 GEMM (torch._int_mm, cuBLASLt) on 8192^3, best of 10, CUDA events -- a library
+# measurement, used as the denominator.  (2) ocs_qlinear on the same shape without and with 2 % duplicated
+# channels.  (3) The 3x3 convolutions of ResNet-50's stages 3 and 4 at batch 128 (configs[3]'s heavy layers)
+# through ocs_qconv, ops-weighted.  Inputs are random codes made on the device: these are timings of the
+# contraction alone, reported beside the headline, not in it.
+def _time_best(torch, fn, reps=10, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    return best
+
+
+def tensor_probe(ocs, torch, dev):
+    out = {}
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    n = 8192
+    ops = 2.0 * n * n * n
+    a8 = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=dev, generator=g)
+    b8 = torch.randint(-127, 128, (n, n), dtype=torch.int8, device=dev, generator=g)
+    try:
+        ms = _time_best(torch, lambda: torch._int_mm(a8, b8))
+        out["int8_peak_tops"] = ops / (ms * 1e-3) / 1e12
+        out["int8_peak_note"] = "measured in this run: torch._int_mm (library int8 GEMM) 8192^3, best of 10, CUDA events"
+    except Exception as e:      # the library routine is missing: fall back to the nominal ratio
+        out["int8_peak_tops"] = None
+        out["int8_peak_note"] = f"torch._int_mm unavailable ({type(e).__name__})"
+    del b8
+    st = ocs.new_status(dev)
+    a_scale = torch.full((1,), 0.01, dtype=torch.float32, device=dev)
+    w_scale = torch.full((1,), 0.001, dtype=torch.float32, device=dev)
+    Au = a8.view(torch.uint8)
+    Y = torch.empty((n, n), dtype=torch.float32, device=dev)
+    ws = torch.empty(int(ocs.lib().ocs_qlinear_workspace_bytes(n, n, n, 164)) + 256, dtype=torch.uint8, device=dev)
+    for S, key in ((0, "qlinear_8192_tops"), (164, "qlinear_8192_dup2pct_tops")):
+        ldw = ocs.round_up(n + S, 16)
+        Wc = torch.randint(-127, 128, (n, ldw), dtype=torch.int8, device=dev, generator=g)
+        idx = torch.cat([torch.arange(n, dtype=torch.int32, device=dev),
+                         torch.randint(0, n, (S,), dtype=torch.int32, device=dev, generator=g)]).contiguous()
+        ms = _time_best(torch, lambda: ocs.ocs_qlinear(Au, a_scale, Wc, w_scale, idx, n, S, out=Y, ws=ws, dev_status=st))
+        out[key] = 2.0 * n * n * (n + S) / (ms * 1e-3) / 1e12
+        del Wc
+    del a8, Au, Y
+    # ResNet-50 stages 3-4, 3x3 convolutions at batch 128: (C = O, H_in, stride, how many such layers)
+    tot_ops, tot_ms = 0.0, 0.0
+    for Cn, H, stride, count in ((256, 28, 2, 1), (256, 14, 1, 5), (512, 14, 2, 1), (512, 7, 1, 2)):
+        S = configs_num_splits(Cn, 0.01)
+        Ho = (H + 2 - 3) // stride + 1
+        X = torch.randint(0, 256, (128, H, H, Cn), dtype=torch.uint8, device=dev, generator=g)
+        Kp = ocs.ocs_conv_packed_k(Cn, S, 3, 3)
+        Wp = torch.randint(-127, 128, (Cn, ocs.round_up(Kp, 16)), dtype=torch.int8, device=dev, generator=g)
+        idx = torch.cat([torch.arange(Cn, dtype=torch.int32, device=dev),
+                         torch.randint(0, Cn, (S,), dtype=torch.int32, device=dev, generator=g)]).contiguous()
+        Yc = torch.empty((128, Ho, Ho, Cn), dtype=torch.float32, device=dev)
+        wsc = torch.empty(int(ocs.lib().ocs_qconv_workspace_bytes(128, H, H, Cn, Cn, S, 3, 3, stride, 1)) + 256,
+                          dtype=torch.uint8, device=dev)
+        ms = _time_best(torch, lambda: ocs.ocs_qconv(X, a_scale, Wp, w_scale, idx, S, 3, 3, stride, 1, out=Yc, ws=wsc,
+                                                     dev_status=st), reps=5)
+        tot_ops += count * 2.0 * 128 * Ho * Ho * Cn * (Cn + S) * 9
+        tot_ms += count * ms
+    out["resnet50_3x3_stage34_tops"] = tot_ops / (tot_ms * 1e-3) / 1e12
+    assert ocs.ocs_poll_status(st) == 0, "device status word set during the tensor probe"
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
 class Fc6Sweep:
     name = "fc6"
 
     def __init__(self, small=False):
         self.O, self.C, self.M = (256, 6272, 128) if small else (4096, 25088, 128)
+        if small:
+            self.name = "fc6-small"
         self.desc = (f"configs[2]: fc6-shaped W [{self.O}, {self.C}] fp32, sweep of 5 expand ratios x 4 weight bit "
                      f"widths (20 points), MSE clip search ({N_CAND} candidates, {N_BINS} bins), int8 containers, "
                      f"activations [{self.M}, {self.C}] 8-bit unsigned; seed 2")
@@ -169,6 +246,13 @@ class Fc6Sweep:
         self.status = ocs.new_status(dev)
         self.W.copy_(host["W"])
         self.A.copy_(host["A"])
+
+    def release(self):
+        """Drops the big device buffers (called after the last timed region)."""
+        for k in ("W", "A", "W_out", "codes", "Wd", "Ad", "Yd", "Y", "slot_graphs", "graph_obj", "ws"):
+            if hasattr(self, k):
+                setattr(self, k, None)
+        self.torch.cuda.empty_cache()
 
     def ledger(self):
         led = Ledger()
@@ -813,6 +897,7 @@ def main():
     ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm", "lstm-folded", "act-ocs"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-tensor-probe", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -906,6 +991,13 @@ def main():
     h2d, d2h = wl.e2e_buffers(host)
     ms_e2e, _ = timed(wl.step_e2e, args.steps, 3)
 
+    # the tensor-bound half of the metric (rank 0, one GPU, default workload): measured int8 peak and three
+    # contraction timings
+    probe = None
+    if rank == 0 and world == 1 and wl.name == "fc6" and not args.no_tensor_probe:
+        wl.release()
+        probe = tensor_probe(ocs, torch, dev)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -919,7 +1011,11 @@ def main():
                              algorithmic_gbs=(nb / (ms * 1e-3) / 1e9) if ms > 0 and nb else None)
     top = next(iter(kernels))
     top_cnt, top_ms = trace[top]
-    int8_peak = pk["bf16_burst"] * INT8_OVER_BF16
+    if probe and probe.get("int8_peak_tops"):
+        int8_peak, int8_note = probe["int8_peak_tops"], probe["int8_peak_note"]
+    else:
+        int8_peak = pk["bf16_burst"] * INT8_OVER_BF16
+        int8_note = f"{pk['source']} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16 ratio; no int8 measurement in this run)"
     gemm_name = "ocs_gemm_kernel(linear)"
     gemm_ms = sum(trace.get(k, (0, 0.0))[1] for k in ("ocs_gemm_kernel(linear)", "ocs_gemm_kernel(conv)",
                                                      "splitk_reduce_kernel"))
@@ -935,7 +1031,7 @@ def main():
         # the contraction: integer ops of the step over the kernel's traced time, against the int8 peak
         ach = led.ops * args.steps / (top_ms * 1e-3) / 1e12
         roofline = dict(kernel=top, bound="tensor", achieved=ach, peak=int8_peak, unit="TOP/s", frac=ach / int8_peak,
-                        traffic=None, peak_source=f"{pk['source']} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16)",
+                        traffic=None, peak_source=int8_note,
                         avg_launch_ms=top_ms / top_cnt, note="ops of every quantized layer of the step (linear and conv "
                         "launches share one kernel); layers with few channels are bound by their output traffic, not by "
                         "the tensor pipe",
@@ -971,9 +1067,12 @@ def main():
                             if use_graph else "eager launches")),
         parts=dict(split_quantize_gbs=sq_gbs, split_quantize_frac_of_hbm=(sq_gbs / pk["hbm"]) if sq_gbs else None,
                    gemm_tops=gemm_tops, gemm_frac_of_int8_peak=(gemm_tops / int8_peak) if gemm_tops else None,
-                   int8_peak_tops=int8_peak,
-                   int8_peak_note=f"{pk['source']} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16 ratio)",
-                   gemm_algorithmic_gbs=kernels.get(gemm_name, {}).get("algorithmic_gbs")),
+                   int8_peak_tops=int8_peak, int8_peak_note=int8_note,
+                   gemm_algorithmic_gbs=kernels.get(gemm_name, {}).get("algorithmic_gbs"),
+                   gemm_frac_of_hbm=(kernels.get(gemm_name, {}).get("algorithmic_gbs") or 0) / pk["hbm"] or None,
+                   **({k: v for k, v in probe.items() if k.endswith("_tops") and k != "int8_peak_tops"} if probe else {}),
+                   **({k.replace("_tops", "_frac_of_int8_peak"): v / int8_peak for k, v in probe.items()
+                       if k.endswith("_tops") and k != "int8_peak_tops" and v} if probe else {})),
         roofline=roofline,
         kernels=kernels,
         cpu_baseline=cpu,

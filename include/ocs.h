@@ -90,6 +90,19 @@ long long ocs_kernel_launches(void);
 ocs_status ocs_trace_start(int max_records);
 int ocs_trace_stop(ocs_trace_row* rows, int capacity);
 
+/* ocs_selftest_wait_expiry (no counterpart in the paper; for tests of the failure path) -------
+ * Every device-side wait of the library is bounded; when one runs out the kernel sets
+ * OCS_DEV_TIMEOUT and returns.  This call shows that path without faulting or hanging anything:
+ * it runs the row-staged copy of ocs_split on W [O][C] (C a multiple of 4, rows 16-byte aligned,
+ * two rows must fit in shared memory) with no splits, but each CTA never requests its last row
+ * group and waits for it for about a millisecond only.  Afterwards *dev_status has
+ * OCS_DEV_TIMEOUT set, rows of the dropped groups of W_out are unwritten, no copy is in flight,
+ * and the stream and context are as usable as before.  Workspace: ocs_split_workspace_bytes(O, C,
+ * 1, 0) + 4*C rounded up to 256. */
+ocs_status ocs_selftest_wait_expiry(const float* W, int O, int C, int64_t ld_in, float* W_out,
+                                    int64_t ld_out, void* ws, size_t ws_bytes, int* dev_status,
+                                    void* stream);
+
 /* ocs_split -------------------------------------------------------------------------------
  * Weight OCS (Section 3.2 Eq. 3, Section 3.3, Section 3.4): S times, take the channel that
  * holds the largest |w| of the CURRENT expanded tensor (ties: the smallest current channel
@@ -320,6 +333,14 @@ ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, 
                        int64_t ldw, const int32_t* idx_map, const float* bias, float* Y,
                        int64_t ldy, int32_t* acc_out, const float* residual, int relu,
                        float* max_abs_out, void* ws, size_t ws_bytes, int* dev_status, void* stream);
+
+/* ocs_selftest_force_gemm_plan (no counterpart in the paper; for tests) ----------------------
+ * ocs_qlinear / ocs_qconv choose the output tile width, the number of K slices and the cluster
+ * size per problem.  The int32 accumulators must not depend on that choice.  This process-wide
+ * hook fixes the choice for the following calls (bn in {64, 128, 256}, split_k in 1..32, cluster
+ * in {1, 2, 4, 8}; values that do not fit a problem fall back to 1) so that a test can run one
+ * problem under several plans; bn = 0 returns the choice to the planner.  Host call. */
+ocs_status ocs_selftest_force_gemm_plan(int bn, int split_k, int cluster);
 
 /* ocs_pack_conv_weights -------------------------------------------------------------------
  * Reorders quantized conv weights from the split's layout [O][C+S][kh*kw] (row stride

@@ -25,13 +25,13 @@ CLIP_NONE, CLIP_MSE, CLIP_MSE_EXACT, CLIP_KL, CLIP_ACIQ = 0, 1, 2, 3, 4
 EXPORTS = [
     "ocs_num_splits", "ocs_poll_status", "ocs_version",
     "ocs_kernel_launches", "ocs_trace_start", "ocs_trace_stop",
-    "ocs_split_workspace_bytes", "ocs_split",
+    "ocs_split_workspace_bytes", "ocs_split", "ocs_selftest_wait_expiry",
     "ocs_range_curve_workspace_bytes", "ocs_range_curve", "ocs_knapsack_workspace_bytes", "ocs_knapsack_allocate",
     "ocs_split_quantize_workspace_bytes", "ocs_split_quantize", "ocs_dup_weight_columns",
     "ocs_fold_workspace_bytes", "ocs_fold_duplicates",
     "ocs_act_select_workspace_bytes", "ocs_act_select_channels", "ocs_act_split_quantize_static",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
-    "ocs_qlinear_workspace_bytes", "ocs_qlinear",
+    "ocs_qlinear_workspace_bytes", "ocs_qlinear", "ocs_selftest_force_gemm_plan",
     "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
     "ocs_add_relu", "ocs_maxpool3x3s2", "ocs_global_avgpool", "ocs_nchw_to_nhwc", "ocs_embedding", "ocs_lstm_cell",
 ]
@@ -483,3 +483,21 @@ def ocs_knapsack_allocate(curves, unit_cost, budget: int):
                                      _ptr(ws), C.c_size_t(ws.numel()), _stream())
     _check(st, "ocs_knapsack_allocate")
     return S, total
+
+
+def ocs_selftest_wait_expiry(W, dev_status):
+    """Runs the row-staged copy with each CTA's last row group never requested: sets DEV_TIMEOUT in dev_status
+    and returns the (partly unwritten) output."""
+    assert W.is_cuda and W.dtype == torch.float32 and W.dim() == 2 and W.is_contiguous()
+    O, Cn = W.shape
+    out = torch.zeros_like(W)
+    ws = _ws(lib().ocs_split_workspace_bytes(O, Cn, 1, 0) + round_up(4 * Cn, 256) + 256, W.device)
+    st = lib().ocs_selftest_wait_expiry(_ptr(W), O, Cn, C.c_int64(Cn), _ptr(out), C.c_int64(Cn), _ptr(ws),
+                                        C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
+    _check(st, "ocs_selftest_wait_expiry")
+    return out
+
+
+def ocs_selftest_force_gemm_plan(bn: int = 0, split_k: int = 0, cluster: int = 0):
+    """Fixes tile width / K slices / cluster size of the following ocs_qlinear / ocs_qconv calls (bn = 0: planner)."""
+    _check(lib().ocs_selftest_force_gemm_plan(int(bn), int(split_k), int(cluster)), "ocs_selftest_force_gemm_plan")

@@ -29,6 +29,9 @@
 // outstanding copies land, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include <atomic>
+#include <random>
+
 #include "common.cuh"
 
 namespace ocs {
@@ -79,6 +82,9 @@ struct GemmParams {
   int relu;                     // max(., 0) applied to Y
   unsigned int* max_bits;       // fp32 bits of max |Y| over the whole output (optional)
   int32_t* acc_ws;              // [split_k][rows][N] partial sums when split_k > 1
+  unsigned long long* slice_flags;   // [m_tiles][n_tiles][split_k]: `nonce` once that slice's partial tile is written
+  unsigned long long nonce;     // this call's tag (a stale or random word in the workspace does not match it)
+  int n_tiles;
   long long out_rows;           // rows of Y
   int a_box_bytes;              // bytes one TMA load of A delivers
   int* dev_status;
@@ -660,7 +666,14 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         for (int c = (warp >= 10 ? 32 : 0); c < BN && c < n_left; c += 64)
           asm volatile("prefetch.global.L2 [%0];" ::"l"(rrow + c));
       }
-      if (!mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag)) { ok = false; break; }
+      // A warp whose wait ran out leaves at once when the output is written directly; with split K it first
+      // goes through this item's three barriers with the other epilogue warps (skipping its own work), so that
+      // all eight stop at the same place
+      const bool got = mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag);
+      if (!got) {
+        ok = false;
+        if (direct) break;
+      }
       tc_fence_after();
       // Each lane holds one row of a 32 x 16 piece of the accumulator; written out that way a store
       // instruction would touch 32 rows with 16 bytes each.  The piece goes through shared memory instead, so
@@ -685,7 +698,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       float tile_max = 0.0f;
       const bool want_max = direct && p.max_bits != nullptr;
       // a warp whose 32 rows are all padding (a short M tile) has nothing to write
-      const bool warp_has_rows = __any_sync(0xffffffffu, ri.out_row >= 0);
+      const bool warp_has_rows = got && __any_sync(0xffffffffu, ri.out_row >= 0);
       for (int c0 = half * kEpiCols; warp_has_rows && c0 < BN; c0 += 2 * kEpiCols) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
@@ -792,7 +805,98 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       // the accumulator has been read out: hand it back to the MMA issuer
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(accempty_bar(acc));
+      if (lane == 0 && got) mbar_arrive(accempty_bar(acc));
+      if (!direct) {
+        // Split K: this slice's partial tile is in the workspace.  The slice that finds every other slice's
+        // tag already set sums the partial tiles (integer sums: exact in any order) and applies the epilogue;
+        // nobody waits for anybody.  Each slice publishes its tag and then looks at the others', so the slice
+        // whose tag lands last sees all of them; if two finish close together both may do the sum -- they
+        // write identical values.
+        int* fin = reinterpret_cast<int*>(ctrl + 8 * kNumBars + 16);
+        asm volatile("bar.sync 2, 256;" ::: "memory");            // all eight epilogue warps have written their pieces
+        if (warp == 6 && lane == 0) {
+          int all = 0;
+          const int aborting = *abort_flag;                       // one reading decides for all eight warps
+          if (!aborting) {
+            unsigned long long* fl = p.slice_flags + ((long long)w.mt * p.n_tiles + nt) * p.split_k;
+            __threadfence();
+            asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(fl + kz), "l"(p.nonce) : "memory");
+            __threadfence();
+            all = 1;
+            for (int z = 0; z < p.split_k; ++z) {
+              unsigned long long v;
+              asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fl + z) : "memory");
+              all &= (v == p.nonce);
+            }
+          }
+          fin[0] = all;
+          fin[1] = aborting;
+        }
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        const bool finisher = fin[0] != 0;
+        if (fin[1]) ok = false;                                   // every epilogue warp leaves after this item
+        asm volatile("bar.sync 2, 256;" ::: "memory");            // everybody has read the verdict before it is reused
+        if (finisher) {
+          const int et = threadIdx.x - 6 * 32;                    // 0..255
+          const int n_lim = min(BN, p.N - nt * BN);
+          const bool vec = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 15) == 0) && (p.ldy % 4 == 0) &&
+                           (!p.acc_out || (reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) &&
+                           (!p.residual || (reinterpret_cast<uintptr_t>(p.residual) & 15) == 0);
+          const long long slice = p.out_rows * (long long)p.N;
+          float fmx = 0.0f;
+          constexpr int kQuads = BN / 4;                          // 4-column groups per tile row
+          for (int g = et; g < BM * kQuads; g += 256) {
+            const int r = g / kQuads, c = (g - r * kQuads) * 4;
+            if (c >= n_lim) continue;
+            const long long orow = row_info(p, w.mt, r).out_row;
+            if (orow < 0) continue;
+            const int n = nt * BN + c;
+            const int32_t* src = p.acc_ws + orow * p.N + n;
+            int4 a = make_int4(0, 0, 0, 0);
+            if (vec) {
+              for (int z = 0; z < p.split_k; ++z) {
+                const int4 b = __ldcg(reinterpret_cast<const int4*>(src + z * slice));
+                a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+              }
+            } else {
+              for (int z = 0; z < p.split_k; ++z) {
+                const int32_t* q = src + z * slice;
+                a.x += __ldcg(q);
+                if (c + 1 < n_lim) a.y += __ldcg(q + 1);
+                if (c + 2 < n_lim) a.z += __ldcg(q + 2);
+                if (c + 3 < n_lim) a.w += __ldcg(q + 3);
+              }
+            }
+            const int av[4] = {a.x, a.y, a.z, a.w};
+            float f[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const bool in = c + e < n_lim;
+              f[e] = fmaf(int_to_float_rn(av[e]), sc, (p.bias && in) ? __ldg(p.bias + n + e) : 0.0f);
+              if (p.residual && in) f[e] = __fadd_rn(f[e], p.residual[orow * p.ldy + n + e]);
+              if (p.relu) f[e] = f[e] > 0.0f ? f[e] : 0.0f;
+              if (in) fmx = fmaxf(fmx, fabsf(f[e]));
+            }
+            float* y = p.Y + orow * p.ldy + n;
+            if (vec) {
+              *reinterpret_cast<float4*>(y) = make_float4(f[0], f[1], f[2], f[3]);
+              if (p.acc_out) *reinterpret_cast<int4*>(p.acc_out + orow * p.ldy + n) = a;
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                if (c + e < n_lim) {
+                  y[e] = f[e];
+                  if (p.acc_out) p.acc_out[orow * p.ldy + n + e] = av[e];
+                }
+              }
+            }
+          }
+          if (p.max_bits) {
+            for (int o = 16; o > 0; o >>= 1) fmx = fmaxf(fmx, __shfl_xor_sync(0xffffffffu, fmx, o));
+            if (lane == 0 && fmx > 0.0f) atomicMax(p.max_bits, __float_as_uint(fmx));
+          }
+        }
+      }
     }
     tc_fence_before();
   }
@@ -805,61 +909,6 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     tmem_dealloc(tmem_base, 2 * BN);
   }
   if (threadIdx.x == 0 && *abort_flag) flag(p.dev_status, OCS_DEV_TIMEOUT);
-}
-
-// Sums the K slices' partial accumulators (integer sums: exact in any order) and applies the epilogue.
-// Thread = 4 consecutive columns of one output row when N % 4 == 0, else one element.
-template <bool VEC>
-__global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const int32_t* __restrict__ part, int split_k, long long rows, int N,
-                     const float* __restrict__ a_scale, const float* __restrict__ w_scale,
-                     const float* __restrict__ bias, float* __restrict__ Y, long long ldy, int32_t* __restrict__ acc_out,
-                     const float* __restrict__ residual, int relu, unsigned int* __restrict__ max_bits) {
-  float m = 0.0f;
-  const float sc = __fmul_rn(__ldg(a_scale), __ldg(w_scale));
-  const long long slice = rows * (long long)N;
-  const int per_row = VEC ? (N >> 2) : N;
-  const long long total = rows * per_row;
-  for (long long t = blockIdx.x * 256ll + threadIdx.x; t < total; t += (long long)gridDim.x * 256) {
-    const long long row = t / per_row;
-    const int n = (int)(t - row * per_row) * (VEC ? 4 : 1);
-    const int32_t* p = part + row * N + n;
-    if (VEC) {
-      int4 a = __ldcg(reinterpret_cast<const int4*>(p));
-#pragma unroll 4
-      for (int z = 1; z < split_k; ++z) {
-        const int4 b = __ldcg(reinterpret_cast<const int4*>(p + z * slice));
-        a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-      }
-      float* y = Y + row * ldy + n;
-      float f[4] = {fmaf((float)a.x, sc, bias ? __ldg(bias + n + 0) : 0.0f), fmaf((float)a.y, sc, bias ? __ldg(bias + n + 1) : 0.0f),
-                    fmaf((float)a.z, sc, bias ? __ldg(bias + n + 2) : 0.0f), fmaf((float)a.w, sc, bias ? __ldg(bias + n + 3) : 0.0f)};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (residual) f[e] = __fadd_rn(f[e], residual[row * ldy + n + e]);
-        if (relu) f[e] = f[e] > 0.0f ? f[e] : 0.0f;
-        m = fmaxf(m, fabsf(f[e]));
-        y[e] = f[e];
-      }
-      if (acc_out) {
-        int32_t* ao = acc_out + row * ldy + n;
-        ao[0] = a.x; ao[1] = a.y; ao[2] = a.z; ao[3] = a.w;
-      }
-    } else {
-      int a = __ldcg(p);
-      for (int z = 1; z < split_k; ++z) a += __ldcg(p + z * slice);
-      float f = fmaf((float)a, sc, bias ? __ldg(bias + n) : 0.0f);
-      if (residual) f = __fadd_rn(f, residual[row * ldy + n]);
-      if (relu) f = f > 0.0f ? f : 0.0f;
-      m = fmaxf(m, fabsf(f));
-      Y[row * ldy + n] = f;
-      if (acc_out) acc_out[row * ldy + n] = a;
-    }
-  }
-  if (max_bits) {
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if ((threadIdx.x & 31) == 0 && m > 0.0f) atomicMax(max_bits, __float_as_uint(m));
-  }
 }
 
 // ------------------------------------------------------------------------------------------------ host
@@ -910,7 +959,21 @@ constexpr int kMaxSplitCtas = 2 * kNumSMs;   // split-K never uses more than two
 // gather of one assembled K-block costs about `gather_cost` such units and is divided by the cluster
 // size; split-K adds the reduction pass.  n_tail = K-blocks whose A tile is assembled by threads,
 // tail_k = contraction indices in them (only 16-index chunks that hold data cost gather time).
+// Self-test override (ocs_selftest_force_gemm_plan): tile width, K slices and cluster size taken as given where
+// they are valid for the problem.
+int g_force_bn = 0, g_force_sk = 0, g_force_cl = 0;
+
 GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, bool conv) {
+  if (g_force_bn) {
+    const int BN = g_force_bn;
+    const int n_tiles = (N + BN - 1) / BN;
+    int sk = g_force_sk < 1 ? 1 : g_force_sk;
+    if (sk > num_kb) sk = num_kb;
+    if ((long long)m_tiles * n_tiles * sk > kMaxSplitCtas && sk > 1) sk = 1;
+    int cl = g_force_cl < 1 ? 1 : g_force_cl;
+    if (n_tail == 0 || n_tiles % cl != 0) cl = 1;
+    return GemmPlan{BN, sk, cl, m_tiles, n_tiles};
+  }
   GemmPlan best{64, 1, 1, m_tiles, (N + 63) / 64};
   double best_cost = 1e300;
   const int bns[3] = {256, 128, 64};
@@ -938,7 +1001,7 @@ GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, boo
         const int cta_k = tail_k < tail_blocks * BK ? tail_k : tail_blocks * BK;
         const double gather_t = (0.5 * tail_blocks + (cta_k / 128.0) * gather_cost) / cl;
         double cost = (double)waves * ((main_t > gather_t ? main_t : gather_t) + 4.0 * t_block);
-        if (sk > 1) cost += 6.0;
+        if (sk > 1) cost += 1.0 + 0.25 * sk * t_block;   // partial tiles written, then summed by the last slice
         cost *= 1.0 + 0.002 * ci + 0.001 * bi;   // ties: smaller cluster, wider tile
         if (cost < best_cost) {
           best_cost = cost;
@@ -950,13 +1013,15 @@ GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, boo
   return best;
 }
 
-// Upper bound of the split-K scratch over every plan choose_plan can return for this output.
+// Upper bound of the split-K scratch (partial tiles and the slices' tags) over every plan choose_plan can
+// return for this output.
+constexpr size_t kSliceFlagBytes = 64 * 1024;   // m_tiles * n_tiles < 148 when K is split, at most 32 slices, 8 bytes each
 size_t splitk_ws_bound(long long rows, int N, long long m_tiles) {
   if (m_tiles * ((N + 255) / 256) >= kNumSMs) return 0;   // enough tiles: never split
   long long ints = 32ll * rows * N;
   const long long cap = (long long)kMaxSplitCtas * BM * 256;
   if (ints > cap) ints = cap;
-  return 4 * (size_t)ints;
+  return align_up(4 * (size_t)ints, 256) + kSliceFlagBytes;
 }
 
 template <int BN>
@@ -990,10 +1055,11 @@ ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const Gem
 
 struct GemmWs {
   int32_t* acc_ws;
+  unsigned long long* flags;
   size_t total;
 };
 
-GemmWs carve_gemm_ws(void* ws, long long rows, int N, int split_k) {
+GemmWs carve_gemm_ws(void* ws, long long rows, int N, int split_k, long long tiles) {
   GemmWs w{};
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -1002,8 +1068,19 @@ GemmWs carve_gemm_ws(void* ws, long long rows, int N, int split_k) {
     return q;
   };
   w.acc_ws = reinterpret_cast<int32_t*>(take(4 * (size_t)split_k * (size_t)rows * (size_t)N));
+  w.flags = reinterpret_cast<unsigned long long*>(take(8 * (size_t)tiles * (size_t)split_k));
   w.total = off;
   return w;
+}
+
+// A tag no earlier call and (but for a 2^-64 accident) no stale workspace content carries.
+unsigned long long next_nonce() {
+  static std::atomic<unsigned long long> counter{0};
+  static const unsigned long long salt = [] {
+    std::random_device rd;
+    return ((unsigned long long)rd() << 32) ^ (unsigned long long)rd() ^ 0x9E3779B97F4A7C15ull;
+  }();
+  return salt + 0x2545F4914F6CDD1Dull * (counter.fetch_add(1) + 1);
 }
 
 ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long long out_rows, int m_tiles, bool tma_a_ok,
@@ -1027,29 +1104,19 @@ ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long lo
   if (p.kb_tma_a > 0) tmA = *tmA_in;
 
   p.out_rows = out_rows;
+  p.n_tiles = plan.n_tiles;
   if (plan.split_k > 1) {
-    const GemmWs w = carve_gemm_ws(ws, out_rows, p.N, plan.split_k);
+    const GemmWs w = carve_gemm_ws(ws, out_rows, p.N, plan.split_k, (long long)plan.m_tiles * plan.n_tiles);
     if (!ws || !aligned(ws, 256) || ws_bytes < w.total) return OCS_ERR_WORKSPACE;
     p.acc_ws = w.acc_ws;
+    p.slice_flags = w.flags;
+    p.nonce = next_nonce();
   }
-  ocs_status st;
   switch (plan.BN) {
-    case 256: st = launch_gemm<256>(tmB, tmA, p, plan, stream); break;
-    case 128: st = launch_gemm<128>(tmB, tmA, p, plan, stream); break;
-    default: st = launch_gemm<64>(tmB, tmA, p, plan, stream); break;
+    case 256: return launch_gemm<256>(tmB, tmA, p, plan, stream);
+    case 128: return launch_gemm<128>(tmB, tmA, p, plan, stream);
+    default: return launch_gemm<64>(tmB, tmA, p, plan, stream);
   }
-  if (st != OCS_OK || plan.split_k == 1) return st;
-  const bool vec = (p.N % 4 == 0);
-  const long long work = out_rows * (long long)(vec ? p.N / 4 : p.N);
-  const int grid = (int)min((work + 255) / 256, (long long)kNumSMs * 8);
-  LaunchScope ls("splitk_reduce_kernel", stream);
-  if (vec)
-    splitk_reduce_kernel<true><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
-                                                         p.bias, p.Y, p.ldy, p.acc_out, p.residual, p.relu, p.max_bits);
-  else
-    splitk_reduce_kernel<false><<<grid, 256, 0, stream>>>(p.acc_ws, plan.split_k, out_rows, p.N, p.a_scale, p.w_scale,
-                                                          p.bias, p.Y, p.ldy, p.acc_out, p.residual, p.relu, p.max_bits);
-  return launch_status();
 }
 
 // M-tile box for the convolution: the (bw, bh, bn) with bw*bh*bn <= 128 that needs the fewest tiles.
@@ -1393,4 +1460,15 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
     if (!encode_u8(&tmA, X_codes, 4, dims, strides, box, estr)) return OCS_ERR_CUDA;
   }
   return run_gemm(p, W_packed, ldw, g.out_rows, (int)g.m_tiles, tma_ok, &tmA, ws, ws_bytes, stream);
+}
+
+// Self-test hook: the next ocs_qlinear / ocs_qconv calls of this process use the given tile width (64, 128, 256),
+// number of K slices and cluster size (1, 2, 4, 8) instead of the planner's choice, wherever the values are
+// valid for the problem; bn = 0 gives the choice back to the planner.
+extern "C" ocs_status ocs_selftest_force_gemm_plan(int bn, int split_k, int cluster) {
+  if (bn != 0 && bn != 64 && bn != 128 && bn != 256) return OCS_ERR_INVALID_ARG;
+  if (split_k < 0 || split_k > 32) return OCS_ERR_INVALID_ARG;
+  if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return OCS_ERR_INVALID_ARG;
+  g_force_bn = bn; g_force_sk = split_k; g_force_cl = cluster;
+  return OCS_OK;
 }

@@ -756,6 +756,8 @@ struct RowsEpilogue {
   int packed_ok;                // QUANT: 32-bit stores of four codes allowed
   float* scale_out;
   float* alpha_out;
+  long long wait_cycles;        // limit of the wait for a row group's copies; 0 = the default (about a second)
+  int drop_last_load;           // self-test only: the CTA's last row group is never requested, so its wait runs out
 };
 
 template <int MODE>
@@ -779,6 +781,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
   const float d = __fmul_rn(*qa_step_dev, 0.5f);
   const int nt = *n_touched;
   const int dep_cap = d == 0.0f ? kMaxHalvings : 64;
+  const long long wait_limit = ep.wait_cycles > 0 ? ep.wait_cycles : kRowWaitCycles;
 
   // epilogue state
   unsigned int* hist_sh = reinterpret_cast<unsigned int*>(row_smem + 2 * (size_t)rows_per_group * srow * sizeof(float));
@@ -854,14 +857,16 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
     }
   }
 
-  if (tid == 0 && my_groups > 0) issue_load(0);
-  int issued = my_groups > 0 ? 1 : 0;
+  // self-test: the last group's copies are never requested (nothing is in flight when its wait gives up)
+  const int load_groups = ep.drop_last_load ? my_groups - 1 : my_groups;
+  if (tid == 0 && load_groups > 0) issue_load(0);
+  int issued = load_groups > 0 ? 1 : 0;
   for (int i = 0; i < my_groups; ++i) {
     const int b = i & 1;
     if (tid == 0) {
       // the stores issued from the other buffer have finished reading it
       asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-      if (i + 1 < my_groups) { issue_load(i + 1); ++issued; }
+      if (i + 1 < load_groups) { issue_load(i + 1); ++issued; }
     }
     {  // bounded wait for this group's rows
       const uint32_t bar = smem_addr(&bars[b]);
@@ -870,7 +875,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
         const long long t0 = clock64();
         for (uint32_t it = 1;; ++it) {
           if (row_bar_try(bar, parity)) break;
-          if ((it & 63u) == 0u && (abort_flag || clock64() - t0 > kRowWaitCycles)) { abort_flag = 1; break; }
+          if ((it & 63u) == 0u && (abort_flag || clock64() - t0 > wait_limit)) { abort_flag = 1; break; }
         }
       }
     }
@@ -1178,6 +1183,44 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     if ((st = launch_status()) != OCS_OK) return st;
   }
   return OCS_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// ocs_selftest_wait_expiry: makes a bounded device wait run out, on purpose and safely.  The row-staged copy
+// kernel runs on W with no splits, but every CTA leaves out the request for its last row group and waits for
+// it with a limit of about a millisecond: the wait expires, the CTA sets OCS_DEV_TIMEOUT and returns with no
+// copy in flight.  Rows of the dropped groups are left unwritten.  Nothing traps and nothing spins unbounded.
+extern "C" ocs_status ocs_selftest_wait_expiry(const float* W, int O, int C, int64_t ld_in, float* W_out, int64_t ld_out,
+                                               void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!W || !W_out || !dev_status) return OCS_ERR_INVALID_ARG;
+  if (O <= 0 || C <= 0 || C % 4 != 0 || ld_in < C || ld_out < C || ld_in % 4 != 0 || ld_out % 4 != 0) return OCS_ERR_SHAPE;
+  if (!aligned(W, 16) || !aligned(W_out, 16)) return OCS_ERR_SHAPE;
+  const size_t row_bytes = 4 * (size_t)C;
+  if (2 * row_bytes > kRowSmemBytes) return OCS_ERR_UNSUPPORTED;
+  const SplitWs w = carve_split_ws(ws, C, 1, 0);
+  const size_t total = w.total + align_up(4 * (size_t)C, 256);
+  if (!ws || !aligned(ws, 256) || ws_bytes < total) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  int32_t* idx_map = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(ws) + w.total);
+  if ((st = run_split_front(W, O, C, 1, ld_in, 0, 0.0f, 0, idx_map, nullptr, nullptr, w, dev_status, stream)) != OCS_OK)
+    return st;
+  long long g = (long long)(kRowSmemBytes / 2 / row_bytes);
+  g = min(g, (long long)max(1, O / kNumSMs));
+  g = min(g, 64ll);
+  const int n_groups = (int)((O + g - 1) / g);
+  if (cudaFuncSetAttribute(split_rows_kernel<ROWS_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)kRowSmemBytes) != cudaSuccess)
+    return OCS_ERR_CUDA;
+  RowsEpilogue ep{};
+  ep.wait_cycles = 2000000ll;   // about a millisecond
+  ep.drop_last_load = 1;
+  LaunchScope ls("split_rows_kernel", stream);
+  split_rows_kernel<ROWS_STORE><<<min(n_groups, kNumSMs), kRowThreads, 2 * (size_t)g * row_bytes, stream>>>(
+      W, O, C, 1, ld_in, 0, W_out, ld_out, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g, C, ep,
+      dev_status);
+  return launch_status();
 }
 
 // ------------------------------------------------------------------------------------------------

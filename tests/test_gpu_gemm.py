@@ -203,3 +203,57 @@ def test_qconv_first_layer_with_and_without_room_for_the_patch_matrix():
         assert ocs.ocs_poll_status(st) == 0
         np.testing.assert_array_equal(host(acc), acco)
         np.testing.assert_array_equal(host(Y), Yo)
+
+
+def test_accumulators_do_not_depend_on_the_tile_plan():
+    """One problem under several forced (tile width, K slices, cluster size) plans: the int32 accumulators and
+    the outputs are identical, and equal the checker's (integer sums do not depend on their order)."""
+    M, Cn, N, S = 200, 2100, 384, 150
+    A = configs.random_codes(31, 0, (M, Cn), 0, 255, np.uint8)
+    Wc = configs.random_codes(31, 1, (N, Cn + S), -127, 127, np.int8)
+    idx = np.concatenate([np.arange(Cn), configs.random_codes(31, 2, (S,), 0, Cn - 1, np.int32)]).astype(np.int32)
+    bias = prng.normal(31, 3, (N,))
+    Yo, acco = orc.qlinear(A, False, 0.013, Wc, 0.0007, idx, bias)
+    ld = ocs.round_up(Cn + S, 16)
+    Wd = torch.zeros((N, ld), dtype=torch.int8, device="cuda")
+    Wd[:, :Cn + S] = dev(Wc)
+    Ad = torch.zeros((M, ocs.round_up(Cn, 16)), dtype=torch.uint8, device="cuda")
+    Ad[:, :Cn] = dev(A)
+    sa, sw = dev(np.array([0.013], np.float32)), dev(np.array([0.0007], np.float32))
+    try:
+        for bn, sk, cl in ((0, 0, 0), (64, 1, 1), (128, 1, 1), (256, 1, 1), (128, 2, 1), (128, 4, 1), (64, 3, 2), (64, 6, 2),
+                           (128, 5, 1), (256, 9, 1), (64, 8, 1)):
+            ocs.ocs_selftest_force_gemm_plan(bn, sk, cl)
+            st = ocs.new_status()
+            for _ in range(2):                                     # twice: the workspace's tags of the first run are stale
+                Y, acc = ocs.ocs_qlinear(Ad, sa, Wd, sw, dev(idx), Cn, S, bias=dev(bias), want_acc=True, dev_status=st)
+                assert ocs.ocs_poll_status(st) == 0
+                np.testing.assert_array_equal(host(acc), acco, err_msg=f"plan {(bn, sk, cl)}")
+                np.testing.assert_array_equal(host(Y), Yo, err_msg=f"plan {(bn, sk, cl)}")
+    finally:
+        ocs.ocs_selftest_force_gemm_plan(0, 0, 0)
+
+
+@pytest.mark.parametrize("split", [False, True])
+def test_shortcut_tensor_that_is_not_16_byte_aligned(split):
+    """A shortcut tensor that starts 4 bytes into its buffer (a view): the epilogue reads it with scalar loads
+    and the result is the checker's."""
+    M, Cn, N, S = 96, 640, 256, 13
+    if split:
+        Cn = 4096                                                   # few tiles, long K: the planner slices K
+    A = configs.random_codes(41, 0, (M, Cn), 0, 255, np.uint8)
+    Wc = configs.random_codes(41, 1, (N, Cn + S), -127, 127, np.int8)
+    idx = _rand_idx(41, Cn, S)
+    Yo, _ = orc.qlinear(A, False, 0.02, Wc, 0.001, idx, None)
+    res = prng.normal(41, 5, (M, N))
+    buf = torch.zeros(M * N + 1, dtype=torch.float32, device="cuda")
+    view = buf[1:].view(M, N)
+    view.copy_(dev(res))
+    assert view.data_ptr() % 16 == 4
+    Wd = torch.zeros((N, ocs.round_up(Cn + S, 16)), dtype=torch.int8, device="cuda")
+    Wd[:, :Cn + S] = dev(Wc)
+    st = ocs.new_status()
+    Y = ocs.ocs_qlinear(dev(A), dev(np.array([0.02], np.float32)), Wd, dev(np.array([0.001], np.float32)), dev(idx), Cn, S,
+                        residual=view, relu=True, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    np.testing.assert_array_equal(host(Y), orc.add_relu(Yo, res, True))
