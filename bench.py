@@ -63,6 +63,8 @@ def algorithmic_bytes(kernel: str, *, N=0, n=0, M=0, C=0, S=0, Nout=0, R=1, rows
         return rows * C + Nout * (C + S) * R + 4 * M * Nout + 4 * (C + S)
     if kernel == "pack_conv_kernel":
         return 2 * n
+    if kernel == "transpose_codes_kernel":
+        return 2 * n
     return 0
 
 
@@ -182,7 +184,9 @@ def tensor_probe(ocs, torch, dev):
         Wc = torch.randint(-127, 128, (n, ldw), dtype=torch.int8, device=dev, generator=g)
         idx = torch.cat([torch.arange(n, dtype=torch.int32, device=dev),
                          torch.randint(0, n, (S,), dtype=torch.int32, device=dev, generator=g)]).contiguous()
-        ms = _time_best(torch, lambda: ocs.ocs_qlinear(Au, a_scale, Wc, w_scale, idx, n, S, out=Y, ws=ws, dev_status=st))
+        AT = ocs.ocs_transpose_codes(Au) if S else None      # channel-major copy: the duplicated channels arrive by TMA
+        ms = _time_best(torch, lambda: ocs.ocs_qlinear(Au, a_scale, Wc, w_scale, idx, n, S, out=Y, ws=ws, dev_status=st,
+                                                       A_codes_T=AT))
         out[key] = 2.0 * n * n * (n + S) / (ms * 1e-3) / 1e12
         del Wc
     del a8, Au, Y
@@ -237,6 +241,7 @@ class Fc6Sweep:
         self.max_abs = torch.zeros(3, dtype=torch.float32, device=dev)
         self.codes = torch.empty((O, self.ld_out), dtype=torch.int8, device=dev)
         self.a_codes = torch.empty((M, ocs.round_up(C, 16)), dtype=torch.uint8, device=dev)
+        self.a_codes_T = torch.empty((C, ocs.round_up(M, 16)), dtype=torch.uint8, device=dev)   # channel-major copy
         self.scal = torch.zeros(4, dtype=torch.float32, device=dev)      # w_scale, alpha, a_scale, a_alpha
         self.Y = [torch.empty((M, O), dtype=torch.float32, device=dev) for _ in self.points]
         L = ocs.lib()
@@ -249,7 +254,7 @@ class Fc6Sweep:
 
     def release(self):
         """Drops the big device buffers (called after the last timed region)."""
-        for k in ("W", "A", "W_out", "codes", "Wd", "Ad", "Yd", "Y", "slot_graphs", "graph_obj", "ws"):
+        for k in ("W", "A", "W_out", "codes", "a_codes_T", "Wd", "Ad", "Yd", "Y", "slot_graphs", "graph_obj", "ws"):
             if hasattr(self, k):
                 setattr(self, k, None)
         self.torch.cuda.empty_cache()
@@ -267,9 +272,21 @@ class Fc6Sweep:
             led.add("quantize_kernel", n=n)
             led.add("maxabs_kernel", n=M * C)
             led.add("quantize_kernel", n=M * C)
+            if S > 0:
+                led.add("transpose_codes_kernel", n=M * C)
             led.add("ocs_gemm_kernel(linear)", rows=M, M=M, C=C, S=S, Nout=O)
             led.ops += 2 * M * O * (C + S)
         return led
+
+    def gemm(self, i, S):
+        """Activation codes -> layer output of sweep point i: with duplicated channels the layer gathers them as
+        whole rows of a channel-major copy of the codes (made here, every point: nothing is cached)."""
+        ocs, C = self.ocs, self.C
+        at = None
+        if S > 0:
+            at = ocs.ocs_transpose_codes(self.a_codes, cols=C, out=self.a_codes_T)
+        ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S,
+                        out=self.Y[i], ws=self.ws, dev_status=self.status, A_codes_T=at)
 
     def step(self):
         ocs, C = self.ocs, self.C
@@ -282,8 +299,7 @@ class Fc6Sweep:
                              ws=self.ws, dev_status=self.status)
             ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(self.a_codes, self.scal[2:3], self.scal[3:4]),
                              ws=self.ws, dev_status=self.status)
-            ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S,
-                            out=self.Y[i], ws=self.ws, dev_status=self.status)
+            self.gemm(i, S)
 
     # The step is a fixed chain of stream-ordered, allocation-free library calls on preallocated buffers: it is
     # captured once in a CUDA graph (after an eager warm-up) and replayed, which removes the host work between
@@ -427,6 +443,8 @@ class Fc6Fused(Fc6Sweep):
             led.add("split_quantize_kernel", N=N, n=n)
             led.add("maxabs_kernel", n=M * C)
             led.add("quantize_kernel", n=M * C)
+            if S > 0:
+                led.add("transpose_codes_kernel", n=M * C)
             led.add("ocs_gemm_kernel(linear)", rows=M, M=M, C=C, S=S, Nout=O)
             led.ops += 2 * M * O * (C + S)
         return led
@@ -440,8 +458,7 @@ class Fc6Fused(Fc6Sweep):
                                    ws=self.ws, dev_status=self.status)
             ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(self.a_codes, self.scal[2:3], self.scal[3:4]),
                              ws=self.ws, dev_status=self.status)
-            ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S,
-                            out=self.Y[i], ws=self.ws, dev_status=self.status)
+            self.gemm(i, S)
 
 
 class ActOcs(Fc6Sweep):
@@ -551,8 +568,7 @@ class SmallFc(Fc6Sweep):
                          out=(self.codes, self.scal[0:1], self.scal[1:2]), ws=self.ws, dev_status=self.status)
         ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(self.a_codes, self.scal[2:3], self.scal[3:4]),
                          ws=self.ws, dev_status=self.status)
-        ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S, out=self.Y[0],
-                        ws=self.ws, dev_status=self.status)
+        self.gemm(0, S)
 
     def ledger(self):
         led = Ledger()
@@ -564,6 +580,7 @@ class SmallFc(Fc6Sweep):
         led.add("quantize_kernel", n=n)
         led.add("maxabs_kernel", n=M * C)
         led.add("quantize_kernel", n=M * C)
+        led.add("transpose_codes_kernel", n=M * C)
         led.add("ocs_gemm_kernel(linear)", rows=M, M=M, C=C, S=S, Nout=O)
         led.ops = 2 * M * O * (C + S)
         return led
@@ -1021,7 +1038,7 @@ def main():
                                                      "splitk_reduce_kernel"))
     gemm_tops = (led.ops * args.steps / (gemm_ms * 1e-3) / 1e12) if gemm_ms > 0 else None
     sq_names = ("col_minmax_kernel", "split_rows_kernel", "split_scatter_kernel", "hist_kernel", "quantize_kernel", "maxabs_kernel",
-                "split_hist_kernel", "split_quantize_kernel")
+                "split_hist_kernel", "split_quantize_kernel", "transpose_codes_kernel")
     sq_ms = sum(trace[k][1] for k in sq_names if k in trace) + sum(
         trace[k][1] for k in ("split_plan_kernel", "score_kernel", "pick_kernel") if k in trace)
     sq_bytes = sum(led.bytes.get(k, 0) for k in sq_names) * args.steps

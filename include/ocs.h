@@ -318,6 +318,11 @@ void ocs_quantize_workspace_views(void* ws, int n_bins, int n_candidates, uint64
  * The duplicated activation channels (the run-time channel duplication of Section 3.5)
  * are gathered through idx_map while the operand tiles are staged; an expanded activation
  * tensor is never written.  idx_map[j] must equal j for j < C (as ocs_split produces).
+ * A_codes_T (nullable), row stride lda_T bytes: a channel-major copy of the same codes, [C][M]
+ * (ocs_transpose_codes makes one); lda_T a multiple of 16, at least M, 16-byte aligned.  With it
+ * the K-blocks that hold duplicated channels are fetched by the copy engine, one channel row per
+ * contraction index, straight into the operand tile -- the gather costs no thread a load.  Without
+ * it the producer warps gather those blocks byte by byte from A_codes.
  * A codes [M][C], row stride lda bytes, uint8 when a_signed = 0 else int8; Wc int8 [N][C+S],
  * row stride ldw bytes, ldw a multiple of 16 and Wc 16-byte aligned; a_scale / w_scale
  * device scalars; Y fp32 [M][N] row stride ldy floats; acc_out (nullable) int32 [M][N] with
@@ -328,19 +333,27 @@ void ocs_quantize_workspace_views(void* ws, int n_bins, int n_candidates, uint64
  * the stored output -- the next layer's activation grid (ocs_quantize's max_abs_in).
  * Device flags: BAD_INDEX, TIMEOUT. */
 size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S);
-ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C,
-                       int64_t lda, const int8_t* W_codes, const float* w_scale, int N, int S,
-                       int64_t ldw, const int32_t* idx_map, const float* bias, float* Y,
-                       int64_t ldy, int32_t* acc_out, const float* residual, int relu,
-                       float* max_abs_out, void* ws, size_t ws_bytes, int* dev_status, void* stream);
+ocs_status ocs_qlinear(const void* A_codes, const void* A_codes_T, int64_t lda_T, int a_signed,
+                       const float* a_scale, int M, int C, int64_t lda, const int8_t* W_codes,
+                       const float* w_scale, int N, int S, int64_t ldw, const int32_t* idx_map,
+                       const float* bias, float* Y, int64_t ldy, int32_t* acc_out,
+                       const float* residual, int relu, float* max_abs_out, void* ws, size_t ws_bytes,
+                       int* dev_status, void* stream);
+
+/* ocs_transpose_codes: codes_T[c][r] = codes[r][c] for 8-bit codes [rows][cols] (row stride ld
+ * bytes) -> [cols][rows] (row stride ld_T bytes).  A pure layout change: the channel-major copy of
+ * an activation matrix that ocs_qlinear can gather whole channels from. */
+ocs_status ocs_transpose_codes(const void* codes, int64_t rows, int64_t cols, int64_t ld,
+                               void* codes_T, int64_t ld_T, void* stream);
 
 /* ocs_selftest_force_gemm_plan (no counterpart in the paper; for tests) ----------------------
- * ocs_qlinear / ocs_qconv choose the output tile width, the number of K slices and the cluster
- * size per problem.  The int32 accumulators must not depend on that choice.  This process-wide
- * hook fixes the choice for the following calls (bn in {64, 128, 256}, split_k in 1..32, cluster
- * in {1, 2, 4, 8}; values that do not fit a problem fall back to 1) so that a test can run one
- * problem under several plans; bn = 0 returns the choice to the planner.  Host call. */
-ocs_status ocs_selftest_force_gemm_plan(int bn, int split_k, int cluster);
+ * ocs_qlinear / ocs_qconv choose the output tile width and, for problems with few tiles, how
+ * many CTAs share a tile and split its K range (their partial sums are exchanged through
+ * distributed shared memory).  The int32 accumulators must not depend on that choice.  This
+ * process-wide hook fixes the choice for the following calls (bn in {64, 128, 256}, split_k in
+ * {1, 2, 4, 8}; a split that does not fit the problem falls back to a smaller one) so that a test
+ * can run one problem under several plans; bn = 0 returns the choice to the planner.  Host call. */
+ocs_status ocs_selftest_force_gemm_plan(int bn, int split_k);
 
 /* ocs_pack_conv_weights -------------------------------------------------------------------
  * Reorders quantized conv weights from the split's layout [O][C+S][kh*kw] (row stride

@@ -31,7 +31,7 @@ EXPORTS = [
     "ocs_fold_workspace_bytes", "ocs_fold_duplicates",
     "ocs_act_select_workspace_bytes", "ocs_act_select_channels", "ocs_act_split_quantize_static",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
-    "ocs_qlinear_workspace_bytes", "ocs_qlinear", "ocs_selftest_force_gemm_plan",
+    "ocs_qlinear_workspace_bytes", "ocs_qlinear", "ocs_transpose_codes", "ocs_selftest_force_gemm_plan",
     "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
     "ocs_add_relu", "ocs_maxpool3x3s2", "ocs_global_avgpool", "ocs_nchw_to_nhwc", "ocs_embedding", "ocs_lstm_cell",
 ]
@@ -196,9 +196,22 @@ def ocs_quantize(T, bits: int, is_signed: bool = True, mode: int = CLIP_NONE, n_
     return codes, scale, alpha, hist, scores
 
 
+def ocs_transpose_codes(codes, cols: int | None = None, out=None):
+    """codes uint8/int8 [rows, ld >= cols] -> channel-major copy [cols, round_up(rows, 16)]."""
+    assert codes.is_cuda and codes.dim() == 2 and codes.stride(1) == 1 and codes.element_size() == 1
+    rows = codes.shape[0]
+    if cols is None:
+        cols = codes.shape[1]
+    T = out if out is not None else torch.empty((cols, round_up(rows, 16)), dtype=codes.dtype, device=codes.device)
+    _check(lib().ocs_transpose_codes(_ptr(codes), C.c_int64(rows), C.c_int64(cols), C.c_int64(codes.stride(0)), _ptr(T),
+                                     C.c_int64(T.stride(0)), _stream()), "ocs_transpose_codes")
+    return T
+
+
 def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, bias=None, want_acc: bool = False,
-                dev_status=None, out=None, ws=None, relu: bool = False, max_out=None, residual=None):
-    """A_codes uint8/int8 [M, lda>=C]; W_codes int8 [N, ldw>=C+S].  Returns Y fp32 [M, N] (and acc int32)."""
+                dev_status=None, out=None, ws=None, relu: bool = False, max_out=None, residual=None, A_codes_T=None):
+    """A_codes uint8/int8 [M, lda>=C]; W_codes int8 [N, ldw>=C+S]; A_codes_T (optional) the channel-major copy
+    [C, ld>=M] from ocs_transpose_codes.  Returns Y fp32 [M, N] (and acc int32)."""
     assert A_codes.is_cuda and A_codes.dim() == 2 and A_codes.stride(1) == 1
     assert W_codes.dtype == torch.int8 and W_codes.dim() == 2 and W_codes.stride(1) == 1
     M, N = A_codes.shape[0], W_codes.shape[0]
@@ -209,7 +222,8 @@ def ocs_qlinear(A_codes, a_scale, W_codes, w_scale, idx_map, C_in: int, S: int, 
     nws = lib().ocs_qlinear_workspace_bytes(M, N, int(C_in), int(S))
     if ws is None:
         ws = _ws(nws, A_codes.device)
-    st = lib().ocs_qlinear(_ptr(A_codes), a_signed, _ptr(a_scale), M, int(C_in), C.c_int64(A_codes.stride(0)),
+    st = lib().ocs_qlinear(_ptr(A_codes), _ptr(A_codes_T), C.c_int64(0 if A_codes_T is None else A_codes_T.stride(0)),
+                           a_signed, _ptr(a_scale), M, int(C_in), C.c_int64(A_codes.stride(0)),
                            _ptr(W_codes), _ptr(w_scale), N, int(S), C.c_int64(W_codes.stride(0)), _ptr(idx_map),
                            _ptr(bias), _ptr(Y), C.c_int64(N), _ptr(acc), _ptr(residual), int(bool(relu)), _ptr(max_out), _ptr(ws),
                            C.c_size_t(ws.numel()), _ptr(dev_status), _stream())
@@ -498,6 +512,6 @@ def ocs_selftest_wait_expiry(W, dev_status):
     return out
 
 
-def ocs_selftest_force_gemm_plan(bn: int = 0, split_k: int = 0, cluster: int = 0):
-    """Fixes tile width / K slices / cluster size of the following ocs_qlinear / ocs_qconv calls (bn = 0: planner)."""
-    _check(lib().ocs_selftest_force_gemm_plan(int(bn), int(split_k), int(cluster)), "ocs_selftest_force_gemm_plan")
+def ocs_selftest_force_gemm_plan(bn: int = 0, split_k: int = 0):
+    """Fixes tile width / K split of the following ocs_qlinear / ocs_qconv calls (bn = 0: planner)."""
+    _check(lib().ocs_selftest_force_gemm_plan(int(bn), int(split_k)), "ocs_selftest_force_gemm_plan")

@@ -104,10 +104,12 @@ __device__ inline float pick_alpha(const double* __restrict__ scores, float m, i
   return __double2float_rn(__ddiv_rn(__dmul_rn((double)m, (double)bc), (double)n_candidates));
 }
 
-// code = clamp(rint(x * inv)): clamping first is the same thing (the bounds are integers) and leaves one
-// conversion with round-to-nearest-even
+// code = clamp(rint(x * inv)): clamping first is the same thing (the bounds are integers).  The rounding is done
+// by one addition instead of a conversion instruction: for |t| <= 255, fl(t + 1.5 * 2^23) has unit spacing, so the
+// addition rounds t to the nearest integer, ties to even, and the integer sits in the low mantissa bits (two's
+// complement for negative t).  Only the low byte of the result is meaningful: that byte is the 8-bit code.
 __device__ __forceinline__ int quant_code(float x, float inv, float lo, float hi) {
-  return __float2int_rn(fminf(fmaxf(__fmul_rn(x, inv), lo), hi));
+  return __float_as_int(__fadd_rn(fminf(fmaxf(__fmul_rn(x, inv), lo), hi), 12582912.0f));
 }
 __device__ __forceinline__ unsigned int pack4(int c0, int c1, int c2, int c3) {
   return __byte_perm(__byte_perm((unsigned)c0, (unsigned)c1, 0x0040), __byte_perm((unsigned)c2, (unsigned)c3, 0x0040),

@@ -11,8 +11,13 @@
 // rules cannot serve) are assembled in shared memory by four producer warps that read the source
 // channels through idx_map and store them in the 128-byte-swizzled layout the tensor core reads.
 //
-// A work item = one 128 x BN output tile (x one K slice when split-K is on).  The grid is
-// persistent: one CTA per SM walks its share of the items.  Warp roles:
+// A work item = one 128 x BN output tile.  The grid is persistent: one CTA per SM, grouped in thread-block
+// clusters of CL = 1, 2, 4 or 8 CTAs; a cluster walks its share of the tiles and its CTAs split the tile's
+// K-blocks among themselves (CTA r takes blocks r, r + CL, ...), so that short-and-wide problems still fill the
+// GPU.  The CL partial accumulators of a tile are summed through distributed shared memory: every CTA sends
+// the rows another CTA owns straight into that CTA's shared memory (st.shared::cluster), barriers in shared
+// memory pace the exchange, and each CTA finishes 128 / CL rows of the tile (integer sums: exact in any order).
+// No second launch, no global scratch, and the only waits are on CTAs the hardware co-schedules.  Warp roles:
 //   warp 0      TMA producer (weights always, activations when the block is TMA-able); its ring of
 //               stages runs on across tiles
 //   warp 1      allocates tensor memory (two accumulators), issues tcgen05.mma, commits to barriers
@@ -22,15 +27,10 @@
 //               the two warps of a tensor-memory lane quadrant take alternate 16-column pieces
 // The K-blocks whose A tile is assembled ("tail" blocks) come last in a CTA's K order and use three
 // dedicated A buffers, so the gather warps start at kernel begin and run ahead of the TMA-fed main
-// loop.  CTAs that share the M tile and the K slice (neighbouring N tiles) form a thread-block
-// cluster: each assembles 1/CL of a tail tile's rows and stores them into every peer's buffer
-// through distributed shared memory, so a tile is gathered once per cluster, not once per CTA.
+// loop.
 // Every mbarrier wait is bounded by a clock limit; on expiry the CTA sets OCS_DEV_TIMEOUT, lets its
 // outstanding copies land, frees its tensor memory and returns.
 #include <cuda.h>
-
-#include <atomic>
-#include <random>
 
 #include "common.cuh"
 
@@ -48,6 +48,7 @@ constexpr long long kWaitCycles = 2000000000ll;  // about one second
 // A waiting thread sleeps inside mbarrier.try_wait until the phase completes or about this many nanoseconds
 // pass, instead of spinning on the issue slots the epilogue warps of the same SM partition need.
 constexpr uint32_t kSuspendHintNs = 2000u;
+constexpr uint32_t kExchangeHintNs = 100u;   // the exchange of partial sums sits on the critical path: short naps
 
 enum { MODE_LINEAR = 0, MODE_CONV = 1 };
 
@@ -61,6 +62,7 @@ struct GemmParams {
   int a_signed;
   const int32_t* idx_map;
   int a_vec16;       // 16-byte loads of A allowed (alignment)
+  int tail_T;        // the tail K-blocks are fetched by TMA from the channel-major copy of A (linear layers)
   // convolution geometry
   int Nb, H, Wd, Ho, Wo, kh, kw, stride, pad;
   int bw, bh, bn;               // output-pixel box of one M tile: bw*bh*bn <= 128
@@ -68,9 +70,9 @@ struct GemmParams {
   // k-blocks
   int num_kb;
   int kb_tma_a;      // K-blocks [0, kb_tma_a) get their A tile by TMA
-  int split_k;
-  // work items of the persistent grid: (K slice, M tile, group of CL neighbouring N tiles)
-  int m_tiles, n_groups, total_items;
+  int split_k;       // = cluster size: CTAs that share one output tile, each taking every split_k-th K-block
+  // work items of the persistent grid: output tiles (M tile, N tile), dealt to the clusters
+  int m_tiles, n_tiles, total_items;
   // epilogue
   const float* a_scale;
   const float* w_scale;
@@ -81,10 +83,6 @@ struct GemmParams {
   const float* residual;        // optional fp32 tensor of Y's shape and stride, added before the ReLU
   int relu;                     // max(., 0) applied to Y
   unsigned int* max_bits;       // fp32 bits of max |Y| over the whole output (optional)
-  int32_t* acc_ws;              // [split_k][rows][N] partial sums when split_k > 1
-  unsigned long long* slice_flags;   // [m_tiles][n_tiles][split_k]: `nonce` once that slice's partial tile is written
-  unsigned long long nonce;     // this call's tag (a stale or random word in the workspace does not match it)
-  int n_tiles;
   long long out_rows;           // rows of Y
   int a_box_bytes;              // bytes one TMA load of A delivers
   int* dev_status;
@@ -132,7 +130,7 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
       "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
+      : "r"(bar), "r"(parity), "r"(kExchangeHintNs)
       : "memory");
   return ok != 0;
 }
@@ -340,9 +338,22 @@ __device__ __forceinline__ KSrc k_source(const GemmParams& p, int k, bool* bad) 
   return e;
 }
 
+// One operand byte, loaded only when `ok` (a predicated load: no branch, and no memory transaction for an index
+// that contributes zero).
+__device__ __forceinline__ uint32_t ldg_u8_if(const uint8_t* addr, bool ok) {
+  uint32_t v;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.u32 p, %2, 0;\n\t"
+      "mov.u32 %0, 0;\n\t"
+      "@p ld.global.nc.u8 %0, [%1];\n\t}"
+      : "=r"(v) : "l"(addr), "r"((uint32_t)ok));
+  return v;
+}
+
 // The operand bytes of one tile row for the 16 contraction indices whose sources are tab[0..16).
-// Every load is unconditional (a source that contributes zero reads the tensor's first byte and is
-// masked afterwards), so the 16 loads are independent and in flight together.
+// The 16 loads are independent (predicated, not branched) and in flight together; indices that contribute zero
+// (K padding, a tap outside the image) issue no load.
 __device__ __forceinline__ uint4 gather_chunk(const GemmParams& p, const RowInfo& ri, const uint8_t* base,
                                               const KSrc* __restrict__ tab) {
   uint32_t b[16];
@@ -354,9 +365,7 @@ __device__ __forceinline__ uint4 gather_chunk(const GemmParams& p, const RowInfo
       const int ih = ri.ih0 + (e.dydx & 255), iw = ri.iw0 + (e.dydx >> 8);
       ok = ok && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd;
     }
-    const uint8_t* addr = ok ? base + e.off : p.A;
-    const uint32_t v = (uint32_t)__ldg(addr);
-    b[i] = ok ? v : 0u;
+    b[i] = ldg_u8_if(base + (ok ? e.off : 0), ok);
   }
   uint32_t w[4];
 #pragma unroll
@@ -384,8 +393,8 @@ struct SmemLayout {
   static constexpr int kBBytes = BN * BK;
   static constexpr int kStageBytes = kABytes + kBBytes;
   // ring depth: shallower when the tail buffers are needed
-  static constexpr int kStagesNoTail = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int kStagesTail = (BN == 256) ? 3 : (BN == 128 ? 4 : 6);
+  static constexpr int kStagesNoTail = (BN == 256) ? 4 : (BN == 192 ? 4 : (BN == 128 ? 6 : 8));
+  static constexpr int kStagesTail = (BN == 256) ? 3 : (BN == 192 ? 3 : (BN == 128 ? 4 : 6));
   static constexpr int kMaxStages = kStagesNoTail;
   static constexpr int kTileBytes =
       (kStagesNoTail * kStageBytes > kStagesTail * kStageBytes + kTailBufs * kABytes)
@@ -401,42 +410,58 @@ struct SmemLayout {
   static constexpr int kDynBytes =
       kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes + kSrcTableBytes + kEpiBytes;
   static_assert(kDynBytes <= 227 * 1024, "more dynamic shared memory than a CTA can have");
+  // exchange buffer of a K split: CL slots of (BN / 4) chunk columns of (128 / CL + 1) cells of 16 bytes
+  static constexpr int kExchangeBytes = (BN / 4) * 16 * (BM + 8);   // CL * (128 / CL + 1) <= 136 for CL <= 8
+  static_assert(kExchangeBytes <= kStagesTail * kStageBytes, "the ring must hold the partial sums of one tile");
 };
 
-// One work item of a CTA: an output tile and a K slice.
+// One work item of a CTA: an output tile, and this CTA's share of its K-blocks.
 struct WorkItem {
-  int mt, nt, kz;
-  int my_kb, n_tma, n_tail;   // K-blocks of the slice: first those with a TMA-fed A tile, then the tail
+  int mt, nt;
+  int my_kb, n_tma, n_tail;   // K-blocks of the share: first those with a TMA-fed A tile, then the tail
 };
 
-// Item j of this CTA's cluster (items are dealt round-robin to the clusters of the grid; the CTAs of
-// a cluster take neighbouring N tiles of the same M tile and K slice).
+// Item j of this CTA's cluster (tiles are dealt round-robin to the clusters of the grid; CTA `crank` of the
+// cluster takes K-blocks crank, crank + CL, ... of every tile).
 __device__ __forceinline__ bool work_item(const GemmParams& p, int j, uint32_t crank, uint32_t CL, WorkItem* w) {
   const long long idx = (long long)blockIdx.x + (long long)j * gridDim.x;
   if (idx >= p.total_items) return false;
-  const int ntg = (int)(idx % p.n_groups);
-  const long long rest = idx / p.n_groups;
-  w->mt = (int)(rest % p.m_tiles);
-  w->kz = (int)(rest / p.m_tiles);
-  w->nt = ntg * (int)CL + (int)crank;
-  w->my_kb = (p.num_kb - w->kz + p.split_k - 1) / p.split_k;
-  w->n_tma = p.kb_tma_a > w->kz ? min(w->my_kb, (p.kb_tma_a - w->kz + p.split_k - 1) / p.split_k) : 0;
+  w->nt = (int)(idx % p.n_tiles);
+  w->mt = (int)(idx / p.n_tiles);
+  const int kz = (int)crank, sk = (int)CL;
+  w->my_kb = p.num_kb > kz ? (p.num_kb - kz + sk - 1) / sk : 0;
+  w->n_tma = p.kb_tma_a > kz ? min(w->my_kb, (p.kb_tma_a - kz + sk - 1) / sk) : 0;
   w->n_tail = w->my_kb - w->n_tma;
   return true;
 }
 
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// 16 bytes into a (peer) CTA's shared memory, asynchronously: the store counts 16 bytes toward the transaction
+// count of the barrier `mbar` in the destination CTA, which is how the receiver learns that the data is there.
+__device__ __forceinline__ void st_async_v4(uint32_t addr, uint4 v, uint32_t mbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(mbar) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmA, const GemmParams p) {
+ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmA,
+                const __grid_constant__ CUtensorMap tmAT, const GemmParams p) {
   using L = SmemLayout<BN>;
   extern __shared__ unsigned char smem_dyn[];
   const uint32_t raw = smem_u32(smem_dyn);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* tiles = smem_dyn + (base - raw);
   unsigned char* ctrl = tiles + L::kTileBytes;
-  // barriers: full[kMaxStages], empty[kMaxStages], gfull[kTailBufs], gempty[kTailBufs], acc_full[2], acc_empty[2]
+  // barriers: full[kMaxStages], empty[kMaxStages], gfull[kTailBufs], gempty[kTailBufs], acc_full[2], acc_empty[2],
+  // xready, xfull, xdone (exchange of the K slices' partial tiles)
   uint64_t* bars = reinterpret_cast<uint64_t*>(ctrl);
-  constexpr int kNumBars = 2 * L::kMaxStages + 2 * kTailBufs + 4;
+  constexpr int kNumBars = 2 * L::kMaxStages + 2 * kTailBufs + 4 + 3;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl + 8 * kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 8 * kNumBars + 8);
   RowInfo* rows = reinterpret_cast<RowInfo*>(ctrl + L::kCtrlBytes);
@@ -448,13 +473,60 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   auto gempty_bar = [&](int g) { return smem_u32(bars + 2 * L::kMaxStages + kTailBufs + g); };
   auto accfull_bar = [&](int a) { return smem_u32(bars + 2 * L::kMaxStages + 2 * kTailBufs + a); };
   auto accempty_bar = [&](int a) { return smem_u32(bars + 2 * L::kMaxStages + 2 * kTailBufs + 2 + a); };
+  const uint32_t xready_bar = smem_u32(bars + 2 * L::kMaxStages + 2 * kTailBufs + 4);
+  const uint32_t xfull_bar = xready_bar + 8, xdone_bar = xready_bar + 16;
   const int stages = p.num_kb > p.kb_tma_a ? L::kStagesTail : L::kStagesNoTail;
   const uint32_t tail_base = base + stages * L::kStageBytes;   // kTailBufs A tiles (only with tail blocks)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // The CTAs of a cluster share the M tile and the K slice and differ in the N tile: they need the
-  // same assembled A tiles, so each assembles 1/CL of the rows and stores them into every peer.
+  // The CTAs of a cluster work on the same output tile and split its K-blocks.
   const uint32_t crank = cluster_rank(), CL = cluster_size();
+
+  // The TMA producer is thread 0, the thread that sets up the barriers: it requests the first ring of operand
+  // tiles right after that, before the CTA waits for the tensor-memory allocation and for its cluster peers, so
+  // that the set-up time overlaps the first bytes' way from DRAM.  (Its own barriers are ready; the tiles land in
+  // this CTA's own shared memory.)
+  int prod_j = 0, prod_i = 0, prod_it = 0;   // producer position: work item, K-block inside it, ring slot counter
+  bool prod_ok = true;
+  // thread 0 only: issue K-blocks until `limit_it` have been issued (first_tile_only: and stay inside the first tile)
+  auto produce = [&](int limit_it, bool first_tile_only) {
+    WorkItem w;
+    while (prod_ok && prod_it < limit_it && work_item(p, prod_j, crank, CL, &w)) {
+      if (prod_i >= w.my_kb) {
+        if (first_tile_only) break;
+        ++prod_j; prod_i = 0;
+        continue;
+      }
+      if (CL > 1 && prod_i == 0 && prod_j > 0) {
+        // the ring doubles as the exchange buffer of the previous tile's partial sums: wait until this CTA
+        // has summed them, then hand the memory back to the copy engine
+        if (!mbar_wait(xdone_bar, (uint32_t)(prod_j - 1) & 1u, abort_flag)) { prod_ok = false; break; }
+        fence_proxy_async_smem();
+      }
+      const int i = prod_i, it = prod_it;
+      const int kb = (int)crank + i * (int)CL;
+      const int s = it % stages;
+      const uint32_t par = ((it / stages) & 1) ^ 1;
+      if (!mbar_wait(empty_bar(s), par, abort_flag)) { prod_ok = false; break; }
+      const uint32_t a_dst = base + s * L::kStageBytes;
+      const uint32_t b_dst = a_dst + L::kABytes;
+      const bool a_tma = i < w.n_tma;
+      mbar_arrive_expect_tx(full_bar(s), L::kBBytes + (a_tma ? p.a_box_bytes : 0));
+      tma_load_2d(b_dst, &tmB, full_bar(s), kb * BK, w.nt * BN);
+      if (a_tma) {
+        if (p.mode == MODE_LINEAR) {
+          tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, w.mt * BM);
+        } else {
+          const int k0 = kb * BK;
+          const int tap = k0 / p.Cp, c0 = k0 - tap * p.Cp;
+          const int tw = w.mt % p.tiles_w, th = (w.mt / p.tiles_w) % p.tiles_h, tn = w.mt / (p.tiles_w * p.tiles_h);
+          tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw * p.stride + tap % p.kw - p.pad,
+                      th * p.bh * p.stride + tap / p.kw - p.pad, tn * p.bn);
+        }
+      }
+      ++prod_i; ++prod_it;
+    }
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -462,56 +534,37 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       mbar_init(empty_bar(s), 1);
     }
     for (int g = 0; g < kTailBufs; ++g) {
-      mbar_init(gfull_bar(g), (kGatherThreads / 32) * CL);   // every gather warp of every CTA of the cluster
-      mbar_init(gempty_bar(g), CL);                          // every CTA's MMA issuer
+      mbar_init(gfull_bar(g), p.tail_T ? 1 : kGatherThreads / 32);   // every gather warp, or the one that issues copies
+      mbar_init(gempty_bar(g), 1);                    // the MMA issuer
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(accfull_bar(a), 1);    // the MMA issuer's commit
       mbar_init(accempty_bar(a), kEpiWarps);   // every epilogue warp
     }
+    mbar_init(xready_bar, CL);               // every CTA of the cluster: "my ring may be written"
+    mbar_init(xfull_bar, 1);                 // this CTA's own announcement of the bytes it expects; the partial rows
+                                             // then arrive as asynchronous stores that count against it
+    mbar_init(xdone_bar, kEpiWarps);         // this CTA's epilogue warps: "the exchange buffer has been read"
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmB);
     if (p.kb_tma_a > 0) prefetch_tmap(&tmA);
+    if (p.tail_T) prefetch_tmap(&tmAT);
+    produce(stages, true);    // the first ring: its slots are free by construction
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 2 * BN);   // two accumulators: the epilogue of one tile
+  constexpr uint32_t kTmemCols = 2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512);   // a power of two
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);   // two accumulators: the epilogue of one tile
   tc_fence_before();                                        // overlaps the main loop of the next
   __syncthreads();
-  cluster_sync_all();   // no peer touches our barriers or tiles before they are set up
+  cluster_sync_all();   // no peer touches our barriers or our ring before they are set up
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      int it = 0;   // K-blocks issued so far (the ring runs on across tiles)
-      WorkItem w;
-      bool ok = true;
-      for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
-        for (int i = 0; i < w.my_kb; ++i, ++it) {
-          const int kb = w.kz + i * p.split_k;
-          const int s = it % stages;
-          const uint32_t par = ((it / stages) & 1) ^ 1;
-          if (!mbar_wait(empty_bar(s), par, abort_flag)) { ok = false; break; }
-          const uint32_t a_dst = base + s * L::kStageBytes;
-          const uint32_t b_dst = a_dst + L::kABytes;
-          const bool a_tma = i < w.n_tma;
-          mbar_arrive_expect_tx(full_bar(s), L::kBBytes + (a_tma ? p.a_box_bytes : 0));
-          tma_load_2d(b_dst, &tmB, full_bar(s), kb * BK, w.nt * BN);
-          if (a_tma) {
-            if (p.mode == MODE_LINEAR) {
-              tma_load_2d(a_dst, &tmA, full_bar(s), kb * BK, w.mt * BM);
-            } else {
-              const int k0 = kb * BK;
-              const int tap = k0 / p.Cp, c0 = k0 - tap * p.Cp;
-              const int tw = w.mt % p.tiles_w, th = (w.mt / p.tiles_w) % p.tiles_h, tn = w.mt / (p.tiles_w * p.tiles_h);
-              tma_load_4d(a_dst, &tmA, full_bar(s), c0, tw * p.bw * p.stride + tap % p.kw - p.pad,
-                          th * p.bh * p.stride + tap / p.kw - p.pad, tn * p.bn);
-            }
-          }
-        }
-      }
-      if (*abort_flag && it > 0) {
+      produce(0x7fffffff, false);
+      if (*abort_flag && prod_it > 0) {
         // give copies that are still in flight time to land before the CTA's shared memory is released
         for (int i = 0; i < 2000; ++i) __nanosleep(100);
       }
@@ -520,7 +573,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       const uint32_t idesc = instr_desc_i8(BN, p.a_signed);
-      const uint16_t all_ctas = (uint16_t)((1u << CL) - 1u);
+      const uint32_t idesc_mn = idesc | (1u << 15);   // A operand stored MN-major (a tail tile made of channel rows)
       WorkItem w;
       int total_tail = 0;   // tail tiles this CTA consumes over all its items
       for (int j = 0; work_item(p, j, crank, CL, &w); ++j) total_tail += w.n_tail;
@@ -538,21 +591,30 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
           uint32_t a_addr = base + s * L::kStageBytes;
           const uint32_t b_addr = a_addr + L::kABytes;
-          const bool tail = i >= w.n_tma;   // the A tile is assembled by the cluster's gather warps
+          const bool tail = i >= w.n_tma;   // the A tile is assembled by the gather warps
           if (tail) {
-            if (!mbar_wait_cluster(gfull_bar(tt % kTailBufs), (uint32_t)(tt / kTailBufs) & 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(gfull_bar(tt % kTailBufs), (uint32_t)(tt / kTailBufs) & 1u, abort_flag)) { ok = false; break; }
             a_addr = tail_base + (tt % kTailBufs) * L::kABytes;
           }
           tc_fence_after();
+          if (tail && p.tail_T) {
+            // the tile holds one 128-byte row per contraction index (MN-major): 32 indices = 4 KB per instruction
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            umma_i8(d_tmem, smem_desc_sw128(a_addr + k * UMMA_K), smem_desc_sw128(b_addr + k * UMMA_K), idesc,
-                    (i > 0 || k > 0) ? 1u : 0u);
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              umma_i8(d_tmem, smem_desc_sw128(a_addr + k * UMMA_K * 128), smem_desc_sw128(b_addr + k * UMMA_K), idesc_mn,
+                      (i > 0 || k > 0) ? 1u : 0u);
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              umma_i8(d_tmem, smem_desc_sw128(a_addr + k * UMMA_K), smem_desc_sw128(b_addr + k * UMMA_K), idesc,
+                      (i > 0 || k > 0) ? 1u : 0u);
+            }
           }
           umma_commit(empty_bar(s));  // frees the stage when these MMAs have read it
           if (tail) {
-            // ... and tells every CTA of the cluster that this CTA is done with the tail buffer, if it is reused
-            if (tt + kTailBufs < total_tail) umma_commit_multicast(gempty_bar(tt % kTailBufs), all_ctas);
+            // ... and the tail buffer, if it is filled again
+            if (tt + kTailBufs < total_tail) umma_commit(gempty_bar(tt % kTailBufs));
             ++tt;
           }
         }
@@ -561,18 +623,58 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     }
   } else if (warp < 6) {
     // ---------------------------------------------------------------- gather producers
-    // This CTA assembles rows [crank * RP, (crank + 1) * RP) of every tail tile: RP * 8 chunks of 16
-    // bytes, dealt so that neighbouring threads work on the same rows (one pixel's channels share
-    // cache lines).  The tail buffers are separate from the TMA ring, so the gather runs ahead of
-    // the TMA-fed main loop (also across tiles).
+    // The four warps assemble every tail tile of this CTA: 128 rows x 8 chunks of 16 bytes, dealt so that
+    // neighbouring threads work on the same rows (one pixel's channels share cache lines).  The tail buffers
+    // are separate from the TMA ring, so the gather runs ahead of the TMA-fed main loop (also across tiles).
     const int gt = threadIdx.x - 64;   // 0..127
-    const int RP = BM / (int)CL;
     bool bad = false;
     bool ok = true;
     int tt = 0;          // tail tiles assembled so far
+    if (p.tail_T) {
+      // Linear layer with a channel-major copy of the activations: contraction index k of a tail block is channel
+      // idx_map[k], and that channel's values for the tile's 128 rows are 128 contiguous bytes of the copy.  One
+      // warp asks the copy engine for them, one row per index; the tile is MN-major (row k = index k).  No thread
+      // touches an activation byte.
+      if (warp == 2) {
+        int buf_kb[kTailBufs];
+        for (int g = 0; g < kTailBufs; ++g) buf_kb[g] = -1;
+        WorkItem w;
+        for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
+          for (int t = 0; t < w.n_tail; ++t, ++tt) {
+            const int kb = (int)crank + (w.n_tma + t) * (int)CL;
+            const int g = tt % kTailBufs;
+            if (tt >= kTailBufs && !mbar_wait(gempty_bar(g), (uint32_t)(tt / kTailBufs - 1) & 1u, abort_flag)) {
+              ok = false;
+              break;
+            }
+            const int n_valid = min(BK, p.Ktot - kb * BK);
+            const uint32_t tile_local = tail_base + g * L::kABytes;
+            if (n_valid < BK && buf_kb[g] != kb) {   // rows past the last contraction index: zero
+              for (int r = n_valid + lane; r < BK; r += 32)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) st_local_v4(tile_local + r * 128 + c * 16, make_uint4(0u, 0u, 0u, 0u));
+            }
+            buf_kb[g] = kb;
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_expect_tx(gfull_bar(g), (uint32_t)n_valid * 128u);
+            __syncwarp();
+            for (int k = lane; k < n_valid; k += 32) {
+              const int kk = kb * BK + k;
+              const int ch = kk < p.C ? kk : checked_src(p, kk, &bad);
+              tma_load_2d(tile_local + k * 128, &tmAT, gfull_bar(g), w.mt * BM, ch);
+            }
+          }
+        }
+        if (*abort_flag && tt > 0)
+          for (int i = 0; i < 2000; ++i) __nanosleep(100);   // copies still in flight land before the CTA leaves
+      }
+      if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
+      ok = false;   // nothing left for the byte gather below
+    }
     int n_tiles_done = 0;
     int table_kb[2] = {-1, -1};   // which K-block each of the two source tables describes
-    int buf_kb[kTailBufs];        // which K-block each tail buffer held last (same for every CTA of the cluster)
+    int buf_kb[kTailBufs];        // which K-block each tail buffer held last
     for (int g = 0; g < kTailBufs; ++g) buf_kb[g] = -1;
     WorkItem w;
     for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
@@ -583,9 +685,9 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       trow[gt] = row_info(p, w.mt, gt);
       asm volatile("bar.sync 1, 128;" ::: "memory");
       for (int t = 0; t < w.n_tail; ++t, ++tt) {
-        const int kb = w.kz + (w.n_tma + t) * p.split_k;
+        const int kb = (int)crank + (w.n_tma + t) * (int)CL;
         const int g = tt % kTailBufs;
-        if (tt >= kTailBufs && !mbar_wait_cluster(gempty_bar(g), (uint32_t)(tt / kTailBufs - 1) & 1u, abort_flag)) {
+        if (tt >= kTailBufs && !mbar_wait(gempty_bar(g), (uint32_t)(tt / kTailBufs - 1) & 1u, abort_flag)) {
           ok = false;
           break;
         }
@@ -603,11 +705,10 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         }
         const uint32_t tile_local = tail_base + g * L::kABytes;
         // (row, chunk) pairs with data, dealt evenly over the threads
-        const int n_valid = RP * valid_chunks;
+        const int n_valid = BM * valid_chunks;
 #pragma unroll 2
         for (int it = gt; it < n_valid; it += kGatherThreads) {
-          const int rl = it / valid_chunks, c = it - rl * valid_chunks;
-          const int r = (int)crank * RP + rl;
+          const int r = it / valid_chunks, c = it - r * valid_chunks;
           const RowInfo ri = trow[r];
           uint4 v;
           if (ri.out_row < 0) {
@@ -620,30 +721,22 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             else rbase = p.A + (((long long)ri.n * p.H + ri.ih0) * p.Wd + ri.iw0) * p.C;
             v = gather_chunk(p, ri, rbase, tab + c * 16);
           }
-          const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
-          if (CL == 1) st_local_v4(off, v);   // a lone CTA: plain shared-memory stores
-          else
-            for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), v);
+          st_local_v4(tile_local + r * 128 + ((c ^ (r & 7)) << 4), v);
         }
         // the K padding: zero, unless this buffer's last occupant was the same K-block (every tile of a layer
         // has the same tail blocks, so the chunks that hold data are overwritten and the padding stays zero)
         const int zero_chunks = 8 - valid_chunks;
         if (buf_kb[g] != kb) {
-          for (int it = gt; it < RP * zero_chunks; it += kGatherThreads) {
-            const int rl = it / zero_chunks, c = valid_chunks + (it - rl * zero_chunks);
-            const int r = (int)crank * RP + rl;
-            const uint32_t off = tile_local + r * 128 + ((c ^ (r & 7)) << 4);
-            if (CL == 1) st_local_v4(off, make_uint4(0u, 0u, 0u, 0u));
-            else
-              for (uint32_t dst = 0; dst < CL; ++dst) st_peer_v4(peer_addr(off, dst), make_uint4(0u, 0u, 0u, 0u));
+          for (int it = gt; it < BM * zero_chunks; it += kGatherThreads) {
+            const int r = it / zero_chunks, c = valid_chunks + (it - r * zero_chunks);
+            st_local_v4(tile_local + r * 128 + ((c ^ (r & 7)) << 4), make_uint4(0u, 0u, 0u, 0u));
           }
           buf_kb[g] = kb;
         }
         // make the generic-proxy stores visible to the tensor cores that read them
-        if (CL == 1) fence_proxy_async_smem(); else fence_proxy_async_cluster();
+        fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0)
-          for (uint32_t dst = 0; dst < CL; ++dst) mbar_arrive_peer(peer_addr(gfull_bar(g), dst));
+        if (lane == 0) mbar_arrive(gfull_bar(g));
       }
     }
     if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
@@ -652,13 +745,14 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     // warp w may read tensor-memory lanes 32*(w%4) .. +31
     const int q = warp & 3;
     const float sc = __fmul_rn(__ldg(p.a_scale), __ldg(p.w_scale));
-    const bool direct = p.split_k == 1;
+    const bool direct = CL == 1;
     WorkItem w;
     bool ok = true;
     for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
       const int acc = j & 1;
       const RowInfo ri = row_info(p, w.mt, q * 32 + lane);
-      const int nt = w.nt, kz = w.kz;
+      const int nt = w.nt;
+      const int ew = warp - 6, half = ew >> 2;
       if (p.residual && direct && ri.out_row >= 0) {
         // the shortcut tensor's part of this tile is asked into L2 while the main loop still runs
         const float* rrow = p.residual + ri.out_row * p.ldy + (long long)nt * BN;
@@ -666,39 +760,159 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         for (int c = (warp >= 10 ? 32 : 0); c < BN && c < n_left; c += 64)
           asm volatile("prefetch.global.L2 [%0];" ::"l"(rrow + c));
       }
-      // A warp whose wait ran out leaves at once when the output is written directly; with split K it first
-      // goes through this item's three barriers with the other epilogue warps (skipping its own work), so that
-      // all eight stop at the same place
-      const bool got = mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag);
-      if (!got) {
-        ok = false;
-        if (direct) break;
-      }
+      if (!mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
+      if (!direct) {
+        // ------------------------------------------------------------ K split over the cluster: exchange and sum
+        // CTA r of the cluster finishes rows [r * RP, (r + 1) * RP) of the tile.  The exchange buffer is the TMA
+        // ring of the owning CTA (idle now: the producer does not start the next tile before the sum is done):
+        // slot s holds sender s's partial sums of the owner's rows, [RP][BN] int32.
+        const int RP = BM / (int)CL;
+        const uint32_t xparity = (uint32_t)j & 1u;
+        // (1) this CTA's tensor cores are done with its ring: it announces the bytes it is about to receive (the
+        // rows it owns, from every CTA of the cluster including itself) and tells every CTA that it may be written
+        const uint32_t cell_stride = (uint32_t)(RP + 1) * 16u;                 // bytes from one chunk to the next
+        const uint32_t slot_bytes = (uint32_t)(BN / 4) * cell_stride;
+        if (ew == 0 && lane == 0) {
+          mbar_arrive_expect_tx(xfull_bar, CL * (uint32_t)(RP * BN) * 4u);
+          for (uint32_t dst = 0; dst < CL; ++dst) mbar_arrive_peer(peer_addr(xready_bar, dst));
+        }
+        // (2) ... and this CTA writes into the others' once they have said the same
+        if (!mbar_wait_cluster(xready_bar, xparity, abort_flag)) { ok = false; break; }
+        // (3) a lane holds one row of the accumulator, 32 columns at a time.  The exchange buffer is laid out in
+        // 16-byte cells [sender][4-column chunk][row of the owner] (+1 cell of padding per chunk): the lanes of a
+        // warp, which hold consecutive rows, store consecutive cells, and the owner later reads consecutive chunks
+        // of one row without bank conflicts.  The stores are asynchronous and count against the owner's barrier.
+        {
+          const int m = q * 32 + lane;
+          const uint32_t owner = (uint32_t)(m / RP);
+          const uint32_t cell0 = base + crank * slot_bytes + (uint32_t)(m - (int)owner * RP) * 16u;
+          const uint32_t dst_cell0 = peer_addr(cell0, owner);
+          const uint32_t dst_bar = peer_addr(xfull_bar, owner);
+          for (int c0 = half * 32; c0 < BN; c0 += 64) {
+            uint32_t v[32];
+            __syncwarp();
+            tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
+#pragma unroll
+            for (int jj = 0; jj < 32; jj += 4)
+              st_async_v4(dst_cell0 + (uint32_t)((c0 + jj) >> 2) * cell_stride, make_uint4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]),
+                          dst_bar);
+          }
+        }
+        // the accumulator has been read out: hand it back to the MMA issuer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(accempty_bar(acc));
+        // (4) all partial sums of this CTA's rows are in place
+        if (!mbar_wait_cluster(xfull_bar, xparity, abort_flag)) { ok = false; break; }
+        // (5) sum the CL slots and finish the rows: a thread takes four consecutive columns
+        {
+          const int et = threadIdx.x - 6 * 32;                    // 0..255
+          const int n_lim = min(BN, p.N - nt * BN);
+          const bool vec = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 15) == 0) && (p.ldy % 4 == 0) &&
+                           (!p.acc_out || (reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) &&
+                           (!p.residual || (reinterpret_cast<uintptr_t>(p.residual) & 15) == 0);
+          // This code runs once per tile and its instructions come straight from L2: on a 40 us kernel every
+          // instruction of it costs about as much as 16 cycles, so the common case (a whole tile of a linear
+          // layer, aligned output, no shortcut tensor, no copy of the accumulators) has its own short loop.
+          constexpr int kQuads = BN / 4;                          // 4-column groups per tile row
+          const int total = RP * kQuads;
+          const unsigned char* ring = tiles;                      // the exchange buffer: this CTA's ring
+          float fmx = 0.0f;
+          const bool lean = vec && p.mode == MODE_LINEAR && n_lim == BN && !p.residual && !p.acc_out &&
+                            (!p.bias || (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0) &&
+                            (long long)(w.mt + 1) * BM <= p.M;
+          if (lean) {
+            const float* bias_n = p.bias ? p.bias + nt * BN : nullptr;
+            float* ybase = p.Y + ((long long)w.mt * BM + (long long)crank * RP) * p.ldy + (long long)nt * BN;
+            for (int g = et; g < total; g += 256) {
+              const int rl = g / kQuads, c = (g - rl * kQuads) * 4;
+              const unsigned char* src = ring + (uint32_t)(c >> 2) * cell_stride + (uint32_t)rl * 16u;
+              int4 a = *reinterpret_cast<const int4*>(src);
+              for (uint32_t sl = 1; sl < CL; ++sl) {
+                const int4 v = *reinterpret_cast<const int4*>(src + sl * slot_bytes);
+                a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+              }
+              float4 b4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+              if (bias_n) b4 = __ldg(reinterpret_cast<const float4*>(bias_n + c));
+              // cvt.rn.f32.s32: the same value as the conversion of the direct epilogue, in one instruction
+              float4 f = make_float4(fmaf(__int2float_rn(a.x), sc, b4.x), fmaf(__int2float_rn(a.y), sc, b4.y),
+                                     fmaf(__int2float_rn(a.z), sc, b4.z), fmaf(__int2float_rn(a.w), sc, b4.w));
+              if (p.relu) { f.x = fmaxf(f.x, 0.0f); f.y = fmaxf(f.y, 0.0f); f.z = fmaxf(f.z, 0.0f); f.w = fmaxf(f.w, 0.0f); }
+              fmx = fmaxf(fmx, fmaxf(fmaxf(fabsf(f.x), fabsf(f.y)), fmaxf(fabsf(f.z), fabsf(f.w))));
+              *reinterpret_cast<float4*>(ybase + (long long)rl * p.ldy + c) = f;
+            }
+          } else {
+            for (int g = et; g < total; g += 256) {
+              const int rl = g / kQuads, cc = g - rl * kQuads, c = cc * 4;
+              if (c >= n_lim) continue;
+              const long long orow = row_info(p, w.mt, (int)crank * RP + rl).out_row;
+              if (orow < 0) continue;
+              const unsigned char* src = ring + (uint32_t)cc * cell_stride + (uint32_t)rl * 16u;
+              int4 a = *reinterpret_cast<const int4*>(src);
+              for (uint32_t sl = 1; sl < CL; ++sl) {
+                const int4 v = *reinterpret_cast<const int4*>(src + sl * slot_bytes);
+                a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+              }
+              const int n = nt * BN + c;
+              const int av[4] = {a.x, a.y, a.z, a.w};
+              float f[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const bool in = c + e < n_lim;
+                f[e] = fmaf(__int2float_rn(av[e]), sc, (p.bias && in) ? __ldg(p.bias + n + e) : 0.0f);
+                if (p.residual && in) f[e] = __fadd_rn(f[e], p.residual[orow * p.ldy + n + e]);
+                if (p.relu) f[e] = f[e] > 0.0f ? f[e] : 0.0f;
+                if (in) fmx = fmaxf(fmx, fabsf(f[e]));
+              }
+              float* y = p.Y + orow * p.ldy + n;
+              if (vec) {
+                *reinterpret_cast<float4*>(y) = make_float4(f[0], f[1], f[2], f[3]);
+                if (p.acc_out) *reinterpret_cast<int4*>(p.acc_out + orow * p.ldy + n) = a;
+              } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  if (c + e < n_lim) {
+                    y[e] = f[e];
+                    if (p.acc_out) p.acc_out[orow * p.ldy + n + e] = av[e];
+                  }
+                }
+              }
+            }
+          }
+          if (p.max_bits) {
+            for (int o = 16; o > 0; o >>= 1) fmx = fmaxf(fmx, __shfl_xor_sync(0xffffffffu, fmx, o));
+            if (lane == 0 && fmx > 0.0f) atomicMax(p.max_bits, __float_as_uint(fmx));
+          }
+        }
+        // (6) the ring may be refilled
+        __syncwarp();
+        if (lane == 0) mbar_arrive(xdone_bar);
+        continue;
+      }
+      // ------------------------------------------------------------ one CTA per tile: straight to the output
       // Each lane holds one row of a 32 x 16 piece of the accumulator; written out that way a store
       // instruction would touch 32 rows with 16 bytes each.  The piece goes through shared memory instead, so
       // that four neighbouring lanes write 64 contiguous bytes of one row (lane -> row i*8 + (qd&1)*4 + qd/2
       // with qd = lane/4, words (lane%4)*4 .. +3; the row order keeps the shared-memory reads conflict-free).
       // The two epilogue warps that share a tensor-memory lane quadrant take alternate pieces.
-      const int ew = warp - 6, half = ew >> 2;
       uint32_t* st_words = reinterpret_cast<uint32_t*>(epi_stage + (size_t)ew * L::kEpiWarpBytes);
       long long* st_rows = reinterpret_cast<long long*>(st_words + 32 * L::kEpiRowWords);
       __syncwarp();
       st_rows[lane] = ri.out_row;
       __syncwarp();
       const int qd = lane >> 2, sub = (qd & 1) * 4 + (qd >> 1), cq = (lane & 3) * 4;
-      // destination of the words: Y (and acc_out), or this slice's partial sums [kz][row][n]
-      uint32_t* dst0 = direct ? reinterpret_cast<uint32_t*>(p.Y) : reinterpret_cast<uint32_t*>(p.acc_ws) + (long long)kz * p.out_rows * p.N;
-      const long long ldd = direct ? p.ldy : (long long)p.N;
+      uint32_t* dst0 = reinterpret_cast<uint32_t*>(p.Y);
+      const long long ldd = p.ldy;
       const bool base_vec = ((reinterpret_cast<uintptr_t>(dst0) & 15) == 0) && (ldd % 4 == 0);
       const bool acc_vec = p.acc_out && ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) && (p.ldy % 4 == 0);
       // the shortcut tensor is read with 128-bit loads only when it is itself 16-byte aligned (a view that
       // starts a few floats into a buffer takes the scalar loads)
       const bool res_vec = p.residual && ((reinterpret_cast<uintptr_t>(p.residual) & 15) == 0) && (p.ldy % 4 == 0);
       float tile_max = 0.0f;
-      const bool want_max = direct && p.max_bits != nullptr;
+      const bool want_max = p.max_bits != nullptr;
       // a warp whose 32 rows are all padding (a short M tile) has nothing to write
-      const bool warp_has_rows = got && __any_sync(0xffffffffu, ri.out_row >= 0);
+      const bool warp_has_rows = __any_sync(0xffffffffu, ri.out_row >= 0);
       for (int c0 = half * kEpiCols; warp_has_rows && c0 < BN; c0 += 2 * kEpiCols) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
@@ -714,7 +928,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         __syncwarp();
         // this lane's four columns of every row it writes: their bias once per piece
         float b4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (direct && p.bias) {
+        if (p.bias) {
 #pragma unroll
           for (int e = 0; e < 4; ++e)
             if (n0 + cq + e < p.N) b4[e] = __ldg(p.bias + n0 + cq + e);
@@ -728,66 +942,62 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           orow[i] = st_rows[r];
           a[i] = *reinterpret_cast<const uint4*>(st_words + r * L::kEpiRowWords + cq);
         }
-        if (direct) {
-          uint4 o[4];
+        uint4 o[4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            float f0 = fmaf(int_to_float_rn((int)a[i].x), sc, b4[0]), f1 = fmaf(int_to_float_rn((int)a[i].y), sc, b4[1]);
-            float f2 = fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]), f3 = fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]);
-            if (p.residual && orow[i] >= 0) {   // the block's shortcut: one more rounded addition per output
-              const float* rr = p.residual + orow[i] * p.ldy + n0 + cq;
-              if (full && res_vec) {
-                const float4 r4 = __ldcs(reinterpret_cast<const float4*>(rr));
-                f0 = __fadd_rn(f0, r4.x); f1 = __fadd_rn(f1, r4.y); f2 = __fadd_rn(f2, r4.z); f3 = __fadd_rn(f3, r4.w);
-              } else {
-                if (n0 + cq + 0 < p.N) f0 = __fadd_rn(f0, rr[0]);
-                if (n0 + cq + 1 < p.N) f1 = __fadd_rn(f1, rr[1]);
-                if (n0 + cq + 2 < p.N) f2 = __fadd_rn(f2, rr[2]);
-                if (n0 + cq + 3 < p.N) f3 = __fadd_rn(f3, rr[3]);
-              }
-            }
-            if (p.relu) {
-              f0 = f0 > 0.0f ? f0 : 0.0f; f1 = f1 > 0.0f ? f1 : 0.0f;
-              f2 = f2 > 0.0f ? f2 : 0.0f; f3 = f3 > 0.0f ? f3 : 0.0f;
-            }
-            if (want_max) {   // padding rows and columns past N are not part of the output
-              float rm;
-              if (full) {
-                rm = fmaxf(fmaxf(fabsf(f0), fabsf(f1)), fmaxf(fabsf(f2), fabsf(f3)));
-              } else {
-                rm = n0 + cq + 0 < p.N ? fabsf(f0) : 0.0f;
-                if (n0 + cq + 1 < p.N) rm = fmaxf(rm, fabsf(f1));
-                if (n0 + cq + 2 < p.N) rm = fmaxf(rm, fabsf(f2));
-                if (n0 + cq + 3 < p.N) rm = fmaxf(rm, fabsf(f3));
-              }
-              tile_max = fmaxf(tile_max, orow[i] >= 0 ? rm : 0.0f);
-            }
-            o[i] = make_uint4(__float_as_uint(f0), __float_as_uint(f1), __float_as_uint(f2), __float_as_uint(f3));
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            if (orow[i] < 0) continue;
-            uint32_t* d = dst0 + orow[i] * ldd + n0 + cq;
-            if (vec0) {
-              *reinterpret_cast<uint4*>(d) = o[i];
+        for (int i = 0; i < 4; ++i) {
+          float f0 = fmaf(int_to_float_rn((int)a[i].x), sc, b4[0]), f1 = fmaf(int_to_float_rn((int)a[i].y), sc, b4[1]);
+          float f2 = fmaf(int_to_float_rn((int)a[i].z), sc, b4[2]), f3 = fmaf(int_to_float_rn((int)a[i].w), sc, b4[3]);
+          if (p.residual && orow[i] >= 0) {   // the block's shortcut: one more rounded addition per output
+            const float* rr = p.residual + orow[i] * p.ldy + n0 + cq;
+            if (full && res_vec) {
+              const float4 r4 = __ldcs(reinterpret_cast<const float4*>(rr));
+              f0 = __fadd_rn(f0, r4.x); f1 = __fadd_rn(f1, r4.y); f2 = __fadd_rn(f2, r4.z); f3 = __fadd_rn(f3, r4.w);
             } else {
-              if (n0 + cq + 0 < p.N) d[0] = o[i].x;
-              if (n0 + cq + 1 < p.N) d[1] = o[i].y;
-              if (n0 + cq + 2 < p.N) d[2] = o[i].z;
-              if (n0 + cq + 3 < p.N) d[3] = o[i].w;
+              if (n0 + cq + 0 < p.N) f0 = __fadd_rn(f0, rr[0]);
+              if (n0 + cq + 1 < p.N) f1 = __fadd_rn(f1, rr[1]);
+              if (n0 + cq + 2 < p.N) f2 = __fadd_rn(f2, rr[2]);
+              if (n0 + cq + 3 < p.N) f3 = __fadd_rn(f3, rr[3]);
             }
+          }
+          if (p.relu) {
+            f0 = f0 > 0.0f ? f0 : 0.0f; f1 = f1 > 0.0f ? f1 : 0.0f;
+            f2 = f2 > 0.0f ? f2 : 0.0f; f3 = f3 > 0.0f ? f3 : 0.0f;
+          }
+          if (want_max) {   // padding rows and columns past N are not part of the output
+            float rm;
+            if (full) {
+              rm = fmaxf(fmaxf(fabsf(f0), fabsf(f1)), fmaxf(fabsf(f2), fabsf(f3)));
+            } else {
+              rm = n0 + cq + 0 < p.N ? fabsf(f0) : 0.0f;
+              if (n0 + cq + 1 < p.N) rm = fmaxf(rm, fabsf(f1));
+              if (n0 + cq + 2 < p.N) rm = fmaxf(rm, fabsf(f2));
+              if (n0 + cq + 3 < p.N) rm = fmaxf(rm, fabsf(f3));
+            }
+            tile_max = fmaxf(tile_max, orow[i] >= 0 ? rm : 0.0f);
+          }
+          o[i] = make_uint4(__float_as_uint(f0), __float_as_uint(f1), __float_as_uint(f2), __float_as_uint(f3));
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (orow[i] < 0) continue;
+          uint32_t* d = dst0 + orow[i] * ldd + n0 + cq;
+          if (vec0) {
+            *reinterpret_cast<uint4*>(d) = o[i];
+          } else {
+            if (n0 + cq + 0 < p.N) d[0] = o[i].x;
+            if (n0 + cq + 1 < p.N) d[1] = o[i].y;
+            if (n0 + cq + 2 < p.N) d[2] = o[i].z;
+            if (n0 + cq + 3 < p.N) d[3] = o[i].w;
           }
         }
-        if (!direct || p.acc_out) {
-          // raw sums: this K slice's partials, or the caller's copy of the accumulators
-          uint32_t* rbase = direct ? reinterpret_cast<uint32_t*>(p.acc_out) : dst0;
-          const long long rld = direct ? p.ldy : ldd;
-          const bool rvec = direct ? vec1 : vec0;
+        if (p.acc_out) {
+          // the caller's copy of the accumulators
+          uint32_t* rbase = reinterpret_cast<uint32_t*>(p.acc_out);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             if (orow[i] < 0) continue;
-            uint32_t* d = rbase + orow[i] * rld + n0 + cq;
-            if (rvec) {
+            uint32_t* d = rbase + orow[i] * p.ldy + n0 + cq;
+            if (vec1) {
               __stcg(reinterpret_cast<uint4*>(d), a[i]);
             } else {
               if (n0 + cq + 0 < p.N) d[0] = a[i].x;
@@ -805,98 +1015,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       // the accumulator has been read out: hand it back to the MMA issuer
       tc_fence_before();
       __syncwarp();
-      if (lane == 0 && got) mbar_arrive(accempty_bar(acc));
-      if (!direct) {
-        // Split K: this slice's partial tile is in the workspace.  The slice that finds every other slice's
-        // tag already set sums the partial tiles (integer sums: exact in any order) and applies the epilogue;
-        // nobody waits for anybody.  Each slice publishes its tag and then looks at the others', so the slice
-        // whose tag lands last sees all of them; if two finish close together both may do the sum -- they
-        // write identical values.
-        int* fin = reinterpret_cast<int*>(ctrl + 8 * kNumBars + 16);
-        asm volatile("bar.sync 2, 256;" ::: "memory");            // all eight epilogue warps have written their pieces
-        if (warp == 6 && lane == 0) {
-          int all = 0;
-          const int aborting = *abort_flag;                       // one reading decides for all eight warps
-          if (!aborting) {
-            unsigned long long* fl = p.slice_flags + ((long long)w.mt * p.n_tiles + nt) * p.split_k;
-            __threadfence();
-            asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(fl + kz), "l"(p.nonce) : "memory");
-            __threadfence();
-            all = 1;
-            for (int z = 0; z < p.split_k; ++z) {
-              unsigned long long v;
-              asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(fl + z) : "memory");
-              all &= (v == p.nonce);
-            }
-          }
-          fin[0] = all;
-          fin[1] = aborting;
-        }
-        asm volatile("bar.sync 2, 256;" ::: "memory");
-        const bool finisher = fin[0] != 0;
-        if (fin[1]) ok = false;                                   // every epilogue warp leaves after this item
-        asm volatile("bar.sync 2, 256;" ::: "memory");            // everybody has read the verdict before it is reused
-        if (finisher) {
-          const int et = threadIdx.x - 6 * 32;                    // 0..255
-          const int n_lim = min(BN, p.N - nt * BN);
-          const bool vec = (p.N % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 15) == 0) && (p.ldy % 4 == 0) &&
-                           (!p.acc_out || (reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0) &&
-                           (!p.residual || (reinterpret_cast<uintptr_t>(p.residual) & 15) == 0);
-          const long long slice = p.out_rows * (long long)p.N;
-          float fmx = 0.0f;
-          constexpr int kQuads = BN / 4;                          // 4-column groups per tile row
-          for (int g = et; g < BM * kQuads; g += 256) {
-            const int r = g / kQuads, c = (g - r * kQuads) * 4;
-            if (c >= n_lim) continue;
-            const long long orow = row_info(p, w.mt, r).out_row;
-            if (orow < 0) continue;
-            const int n = nt * BN + c;
-            const int32_t* src = p.acc_ws + orow * p.N + n;
-            int4 a = make_int4(0, 0, 0, 0);
-            if (vec) {
-              for (int z = 0; z < p.split_k; ++z) {
-                const int4 b = __ldcg(reinterpret_cast<const int4*>(src + z * slice));
-                a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-              }
-            } else {
-              for (int z = 0; z < p.split_k; ++z) {
-                const int32_t* q = src + z * slice;
-                a.x += __ldcg(q);
-                if (c + 1 < n_lim) a.y += __ldcg(q + 1);
-                if (c + 2 < n_lim) a.z += __ldcg(q + 2);
-                if (c + 3 < n_lim) a.w += __ldcg(q + 3);
-              }
-            }
-            const int av[4] = {a.x, a.y, a.z, a.w};
-            float f[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const bool in = c + e < n_lim;
-              f[e] = fmaf(int_to_float_rn(av[e]), sc, (p.bias && in) ? __ldg(p.bias + n + e) : 0.0f);
-              if (p.residual && in) f[e] = __fadd_rn(f[e], p.residual[orow * p.ldy + n + e]);
-              if (p.relu) f[e] = f[e] > 0.0f ? f[e] : 0.0f;
-              if (in) fmx = fmaxf(fmx, fabsf(f[e]));
-            }
-            float* y = p.Y + orow * p.ldy + n;
-            if (vec) {
-              *reinterpret_cast<float4*>(y) = make_float4(f[0], f[1], f[2], f[3]);
-              if (p.acc_out) *reinterpret_cast<int4*>(p.acc_out + orow * p.ldy + n) = a;
-            } else {
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                if (c + e < n_lim) {
-                  y[e] = f[e];
-                  if (p.acc_out) p.acc_out[orow * p.ldy + n + e] = av[e];
-                }
-              }
-            }
-          }
-          if (p.max_bits) {
-            for (int o = 16; o > 0; o >>= 1) fmx = fmaxf(fmx, __shfl_xor_sync(0xffffffffu, fmx, o));
-            if (lane == 0 && fmx > 0.0f) atomicMax(p.max_bits, __float_as_uint(fmx));
-          }
-        }
-      }
+      if (lane == 0) mbar_arrive(accempty_bar(acc));
     }
     tc_fence_before();
   }
@@ -906,7 +1025,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    tmem_dealloc(tmem_base, 2 * BN);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
   if (threadIdx.x == 0 && *abort_flag) flag(p.dev_status, OCS_DEV_TIMEOUT);
 }
@@ -943,8 +1062,7 @@ bool encode_u8(CUtensorMap* map, const void* base, int rank, const cuuint64_t* d
 
 struct GemmPlan {
   int BN;
-  int split_k;
-  int cluster;   // CTAs along N that share assembled A tiles
+  int split_k;   // = cluster size: CTAs that share an output tile and split its K-blocks
   int m_tiles, n_tiles;
 };
 
@@ -952,81 +1070,75 @@ struct GemmPlan {
 // a cluster must fit inside one GPC, so larger clusters leave SMs unused).
 constexpr int kClusterSizes[4] = {1, 2, 4, 8};
 constexpr int kClusterCapacity[4] = {148, 148, 132, 120};
-constexpr int kMaxSplitCtas = 2 * kNumSMs;   // split-K never uses more than two waves of CTAs
 
-// Tile width, K split and cluster size by a small time model in units of one TMA-fed K-block of a
-// 128 x 256 tile: a wave costs max(main loop, gather beside it) plus a fixed prologue/epilogue; the
-// gather of one assembled K-block costs about `gather_cost` such units and is divided by the cluster
-// size; split-K adds the reduction pass.  n_tail = K-blocks whose A tile is assembled by threads,
-// tail_k = contraction indices in them (only 16-index chunks that hold data cost gather time).
-// Self-test override (ocs_selftest_force_gemm_plan): tile width, K slices and cluster size taken as given where
-// they are valid for the problem.
-int g_force_bn = 0, g_force_sk = 0, g_force_cl = 0;
+// Self-test override (ocs_selftest_force_gemm_plan): tile width and K split taken as given where they are
+// valid for the problem.
+int g_force_bn = 0, g_force_sk = 0;
 
-GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, bool conv) {
+// Tile width and K split by a small time model (microseconds).  Measured on this part: an SM takes in about
+// 105 GB/s of operand tiles, all SMs together about 9.5 TB/s from L2 (the activation tile of a K-block is re-read
+// from L2 by every N tile, so narrow tiles spend that budget on re-reads), DRAM delivers about 6.3 TB/s, and a
+// 128 x 256 x 128 block of int8 MMAs takes about 0.27 us.  A wave of tiles costs the largest of those terms for
+// the most loaded CTA, or the gather beside it; a K split adds the exchange of the partial tiles.  K is split
+// only so far that all clusters are resident at once.  n_tail = K-blocks whose A tile is assembled by threads
+// or fetched as channel rows, tail_k = contraction indices in them.
+GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, bool conv, bool tail_by_tma) {
   if (g_force_bn) {
     const int BN = g_force_bn;
     const int n_tiles = (N + BN - 1) / BN;
-    int sk = g_force_sk < 1 ? 1 : g_force_sk;
-    if (sk > num_kb) sk = num_kb;
-    if ((long long)m_tiles * n_tiles * sk > kMaxSplitCtas && sk > 1) sk = 1;
-    int cl = g_force_cl < 1 ? 1 : g_force_cl;
-    if (n_tail == 0 || n_tiles % cl != 0) cl = 1;
-    return GemmPlan{BN, sk, cl, m_tiles, n_tiles};
+    int ci = 0;
+    while (ci < 3 && kClusterSizes[ci + 1] <= g_force_sk) ++ci;
+    while (ci > 0 && ((long long)m_tiles * n_tiles * kClusterSizes[ci] > kClusterCapacity[ci] || kClusterSizes[ci] > num_kb)) --ci;
+    return GemmPlan{BN, kClusterSizes[ci], m_tiles, n_tiles};
   }
-  GemmPlan best{64, 1, 1, m_tiles, (N + 63) / 64};
+  GemmPlan best{64, 1, m_tiles, (N + 63) / 64};
   double best_cost = 1e300;
-  const int bns[3] = {256, 128, 64};
-  const double gather_cost = conv ? 16.0 : 60.0;
-  for (int bi = 0; bi < 3; ++bi) {
+  const int bns[4] = {256, 192, 128, 64};
+  const double kSmIngest = 105e3, kL2Total = 9.5e6, kDram = 6.3e6;   // bytes per microsecond
+  const double gather_us = tail_by_tma ? 0.0 : (conv ? 4.0 : 16.0);  // per assembled K-block full of data
+  const double K = (double)num_kb * BK, Mrows = (double)m_tiles * BM;
+  const double dram_us = ((double)N * K + Mrows * K + 4.0 * Mrows * N) / kDram;
+  for (int bi = 0; bi < 4; ++bi) {
     const int BN = bns[bi];
     if (BN > 64 && N <= BN / 2) continue;  // tile mostly empty
     const int n_tiles = (N + BN - 1) / BN;
     const long long tiles = (long long)m_tiles * n_tiles;
-    const double t_block = (128.0 + BN) / 384.0;
-    int max_split = num_kb / 4;            // keep at least 4 K-blocks per slice
-    if (max_split < 1 || tiles >= kNumSMs) max_split = 1;
-    if (max_split > 32) max_split = 32;
-    for (int sk = 1; sk <= max_split; ++sk) {
-      const long long ctas = tiles * sk;
-      if (sk > 1 && ctas > kMaxSplitCtas) break;
-      const int main_blocks = (num_kb + sk - 1) / sk;
+    const double block_bytes = (double)(BM + BN) * BK;
+    const double mma_block_us = 0.27 * BN / 256.0;
+    for (int ci = 0; ci < 4; ++ci) {
+      const int sk = kClusterSizes[ci];
+      if (sk > 1 && (tiles * sk > kClusterCapacity[ci] || num_kb < 4 * sk)) continue;   // one resident wave, >= 4 blocks each
+      const long long waves = (tiles * sk + kClusterCapacity[ci] - 1) / kClusterCapacity[ci];
+      const int cta_blocks = (num_kb + sk - 1) / sk;
       const int tail_blocks = (n_tail + sk - 1) / sk;
-      for (int ci = 0; ci < 4; ++ci) {
-        const int cl = kClusterSizes[ci];
-        if (cl > 1 && (n_tail == 0 || n_tiles % cl != 0)) continue;
-        const long long waves = (ctas + kClusterCapacity[ci] - 1) / kClusterCapacity[ci];
-        const double main_t = main_blocks * t_block;
-        // the most loaded CTA assembles tail_blocks K-blocks, of which at most tail_k indices hold data
-        const int cta_k = tail_k < tail_blocks * BK ? tail_k : tail_blocks * BK;
-        const double gather_t = (0.5 * tail_blocks + (cta_k / 128.0) * gather_cost) / cl;
-        double cost = (double)waves * ((main_t > gather_t ? main_t : gather_t) + 4.0 * t_block);
-        if (sk > 1) cost += 1.0 + 0.25 * sk * t_block;   // partial tiles written, then summed by the last slice
-        cost *= 1.0 + 0.002 * ci + 0.001 * bi;   // ties: smaller cluster, wider tile
-        if (cost < best_cost) {
-          best_cost = cost;
-          best = GemmPlan{BN, sk, cl, m_tiles, n_tiles};
-        }
+      const double cta_bytes = (double)waves * cta_blocks * block_bytes;
+      const double total_bytes = (double)tiles * num_kb * block_bytes;
+      double stream = cta_bytes / kSmIngest;
+      if (total_bytes / kL2Total > stream) stream = total_bytes / kL2Total;
+      if (dram_us > stream) stream = dram_us;
+      if ((double)waves * cta_blocks * mma_block_us > stream) stream = (double)waves * cta_blocks * mma_block_us;
+      // the most loaded CTA assembles tail_blocks K-blocks per tile, of which at most tail_k indices hold data
+      const int cta_k = tail_k < tail_blocks * BK ? tail_k : tail_blocks * BK;
+      const double gather = (double)waves * (0.1 * tail_blocks + (cta_k / 128.0) * gather_us);
+      if (gather > stream) stream = gather;
+      double cost = 5.0 + stream + (double)waves * 1.0 * BN / 256.0;   // start-up, main loops, last epilogue
+      if (sk > 1) cost += 3.0 + 6.0 * BN / 256.0;                        // exchange and sum of the partial tiles
+      cost *= 1.0 + 0.002 * ci + 0.001 * bi;                             // ties: fewer slices, wider tile
+      if (cost < best_cost) {
+        best_cost = cost;
+        best = GemmPlan{BN, sk, m_tiles, n_tiles};
       }
     }
   }
   return best;
 }
 
-// Upper bound of the split-K scratch (partial tiles and the slices' tags) over every plan choose_plan can
-// return for this output.
-constexpr size_t kSliceFlagBytes = 64 * 1024;   // m_tiles * n_tiles < 148 when K is split, at most 32 slices, 8 bytes each
-size_t splitk_ws_bound(long long rows, int N, long long m_tiles) {
-  if (m_tiles * ((N + 255) / 256) >= kNumSMs) return 0;   // enough tiles: never split
-  long long ints = 32ll * rows * N;
-  const long long cap = (long long)kMaxSplitCtas * BM * 256;
-  if (ints > cap) ints = cap;
-  return align_up(4 * (size_t)ints, 256) + kSliceFlagBytes;
-}
+// The K split needs no global scratch (kept for the workspace queries' layout).
+size_t splitk_ws_bound(long long, int, long long) { return 0; }
 
 template <int BN>
-ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const GemmParams& p, const GemmPlan& plan,
-                       cudaStream_t stream) {
+ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const CUtensorMap& tmAT, const GemmParams& p,
+                       const GemmPlan& plan, cudaStream_t stream) {
   using L = SmemLayout<BN>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -1036,62 +1148,35 @@ ocs_status launch_gemm(const CUtensorMap& tmB, const CUtensorMap& tmA, const Gem
   }
   // persistent grid: as many clusters as fit on the device at once (or fewer, if there is less work)
   int ci = 0;
-  while (ci < 3 && kClusterSizes[ci] != plan.cluster) ++ci;
-  const long long slots = kClusterCapacity[ci] / plan.cluster;
+  while (ci < 3 && kClusterSizes[ci] != plan.split_k) ++ci;
+  const long long slots = kClusterCapacity[ci] / plan.split_k;
   const long long n_clusters = p.total_items < slots ? p.total_items : slots;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)n_clusters, plan.cluster, 1);
+  cfg.gridDim = dim3((unsigned)n_clusters, plan.split_k, 1);
   cfg.blockDim = dim3(kGemmThreads, 1, 1);
   cfg.dynamicSmemBytes = L::kDynBytes;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = plan.cluster; attr[0].val.clusterDim.z = 1;
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = plan.split_k; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   LaunchScope ls(p.mode == MODE_CONV ? "ocs_gemm_kernel(conv)" : "ocs_gemm_kernel(linear)", stream);
-  if (cudaLaunchKernelEx(&cfg, ocs_gemm_kernel<BN>, tmB, tmA, p) != cudaSuccess) return OCS_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, ocs_gemm_kernel<BN>, tmB, tmA, tmAT, p) != cudaSuccess) return OCS_ERR_CUDA;
   return launch_status();
 }
 
-struct GemmWs {
-  int32_t* acc_ws;
-  unsigned long long* flags;
-  size_t total;
-};
-
-GemmWs carve_gemm_ws(void* ws, long long rows, int N, int split_k, long long tiles) {
-  GemmWs w{};
-  size_t off = 0;
-  auto take = [&](size_t bytes) {
-    unsigned char* q = ws ? reinterpret_cast<unsigned char*>(ws) + off : nullptr;
-    off += align_up(bytes, 256);
-    return q;
-  };
-  w.acc_ws = reinterpret_cast<int32_t*>(take(4 * (size_t)split_k * (size_t)rows * (size_t)N));
-  w.flags = reinterpret_cast<unsigned long long*>(take(8 * (size_t)tiles * (size_t)split_k));
-  w.total = off;
-  return w;
-}
-
-// A tag no earlier call and (but for a 2^-64 accident) no stale workspace content carries.
-unsigned long long next_nonce() {
-  static std::atomic<unsigned long long> counter{0};
-  static const unsigned long long salt = [] {
-    std::random_device rd;
-    return ((unsigned long long)rd() << 32) ^ (unsigned long long)rd() ^ 0x9E3779B97F4A7C15ull;
-  }();
-  return salt + 0x2545F4914F6CDD1Dull * (counter.fetch_add(1) + 1);
-}
-
 ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long long out_rows, int m_tiles, bool tma_a_ok,
-                    const CUtensorMap* tmA_in, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                    const CUtensorMap* tmA_in, void* ws, size_t ws_bytes, cudaStream_t stream,
+                    const CUtensorMap* tmAT_in = nullptr) {
   p.num_kb = (p.Ktot + BK - 1) / BK;
   if (!tma_a_ok) p.kb_tma_a = 0;
-  const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb, p.num_kb - p.kb_tma_a, p.Ktot - p.kb_tma_a * BK, p.mode == MODE_CONV);
+  p.tail_T = tmAT_in != nullptr && p.num_kb > p.kb_tma_a;
+  const GemmPlan plan = choose_plan(m_tiles, p.N, p.num_kb, p.num_kb - p.kb_tma_a, p.Ktot - p.kb_tma_a * BK,
+                                    p.mode == MODE_CONV, p.tail_T != 0);
   p.split_k = plan.split_k;
   p.m_tiles = plan.m_tiles;
-  p.n_groups = plan.n_tiles / plan.cluster;
-  p.total_items = (int)((long long)plan.m_tiles * p.n_groups * plan.split_k);
+  p.n_tiles = plan.n_tiles;
+  p.total_items = (int)((long long)plan.m_tiles * plan.n_tiles);
 
   CUtensorMap tmB;
   {
@@ -1102,20 +1187,16 @@ ocs_status run_gemm(GemmParams& p, const int8_t* W_codes, long long ldw, long lo
   }
   CUtensorMap tmA = tmB;  // a valid map even when unused
   if (p.kb_tma_a > 0) tmA = *tmA_in;
+  CUtensorMap tmAT = tmB;
+  if (p.tail_T) tmAT = *tmAT_in;
 
   p.out_rows = out_rows;
-  p.n_tiles = plan.n_tiles;
-  if (plan.split_k > 1) {
-    const GemmWs w = carve_gemm_ws(ws, out_rows, p.N, plan.split_k, (long long)plan.m_tiles * plan.n_tiles);
-    if (!ws || !aligned(ws, 256) || ws_bytes < w.total) return OCS_ERR_WORKSPACE;
-    p.acc_ws = w.acc_ws;
-    p.slice_flags = w.flags;
-    p.nonce = next_nonce();
-  }
+  (void)ws; (void)ws_bytes;   // the K split exchanges its partial sums through shared memory: no global scratch
   switch (plan.BN) {
-    case 256: return launch_gemm<256>(tmB, tmA, p, plan, stream);
-    case 128: return launch_gemm<128>(tmB, tmA, p, plan, stream);
-    default: return launch_gemm<64>(tmB, tmA, p, plan, stream);
+    case 256: return launch_gemm<256>(tmB, tmA, tmAT, p, plan, stream);
+    case 192: return launch_gemm<192>(tmB, tmA, tmAT, p, plan, stream);
+    case 128: return launch_gemm<128>(tmB, tmA, tmAT, p, plan, stream);
+    default: return launch_gemm<64>(tmB, tmA, tmAT, p, plan, stream);
   }
 }
 
@@ -1255,8 +1336,9 @@ extern "C" size_t ocs_qlinear_workspace_bytes(int M, int N, int C, int S) {
   return 256 + align_up(splitk_ws_bound(M, N, m_tiles), 256);
 }
 
-extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float* a_scale, int M, int C, int64_t lda,
-                                  const int8_t* W_codes, const float* w_scale, int N, int S, int64_t ldw,
+extern "C" ocs_status ocs_qlinear(const void* A_codes, const void* A_codes_T, int64_t lda_T, int a_signed, const float* a_scale,
+                                  int M, int C, int64_t lda, const int8_t* W_codes, const float* w_scale, int N, int S,
+                                  int64_t ldw,
                                   const int32_t* idx_map, const float* bias, float* Y, int64_t ldy, int32_t* acc_out,
                                   const float* residual, int relu, float* max_abs_out, void* ws, size_t ws_bytes,
                                   int* dev_status, void* stream_) {
@@ -1267,6 +1349,7 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
   const long long Ktot = (long long)C + S;
   if (lda < C || ldw < Ktot || ldy < N) return OCS_ERR_SHAPE;
   if (ldw % 16 != 0 || !aligned(W_codes, 16) || !aligned(Y, 4)) return OCS_ERR_SHAPE;
+  if (A_codes_T && (lda_T < M || lda_T % 16 != 0 || !aligned(A_codes_T, 16))) return OCS_ERR_SHAPE;
   if ((residual && !aligned(residual, 4)) || (acc_out && !aligned(acc_out, 4)) || (bias && !aligned(bias, 4)))
     return OCS_ERR_SHAPE;
   if (Ktot * 255ll * 127ll > 2147483647ll) return OCS_ERR_UNSUPPORTED;
@@ -1298,7 +1381,15 @@ extern "C" ocs_status ocs_qlinear(const void* A_codes, int a_signed, const float
     const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
     if (!encode_u8(&tmA, A_codes, 2, dims, strides, box)) return OCS_ERR_CUDA;
   }
-  return run_gemm(p, W_codes, ldw, M, m_tiles, tma_ok, &tmA, ws, ws_bytes, stream);
+  // the channel-major copy, if the caller has one: [C][lda_T], one channel's values for all rows contiguous
+  CUtensorMap tmAT;
+  if (A_codes_T) {
+    const cuuint64_t dims[2] = {(cuuint64_t)M, (cuuint64_t)C};
+    const cuuint64_t strides[1] = {(cuuint64_t)lda_T};
+    const cuuint32_t box[2] = {(cuuint32_t)BM, 1u};
+    if (!encode_u8(&tmAT, A_codes_T, 2, dims, strides, box)) return OCS_ERR_CUDA;
+  }
+  return run_gemm(p, W_codes, ldw, M, m_tiles, tma_ok, &tmA, ws, ws_bytes, stream, A_codes_T ? &tmAT : nullptr);
 }
 
 extern "C" int64_t ocs_conv_packed_k(int C, int S, int kh, int kw) {
@@ -1462,13 +1553,12 @@ extern "C" ocs_status ocs_qconv(const void* X_codes, int a_signed, const float* 
   return run_gemm(p, W_packed, ldw, g.out_rows, (int)g.m_tiles, tma_ok, &tmA, ws, ws_bytes, stream);
 }
 
-// Self-test hook: the next ocs_qlinear / ocs_qconv calls of this process use the given tile width (64, 128, 256),
-// number of K slices and cluster size (1, 2, 4, 8) instead of the planner's choice, wherever the values are
-// valid for the problem; bn = 0 gives the choice back to the planner.
-extern "C" ocs_status ocs_selftest_force_gemm_plan(int bn, int split_k, int cluster) {
-  if (bn != 0 && bn != 64 && bn != 128 && bn != 256) return OCS_ERR_INVALID_ARG;
-  if (split_k < 0 || split_k > 32) return OCS_ERR_INVALID_ARG;
-  if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return OCS_ERR_INVALID_ARG;
-  g_force_bn = bn; g_force_sk = split_k; g_force_cl = cluster;
+// Self-test hook: the next ocs_qlinear / ocs_qconv calls of this process use the given tile width (64, 128, 256)
+// and K split (1, 2, 4, 8; the cluster size) instead of the planner's choice, wherever the values are valid for
+// the problem; bn = 0 gives the choice back to the planner.
+extern "C" ocs_status ocs_selftest_force_gemm_plan(int bn, int split_k) {
+  if (bn != 0 && bn != 64 && bn != 128 && bn != 192 && bn != 256) return OCS_ERR_INVALID_ARG;
+  if (split_k < 0 || split_k > 8) return OCS_ERR_INVALID_ARG;
+  g_force_bn = bn; g_force_sk = split_k;
   return OCS_OK;
 }

@@ -264,3 +264,46 @@ extern "C" ocs_status ocs_lstm_cell(const float* g_ih, const float* g_hh, int ba
   lstm_cell_kernel<<<ew_grid((long long)batch * hidden, 1), 256, 0, stream>>>(g_ih, g_hh, batch, hidden, c, h);
   return launch_status();
 }
+
+// ------------------------------------------------------------------------------------------------
+// ocs_transpose_codes: channel-major copy of a code matrix, T[c][r] = A[r][c].  A 64 x 64 byte tile goes
+// through shared memory so that both the reads (along c) and the writes (along r) are coalesced.
+namespace ocs {
+namespace {
+__global__ void __launch_bounds__(256)
+transpose_codes_kernel(const uint8_t* __restrict__ A, long long rows, long long cols, long long ld,
+                       uint8_t* __restrict__ T, long long ld_t) {
+  __shared__ uint8_t tile[64][65];
+  const long long tiles_c = (cols + 63) / 64, tiles_r = (rows + 63) / 64;
+  for (long long t = blockIdx.x; t < tiles_c * tiles_r; t += gridDim.x) {
+    const long long tr = t / tiles_c, tc = t - tr * tiles_c;
+    const long long r0 = tr * 64, c0 = tc * 64;
+    __syncthreads();
+    for (int i = threadIdx.x; i < 64 * 64; i += 256) {
+      const int r = i >> 6, c = i & 63;
+      tile[r][c] = (r0 + r < rows && c0 + c < cols) ? __ldg(A + (r0 + r) * ld + c0 + c) : (uint8_t)0;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 64 * 64; i += 256) {
+      const int c = i >> 6, r = i & 63;
+      if (c0 + c < cols && r0 + r < rows) T[(c0 + c) * ld_t + r0 + r] = tile[r][c];
+    }
+  }
+}
+}  // namespace
+}  // namespace ocs
+
+extern "C" ocs_status ocs_transpose_codes(const void* codes, int64_t rows, int64_t cols, int64_t ld, void* codes_T,
+                                          int64_t ld_T, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!codes || !codes_T) return OCS_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ld < cols || ld_T < rows) return OCS_ERR_SHAPE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  const long long tiles = ((rows + 63) / 64) * ((cols + 63) / 64);
+  const int grid = (int)(tiles < (long long)kNumSMs * 8 ? tiles : (long long)kNumSMs * 8);
+  LaunchScope ls("transpose_codes_kernel", stream);
+  transpose_codes_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint8_t*>(codes), rows, cols, ld,
+                                                   reinterpret_cast<uint8_t*>(codes_T), ld_T);
+  return launch_status();
+}

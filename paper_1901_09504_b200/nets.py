@@ -87,7 +87,11 @@ def linear_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=Non
     M, Cn = x.shape
     ld = B.round_up(Cn, 16)
     codes, scale, _ = B.ocs_quantize(x.contiguous(), a_bits, a_signed, B.CLIP_NONE, ld_codes=ld, dev_status=dev_status)
-    return B.ocs_qlinear(codes, scale, L.codes, L.w_scale, L.idx_map, Cn, L.S, bias=L.bias, dev_status=dev_status)
+    # with many rows and duplicated channels the layer gathers whole channels from a channel-major copy of the
+    # codes; a handful of rows (a recurrent net's time step) is not worth the extra launch
+    codes_T = B.ocs_transpose_codes(codes, cols=Cn) if (L.S > 0 and M >= 64) else None
+    return B.ocs_qlinear(codes, scale, L.codes, L.w_scale, L.idx_map, Cn, L.S, bias=L.bias, dev_status=dev_status,
+                         A_codes_T=codes_T)
 
 
 # ------------------------------------------------------------------------------------------ ResNet-50

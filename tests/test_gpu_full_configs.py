@@ -70,8 +70,13 @@ def test_config3_fc6_full_size_points(ratio, bits, qa_bits):
     del Wout
     a_codes, a_scale, _ = ocs.ocs_quantize(dev(A), 8, False, ocs.CLIP_NONE, dev_status=st)
     np.testing.assert_array_equal(host(a_codes)[:, :Cn], ac)
-    Y, acc = ocs.ocs_qlinear(a_codes, a_scale, codes, scale, idx_d, Cn, S, want_acc=True, dev_status=st)
+    # the launch configuration the bench times: with duplicated channels, gathered from the channel-major copy
+    a_T = ocs.ocs_transpose_codes(a_codes, cols=Cn) if S > 0 else None
+    Y, acc = ocs.ocs_qlinear(a_codes, a_scale, codes, scale, idx_d, Cn, S, want_acc=True, dev_status=st, A_codes_T=a_T)
     assert ocs.ocs_poll_status(st) == 0
+    if S > 0:        # and the byte gather from the row-major codes gives the same accumulators
+        acc_b = ocs.ocs_qlinear(a_codes, a_scale, codes, scale, idx_d, Cn, S, want_acc=True, dev_status=st)[1]
+        assert torch.equal(acc, acc_b)
     rng = np.random.default_rng(3)
     ms = np.concatenate([rng.integers(0, A.shape[0], 3996), [0, 0, 127, 127]]).astype(np.int32)
     ns = np.concatenate([rng.integers(0, W.shape[0], 3996), [0, 4095, 0, 4095]]).astype(np.int32)

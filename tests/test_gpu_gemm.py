@@ -39,6 +39,16 @@ def _check_linear(seed, M, Cn, N, S, a_signed=False, lda=None, bias=True, a_scal
     np.testing.assert_array_equal(host(acc), acco)
     np.testing.assert_allclose(host(Y), Yo, rtol=1e-5, atol=0)
     np.testing.assert_array_equal(host(Y), Yo)
+    # the same layer with the channel-major copy of the activations: the duplicated channels arrive as whole rows
+    # of that copy (no byte gather); identical accumulators
+    AT = ocs.ocs_transpose_codes(Ad, cols=Cn)
+    np.testing.assert_array_equal(host(AT)[:, :M], A.T)
+    Yt, acct = ocs.ocs_qlinear(Ad, dev(np.array([a_scale], np.float32)), Wd, dev(np.array([w_scale], np.float32)),
+                               dev(idx), Cn, S, bias=None if b is None else dev(b), want_acc=True, dev_status=st,
+                               A_codes_T=AT)
+    assert ocs.ocs_poll_status(st) == 0
+    np.testing.assert_array_equal(host(acct), acco)
+    np.testing.assert_array_equal(host(Yt), Yo)
     # ReLU and max |Y| taken in the layer's epilogue: the checker's relu and maxabs of its own output
     m = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
     Yr = ocs.ocs_qlinear(Ad, dev(np.array([a_scale], np.float32)), Wd, dev(np.array([w_scale], np.float32)),
@@ -206,7 +216,7 @@ def test_qconv_first_layer_with_and_without_room_for_the_patch_matrix():
 
 
 def test_accumulators_do_not_depend_on_the_tile_plan():
-    """One problem under several forced (tile width, K slices, cluster size) plans: the int32 accumulators and
+    """One problem under several forced (tile width, K split) plans: the int32 accumulators and
     the outputs are identical, and equal the checker's (integer sums do not depend on their order)."""
     M, Cn, N, S = 200, 2100, 384, 150
     A = configs.random_codes(31, 0, (M, Cn), 0, 255, np.uint8)
@@ -220,18 +230,21 @@ def test_accumulators_do_not_depend_on_the_tile_plan():
     Ad = torch.zeros((M, ocs.round_up(Cn, 16)), dtype=torch.uint8, device="cuda")
     Ad[:, :Cn] = dev(A)
     sa, sw = dev(np.array([0.013], np.float32)), dev(np.array([0.0007], np.float32))
+    AT = ocs.ocs_transpose_codes(Ad, cols=Cn)
     try:
-        for bn, sk, cl in ((0, 0, 0), (64, 1, 1), (128, 1, 1), (256, 1, 1), (128, 2, 1), (128, 4, 1), (64, 3, 2), (64, 6, 2),
-                           (128, 5, 1), (256, 9, 1), (64, 8, 1)):
-            ocs.ocs_selftest_force_gemm_plan(bn, sk, cl)
+        for bn, sk in ((0, 0), (64, 1), (128, 1), (256, 1), (128, 2), (128, 4), (64, 2), (64, 4), (64, 8), (256, 2),
+                       (256, 4), (256, 8), (128, 8), (192, 1), (192, 2), (192, 4)):
+            ocs.ocs_selftest_force_gemm_plan(bn, sk)
             st = ocs.new_status()
-            for _ in range(2):                                     # twice: the workspace's tags of the first run are stale
-                Y, acc = ocs.ocs_qlinear(Ad, sa, Wd, sw, dev(idx), Cn, S, bias=dev(bias), want_acc=True, dev_status=st)
-                assert ocs.ocs_poll_status(st) == 0
-                np.testing.assert_array_equal(host(acc), acco, err_msg=f"plan {(bn, sk, cl)}")
-                np.testing.assert_array_equal(host(Y), Yo, err_msg=f"plan {(bn, sk, cl)}")
+            for _ in range(2):
+                for at in (None, AT):
+                    Y, acc = ocs.ocs_qlinear(Ad, sa, Wd, sw, dev(idx), Cn, S, bias=dev(bias), want_acc=True, dev_status=st,
+                                             A_codes_T=at)
+                    assert ocs.ocs_poll_status(st) == 0
+                    np.testing.assert_array_equal(host(acc), acco, err_msg=f"plan {(bn, sk)}")
+                    np.testing.assert_array_equal(host(Y), Yo, err_msg=f"plan {(bn, sk)}")
     finally:
-        ocs.ocs_selftest_force_gemm_plan(0, 0, 0)
+        ocs.ocs_selftest_force_gemm_plan(0, 0)
 
 
 @pytest.mark.parametrize("split", [False, True])
