@@ -1,6 +1,6 @@
 """Benchmark of the OCS hot path on B200: split -> clip search -> quantize -> int8 GEMM/conv.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-fused|fc6-small|fc|conv|resnet50|lstm|act-ocs] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload fc6|fc6-fused|fc6-small|fc|conv|resnet50|lstm|act-ocs|exact-mse] [--impl reference]
 
 One step is one pass of the whole path over one batch of synthetic input:
   fc6   (default) the VGG-16-fc6-shaped sweep: W [4096, 25088], 5 expand ratios x 4 weight bit
@@ -546,6 +546,75 @@ class ActOcs(Fc6Sweep):
         return sec, led.total
 
 
+class ExactMse(Fc6Sweep):
+    l2_note = "input larger than L2 (103 MB, no flush)"
+    """The element-wise MSE scorer (no histogram): every candidate threshold scored on every element in double.
+    Bound by fp64 arithmetic, not by memory: reported against an fp64 instruction rate, not against HBM."""
+    name = "exact-mse"
+    graph = False
+    N_INSTR = 8          # fp64 instructions per element and candidate: div, rint, min, max, mul, sub, mul, add
+
+    def __init__(self):
+        self.O, self.C, self.M = 1024, 25088, 128
+        self.bits = 4
+        self.desc = (f"Section 4.1's MSE on the elements themselves (OCS_CLIP_MSE_EXACT): W [{self.O}, {self.C}] fp32 (a quarter "
+                     f"of the fc6-shaped tensor of configs[2]), {N_CAND} candidates, {self.bits}-bit codes; a step = max |W|, the "
+                     "scorer, the combine and the quantization; seed 2")
+        self.points = [(0.0, self.bits)]
+        self.oracle_sample_desc = "the same search on the first 64 rows (1.6 M elements)"
+
+    def setup(self, ocs, torch, dev, host):
+        self.ocs, self.torch = ocs, torch
+        self.W = host["W"].to(dev)
+        self.codes = torch.empty((self.O, ocs.round_up(self.C, 16)), dtype=torch.int8, device=dev)
+        self.scal = torch.zeros(2, dtype=torch.float32, device=dev)
+        self.ws = torch.empty(int(ocs.lib().ocs_quantize_workspace_bytes(0, N_CAND)) + 256, dtype=torch.uint8, device=dev)
+        self.status = ocs.new_status(dev)
+
+    def host_inputs(self):
+        c = configs.config3(O=self.O, C=self.C, M=self.M)
+        return dict(W=c["W"])
+
+    def ledger(self):
+        led = Ledger()
+        n = self.O * self.C
+        led.add("maxabs_kernel", n=n)
+        led.bytes["exact_score_kernel"] = 4 * n
+        led.add("quantize_kernel", n=n)
+        led.ops = n * N_CAND * self.N_INSTR
+        return led
+
+    def step(self):
+        ocs = self.ocs
+        ocs.ocs_quantize(self.W, self.bits, True, ocs.CLIP_MSE_EXACT, N_CAND, out=(self.codes, self.scal[0:1], self.scal[1:2]),
+                         ws=self.ws, dev_status=self.status)
+
+    def e2e_buffers(self, host):
+        torch = self.torch
+        self.hW = torch.from_numpy(host["W"]).pin_memory()
+        self.hC = torch.empty(self.codes.shape, dtype=torch.int8).pin_memory()
+        return self.hW.numel() * 4, self.hC.numel()
+
+    def step_e2e(self):
+        self.W.copy_(self.hW, non_blocking=True)
+        self.step()
+        self.hC.copy_(self.codes, non_blocking=True)
+
+    def oracle_sample(self, orc, host):
+        W = host["W"][:64]
+        t0 = time.perf_counter()
+        a = orc.clip_mse_exact(W, self.bits, True, N_CAND)["alpha"]
+        orc.quantize(W, self.bits, True, a)
+        return time.perf_counter() - t0, 13 * W.size
+
+    def fp64_peak(self, torch, dev):
+        """fp64 instruction rate of this GPU, measured: the library's double-precision matrix product (4096^3, best
+        of 5) issues one fused multiply-add per two counted operations, so instructions/s = flop/s / 2."""
+        a = torch.randn((4096, 4096), dtype=torch.float64, device=dev)
+        ms = _time_best(torch, lambda: torch.matmul(a, a), reps=5)
+        return 2.0 * 4096 ** 3 / (ms * 1e-3) / 2.0
+
+
 class SmallFc(Fc6Sweep):
     """configs[0]: one fully-connected layer, no clip search."""
     name = "fc"
@@ -686,11 +755,17 @@ class ResNet50(NetWorkload):
         self.ev_start = torch.cuda.Event()
         self.ev_done = [torch.cuda.Event() for _ in self.prep_streams]
 
+    batched = True
+
     def step(self):
-        """The 54 layers are prepared independently of one another: their small, latency-bound kernels (a single
-        CTA for the split plan) are spread over a few streams so that they run side by side; the forward pass
-        starts when all of them are done."""
+        """Preparation of the 54 layers, then the forward pass.  Batched (default): every layer but the first goes
+        through ocs_split_quantize_batch -- five launches for 53 layers -- and the weight reordering of the
+        convolutions follows layer by layer.  Otherwise the layers are prepared one by one, spread over a few
+        streams so that their small, latency-bound kernels run side by side."""
         nets, cfg, torch = self.nets, self.cfg, self.torch
+        if self.batched:
+            layers = nets.prepare_resnet50(cfg, self.dev, dev_status=self.status, batched=True, weights=self.Wd)
+            return nets.resnet50_forward(cfg, layers, self.dev_in["X"], dev_status=self.status)
         main = torch.cuda.current_stream()
         self.ev_start.record(main)
         layers = {}
@@ -781,6 +856,12 @@ class Lstm(NetWorkload):
         h = small["hidden"]
         S = configs_num_splits(h, 0.02)
         return sec, 2 * (h + S) * (6 * 4 * 4 * h * 4 + 6 * 4 * 3000)
+
+
+class ResNet50PerLayer(ResNet50):
+    """The same step with every layer prepared by its own calls (eight streams), for comparison."""
+    name = "resnet50-per-layer"
+    batched = False
 
 
 class LstmFolded(Lstm):
@@ -911,7 +992,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm", "lstm-folded", "act-ocs"])
+    ap.add_argument("--workload", default="fc6", choices=["fc6", "fc6-fused", "fc6-small", "fc", "conv", "resnet50", "lstm", "lstm-folded", "act-ocs", "exact-mse", "resnet50-per-layer"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-tensor-probe", action="store_true")
@@ -922,7 +1003,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     wl = {"fc6": Fc6Sweep, "fc6-fused": Fc6Fused, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc, "conv": Conv3x3,
-          "resnet50": ResNet50, "lstm": Lstm, "lstm-folded": LstmFolded, "act-ocs": ActOcs}[args.workload]()
+          "resnet50": ResNet50, "resnet50-per-layer": ResNet50PerLayer, "lstm": Lstm, "lstm-folded": LstmFolded, "act-ocs": ActOcs, "exact-mse": ExactMse}[args.workload]()
     net = getattr(wl, "kind", "") == "net"
 
     if args.impl == "reference":
@@ -1052,6 +1133,17 @@ def main():
                         avg_launch_ms=top_ms / top_cnt, note="ops of every quantized layer of the step (linear and conv "
                         "launches share one kernel); layers with few channels are bound by their output traffic, not by "
                         "the tensor pipe",
+                        timed="second pass over the same steps with CUDA events around every kernel launch")
+    elif top == "exact_score_kernel":
+        # bound by fp64 arithmetic: counted fp64 instructions of the scorer over its traced time, against the fp64
+        # instruction rate measured in this run
+        peak_i = wl.fp64_peak(torch, dev) / 1e12
+        ach = led.ops * args.steps / (top_ms * 1e-3) / 1e12
+        roofline = dict(kernel=top, bound="alu", achieved=ach, peak=peak_i, unit="T fp64 instr/s", frac=ach / peak_i,
+                        traffic=None, peak_source="measured in this run: fp64 matrix product 4096^3 (library), flop/s / 2",
+                        avg_launch_ms=top_ms / top_cnt,
+                        note=f"{wl.N_INSTR} counted instructions per element and candidate (the division alone expands to "
+                        "a dozen machine instructions, so the fraction understates the pipe's load)",
                         timed="second pass over the same steps with CUDA events around every kernel launch")
     elif top_bytes:
         roof_achieved = top_bytes * args.steps / (top_ms * 1e-3) / 1e9

@@ -219,6 +219,30 @@ ocs_status ocs_split_quantize(const float* W, int O, int C, int R, int64_t ld_in
                               float* max_abs_out, float* scale, float* alpha, void* ws, size_t ws_bytes,
                               int* dev_status, void* stream);
 
+/* ocs_split_quantize_batch -------------------------------------------------------------------
+ * ocs_split_quantize with plain halving and no clip search (Sections 3.2-3.4, Eq. 1) for all
+ * the layers of a network at once: five launches in total instead of five per layer (one
+ * extrema pass over all weights, the greedy plans side by side -- one CTA per layer --, one
+ * code pass for the short-row layers and one for the long-row layers).  The results of every
+ * layer are bit-identical to its own ocs_split_quantize call (qa_step = 0, qa_bits = 0, mode
+ * OCS_CLIP_NONE).  layers: HOST array of n_layers descriptors (read before the call returns);
+ * W dense [O][C][R]; codes [O][ld_codes]; idx_map [C+S]; scale [1]; max_abs3 [3] nullable.
+ * Limits: n_layers <= 64; every layer must satisfy ocs_split_quantize's staging limits (W 16-byte
+ * aligned, C*R a multiple of 4, two expanded rows in shared memory), otherwise
+ * OCS_ERR_UNSUPPORTED -- prepare that layer with its own call.  Device flags: NONFINITE, TIMEOUT. */
+typedef struct {
+  const float* W;
+  int O, C, R, S;
+  int8_t* codes;
+  int64_t ld_codes;
+  int32_t* idx_map;
+  float* scale;
+  float* max_abs3;
+} ocs_layer_desc;
+size_t ocs_split_quantize_batch_workspace_bytes(const ocs_layer_desc* layers, int n_layers);
+ocs_status ocs_split_quantize_batch(const ocs_layer_desc* layers, int n_layers, int bits, int is_signed,
+                                    void* ws, size_t ws_bytes, int* dev_status, void* stream);
+
 /* ocs_dup_weight_columns ------------------------------------------------------------------
  * Weight side of activation OCS (Eq. 4: the activation channel is halved in both copies, its
  * weights are duplicated unchanged).  W_codes (device) int8 [N][ldw >= (C+S)*R] holds the layer's
@@ -368,6 +392,18 @@ ocs_status ocs_selftest_force_gemm_plan(int bn, int split_k);
 int64_t ocs_conv_packed_k(int C, int S, int kh, int kw);
 ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, int S, int kh, int kw,
                                  int64_t ld_src, int8_t* packed, int64_t ld_dst, void* stream);
+
+/* ocs_pack_conv_weights_batch: ocs_pack_conv_weights for up to 64 layers in one launch (the
+ * reordering of a whole network's convolutions after ocs_split_quantize_batch).  jobs: HOST array,
+ * read before the call returns; fields as the arguments of ocs_pack_conv_weights. */
+typedef struct {
+  const int8_t* codes;
+  int O, C, S, kh, kw;
+  int64_t ld_src;
+  int8_t* packed;
+  int64_t ld_dst;
+} ocs_pack_desc;
+ocs_status ocs_pack_conv_weights_batch(const ocs_pack_desc* jobs, int n_jobs, void* stream);
 
 /* ocs_qconv -------------------------------------------------------------------------------
  * Convolution form of ocs_qlinear (Section 3.2: a split duplicates a whole 2-D activation

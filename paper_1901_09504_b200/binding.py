@@ -28,11 +28,12 @@ EXPORTS = [
     "ocs_split_workspace_bytes", "ocs_split", "ocs_selftest_wait_expiry",
     "ocs_range_curve_workspace_bytes", "ocs_range_curve", "ocs_knapsack_workspace_bytes", "ocs_knapsack_allocate",
     "ocs_split_quantize_workspace_bytes", "ocs_split_quantize", "ocs_dup_weight_columns",
+    "ocs_split_quantize_batch_workspace_bytes", "ocs_split_quantize_batch",
     "ocs_fold_workspace_bytes", "ocs_fold_duplicates",
     "ocs_act_select_workspace_bytes", "ocs_act_select_channels", "ocs_act_split_quantize_static",
     "ocs_quantize_workspace_bytes", "ocs_quantize", "ocs_quantize_workspace_views", "ocs_quantize_noalloc",
     "ocs_qlinear_workspace_bytes", "ocs_qlinear", "ocs_transpose_codes", "ocs_selftest_force_gemm_plan",
-    "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_qconv_workspace_bytes", "ocs_qconv",
+    "ocs_conv_packed_k", "ocs_pack_conv_weights", "ocs_pack_conv_weights_batch", "ocs_qconv_workspace_bytes", "ocs_qconv",
     "ocs_add_relu", "ocs_maxpool3x3s2", "ocs_global_avgpool", "ocs_nchw_to_nhwc", "ocs_embedding", "ocs_lstm_cell",
 ]
 
@@ -54,7 +55,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.ocs_num_splits.argtypes = [C.c_int, C.c_double]
         L.ocs_version.restype = C.c_char_p
-        for name in ("ocs_range_curve_workspace_bytes", "ocs_knapsack_workspace_bytes", "ocs_fold_workspace_bytes", "ocs_act_select_workspace_bytes", "ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
+        for name in ("ocs_split_quantize_batch_workspace_bytes", "ocs_range_curve_workspace_bytes", "ocs_knapsack_workspace_bytes", "ocs_fold_workspace_bytes", "ocs_act_select_workspace_bytes", "ocs_split_quantize_workspace_bytes", "ocs_split_workspace_bytes", "ocs_quantize_workspace_bytes", "ocs_qlinear_workspace_bytes",
                      "ocs_qconv_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.ocs_quantize_workspace_views.restype = None
@@ -515,3 +516,59 @@ def ocs_selftest_wait_expiry(W, dev_status):
 def ocs_selftest_force_gemm_plan(bn: int = 0, split_k: int = 0):
     """Fixes tile width / K split of the following ocs_qlinear / ocs_qconv calls (bn = 0: planner)."""
     _check(lib().ocs_selftest_force_gemm_plan(int(bn), int(split_k)), "ocs_selftest_force_gemm_plan")
+
+
+class _LayerDesc(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("O", C.c_int), ("C", C.c_int), ("R", C.c_int), ("S", C.c_int),
+                ("codes", C.c_void_p), ("ld_codes", C.c_int64), ("idx_map", C.c_void_p), ("scale", C.c_void_p),
+                ("max_abs3", C.c_void_p)]
+
+
+def ocs_split_quantize_batch(Ws, Ss, bits: int, is_signed: bool = True, dev_status=None, ws=None):
+    """ocs_split_quantize (plain halving, no clip search) for a list of weight tensors in five launches.
+    Ws: fp32 [O, C] or [O, C, kh, kw] device tensors; Ss: split counts.  Returns per layer (codes int8
+    [O, ld_codes], scale fp32 [1], idx_map int32 [C+S])."""
+    n = len(Ws)
+    descs = (_LayerDesc * n)()
+    outs = []
+    for i, (W, S) in enumerate(zip(Ws, Ss)):
+        assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+        O, Cn = W.shape[0], W.shape[1]
+        R = 1
+        for d in W.shape[2:]:
+            R *= d
+        ld = round_up((Cn + int(S)) * R, 16)
+        codes = torch.empty((O, ld), dtype=torch.int8 if is_signed else torch.uint8, device=W.device)
+        scale = torch.empty(1, dtype=torch.float32, device=W.device)
+        idx_map = torch.empty(Cn + int(S), dtype=torch.int32, device=W.device)
+        descs[i] = _LayerDesc(W.data_ptr(), O, Cn, R, int(S), codes.data_ptr(), ld, idx_map.data_ptr(), scale.data_ptr(), None)
+        outs.append((codes, scale, idx_map))
+    nws = lib().ocs_split_quantize_batch_workspace_bytes(descs, n)
+    if nws == 0:
+        raise OcsError("ocs_split_quantize_batch_workspace_bytes", 4)
+    if ws is None:
+        ws = _ws(nws, Ws[0].device)
+    st = lib().ocs_split_quantize_batch(descs, n, int(bits), int(bool(is_signed)), _ptr(ws), C.c_size_t(ws.numel()),
+                                        _ptr(dev_status), _stream())
+    _check(st, "ocs_split_quantize_batch")
+    return outs
+
+
+class _PackDesc(C.Structure):
+    _fields_ = [("codes", C.c_void_p), ("O", C.c_int), ("C", C.c_int), ("S", C.c_int), ("kh", C.c_int), ("kw", C.c_int),
+                ("ld_src", C.c_int64), ("packed", C.c_void_p), ("ld_dst", C.c_int64)]
+
+
+def ocs_pack_conv_weights_batch(jobs):
+    """jobs: list of (codes int8 [O, ld_src], O, C, S, kh, kw) -> list of packed int8 [O, ld_dst], one launch."""
+    n = len(jobs)
+    descs = (_PackDesc * n)()
+    outs = []
+    for i, (codes, O, Cn, S, kh, kw) in enumerate(jobs):
+        assert codes.is_cuda and codes.dtype == torch.int8 and codes.dim() == 2 and codes.stride(1) == 1
+        ld = round_up(ocs_conv_packed_k(Cn, S, kh, kw), 16)
+        packed = torch.empty((O, ld), dtype=torch.int8, device=codes.device)
+        descs[i] = _PackDesc(codes.data_ptr(), int(O), int(Cn), int(S), int(kh), int(kw), codes.stride(0), packed.data_ptr(), ld)
+        outs.append(packed)
+    _check(lib().ocs_pack_conv_weights_batch(descs, n, _stream()), "ocs_pack_conv_weights_batch")
+    return outs

@@ -32,6 +32,8 @@
 // outstanding copies land, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace ocs {
@@ -342,8 +344,8 @@ __device__ __forceinline__ KSrc k_source(const GemmParams& p, int k, bool* bad) 
 // that contributes zero).
 __device__ __forceinline__ uint32_t ldg_u8_if(const uint8_t* addr, bool ok) {
   uint32_t v;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+  // not volatile: a read-only load, free to be scheduled early and side by side with its fifteen siblings
+  asm("{\n\t.reg .pred p;\n\t"
       "setp.ne.u32 p, %2, 0;\n\t"
       "mov.u32 %0, 0;\n\t"
       "@p ld.global.nc.u8 %0, [%1];\n\t}"
@@ -489,9 +491,15 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   int prod_j = 0, prod_i = 0, prod_it = 0;   // producer position: work item, K-block inside it, ring slot counter
   bool prod_ok = true;
   // thread 0 only: issue K-blocks until `limit_it` have been issued (first_tile_only: and stay inside the first tile)
+  WorkItem prod_w;
+  int prod_w_j = -1;                         // the work item prod_w describes (-1: none yet)
   auto produce = [&](int limit_it, bool first_tile_only) {
-    WorkItem w;
-    while (prod_ok && prod_it < limit_it && work_item(p, prod_j, crank, CL, &w)) {
+    while (prod_ok && prod_it < limit_it) {
+      if (prod_w_j != prod_j) {              // look the tile up once, not once per K-block
+        if (!work_item(p, prod_j, crank, CL, &prod_w)) break;
+        prod_w_j = prod_j;
+      }
+      const WorkItem& w = prod_w;
       if (prod_i >= w.my_kb) {
         if (first_tile_only) break;
         ++prod_j; prod_i = 0;
@@ -1075,13 +1083,13 @@ constexpr int kClusterCapacity[4] = {148, 148, 132, 120};
 // valid for the problem.
 int g_force_bn = 0, g_force_sk = 0;
 
-// Tile width and K split by a small time model (microseconds).  Measured on this part: an SM takes in about
-// 105 GB/s of operand tiles, all SMs together about 9.5 TB/s from L2 (the activation tile of a K-block is re-read
-// from L2 by every N tile, so narrow tiles spend that budget on re-reads), DRAM delivers about 6.3 TB/s, and a
-// 128 x 256 x 128 block of int8 MMAs takes about 0.27 us.  A wave of tiles costs the largest of those terms for
-// the most loaded CTA, or the gather beside it; a K split adds the exchange of the partial tiles.  K is split
-// only so far that all clusters are resident at once.  n_tail = K-blocks whose A tile is assembled by threads
-// or fetched as channel rows, tail_k = contraction indices in them.
+// Tile width and K split by a small time model (microseconds), fitted to measurements on this part: an SM takes
+// in about 105 GB/s of operand tiles, all SMs together about 9.5 TB/s from L2 (the activation tile of a K-block is
+// re-read from L2 by every N tile), DRAM delivers about 6.3 TB/s, a 128 x 256 x 128 block of int8 MMAs takes about
+// 0.27 us, the epilogue writes a tile at about 22 GB/s per SM (it overlaps the next tile's main loop, so a tile
+// costs the longer of the two), and every tile costs about 1.5 us of hand-offs.  A K split adds the exchange of
+// the partial tiles; K is split only so far that all clusters are resident at once.  n_tail = K-blocks whose A
+// tile is assembled by threads or fetched as channel rows, tail_k = contraction indices in them.
 GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, bool conv, bool tail_by_tma) {
   if (g_force_bn) {
     const int BN = g_force_bn;
@@ -1094,7 +1102,7 @@ GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, boo
   GemmPlan best{64, 1, m_tiles, (N + 63) / 64};
   double best_cost = 1e300;
   const int bns[4] = {256, 192, 128, 64};
-  const double kSmIngest = 105e3, kL2Total = 9.5e6, kDram = 6.3e6;   // bytes per microsecond
+  const double kSmIngest = 105e3, kL2Total = 9.5e6, kDram = 6.3e6, kEpilogue = 22e3;   // bytes per microsecond
   const double gather_us = tail_by_tma ? 0.0 : (conv ? 4.0 : 16.0);  // per assembled K-block full of data
   const double K = (double)num_kb * BK, Mrows = (double)m_tiles * BM;
   const double dram_us = ((double)N * K + Mrows * K + 4.0 * Mrows * N) / kDram;
@@ -1104,25 +1112,26 @@ GemmPlan choose_plan(int m_tiles, int N, int num_kb, int n_tail, int tail_k, boo
     const int n_tiles = (N + BN - 1) / BN;
     const long long tiles = (long long)m_tiles * n_tiles;
     const double block_bytes = (double)(BM + BN) * BK;
-    const double mma_block_us = 0.27 * BN / 256.0;
+    double block_us = block_bytes / kSmIngest;                       // one K-block: operand intake or the MMAs
+    if (0.27 * BN / 256.0 > block_us) block_us = 0.27 * BN / 256.0;
+    const double epi_us = (double)BM * ((double)N / n_tiles) * 4.0 / kEpilogue;
     for (int ci = 0; ci < 4; ++ci) {
       const int sk = kClusterSizes[ci];
       if (sk > 1 && (tiles * sk > kClusterCapacity[ci] || num_kb < 4 * sk)) continue;   // one resident wave, >= 4 blocks each
       const long long waves = (tiles * sk + kClusterCapacity[ci] - 1) / kClusterCapacity[ci];
       const int cta_blocks = (num_kb + sk - 1) / sk;
       const int tail_blocks = (n_tail + sk - 1) / sk;
-      const double cta_bytes = (double)waves * cta_blocks * block_bytes;
-      const double total_bytes = (double)tiles * num_kb * block_bytes;
-      double stream = cta_bytes / kSmIngest;
-      if (total_bytes / kL2Total > stream) stream = total_bytes / kL2Total;
-      if (dram_us > stream) stream = dram_us;
-      if ((double)waves * cta_blocks * mma_block_us > stream) stream = (double)waves * cta_blocks * mma_block_us;
       // the most loaded CTA assembles tail_blocks K-blocks per tile, of which at most tail_k indices hold data
       const int cta_k = tail_k < tail_blocks * BK ? tail_k : tail_blocks * BK;
-      const double gather = (double)waves * (0.1 * tail_blocks + (cta_k / 128.0) * gather_us);
-      if (gather > stream) stream = gather;
-      double cost = 5.0 + stream + (double)waves * 1.0 * BN / 256.0;   // start-up, main loops, last epilogue
-      if (sk > 1) cost += 3.0 + 6.0 * BN / 256.0;                        // exchange and sum of the partial tiles
+      const double gather = tail_blocks > 0 ? 0.5 + (cta_k / 128.0) * gather_us : 0.0;
+      double tile_us = cta_blocks * block_us;
+      if (sk == 1 && epi_us > tile_us) tile_us = epi_us;
+      if (gather > tile_us) tile_us = gather;
+      double body = (double)waves * (tile_us + 1.5);
+      const double total_bytes = (double)tiles * num_kb * block_bytes;
+      if (total_bytes / kL2Total > body) body = total_bytes / kL2Total;
+      if (dram_us > body) body = dram_us;
+      double cost = 5.0 + body + (sk == 1 ? epi_us : 3.0 + 6.0 * BN / 256.0);   // start-up; last epilogue or exchange
       cost *= 1.0 + 0.002 * ci + 0.001 * bi;                             // ties: fewer slices, wider tile
       if (cost < best_cost) {
         best_cost = cost;
@@ -1224,11 +1233,12 @@ void choose_conv_box(int Wo, int Ho, int Nb, int* bw_o, int* bh_o, int* bn_o) {
 // with zero-filled out-of-range channels).
 int conv_tap_stride(int C) { return (C % 16 == 0 && C % BK != 0) ? (C + BK - 1) / BK * BK : C; }
 
-__global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, int Cp, int S, int R, long long ld_src,
-                                 int8_t* __restrict__ dst, long long ld_dst) {
+// (vb, vg): this CTA's index and the number of CTAs working on this layer (a whole launch, or a share of one)
+__device__ __forceinline__ void pack_conv_body(const int8_t* __restrict__ src, int O, int C, int Cp, int S, int R,
+                                               long long ld_src, int8_t* __restrict__ dst, long long ld_dst, int vb, int vg) {
   const long long total = (long long)O * ld_dst;
   const int KO = R * Cp, Kt = KO + R * S;
-  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+  for (long long i = vb * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)vg * blockDim.x) {
     const long long o = i / ld_dst;
     const int k = (int)(i - o * ld_dst);
     int8_t v = 0;
@@ -1240,6 +1250,29 @@ __global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, i
     }
     dst[i] = v;
   }
+}
+
+__global__ void pack_conv_kernel(const int8_t* __restrict__ src, int O, int C, int Cp, int S, int R, long long ld_src,
+                                 int8_t* __restrict__ dst, long long ld_dst) {
+  pack_conv_body(src, O, C, Cp, S, R, ld_src, dst, ld_dst, blockIdx.x, gridDim.x);
+}
+
+// The same reordering for many layers in one launch: a CTA looks up its layer and its place among that layer's CTAs.
+constexpr int kMaxPackBatch = 64;
+struct PackJob {
+  const int8_t* src; int8_t* dst;
+  long long ld_src, ld_dst;
+  int O, C, Cp, S, R, blk0, blks, pad;
+};
+struct PackTable {
+  int n, pad[3];
+  PackJob j[kMaxPackBatch];
+};
+__global__ void __launch_bounds__(256) batch_pack_kernel(const __grid_constant__ PackTable t) {
+  int li = 0;
+  while (li + 1 < t.n && (int)blockIdx.x >= t.j[li + 1].blk0) ++li;
+  const PackJob& y = t.j[li];
+  pack_conv_body(y.src, y.O, y.C, y.Cp, y.S, y.R, y.ld_src, y.dst, y.ld_dst, (int)blockIdx.x - y.blk0, y.blks);
 }
 
 
@@ -1411,6 +1444,38 @@ extern "C" ocs_status ocs_pack_conv_weights(const int8_t* codes, int O, int C, i
   const int grid = (int)((total + 255) / 256 < kNumSMs * 8 ? (total + 255) / 256 : kNumSMs * 8);
   LaunchScope ls("pack_conv_kernel", stream);
   pack_conv_kernel<<<grid, 256, 0, stream>>>(codes, O, C, conv_tap_stride(C), S, kh * kw, ld_src, packed, ld_dst);
+  return launch_status();
+}
+
+extern "C" ocs_status ocs_pack_conv_weights_batch(const ocs_pack_desc* jobs, int n_jobs, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!jobs || n_jobs < 1) return OCS_ERR_INVALID_ARG;
+  if (n_jobs > kMaxPackBatch) return OCS_ERR_UNSUPPORTED;
+  static PackTable t;                  // 5 KB, kept off the stack; calls are serialised
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  t.n = n_jobs;
+  int blk = 0;
+  for (int i = 0; i < n_jobs; ++i) {
+    const ocs_pack_desc& d = jobs[i];
+    if (!d.codes || !d.packed || d.S < 0) return OCS_ERR_INVALID_ARG;
+    if (d.O <= 0 || d.C <= 0 || d.kh <= 0 || d.kw <= 0) return OCS_ERR_SHAPE;
+    const long long Ksrc = (long long)d.kh * d.kw * ((long long)d.C + d.S);
+    const long long Kt = (long long)d.kh * d.kw * ((long long)conv_tap_stride(d.C) + d.S);
+    if (d.ld_src < Ksrc || d.ld_dst < Kt || d.ld_dst % 16 != 0 || Kt >= (1ll << 31)) return OCS_ERR_SHAPE;
+    PackJob& y = t.j[i];
+    y.src = d.codes; y.dst = d.packed; y.ld_src = d.ld_src; y.ld_dst = d.ld_dst;
+    y.O = d.O; y.C = d.C; y.Cp = conv_tap_stride(d.C); y.S = d.S; y.R = d.kh * d.kw;
+    const long long total = (long long)d.O * d.ld_dst;
+    long long want = (total + 256 * 16 - 1) / (256 * 16);     // sixteen bytes per thread
+    if (want < 1) want = 1;
+    if (want > kNumSMs) want = kNumSMs;
+    y.blk0 = blk; y.blks = (int)want; blk += (int)want;
+  }
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  LaunchScope ls("batch_pack_kernel", stream);
+  batch_pack_kernel<<<blk, 256, 0, stream>>>(t);
   return launch_status();
 }
 

@@ -12,6 +12,8 @@
 //                        in shared memory by bulk copies, duplicated channels gathered there
 //   split_scatter_kernel the same pass with plain loads and stores, for shapes the bulk copies
 //                        cannot serve (rows longer than the buffers, unaligned rows)
+#include <mutex>
+
 #include "common.cuh"
 
 namespace ocs {
@@ -31,19 +33,21 @@ __device__ __forceinline__ float split_new(float w, float d) { return __fmul_rn(
 // columns (a thread owns 4 consecutive columns); the (column block, row) pairs are numbered
 // column-block-major and every CTA of a grid sized to one resident wave takes one contiguous
 // range of them, so all CTAs stream the same number of rows (to within one).
-__device__ __forceinline__ void cta_range(long long total, long long* u0, long long* u1) {
-  *u0 = total * (long long)blockIdx.x / (long long)gridDim.x;
-  *u1 = total * ((long long)blockIdx.x + 1) / (long long)gridDim.x;
+__device__ __forceinline__ void cta_range(long long total, long long* u0, long long* u1, int vb, int vg) {
+  *u0 = total * (long long)vb / (long long)vg;
+  *u1 = total * ((long long)vb + 1) / (long long)vg;
 }
 
 // K1 for a narrow matrix (ncols <= 512): a row needs only ncols/4 threads, so the CTA walks 256 / (ncols/4)
 // rows side by side and combines them in shared memory before touching the global extrema.
+// (vb, vg): this CTA's index and the number of CTAs working on this matrix -- the block index and grid size of a
+// launch for one matrix, or a share of a launch that covers many matrices.
 template <bool VEC>
-__global__ void __launch_bounds__(256)
-col_minmax_narrow_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
-                         uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map,
-                         int32_t* __restrict__ depth, unsigned long long* __restrict__ bits, int* dev_status) {
-  for (int c = blockIdx.x * 256 + threadIdx.x; c < C; c += gridDim.x * 256) {
+__device__ __forceinline__ void
+col_minmax_narrow_body(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
+                       uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map,
+                       int32_t* __restrict__ depth, unsigned long long* __restrict__ bits, int* dev_status, int vb, int vg) {
+  for (int c = vb * 256 + threadIdx.x; c < C; c += vg * 256) {
     idx_map[c] = c; depth[c] = 0; bits[c] = 0ull;
   }
   bool bad = false;
@@ -57,7 +61,7 @@ col_minmax_narrow_kernel(const float* __restrict__ W, int O, int ncols, int64_t 
     const int side = 256 / tpr;
     const int lr = threadIdx.x / tpr, col0 = (threadIdx.x - lr * tpr) * 4;
     long long r0, r1;
-    cta_range((long long)O, &r0, &r1);
+    cta_range((long long)O, &r0, &r1, vb, vg);
     if (lr < side) {
       float mn[4], mx[4];
 #pragma unroll
@@ -109,20 +113,28 @@ col_minmax_narrow_kernel(const float* __restrict__ W, int O, int ncols, int64_t 
   }
 }
 
-// K1: per-column signed extrema of a row-major [O][ncols] fp32 matrix.
 template <bool VEC>
 __global__ void __launch_bounds__(256)
-col_minmax_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
-                  uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map, int32_t* __restrict__ depth,
-                  unsigned long long* __restrict__ bits, int* dev_status) {
+col_minmax_narrow_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
+                         uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map,
+                         int32_t* __restrict__ depth, unsigned long long* __restrict__ bits, int* dev_status) {
+  col_minmax_narrow_body<VEC>(W, O, ncols, ld, colmin, colmax, C, idx_map, depth, bits, dev_status, blockIdx.x, gridDim.x);
+}
+
+// K1: per-column signed extrema of a row-major [O][ncols] fp32 matrix.
+template <bool VEC>
+__device__ __forceinline__ void
+col_minmax_body(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
+                uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map, int32_t* __restrict__ depth,
+                unsigned long long* __restrict__ bits, int* dev_status, int vb, int vg) {
   // identity part of the plan's outputs: original channel c maps to itself and has no split yet
-  for (int c = blockIdx.x * 256 + threadIdx.x; c < C; c += gridDim.x * 256) {
+  for (int c = vb * 256 + threadIdx.x; c < C; c += vg * 256) {
     idx_map[c] = c; depth[c] = 0; bits[c] = 0ull;
   }
   bool bad = false;
   const int col_blocks = (ncols + 1023) / 1024;
   long long u, u1;
-  cta_range((long long)col_blocks * O, &u, &u1);
+  cta_range((long long)col_blocks * O, &u, &u1, vb, vg);
   while (u < u1) {
     const int cb = (int)(u / O);
     const int r0 = (int)(u - (long long)cb * O);
@@ -168,6 +180,14 @@ col_minmax_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uin
     }
   }
   if (bad) flag(dev_status, OCS_DEV_NONFINITE);
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(256)
+col_minmax_kernel(const float* __restrict__ W, int O, int ncols, int64_t ld, uint32_t* __restrict__ colmin,
+                  uint32_t* __restrict__ colmax, int C, int32_t* __restrict__ idx_map, int32_t* __restrict__ depth,
+                  unsigned long long* __restrict__ bits, int* dev_status) {
+  col_minmax_body<VEC>(W, O, ncols, ld, colmin, colmax, C, idx_map, depth, bits, dev_status, blockIdx.x, gridDim.x);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -417,8 +437,7 @@ __device__ float greedy_rounds(const PlanArgs& a, PlanShared& sh, unsigned long 
   return prio_key(block_max_u64(m, sh.red));
 }
 
-__global__ void __launch_bounds__(kPlanThreads, 1) split_plan_kernel(PlanArgs a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ void split_plan_body(const PlanArgs& a, unsigned char* smem_raw) {
   __shared__ PlanShared sh;
 
   const int tid = threadIdx.x;
@@ -606,6 +625,11 @@ __global__ void __launch_bounds__(kPlanThreads, 1) split_plan_kernel(PlanArgs a)
   }
 }
 
+__global__ void __launch_bounds__(kPlanThreads, 1) split_plan_kernel(PlanArgs a) {
+  extern __shared__ __align__(16) unsigned char plan_smem[];
+  split_plan_body(a, plan_smem);
+}
+
 // ------------------------------------------------------------------------------------------------
 // K3: W'[o][j][r] = path_j(W[o][idx_map[j]][r]).  Threads own 4 consecutive output columns.
 template <bool VEC>
@@ -617,7 +641,7 @@ split_scatter_kernel(const float* __restrict__ W, int O, int C, int R, int64_t l
   const int ncols_out = (C + S) * R;
   const int col_blocks = (ncols_out + 1023) / 1024;
   long long u, u1;
-  cta_range((long long)col_blocks * O, &u, &u1);
+  cta_range((long long)col_blocks * O, &u, &u1, blockIdx.x, gridDim.x);
   const float d = __fmul_rn(*qa_step_dev, 0.5f);
   while (u < u1) {
     const int cb = (int)(u / O);
@@ -761,13 +785,13 @@ struct RowsEpilogue {
 };
 
 template <int MODE>
-__global__ void __launch_bounds__(kRowThreads, 1)
-split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_in, int S, float* __restrict__ Wout,
-                  int64_t ld_out, const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
-                  const unsigned long long* __restrict__ bits, const float* __restrict__ qa_step_dev,
-                  const int32_t* __restrict__ touched, const int* __restrict__ n_touched, int rows_per_group,
-                  int srow /*floats between rows in shared memory*/, RowsEpilogue ep, int* dev_status) {
-  extern __shared__ __align__(128) unsigned char row_smem[];
+__device__ __forceinline__ void
+split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in, int S, float* __restrict__ Wout,
+                int64_t ld_out, const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
+                const unsigned long long* __restrict__ bits, const float* __restrict__ qa_step_dev,
+                const int32_t* __restrict__ touched, const int* __restrict__ n_touched, int rows_per_group,
+                int srow /*floats between rows in shared memory*/, RowsEpilogue ep, int* dev_status,
+                unsigned char* row_smem, int vb, int vg) {
   __shared__ __align__(8) unsigned long long bars[2];
   __shared__ int abort_flag;
   float* buf[2] = {reinterpret_cast<float*>(row_smem),
@@ -777,7 +801,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
   const int out_cols = (C + S) * R;
   const int out_bulk = out_cols & ~3;        // floats per row that leave by bulk store
   const int n_groups = (O + rows_per_group - 1) / rows_per_group;
-  const int my_groups = blockIdx.x < n_groups ? (n_groups - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+  const int my_groups = vb < n_groups ? (n_groups - 1 - vb) / vg + 1 : 0;
   const float d = __fmul_rn(*qa_step_dev, 0.5f);
   const int nt = *n_touched;
   const int dep_cap = d == 0.0f ? kMaxHalvings : 64;
@@ -798,7 +822,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
     const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)ep.L);
     q_inv = zero ? 0.0f : __fdiv_rn((float)ep.L, alpha);
     q_lo = ep.is_signed ? -(float)ep.L : 0.0f; q_hi = (float)ep.L;
-    if (blockIdx.x == 0 && tid == 0) {
+    if (vb == 0 && tid == 0) {
       *ep.scale_out = step;
       if (ep.alpha_out) *ep.alpha_out = zero ? 0.0f : alpha;
     }
@@ -813,7 +837,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
   __syncthreads();
 
   auto issue_load = [&](int i) {   // thread 0 only
-    const int g = blockIdx.x + i * gridDim.x;
+    const int g = vb + i * vg;
     const int r0 = g * rows_per_group;
     const int gn = min(rows_per_group, O - r0);
     const uint32_t bar = smem_addr(&bars[i & 1]);
@@ -881,7 +905,7 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
     }
     __syncthreads();
     if (abort_flag) break;
-    const int g = blockIdx.x + i * gridDim.x;
+    const int g = vb + i * vg;
     const int r0 = g * rows_per_group;
     const int gn = min(rows_per_group, O - r0);
     float* rows = buf[b];
@@ -992,6 +1016,18 @@ split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_i
     }
   }
   __syncthreads();
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kRowThreads, 1)
+split_rows_kernel(const float* __restrict__ W, int O, int C, int R, int64_t ld_in, int S, float* __restrict__ Wout,
+                  int64_t ld_out, const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
+                  const unsigned long long* __restrict__ bits, const float* __restrict__ qa_step_dev,
+                  const int32_t* __restrict__ touched, const int* __restrict__ n_touched, int rows_per_group,
+                  int srow /*floats between rows in shared memory*/, RowsEpilogue ep, int* dev_status) {
+  extern __shared__ __align__(128) unsigned char row_smem_dyn[];
+  split_rows_body<MODE>(W, O, C, R, ld_in, S, Wout, ld_out, idx_map, depth, bits, qa_step_dev, touched, n_touched,
+                        rows_per_group, srow, ep, dev_status, row_smem_dyn, blockIdx.x, gridDim.x);
 }
 
 struct SplitWs {
@@ -1288,19 +1324,19 @@ namespace {
 // channels (four loads of source columns whose lines the main group has just read).  Keeping the two kinds
 // of work in different warps keeps either from waiting on the other's divergent path.  Repeated halving
 // keeps the checker's rounding, subnormals included.
-__global__ void __launch_bounds__(256, 4)
-rows_quant_narrow_kernel(const float* __restrict__ W, int O, int C, int R, long long ld_in, int S,
-                         const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
-                         const float* __restrict__ maxp, const double* __restrict__ scores, int n_candidates, int L,
-                         int is_signed, int8_t* __restrict__ codes, long long ld_codes, int packed_ok, int vec_ok,
-                         int tail_warps, float* __restrict__ scale_out, float* __restrict__ alpha_out) {
+__device__ __forceinline__ void
+rows_quant_narrow_body(const float* __restrict__ W, int O, int C, int R, long long ld_in, int S,
+                       const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
+                       const float* __restrict__ maxp, const double* __restrict__ scores, int n_candidates, int L,
+                       int is_signed, int8_t* __restrict__ codes, long long ld_codes, int packed_ok, int vec_ok,
+                       int tail_warps, float* __restrict__ scale_out, float* __restrict__ alpha_out, int vb, int vg) {
   float alpha = *maxp;
   if (scores && alpha > 0.0f) alpha = pick_alpha(scores, alpha, n_candidates);
   const bool zero = !(alpha > 0.0f);
   const float step = zero ? 0.0f : __fdiv_rn(alpha, (float)L);
   const float inv = zero ? 0.0f : __fdiv_rn((float)L, alpha);
   const float lo = is_signed ? -(float)L : 0.0f, hi = (float)L;
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
+  if (vb == 0 && threadIdx.x == 0) {
     *scale_out = step;
     if (alpha_out) *alpha_out = zero ? 0.0f : alpha;
   }
@@ -1331,7 +1367,7 @@ rows_quant_narrow_kernel(const float* __restrict__ W, int O, int C, int R, long 
   const bool contiguous = !is_tail && vec_ok && valid[3];
   const bool any_dep = (dep[0] | dep[1] | dep[2] | dep[3]) != 0;
   long long r0, r1;
-  cta_range((long long)O, &r0, &r1);
+  cta_range((long long)O, &r0, &r1, vb, vg);
   auto emit = [&](long long r, float (&x)[4]) {
     if (any_dep) {
 #pragma unroll
@@ -1378,6 +1414,15 @@ rows_quant_narrow_kernel(const float* __restrict__ W, int O, int C, int R, long 
       emit(r, x);
     }
   }
+}
+__global__ void __launch_bounds__(256, 4)
+rows_quant_narrow_kernel(const float* __restrict__ W, int O, int C, int R, long long ld_in, int S,
+                         const int32_t* __restrict__ idx_map, const int32_t* __restrict__ depth,
+                         const float* __restrict__ maxp, const double* __restrict__ scores, int n_candidates, int L,
+                         int is_signed, int8_t* __restrict__ codes, long long ld_codes, int packed_ok, int vec_ok,
+                         int tail_warps, float* __restrict__ scale_out, float* __restrict__ alpha_out) {
+  rows_quant_narrow_body(W, O, C, R, ld_in, S, idx_map, depth, maxp, scores, n_candidates, L, is_signed, codes, ld_codes,
+                         packed_ok, vec_ok, tail_warps, scale_out, alpha_out, blockIdx.x, gridDim.x);
 }
 }  // namespace
 }  // namespace ocs
@@ -1524,6 +1569,263 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
   ep.n_candidates = n_candidates;
   return launch_rows_quant(W, O, C, R, ld_in, S, idx_map, w, ep, codes, ld_codes, scale, alpha, (int)g, srow, n_groups,
                            rows_smem, qa_step == 0.0f && qa_bits == 0, dev_status, stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// ocs_split_quantize_batch: ocs_split_quantize (plain halving, no clip search) for many layers in five launches
+// instead of five per layer: one extrema pass, one plan launch with a CTA per layer, one code pass each for
+// the short-row and the row-staged layers.  A network's layers are small next to the GPU (ResNet-50: 97 MiB of
+// weights in 54 layers); launched one by one their kernels are latency-bound, together they stream at memory rate.
+// The per-layer kernels' bodies are reused: a CTA of a batched launch looks up its layer and its position among
+// that layer's CTAs.
+namespace ocs {
+namespace {
+constexpr int kMaxBatch = 64;
+
+struct BatchLayer {
+  const float* W;
+  int O, C, R, S;
+  uint32_t* colmin; uint32_t* colmax;
+  float* chmin; float* chmax; float* chkey;
+  int32_t* depth; unsigned long long* bits;
+  float* qa_step_dev; int32_t* touched; int* n_touched; unsigned long long* g_buf;
+  int cap, npad, Sp, hist_off, keys_off;
+  int32_t* idx_map; float* mx3;
+  int8_t* codes; long long ld_codes; float* scale;
+  int mm_blk0, mm_blks, mm_narrow, vec;            // extrema pass: first CTA, CTAs, kernel form, 128-bit loads
+  int cp_kind, cp_blk0, cp_blks;                   // code pass: 0 = short rows, 1 = row-staged; first CTA, CTAs
+  int tail_warps, packed_ok, rows_per_group, srow; // code pass geometry
+};
+struct BatchTable {
+  int n, L, is_signed, pad;
+  BatchLayer l[kMaxBatch];
+};
+
+__global__ void __launch_bounds__(256)
+batch_minmax_kernel(const __grid_constant__ BatchTable t, int* dev_status) {
+  int li = 0;
+  while (li + 1 < t.n && (int)blockIdx.x >= t.l[li + 1].mm_blk0) ++li;
+  const BatchLayer& y = t.l[li];
+  const int vb = (int)blockIdx.x - y.mm_blk0, vg = y.mm_blks;
+  const int ncols = y.C * y.R;
+  if (y.mm_narrow) {
+    if (y.vec) col_minmax_narrow_body<true>(y.W, y.O, ncols, ncols, y.colmin, y.colmax, y.C, y.idx_map, y.depth, y.bits, dev_status, vb, vg);
+    else col_minmax_narrow_body<false>(y.W, y.O, ncols, ncols, y.colmin, y.colmax, y.C, y.idx_map, y.depth, y.bits, dev_status, vb, vg);
+  } else {
+    if (y.vec) col_minmax_body<true>(y.W, y.O, ncols, ncols, y.colmin, y.colmax, y.C, y.idx_map, y.depth, y.bits, dev_status, vb, vg);
+    else col_minmax_body<false>(y.W, y.O, ncols, ncols, y.colmin, y.colmax, y.C, y.idx_map, y.depth, y.bits, dev_status, vb, vg);
+  }
+}
+
+__global__ void __launch_bounds__(kPlanThreads, 1)
+batch_plan_kernel(const __grid_constant__ BatchTable t, int* dev_status) {
+  extern __shared__ __align__(16) unsigned char plan_smem_b[];
+  const BatchLayer& y = t.l[blockIdx.x];
+  PlanArgs a{};
+  a.colmin = y.colmin; a.colmax = y.colmax;
+  a.C = y.C; a.R = y.R; a.S = y.S; a.qa_step = 0.0f; a.qa_bits = 0;
+  a.chmin = y.chmin; a.chmax = y.chmax; a.chkey = y.chkey;
+  a.idx_map = y.idx_map; a.split_order = nullptr; a.depth = y.depth; a.bits = y.bits;
+  a.max_abs_out = y.mx3; a.qa_step_dev = y.qa_step_dev;
+  a.touched = y.touched; a.n_touched = y.n_touched;
+  a.g_buf = y.g_buf; a.cap = y.cap; a.npad = y.npad; a.Sp = y.Sp;
+  a.hist_off = y.hist_off; a.keys_off = y.keys_off;
+  a.curve = nullptr;
+  a.dev_status = dev_status;
+  split_plan_body(a, plan_smem_b);
+}
+
+// the layer of kind `kind` that CTA b of a code-pass launch belongs to (the launches of the two kinds number
+// their CTAs separately)
+__device__ __forceinline__ int code_layer(const BatchTable& t, int b, int kind) {
+  int li = -1;
+  for (int i = 0; i < t.n; ++i)
+    if (t.l[i].cp_kind == kind && b >= t.l[i].cp_blk0) li = i;
+  return li;
+}
+
+__global__ void __launch_bounds__(256, 4)
+batch_narrow_code_kernel(const __grid_constant__ BatchTable t) {
+  const BatchLayer& y = t.l[code_layer(t, (int)blockIdx.x, 0)];
+  rows_quant_narrow_body(y.W, y.O, y.C, y.R, (long long)y.C * y.R, y.S, y.idx_map, y.depth, y.mx3 + 1, nullptr, 1, t.L,
+                         t.is_signed, y.codes, y.ld_codes, y.packed_ok, y.vec, y.tail_warps, y.scale, nullptr,
+                         (int)blockIdx.x - y.cp_blk0, y.cp_blks);
+}
+
+__global__ void __launch_bounds__(kRowThreads, 1)
+batch_staged_code_kernel(const __grid_constant__ BatchTable t, int* dev_status) {
+  extern __shared__ __align__(128) unsigned char row_smem_b[];
+  const BatchLayer& y = t.l[code_layer(t, (int)blockIdx.x, 1)];
+  RowsEpilogue ep{};
+  ep.maxp = y.mx3 + 1;
+  ep.L = t.L;
+  ep.is_signed = t.is_signed;
+  ep.scores = nullptr;
+  ep.n_candidates = 1;
+  ep.codes = y.codes;
+  ep.ld_codes = y.ld_codes;
+  ep.packed_ok = y.packed_ok;
+  ep.scale_out = y.scale;
+  ep.alpha_out = nullptr;
+  split_rows_body<ROWS_QUANT>(y.W, y.O, y.C, y.R, (int64_t)y.C * y.R, y.S, nullptr, 0, y.idx_map, y.depth, y.bits,
+                              y.qa_step_dev, y.touched, y.n_touched, y.rows_per_group, y.srow, ep, dev_status, row_smem_b,
+                              (int)blockIdx.x - y.cp_blk0, y.cp_blks);
+}
+
+// Table and workspace layout of a batch; false if a layer cannot go through the fused path.
+struct BatchPlan {
+  BatchTable t;
+  int mm_grid, narrow_grid, staged_grid;
+  size_t plan_smem, staged_smem;
+  size_t colmin_bytes;   // all layers' column minima are one region (one memset), then all maxima
+  size_t total;
+};
+
+bool plan_batch(const ocs_layer_desc* layers, int n, int bits, int is_signed, void* ws, BatchPlan* bp, ocs_status* why) {
+  *why = OCS_OK;
+  if (n < 1 || n > kMaxBatch) { *why = OCS_ERR_UNSUPPORTED; return false; }
+  BatchTable& t = bp->t;
+  memset(&t, 0, sizeof(t));
+  t.n = n;
+  t.L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
+  t.is_signed = is_signed ? 1 : 0;
+  size_t cm = 0;
+  for (int i = 0; i < n; ++i) cm += align_up(4 * (size_t)layers[i].C * layers[i].R, 256);
+  bp->colmin_bytes = cm;
+  size_t off_min = 0, off = 2 * cm;
+  auto at = [&](size_t o) { return ws ? reinterpret_cast<unsigned char*>(ws) + o : nullptr; };
+  auto take = [&](size_t bytes) { unsigned char* q = at(off); off += align_up(bytes, 256); return q; };
+  int mm_blk = 0, nb = 0, sb = 0;
+  bp->plan_smem = 0; bp->staged_smem = 0;
+  for (int i = 0; i < n; ++i) {
+    const ocs_layer_desc& d = layers[i];
+    BatchLayer& y = t.l[i];
+    if (!d.W || !d.codes || !d.idx_map || !d.scale) { *why = OCS_ERR_INVALID_ARG; return false; }
+    if (d.O <= 0 || d.C <= 0 || d.R <= 0 || d.S < 0) { *why = OCS_ERR_SHAPE; return false; }
+    const long long ncols = (long long)d.C * d.R, ncols_out = ((long long)d.C + d.S) * d.R;
+    if (ncols_out >= (1ll << 31) || d.ld_codes < ncols_out) { *why = OCS_ERR_SHAPE; return false; }
+    const int srow = (int)((ncols_out + 3) & ~3ll);
+    const size_t row_bytes = 4 * (size_t)srow;
+    if (!(aligned(d.W, 16) && ncols % 4 == 0 && 2 * row_bytes <= kRowSmemBytes)) { *why = OCS_ERR_UNSUPPORTED; return false; }
+    y.W = d.W; y.O = d.O; y.C = d.C; y.R = d.R; y.S = d.S;
+    y.colmin = reinterpret_cast<uint32_t*>(at(off_min));
+    y.colmax = reinterpret_cast<uint32_t*>(at(cm + off_min));
+    off_min += align_up(4 * (size_t)ncols, 256);
+    const size_t CS = (size_t)d.C + d.S;
+    y.chmin = reinterpret_cast<float*>(take(4 * CS));
+    y.chmax = reinterpret_cast<float*>(take(4 * CS));
+    y.chkey = reinterpret_cast<float*>(take(4 * (size_t)d.C));
+    y.depth = reinterpret_cast<int32_t*>(take(4 * CS));
+    y.bits = reinterpret_cast<unsigned long long*>(take(8 * CS));
+    y.qa_step_dev = reinterpret_cast<float*>(take(256));
+    y.n_touched = reinterpret_cast<int*>(take(256));
+    y.Sp = d.S < d.C ? d.S : d.C;
+    y.touched = reinterpret_cast<int32_t*>(take(4 * (size_t)(y.Sp > 0 ? y.Sp : 1)));
+    y.cap = y.Sp + d.S;
+    y.npad = 1;
+    while (y.npad < y.cap) y.npad <<= 1;
+    const size_t plan_words = (size_t)y.Sp + 2 * (size_t)y.cap + (size_t)y.npad;
+    y.g_buf = d.S > kPlanSmemSplits ? reinterpret_cast<unsigned long long*>(take(8 * plan_words)) : nullptr;
+    y.mx3 = d.max_abs3 ? d.max_abs3 : reinterpret_cast<float*>(take(256));
+    y.idx_map = d.idx_map; y.codes = d.codes; y.ld_codes = d.ld_codes; y.scale = d.scale;
+    // plan kernel's shared memory, as in the single-layer call
+    const size_t plan_bytes = (d.S <= kPlanSmemSplits) ? 8 * plan_words : 0;
+    const size_t hist_off = (d.S <= kPlanSmemSplits) ? align_up(8 * (size_t)y.Sp, 16) : 0;
+    const size_t keys_off = hist_off + kSelHistBytes;
+    const bool keys_fit = keys_off + 4 * (size_t)d.C <= (size_t)kPlanSmemBytes;
+    y.hist_off = (int)hist_off;
+    y.keys_off = keys_fit ? (int)keys_off : -1;
+    size_t smem = keys_fit ? keys_off + 4 * (size_t)d.C : keys_off;
+    if (plan_bytes > smem) smem = plan_bytes;
+    if (smem > bp->plan_smem) bp->plan_smem = smem;
+    // extrema pass: CTAs in proportion to the (column block, row) units, eight rows per CTA at least
+    const long long units = ((ncols + 1023) / 1024) * d.O;
+    long long want = (units + 7) / 8;
+    if (want < 1) want = 1;
+    if (want > 4 * kNumSMs) want = 4 * kNumSMs;
+    y.mm_blk0 = mm_blk; y.mm_blks = (int)want; mm_blk += (int)want;
+    y.mm_narrow = ncols <= 512;
+    y.vec = 1;
+    // code pass: the same choice of form and geometry as the single-layer call
+    y.packed_ok = aligned(d.codes, 4) && (d.ld_codes % 4 == 0);
+    const int main_quads = (int)((ncols + 3) / 4), tail_quads = (d.S * d.R + 3) / 4;
+    const int tail_warps = d.S == 0 ? 0 : (12 * tail_quads >= main_quads ? 2 : 1);
+    y.tail_warps = tail_warps;
+    y.srow = srow;
+    if (main_quads <= 256 - 32 * tail_warps && tail_quads <= 32 * tail_warps) {
+      const int side = (256 - 32 * tail_warps) / main_quads;
+      long long g = (((long long)d.O + side - 1) / side + 7) / 8;
+      if (g < 1) g = 1;
+      if (g > 2 * kNumSMs) g = 2 * kNumSMs;
+      y.cp_kind = 0; y.cp_blk0 = nb; y.cp_blks = (int)g; nb += (int)g;
+    } else {
+      const RowsGeometry geo = rows_geometry(d.O, row_bytes, 0);
+      y.rows_per_group = (int)geo.g;
+      int g = geo.n_groups < kNumSMs / 4 ? geo.n_groups : kNumSMs / 4;   // a layer takes a quarter of the SMs at most
+      if (g < 1) g = 1;
+      y.cp_kind = 1; y.cp_blk0 = sb; y.cp_blks = g; sb += g;
+      if (geo.rows_smem > bp->staged_smem) bp->staged_smem = geo.rows_smem;
+    }
+  }
+  bp->mm_grid = mm_blk; bp->narrow_grid = nb; bp->staged_grid = sb;
+  bp->total = off;
+  return true;
+}
+}  // namespace
+}  // namespace ocs
+
+extern "C" size_t ocs_split_quantize_batch_workspace_bytes(const ocs_layer_desc* layers, int n_layers) {
+  BatchPlan bp;
+  ocs_status why;
+  if (!layers || !plan_batch(layers, n_layers, 8, 1, nullptr, &bp, &why)) return 0;
+  return bp.total;
+}
+
+extern "C" ocs_status ocs_split_quantize_batch(const ocs_layer_desc* layers, int n_layers, int bits, int is_signed,
+                                               void* ws, size_t ws_bytes, int* dev_status, void* stream_) {
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+  if (!layers) return OCS_ERR_INVALID_ARG;
+  if (bits < 2 || bits > 8) return OCS_ERR_INVALID_ARG;
+  if (!ws || !aligned(ws, 256)) return OCS_ERR_WORKSPACE;
+  static BatchPlan bp;                 // 14 KB: kept off the stack (calls are serialised by the mutex below)
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  ocs_status why;
+  if (!plan_batch(layers, n_layers, bits, is_signed, ws, &bp, &why)) return why;
+  if (ws_bytes < bp.total) return OCS_ERR_WORKSPACE;
+  ocs_status st = check_device();
+  if (st != OCS_OK) return st;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(batch_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPlanSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(batch_staged_code_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRowSmemBytes) != cudaSuccess)
+      return OCS_ERR_CUDA;
+    attr_set = true;
+  }
+  if (cudaMemsetAsync(ws, 0xFF, bp.colmin_bytes, stream) != cudaSuccess) return OCS_ERR_CUDA;
+  if (cudaMemsetAsync(reinterpret_cast<unsigned char*>(ws) + bp.colmin_bytes, 0x00, bp.colmin_bytes, stream) != cudaSuccess)
+    return OCS_ERR_CUDA;
+  {
+    LaunchScope ls("batch_minmax_kernel", stream);
+    batch_minmax_kernel<<<bp.mm_grid, 256, 0, stream>>>(bp.t, dev_status);
+    if ((st = launch_status()) != OCS_OK) return st;
+  }
+  {
+    LaunchScope ls("batch_plan_kernel", stream);
+    batch_plan_kernel<<<n_layers, kPlanThreads, bp.plan_smem, stream>>>(bp.t, dev_status);
+    if ((st = launch_status()) != OCS_OK) return st;
+  }
+  if (bp.narrow_grid > 0) {
+    LaunchScope ls("batch_narrow_code_kernel", stream);
+    batch_narrow_code_kernel<<<bp.narrow_grid, 256, 0, stream>>>(bp.t);
+    if ((st = launch_status()) != OCS_OK) return st;
+  }
+  if (bp.staged_grid > 0) {
+    LaunchScope ls("batch_staged_code_kernel", stream);
+    batch_staged_code_kernel<<<bp.staged_grid, kRowThreads, bp.staged_smem, stream>>>(bp.t, dev_status);
+    if ((st = launch_status()) != OCS_OK) return st;
+  }
+  return OCS_OK;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -95,20 +95,66 @@ def linear_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=Non
 
 
 # ------------------------------------------------------------------------------------------ ResNet-50
-def prepare_resnet50(cfg, device, dev_status=None):
-    """cfg from ocs_inputs.configs.config4 -> {layer name: QLayer}."""
+def batchable(W) -> bool:
+    """True when ocs_split_quantize_batch can take this layer (the fused path's staging limits)."""
+    R = 1
+    for d in W.shape[2:]:
+        R *= d
+    Cn = W.shape[1]
+    return (Cn * R) % 4 == 0 and 2 * 4 * (Cn + Cn // 8 + 8) * R <= 226 * 1024 and W.data_ptr() % 16 == 0
+
+
+def prepare_layers_batch(Ws, biases, ratio: float, bits: int, conv_flags, strides, pads, dev_status=None):
+    """All layers that fit the batched call are split and quantized together (ocs_split_quantize_batch: no clip
+    search, plain halving); the convolution weights are then reordered in one more launch.  -> list of QLayer."""
+    Ss = [B.ocs_num_splits(W.shape[1], ratio) for W in Ws]
+    outs = B.ocs_split_quantize_batch([W.contiguous() for W in Ws], Ss, bits, dev_status=dev_status)
+    jobs, where = [], []
+    for i, (W, S, (codes, _, _), conv) in enumerate(zip(Ws, Ss, outs, conv_flags)):
+        if conv:
+            jobs.append((codes, W.shape[0], W.shape[1], S, W.shape[2], W.shape[3]))
+            where.append(i)
+    packed = dict(zip(where, B.ocs_pack_conv_weights_batch(jobs))) if jobs else {}
+    layers = []
+    for i, (W, b, S, (codes, scale, idx_map), stride, pad) in enumerate(zip(Ws, biases, Ss, outs, strides, pads)):
+        O, Cn = W.shape[0], W.shape[1]
+        k = W.shape[2] if W.dim() == 4 else 1
+        layers.append(QLayer(packed.get(i, codes), scale, idx_map, b, Cn, O, S, k, stride, pad))
+    return layers
+
+
+def prepare_resnet50(cfg, device, dev_status=None, batched: bool = True, weights=None):
+    """cfg from ocs_inputs.configs.config4 -> {layer name: QLayer}.  weights: {name: (W, bias)} already on the device
+    (else they are uploaded from cfg).  With `batched` (and no clip search) every layer the batched call can take is
+    prepared by ocs_split_quantize_batch; the rest (the first layer: 3 x 49 weights per filter) go one by one."""
     mode = B.CLIP_MSE if cfg["clip"] == "mse" else B.CLIP_NONE
     out = {}
-    for spec in cfg["layers"] + [cfg["fc"]]:
-        W, bias = cfg["params"][spec.name]
-        Wd = torch.from_numpy(W).to(device)
-        bd = torch.from_numpy(bias).to(device)
+    specs = cfg["layers"] + [cfg["fc"]]
+    dev_w = {}
+    for spec in specs:
+        if weights is not None:
+            dev_w[spec.name] = weights[spec.name]
+        else:
+            W, bias = cfg["params"][spec.name]
+            dev_w[spec.name] = (torch.from_numpy(W).to(device), torch.from_numpy(bias).to(device))
+    group = []
+    for spec in specs:
+        Wd, bd = dev_w[spec.name]
         if spec.name == "fc":
-            out["fc"] = prepare_layer(Wd.reshape(spec.O, spec.C), bd, cfg["ratio"], cfg["w_bits"], mode,
-                                      dev_status=dev_status)
+            Wd = Wd.reshape(spec.O, spec.C)
+        if batched and mode == B.CLIP_NONE and batchable(Wd):
+            group.append((spec, Wd, bd))
+        elif spec.name == "fc":
+            out["fc"] = prepare_layer(Wd, bd, cfg["ratio"], cfg["w_bits"], mode, dev_status=dev_status)
         else:
             out[spec.name] = prepare_layer(Wd, bd, cfg["ratio"], cfg["w_bits"], mode, conv=True, stride=spec.stride,
                                            pad=spec.pad, dev_status=dev_status)
+    if group:
+        ql = prepare_layers_batch([g[1] for g in group], [g[2] for g in group], cfg["ratio"], cfg["w_bits"],
+                                  [g[0].name != "fc" for g in group], [g[0].stride for g in group],
+                                  [g[0].pad for g in group], dev_status=dev_status)
+        for (spec, _, _), L in zip(group, ql):
+            out[spec.name] = L
     return out
 
 

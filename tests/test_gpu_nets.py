@@ -99,3 +99,35 @@ def test_lstm_with_folded_duplicates_gives_the_same_logits():
     assert ocs.ocs_poll_status(st) == 0
     np.testing.assert_array_equal(host(t["tops"]), ref["tops"])
     np.testing.assert_array_equal(host(logits), ref_logits)
+
+
+def test_batched_preparation_equals_per_layer_calls():
+    """ocs_split_quantize_batch on a mix of layer shapes (short rows, long rows, 1x1 and 3x3, fully connected, S = 0)
+    gives every layer the bytes of its own ocs_split_quantize call, which in turn equal the checker's."""
+    shapes = [(64, 64, 1, 1), (64, 64, 3, 3), (256, 64, 1, 1), (128, 128, 3, 3), (512, 256, 1, 1), (128, 1024, 1, 1),
+              (96, 512, 3, 3), (1000, 2048), (33, 20), (16, 8)]
+    Ws = []
+    for i, sh in enumerate(shapes):
+        W = prng.laplace(61, i, sh, 0.02)
+        W.reshape(-1)[prng.distinct_positions(61, 100 + i, W.size, 4)] *= 20
+        Ws.append(W)
+    Ss = [ocs.ocs_num_splits(W.shape[1], 0.02) for W in Ws]
+    Ss[-1] = 0
+    st = ocs.new_status()
+    outs = ocs.ocs_split_quantize_batch([dev(W) for W in Ws], Ss, 8, dev_status=st)
+    assert ocs.ocs_poll_status(st) == 0
+    for W, S, (codes, scale, idx_map) in zip(Ws, Ss, outs):
+        c1, s1, _, i1, _, _ = ocs.ocs_split_quantize(dev(W), S, 8, ocs.CLIP_NONE, dev_status=st)
+        cols = (W.shape[1] + S) * int(np.prod(W.shape[2:]))
+        np.testing.assert_array_equal(host(idx_map), host(i1))
+        assert host(scale)[0] == host(s1)[0]
+        np.testing.assert_array_equal(host(codes)[:, :cols], host(c1)[:, :cols])
+        Wp, idx_o, _, _ = orc.split(W, S, 0.0)
+        wc, wscale = orc.quantize(Wp, 8, True, orc.maxabs(Wp))
+        np.testing.assert_array_equal(host(idx_map), idx_o)
+        assert host(scale)[0] == np.float32(wscale)
+        np.testing.assert_array_equal(host(codes)[:, :cols], wc.reshape(W.shape[0], -1))
+    assert ocs.ocs_poll_status(st) == 0
+    with pytest.raises(ocs.OcsError) as e:                       # 3 x 49 weights per filter: not a multiple of 4
+        ocs.ocs_split_quantize_batch([dev(prng.laplace(61, 50, (8, 3, 7, 7), 0.1))], [1], 8)
+    assert e.value.status == 4
