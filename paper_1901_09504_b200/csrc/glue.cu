@@ -266,13 +266,65 @@ extern "C" ocs_status ocs_lstm_cell(const float* g_ih, const float* g_hh, int ba
 }
 
 // ------------------------------------------------------------------------------------------------
-// ocs_transpose_codes: channel-major copy of a code matrix, T[c][r] = A[r][c].  A 64 x 64 byte tile goes
-// through shared memory so that both the reads (along c) and the writes (along r) are coalesced.
+// ocs_transpose_codes: channel-major copy of a code matrix, T[c][r] = A[r][c].  A CTA moves a 128 x 128 byte tile:
+// a thread loads four 32-bit words -- the same four columns of four consecutive rows --, transposes the 4 x 4 bytes
+// in registers (byte permutes) and writes four words into a shared-memory tile laid out like T; the tile's rows
+// then leave as whole 128-byte lines.  Reads and writes are both coalesced 32-bit accesses.  A plain byte-by-byte
+// form covers matrices whose rows are not 4-byte addressable.
 namespace ocs {
 namespace {
 __global__ void __launch_bounds__(256)
 transpose_codes_kernel(const uint8_t* __restrict__ A, long long rows, long long cols, long long ld,
                        uint8_t* __restrict__ T, long long ld_t) {
+  __shared__ uint32_t tile[128][33];    // [column of A][four rows of A per word], one word of padding
+  const long long tiles_c = (cols + 127) / 128, tiles_r = (rows + 127) / 128;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (long long t = blockIdx.x; t < tiles_c * tiles_r; t += gridDim.x) {
+    const long long tr = t / tiles_c, tc = t - tr * tiles_c;
+    const long long r0 = tr * 128, c0 = tc * 128;
+    __syncthreads();
+    // warp w takes row groups w, w + 8, ... (four rows each); lane l takes columns 4l .. 4l + 3
+#pragma unroll
+    for (int gi = 0; gi < 4; ++gi) {
+      const int rg = warp + gi * 8;                         // row group 0..31
+      uint32_t w[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const long long r = r0 + rg * 4 + k, c = c0 + lane * 4;
+        w[k] = 0u;
+        if (r < rows) {
+          if (c + 3 < cols) w[k] = __ldg(reinterpret_cast<const uint32_t*>(A + r * ld + c));
+          else
+            for (int e = 0; e < 4; ++e)
+              if (c + e < cols) w[k] |= (uint32_t)__ldg(A + r * ld + c + e) << (8 * e);
+        }
+      }
+      // 4 x 4 byte transpose: out[j] = bytes j of w[0..3]
+      const uint32_t a01 = __byte_perm(w[0], w[1], 0x5140), b01 = __byte_perm(w[0], w[1], 0x7362);
+      const uint32_t a23 = __byte_perm(w[2], w[3], 0x5140), b23 = __byte_perm(w[2], w[3], 0x7362);
+      tile[lane * 4 + 0][rg] = __byte_perm(a01, a23, 0x5410);
+      tile[lane * 4 + 1][rg] = __byte_perm(a01, a23, 0x7632);
+      tile[lane * 4 + 2][rg] = __byte_perm(b01, b23, 0x5410);
+      tile[lane * 4 + 3][rg] = __byte_perm(b01, b23, 0x7632);
+    }
+    __syncthreads();
+    // row c of the tile = 128 consecutive rows of A for one column: one 128-byte line of T per warp instruction
+    for (int c = warp; c < 128; c += 8) {
+      if (c0 + c >= cols) break;
+      const long long r = r0 + lane * 4;
+      uint8_t* dst = T + (c0 + c) * ld_t + r;
+      const uint32_t v = tile[c][lane];
+      if (r + 3 < rows) *reinterpret_cast<uint32_t*>(dst) = v;
+      else
+        for (int e = 0; e < 4; ++e)
+          if (r + e < rows) dst[e] = (uint8_t)(v >> (8 * e));
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+transpose_codes_bytes_kernel(const uint8_t* __restrict__ A, long long rows, long long cols, long long ld,
+                             uint8_t* __restrict__ T, long long ld_t) {
   __shared__ uint8_t tile[64][65];
   const long long tiles_c = (cols + 63) / 64, tiles_r = (rows + 63) / 64;
   for (long long t = blockIdx.x; t < tiles_c * tiles_r; t += gridDim.x) {
@@ -300,10 +352,16 @@ extern "C" ocs_status ocs_transpose_codes(const void* codes, int64_t rows, int64
   if (rows <= 0 || cols <= 0 || ld < cols || ld_T < rows) return OCS_ERR_SHAPE;
   ocs_status st = check_device();
   if (st != OCS_OK) return st;
-  const long long tiles = ((rows + 63) / 64) * ((cols + 63) / 64);
+  const bool words = aligned(codes, 4) && aligned(codes_T, 4) && ld % 4 == 0 && ld_T % 4 == 0;
+  const long long edge = words ? 128 : 64;
+  const long long tiles = ((rows + edge - 1) / edge) * ((cols + edge - 1) / edge);
   const int grid = (int)(tiles < (long long)kNumSMs * 8 ? tiles : (long long)kNumSMs * 8);
   LaunchScope ls("transpose_codes_kernel", stream);
-  transpose_codes_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint8_t*>(codes), rows, cols, ld,
-                                                   reinterpret_cast<uint8_t*>(codes_T), ld_T);
+  if (words)
+    transpose_codes_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint8_t*>(codes), rows, cols, ld,
+                                                     reinterpret_cast<uint8_t*>(codes_T), ld_T);
+  else
+    transpose_codes_bytes_kernel<<<grid, 256, 0, stream>>>(reinterpret_cast<const uint8_t*>(codes), rows, cols, ld,
+                                                           reinterpret_cast<uint8_t*>(codes_T), ld_T);
   return launch_status();
 }

@@ -270,3 +270,16 @@ def test_shortcut_tensor_that_is_not_16_byte_aligned(split):
                         residual=view, relu=True, dev_status=st)
     assert ocs.ocs_poll_status(st) == 0
     np.testing.assert_array_equal(host(Y), orc.add_relu(Yo, res, True))
+
+
+@pytest.mark.parametrize("rows,cols,ld,ld_t", [(128, 25088, 25088, 128), (20, 650, 656, 32), (7, 5, 5, 7), (300, 1031, 1040, 304),
+                                                (129, 130, 131, 133), (4, 4, 4, 4)])
+def test_transpose_codes(rows, cols, ld, ld_t):
+    A = configs.random_codes(51, 0, (rows, cols), 0, 255, np.uint8)
+    Ad = torch.zeros((rows, ld), dtype=torch.uint8, device="cuda")
+    Ad[:, :cols] = dev(A)
+    T = torch.full((cols, ld_t), 7, dtype=torch.uint8, device="cuda")
+    ocs.ocs_transpose_codes(Ad, cols=cols, out=T)
+    got = host(T)
+    np.testing.assert_array_equal(got[:, :rows], A.T)
+    assert (got[:, rows:] == 7).all()                      # padding beyond the rows is left alone
