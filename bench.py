@@ -1115,8 +1115,7 @@ def main():
         int8_peak = pk["bf16_burst"] * INT8_OVER_BF16
         int8_note = f"{pk['source']} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16 ratio; no int8 measurement in this run)"
     gemm_name = "ocs_gemm_kernel(linear)"
-    gemm_ms = sum(trace.get(k, (0, 0.0))[1] for k in ("ocs_gemm_kernel(linear)", "ocs_gemm_kernel(conv)",
-                                                     "splitk_reduce_kernel"))
+    gemm_ms = sum(trace.get(k, (0, 0.0))[1] for k in ("ocs_gemm_kernel(linear)", "ocs_gemm_kernel(conv)"))
     gemm_tops = (led.ops * args.steps / (gemm_ms * 1e-3) / 1e12) if gemm_ms > 0 else None
     sq_names = ("col_minmax_kernel", "split_rows_kernel", "split_scatter_kernel", "hist_kernel", "quantize_kernel", "maxabs_kernel",
                 "split_hist_kernel", "split_quantize_kernel", "transpose_codes_kernel")

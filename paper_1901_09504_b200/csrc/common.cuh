@@ -111,6 +111,14 @@ __device__ inline float pick_alpha(const double* __restrict__ scores, float m, i
 __device__ __forceinline__ int quant_code(float x, float inv, float lo, float hi) {
   return __float_as_int(__fadd_rn(fminf(fmaxf(__fmul_rn(x, inv), lo), hi), 12582912.0f));
 }
+// Histogram bin of the clip search: min(last, trunc(|x| * invw)).  last is an integer, so clamping the product
+// first gives the same bin (and sends NaN and infinity to the last bin instead of out of range).  The truncation
+// is one addition rounded toward zero: for 0 <= t < 2^23, fl_rz(t + 2^23) has unit spacing and its bit pattern is
+// that of 2^23 plus floor(t) -- no conversion instruction, which runs at a quarter of the addition's rate.
+__device__ __forceinline__ int hist_bin(float x, float invw, int last) {
+  const float t = fminf(__fmul_rn(fabsf(x), invw), (float)last);
+  return __float_as_int(__fadd_rz(t, 8388608.0f)) - 0x4B000000;
+}
 __device__ __forceinline__ unsigned int pack4(int c0, int c1, int c2, int c3) {
   return __byte_perm(__byte_perm((unsigned)c0, (unsigned)c1, 0x0040), __byte_perm((unsigned)c2, (unsigned)c3, 0x0040),
                      0x5410);

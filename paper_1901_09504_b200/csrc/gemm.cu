@@ -15,13 +15,16 @@
 // clusters of CL = 1, 2, 4 or 8 CTAs; a cluster walks its share of the tiles and its CTAs split the tile's
 // K-blocks among themselves (CTA r takes blocks r, r + CL, ...), so that short-and-wide problems still fill the
 // GPU.  The CL partial accumulators of a tile are summed through distributed shared memory: every CTA sends
-// the rows another CTA owns straight into that CTA's shared memory (st.shared::cluster), barriers in shared
-// memory pace the exchange, and each CTA finishes 128 / CL rows of the tile (integer sums: exact in any order).
+// the rows another CTA owns straight into that CTA's shared memory (st.async, counted as transaction bytes on
+// the owner's barrier), barriers in shared memory pace the exchange, and each CTA finishes 128 / CL rows of the
+// tile (integer sums: exact in any order).
 // No second launch, no global scratch, and the only waits are on CTAs the hardware co-schedules.  Warp roles:
 //   warp 0      TMA producer (weights always, activations when the block is TMA-able); its ring of
 //               stages runs on across tiles
 //   warp 1      allocates tensor memory (two accumulators), issues tcgen05.mma, commits to barriers
-//   warps 2..5  gather producers: assemble the A tiles of the K-blocks that hold duplicated channels
+//   warps 2..5  gather producers: assemble the A tiles of the K-blocks that hold duplicated channels -- or, when
+//               the caller supplies a channel-major copy of the activations, warp 2 alone requests each
+//               duplicated channel as one row of that copy by TMA (an MN-major operand tile)
 //   warps 6..13 epilogue of tile i while the main loop of tile i+1 runs: tcgen05.ld, transposition through
 //               shared memory for full-sector stores, int32 -> fp32, fmaf (optionally ReLU and max |Y|);
 //               the two warps of a tensor-memory lane quadrant take alternate 16-column pieces
@@ -161,9 +164,6 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void st_peer_v4(uint32_t addr, uint4 v) {
-  asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
 __device__ __forceinline__ void st_local_v4(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -245,6 +245,38 @@ __device__ __forceinline__ float int_to_float_rn(int acc) {
   return fmaf(fh, 65536.0f, fl);
 }
 
+// Two fp32 values in one 64-bit register, and the packed arithmetic on them (each half rounds on its own,
+// exactly as the scalar instruction would).
+__device__ __forceinline__ unsigned long long pack_f32x2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long sub_f32x2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+// int_to_float_rn for two accumulators at once (the same five steps, the floating-point ones packed).
+__device__ __forceinline__ unsigned long long int2_to_float2_rn(int acc0, int acc1) {
+  const uint32_t u0 = (uint32_t)acc0 ^ 0x80000000u, u1 = (uint32_t)acc1 ^ 0x80000000u;
+  const unsigned long long hi = pack_f32x2(__uint_as_float(__byte_perm(u0, 0x4B400000u, 0x7632)),
+                                           __uint_as_float(__byte_perm(u1, 0x4B400000u, 0x7632)));
+  const unsigned long long lo = pack_f32x2(__uint_as_float(__byte_perm(u0, 0x4B400000u, 0x7610)),
+                                           __uint_as_float(__byte_perm(u1, 0x4B400000u, 0x7610)));
+  const unsigned long long fh = sub_f32x2(hi, pack_f32x2(12615680.0f, 12615680.0f));   // 1.5*2^23 + 2^15
+  const unsigned long long fl = sub_f32x2(lo, pack_f32x2(12582912.0f, 12582912.0f));
+  return fma_f32x2(fh, pack_f32x2(65536.0f, 65536.0f), fl);
+}
+
 // 32 lanes x 16 consecutive 32-bit columns
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t v[16]) {
   asm volatile(
@@ -283,25 +315,43 @@ struct RowInfo {
   int n, ih0, iw0;     // conv: image and top-left input coordinate of the receptive field
 };
 
-__device__ __forceinline__ RowInfo row_info(const GemmParams& p, int mt, int r) {
+// Where row r of an M tile sits inside the tile's box of output pixels: the same for every tile, so a thread that
+// keeps its row works it out once.
+struct RowPos {
+  int wl, hl, nl;
+};
+__device__ __forceinline__ RowPos row_pos(const GemmParams& p, int r) {
+  RowPos rp;
+  rp.wl = r; rp.hl = 0; rp.nl = 0;
+  if (p.mode == MODE_LINEAR) return rp;
+  const int t = r / p.bw;
+  rp.wl = r - t * p.bw;
+  rp.nl = t / p.bh;
+  rp.hl = t - rp.nl * p.bh;
+  return rp;
+}
+
+__device__ __forceinline__ RowInfo row_info_at(const GemmParams& p, int mt, const RowPos& rp) {
   RowInfo ri;
   ri.n = 0; ri.ih0 = 0; ri.iw0 = 0;
   if (p.mode == MODE_LINEAR) {
-    const long long m = (long long)mt * BM + r;
+    const long long m = (long long)mt * BM + rp.wl;
     ri.out_row = m < p.M ? m : -1;
     return ri;
   }
-  const int tw = mt % p.tiles_w;
-  const int th = (mt / p.tiles_w) % p.tiles_h;
-  const int tn = mt / (p.tiles_w * p.tiles_h);
-  const int wl = r % p.bw;
-  const int hl = (r / p.bw) % p.bh;
-  const int nl = r / (p.bw * p.bh);
+  const int t = mt / p.tiles_w;
+  const int tw = mt - t * p.tiles_w;
+  const int tn = t / p.tiles_h;
+  const int th = t - tn * p.tiles_h;
+  const int wl = rp.wl, hl = rp.hl, nl = rp.nl;
   const int ow = tw * p.bw + wl, oh = th * p.bh + hl, n = tn * p.bn + nl;
   if (nl >= p.bn || ow >= p.Wo || oh >= p.Ho || n >= p.Nb) { ri.out_row = -1; return ri; }
   ri.out_row = ((long long)n * p.Ho + oh) * p.Wo + ow;
   ri.n = n; ri.ih0 = oh * p.stride - p.pad; ri.iw0 = ow * p.stride - p.pad;
   return ri;
+}
+__device__ __forceinline__ RowInfo row_info(const GemmParams& p, int mt, int r) {
+  return row_info_at(p, mt, row_pos(p, r));
 }
 
 // Where contraction index k of a K-block reads from, relative to the row's base address (linear:
@@ -426,10 +476,11 @@ struct WorkItem {
 // Item j of this CTA's cluster (tiles are dealt round-robin to the clusters of the grid; CTA `crank` of the
 // cluster takes K-blocks crank, crank + CL, ... of every tile).
 __device__ __forceinline__ bool work_item(const GemmParams& p, int j, uint32_t crank, uint32_t CL, WorkItem* w) {
-  const long long idx = (long long)blockIdx.x + (long long)j * gridDim.x;
-  if (idx >= p.total_items) return false;
-  w->nt = (int)(idx % p.n_tiles);
-  w->mt = (int)(idx / p.n_tiles);
+  // total_items fits an int, and so does every index a CTA looks at before it finds the end (32-bit divisions)
+  const unsigned idx = blockIdx.x + (unsigned)j * gridDim.x;
+  if (idx >= (unsigned)p.total_items) return false;
+  w->mt = (int)(idx / (unsigned)p.n_tiles);
+  w->nt = (int)(idx - (unsigned)w->mt * (unsigned)p.n_tiles);
   const int kz = (int)crank, sk = (int)CL;
   w->my_kb = p.num_kb > kz ? (p.num_kb - kz + sk - 1) / sk : 0;
   w->n_tma = p.kb_tma_a > kz ? min(w->my_kb, (p.kb_tma_a - kz + sk - 1) / sk) : 0;
@@ -754,11 +805,12 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     const int q = warp & 3;
     const float sc = __fmul_rn(__ldg(p.a_scale), __ldg(p.w_scale));
     const bool direct = CL == 1;
+    const RowPos my_pos = row_pos(p, q * 32 + lane);
     WorkItem w;
     bool ok = true;
     for (int j = 0; ok && work_item(p, j, crank, CL, &w); ++j) {
       const int acc = j & 1;
-      const RowInfo ri = row_info(p, w.mt, q * 32 + lane);
+      const RowInfo ri = row_info_at(p, w.mt, my_pos);
       const int nt = w.nt;
       const int ew = warp - 6, half = ew >> 2;
       if (p.residual && direct && ri.out_row >= 0) {
@@ -905,11 +957,11 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       // with qd = lane/4, words (lane%4)*4 .. +3; the row order keeps the shared-memory reads conflict-free).
       // The two epilogue warps that share a tensor-memory lane quadrant take alternate pieces.
       uint32_t* st_words = reinterpret_cast<uint32_t*>(epi_stage + (size_t)ew * L::kEpiWarpBytes);
-      long long* st_rows = reinterpret_cast<long long*>(st_words + 32 * L::kEpiRowWords);
-      __syncwarp();
-      st_rows[lane] = ri.out_row;
-      __syncwarp();
       const int qd = lane >> 2, sub = (qd & 1) * 4 + (qd >> 1), cq = (lane & 3) * 4;
+      // the four rows this lane writes, the same for every piece of the tile
+      long long orow[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) orow[i] = __shfl_sync(0xffffffffu, ri.out_row, i * 8 + sub);
       uint32_t* dst0 = reinterpret_cast<uint32_t*>(p.Y);
       const long long ldd = p.ldy;
       const bool base_vec = ((reinterpret_cast<uintptr_t>(dst0) & 15) == 0) && (ldd % 4 == 0);
@@ -917,6 +969,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       // the shortcut tensor is read with 128-bit loads only when it is itself 16-byte aligned (a view that
       // starts a few floats into a buffer takes the scalar loads)
       const bool res_vec = p.residual && ((reinterpret_cast<uintptr_t>(p.residual) & 15) == 0) && (p.ldy % 4 == 0);
+      const bool bias_vec = p.bias && ((reinterpret_cast<uintptr_t>(p.bias) & 15) == 0);
       float tile_max = 0.0f;
       const bool want_max = p.max_bits != nullptr;
       // a warp whose 32 rows are all padding (a short M tile) has nothing to write
@@ -924,31 +977,54 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       for (int c0 = half * kEpiCols; warp_has_rows && c0 < BN; c0 += 2 * kEpiCols) {
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
+        const bool full = n0 + kEpiCols <= p.N;   // warp-uniform
+        // this lane's four columns of every row it writes: their bias once per piece, asked for before the
+        // accumulator so that the two latencies overlap
+        float b4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (p.bias) {
+          if (full && bias_vec) {
+            const float4 t = __ldg(reinterpret_cast<const float4*>(p.bias + n0 + cq));
+            b4[0] = t.x; b4[1] = t.y; b4[2] = t.z; b4[3] = t.w;
+          } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              if (n0 + cq + e < p.N) b4[e] = __ldg(p.bias + n0 + cq + e);
+          }
+        }
         uint32_t v[kEpiCols];
         __syncwarp();
         tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
-        const bool full = n0 + kEpiCols <= p.N;   // warp-uniform
         // raw accumulators -> shared memory, one row per lane
         uint32_t* mine = st_words + lane * L::kEpiRowWords;
 #pragma unroll
         for (int jj = 0; jj < kEpiCols; jj += 4)
           *reinterpret_cast<uint4*>(mine + jj) = make_uint4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
         __syncwarp();
-        // this lane's four columns of every row it writes: their bias once per piece
-        float b4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (p.bias) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            if (n0 + cq + e < p.N) b4[e] = __ldg(p.bias + n0 + cq + e);
-        }
         const bool vec0 = full && base_vec, vec1 = full && acc_vec;
-        long long orow[4];
         uint4 a[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int r = i * 8 + sub;
-          orow[i] = st_rows[r];
-          a[i] = *reinterpret_cast<const uint4*>(st_words + r * L::kEpiRowWords + cq);
+        for (int i = 0; i < 4; ++i)
+          a[i] = *reinterpret_cast<const uint4*>(st_words + (i * 8 + sub) * L::kEpiRowWords + cq);
+        if (vec0 && !p.residual && !p.acc_out) {
+          // the common case, without per-element tests: whole piece inside N, 16-byte aligned output, nothing
+          // but scale, bias, ReLU and the maximum; the floating-point steps work on pairs
+          const unsigned long long sc2 = pack_f32x2(sc, sc);
+          const unsigned long long b01 = pack_f32x2(b4[0], b4[1]), b23 = pack_f32x2(b4[2], b4[3]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float f0, f1, f2, f3;
+            unpack_f32x2(fma_f32x2(int2_to_float2_rn((int)a[i].x, (int)a[i].y), sc2, b01), f0, f1);
+            unpack_f32x2(fma_f32x2(int2_to_float2_rn((int)a[i].z, (int)a[i].w), sc2, b23), f2, f3);
+            if (p.relu) {
+              f0 = f0 > 0.0f ? f0 : 0.0f; f1 = f1 > 0.0f ? f1 : 0.0f;
+              f2 = f2 > 0.0f ? f2 : 0.0f; f3 = f3 > 0.0f ? f3 : 0.0f;
+            }
+            if (orow[i] >= 0) {
+              if (want_max) tile_max = fmaxf(tile_max, fmaxf(fmaxf(fabsf(f0), fabsf(f1)), fmaxf(fabsf(f2), fabsf(f3))));
+              *reinterpret_cast<float4*>(p.Y + orow[i] * ldd + n0 + cq) = make_float4(f0, f1, f2, f3);
+            }
+          }
+          continue;
         }
         uint4 o[4];
 #pragma unroll

@@ -135,8 +135,7 @@ hist_kernel(View v, const float* __restrict__ maxp, int n_bins, unsigned long lo
     unsigned int* mine = sh + ((threadIdx.x >> 5) % kHistCopies) * n_bins;
     const int last = n_bins - 1;
     auto count = [&](float xv) {
-      const int b = min(last, (int)__fmul_rn(fabsf(xv), invw));  // truncation
-      atomicAdd(&mine[b], 1u);
+      atomicAdd(&mine[hist_bin(xv, invw, last)], 1u);
     };
     for (TileWalk w(v); w.left > 0; w.next(v)) {
       float4 x[kTileQuads];

@@ -740,6 +740,7 @@ split_scatter_kernel(const float* __restrict__ W, int O, int C, int R, int64_t l
 // Two row-group buffers alternate: the load of group i+1 and the store of group i-1 overlap the
 // (small) compute of group i.  One CTA per SM; row groups are dealt round-robin.
 constexpr int kRowThreads = 512;
+constexpr int kRowRing = 4;                         // row-group buffers a CTA may cycle through
 constexpr long long kRowWaitCycles = 2000000000ll;  // about one second
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -770,7 +771,7 @@ struct RowsEpilogue {
   const float* maxp;            // max|W'| (device scalar from the plan)
   int n_bins;                   // HIST
   unsigned long long* hist;     // HIST: global histogram [n_bins]
-  int hist_copies;              // HIST: private copies in shared memory behind the row buffers
+  int hist_copies;              // HIST: private copies of the counters (one per group of warps) behind the row buffers
   const double* scores;         // QUANT: candidate scores (null: no clipping)
   int n_candidates;
   int L;                        // QUANT: code range [-L, L], or [0, L] for unsigned codes
@@ -782,6 +783,7 @@ struct RowsEpilogue {
   float* alpha_out;
   long long wait_cycles;        // limit of the wait for a row group's copies; 0 = the default (about a second)
   int drop_last_load;           // self-test only: the CTA's last row group is never requested, so its wait runs out
+  int n_buf;                    // row-group buffers in the ring (2..kRowRing; 0 means 2)
 };
 
 template <int MODE>
@@ -792,10 +794,17 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
                 const int32_t* __restrict__ touched, const int* __restrict__ n_touched, int rows_per_group,
                 int srow /*floats between rows in shared memory*/, RowsEpilogue ep, int* dev_status,
                 unsigned char* row_smem, int vb, int vg) {
-  __shared__ __align__(8) unsigned long long bars[2];
+  __shared__ __align__(8) unsigned long long bars[kRowRing];
   __shared__ int abort_flag;
-  float* buf[2] = {reinterpret_cast<float*>(row_smem),
-                   reinterpret_cast<float*>(row_smem) + (size_t)rows_per_group * srow};
+  const int n_buf = ep.n_buf >= 2 ? min(ep.n_buf, kRowRing) : 2;
+  const size_t buf_floats = (size_t)rows_per_group * srow;
+  auto buf_at = [&](int b) { return reinterpret_cast<float*>(row_smem) + (size_t)b * buf_floats; };
+  // Row groups requested ahead of the one in work.  A buffer is refilled once its last user is done
+  // with it: the threads, as soon as the CTA barrier that ends their group is passed; a bulk store,
+  // once it has read the buffer -- so with stores the ring keeps one buffer more out of the loads'
+  // way (the newest store may still be reading) whenever it has three or more.
+  const int store_lag = (MODE == ROWS_STORE && n_buf >= 3) ? 1 : 0;
+  const int ahead = n_buf - 1 - store_lag;
   const int tid = threadIdx.x;
   const int in_cols = C * R;                 // a multiple of 4 (checked by the host)
   const int out_cols = (C + S) * R;
@@ -808,7 +817,7 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
   const long long wait_limit = ep.wait_cycles > 0 ? ep.wait_cycles : kRowWaitCycles;
 
   // epilogue state
-  unsigned int* hist_sh = reinterpret_cast<unsigned int*>(row_smem + 2 * (size_t)rows_per_group * srow * sizeof(float));
+  unsigned int* hist_sh = reinterpret_cast<unsigned int*>(row_smem + (size_t)n_buf * buf_floats * sizeof(float));
   float invw = 0.0f, q_inv = 0.0f, q_lo = 0.0f, q_hi = 0.0f;
   if (MODE == ROWS_HIST) {
     for (int i = tid; i < ep.hist_copies * ep.n_bins; i += kRowThreads) hist_sh[i] = 0u;
@@ -829,25 +838,26 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
   }
 
   if (tid == 0) {
-    for (int b = 0; b < 2; ++b)
+    for (int b = 0; b < kRowRing; ++b)
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[b])) : "memory");
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
 
-  auto issue_load = [&](int i) {   // thread 0 only
+  auto issue_load = [&](int i, int slot) {   // thread 0 only; slot = i mod n_buf
     const int g = vb + i * vg;
     const int r0 = g * rows_per_group;
     const int gn = min(rows_per_group, O - r0);
-    const uint32_t bar = smem_addr(&bars[i & 1]);
+    const uint32_t bar = smem_addr(&bars[slot]);
+    float* dst = buf_at(slot);
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)gn * in_cols * 4u)
                  : "memory");
     for (int rl = 0; rl < gn; ++rl) {
       const float* src = W + (int64_t)(r0 + rl) * ld_in;
       asm volatile(
           "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-          ::"r"(smem_addr(buf[i & 1] + (size_t)rl * srow)), "l"(src), "r"((uint32_t)in_cols * 4u), "r"(bar)
+          ::"r"(smem_addr(dst + (size_t)rl * srow)), "l"(src), "r"((uint32_t)in_cols * 4u), "r"(bar)
           : "memory");
     }
   };
@@ -883,18 +893,32 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
 
   // self-test: the last group's copies are never requested (nothing is in flight when its wait gives up)
   const int load_groups = ep.drop_last_load ? my_groups - 1 : my_groups;
-  if (tid == 0 && load_groups > 0) issue_load(0);
-  int issued = load_groups > 0 ? 1 : 0;
+  int issued = 0;
+  int load_slot = 0;                       // buffer of the next group to request (thread 0)
+  if (tid == 0) {
+    for (int k = 0; k < ahead && k < load_groups; ++k) {
+      issue_load(k, load_slot);
+      ++issued;
+      load_slot = load_slot + 1 == n_buf ? 0 : load_slot + 1;
+    }
+  }
+  int b = 0;                               // buffer of the group in work, and how often the ring has wrapped
+  uint32_t parity = 0;
   for (int i = 0; i < my_groups; ++i) {
-    const int b = i & 1;
     if (tid == 0) {
-      // the stores issued from the other buffer have finished reading it
-      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-      if (i + 1 < load_groups) { issue_load(i + 1); ++issued; }
+      // the bulk stores that read the buffer about to be refilled have finished reading it
+      if (MODE == ROWS_STORE) {
+        if (store_lag) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      }
+      if (i + ahead < load_groups) {
+        issue_load(i + ahead, load_slot);
+        ++issued;
+        load_slot = load_slot + 1 == n_buf ? 0 : load_slot + 1;
+      }
     }
     {  // bounded wait for this group's rows
       const uint32_t bar = smem_addr(&bars[b]);
-      const uint32_t parity = (uint32_t)(i >> 1) & 1u;
       if (!row_bar_try(bar, parity)) {
         const long long t0 = clock64();
         for (uint32_t it = 1;; ++it) {
@@ -908,7 +932,7 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
     const int g = vb + i * vg;
     const int r0 = g * rows_per_group;
     const int gn = min(rows_per_group, O - r0);
-    float* rows = buf[b];
+    float* rows = buf_at(b);
     if (cached) {
       // appended copies: channel C + s reads its source channel's original values
 #pragma unroll
@@ -947,8 +971,8 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
     }
     // The threads' (generic-proxy) writes into the row buffer are ordered before what the copy engine (async
     // proxy) does with the same bytes next: the bulk store that reads them (ROWS_STORE), and in every mode the
-    // bulk load that refills this buffer two groups later.  Each writing thread fences, then the CTA barrier
-    // orders the fences before thread 0's next copy.
+    // bulk load that refills this buffer later.  Each writing thread fences, then the CTA barrier orders the
+    // fences before thread 0's next copy.
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
     if (MODE == ROWS_STORE) {
@@ -970,13 +994,26 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
           if (invw > 0.0f) {
             unsigned int* mine = hist_sh + ((tid >> 5) % ep.hist_copies) * ep.n_bins;
             const int last = ep.n_bins - 1;
-            auto count = [&](float xv) {
-              const int bin = min(last, (int)__fmul_rn(fabsf(xv), invw));  // truncation
-              atomicAdd(&mine[bin], 1u);
-            };
-            for (int q = tid; q < quads; q += kRowThreads) {
-              const float4 v = reinterpret_cast<const float4*>(row)[q];
-              count(v.x); count(v.y); count(v.z); count(v.w);
+            auto count = [&](float xv) { atomicAdd(&mine[hist_bin(xv, invw, last)], 1u); };
+            // A thread's share of the row is loaded first and counted afterwards: the loads are in flight together
+            // and the counter updates (which return nothing) follow one another without a dependent load between.
+            constexpr int kQ = 6;
+            if (quads <= kQ * kRowThreads) {
+              float4 v[kQ];
+#pragma unroll
+              for (int k = 0; k < kQ; ++k) {
+                const int q = tid + k * kRowThreads;
+                if (q < quads) v[k] = reinterpret_cast<const float4*>(row)[q];
+              }
+#pragma unroll
+              for (int k = 0; k < kQ; ++k) {
+                if (tid + k * kRowThreads < quads) { count(v[k].x); count(v[k].y); count(v[k].z); count(v[k].w); }
+              }
+            } else {
+              for (int q = tid; q < quads; q += kRowThreads) {
+                const float4 v = reinterpret_cast<const float4*>(row)[q];
+                count(v.x); count(v.y); count(v.z); count(v.w);
+              }
             }
             if (tid < (out_cols & 3)) count(row[(quads << 2) + tid]);
           }
@@ -998,6 +1035,8 @@ split_rows_body(const float* __restrict__ W, int O, int C, int R, int64_t ld_in,
       }
       __syncthreads();   // the buffer may be refilled now
     }
+    b = b + 1 == n_buf ? 0 : b + 1;
+    if (b == 0) parity ^= 1u;
   }
   if (MODE == ROWS_HIST) {
     __syncthreads();
@@ -1069,6 +1108,26 @@ SplitWs carve_split_ws(void* ws, int C, int R, int S) {
   if (S > kPlanSmemSplits) w.g_buf = reinterpret_cast<unsigned long long*>(take(8 * w.plan_words));
   w.total = off;
   return w;
+}
+
+// Rows-per-buffer, row-group count and shared-memory bytes of the row-staged kernels.
+struct RowsGeometry {
+  long long g;
+  int n_groups;
+  int n_buf;
+  size_t rows_smem;
+};
+RowsGeometry rows_geometry(int O, size_t row_bytes, size_t hist_bytes) {
+  RowsGeometry q{};
+  // rows that fit beside the histogram counters (the caller checked that two do)
+  const size_t n_fit = (kRowSmemBytes - hist_bytes) / row_bytes;
+  q.n_buf = n_fit >= (size_t)kRowRing ? kRowRing : (int)n_fit;
+  q.g = (long long)(n_fit / q.n_buf);
+  q.g = min(q.g, (long long)max(1, O / (kNumSMs * q.n_buf)));   // every SM should get a ring's worth of groups
+  q.g = min(q.g, 64ll);
+  q.n_groups = (int)((O + q.g - 1) / q.g);
+  q.rows_smem = (size_t)q.n_buf * (size_t)q.g * row_bytes;
+  return q;
 }
 
 // Grid of a streaming kernel: one resident wave, but no more CTAs than there are 8-row slices.
@@ -1192,11 +1251,11 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
     const bool staged = vec && (C * R) % 4 == 0 && 2 * row_bytes <= kRowSmemBytes;
     LaunchScope ls(staged ? "split_rows_kernel" : "split_scatter_kernel", stream);
     if (staged) {
-      // rows per group: as many as fit in half the buffer space, but keep at least one group per SM
-      long long g = (long long)(kRowSmemBytes / 2 / row_bytes);
-      g = min(g, (long long)max(1, O / kNumSMs));
-      g = min(g, 64ll);
-      const int n_groups = (int)((O + g - 1) / g);
+      const RowsGeometry geo = rows_geometry(O, row_bytes, 0);
+      const long long g = geo.g;
+      const int n_groups = geo.n_groups;
+      RowsEpilogue ep{};
+      ep.n_buf = geo.n_buf;
       static bool attr_set = false;
       if (!attr_set) {
         if (cudaFuncSetAttribute(split_rows_kernel<ROWS_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1204,9 +1263,9 @@ extern "C" ocs_status ocs_split(const float* W, int O, int C, int R, int64_t ld_
           return OCS_ERR_CUDA;
         attr_set = true;
       }
-      split_rows_kernel<ROWS_STORE><<<min(n_groups, kNumSMs), kRowThreads, 2 * (size_t)g * row_bytes, stream>>>(
+      split_rows_kernel<ROWS_STORE><<<min(n_groups, kNumSMs), kRowThreads, geo.rows_smem, stream>>>(
           W, O, C, R, ld_in, S, W_out, ld_out, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g,
-          srow, RowsEpilogue{}, dev_status);
+          srow, ep, dev_status);
     } else {
       const long long units = (long long)((ncols_out + 1023) / 1024) * O;
       if (vec)
@@ -1429,22 +1488,6 @@ rows_quant_narrow_kernel(const float* __restrict__ W, int O, int C, int R, long 
 
 namespace ocs {
 namespace {
-// Rows-per-buffer, row-group count and shared-memory bytes of the row-staged kernels.
-struct RowsGeometry {
-  long long g;
-  int n_groups;
-  size_t rows_smem;
-};
-RowsGeometry rows_geometry(int O, size_t row_bytes, size_t hist_bytes) {
-  RowsGeometry q{};
-  q.g = (long long)((kRowSmemBytes - hist_bytes) / 2 / row_bytes);
-  q.g = min(q.g, (long long)max(1, O / kNumSMs));
-  q.g = min(q.g, 64ll);
-  q.n_groups = (int)((O + q.g - 1) / q.g);
-  q.rows_smem = 2 * (size_t)q.g * row_bytes;
-  return q;
-}
-
 ocs_status rows_attr_once() {
   static bool attr_set = false;
   if (!attr_set) {
@@ -1534,7 +1577,7 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
       OCS_OK)
     return st;
 
-  const RowsGeometry geo = rows_geometry(O, row_bytes, hist_bytes);
+  const RowsGeometry geo = rows_geometry(O, row_bytes, 0);   // the code pass keeps no counters
   const long long g = geo.g;
   const int n_groups = geo.n_groups;
   const size_t rows_smem = geo.rows_smem;
@@ -1542,6 +1585,7 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
   const int L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
   RowsEpilogue ep{};
   ep.maxp = mx3 + 1;   // max|W'| as the plan computed it
+  ep.n_buf = geo.n_buf;
   ep.L = L;
   ep.is_signed = is_signed ? 1 : 0;
   const double* scores = nullptr;
@@ -1549,15 +1593,19 @@ extern "C" ocs_status ocs_split_quantize(const float* W, int O, int C, int R, in
     if (cudaMemsetAsync(f.hist, 0, 8 * (size_t)n_bins, stream) != cudaSuccess) return OCS_ERR_CUDA;
     ep.n_bins = n_bins;
     ep.hist = f.hist;
-    int copies = (int)((kRowSmemBytes - rows_smem) / (4 * (size_t)n_bins));
-    ep.hist_copies = copies >= 4 ? 4 : (copies >= 2 ? 2 : 1);
+    // four counter copies when a full ring of rows fits beside them, else two or one
+    int copies = 4;
+    while (copies > 1 && (kRowSmemBytes - copies * hist_bytes) / row_bytes < (size_t)kRowRing) copies >>= 1;
+    const RowsGeometry gh = rows_geometry(O, row_bytes, copies * hist_bytes);
+    ep.hist_copies = copies;
+    ep.n_buf = gh.n_buf;
     {
       LaunchScope ls("split_hist_kernel", stream);
-      split_rows_kernel<ROWS_HIST><<<min(n_groups, kNumSMs), kRowThreads,
-                                     rows_smem + 4 * (size_t)ep.hist_copies * n_bins, stream>>>(
-          W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)g, srow,
-          ep, dev_status);
+      split_rows_kernel<ROWS_HIST><<<min(gh.n_groups, kNumSMs), kRowThreads, gh.rows_smem + copies * hist_bytes, stream>>>(
+          W, O, C, R, ld_in, S, nullptr, 0, idx_map, w.depth, w.bits, w.qa_step_dev, w.touched, w.n_touched, (int)gh.g,
+          srow, ep, dev_status);
     }
+    ep.n_buf = geo.n_buf;
     if ((st = launch_status()) != OCS_OK) return st;
     if ((st = launch_clip_search(mode, f.hist, ep.maxp, n_bins, n_candidates, L, is_signed ? 1 : 0, f.scores,
                                  f.mx3 + 8, stream)) != OCS_OK)
@@ -1594,7 +1642,7 @@ struct BatchLayer {
   int8_t* codes; long long ld_codes; float* scale;
   int mm_blk0, mm_blks, mm_narrow, vec;            // extrema pass: first CTA, CTAs, kernel form, 128-bit loads
   int cp_kind, cp_blk0, cp_blks;                   // code pass: 0 = short rows, 1 = row-staged; first CTA, CTAs
-  int tail_warps, packed_ok, rows_per_group, srow; // code pass geometry
+  int tail_warps, packed_ok, rows_per_group, srow, n_buf; // code pass geometry
 };
 struct BatchTable {
   int n, L, is_signed, pad;
@@ -1667,6 +1715,7 @@ batch_staged_code_kernel(const __grid_constant__ BatchTable t, int* dev_status) 
   ep.packed_ok = y.packed_ok;
   ep.scale_out = y.scale;
   ep.alpha_out = nullptr;
+  ep.n_buf = y.n_buf;
   split_rows_body<ROWS_QUANT>(y.W, y.O, y.C, y.R, (int64_t)y.C * y.R, y.S, nullptr, 0, y.idx_map, y.depth, y.bits,
                               y.qa_step_dev, y.touched, y.n_touched, y.rows_per_group, y.srow, ep, dev_status, row_smem_b,
                               (int)blockIdx.x - y.cp_blk0, y.cp_blks);
@@ -1761,6 +1810,7 @@ bool plan_batch(const ocs_layer_desc* layers, int n, int bits, int is_signed, vo
     } else {
       const RowsGeometry geo = rows_geometry(d.O, row_bytes, 0);
       y.rows_per_group = (int)geo.g;
+      y.n_buf = geo.n_buf;
       int g = geo.n_groups < kNumSMs / 4 ? geo.n_groups : kNumSMs / 4;   // a layer takes a quarter of the SMs at most
       if (g < 1) g = 1;
       y.cp_kind = 1; y.cp_blk0 = sb; y.cp_blks = g; sb += g;
@@ -1934,6 +1984,7 @@ extern "C" ocs_status ocs_act_split_quantize_static(const float* A, int rows, in
   if ((st = rows_attr_once()) != OCS_OK) return st;
   RowsEpilogue ep{};
   ep.maxp = f.mx3 + 1;
+  ep.n_buf = geo.n_buf;
   ep.L = is_signed ? (1 << (bits - 1)) - 1 : (1 << bits) - 1;
   ep.is_signed = is_signed ? 1 : 0;
   ep.scores = nullptr;
