@@ -457,7 +457,7 @@ struct SmemLayout {
   // epilogue staging: per epilogue warp a 32 x 32 tile of 32-bit words, rows padded to 36 words (16-byte
   // aligned, conflict-free for 128-bit accesses by quarter warps), and the 32 output-row numbers
   static constexpr int kEpiRowWords = kEpiCols + 4;
-  static constexpr int kEpiWarpBytes = 32 * kEpiRowWords * 4 + 32 * 8;
+  static constexpr int kEpiWarpBytes = 32 * kEpiRowWords * 4 + 128 * 4;   // + the bias of the warp's pieces of a tile
   static constexpr int kEpiBytes = kEpiWarps * kEpiWarpBytes;
   static constexpr int kDynBytes =
       kTileBytes + 1024 /*alignment slack*/ + kCtrlBytes + kRowTableBytes + kSrcTableBytes + kEpiBytes;
@@ -820,6 +820,24 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         for (int c = (warp >= 10 ? 32 : 0); c < BN && c < n_left; c += 64)
           asm volatile("prefetch.global.L2 [%0];" ::"l"(rrow + c));
       }
+      // The bias of this warp's pieces of the tile (piece k = columns half*16 + 32k .. +15): lane l asks for four
+      // values of piece l/4 now, before the wait for the accumulator, and parks them in shared memory afterwards, so
+      // that the pieces read them from there instead of waiting for global memory once each.
+      float4 bias_mine = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      if (direct && p.bias) {
+        const int col = half * kEpiCols + 2 * kEpiCols * (lane >> 2) + (lane & 3) * 4;   // inside the tile
+        const int n = nt * BN + col;
+        if (col < BN) {
+          if (n + 3 < p.N && ((reinterpret_cast<uintptr_t>(p.bias) & 15) == 0)) {
+            bias_mine = __ldg(reinterpret_cast<const float4*>(p.bias + n));
+          } else {
+            if (n < p.N) bias_mine.x = __ldg(p.bias + n);
+            if (n + 1 < p.N) bias_mine.y = __ldg(p.bias + n + 1);
+            if (n + 2 < p.N) bias_mine.z = __ldg(p.bias + n + 2);
+            if (n + 3 < p.N) bias_mine.w = __ldg(p.bias + n + 3);
+          }
+        }
+      }
       if (!mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       if (!direct) {
@@ -957,11 +975,22 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       // with qd = lane/4, words (lane%4)*4 .. +3; the row order keeps the shared-memory reads conflict-free).
       // The two epilogue warps that share a tensor-memory lane quadrant take alternate pieces.
       uint32_t* st_words = reinterpret_cast<uint32_t*>(epi_stage + (size_t)ew * L::kEpiWarpBytes);
+      float* st_bias = reinterpret_cast<float*>(st_words + 32 * L::kEpiRowWords);   // [piece][16]
+      __syncwarp();   // the previous tile's pieces have read their bias
+      *reinterpret_cast<float4*>(st_bias + lane * 4) = bias_mine;   // read after the piece loop's first __syncwarp
       const int qd = lane >> 2, sub = (qd & 1) * 4 + (qd >> 1), cq = (lane & 3) * 4;
       // the four rows this lane writes, the same for every piece of the tile
       long long orow[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) orow[i] = __shfl_sync(0xffffffffu, ri.out_row, i * 8 + sub);
+      // ... and where their part of the tile starts in Y (for the common case below)
+      float* yrow[4];
+      bool rok[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        rok[i] = orow[i] >= 0;
+        yrow[i] = p.Y + (rok[i] ? orow[i] : 0) * p.ldy + (long long)nt * BN + cq;
+      }
       uint32_t* dst0 = reinterpret_cast<uint32_t*>(p.Y);
       const long long ldd = p.ldy;
       const bool base_vec = ((reinterpret_cast<uintptr_t>(dst0) & 15) == 0) && (ldd % 4 == 0);
@@ -969,7 +998,6 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       // the shortcut tensor is read with 128-bit loads only when it is itself 16-byte aligned (a view that
       // starts a few floats into a buffer takes the scalar loads)
       const bool res_vec = p.residual && ((reinterpret_cast<uintptr_t>(p.residual) & 15) == 0) && (p.ldy % 4 == 0);
-      const bool bias_vec = p.bias && ((reinterpret_cast<uintptr_t>(p.bias) & 15) == 0);
       float tile_max = 0.0f;
       const bool want_max = p.max_bits != nullptr;
       // a warp whose 32 rows are all padding (a short M tile) has nothing to write
@@ -978,21 +1006,11 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
         const bool full = n0 + kEpiCols <= p.N;   // warp-uniform
-        // this lane's four columns of every row it writes: their bias once per piece, asked for before the
-        // accumulator so that the two latencies overlap
-        float b4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (p.bias) {
-          if (full && bias_vec) {
-            const float4 t = __ldg(reinterpret_cast<const float4*>(p.bias + n0 + cq));
-            b4[0] = t.x; b4[1] = t.y; b4[2] = t.z; b4[3] = t.w;
-          } else {
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-              if (n0 + cq + e < p.N) b4[e] = __ldg(p.bias + n0 + cq + e);
-          }
-        }
         uint32_t v[kEpiCols];
         __syncwarp();
+        // this lane's four columns of every row it writes: their bias (zero without one, and past column N)
+        const float4 bq = *reinterpret_cast<const float4*>(st_bias + (c0 >> 5) * kEpiCols + cq);
+        const float b4[4] = {bq.x, bq.y, bq.z, bq.w};
         tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
         // raw accumulators -> shared memory, one row per lane
         uint32_t* mine = st_words + lane * L::kEpiRowWords;
@@ -1019,9 +1037,9 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
               f0 = f0 > 0.0f ? f0 : 0.0f; f1 = f1 > 0.0f ? f1 : 0.0f;
               f2 = f2 > 0.0f ? f2 : 0.0f; f3 = f3 > 0.0f ? f3 : 0.0f;
             }
-            if (orow[i] >= 0) {
+            if (rok[i]) {
               if (want_max) tile_max = fmaxf(tile_max, fmaxf(fmaxf(fabsf(f0), fabsf(f1)), fmaxf(fabsf(f2), fabsf(f3))));
-              *reinterpret_cast<float4*>(p.Y + orow[i] * ldd + n0 + cq) = make_float4(f0, f1, f2, f3);
+              *reinterpret_cast<float4*>(yrow[i] + c0) = make_float4(f0, f1, f2, f3);
             }
           }
           continue;
