@@ -1006,6 +1006,15 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
         const int n0 = nt * BN + c0;
         if (n0 >= p.N) break;  // warp-uniform
         const bool full = n0 + kEpiCols <= p.N;   // warp-uniform
+        // the shortcut values of the piece (common case below): asked for first, so that their way from L2 -- where
+        // the tile's part of the shortcut tensor was prefetched -- overlaps the accumulator's way through shared memory
+        float4 r4[4];
+        if (p.residual && full && base_vec && res_vec && !p.acc_out) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            r4[i] = rok[i] ? __ldcs(reinterpret_cast<const float4*>(p.residual + (yrow[i] - p.Y) + c0))
+                           : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
         uint32_t v[kEpiCols];
         __syncwarp();
         // this lane's four columns of every row it writes: their bias (zero without one, and past column N)
@@ -1023,9 +1032,9 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
 #pragma unroll
         for (int i = 0; i < 4; ++i)
           a[i] = *reinterpret_cast<const uint4*>(st_words + (i * 8 + sub) * L::kEpiRowWords + cq);
-        if (vec0 && !p.residual && !p.acc_out) {
-          // the common case, without per-element tests: whole piece inside N, 16-byte aligned output, nothing
-          // but scale, bias, ReLU and the maximum; the floating-point steps work on pairs
+        if (vec0 && !p.acc_out && (!p.residual || res_vec)) {
+          // the common case, without per-element tests: whole piece inside N, 16-byte aligned output (and
+          // shortcut tensor), scale, bias, shortcut, ReLU and the maximum; the floating-point steps work on pairs
           const unsigned long long sc2 = pack_f32x2(sc, sc);
           const unsigned long long b01 = pack_f32x2(b4[0], b4[1]), b23 = pack_f32x2(b4[2], b4[3]);
 #pragma unroll
@@ -1033,6 +1042,9 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             float f0, f1, f2, f3;
             unpack_f32x2(fma_f32x2(int2_to_float2_rn((int)a[i].x, (int)a[i].y), sc2, b01), f0, f1);
             unpack_f32x2(fma_f32x2(int2_to_float2_rn((int)a[i].z, (int)a[i].w), sc2, b23), f2, f3);
+            if (p.residual) {   // one more rounded addition per output
+              f0 = __fadd_rn(f0, r4[i].x); f1 = __fadd_rn(f1, r4[i].y); f2 = __fadd_rn(f2, r4[i].z); f3 = __fadd_rn(f3, r4[i].w);
+            }
             if (p.relu) {
               f0 = f0 > 0.0f ? f0 : 0.0f; f1 = f1 > 0.0f ? f1 : 0.0f;
               f2 = f2 > 0.0f ? f2 : 0.0f; f3 = f3 > 0.0f ? f3 : 0.0f;

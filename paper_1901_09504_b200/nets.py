@@ -167,16 +167,16 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
     for spec in cfg["layers"]:
         src = t[spec.input_from] if spec.input_from else x
         m = torch.empty(1, dtype=torch.float32, device=x.device)
-        # A ReLU straight after the layer is taken in its epilogue, with the maximum of the result.  The shortcut
-        # addition stays a separate streaming pass (ocs_add_relu, which also takes the maximum): in the epilogue
-        # it makes the output-bound layers wait for the shortcut tensor's loads and costs more than it saves.
-        fused_relu = spec.relu and not spec.residual_from
+        # The ReLU after the layer is taken in its epilogue, with the maximum of the result, and so is the shortcut
+        # addition of a bottleneck block's last convolution (one more rounded addition per output, before the
+        # ReLU): the block's output is written once instead of written, read back with the shortcut and rewritten.
+        take_max = spec.relu or bool(spec.residual_from)
         y = conv_forward(layers[spec.name], src, a_signed=first, a_bits=a_bits, dev_status=dev_status,
-                         max_abs=mx.get(id(src)), relu=fused_relu, max_out=m if fused_relu else None)
+                         max_abs=mx.get(id(src)), relu=spec.relu, max_out=m if take_max else None,
+                         residual=t[spec.residual_from] if spec.residual_from else None)
         if spec.residual_from:
-            y = B.ocs_add_relu(y, t[spec.residual_from], relu=spec.relu, out=y, max_out=m)
             t[spec.name.rsplit(".", 1)[0] + ".out"] = y
-        if fused_relu or spec.residual_from:
+        if take_max:
             mx[id(y)] = m
         t[spec.name] = y
         x = y
