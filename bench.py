@@ -976,7 +976,7 @@ def run_reference(args, wl):
     line = dict(impl="reference", metric=NET_METRIC if net else METRIC, value=val, unit=unit, n_gpus=args.gpus,
                 steps=args.steps,
                 warmup=min(args.warmup, 1), ms_per_step=sec * 1e3, higher_is_better=True, scaling="weak",
-                vs_baseline=None, dtype="int8 codes / int32 accumulate / fp32 scales", data="synthetic",
+                vs_baseline=None, dtype="f32 (split, clip search, quantize) + int8 x int8 -> int32 (GEMM)", data="synthetic",
                 config=dict(workload=wl.desc, sample=wl.oracle_sample_desc),
                 cpu_baseline=dict(value=val, unit=unit, cores=orc.threads(), kind="oracle",
                                   sample=wl.oracle_sample_desc),
@@ -1167,7 +1167,7 @@ def main():
     line = dict(
         metric=metric, value=value, unit=unit, n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=ms_step, higher_is_better=True, scaling="weak", vs_baseline=None,
-        dtype="int8 codes / int32 accumulate / fp32 scales", data="synthetic",
+        dtype="f32 (split, clip search, quantize) + int8 x int8 -> int32 (GEMM)", data="synthetic",
         config=dict(workload=wl.desc, l2=getattr(wl, "l2_note", None) or (
             "inputs larger than L2 (no flush)" if wl.name.startswith("fc6") else "inputs fit in L2; nothing is flushed between steps"),
                     bytes_per_step=led.total, int_ops_per_step=led.ops,
