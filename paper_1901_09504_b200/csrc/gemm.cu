@@ -535,24 +535,21 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   // The CTAs of a cluster work on the same output tile and split its K-blocks.
   const uint32_t crank = cluster_rank(), CL = cluster_size();
 
-  // The TMA producer is thread 0, the thread that sets up the barriers: it requests the first ring of operand
-  // tiles right after that, before the CTA waits for the tensor-memory allocation and for its cluster peers, so
-  // that the set-up time overlaps the first bytes' way from DRAM.  (Its own barriers are ready; the tiles land in
-  // this CTA's own shared memory.)
+  // The TMA producer is thread 0.  (Requesting the first ring of operand tiles before the set-up barriers, to
+  // overlap the set-up with the first bytes' way from DRAM, was measured: the whole CTA then waits for that thread's
+  // cold code, and the fc6 GEMM takes 4 us longer.)
   int prod_j = 0, prod_i = 0, prod_it = 0;   // producer position: work item, K-block inside it, ring slot counter
   bool prod_ok = true;
-  // thread 0 only: issue K-blocks until `limit_it` have been issued (first_tile_only: and stay inside the first tile)
   WorkItem prod_w;
   int prod_w_j = -1;                         // the work item prod_w describes (-1: none yet)
-  auto produce = [&](int limit_it, bool first_tile_only) {
-    while (prod_ok && prod_it < limit_it) {
+  auto produce = [&]() {                     // thread 0 only: issue the K-blocks of all of this CTA's work items
+    while (prod_ok) {
       if (prod_w_j != prod_j) {              // look the tile up once, not once per K-block
         if (!work_item(p, prod_j, crank, CL, &prod_w)) break;
         prod_w_j = prod_j;
       }
       const WorkItem& w = prod_w;
       if (prod_i >= w.my_kb) {
-        if (first_tile_only) break;
         ++prod_j; prod_i = 0;
         continue;
       }
@@ -609,7 +606,6 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
     prefetch_tmap(&tmB);
     if (p.kb_tma_a > 0) prefetch_tmap(&tmA);
     if (p.tail_T) prefetch_tmap(&tmAT);
-    produce(stages, true);    // the first ring: its slots are free by construction
   }
   constexpr uint32_t kTmemCols = 2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512);   // a power of two
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);   // two accumulators: the epilogue of one tile
@@ -622,7 +618,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      produce(0x7fffffff, false);
+      produce();
       if (*abort_flag && prod_it > 0) {
         // give copies that are still in flight time to land before the CTA's shared memory is released
         for (int i = 0; i < 2000; ++i) __nanosleep(100);
