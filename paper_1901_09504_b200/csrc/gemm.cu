@@ -834,6 +834,13 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
           }
         }
       }
+      // K split: a thread of the summing step below keeps one 4-column group for all the rows it finishes (256
+      // threads step over the row-major quads of the tile's part in strides that are multiples of a row), so its
+      // bias is fetched here, while the main loop runs, instead of from a cold cache at the end of the tile
+      constexpr bool kBiasOnce = 256 % (BN / 4) == 0;
+      float4 bias_split = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      if (!direct && kBiasOnce && p.bias && (reinterpret_cast<uintptr_t>(p.bias) & 15) == 0 && (nt + 1) * BN <= p.N)
+        bias_split = __ldg(reinterpret_cast<const float4*>(p.bias + nt * BN + ((threadIdx.x - 6 * 32) % (BN / 4)) * 4));
       if (!mbar_wait(accfull_bar(acc), ((uint32_t)j >> 1) & 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       if (!direct) {
@@ -907,8 +914,8 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
                 const int4 v = *reinterpret_cast<const int4*>(src + sl * slot_bytes);
                 a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
               }
-              float4 b4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-              if (bias_n) b4 = __ldg(reinterpret_cast<const float4*>(bias_n + c));
+              float4 b4 = bias_split;   // zero without a bias
+              if (!kBiasOnce && bias_n) b4 = __ldg(reinterpret_cast<const float4*>(bias_n + c));
               // cvt.rn.f32.s32: the same value as the conversion of the direct epilogue, in one instruction
               float4 f = make_float4(fmaf(__int2float_rn(a.x), sc, b4.x), fmaf(__int2float_rn(a.y), sc, b4.y),
                                      fmaf(__int2float_rn(a.z), sc, b4.z), fmaf(__int2float_rn(a.w), sc, b4.w));
