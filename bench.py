@@ -215,6 +215,7 @@ def tensor_probe(ocs, torch, dev):
 # ----------------------------------------------------------------------------------------------
 class Fc6Sweep:
     name = "fc6"
+    LANES = 3      # sweep points in flight (measured on the fc6 sweep: 9.44 / 8.62 / 8.40 / 8.45 ms with 1 / 2 / 3 / 4)
 
     def __init__(self, small=False):
         self.O, self.C, self.M = (256, 6272, 128) if small else (4096, 25088, 128)
@@ -251,9 +252,20 @@ class Fc6Sweep:
         self.status = ocs.new_status(dev)
         self.W.copy_(host["W"])
         self.A.copy_(host["A"])
+        # Sweep points are independent: they run in two lanes (two streams, each with its own working buffers), so
+        # that the latency-bound kernels of one point (the single-CTA split plan, the candidate scores, the short
+        # GEMM) overlap the streaming kernels of the other.
+        self.lanes = min(self.LANES, len(self.points))
+        self.lane_bufs = [dict(W_out=self.W_out, idx_map=self.idx_map, max_abs=self.max_abs, codes=self.codes,
+                               a_codes=self.a_codes, a_codes_T=self.a_codes_T, scal=self.scal, ws=self.ws)]
+        for _ in range(1, self.lanes):
+            self.lane_bufs.append({k: torch.zeros_like(v) if k in ("scal", "max_abs") else torch.empty_like(v)
+                                   for k, v in self.lane_bufs[0].items()})
+        self.lane_streams = [torch.cuda.Stream() for _ in range(self.lanes)] if self.lanes > 1 else []
 
     def release(self):
         """Drops the big device buffers (called after the last timed region)."""
+        self.lane_bufs = None
         for k in ("W", "A", "W_out", "codes", "a_codes_T", "Wd", "Ad", "Yd", "Y", "slot_graphs", "graph_obj", "ws"):
             if hasattr(self, k):
                 setattr(self, k, None)
@@ -278,28 +290,43 @@ class Fc6Sweep:
             led.ops += 2 * M * O * (C + S)
         return led
 
-    def gemm(self, i, S):
+    def gemm(self, i, S, b):
         """Activation codes -> layer output of sweep point i: with duplicated channels the layer gathers them as
         whole rows of a channel-major copy of the codes (made here, every point: nothing is cached)."""
         ocs, C = self.ocs, self.C
         at = None
         if S > 0:
-            at = ocs.ocs_transpose_codes(self.a_codes, cols=C, out=self.a_codes_T)
-        ocs.ocs_qlinear(self.a_codes, self.scal[2:3], self.codes, self.scal[0:1], self.idx_map, C, S,
-                        out=self.Y[i], ws=self.ws, dev_status=self.status, A_codes_T=at)
+            at = ocs.ocs_transpose_codes(b["a_codes"], cols=C, out=b["a_codes_T"])
+        ocs.ocs_qlinear(b["a_codes"], b["scal"][2:3], b["codes"], b["scal"][0:1], b["idx_map"], C, S,
+                        out=self.Y[i], ws=b["ws"], dev_status=self.status, A_codes_T=at)
+
+    def point(self, i, b):
+        ocs, C = self.ocs, self.C
+        r, bits = self.points[i]
+        S = ocs.ocs_num_splits(C, r)
+        ocs.ocs_split(self.W, S, out=(b["W_out"], b["idx_map"], None, b["max_abs"]), ws=b["ws"],
+                      dev_status=self.status)
+        ocs.ocs_quantize(b["W_out"], bits, True, ocs.CLIP_MSE, N_CAND, N_BINS, cols=C + S,
+                         max_abs_in=b["max_abs"][1:2], out=(b["codes"], b["scal"][0:1], b["scal"][1:2]),
+                         ws=b["ws"], dev_status=self.status)
+        ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(b["a_codes"], b["scal"][2:3], b["scal"][3:4]),
+                         ws=b["ws"], dev_status=self.status)
+        self.gemm(i, S, b)
 
     def step(self):
-        ocs, C = self.ocs, self.C
-        for i, (r, bits) in enumerate(self.points):
-            S = ocs.ocs_num_splits(C, r)
-            ocs.ocs_split(self.W, S, out=(self.W_out, self.idx_map, None, self.max_abs), ws=self.ws,
-                          dev_status=self.status)
-            ocs.ocs_quantize(self.W_out, bits, True, ocs.CLIP_MSE, N_CAND, N_BINS, cols=C + S,
-                             max_abs_in=self.max_abs[1:2], out=(self.codes, self.scal[0:1], self.scal[1:2]),
-                             ws=self.ws, dev_status=self.status)
-            ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(self.a_codes, self.scal[2:3], self.scal[3:4]),
-                             ws=self.ws, dev_status=self.status)
-            self.gemm(i, S)
+        torch = self.torch
+        if self.lanes <= 1:
+            for i in range(len(self.points)):
+                self.point(i, self.lane_bufs[0])
+            return
+        main = torch.cuda.current_stream()
+        for k, st in enumerate(self.lane_streams):
+            st.wait_stream(main)
+            with torch.cuda.stream(st):
+                for i in range(k, len(self.points), self.lanes):
+                    self.point(i, self.lane_bufs[k])
+        for st in self.lane_streams:
+            main.wait_stream(st)
 
     # The step is a fixed chain of stream-ordered, allocation-free library calls on preallocated buffers: it is
     # captured once in a CUDA graph (after an eager warm-up) and replayed, which removes the host work between
@@ -427,9 +454,12 @@ class Fc6Fused(Fc6Sweep):
     def setup(self, ocs, torch, dev, host):
         super().setup(ocs, torch, dev, host)
         nws = ocs.lib().ocs_split_quantize_workspace_bytes(self.O, self.C, 1, self.idx_map.numel() - self.C, N_BINS, N_CAND)
-        if nws + 256 > self.ws.numel():
-            self.ws = torch.empty(int(nws) + 256, dtype=torch.uint8, device=dev)
         self.W_out = None      # never written
+        for b in self.lane_bufs:
+            b["W_out"] = None
+            if nws + 256 > b["ws"].numel():
+                b["ws"] = torch.empty(int(nws) + 256, dtype=torch.uint8, device=dev)
+        self.ws = self.lane_bufs[0]["ws"]
 
     def ledger(self):
         led = Ledger()
@@ -449,16 +479,16 @@ class Fc6Fused(Fc6Sweep):
             led.ops += 2 * M * O * (C + S)
         return led
 
-    def step(self):
+    def point(self, i, b):
         ocs, C = self.ocs, self.C
-        for i, (r, bits) in enumerate(self.points):
-            S = ocs.ocs_num_splits(C, r)
-            ocs.ocs_split_quantize(self.W, S, bits, ocs.CLIP_MSE, n_candidates=N_CAND, n_bins=N_BINS,
-                                   out=(self.codes, self.scal[0:1], self.scal[1:2], self.idx_map, None, self.max_abs),
-                                   ws=self.ws, dev_status=self.status)
-            ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(self.a_codes, self.scal[2:3], self.scal[3:4]),
-                             ws=self.ws, dev_status=self.status)
-            self.gemm(i, S)
+        r, bits = self.points[i]
+        S = ocs.ocs_num_splits(C, r)
+        ocs.ocs_split_quantize(self.W, S, bits, ocs.CLIP_MSE, n_candidates=N_CAND, n_bins=N_BINS,
+                               out=(b["codes"], b["scal"][0:1], b["scal"][1:2], b["idx_map"], None, b["max_abs"]),
+                               ws=b["ws"], dev_status=self.status)
+        ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(b["a_codes"], b["scal"][2:3], b["scal"][3:4]),
+                         ws=b["ws"], dev_status=self.status)
+        self.gemm(i, S, b)
 
 
 class ActOcs(Fc6Sweep):
@@ -637,7 +667,7 @@ class SmallFc(Fc6Sweep):
                          out=(self.codes, self.scal[0:1], self.scal[1:2]), ws=self.ws, dev_status=self.status)
         ocs.ocs_quantize(self.A, 8, False, ocs.CLIP_NONE, out=(self.a_codes, self.scal[2:3], self.scal[3:4]),
                          ws=self.ws, dev_status=self.status)
-        self.gemm(0, S)
+        self.gemm(0, S, self.lane_bufs[0])
 
     def ledger(self):
         led = Ledger()
@@ -1080,8 +1110,13 @@ def main():
     # second pass over the same K steps with per-kernel CUDA events (the launches are identical)
     barrier()
     ocs.ocs_trace_start(launches * args.steps + 16)
+    lanes = getattr(wl, "lanes", 1)
+    if lanes > 1:
+        wl.lanes = 1          # one kernel at a time: a launch's duration is then its own
     for _ in range(args.steps):
         wl.step()
+    if lanes > 1:
+        wl.lanes = lanes
     trace = ocs.ocs_trace_stop()
     barrier()
 
@@ -1172,7 +1207,9 @@ def main():
             "inputs larger than L2 (no flush)" if wl.name.startswith("fc6") else "inputs fit in L2; nothing is flushed between steps"),
                     bytes_per_step=led.total, int_ops_per_step=led.ops,
                     launch=("the step's kernel launches are captured once in a CUDA graph and replayed"
-                            if use_graph else "eager launches")),
+                            if use_graph else "eager launches"),
+                    **({"lanes": f"{wl.lanes} sweep points in flight on {wl.lanes} streams (independent points; the "
+                                 "per-kernel timings are taken one kernel at a time)"} if getattr(wl, "lanes", 1) > 1 else {})),
         parts=dict(split_quantize_gbs=sq_gbs, split_quantize_frac_of_hbm=(sq_gbs / pk["hbm"]) if sq_gbs else None,
                    gemm_tops=gemm_tops, gemm_frac_of_int8_peak=(gemm_tops / int8_peak) if gemm_tops else None,
                    int8_peak_tops=int8_peak, int8_peak_note=int8_note,
