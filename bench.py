@@ -1026,6 +1026,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-tensor-probe", action="store_true")
+    ap.add_argument("--lanes", type=int, default=0,
+                    help="sweep points in flight in the fc6 sweeps (0: the workload's default; 1 gives the launch "
+                         "order the ncu summaries under profiles/ index into)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -1035,6 +1038,8 @@ def main():
     wl = {"fc6": Fc6Sweep, "fc6-fused": Fc6Fused, "fc6-small": lambda: Fc6Sweep(small=True), "fc": SmallFc, "conv": Conv3x3,
           "resnet50": ResNet50, "resnet50-per-layer": ResNet50PerLayer, "lstm": Lstm, "lstm-folded": LstmFolded, "act-ocs": ActOcs, "exact-mse": ExactMse}[args.workload]()
     net = getattr(wl, "kind", "") == "net"
+    if args.lanes > 0 and hasattr(wl, "LANES"):
+        wl.LANES = args.lanes
 
     if args.impl == "reference":
         if rank == 0:
