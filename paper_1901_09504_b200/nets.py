@@ -74,10 +74,10 @@ def quantize_activations(x, signed: bool, bits: int = 8, dev_status=None, max_ab
 
 
 def conv_forward(L: QLayer, x, a_signed: bool, a_bits: int = 8, dev_status=None, max_abs=None, relu: bool = False,
-                 max_out=None, residual=None):
+                 max_out=None, residual=None, xq=None):
     """x fp32 NHWC -> fp32 NHWC (activation quantization + ocs_qconv; the shortcut addition, ReLU and max |y|
-    in the layer's epilogue on request)."""
-    xc, xs = quantize_activations(x, a_signed, a_bits, dev_status, max_abs)
+    in the layer's epilogue on request).  xq: (codes, scale) of x when another layer has quantized it already."""
+    xc, xs = xq if xq is not None else quantize_activations(x, a_signed, a_bits, dev_status, max_abs)
     return B.ocs_qconv(xc, xs, L.codes, L.w_scale, L.idx_map, L.S, L.k, L.k, L.stride, L.pad, bias=L.bias,
                        dev_status=dev_status, relu=relu, max_out=max_out, residual=residual)
 
@@ -162,6 +162,10 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
     """X fp32 NCHW on the device -> logits fp32 [Nb, 1000]; with keep, also every named tensor."""
     t = {}
     mx = {}     # max |tensor| of the tensors whose producing layer took it in its epilogue
+    xq = {}     # codes and scale of a tensor that two layers read (a block's first convolution and its projection)
+    readers = {}
+    for spec in cfg["layers"]:
+        readers[spec.input_from] = readers.get(spec.input_from, 0) + 1
     x = B.ocs_nchw_to_nhwc(X_nchw.contiguous())
     first = True
     for spec in cfg["layers"]:
@@ -171,9 +175,12 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
         # addition of a bottleneck block's last convolution (one more rounded addition per output, before the
         # ReLU): the block's output is written once instead of written, read back with the shortcut and rewritten.
         take_max = spec.relu or bool(spec.residual_from)
+        q = xq.get(id(src))
+        if q is None and spec.input_from and readers[spec.input_from] > 1:
+            q = xq[id(src)] = quantize_activations(src, first, a_bits, dev_status, mx.get(id(src)))
         y = conv_forward(layers[spec.name], src, a_signed=first, a_bits=a_bits, dev_status=dev_status,
                          max_abs=mx.get(id(src)), relu=spec.relu, max_out=m if take_max else None,
-                         residual=t[spec.residual_from] if spec.residual_from else None)
+                         residual=t[spec.residual_from] if spec.residual_from else None, xq=q)
         if spec.residual_from:
             t[spec.name.rsplit(".", 1)[0] + ".out"] = y
         if take_max:
