@@ -190,6 +190,8 @@ def resnet50_forward(cfg, layers, X_nchw, a_bits: int = 8, keep: bool = False, d
         if first:
             x = B.ocs_maxpool3x3s2(y)
             t["pool"] = x
+            if spec.relu:
+                mx[id(x)] = m   # the windows cover every value of y and none is negative: max |pool| = max |y|
             first = False
     feat = B.ocs_global_avgpool(x)
     t["avgpool"] = feat

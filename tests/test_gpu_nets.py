@@ -27,6 +27,8 @@ def test_elementwise_and_pooling_steps():
     odd = x.reshape(-1)[:4099].copy()                                        # ragged tail of the vector path
     np.testing.assert_array_equal(host(ocs.ocs_add_relu(dev(odd), None, True)), orc.relu(odd))
     np.testing.assert_array_equal(host(ocs.ocs_maxpool3x3s2(dev(x))), orc.maxpool3x3s2(x))
+    x4 = prng.normal(21, 4, (2, 11, 14, 24), std=2.0)                       # C % 4 == 0: the 128-bit form
+    np.testing.assert_array_equal(host(ocs.ocs_maxpool3x3s2(dev(x4))), orc.maxpool3x3s2(x4))
     np.testing.assert_array_equal(host(ocs.ocs_global_avgpool(dev(x))), orc.global_avgpool(x))
     nchw = prng.normal(21, 2, (2, 5, 9, 11))
     np.testing.assert_array_equal(host(ocs.ocs_nchw_to_nhwc(dev(nchw))), orc.nchw_to_nhwc(nchw))
