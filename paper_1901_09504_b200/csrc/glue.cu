@@ -125,6 +125,24 @@ global_avgpool_kernel(const float* __restrict__ x, int Nb, int HW, int C, float*
   }
 }
 
+// NCHW -> NHWC for a handful of channels (an image batch): a CTA takes 256 pixels of one image; the C planes are
+// read one after the other (coalesced) into shared memory and the 256 * C interleaved values leave as one
+// contiguous run.  grid = (ceil(HW / 256), Nb).
+constexpr int kFewChannels = 8;
+__global__ void __launch_bounds__(256)
+nchw_to_nhwc_few_kernel(const float* __restrict__ x, int C, int HW, float* __restrict__ y) {
+  __shared__ float tile[256 * kFewChannels];
+  const int n = blockIdx.y;
+  const int p0 = blockIdx.x * 256;
+  const int np = min(256, HW - p0);
+  const float* xin = x + (long long)n * C * HW + p0;
+  for (int c = 0; c < C; ++c)
+    if ((int)threadIdx.x < np) tile[threadIdx.x * C + c] = xin[(long long)c * HW + threadIdx.x];
+  __syncthreads();
+  float* yout = y + ((long long)n * HW + p0) * C;
+  for (int i = threadIdx.x; i < np * C; i += 256) yout[i] = tile[i];
+}
+
 // NCHW -> NHWC through a 32 x 33 shared-memory tile over (c, hw) so both sides are coalesced.
 __global__ void __launch_bounds__(256)
 nchw_to_nhwc_kernel(const float* __restrict__ x, int C, int HW, float* __restrict__ y) {
@@ -267,9 +285,14 @@ extern "C" ocs_status ocs_nchw_to_nhwc(const float* x, int Nb, int C, int H, int
   ocs_status st = check_device();
   if (st != OCS_OK) return st;
   const int HW = H * Wd;
-  dim3 grid((HW + 31) / 32, (C + 31) / 32, Nb);
   LaunchScope ls("nchw_to_nhwc_kernel", stream);
-  nchw_to_nhwc_kernel<<<grid, 256, 0, stream>>>(x, C, HW, y);
+  if (C <= kFewChannels && (HW + 255) / 256 <= 0x7fffffff) {
+    dim3 grid((HW + 255) / 256, Nb);
+    nchw_to_nhwc_few_kernel<<<grid, 256, 0, stream>>>(x, C, HW, y);
+  } else {
+    dim3 grid((HW + 31) / 32, (C + 31) / 32, Nb);
+    nchw_to_nhwc_kernel<<<grid, 256, 0, stream>>>(x, C, HW, y);
+  }
   return launch_status();
 }
 

@@ -32,6 +32,8 @@ def test_elementwise_and_pooling_steps():
     np.testing.assert_array_equal(host(ocs.ocs_global_avgpool(dev(x))), orc.global_avgpool(x))
     nchw = prng.normal(21, 2, (2, 5, 9, 11))
     np.testing.assert_array_equal(host(ocs.ocs_nchw_to_nhwc(dev(nchw))), orc.nchw_to_nhwc(nchw))
+    img = prng.normal(21, 5, (2, 3, 20, 30))                                # few channels, several CTAs per image
+    np.testing.assert_array_equal(host(ocs.ocs_nchw_to_nhwc(dev(img))), orc.nchw_to_nhwc(img))
     big = prng.normal(21, 3, (2, 70, 33, 35))
     np.testing.assert_array_equal(host(ocs.ocs_nchw_to_nhwc(dev(big))), orc.nchw_to_nhwc(big))
 
