@@ -406,22 +406,29 @@ __device__ __forceinline__ uint32_t ldg_u8_if(const uint8_t* addr, bool ok) {
 // The operand bytes of one tile row for the 16 contraction indices whose sources are tab[0..16).
 // The 16 loads are independent (predicated, not branched) and in flight together; indices that contribute zero
 // (K padding, a tap outside the image) issue no load.
+// n = how many of the 16 indices lie below the last contraction index (the K padding comes last): groups of four
+// indices beyond it are skipped altogether -- with a handful of duplicated channels most of a chunk is padding.
 __device__ __forceinline__ uint4 gather_chunk(const GemmParams& p, const RowInfo& ri, const uint8_t* base,
-                                              const KSrc* __restrict__ tab) {
-  uint32_t b[16];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const KSrc e = tab[i];
-    bool ok = ri.out_row >= 0 && e.off >= 0;
-    if (p.mode == MODE_CONV) {
-      const int ih = ri.ih0 + (e.dydx & 255), iw = ri.iw0 + (e.dydx >> 8);
-      ok = ok && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd;
-    }
-    b[i] = ldg_u8_if(base + (ok ? e.off : 0), ok);
-  }
+                                              const KSrc* __restrict__ tab, int n) {
   uint32_t w[4];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) w[q] = b[4 * q] | (b[4 * q + 1] << 8) | (b[4 * q + 2] << 16) | (b[4 * q + 3] << 24);
+  for (int q = 0; q < 4; ++q) {
+    w[q] = 0u;
+    if (4 * q < n) {
+      uint32_t b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const KSrc e = tab[4 * q + i];
+        bool ok = ri.out_row >= 0 && e.off >= 0;
+        if (p.mode == MODE_CONV) {
+          const int ih = ri.ih0 + (e.dydx & 255), iw = ri.iw0 + (e.dydx >> 8);
+          ok = ok && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.Wd;
+        }
+        b[i] = ldg_u8_if(base + (ok ? e.off : 0), ok);
+      }
+      w[q] = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+    }
+  }
   return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
@@ -727,6 +734,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       if (bad) flag(p.dev_status, OCS_DEV_BAD_INDEX);
       ok = false;   // nothing left for the byte gather below
     }
+    const RowPos gather_pos = row_pos(p, gt);   // this thread's row of every tile's row table
     int n_tiles_done = 0;
     int table_kb[2] = {-1, -1};   // which K-block each of the two source tables describes
     int buf_kb[kTailBufs];        // which K-block each tail buffer held last
@@ -737,7 +745,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
       // row table of this tile (two tables alternate, so the previous tile's may still be in use)
       RowInfo* trow = rows + (n_tiles_done & 1) * BM;
       ++n_tiles_done;
-      trow[gt] = row_info(p, w.mt, gt);
+      trow[gt] = row_info_at(p, w.mt, gather_pos);
       asm volatile("bar.sync 1, 128;" ::: "memory");
       for (int t = 0; t < w.n_tail; ++t, ++tt) {
         const int kb = (int)crank + (w.n_tma + t) * (int)CL;
@@ -774,7 +782,7 @@ ocs_gemm_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__
             const uint8_t* rbase;
             if (p.mode == MODE_LINEAR) rbase = p.A + ri.out_row * p.lda;
             else rbase = p.A + (((long long)ri.n * p.H + ri.ih0) * p.Wd + ri.iw0) * p.C;
-            v = gather_chunk(p, ri, rbase, tab + c * 16);
+            v = gather_chunk(p, ri, rbase, tab + c * 16, p.Ktot - (kb * BK + c * 16));
           }
           st_local_v4(tile_local + r * 128 + ((c ^ (r & 7)) << 4), v);
         }
